@@ -1,0 +1,201 @@
+"""ctypes binding of libhorizonserve.so: the same names as the C ABI, argument marshalling only.
+
+PyTorch appears here for what the library leaves to its caller: device memory (weights, KV pool,
+workspace, inputs, outputs) and streams.  Every step of the hot path runs inside the library's CUDA
+kernels; if the library is missing this module raises instead of falling back to anything.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libhorizonserve.so")
+
+HS_ABI_VERSION = 1
+HS_OK, HS_ERR_INVALID_ARG, HS_ERR_INVALID_BUDGET, HS_ERR_UNSUPPORTED_SHAPE, HS_ERR_OUT_OF_PAGES, \
+    HS_ERR_BAD_BLOCK_TABLE, HS_ERR_CUDA, HS_ERR_TIMEOUT, HS_ERR_NO_DEVICE, HS_ERR_UNKNOWN_SEQ = range(10)
+
+EXPORTS = ("hs_status_str", "hs_kv_pool_bytes", "hs_workspace_bytes", "hs_stage_create", "hs_stage_destroy",
+           "hs_kv_alloc", "hs_kv_free", "hs_kv_free_pages", "hs_stage_plan", "hs_stage_step", "hs_stage_status",
+           "hs_stage_sm_count", "hs_op_gemm_bf16", "hs_stage_debug_buffer")
+
+
+class hs_stage_config_t(C.Structure):
+    _fields_ = [("abi_version", C.c_uint32), ("device", C.c_int32),
+                ("n_layers", C.c_int32), ("d_model", C.c_int32), ("n_q_heads", C.c_int32),
+                ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("d_ffn", C.c_int32),
+                ("rms_eps", C.c_float), ("rope_base", C.c_float),
+                ("page_size", C.c_int32), ("num_pages", C.c_int32), ("max_tokens", C.c_int32),
+                ("max_seqs", C.c_int32), ("max_pages_per_seq", C.c_int32), ("max_position", C.c_int32),
+                ("flags", C.c_uint32)]
+
+
+WEIGHT_NAMES = ("g_attn", "w_q", "w_k", "w_v", "w_o", "g_mlp", "w_gate", "w_up", "w_down")
+
+
+class hs_layer_weights_t(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES]
+
+
+class hs_batch_t(C.Structure):
+    _fields_ = [("n_seqs", C.c_int32), ("n_tokens", C.c_int32), ("q_len", C.c_void_p), ("ctx_len", C.c_void_p),
+                ("block_tables", C.c_void_p), ("x_in", C.c_void_p), ("y_out", C.c_void_p)]
+
+
+class HsError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_str(status)}")
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def lib() -> C.CDLL:
+    """Loads the library (once).  Raises if it has not been built: there is no other code path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2608_01785_b200.build` "
+                               "(the CUDA library is the only implementation)")
+        l = C.CDLL(LIB_PATH)
+        l.hs_status_str.restype = C.c_char_p
+        l.hs_status_str.argtypes = [C.c_int]
+        l.hs_kv_pool_bytes.restype = C.c_size_t
+        l.hs_kv_pool_bytes.argtypes = [C.POINTER(hs_stage_config_t)]
+        l.hs_workspace_bytes.restype = C.c_size_t
+        l.hs_workspace_bytes.argtypes = [C.POINTER(hs_stage_config_t)]
+        l.hs_stage_create.argtypes = [C.POINTER(hs_stage_config_t), C.POINTER(hs_layer_weights_t), C.c_void_p,
+                                      C.c_void_p, C.POINTER(C.c_void_p)]
+        l.hs_stage_destroy.argtypes = [C.c_void_p]
+        l.hs_kv_alloc.argtypes = [C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]
+        l.hs_kv_free.argtypes = [C.c_void_p, C.c_int64]
+        l.hs_kv_free_pages.argtypes = [C.c_void_p]
+        l.hs_kv_free_pages.restype = C.c_int32
+        l.hs_stage_plan.argtypes = [C.c_void_p, C.POINTER(hs_batch_t), C.c_void_p, C.c_void_p, C.c_void_p]
+        l.hs_stage_step.argtypes = [C.c_void_p, C.POINTER(hs_batch_t), C.c_int32, C.c_void_p]
+        l.hs_stage_status.argtypes = [C.c_void_p]
+        l.hs_stage_sm_count.argtypes = [C.c_void_p]
+        l.hs_stage_sm_count.restype = C.c_int32
+        l.hs_op_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                      C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        l.hs_stage_debug_buffer.argtypes = [C.c_void_p, C.c_char_p, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
+        _lib = l
+    return _lib
+
+
+def status_str(status: int) -> str:
+    return lib().hs_status_str(int(status)).decode()
+
+
+def make_config(dims, num_pages: int, max_tokens: int, max_seqs: int, max_pages_per_seq: int, max_position: int,
+                device: int = 0) -> hs_stage_config_t:
+    """dims: any object with n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, rms_eps, rope_base, page_size."""
+    return hs_stage_config_t(HS_ABI_VERSION, device, dims.n_layers, dims.d_model, dims.n_q_heads, dims.n_kv_heads,
+                             dims.head_dim, dims.d_ffn, dims.rms_eps, dims.rope_base, dims.page_size, num_pages,
+                             max_tokens, max_seqs, max_pages_per_seq, max_position, 0)
+
+
+def hs_kv_pool_bytes(cfg: hs_stage_config_t) -> int:
+    return int(lib().hs_kv_pool_bytes(C.byref(cfg)))
+
+
+def hs_workspace_bytes(cfg: hs_stage_config_t) -> int:
+    return int(lib().hs_workspace_bytes(C.byref(cfg)))
+
+
+def hs_stage_create(cfg: hs_stage_config_t, layer_ptrs: Optional[Sequence[Dict[str, int]]], kv_pool_ptr: int,
+                    workspace_ptr: int) -> int:
+    """Returns the stage handle (an integer address).  layer_ptrs: one dict of device addresses per layer."""
+    arr = None
+    if layer_ptrs is not None:
+        arr = (hs_layer_weights_t * len(layer_ptrs))()
+        for i, lw in enumerate(layer_ptrs):
+            for n in WEIGHT_NAMES:
+                setattr(arr[i], n, lw[n])
+    out = C.c_void_p()
+    st = lib().hs_stage_create(C.byref(cfg), arr, C.c_void_p(kv_pool_ptr), C.c_void_p(workspace_ptr), C.byref(out))
+    if st != HS_OK:
+        raise HsError(st, "hs_stage_create")
+    return out.value
+
+
+def hs_stage_destroy(stage: int) -> None:
+    st = lib().hs_stage_destroy(C.c_void_p(stage))
+    if st != HS_OK:
+        raise HsError(st, "hs_stage_destroy")
+
+
+def hs_kv_alloc(stage: int, seq_id: int, total_tokens: int, cap: int) -> List[int]:
+    """Returns the sequence's whole block table."""
+    table = (C.c_int32 * max(cap, 1))()
+    n = C.c_int32(0)
+    st = lib().hs_kv_alloc(C.c_void_p(stage), seq_id, total_tokens, table, cap, C.byref(n))
+    if st != HS_OK:
+        raise HsError(st, "hs_kv_alloc")
+    return list(table[: n.value])
+
+
+def hs_kv_free(stage: int, seq_id: int) -> None:
+    st = lib().hs_kv_free(C.c_void_p(stage), seq_id)
+    if st != HS_OK:
+        raise HsError(st, "hs_kv_free")
+
+
+def hs_kv_free_pages(stage: int) -> int:
+    return int(lib().hs_kv_free_pages(C.c_void_p(stage)))
+
+
+def hs_stage_sm_count(stage: int) -> int:
+    return int(lib().hs_stage_sm_count(C.c_void_p(stage)))
+
+
+class Batch:
+    """Owns the host arrays of one hs_batch_t (they must stay alive across the call)."""
+
+    def __init__(self, q_len, ctx_len, block_tables, x_in_ptr: int = 0, y_out_ptr: int = 0):
+        self.q_len = np.ascontiguousarray(q_len, dtype=np.int32)
+        self.ctx_len = np.ascontiguousarray(ctx_len, dtype=np.int32)
+        self.block_tables = np.ascontiguousarray(block_tables, dtype=np.int32)
+        self.c = hs_batch_t(len(self.q_len), int(self.q_len.sum()), self.q_len.ctypes.data, self.ctx_len.ctypes.data,
+                            self.block_tables.ctypes.data, x_in_ptr, y_out_ptr)
+
+
+def hs_stage_plan(stage: int, batch: Batch):
+    """Returns (tok_seq, tok_pos, tok_slot) int32 arrays."""
+    n = batch.c.n_tokens
+    seq, pos, slot = (np.empty(max(n, 1), dtype=np.int32) for _ in range(3))
+    st = lib().hs_stage_plan(C.c_void_p(stage), C.byref(batch.c), seq.ctypes.data, pos.ctypes.data, slot.ctypes.data)
+    if st != HS_OK:
+        raise HsError(st, "hs_stage_plan")
+    return seq[:n], pos[:n], slot[:n]
+
+
+def hs_stage_step(stage: int, batch: Batch, sm_budget: int, cuda_stream: int = 0) -> None:
+    st = lib().hs_stage_step(C.c_void_p(stage), C.byref(batch.c), sm_budget, C.c_void_p(cuda_stream))
+    if st != HS_OK:
+        raise HsError(st, "hs_stage_step")
+
+
+def hs_stage_status(stage: int) -> int:
+    return int(lib().hs_stage_status(C.c_void_p(stage)))
+
+
+def hs_stage_debug_buffer(stage: int, name: str):
+    ptr, size = C.c_void_p(), C.c_size_t()
+    st = lib().hs_stage_debug_buffer(C.c_void_p(stage), name.encode(), C.byref(ptr), C.byref(size))
+    if st != HS_OK:
+        raise HsError(st, "hs_stage_debug_buffer")
+    return ptr.value, size.value
+
+
+def hs_op_gemm_bf16(a_ptr: int, w_ptr: int, resid_ptr: int, out_ptr: int, M: int, N: int, K: int, sm_budget: int,
+                    status_ptr: int, cuda_stream: int = 0) -> None:
+    st = lib().hs_op_gemm_bf16(C.c_void_p(a_ptr), C.c_void_p(w_ptr), C.c_void_p(resid_ptr or None), C.c_void_p(out_ptr),
+                               M, N, K, sm_budget, C.c_void_p(status_ptr), C.c_void_p(cuda_stream))
+    if st != HS_OK:
+        raise HsError(st, "hs_op_gemm_bf16")

@@ -1,0 +1,475 @@
+// C ABI of the library: stage object, page allocator front end, step orchestration.
+#include <math.h>
+#include <string.h>
+
+#include <memory>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "../../include/horizonserve_ops.h"
+#include "hs_internal.h"
+#include "kernels.h"
+
+namespace hs {
+namespace {
+
+constexpr int kRing = 4;   // pinned staging slots for step metadata
+
+struct WsLayout {
+  size_t rope, x, h, q, o, act, meta, part_o, part_ml, status, total;
+};
+
+WsLayout make_ws_layout(const hs_stage_config_t& c, const MetaLayout& ml) {
+  WsLayout w{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    size_t o = off;
+    off += align_up(bytes, 1024);
+    return o;
+  };
+  const size_t T = c.max_tokens, q_dim = size_t(c.n_q_heads) * c.head_dim;
+  w.rope = take(size_t(c.max_position) * (c.head_dim / 2) * sizeof(float2));
+  w.x = take(T * c.d_model * 4);
+  w.h = take(T * c.d_model * 2);
+  w.q = take(T * q_dim * 2);
+  w.o = take(T * q_dim * 2);
+  w.act = take(T * c.d_ffn * 2);
+  w.meta = take(size_t(ml.total) * 4);
+  w.part_o = take(size_t(ml.max_decode_items) * 16 * c.head_dim * 4);
+  w.part_ml = take(size_t(ml.max_decode_items) * 16 * 2 * 4);
+  w.status = take(256);
+  w.total = off;
+  return w;
+}
+
+// cuTensorMapEncodeTiled, fetched through the runtime so that the library has no link-time dependency
+// on the driver library (it must load on machines without a GPU).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// bf16 matrix [rows, cols] with cols contiguous; box = 64 columns x box_rows rows, 128-byte swizzle,
+// out-of-range elements read as zero.
+bool encode_2d(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct LayerMaps {
+  CUtensorMap wq, wk, wv, wo, wgate, wup, wdown;
+};
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    if (prev == dev) prev = -1;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+bool g_attrs_set[64] = {};
+hs_status_t ensure_attributes(int device) {
+  if (device >= 0 && device < 64 && g_attrs_set[device]) return HS_OK;
+  if (gemm_set_attributes() != cudaSuccess || norm_set_attributes() != cudaSuccess ||
+      attention_set_attributes() != cudaSuccess)
+    return HS_ERR_CUDA;
+  if (device >= 0 && device < 64) g_attrs_set[device] = true;
+  return HS_OK;
+}
+
+}  // namespace
+}  // namespace hs
+
+using namespace hs;
+
+struct hs_stage {
+  hs_stage_config_t cfg;
+  MetaLayout ml;
+  WsLayout ws;
+  std::unique_ptr<PageAllocator> alloc;
+  std::vector<int32_t> page_stamp;
+  int32_t stamp = 0;
+  int sm_count = 0;
+  uint8_t* ws_dev = nullptr;
+  __nv_bfloat16* kv_pool = nullptr;
+  std::vector<hs_layer_weights_t> layers;
+  std::vector<LayerMaps> maps;
+  CUtensorMap tm_h, tm_o, tm_act, tm_kv;
+  int32_t* pinned[kRing] = {};
+  cudaEvent_t ev[kRing] = {};
+  bool ev_pending[kRing] = {};
+  int ring_pos = 0;
+};
+
+extern "C" {
+
+const char* hs_status_str(hs_status_t s) {
+  switch (s) {
+    case HS_OK: return "HS_OK";
+    case HS_ERR_INVALID_ARG: return "HS_ERR_INVALID_ARG";
+    case HS_ERR_INVALID_BUDGET: return "HS_ERR_INVALID_BUDGET";
+    case HS_ERR_UNSUPPORTED_SHAPE: return "HS_ERR_UNSUPPORTED_SHAPE";
+    case HS_ERR_OUT_OF_PAGES: return "HS_ERR_OUT_OF_PAGES";
+    case HS_ERR_BAD_BLOCK_TABLE: return "HS_ERR_BAD_BLOCK_TABLE";
+    case HS_ERR_CUDA: return "HS_ERR_CUDA";
+    case HS_ERR_TIMEOUT: return "HS_ERR_TIMEOUT";
+    case HS_ERR_NO_DEVICE: return "HS_ERR_NO_DEVICE";
+    case HS_ERR_UNKNOWN_SEQ: return "HS_ERR_UNKNOWN_SEQ";
+  }
+  return "HS_ERR_?";
+}
+
+size_t hs_kv_pool_bytes(const hs_stage_config_t* cfg) {
+  if (!cfg || validate_config(*cfg) != HS_OK) return 0;
+  return size_t(cfg->n_layers) * 2 * cfg->num_pages * cfg->n_kv_heads * kPage * cfg->head_dim * 2;
+}
+
+size_t hs_workspace_bytes(const hs_stage_config_t* cfg) {
+  if (!cfg || validate_config(*cfg) != HS_OK) return 0;
+  return make_ws_layout(*cfg, make_meta_layout(*cfg)).total;
+}
+
+hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights_t* layers, void* kv_pool_dev,
+                            void* workspace_dev, hs_stage_t** out) {
+  if (!cfg || !out) return HS_ERR_INVALID_ARG;
+  *out = nullptr;
+  hs_status_t st = validate_config(*cfg);
+  if (st != HS_OK) return st;
+  const bool host_only = cfg->device < 0;
+  if (!host_only) {
+    if (!layers || !kv_pool_dev || !workspace_dev) return HS_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(kv_pool_dev) & 1023) || (reinterpret_cast<uintptr_t>(workspace_dev) & 1023))
+      return HS_ERR_INVALID_ARG;
+    for (int l = 0; l < cfg->n_layers; ++l) {
+      const void* ptrs[9] = {layers[l].g_attn, layers[l].w_q,    layers[l].w_k,  layers[l].w_v,   layers[l].w_o,
+                             layers[l].g_mlp,  layers[l].w_gate, layers[l].w_up, layers[l].w_down};
+      for (const void* ptr : ptrs)
+        if (!ptr || (reinterpret_cast<uintptr_t>(ptr) & 15)) return HS_ERR_INVALID_ARG;
+    }
+  }
+  std::unique_ptr<hs_stage> s(new (std::nothrow) hs_stage());
+  if (!s) return HS_ERR_INVALID_ARG;
+  s->cfg = *cfg;
+  s->ml = make_meta_layout(*cfg);
+  s->ws = make_ws_layout(*cfg, s->ml);
+  s->alloc.reset(new PageAllocator(cfg->num_pages));
+  s->page_stamp.assign(cfg->num_pages, 0);
+  if (host_only) {
+    *out = s.release();
+    return HS_OK;
+  }
+
+  DeviceGuard guard(cfg->device);
+  if (!guard.ok) return HS_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return HS_ERR_CUDA;
+  if (prop.major != 10) return HS_ERR_CUDA;   // the kernels exist for sm_100a only
+  s->sm_count = prop.multiProcessorCount;
+  if ((st = ensure_attributes(cfg->device)) != HS_OK) return st;
+  s->ws_dev = static_cast<uint8_t*>(workspace_dev);
+  s->kv_pool = static_cast<__nv_bfloat16*>(kv_pool_dev);
+  s->layers.assign(layers, layers + cfg->n_layers);
+
+  // RoPE table: angle and cos/sin in double, stored as fp32 (cos, sin)
+  const int half = cfg->head_dim / 2;
+  std::vector<float2> rope(size_t(cfg->max_position) * half);
+  for (int i = 0; i < half; ++i) {
+    const double theta = pow(double(cfg->rope_base), -2.0 * i / double(cfg->head_dim));
+    for (int pos = 0; pos < cfg->max_position; ++pos) {
+      const double phi = double(pos) * theta;
+      rope[size_t(pos) * half + i] = make_float2(float(cos(phi)), float(sin(phi)));
+    }
+  }
+  if (cudaMemcpy(s->ws_dev + s->ws.rope, rope.data(), rope.size() * sizeof(float2), cudaMemcpyHostToDevice) !=
+          cudaSuccess ||
+      cudaMemset(s->ws_dev + s->ws.status, 0, 256) != cudaSuccess)
+    return HS_ERR_CUDA;
+
+  // tensor maps
+  const uint64_t T = cfg->max_tokens, d = cfg->d_model, F = cfg->d_ffn;
+  const uint64_t q_dim = uint64_t(cfg->n_q_heads) * cfg->head_dim, kv_dim = uint64_t(cfg->n_kv_heads) * cfg->head_dim;
+  bool ok = encode_2d(&s->tm_h, s->ws_dev + s->ws.h, T, d, 128) && encode_2d(&s->tm_o, s->ws_dev + s->ws.o, T, q_dim, 128) &&
+            encode_2d(&s->tm_act, s->ws_dev + s->ws.act, T, F, 128);
+  const uint64_t pool_rows = uint64_t(cfg->n_layers) * 2 * cfg->num_pages * cfg->n_kv_heads * kPage;
+  ok = ok && encode_2d(&s->tm_kv, s->kv_pool, pool_rows, cfg->head_dim, 16);
+  s->maps.resize(cfg->n_layers);
+  for (int l = 0; l < cfg->n_layers && ok; ++l) {
+    LayerMaps& m = s->maps[l];
+    const hs_layer_weights_t& w = s->layers[l];
+    ok = encode_2d(&m.wq, w.w_q, q_dim, d, 128) && encode_2d(&m.wk, w.w_k, kv_dim, d, 128) &&
+         encode_2d(&m.wv, w.w_v, kv_dim, d, 128) && encode_2d(&m.wo, w.w_o, d, q_dim, 128) &&
+         encode_2d(&m.wgate, w.w_gate, F, d, 128) && encode_2d(&m.wup, w.w_up, F, d, 128) &&
+         encode_2d(&m.wdown, w.w_down, d, F, 128);
+  }
+  if (!ok) return HS_ERR_CUDA;
+
+  for (int i = 0; i < kRing; ++i) {
+    if (cudaHostAlloc(reinterpret_cast<void**>(&s->pinned[i]), size_t(s->ml.total) * 4, cudaHostAllocDefault) !=
+            cudaSuccess ||
+        cudaEventCreateWithFlags(&s->ev[i], cudaEventDisableTiming) != cudaSuccess) {
+      hs_stage_destroy(s.release());
+      return HS_ERR_CUDA;
+    }
+  }
+  if (cudaDeviceSynchronize() != cudaSuccess) {
+    hs_stage_destroy(s.release());
+    return HS_ERR_CUDA;
+  }
+  *out = s.release();
+  return HS_OK;
+}
+
+hs_status_t hs_stage_destroy(hs_stage_t* s) {
+  if (!s) return HS_ERR_INVALID_ARG;
+  if (s->cfg.device >= 0) {
+    DeviceGuard guard(s->cfg.device);
+    for (int i = 0; i < kRing; ++i) {
+      if (s->ev[i]) {
+        if (s->ev_pending[i]) cudaEventSynchronize(s->ev[i]);
+        cudaEventDestroy(s->ev[i]);
+      }
+      if (s->pinned[i]) cudaFreeHost(s->pinned[i]);
+    }
+  }
+  delete s;
+  return HS_OK;
+}
+
+hs_status_t hs_kv_alloc(hs_stage_t* s, int64_t seq_id, int32_t total_tokens, int32_t* table_out, int32_t cap,
+                        int32_t* n_pages_out) {
+  if (!s || total_tokens < 0 || cap < 0 || (cap > 0 && !table_out)) return HS_ERR_INVALID_ARG;
+  if (ceil_div(total_tokens, kPage) > cap) return HS_ERR_INVALID_ARG;
+  const std::vector<int32_t>* table = nullptr;
+  const hs_status_t st = s->alloc->grow(seq_id, total_tokens, &table);
+  if (st != HS_OK) return st;
+  if (int(table->size()) > cap) return HS_ERR_INVALID_ARG;   // owned more than asked before: still reported whole
+  for (size_t i = 0; i < table->size(); ++i) table_out[i] = (*table)[i];
+  if (n_pages_out) *n_pages_out = int32_t(table->size());
+  return HS_OK;
+}
+
+hs_status_t hs_kv_free(hs_stage_t* s, int64_t seq_id) {
+  if (!s) return HS_ERR_INVALID_ARG;
+  return s->alloc->release(seq_id);
+}
+
+int32_t hs_kv_free_pages(const hs_stage_t* s) { return s ? s->alloc->free_pages() : -1; }
+
+int32_t hs_stage_sm_count(const hs_stage_t* s) { return s ? s->sm_count : 0; }
+
+hs_status_t hs_stage_plan(hs_stage_t* s, const hs_batch_t* b, int32_t* tok_seq, int32_t* tok_pos, int32_t* tok_slot) {
+  if (!s || !b) return HS_ERR_INVALID_ARG;
+  std::vector<int32_t> meta(s->ml.total);
+  StepPlan plan;
+  const hs_status_t st = plan_step(s->cfg, s->ml, *b, s->page_stamp, ++s->stamp, meta.data(), tok_seq, &plan);
+  if (st != HS_OK) return st;
+  if (tok_pos) memcpy(tok_pos, meta.data() + s->ml.tok_pos, size_t(plan.n_tokens) * 4);
+  if (tok_slot) memcpy(tok_slot, meta.data() + s->ml.tok_slot, size_t(plan.n_tokens) * 4);
+  return HS_OK;
+}
+
+hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget, void* cuda_stream) {
+  if (!s || !b) return HS_ERR_INVALID_ARG;
+  if (s->cfg.device < 0) return HS_ERR_NO_DEVICE;
+  if (sm_budget < 1 || sm_budget > s->sm_count) return HS_ERR_INVALID_BUDGET;
+  if (!b->x_in || !b->y_out || (reinterpret_cast<uintptr_t>(b->x_in) & 15) || (reinterpret_cast<uintptr_t>(b->y_out) & 15))
+    return HS_ERR_INVALID_ARG;
+  const hs_stage_config_t& c = s->cfg;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  DeviceGuard guard(c.device);
+  if (!guard.ok) return HS_ERR_CUDA;
+
+  // plan into the next pinned slot (waiting for the copy that last used it)
+  const int slot = s->ring_pos;
+  if (s->ev_pending[slot]) {
+    if (cudaEventSynchronize(s->ev[slot]) != cudaSuccess) return HS_ERR_CUDA;
+    s->ev_pending[slot] = false;
+  }
+  StepPlan plan;
+  hs_status_t st = plan_step(c, s->ml, *b, s->page_stamp, ++s->stamp, s->pinned[slot], nullptr, &plan);
+  if (st != HS_OK) return st;
+  s->ring_pos = (slot + 1) % kRing;
+
+  int32_t* meta = reinterpret_cast<int32_t*>(s->ws_dev + s->ws.meta);
+  if (cudaMemcpyAsync(meta, s->pinned[slot], size_t(s->ml.total) * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaEventRecord(s->ev[slot], stream) != cudaSuccess)
+    return HS_ERR_CUDA;
+  s->ev_pending[slot] = true;
+
+  const int T = plan.n_tokens, d = c.d_model, F = c.d_ffn, Dh = c.head_dim;
+  const int q_dim = c.n_q_heads * Dh, kv_dim = c.n_kv_heads * Dh;
+  float* x = reinterpret_cast<float*>(s->ws_dev + s->ws.x);
+  __nv_bfloat16* h = reinterpret_cast<__nv_bfloat16*>(s->ws_dev + s->ws.h);
+  __nv_bfloat16* q = reinterpret_cast<__nv_bfloat16*>(s->ws_dev + s->ws.q);
+  __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(s->ws_dev + s->ws.o);
+  __nv_bfloat16* act = reinterpret_cast<__nv_bfloat16*>(s->ws_dev + s->ws.act);
+  int* status = reinterpret_cast<int*>(s->ws_dev + s->ws.status);
+  const size_t layer_kv_elems = size_t(c.num_pages) * c.n_kv_heads * kPage * Dh;
+  cudaError_t e = cudaSuccess;
+
+  for (int l = 0; l < c.n_layers && e == cudaSuccess; ++l) {
+    const hs_layer_weights_t& w = s->layers[l];
+    const LayerMaps& m = s->maps[l];
+    const bool last = l == c.n_layers - 1;
+
+    NormParams np{};
+    np.x_bf16 = l == 0 ? static_cast<const __nv_bfloat16*>(b->x_in) : nullptr;
+    np.x_f32 = x;
+    np.x_f32_out = x;
+    np.gain = static_cast<const __nv_bfloat16*>(w.g_attn);
+    np.h = h;
+    np.T = T;
+    np.d = d;
+    np.eps = c.rms_eps;
+    if ((e = launch_rmsnorm(np, sm_budget, stream)) != cudaSuccess) break;
+
+    GemmParams g{};
+    g.tm_a = s->tm_h;
+    g.tm_b[0] = m.wq; g.tm_b[1] = m.wk; g.tm_b[2] = m.wv;
+    g.M = T; g.N = q_dim + 2 * kv_dim; g.K = d;
+    g.mode = kGemmQkv;
+    g.q_dim = q_dim; g.kv_dim = kv_dim; g.head_dim = Dh; g.n_kv_heads = c.n_kv_heads;
+    g.q_out = q;
+    g.k_cache = s->kv_pool + (size_t(l) * 2 + 0) * layer_kv_elems;
+    g.v_cache = s->kv_pool + (size_t(l) * 2 + 1) * layer_kv_elems;
+    g.tok_pos = meta + s->ml.tok_pos;
+    g.tok_slot = meta + s->ml.tok_slot;
+    g.rope = reinterpret_cast<const float2*>(s->ws_dev + s->ws.rope);
+    g.status = status;
+    if ((e = launch_gemm(g, sm_budget, stream)) != cudaSuccess) break;
+
+    AttnParams a{};
+    a.tm_kv = s->tm_kv;
+    a.q = q; a.o = o;
+    a.n_q_heads = c.n_q_heads; a.n_kv_heads = c.n_kv_heads; a.head_dim = Dh;
+    a.num_pages = c.num_pages; a.max_pages_per_seq = c.max_pages_per_seq; a.layer = l;
+    a.seq_tok0 = meta + s->ml.seq_tok0;
+    a.seq_ctx = meta + s->ml.seq_ctx;
+    a.block_tables = meta + s->ml.block_tables;
+    a.prefill_items = meta + s->ml.prefill_items;
+    a.n_prefill_items = plan.n_prefill_items;
+    a.decode_items = meta + s->ml.decode_items;
+    a.n_decode_items = plan.n_decode_items;
+    a.decode_rows = meta + s->ml.decode_rows;
+    a.n_decode_rows = plan.n_decode_rows;
+    a.part_o = reinterpret_cast<float*>(s->ws_dev + s->ws.part_o);
+    a.part_ml = reinterpret_cast<float*>(s->ws_dev + s->ws.part_ml);
+    a.counters = meta + s->ml.counters + 2 * l;
+    a.status = status;
+    if ((e = launch_attention_prefill(a, sm_budget, stream)) != cudaSuccess) break;
+    if ((e = launch_attention_decode(a, sm_budget, stream)) != cudaSuccess) break;
+    if ((e = launch_attention_combine(a, sm_budget, stream)) != cudaSuccess) break;
+
+    GemmParams go{};
+    go.tm_a = s->tm_o;
+    go.tm_b[0] = m.wo; go.tm_b[1] = m.wo; go.tm_b[2] = m.wo;
+    go.M = T; go.N = d; go.K = q_dim;
+    go.mode = kGemmResid;
+    go.resid = x; go.out = x;
+    go.status = status;
+    if ((e = launch_gemm(go, sm_budget, stream)) != cudaSuccess) break;
+
+    np.x_bf16 = nullptr;
+    np.gain = static_cast<const __nv_bfloat16*>(w.g_mlp);
+    if ((e = launch_rmsnorm(np, sm_budget, stream)) != cudaSuccess) break;
+
+    GemmParams gu{};
+    gu.tm_a = s->tm_h;
+    gu.tm_b[0] = m.wgate; gu.tm_b[1] = m.wup; gu.tm_b[2] = m.wup;
+    gu.M = T; gu.N = F; gu.K = d;
+    gu.mode = kGemmGateUp;
+    gu.act = act;
+    gu.status = status;
+    if ((e = launch_gemm(gu, sm_budget, stream)) != cudaSuccess) break;
+
+    GemmParams gd{};
+    gd.tm_a = s->tm_act;
+    gd.tm_b[0] = m.wdown; gd.tm_b[1] = m.wdown; gd.tm_b[2] = m.wdown;
+    gd.M = T; gd.N = d; gd.K = F;
+    gd.mode = kGemmResid;
+    gd.resid = x;
+    gd.out = last ? static_cast<float*>(b->y_out) : x;
+    gd.status = status;
+    if ((e = launch_gemm(gd, sm_budget, stream)) != cudaSuccess) break;
+  }
+  return e == cudaSuccess ? HS_OK : HS_ERR_CUDA;
+}
+
+hs_status_t hs_stage_status(hs_stage_t* s) {
+  if (!s) return HS_ERR_INVALID_ARG;
+  if (s->cfg.device < 0) return HS_ERR_NO_DEVICE;
+  DeviceGuard guard(s->cfg.device);
+  int v = 0;
+  if (cudaMemcpy(&v, s->ws_dev + s->ws.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return HS_ERR_CUDA;
+  return v == 0 ? HS_OK : static_cast<hs_status_t>(v);
+}
+
+hs_status_t hs_stage_debug_buffer(hs_stage_t* s, const char* name, void** dev_ptr, size_t* bytes) {
+  if (!s || !name || !dev_ptr || !bytes) return HS_ERR_INVALID_ARG;
+  if (s->cfg.device < 0) return HS_ERR_NO_DEVICE;
+  const hs_stage_config_t& c = s->cfg;
+  const size_t T = c.max_tokens, q_dim = size_t(c.n_q_heads) * c.head_dim;
+  const std::string n(name);
+  size_t off, sz;
+  if (n == "x") { off = s->ws.x; sz = T * c.d_model * 4; }
+  else if (n == "h") { off = s->ws.h; sz = T * c.d_model * 2; }
+  else if (n == "q") { off = s->ws.q; sz = T * q_dim * 2; }
+  else if (n == "o") { off = s->ws.o; sz = T * q_dim * 2; }
+  else if (n == "act") { off = s->ws.act; sz = T * c.d_ffn * 2; }
+  else return HS_ERR_INVALID_ARG;
+  *dev_ptr = s->ws_dev + off;
+  *bytes = sz;
+  return HS_OK;
+}
+
+hs_status_t hs_op_gemm_bf16(const void* a, const void* w, const float* resid, float* out, int32_t M, int32_t N, int32_t K,
+                            int32_t sm_budget, int32_t* status_dev, void* cuda_stream) {
+  if (!a || !w || !out || !status_dev || M < 1 || N < 1 || K < 1) return HS_ERR_INVALID_ARG;
+  if ((N & 7) || (K & 7)) return HS_ERR_UNSUPPORTED_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(a) & 15) || (reinterpret_cast<uintptr_t>(w) & 15) ||
+      (reinterpret_cast<uintptr_t>(out) & 15) || (reinterpret_cast<uintptr_t>(resid) & 15))
+    return HS_ERR_INVALID_ARG;
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return HS_ERR_CUDA;
+  if (prop.major != 10) return HS_ERR_CUDA;
+  if (sm_budget < 1 || sm_budget > prop.multiProcessorCount) return HS_ERR_INVALID_BUDGET;
+  if (ensure_attributes(dev) != HS_OK) return HS_ERR_CUDA;
+  GemmParams g{};
+  if (!encode_2d(&g.tm_a, a, M, K, 128) || !encode_2d(&g.tm_b[0], w, N, K, 128)) return HS_ERR_CUDA;
+  g.tm_b[1] = g.tm_b[0];
+  g.tm_b[2] = g.tm_b[0];
+  g.M = M; g.N = N; g.K = K;
+  g.mode = kGemmResid;
+  g.resid = resid;
+  g.out = out;
+  g.status = status_dev;
+  return launch_gemm(g, sm_budget, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? HS_OK : HS_ERR_CUDA;
+}
+
+}  // extern "C"

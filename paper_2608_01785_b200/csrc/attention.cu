@@ -1,0 +1,583 @@
+// Causal GQA attention over the paged bf16 KV cache: TMA-staged K/V pages, warp-level tensor-core tiles
+// (mma.sync m16n8k16) and an fp32 online softmax in the log2 domain.
+//
+//   prefill kernel   work item = (sequence, KV head, tile of 128/G tokens); the G query heads that share
+//                    the KV head are stacked as rows, so K/V are streamed once per KV head.  8 compute
+//                    warps x 16 rows, key blocks of 64 keys (4 pages) in a 4-stage ring fed by one
+//                    producer thread.
+//   decode kernel    work item = (sequence, KV head, run of <= 512 keys); rows = the G query heads of the
+//                    single new token.  4 compute warps each take one page of every 4-page stage; their
+//                    partial (max, sum, output) triples are merged in shared memory in warp order and
+//                    written as one partial per item.  HBM-bound: 5 stages x 32 KB in flight per SM.
+//   combine kernel   merges the partials of a sequence's splits in split order.
+// Work items are listed on the host independently of the SM budget and handed out through an atomic
+// queue head; an item's result does not depend on which block ran it, and every reduction has a fixed
+// order, so outputs are bit-identical across budgets.
+//
+// A page block [16 keys][Dh] arrives as Dh/64 tiles of [16][64] with the 128-byte swizzle, which makes
+// every ldmatrix below bank-conflict free.  Keys past the end of a sequence (the unused tail of its last
+// page, or pages of a ragged last block that were never fetched) may hold arbitrary bytes: scores are
+// masked by selection and the matching V fragments are zeroed, so they cannot reach the output.
+#include <math.h>
+
+#include "kernels.h"
+#include "ptx.cuh"
+
+namespace hs {
+namespace {
+
+constexpr float kLog2e = 1.4426950408889634f;
+
+template <int DH>
+struct Geom {
+  static constexpr int HALVES = DH / 64;
+  static constexpr int PAGE_BYTES = HALVES * 2048;   // [HALVES][16 keys][128 B]
+  static constexpr int CHUNKS = DH / 8;              // 16-byte chunks per row
+};
+
+// Byte offset of (key kk, 16-byte chunk cc) inside a page block.
+__device__ __forceinline__ int kv_off(int kk, int cc) {
+  return (cc >> 3) * 2048 + kk * 128 + (((cc & 7) ^ (kk & 7)) << 4);
+}
+// First pool row (unit: one key's Dh elements of one KV head) of (layer, K|V, page, head).
+__device__ __forceinline__ int pool_row(const AttnParams& p, int kv, int page, int hk) {
+  return (((p.layer * 2 + kv) * p.num_pages + page) * p.n_kv_heads + hk) * 16;
+}
+template <int DH>
+__device__ __forceinline__ void load_page(const AttnParams& p, uint8_t* dst, uint64_t* bar, int kv, int page, int hk) {
+  const int row = pool_row(p, kv, page, hk);
+#pragma unroll
+  for (int h = 0; h < Geom<DH>::HALVES; ++h) tma_load_2d(dst + h * 2048, &p.tm_kv, bar, h * 64, row);
+}
+__device__ __forceinline__ float quad_max(float v) {
+  v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 1));
+  return fmaxf(v, __shfl_xor_sync(0xffffffffu, v, 2));
+}
+__device__ __forceinline__ float quad_sum(float v) {
+  v += __shfl_xor_sync(0xffffffffu, v, 1);
+  return v + __shfl_xor_sync(0xffffffffu, v, 2);
+}
+// Zeroes the halves of a V fragment register whose keys (k, k + 1) are not below n_valid.
+__device__ __forceinline__ uint32_t mask_v(uint32_t r, int k, int n_valid) {
+  if (k >= n_valid) return 0u;
+  if (k + 1 >= n_valid) return r & 0x0000ffffu;
+  return r;
+}
+
+// =================================================================== prefill ==
+constexpr int PF_WARPS = 8, PF_THREADS = (PF_WARPS + 1) * 32, PF_STAGES = 4, PF_BLOCK_KEYS = 64;
+
+template <int DH>
+constexpr int pf_smem_bytes() {
+  int b = 1024 + Geom<DH>::HALVES * 16384 + PF_STAGES * 8 * Geom<DH>::PAGE_BYTES + 256;
+  return b > kMinSmemBytes ? b : kMinSmemBytes;
+}
+
+template <int DH>
+__global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __grid_constant__ AttnParams p) {
+  using G_ = Geom<DH>;
+  constexpr int STAGE_BYTES = 8 * G_::PAGE_BYTES;   // 4 K pages then 4 V pages
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* q_smem = smem;                                      // [HALVES][128 rows][128 B], swizzled
+  uint8_t* stages = smem + G_::HALVES * 16384;
+  uint64_t* full = reinterpret_cast<uint64_t*>(stages + PF_STAGES * STAGE_BYTES);
+  uint64_t* empty = full + PF_STAGES;
+  int* s_item = reinterpret_cast<int*>(empty + PF_STAGES);   // two slots, used alternately
+  volatile int* abort_flag = s_item + 2;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = p.n_q_heads / p.n_kv_heads;
+  const int q_dim = p.n_q_heads * DH;
+  const float scale_log2 = kLog2e / sqrtf(float(DH));
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < PF_STAGES; ++i) {
+      mbar_init(&full[i], 1);
+      mbar_init(&empty[i], PF_WARPS);
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+    tma_prefetch_desc(&p.tm_kv);
+  }
+  __syncthreads();
+
+  int s = 0;
+  uint32_t ph = 0;
+  bool alive = true;
+  for (int round = 0;; round ^= 1) {
+    // one barrier per item: a thread is never more than one item ahead, so two slots suffice
+    if (threadIdx.x == 0) s_item[round] = atomicAdd(p.counters, 1);
+    __syncthreads();
+    const int item = s_item[round];
+    if (item >= p.n_prefill_items || *abort_flag) break;
+    const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
+    const int seq = it.x, hk = it.y, tok_begin = it.z, n_tok = it.w;
+    const int ctx = p.seq_ctx[seq];
+    const int tok0 = p.seq_tok0[seq] + tok_begin;
+    const int pos0 = ctx + tok_begin;                 // position of the tile's first token
+    const int n_keys = pos0 + n_tok;
+    const int n_kblocks = (n_keys + PF_BLOCK_KEYS - 1) / PF_BLOCK_KEYS;
+    const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq;
+
+    if (warp == PF_WARPS) {
+      // ----------------------------------------------------------- producer --
+      if (lane == 0 && alive) {
+        for (int kb = 0; kb < n_kblocks; ++kb) {
+          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status)) { alive = false; break; }
+          const int rem = n_keys - kb * PF_BLOCK_KEYS;
+          const int np = rem >= PF_BLOCK_KEYS ? 4 : (rem + 15) >> 4;
+          uint8_t* st = stages + s * STAGE_BYTES;
+          mbar_expect_tx(&full[s], np * 2 * G_::PAGE_BYTES);
+          for (int w = 0; w < np; ++w) {
+            const int page = table[kb * 4 + w];
+            load_page<DH>(p, st + w * G_::PAGE_BYTES, &full[s], 0, page, hk);
+            load_page<DH>(p, st + (4 + w) * G_::PAGE_BYTES, &full[s], 1, page, hk);
+          }
+          if (++s == PF_STAGES) { s = 0; ph ^= 1; }
+        }
+      }
+    } else {
+      // ---------------------------------------------------------- consumers --
+      const int n_rows = n_tok * G;
+      // stage the Q tile: row r = (token r / G, query head hk*G + r % G)
+      for (int idx = threadIdx.x; idx < 128 * G_::CHUNKS; idx += PF_WARPS * 32) {
+        const int r = idx / G_::CHUNKS, cc = idx % G_::CHUNKS;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (r < n_rows) {
+          const __nv_bfloat16* src = p.q + size_t(tok0 + r / G) * q_dim + (hk * G + r % G) * DH + cc * 8;
+          v = *reinterpret_cast<const uint4*>(src);
+        }
+        *reinterpret_cast<uint4*>(q_smem + (cc >> 3) * 16384 + r * 128 + (((cc & 7) ^ (r & 7)) << 4)) = v;
+      }
+      named_barrier_sync(1, PF_WARPS * 32);
+      uint32_t qf[DH / 16][4];
+#pragma unroll
+      for (int ks = 0; ks < DH / 16; ++ks) {
+        const int r = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, cc = 2 * ks + (lane >> 4);
+        ldmatrix_x4(qf[ks], smem_u32(q_smem + (cc >> 3) * 16384 + r * 128 + (((cc & 7) ^ (r & 7)) << 4)));
+      }
+      // positions of this thread's two rows (padding rows behave like the tile's last token)
+      const int row_a = warp * 16 + (lane >> 2), row_b = row_a + 8;
+      const int pos_a = pos0 + min(row_a / G, n_tok - 1), pos_b = pos0 + min(row_b / G, n_tok - 1);
+      const bool warp_has_rows = warp * 16 < n_rows;
+      const int warp_min_pos = pos0 + min((warp * 16) / G, n_tok - 1);
+      const int warp_max_pos = pos0 + min((warp * 16 + 15) / G, n_tok - 1);
+
+      float o_acc[DH / 8][4];
+#pragma unroll
+      for (int j = 0; j < DH / 8; ++j) o_acc[j][0] = o_acc[j][1] = o_acc[j][2] = o_acc[j][3] = 0.f;
+      float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
+
+      for (int kb = 0; kb < n_kblocks; ++kb) {
+        const bool ok = alive && mbar_wait(&full[s], ph, abort_flag, p.status);
+        if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+        const int key0 = kb * PF_BLOCK_KEYS;
+        if (warp_has_rows && key0 <= warp_max_pos) {
+          const uint32_t k_base = smem_u32(stages + s * STAGE_BYTES);
+          const uint32_t v_base = k_base + 4 * G_::PAGE_BYTES;
+          const int rem = n_keys - key0;
+          const int np = rem >= PF_BLOCK_KEYS ? 4 : (rem + 15) >> 4;   // pages present in this stage
+          float sc[8][4];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f;
+#pragma unroll
+          for (int ks = 0; ks < DH / 16; ++ks) {
+#pragma unroll
+            for (int pg = 0; pg < 4; ++pg) {
+              uint32_t kf[4];
+              const int kk = (lane & 7) + (lane >> 4) * 8, cc = 2 * ks + ((lane >> 3) & 1);
+              ldmatrix_x4(kf, k_base + pg * G_::PAGE_BYTES + kv_off(kk, cc));
+              mma_bf16_16816(sc[2 * pg], qf[ks], kf[0], kf[1]);
+              mma_bf16_16816(sc[2 * pg + 1], qf[ks], kf[2], kf[3]);
+            }
+          }
+          // scale, causal mask (by selection), block max
+          const bool need_mask = key0 + PF_BLOCK_KEYS - 1 > warp_min_pos;
+          float mx_a = -INFINITY, mx_b = -INFINITY;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              float v = sc[j][e] * scale_log2;
+              if (need_mask) {
+                const int key = key0 + 8 * j + 2 * (lane & 3) + (e & 1);
+                if (key > (e < 2 ? pos_a : pos_b)) v = -INFINITY;
+              }
+              sc[j][e] = v;
+            }
+            mx_a = fmaxf(mx_a, fmaxf(sc[j][0], sc[j][1]));
+            mx_b = fmaxf(mx_b, fmaxf(sc[j][2], sc[j][3]));
+          }
+          mx_a = quad_max(mx_a);
+          mx_b = quad_max(mx_b);
+          const float mn_a = fmaxf(m_a, mx_a), mn_b = fmaxf(m_b, mx_b);
+          const float al_a = exp2f(m_a - mn_a), al_b = exp2f(m_b - mn_b);
+          m_a = mn_a;
+          m_b = mn_b;
+          float sum_a = 0.f, sum_b = 0.f;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            sc[j][0] = exp2f(sc[j][0] - mn_a);
+            sc[j][1] = exp2f(sc[j][1] - mn_a);
+            sc[j][2] = exp2f(sc[j][2] - mn_b);
+            sc[j][3] = exp2f(sc[j][3] - mn_b);
+            sum_a += sc[j][0] + sc[j][1];
+            sum_b += sc[j][2] + sc[j][3];
+          }
+          l_a = l_a * al_a + sum_a;
+          l_b = l_b * al_b + sum_b;
+#pragma unroll
+          for (int j = 0; j < DH / 8; ++j) {
+            o_acc[j][0] *= al_a; o_acc[j][1] *= al_a;
+            o_acc[j][2] *= al_b; o_acc[j][3] *= al_b;
+          }
+          // O += P V, one page (16 keys) per k-step
+#pragma unroll
+          for (int pg = 0; pg < 4; ++pg) {
+            if (pg < np) {
+              uint32_t pf[4];
+              pf[0] = pack_bf16(sc[2 * pg][0], sc[2 * pg][1]);
+              pf[1] = pack_bf16(sc[2 * pg][2], sc[2 * pg][3]);
+              pf[2] = pack_bf16(sc[2 * pg + 1][0], sc[2 * pg + 1][1]);
+              pf[3] = pack_bf16(sc[2 * pg + 1][2], sc[2 * pg + 1][3]);
+              const int n_valid = rem - pg * 16;      // keys of this page that exist
+#pragma unroll
+              for (int dp = 0; dp < DH / 16; ++dp) {
+                uint32_t vf[4];
+                const int kk = (lane & 7) + ((lane >> 3) & 1) * 8, cc = 2 * dp + (lane >> 4);
+                ldmatrix_x4_trans(vf, v_base + pg * G_::PAGE_BYTES + kv_off(kk, cc));
+                if (n_valid < 16) {
+                  const int k = 2 * (lane & 3);
+                  vf[0] = mask_v(vf[0], k, n_valid);
+                  vf[1] = mask_v(vf[1], k + 8, n_valid);
+                  vf[2] = mask_v(vf[2], k, n_valid);
+                  vf[3] = mask_v(vf[3], k + 8, n_valid);
+                }
+                mma_bf16_16816(o_acc[2 * dp], pf, vf[0], vf[1]);
+                mma_bf16_16816(o_acc[2 * dp + 1], pf, vf[2], vf[3]);
+              }
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[s]);
+        if (++s == PF_STAGES) { s = 0; ph ^= 1; }
+      }
+      if (alive && warp_has_rows) {
+        l_a = quad_sum(l_a);
+        l_b = quad_sum(l_b);
+        const float inv_a = 1.f / l_a, inv_b = 1.f / l_b;
+#pragma unroll
+        for (int j = 0; j < DH / 8; ++j) {
+          const int col = 8 * j + 2 * (lane & 3);
+          if (row_a < n_rows) {
+            __nv_bfloat16* dst = p.o + size_t(tok0 + row_a / G) * q_dim + (hk * G + row_a % G) * DH + col;
+            *reinterpret_cast<uint32_t*>(dst) = pack_bf16(o_acc[j][0] * inv_a, o_acc[j][1] * inv_a);
+          }
+          if (row_b < n_rows) {
+            __nv_bfloat16* dst = p.o + size_t(tok0 + row_b / G) * q_dim + (hk * G + row_b % G) * DH + col;
+            *reinterpret_cast<uint32_t*>(dst) = pack_bf16(o_acc[j][2] * inv_b, o_acc[j][3] * inv_b);
+          }
+        }
+      }
+    }
+  }
+  __syncwarp();
+  if (*abort_flag) drain_after_abort();
+}
+
+// ==================================================================== decode ==
+constexpr int DC_WARPS = 4, DC_THREADS = (DC_WARPS + 1) * 32, DC_STAGES = 5;
+
+template <int DH>
+constexpr int dc_smem_bytes() {
+  int b = 1024 + DC_STAGES * 8 * Geom<DH>::PAGE_BYTES + DC_WARPS * 16 * DH * 4 + DC_WARPS * 16 * 2 * 4 + 256;
+  return b > kMinSmemBytes ? b : kMinSmemBytes;
+}
+
+template <int DH>
+__global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid_constant__ AttnParams p) {
+  using G_ = Geom<DH>;
+  constexpr int STAGE_BYTES = 8 * G_::PAGE_BYTES;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* stages = smem;
+  float* sm_o = reinterpret_cast<float*>(stages + DC_STAGES * STAGE_BYTES);   // [warp][16][DH]
+  float* sm_ml = sm_o + DC_WARPS * 16 * DH;                                   // [warp][16][2]
+  uint64_t* full = reinterpret_cast<uint64_t*>(sm_ml + DC_WARPS * 16 * 2);
+  uint64_t* empty = full + DC_STAGES;
+  int* s_item = reinterpret_cast<int*>(empty + DC_STAGES);   // two slots, used alternately
+  volatile int* abort_flag = s_item + 2;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = p.n_q_heads / p.n_kv_heads;
+  const int q_dim = p.n_q_heads * DH;
+  const float scale_log2 = kLog2e / sqrtf(float(DH));
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < DC_STAGES; ++i) {
+      mbar_init(&full[i], 1);
+      mbar_init(&empty[i], DC_WARPS);
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+    tma_prefetch_desc(&p.tm_kv);
+  }
+  __syncthreads();
+
+  int s = 0;
+  uint32_t ph = 0;
+  bool alive = true;
+  for (int round = 0;; round ^= 1) {
+    if (threadIdx.x == 0) s_item[round] = atomicAdd(p.counters + 1, 1);
+    __syncthreads();
+    const int item = s_item[round];
+    if (item >= p.n_decode_items || *abort_flag) break;
+    const int4 it = reinterpret_cast<const int4*>(p.decode_items)[item];
+    const int seq = it.x, hk = it.y, k0 = it.z, k1 = it.w;
+    const int n_pages = (k1 - k0 + 15) >> 4, first_page = k0 >> 4;
+    const int n_iters = (n_pages + 3) >> 2;
+    const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq + first_page;
+
+    if (warp == DC_WARPS) {
+      if (lane == 0 && alive) {
+        for (int i = 0; i < n_iters; ++i) {
+          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status)) { alive = false; break; }
+          const int np = min(4, n_pages - i * 4);
+          uint8_t* st = stages + s * STAGE_BYTES;
+          mbar_expect_tx(&full[s], np * 2 * G_::PAGE_BYTES);
+          for (int w = 0; w < np; ++w) {
+            const int page = table[i * 4 + w];
+            load_page<DH>(p, st + w * G_::PAGE_BYTES, &full[s], 0, page, hk);
+            load_page<DH>(p, st + (4 + w) * G_::PAGE_BYTES, &full[s], 1, page, hk);
+          }
+          if (++s == DC_STAGES) { s = 0; ph ^= 1; }
+        }
+      }
+    } else {
+      // Q fragments straight from global memory: rows = query heads hk*G .. hk*G + G - 1 of the new token
+      const int tok = p.seq_tok0[seq];
+      const __nv_bfloat16* qrow = p.q + size_t(tok) * q_dim + size_t(hk) * G * DH;
+      const int ra = lane >> 2, rb = ra + 8;
+      uint32_t qf[DH / 16][4];
+#pragma unroll
+      for (int ks = 0; ks < DH / 16; ++ks) {
+        const int c = ks * 16 + 2 * (lane & 3);
+        qf[ks][0] = ra < G ? *reinterpret_cast<const uint32_t*>(qrow + ra * DH + c) : 0u;
+        qf[ks][1] = rb < G ? *reinterpret_cast<const uint32_t*>(qrow + rb * DH + c) : 0u;
+        qf[ks][2] = ra < G ? *reinterpret_cast<const uint32_t*>(qrow + ra * DH + c + 8) : 0u;
+        qf[ks][3] = rb < G ? *reinterpret_cast<const uint32_t*>(qrow + rb * DH + c + 8) : 0u;
+      }
+      float o_acc[DH / 8][4];
+#pragma unroll
+      for (int j = 0; j < DH / 8; ++j) o_acc[j][0] = o_acc[j][1] = o_acc[j][2] = o_acc[j][3] = 0.f;
+      float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
+
+      for (int i = 0; i < n_iters; ++i) {
+        const bool ok = alive && mbar_wait(&full[s], ph, abort_flag, p.status);
+        if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+        const int pi = i * 4 + warp;
+        if (pi < n_pages) {
+          const uint32_t k_base = smem_u32(stages + s * STAGE_BYTES + warp * G_::PAGE_BYTES);
+          const uint32_t v_base = k_base + 4 * G_::PAGE_BYTES;
+          const int n_valid = k1 - (k0 + pi * 16);          // keys of this page that belong to the item
+          float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+#pragma unroll
+          for (int ks = 0; ks < DH / 16; ++ks) {
+            uint32_t kf[4];
+            const int kk = (lane & 7) + (lane >> 4) * 8, cc = 2 * ks + ((lane >> 3) & 1);
+            ldmatrix_x4(kf, k_base + kv_off(kk, cc));
+            mma_bf16_16816(sc[0], qf[ks], kf[0], kf[1]);
+            mma_bf16_16816(sc[1], qf[ks], kf[2], kf[3]);
+          }
+          float mx_a = -INFINITY, mx_b = -INFINITY;
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              float v = sc[j][e] * scale_log2;
+              if (8 * j + 2 * (lane & 3) + (e & 1) >= n_valid) v = -INFINITY;
+              sc[j][e] = v;
+            }
+            mx_a = fmaxf(mx_a, fmaxf(sc[j][0], sc[j][1]));
+            mx_b = fmaxf(mx_b, fmaxf(sc[j][2], sc[j][3]));
+          }
+          mx_a = quad_max(mx_a);
+          mx_b = quad_max(mx_b);
+          const float mn_a = fmaxf(m_a, mx_a), mn_b = fmaxf(m_b, mx_b);
+          const float al_a = exp2f(m_a - mn_a), al_b = exp2f(m_b - mn_b);
+          m_a = mn_a;
+          m_b = mn_b;
+          float sum_a = 0.f, sum_b = 0.f;
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            sc[j][0] = exp2f(sc[j][0] - mn_a);
+            sc[j][1] = exp2f(sc[j][1] - mn_a);
+            sc[j][2] = exp2f(sc[j][2] - mn_b);
+            sc[j][3] = exp2f(sc[j][3] - mn_b);
+            sum_a += sc[j][0] + sc[j][1];
+            sum_b += sc[j][2] + sc[j][3];
+          }
+          l_a = l_a * al_a + sum_a;
+          l_b = l_b * al_b + sum_b;
+          uint32_t pf[4];
+          pf[0] = pack_bf16(sc[0][0], sc[0][1]);
+          pf[1] = pack_bf16(sc[0][2], sc[0][3]);
+          pf[2] = pack_bf16(sc[1][0], sc[1][1]);
+          pf[3] = pack_bf16(sc[1][2], sc[1][3]);
+#pragma unroll
+          for (int dp = 0; dp < DH / 16; ++dp) {
+            uint32_t vf[4];
+            const int kk = (lane & 7) + ((lane >> 3) & 1) * 8, cc = 2 * dp + (lane >> 4);
+            ldmatrix_x4_trans(vf, v_base + kv_off(kk, cc));
+            if (n_valid < 16) {
+              const int k = 2 * (lane & 3);
+              vf[0] = mask_v(vf[0], k, n_valid);
+              vf[1] = mask_v(vf[1], k + 8, n_valid);
+              vf[2] = mask_v(vf[2], k, n_valid);
+              vf[3] = mask_v(vf[3], k + 8, n_valid);
+            }
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+              float* oc = o_acc[2 * dp + t];
+              oc[0] *= al_a; oc[1] *= al_a; oc[2] *= al_b; oc[3] *= al_b;
+            }
+            mma_bf16_16816(o_acc[2 * dp], pf, vf[0], vf[1]);
+            mma_bf16_16816(o_acc[2 * dp + 1], pf, vf[2], vf[3]);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[s]);
+        if (++s == DC_STAGES) { s = 0; ph ^= 1; }
+      }
+      // merge the four warps' partials in warp order
+      l_a = quad_sum(l_a);
+      l_b = quad_sum(l_b);
+      float* my_o = sm_o + warp * 16 * DH;
+#pragma unroll
+      for (int j = 0; j < DH / 8; ++j) {
+        const int col = 8 * j + 2 * (lane & 3);
+        *reinterpret_cast<float2*>(my_o + ra * DH + col) = make_float2(o_acc[j][0], o_acc[j][1]);
+        *reinterpret_cast<float2*>(my_o + rb * DH + col) = make_float2(o_acc[j][2], o_acc[j][3]);
+      }
+      if ((lane & 3) == 0) {
+        sm_ml[(warp * 16 + ra) * 2] = m_a;
+        sm_ml[(warp * 16 + ra) * 2 + 1] = l_a;
+        sm_ml[(warp * 16 + rb) * 2] = m_b;
+        sm_ml[(warp * 16 + rb) * 2 + 1] = l_b;
+      }
+      named_barrier_sync(1, DC_WARPS * 32);
+      if (alive) {
+        float* po = p.part_o + size_t(item) * 16 * DH;
+        float* pml = p.part_ml + size_t(item) * 16 * 2;
+        for (int idx = threadIdx.x; idx < G * DH; idx += DC_WARPS * 32) {
+          const int r = idx / DH, e = idx % DH;
+          float mm = -INFINITY;
+#pragma unroll
+          for (int w = 0; w < DC_WARPS; ++w) mm = fmaxf(mm, sm_ml[(w * 16 + r) * 2]);
+          float acc = 0.f, ll = 0.f;
+#pragma unroll
+          for (int w = 0; w < DC_WARPS; ++w) {
+            const float f = exp2f(sm_ml[(w * 16 + r) * 2] - mm);
+            acc += f * sm_o[(w * 16 + r) * DH + e];
+            ll += f * sm_ml[(w * 16 + r) * 2 + 1];
+          }
+          po[r * DH + e] = acc;
+          if (e == 0) {
+            pml[r * 2] = mm;
+            pml[r * 2 + 1] = ll;
+          }
+        }
+      }
+    }
+  }
+  __syncwarp();
+  if (*abort_flag) drain_after_abort();
+}
+
+// =================================================================== combine ==
+constexpr int CB_THREADS = 256;
+
+template <int DH>
+__global__ void __launch_bounds__(CB_THREADS, 1) attn_combine_kernel(const AttnParams p) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = p.n_q_heads / p.n_kv_heads;
+  const int q_dim = p.n_q_heads * DH;
+  constexpr int PER = DH / 32;
+  const int total = p.n_decode_rows * p.n_q_heads;
+  for (int w = blockIdx.x * (CB_THREADS / 32) + warp; w < total; w += gridDim.x * (CB_THREADS / 32)) {
+    const int4 row = reinterpret_cast<const int4*>(p.decode_rows)[w / p.n_q_heads];
+    const int hq = w % p.n_q_heads, hk = hq / G, g = hq % G;
+    const int tok = row.y, first = row.z + hk * row.w, splits = row.w;
+    float mm = -INFINITY;
+    for (int j = 0; j < splits; ++j) mm = fmaxf(mm, p.part_ml[(size_t(first + j) * 16 + g) * 2]);
+    float acc[PER];
+#pragma unroll
+    for (int i = 0; i < PER; ++i) acc[i] = 0.f;
+    float ll = 0.f;
+    for (int j = 0; j < splits; ++j) {
+      const float* ml = p.part_ml + (size_t(first + j) * 16 + g) * 2;
+      const float f = exp2f(ml[0] - mm);
+      ll += f * ml[1];
+      const float* po = p.part_o + (size_t(first + j) * 16 + g) * DH + lane * PER;
+#pragma unroll
+      for (int i = 0; i < PER; ++i) acc[i] += f * po[i];
+    }
+    const float inv = 1.f / ll;
+    __nv_bfloat16* dst = p.o + size_t(tok) * q_dim + hq * DH + lane * PER;
+#pragma unroll
+    for (int i = 0; i < PER; i += 2) *reinterpret_cast<uint32_t*>(dst + i) = pack_bf16(acc[i] * inv, acc[i + 1] * inv);
+  }
+}
+
+template <typename K>
+cudaError_t set_smem(K kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
+
+}  // namespace
+
+cudaError_t attention_set_attributes() {
+  cudaError_t e;
+  if ((e = set_smem(attn_prefill_kernel<64>, pf_smem_bytes<64>())) != cudaSuccess) return e;
+  if ((e = set_smem(attn_prefill_kernel<128>, pf_smem_bytes<128>())) != cudaSuccess) return e;
+  if ((e = set_smem(attn_decode_kernel<64>, dc_smem_bytes<64>())) != cudaSuccess) return e;
+  if ((e = set_smem(attn_decode_kernel<128>, dc_smem_bytes<128>())) != cudaSuccess) return e;
+  if ((e = set_smem(attn_combine_kernel<64>, kMinSmemBytes)) != cudaSuccess) return e;
+  return set_smem(attn_combine_kernel<128>, kMinSmemBytes);
+}
+
+cudaError_t launch_attention_prefill(const AttnParams& p, int sm_budget, cudaStream_t stream) {
+  if (p.n_prefill_items <= 0) return cudaSuccess;
+  const int grid = p.n_prefill_items < sm_budget ? p.n_prefill_items : sm_budget;
+  if (p.head_dim == 128)
+    attn_prefill_kernel<128><<<grid, PF_THREADS, pf_smem_bytes<128>(), stream>>>(p);
+  else
+    attn_prefill_kernel<64><<<grid, PF_THREADS, pf_smem_bytes<64>(), stream>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attention_decode(const AttnParams& p, int sm_budget, cudaStream_t stream) {
+  if (p.n_decode_items <= 0) return cudaSuccess;
+  const int grid = p.n_decode_items < sm_budget ? p.n_decode_items : sm_budget;
+  if (p.head_dim == 128)
+    attn_decode_kernel<128><<<grid, DC_THREADS, dc_smem_bytes<128>(), stream>>>(p);
+  else
+    attn_decode_kernel<64><<<grid, DC_THREADS, dc_smem_bytes<64>(), stream>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_attention_combine(const AttnParams& p, int sm_budget, cudaStream_t stream) {
+  if (p.n_decode_rows <= 0) return cudaSuccess;
+  const int total = p.n_decode_rows * p.n_q_heads;
+  const int blocks = (total + CB_THREADS / 32 - 1) / (CB_THREADS / 32);
+  const int grid = blocks < sm_budget ? blocks : sm_budget;
+  if (p.head_dim == 128)
+    attn_combine_kernel<128><<<grid, CB_THREADS, kMinSmemBytes, stream>>>(p);
+  else
+    attn_combine_kernel<64><<<grid, CB_THREADS, kMinSmemBytes, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace hs

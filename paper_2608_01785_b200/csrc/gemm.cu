@@ -1,0 +1,294 @@
+// Persistent, SM-budgeted bf16 GEMM on the 5th-generation tensor cores (tcgen05) with the step's
+// element-wise work fused into its epilogues.
+//
+//   tile        128 (tokens) x 256 (output columns), K consumed in blocks of 64
+//   operands    TMA (128-byte swizzle) -> 4-stage shared-memory ring -> tcgen05.mma, fp32 accumulators
+//               in tensor memory, two accumulator buffers so the epilogue of tile i overlaps the main
+//               loop of tile i+1
+//   roles       warp 0: TMA producer, warp 1: MMA issuer (one thread), warps 2..5: epilogue
+//   schedule    tile = blockIdx.x + i * gridDim.x, gridDim.x <= sm_budget, one block per SM.  Each output
+//               tile is produced by exactly one block with a fixed K order, so results do not depend on
+//               the budget.
+//
+// Epilogues: residual add (fp32 in / out), QKV (rotate-half RoPE + bf16 q + scatter of k, v into the
+// paged cache), gate/up (silu(gate) * up -> bf16).
+#include "kernels.h"
+#include "ptx.cuh"
+
+namespace hs {
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int A_BYTES = BM * BK * 2;            // 16 KB
+constexpr int BH_BYTES = 128 * BK * 2;          // one 128-row half of the B tile, 16 KB
+constexpr int STAGE_BYTES = A_BYTES + 2 * BH_BYTES;
+constexpr int GEMM_THREADS = 192;
+constexpr int TMEM_COLS = 512;                  // two 128 x 256 fp32 accumulators
+constexpr int GEMM_SMEM = 1024 + STAGES * STAGE_BYTES + 256;
+static_assert(GEMM_SMEM >= kMinSmemBytes, "one block per SM");
+
+struct BSource { int map, row; };
+__device__ __forceinline__ BSource b_source(const GemmParams& p, int n_tile, int half) {
+  if (p.mode == kGemmResid) return {0, n_tile * BN + half * 128};
+  if (p.mode == kGemmGateUp) return {half, n_tile * 128};
+  int v = n_tile * BN + half * 128;
+  if (v < p.q_dim) return {0, v};
+  v -= p.q_dim;
+  if (v < p.kv_dim) return {1, v};
+  return {2, v - p.kv_dim};
+}
+
+__device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+
+__device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float (&v)[32], int n_valid) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    if (i * 8 < n_valid) {
+      uint4 w;
+      w.x = pack_bf16(v[i * 8 + 0], v[i * 8 + 1]);
+      w.y = pack_bf16(v[i * 8 + 2], v[i * 8 + 3]);
+      w.z = pack_bf16(v[i * 8 + 4], v[i * 8 + 5]);
+      w.w = pack_bf16(v[i * 8 + 6], v[i * 8 + 7]);
+      *reinterpret_cast<uint4*>(dst + i * 8) = w;
+    }
+  }
+}
+
+// Address of element e of (slot, kv head) in one layer's K or V pages.
+__device__ __forceinline__ __nv_bfloat16* cache_ptr(__nv_bfloat16* base, int slot, int hk, int n_kv_heads, int Dh,
+                                                    int e) {
+  const size_t row = (size_t(slot >> 4) * n_kv_heads + hk) * 16 + (slot & 15);
+  return base + row * Dh + e;
+}
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  uint64_t* empty = full + STAGES;
+  uint64_t* tfull = empty + STAGES;
+  uint64_t* tempty = tfull + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_m_tiles = (p.M + BM - 1) / BM;
+  const int n_n_tiles = p.mode == kGemmGateUp ? (p.N + 127) / 128 : (p.N + BN - 1) / BN;
+  const int n_tiles = n_m_tiles * n_n_tiles;
+  const int k_blocks = (p.K + BK - 1) / BK;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; ++i) {
+      mbar_init(&full[i], 1);
+      mbar_init(&empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&tfull[i], 1);
+      mbar_init(&tempty[i], 128);
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+    tma_prefetch_desc(&p.tm_a);
+    tma_prefetch_desc(&p.tm_b[0]);
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------- TMA producer --
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int m = tile % n_m_tiles, n = tile / n_m_tiles;
+        const BSource b0 = b_source(p, n, 0), b1 = b_source(p, n, 1);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+          uint8_t* st = smem + s * STAGE_BYTES;
+          mbar_expect_tx(&full[s], STAGE_BYTES);
+          tma_load_2d(st, &p.tm_a, &full[s], kb * BK, m * BM);
+          tma_load_2d(st + A_BYTES, &p.tm_b[b0.map], &full[s], kb * BK, b0.row);
+          tma_load_2d(st + A_BYTES + BH_BYTES, &p.tm_b[b1.map], &full[s], kb * BK, b1.row);
+          if (++s == STAGES) { s = 0; ph ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // --------------------------------------------------------- MMA issuer --
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_bf16_f32(BM, BN);
+      int s = 0, acc = 0;
+      uint32_t ph = 0, acc_ph = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        if (!mbar_wait(&tempty[acc], acc_ph ^ 1, abort_flag, p.status)) break;
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!mbar_wait(&full[s], ph, abort_flag, p.status)) { ok = false; break; }
+          tc_fence_after_sync();
+          const uint32_t a_addr = smem_u32(smem + s * STAGE_BYTES);
+          const uint64_t a_desc = umma_desc_kmajor_sw128(a_addr);
+          const uint64_t b_desc = umma_desc_kmajor_sw128(a_addr + A_BYTES);
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)   // 16 bf16 = 32 B along K: +2 in the (address / 16) field
+            umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+          umma_commit(&empty[s]);             // frees the stage once these MMAs have read it
+          if (++s == STAGES) { s = 0; ph ^= 1; }
+        }
+        if (ok) umma_commit(&tfull[acc]);
+        acc ^= 1;
+        if (acc == 0) acc_ph ^= 1;
+      }
+    }
+  } else {
+    // ----------------------------------------------------------- epilogue --
+    const int quarter = warp & 3;             // the TMEM lane quarter this warp may read
+    int acc = 0;
+    uint32_t acc_ph = 0;
+    const int Dh = p.head_dim;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+      const int m = tile % n_m_tiles, n = tile / n_m_tiles;
+      const bool ok = mbar_wait(&tfull[acc], acc_ph, abort_flag, p.status);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      tc_fence_after_sync();
+      const uint32_t taddr = tmem_base + acc * BN + (uint32_t(quarter * 32) << 16);
+      const int row = m * BM + quarter * 32 + lane;
+      const bool row_ok = row < p.M;
+      uint32_t r0[32], r1[32];
+      float v0[32], v1[32];
+
+      if (p.mode == kGemmResid) {
+        for (int c = 0; c < BN / 32; ++c) {
+          const int col0 = n * BN + c * 32;
+          if (col0 >= p.N) break;
+          tmem_ld32(taddr + c * 32, r0);
+          tmem_ld_wait();
+          if (row_ok) {
+            float* o = p.out + size_t(row) * p.N + col0;
+            const float* rs = p.resid ? p.resid + size_t(row) * p.N + col0 : nullptr;
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+              if (col0 + v * 4 < p.N) {
+                float4 a = make_float4(__uint_as_float(r0[4 * v]), __uint_as_float(r0[4 * v + 1]),
+                                       __uint_as_float(r0[4 * v + 2]), __uint_as_float(r0[4 * v + 3]));
+                if (rs) {
+                  const float4 b = ld4(rs + 4 * v);
+                  a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+                }
+                *reinterpret_cast<float4*>(o + 4 * v) = a;
+              }
+            }
+          }
+        }
+      } else if (p.mode == kGemmGateUp) {
+        for (int c = 0; c < 4; ++c) {
+          const int col0 = n * 128 + c * 32;
+          if (col0 >= p.N) break;
+          tmem_ld32(taddr + c * 32, r0);          // gate
+          tmem_ld32(taddr + 128 + c * 32, r1);    // up
+          tmem_ld_wait();
+          if (row_ok) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              const float g = __uint_as_float(r0[e]), u = __uint_as_float(r1[e]);
+              v0[e] = g / (1.f + __expf(-g)) * u;
+            }
+            store_bf16x32(p.act + size_t(row) * p.N + col0, v0, p.N - col0);
+          }
+        }
+      } else {
+        const int pos = row_ok ? p.tok_pos[row] : 0;
+        const int slot = row_ok ? p.tok_slot[row] : 0;
+        const int half_dh = Dh >> 1;
+        for (int half = 0; half < 2; ++half) {
+          int vcol = n * BN + half * 128;         // virtual column of this half in [q | k | v]
+          if (vcol >= p.N) break;
+          int region = 0;
+          if (vcol >= p.q_dim) { region = 1; vcol -= p.q_dim; }
+          if (region == 1 && vcol >= p.kv_dim) { region = 2; vcol -= p.kv_dim; }
+          if (region == 2) {
+            for (int c = 0; c < 4; ++c) {
+              tmem_ld32(taddr + half * 128 + c * 32, r0);
+              tmem_ld_wait();
+              if (row_ok) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) v0[e] = __uint_as_float(r0[e]);
+                const int col = vcol + c * 32;
+                store_bf16x32(cache_ptr(p.v_cache, slot, col / Dh, p.n_kv_heads, Dh, col % Dh), v0, 32);
+              }
+            }
+          } else {
+            for (int j = 0; j < 2; ++j) {
+              const int lo = Dh == 128 ? j : 2 * j, hi = lo + (Dh == 128 ? 2 : 1);
+              const int i0 = Dh == 128 ? 32 * j : 0;       // index of the first rotation pair
+              tmem_ld32(taddr + half * 128 + lo * 32, r0);
+              tmem_ld32(taddr + half * 128 + hi * 32, r1);
+              tmem_ld_wait();
+              if (row_ok) {
+                const float2* cs = p.rope + size_t(pos) * half_dh + i0;
+#pragma unroll
+                for (int e = 0; e < 32; e += 2) {
+                  const float4 t = *reinterpret_cast<const float4*>(cs + e);   // cos,sin of pairs e, e+1
+                  const float a0 = __uint_as_float(r0[e]), b0 = __uint_as_float(r1[e]);
+                  const float a1 = __uint_as_float(r0[e + 1]), b1 = __uint_as_float(r1[e + 1]);
+                  v0[e] = a0 * t.x - b0 * t.y;
+                  v1[e] = b0 * t.x + a0 * t.y;
+                  v0[e + 1] = a1 * t.z - b1 * t.w;
+                  v1[e + 1] = b1 * t.z + a1 * t.w;
+                }
+                const int col_lo = vcol + lo * 32, col_hi = vcol + hi * 32;
+                if (region == 0) {
+                  store_bf16x32(p.q_out + size_t(row) * p.q_dim + col_lo, v0, 32);
+                  store_bf16x32(p.q_out + size_t(row) * p.q_dim + col_hi, v1, 32);
+                } else {
+                  store_bf16x32(cache_ptr(p.k_cache, slot, col_lo / Dh, p.n_kv_heads, Dh, col_lo % Dh), v0, 32);
+                  store_bf16x32(cache_ptr(p.k_cache, slot, col_hi / Dh, p.n_kv_heads, Dh, col_hi % Dh), v1, 32);
+                }
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before_sync();
+      mbar_arrive(&tempty[acc]);
+      acc ^= 1;
+      if (acc == 0) acc_ph ^= 1;
+    }
+  }
+
+  // ------------------------------------------------------------- teardown --
+  __syncwarp();
+  if (*abort_flag) drain_after_abort();
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+}  // namespace
+
+cudaError_t gemm_set_attributes() {
+  return cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
+}
+
+cudaError_t launch_gemm(const GemmParams& p, int sm_budget, cudaStream_t stream) {
+  const int n_m_tiles = (p.M + BM - 1) / BM;
+  const int n_n_tiles = p.mode == kGemmGateUp ? (p.N + 127) / 128 : (p.N + BN - 1) / BN;
+  const int n_tiles = n_m_tiles * n_n_tiles;
+  if (n_tiles <= 0) return cudaSuccess;
+  const int grid = n_tiles < sm_budget ? n_tiles : sm_budget;
+  gemm_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace hs

@@ -1,0 +1,69 @@
+// Internal declarations shared by the host side (allocator, planner, C ABI) and the kernel launchers.
+#pragma once
+#include <stdint.h>
+
+#include <unordered_map>
+#include <vector>
+
+#include "../../include/horizonserve.h"
+
+namespace hs {
+
+constexpr int kPage = HS_PAGE_SIZE;      // tokens per KV page
+constexpr int kDecodeSplit = 512;        // keys per decode split-KV work item (budget independent)
+constexpr int kPrefillRows = 128;        // (token, query head of one KV head) rows per prefill work item
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Tokens per prefill work item: the G query heads of one KV head are stacked as rows of the tile.
+inline int prefill_tokens_per_item(int G) { return kPrefillRows / G; }
+
+// ------------------------------------------------------------------ pages --
+// LIFO page allocator: pops on a fresh pool give 0, 1, 2, ...; a freed sequence returns its pages in
+// reverse order of acquisition.
+class PageAllocator {
+ public:
+  explicit PageAllocator(int num_pages);
+  // Grows seq to ceil(total_tokens / kPage) pages.  Returns HS_OK or HS_ERR_OUT_OF_PAGES (unchanged).
+  hs_status_t grow(int64_t seq, int total_tokens, const std::vector<int32_t>** table);
+  hs_status_t release(int64_t seq);
+  int free_pages() const { return static_cast<int>(free_.size()); }
+
+ private:
+  std::vector<int32_t> free_;   // stack; back() is popped next
+  std::unordered_map<int64_t, std::vector<int32_t>> owned_;
+};
+
+// --------------------------------------------------------- step metadata --
+// Offsets (in int32 units) of the arrays inside the per-step metadata block that is copied to the
+// device once per step.  Fixed at stage creation from the configuration's maxima.
+struct MetaLayout {
+  int tok_pos, tok_slot;             // [max_tokens]      absolute position / cache slot of each new token
+  int seq_tok0, seq_ctx, seq_qlen;   // [max_seqs]        first token row, cached tokens, new tokens
+  int block_tables;                  // [max_seqs * max_pages_per_seq]
+  int prefill_items;                 // [max_prefill_items * 4]  {seq, kv_head, first token of the tile, tokens}
+  int decode_items;                  // [max_decode_items * 4]   {seq, kv_head, first key, end key}
+  int decode_rows;                   // [max_seqs * 4]           {seq, token row, first item, splits}
+  int counters;                      // [n_layers * 2]           work-queue heads, zero at step start
+  int total;                         // int32 words in the block
+  int max_prefill_items, max_decode_items;
+};
+MetaLayout make_meta_layout(const hs_stage_config_t& c);
+
+struct StepPlan {
+  int n_tokens = 0, n_seqs = 0;
+  int n_prefill_items = 0, n_decode_items = 0, n_decode_rows = 0;
+};
+
+// Validates `b` against `c` and, when `meta` is non-NULL, fills the metadata block (layout `ml`).
+// `page_stamp` is scratch of num_pages entries used to detect a page named by two sequences; `stamp`
+// must be a value not used by an earlier call.  tok_seq (nullable) receives the owning sequence of each
+// token.  Returns HS_OK, HS_ERR_INVALID_ARG or HS_ERR_BAD_BLOCK_TABLE.
+hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs_batch_t& b,
+                      std::vector<int32_t>& page_stamp, int32_t stamp, int32_t* meta, int32_t* tok_seq,
+                      StepPlan* plan);
+
+hs_status_t validate_config(const hs_stage_config_t& c);
+
+}  // namespace hs

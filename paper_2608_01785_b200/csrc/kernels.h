@@ -1,0 +1,88 @@
+// Launcher interfaces of the step's kernels.  Every launcher enqueues one persistent kernel of at most
+// `sm_budget` thread blocks (one per SM: each block asks for more than half of an SM's shared memory)
+// on `stream` and returns the launch status.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace hs {
+
+// Dynamic shared memory every kernel requests at least, so that two blocks (of this or of a co-running
+// stage's kernel) never share an SM: more than half of the 227 KB an SM offers.
+constexpr int kMinSmemBytes = 117 * 1024;
+
+// ------------------------------------------------------------------ GEMM --
+// out = A[M,K] * W^T with W given as up to three row blocks [rows, K] (bf16, K contiguous).  The output
+// tile is 128 x 256 "virtual" columns; each 128-column half of a tile is fetched from one weight matrix.
+enum GemmMode : int {
+  kGemmResid = 0,   // out[M,N] fp32 = (resid ? resid : 0) + A W^T                     (out-proj, down)
+  kGemmQkv = 1,     // virtual columns [q | k | v]; RoPE on q,k; q -> bf16 buffer, k,v -> paged cache
+  kGemmGateUp = 2   // tile = 128 gate columns + the same 128 up columns; act = silu(gate) * up -> bf16
+};
+
+struct GemmParams {
+  CUtensorMap tm_a;          // activations [rows >= M, K], box 64 x 128
+  CUtensorMap tm_b[3];       // weights, box 64 x 128: Resid {W}, Qkv {Wq, Wk, Wv}, GateUp {Wgate, Wup}
+  int M, N, K;               // N: Resid output width; Qkv (Hq + 2 Hkv) * Dh; GateUp F (activation width)
+  int mode;
+  // Resid
+  const float* resid;        // nullable; may alias out
+  float* out;                // [M, N]
+  // Qkv
+  int q_dim, kv_dim, head_dim, n_kv_heads;
+  __nv_bfloat16* q_out;      // [M, q_dim]
+  __nv_bfloat16* k_cache;    // this layer's K pages: [page][kv_head][16][Dh]
+  __nv_bfloat16* v_cache;
+  const int32_t* tok_pos;    // [M]
+  const int32_t* tok_slot;   // [M]
+  const float2* rope;        // [max_position][Dh/2] (cos, sin)
+  // GateUp
+  __nv_bfloat16* act;        // [M, N]
+  int* status;               // device status word
+};
+cudaError_t launch_gemm(const GemmParams& p, int sm_budget, cudaStream_t stream);
+cudaError_t gemm_set_attributes();
+
+// ---------------------------------------------------------------- RMSNorm --
+// h[t,:] = bf16(x[t,:] * rsqrt(mean(x[t,:]^2) + eps) * g).  x comes either as bf16 (x_bf16, first layer;
+// x_f32_out then receives the widened copy that starts the fp32 residual stream) or as fp32 (x_f32).
+struct NormParams {
+  const __nv_bfloat16* x_bf16;
+  const float* x_f32;
+  float* x_f32_out;
+  const __nv_bfloat16* gain;
+  __nv_bfloat16* h;
+  int T, d;
+  float eps;
+};
+cudaError_t launch_rmsnorm(const NormParams& p, int sm_budget, cudaStream_t stream);
+cudaError_t norm_set_attributes();
+
+// -------------------------------------------------------------- attention --
+struct AttnParams {
+  CUtensorMap tm_kv;               // whole pool as rows of Dh bf16: box 64 x 16, 128-byte swizzle
+  const __nv_bfloat16* q;          // [T, q_dim] (after RoPE)
+  __nv_bfloat16* o;                // [T, q_dim]
+  int n_q_heads, n_kv_heads, head_dim, num_pages, max_pages_per_seq, layer;
+  const int32_t* seq_tok0;
+  const int32_t* seq_ctx;
+  const int32_t* block_tables;
+  const int32_t* prefill_items;    // int4 per item
+  int n_prefill_items;
+  const int32_t* decode_items;     // int4 per item
+  int n_decode_items;
+  const int32_t* decode_rows;      // int4 per decode sequence
+  int n_decode_rows;
+  float* part_o;                   // [max_decode_items][16][Dh] unnormalised partial outputs
+  float* part_ml;                  // [max_decode_items][16][2]  running max (log2 domain) and sum
+  int* counters;                   // two work-queue heads of this layer (prefill, decode), zero at entry
+  int* status;
+};
+cudaError_t launch_attention_prefill(const AttnParams& p, int sm_budget, cudaStream_t stream);
+cudaError_t launch_attention_decode(const AttnParams& p, int sm_budget, cudaStream_t stream);
+cudaError_t launch_attention_combine(const AttnParams& p, int sm_budget, cudaStream_t stream);
+cudaError_t attention_set_attributes();
+
+}  // namespace hs

@@ -1,0 +1,177 @@
+// Host-only logic of the stage: configuration checks, the page allocator, and the per-step planner
+// that turns a batch descriptor into the integer metadata the kernels consume.  Nothing here depends
+// on the SM budget, which is what keeps results identical across budgets.
+#include <algorithm>
+#include <numeric>
+
+#include "hs_internal.h"
+
+namespace hs {
+
+hs_status_t validate_config(const hs_stage_config_t& c) {
+  if (c.abi_version != HS_ABI_VERSION || c.flags != 0) return HS_ERR_INVALID_ARG;
+  if (c.n_layers < 1 || c.d_model < 64 || c.n_q_heads < 1 || c.n_kv_heads < 1 || c.d_ffn < 64) return HS_ERR_INVALID_ARG;
+  if (c.num_pages < 1 || c.max_tokens < 1 || c.max_seqs < 1 || c.max_pages_per_seq < 1 || c.max_position < 1)
+    return HS_ERR_INVALID_ARG;
+  if (c.max_seqs > c.max_tokens) return HS_ERR_INVALID_ARG;
+  if (!(c.rms_eps >= 0.f) || !(c.rope_base > 1.f)) return HS_ERR_INVALID_ARG;
+  if (c.page_size != kPage) return HS_ERR_UNSUPPORTED_SHAPE;
+  if (c.head_dim != 64 && c.head_dim != 128) return HS_ERR_UNSUPPORTED_SHAPE;
+  if (c.n_q_heads % c.n_kv_heads != 0 || c.n_q_heads / c.n_kv_heads > 16) return HS_ERR_UNSUPPORTED_SHAPE;
+  // A 128-wide half of a GEMM tile must lie inside one of q / k / v
+  if ((c.n_q_heads * c.head_dim) % 128 != 0 || (c.n_kv_heads * c.head_dim) % 128 != 0) return HS_ERR_UNSUPPORTED_SHAPE;
+  // 16-byte rows for tiled copies and vector stores
+  if (c.d_model % 8 != 0 || c.d_ffn % 8 != 0) return HS_ERR_UNSUPPORTED_SHAPE;
+  // total rows of the pool as seen by a tiled copy must fit a 32-bit coordinate
+  const int64_t rows = int64_t(c.n_layers) * 2 * c.num_pages * c.n_kv_heads * kPage;
+  if (rows >= (int64_t(1) << 31)) return HS_ERR_UNSUPPORTED_SHAPE;
+  return HS_OK;
+}
+
+// ------------------------------------------------------------------ pages --
+PageAllocator::PageAllocator(int num_pages) {
+  free_.resize(num_pages);
+  for (int i = 0; i < num_pages; ++i) free_[i] = num_pages - 1 - i;
+}
+
+hs_status_t PageAllocator::grow(int64_t seq, int total_tokens, const std::vector<int32_t>** table) {
+  auto it = owned_.find(seq);
+  const int have = it == owned_.end() ? 0 : static_cast<int>(it->second.size());
+  const int need = ceil_div(total_tokens, kPage) - have;
+  if (need > static_cast<int>(free_.size())) return HS_ERR_OUT_OF_PAGES;
+  std::vector<int32_t>& pages = owned_[seq];
+  for (int i = 0; i < need; ++i) {
+    pages.push_back(free_.back());
+    free_.pop_back();
+  }
+  *table = &pages;
+  return HS_OK;
+}
+
+hs_status_t PageAllocator::release(int64_t seq) {
+  auto it = owned_.find(seq);
+  if (it == owned_.end()) return HS_ERR_UNKNOWN_SEQ;
+  for (auto p = it->second.rbegin(); p != it->second.rend(); ++p) free_.push_back(*p);
+  owned_.erase(it);
+  return HS_OK;
+}
+
+// --------------------------------------------------------- step metadata --
+MetaLayout make_meta_layout(const hs_stage_config_t& c) {
+  MetaLayout m{};
+  const int G = c.n_q_heads / c.n_kv_heads;
+  m.max_prefill_items = c.n_kv_heads * (c.max_tokens / prefill_tokens_per_item(G) + c.max_seqs);
+  // every decode sequence has one ragged split plus one per kDecodeSplit cached keys; cached keys are
+  // bounded by the pool
+  m.max_decode_items = c.n_kv_heads * (c.max_seqs + int((int64_t(c.num_pages) * kPage) / kDecodeSplit) + 1);
+  int off = 0;
+  auto take = [&](int n) {
+    int o = off;
+    off += (n + 3) & ~3;   // keep every array 16-byte aligned
+    return o;
+  };
+  m.tok_pos = take(c.max_tokens);
+  m.tok_slot = take(c.max_tokens);
+  m.seq_tok0 = take(c.max_seqs);
+  m.seq_ctx = take(c.max_seqs);
+  m.seq_qlen = take(c.max_seqs);
+  m.block_tables = take(c.max_seqs * c.max_pages_per_seq);
+  m.prefill_items = take(m.max_prefill_items * 4);
+  m.decode_items = take(m.max_decode_items * 4);
+  m.decode_rows = take(c.max_seqs * 4);
+  m.counters = take(c.n_layers * 2);
+  m.total = off;
+  return m;
+}
+
+hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs_batch_t& b,
+                      std::vector<int32_t>& page_stamp, int32_t stamp, int32_t* meta, int32_t* tok_seq,
+                      StepPlan* plan) {
+  if (!b.q_len || !b.ctx_len || !b.block_tables) return HS_ERR_INVALID_ARG;
+  if (b.n_seqs < 1 || b.n_seqs > c.max_seqs || b.n_tokens < 1 || b.n_tokens > c.max_tokens) return HS_ERR_INVALID_ARG;
+  const int mpps = c.max_pages_per_seq;
+  int64_t total = 0;
+  for (int s = 0; s < b.n_seqs; ++s) {
+    if (b.q_len[s] < 1 || b.ctx_len[s] < 0) return HS_ERR_INVALID_ARG;
+    if (int64_t(b.ctx_len[s]) + b.q_len[s] > c.max_position) return HS_ERR_INVALID_ARG;
+    total += b.q_len[s];
+  }
+  if (total != b.n_tokens) return HS_ERR_INVALID_ARG;
+  // block tables: enough pages, ids in range, no page named twice in this step
+  for (int s = 0; s < b.n_seqs; ++s) {
+    const int need = ceil_div(b.ctx_len[s] + b.q_len[s], kPage);
+    if (need > mpps) return HS_ERR_BAD_BLOCK_TABLE;
+    for (int i = 0; i < need; ++i) {
+      const int32_t pg = b.block_tables[size_t(s) * mpps + i];
+      if (pg < 0 || pg >= c.num_pages) return HS_ERR_BAD_BLOCK_TABLE;
+      if (page_stamp[pg] == stamp) return HS_ERR_BAD_BLOCK_TABLE;
+      page_stamp[pg] = stamp;
+    }
+  }
+
+  const int G = c.n_q_heads / c.n_kv_heads;
+  const int Mt = prefill_tokens_per_item(G);
+  StepPlan p;
+  p.n_tokens = b.n_tokens;
+  p.n_seqs = b.n_seqs;
+
+  struct Item { int32_t v[4]; int32_t cost; };
+  std::vector<Item> pre;
+  int n_dec_items = 0, n_dec_rows = 0;
+  int t = 0;
+  for (int s = 0; s < b.n_seqs; ++s) {
+    const int n = b.q_len[s], ctx = b.ctx_len[s];
+    if (meta) {
+      meta[ml.seq_tok0 + s] = t;
+      meta[ml.seq_ctx + s] = ctx;
+      meta[ml.seq_qlen + s] = n;
+      for (int i = 0; i < mpps; ++i) meta[ml.block_tables + s * mpps + i] = b.block_tables[size_t(s) * mpps + i];
+    }
+    for (int j = 0; j < n; ++j) {
+      const int pos = ctx + j;
+      const int slot = b.block_tables[size_t(s) * mpps + pos / kPage] * kPage + pos % kPage;
+      if (meta) {
+        meta[ml.tok_pos + t + j] = pos;
+        meta[ml.tok_slot + t + j] = slot;
+      }
+      if (tok_seq) tok_seq[t + j] = s;
+    }
+    if (n == 1) {
+      // decode: keys 0..ctx split into fixed runs of kDecodeSplit
+      const int keys = ctx + 1, splits = ceil_div(keys, kDecodeSplit);
+      if (meta) {
+        int32_t* row = meta + ml.decode_rows + n_dec_rows * 4;
+        row[0] = s; row[1] = t; row[2] = n_dec_items; row[3] = splits;
+        for (int hk = 0; hk < c.n_kv_heads; ++hk)
+          for (int j = 0; j < splits; ++j) {
+            int32_t* it = meta + ml.decode_items + (n_dec_items + hk * splits + j) * 4;
+            it[0] = s; it[1] = hk; it[2] = j * kDecodeSplit; it[3] = std::min(keys, (j + 1) * kDecodeSplit);
+          }
+      }
+      n_dec_items += c.n_kv_heads * splits;
+      ++n_dec_rows;
+    } else {
+      for (int t0 = 0; t0 < n; t0 += Mt)
+        for (int hk = 0; hk < c.n_kv_heads; ++hk) {
+          const int nt = std::min(Mt, n - t0);
+          pre.push_back(Item{{s, hk, t0, nt}, ctx + t0 + nt});
+        }
+    }
+    t += n;
+  }
+  if (int(pre.size()) > ml.max_prefill_items || n_dec_items > ml.max_decode_items) return HS_ERR_INVALID_ARG;
+  // longest first, so that the dynamic queue finishes evenly; ties keep batch order
+  std::stable_sort(pre.begin(), pre.end(), [](const Item& a, const Item& b2) { return a.cost > b2.cost; });
+  if (meta) {
+    for (size_t i = 0; i < pre.size(); ++i)
+      for (int k = 0; k < 4; ++k) meta[ml.prefill_items + int(i) * 4 + k] = pre[i].v[k];
+    for (int i = 0; i < c.n_layers * 2; ++i) meta[ml.counters + i] = 0;
+  }
+  p.n_prefill_items = int(pre.size());
+  p.n_decode_items = n_dec_items;
+  p.n_decode_rows = n_dec_rows;
+  if (plan) *plan = p;
+  return HS_OK;
+}
+
+}  // namespace hs
