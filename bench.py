@@ -1,0 +1,328 @@
+#!/usr/bin/env python
+"""Benchmark of the shared-stage step: tokens/s and step latency under an SM budget, with the fraction of
+the tensor-core roofline reached by the dominant kernel and the CPU oracle timed beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload c2_shared|c3_7b|c4_talker|c1_tiny] [--sm-budget B]
+
+A "step" is one hs_stage_step over the whole batch (every layer: RMSNorm, QKV GEMM + RoPE + cache write,
+paged attention, out-proj, gate/up + SwiGLU, down).  Inputs are seeded and synthetic.  With N > 1 (one
+process per GPU under torch.distributed.run) every rank runs an independent replica of the same workload:
+the step has no exchange between GPUs, so the data path uses no collective; ranks meet only at the timing
+barriers.  `--impl reference` times the CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_01785_b200 import workloads as wl  # noqa: E402
+
+METRIC = "shared_stage_tokens_per_s"
+UNIT = "tokens/s"
+SEED = {"c1_tiny": 0, "c2_shared": 1, "c3_7b": 2, "c4_talker": 3}
+# DRAM bytes (read + write) of one gate/up GEMM launch, from the ncu capture summarised under profiles/
+# (None until a capture of this workload's launch exists).
+GATEUP_DRAM_TRAFFIC_BYTES = {"c2_shared": None}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_burst": p["bf16_tflops"], "bf16_sustained": p["bf16_tflops_sustained"],
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def build_stage(name: str, device: int):
+    """Weights, KV pool with random-filled context, block tables and input of the named workload."""
+    from paper_2608_01785_b200.stage import Stage
+    dims = wl.DIMS[name]
+    seed = SEED[name]
+    batch = wl.make_batch(name, seed)
+    dev = torch.device("cuda", device)
+    weights = wl.make_weights(dims, seed, dev)
+    num_pages = wl.pages_needed(batch) + 8
+    mpps = max(-(-t // 16) for t in batch.total_len())
+    stage = Stage(dims, weights, num_pages, batch.n_tokens, batch.n_seqs, mpps, max(batch.total_len()), device)
+    # context of the decode sequences: values do not change the timing; N(0,1) bf16 stands in for K/V
+    # written by earlier steps
+    g = torch.Generator(device=dev)
+    g.manual_seed(seed + 1000)
+    chunk = 1 << 24
+    flat = stage.kv_pool
+    for o in range(0, flat.numel(), chunk):
+        n = min(chunk, flat.numel() - o)
+        flat[o:o + n] = torch.randn(n, generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    tables = [stage.kv_alloc(s, t) for s, t in enumerate(batch.total_len())]
+    bt = stage.block_table_array(tables)
+    x = wl.make_x(batch.n_tokens, dims.d_model, seed, dev)
+    return stage, dims, batch, bt, x
+
+
+def flops_per_step(dims: wl.StageDims, batch: wl.BatchSpec):
+    T = batch.n_tokens
+    gemm = 2.0 * T * dims.params_per_layer() * dims.n_layers
+    attn = 0.0
+    for n, c in zip(batch.q_len, batch.ctx_len):
+        attn += 4.0 * dims.n_q_heads * dims.head_dim * (c * n + n * (n + 1) / 2.0)
+    return gemm, attn * dims.n_layers
+
+
+def cpu_oracle_sample(name: str, target_s: float):
+    """Times the oracle on a bounded sample: one layer of the workload's batch, K/V of every token plus
+    `rows` fully evaluated rows.  Returns (tokens/s extrapolated to the whole step, description, threads)."""
+    from oracle.oracle import Oracle, OracleConfig
+    from oracle.paging import PageAllocator, block_table_array
+    dims = wl.DIMS[name]
+    seed = SEED[name]
+    batch = wl.make_batch(name, seed)
+    one = wl.StageDims(1, dims.d_model, dims.n_q_heads, dims.n_kv_heads, dims.head_dim, dims.d_ffn)
+    num_pages = wl.pages_needed(batch) + 8
+    alloc = PageAllocator(num_pages, 16)
+    tables = [alloc.alloc(s, t) for s, t in enumerate(batch.total_len())]
+    bt = block_table_array(tables, max(len(t) for t in tables))
+    cfg = OracleConfig(1, dims.d_model, dims.n_q_heads, dims.n_kv_heads, dims.head_dim, dims.d_ffn, 16, num_pages,
+                       dims.rms_eps, dims.rope_base)
+    w = wl.weights_to_numpy([wl.make_layer_weights(one, seed, 0)])
+    pool = wl.bf16_bits_numpy(wl.make_kv_fill(one, num_pages, seed)).reshape(-1).copy()
+    x = wl.to_f32_numpy(wl.make_x(batch.n_tokens, dims.d_model, seed))
+    orc = Oracle("f32")
+    T = batch.n_tokens
+    # ~2 * params flops per fully evaluated row; the plain loops run at a few tens of GFLOP/s
+    rows = int(max(16, min(T, target_s * 40e9 / (2.0 * dims.params_per_layer()))))
+    mask = np.zeros(T, dtype=np.uint8)
+    mask[np.linspace(0, T - 1, rows).astype(np.int64)] = 1
+    rows = int(mask.sum())
+    t0 = time.perf_counter()
+    orc.step(cfg, w, pool, batch.q_len, batch.ctx_len, bt, x, mask)
+    dt = time.perf_counter() - t0
+    value = rows / (dt * dims.n_layers)
+    desc = (f"one layer of {dims.n_layers}, batch of {name}: K/V of all {T} tokens + {rows} evenly spaced rows "
+            f"evaluated in full, {dt:.2f} s; tokens/s = rows / (seconds x layers)")
+    threads = int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+    return value, desc, threads, dt
+
+
+def run_reference(args, rank: int):
+    if rank != 0:
+        return
+    name = args.workload
+    per_step = max(1.0, min(20.0, 150.0 / (args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        cpu_oracle_sample(name, per_step)
+    vals, times, desc, threads = [], [], "", 1
+    for _ in range(args.steps):
+        v, desc, threads, dt = cpu_oracle_sample(name, per_step)
+        vals.append(v); times.append(dt)
+    value = len(vals) / sum(1.0 / v for v in vals)          # harmonic mean = total tokens / total time
+    dims, batch = wl.DIMS[name], wl.make_batch(name, SEED[name])
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * batch.n_tokens / value,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": name, "n_tokens": batch.n_tokens, "n_seqs": batch.n_seqs,
+                       "n_layers": dims.n_layers},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c2_shared", choices=sorted(SEED))
+    ap.add_argument("--sm-budget", type=int, default=0, help="0 = all SMs")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only implementation of the step")
+
+    import torch.distributed as dist
+    from paper_2608_01785_b200 import binding as B
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    name = args.workload
+    stage, dims, batch, bt, x = build_stage(name, local_rank)
+    budget = args.sm_budget or stage.sm_count
+    T, d = batch.n_tokens, dims.d_model
+    dev = stage.device
+    y = torch.empty(T, d, dtype=torch.float32, device=dev)
+    b = stage.make_batch(batch.q_len, batch.ctx_len, bt, x, y)
+    stream = torch.cuda.Stream(device=dev)
+
+    def timed_steps(k: int, fn):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for _ in range(k):
+                fn()
+            e1.record(stream)
+        barrier()
+        ms = torch.tensor([e0.elapsed_time(e1)], device=dev)
+        if world > 1:
+            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+        return float(ms.item())
+
+    step_dev = lambda: stage.step(b, budget, stream)
+
+    # ---- device-resident throughput -------------------------------------
+    timed_steps(args.warmup, step_dev)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms_total = timed_steps(args.steps, step_dev)
+    clocks = sampler.stop() if rank == 0 else None
+    assert stage.status() == 0, "device status word is set"
+    ms_step = ms_total / args.steps
+    value = world * T / (ms_step * 1e-3)
+
+    # ---- per-kernel timing (same launches, events around each kernel) ----
+    B.hs_stage_profile_enable(stage.handle, True)
+    timed_steps(args.steps, step_dev)
+    prof = B.hs_stage_profile_read(stage.handle)
+    B.hs_stage_profile_enable(stage.handle, False)
+    launches_per_step = sum(n for _, n in prof.values()) // args.steps
+
+    # ---- end to end: host buffers in, host buffers out -------------------
+    x_host = x.cpu().pin_memory()
+    y_host = torch.empty(T, d, dtype=torch.float32).pin_memory()
+    x_dev2 = torch.empty_like(x)
+    b2 = stage.make_batch(batch.q_len, batch.ctx_len, bt, x_dev2, y)
+
+    def step_e2e():
+        x_dev2.copy_(x_host, non_blocking=True)
+        stage.step(b2, budget, stream)
+        y_host.copy_(y, non_blocking=True)
+
+    timed_steps(3, step_e2e)
+    ms_e2e = timed_steps(args.steps, step_e2e) / args.steps
+    e2e_value = world * T / (ms_e2e * 1e-3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (gate/up GEMM) -------------------
+    peaks = measured_peaks()
+    gu_ms, gu_n = prof["gemm_gateup"]
+    gu_flops = 2.0 * T * dims.d_model * 2 * dims.d_ffn
+    gu_avg_s = gu_ms * 1e-3 / max(gu_n, 1)
+    achieved = gu_flops / gu_avg_s / 1e12
+    peak = peaks["bf16_sustained"] * budget / stage.sm_count
+    gemm_flops, attn_flops = flops_per_step(dims, batch)
+    roofline = {"bound": "tensor", "kernel": "gemm_kernel (gate/up + SwiGLU epilogue)", "achieved": achieved,
+                "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                "peak_source": f"{peaks['source']} sustained bf16 x sm_budget/{stage.sm_count}",
+                "frac_of_burst_peak": achieved / (peaks["bf16_burst"] * budget / stage.sm_count),
+                "traffic": GATEUP_DRAM_TRAFFIC_BYTES.get(name),
+                "avg_launch_ms": gu_avg_s * 1e3, "launches": gu_n,
+                "step_tflops": (gemm_flops + attn_flops) / (ms_step * 1e-3) / 1e12}
+    kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps} for k, v in prof.items()}
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        v, desc, threads, _ = cpu_oracle_sample(name, 12.0)
+        cpu = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": name, "n_layers": dims.n_layers, "d_model": d, "n_tokens": T,
+                       "n_seqs": batch.n_seqs, "prefill_tokens": int(sum(q for q in batch.q_len if q > 1)),
+                       "decode_seqs": int(sum(1 for q in batch.q_len if q == 1)), "sm_budget": budget,
+                       "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
+                       "l2": "inputs larger than L2: weights + KV read per step exceed the 126 MB L2"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e, "h2d_bytes_per_step": T * d * 2,
+                    "d2h_bytes_per_step": T * d * 4},
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -40,6 +40,20 @@ hs_status_t hs_op_gemm_bf16(const void *a, const void *w, const float *resid, fl
  */
 hs_status_t hs_stage_debug_buffer(hs_stage_t *stage, const char *name, void **dev_ptr, size_t *bytes);
 
+/*
+ * Per-kernel timing of hs_stage_step (measurement support; the paper's analogue is its fixed-SM
+ * profiling sweep, Sec. 3.3).  While enabled, every kernel launch of a step is bracketed by CUDA
+ * events on the step's stream.  hs_stage_profile_read synchronises those events and adds, per
+ * kernel class, the elapsed milliseconds to ms[class] and the launch count to launches[class]
+ * (host arrays of HS_PROFILE_CLASSES entries, accumulated since the last read), then forgets them.
+ * Classes: 0 rmsnorm, 1 qkv gemm, 2 prefill attention, 3 decode attention, 4 decode combine,
+ * 5 out-proj gemm, 6 gate/up gemm, 7 down gemm.
+ * Errors: INVALID_ARG, NO_DEVICE, CUDA.
+ */
+#define HS_PROFILE_CLASSES 8
+hs_status_t hs_stage_profile_enable(hs_stage_t *stage, int32_t enable);
+hs_status_t hs_stage_profile_read(hs_stage_t *stage, float *ms, int32_t *launches);
+
 #if defined(__GNUC__)
 #pragma GCC visibility pop
 #endif

@@ -21,7 +21,10 @@ HS_OK, HS_ERR_INVALID_ARG, HS_ERR_INVALID_BUDGET, HS_ERR_UNSUPPORTED_SHAPE, HS_E
 
 EXPORTS = ("hs_status_str", "hs_kv_pool_bytes", "hs_workspace_bytes", "hs_stage_create", "hs_stage_destroy",
            "hs_kv_alloc", "hs_kv_free", "hs_kv_free_pages", "hs_stage_plan", "hs_stage_step", "hs_stage_status",
-           "hs_stage_sm_count", "hs_op_gemm_bf16", "hs_stage_debug_buffer")
+           "hs_stage_sm_count", "hs_op_gemm_bf16", "hs_stage_debug_buffer", "hs_stage_profile_enable",
+           "hs_stage_profile_read")
+PROFILE_CLASSES = ("rmsnorm", "gemm_qkv", "attn_prefill", "attn_decode", "attn_combine", "gemm_out", "gemm_gateup",
+                   "gemm_down")
 
 
 class hs_stage_config_t(C.Structure):
@@ -84,6 +87,8 @@ def lib() -> C.CDLL:
         l.hs_op_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                       C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         l.hs_stage_debug_buffer.argtypes = [C.c_void_p, C.c_char_p, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
+        l.hs_stage_profile_enable.argtypes = [C.c_void_p, C.c_int32]
+        l.hs_stage_profile_read.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = l
     return _lib
 
@@ -199,3 +204,19 @@ def hs_op_gemm_bf16(a_ptr: int, w_ptr: int, resid_ptr: int, out_ptr: int, M: int
                                M, N, K, sm_budget, C.c_void_p(status_ptr), C.c_void_p(cuda_stream))
     if st != HS_OK:
         raise HsError(st, "hs_op_gemm_bf16")
+
+
+def hs_stage_profile_enable(stage: int, enable: bool) -> None:
+    st = lib().hs_stage_profile_enable(C.c_void_p(stage), int(enable))
+    if st != HS_OK:
+        raise HsError(st, "hs_stage_profile_enable")
+
+
+def hs_stage_profile_read(stage: int):
+    """Returns {class name: (milliseconds, launches)} accumulated since the last read."""
+    ms = np.zeros(len(PROFILE_CLASSES), dtype=np.float32)
+    n = np.zeros(len(PROFILE_CLASSES), dtype=np.int32)
+    st = lib().hs_stage_profile_read(C.c_void_p(stage), ms.ctypes.data, n.ctypes.data)
+    if st != HS_OK:
+        raise HsError(st, "hs_stage_profile_read")
+    return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(PROFILE_CLASSES)}

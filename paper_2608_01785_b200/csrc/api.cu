@@ -124,7 +124,38 @@ struct hs_stage {
   cudaEvent_t ev[kRing] = {};
   bool ev_pending[kRing] = {};
   int ring_pos = 0;
+  // optional per-kernel timing
+  bool profile = false;
+  struct Timed { int cls; cudaEvent_t a, b; };
+  std::vector<Timed> timed;
+  std::vector<cudaEvent_t> event_pool;
 };
+
+namespace {
+// Brackets one launch with events when the stage is being profiled.
+struct LaunchTimer {
+  hs_stage* s;
+  cudaStream_t stream;
+  cudaEvent_t a = nullptr, b = nullptr;
+  int cls;
+  LaunchTimer(hs_stage* st, int c, cudaStream_t str) : s(st), stream(str), cls(c) {
+    if (!s->profile) return;
+    auto get = [&]() {
+      cudaEvent_t e = nullptr;
+      if (!s->event_pool.empty()) { e = s->event_pool.back(); s->event_pool.pop_back(); }
+      else cudaEventCreate(&e);
+      return e;
+    };
+    a = get(); b = get();
+    cudaEventRecord(a, stream);
+  }
+  ~LaunchTimer() {
+    if (!a) return;
+    cudaEventRecord(b, stream);
+    s->timed.push_back({cls, a, b});
+  }
+};
+}  // namespace
 
 extern "C" {
 
@@ -255,6 +286,8 @@ hs_status_t hs_stage_destroy(hs_stage_t* s) {
       }
       if (s->pinned[i]) cudaFreeHost(s->pinned[i]);
     }
+    for (const hs_stage::Timed& t : s->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
+    for (cudaEvent_t e : s->event_pool) cudaEventDestroy(e);
   }
   delete s;
   return HS_OK;
@@ -346,7 +379,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     np.T = T;
     np.d = d;
     np.eps = c.rms_eps;
-    if ((e = launch_rmsnorm(np, sm_budget, stream)) != cudaSuccess) break;
+    { LaunchTimer t(s, 0, stream); e = launch_rmsnorm(np, sm_budget, stream); }
+    if (e != cudaSuccess) break;
 
     GemmParams g{};
     g.tm_a = s->tm_h;
@@ -361,7 +395,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     g.tok_slot = meta + s->ml.tok_slot;
     g.rope = reinterpret_cast<const float2*>(s->ws_dev + s->ws.rope);
     g.status = status;
-    if ((e = launch_gemm(g, sm_budget, stream)) != cudaSuccess) break;
+    { LaunchTimer t(s, 1, stream); e = launch_gemm(g, sm_budget, stream); }
+    if (e != cudaSuccess) break;
 
     AttnParams a{};
     a.tm_kv = s->tm_kv;
@@ -381,9 +416,12 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     a.part_ml = reinterpret_cast<float*>(s->ws_dev + s->ws.part_ml);
     a.counters = meta + s->ml.counters + 2 * l;
     a.status = status;
-    if ((e = launch_attention_prefill(a, sm_budget, stream)) != cudaSuccess) break;
-    if ((e = launch_attention_decode(a, sm_budget, stream)) != cudaSuccess) break;
-    if ((e = launch_attention_combine(a, sm_budget, stream)) != cudaSuccess) break;
+    if (a.n_prefill_items > 0) { LaunchTimer t(s, 2, stream); e = launch_attention_prefill(a, sm_budget, stream); }
+    if (e != cudaSuccess) break;
+    if (a.n_decode_items > 0) { LaunchTimer t(s, 3, stream); e = launch_attention_decode(a, sm_budget, stream); }
+    if (e != cudaSuccess) break;
+    if (a.n_decode_rows > 0) { LaunchTimer t(s, 4, stream); e = launch_attention_combine(a, sm_budget, stream); }
+    if (e != cudaSuccess) break;
 
     GemmParams go{};
     go.tm_a = s->tm_o;
@@ -392,11 +430,13 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     go.mode = kGemmResid;
     go.resid = x; go.out = x;
     go.status = status;
-    if ((e = launch_gemm(go, sm_budget, stream)) != cudaSuccess) break;
+    { LaunchTimer t(s, 5, stream); e = launch_gemm(go, sm_budget, stream); }
+    if (e != cudaSuccess) break;
 
     np.x_bf16 = nullptr;
     np.gain = static_cast<const __nv_bfloat16*>(w.g_mlp);
-    if ((e = launch_rmsnorm(np, sm_budget, stream)) != cudaSuccess) break;
+    { LaunchTimer t(s, 0, stream); e = launch_rmsnorm(np, sm_budget, stream); }
+    if (e != cudaSuccess) break;
 
     GemmParams gu{};
     gu.tm_a = s->tm_h;
@@ -405,7 +445,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gu.mode = kGemmGateUp;
     gu.act = act;
     gu.status = status;
-    if ((e = launch_gemm(gu, sm_budget, stream)) != cudaSuccess) break;
+    { LaunchTimer t(s, 6, stream); e = launch_gemm(gu, sm_budget, stream); }
+    if (e != cudaSuccess) break;
 
     GemmParams gd{};
     gd.tm_a = s->tm_act;
@@ -415,7 +456,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gd.resid = x;
     gd.out = last ? static_cast<float*>(b->y_out) : x;
     gd.status = status;
-    if ((e = launch_gemm(gd, sm_budget, stream)) != cudaSuccess) break;
+    { LaunchTimer t(s, 7, stream); e = launch_gemm(gd, sm_budget, stream); }
+    if (e != cudaSuccess) break;
   }
   return e == cudaSuccess ? HS_OK : HS_ERR_CUDA;
 }
@@ -427,6 +469,32 @@ hs_status_t hs_stage_status(hs_stage_t* s) {
   int v = 0;
   if (cudaMemcpy(&v, s->ws_dev + s->ws.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return HS_ERR_CUDA;
   return v == 0 ? HS_OK : static_cast<hs_status_t>(v);
+}
+
+hs_status_t hs_stage_profile_enable(hs_stage_t* s, int32_t enable) {
+  if (!s) return HS_ERR_INVALID_ARG;
+  if (s->cfg.device < 0) return HS_ERR_NO_DEVICE;
+  s->profile = enable != 0;
+  return HS_OK;
+}
+
+hs_status_t hs_stage_profile_read(hs_stage_t* s, float* ms, int32_t* launches) {
+  if (!s || !ms || !launches) return HS_ERR_INVALID_ARG;
+  if (s->cfg.device < 0) return HS_ERR_NO_DEVICE;
+  DeviceGuard guard(s->cfg.device);
+  hs_status_t st = HS_OK;
+  for (const hs_stage::Timed& t : s->timed) {
+    float v = 0.f;
+    if (cudaEventSynchronize(t.b) != cudaSuccess || cudaEventElapsedTime(&v, t.a, t.b) != cudaSuccess) st = HS_ERR_CUDA;
+    if (t.cls >= 0 && t.cls < HS_PROFILE_CLASSES) {
+      ms[t.cls] += v;
+      launches[t.cls] += 1;
+    }
+    s->event_pool.push_back(t.a);
+    s->event_pool.push_back(t.b);
+  }
+  s->timed.clear();
+  return st;
 }
 
 hs_status_t hs_stage_debug_buffer(hs_stage_t* s, const char* name, void** dev_ptr, size_t* bytes) {

@@ -1,0 +1,279 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same seeded inputs.
+
+Tolerances (from the arithmetic: bf16 tensor-core operands, fp32 accumulation, fp32 residual stream):
+  y_out      max |y_gpu - y_oracle| <= 2e-2 * RMS(y_oracle), per tensor;
+  K/V bytes  each element written this step against the oracle's value BEFORE its bf16 rounding:
+             |k_gpu - k_ref| <= 2^-8 |k_ref| + 1e-2 RMS(k_ref) (one bf16 rounding plus operand noise; two
+             independently rounded bf16 tensors legitimately differ by an ulp in many elements);
+  integers   block tables, slots, and the set of cache bytes a step touches: bit-exact;
+  budgets    y_out and the whole KV pool bit-identical for every sm_budget.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle.oracle import Oracle
+from paper_2608_01785_b200 import binding as B
+from paper_2608_01785_b200 import workloads as wl
+from tests.gpu_helpers import bits_to_f32, make_stage, run_step
+from tests.helpers import make_case, rel_err
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+
+@pytest.fixture(scope="module")
+def orc():
+    return Oracle("f32")
+
+
+def one_layer(dims):
+    return wl.StageDims(1, dims.d_model, dims.n_q_heads, dims.n_kv_heads, dims.head_dim, dims.d_ffn)
+
+
+def check_kv_written(case, pool_in, pool_gpu, kv_pre, layer=0):
+    """Slots of `layer` written by the step obey the element rule; every other byte of the pool is unchanged."""
+    d = case.dims
+    shape = (d.n_layers, 2, case.cfg.num_pages, d.n_kv_heads, d.page_size, d.head_dim)
+    g = bits_to_f32(pool_gpu).reshape(shape)
+    touched = np.zeros(shape, dtype=bool)
+    t = 0
+    for s, (n, c) in enumerate(zip(case.batch.q_len, case.batch.ctx_len)):
+        for j in range(n):
+            p = c + j
+            page, slot = case.block_tables[s, p // 16], p % 16
+            touched[:, :, page, :, slot, :] = True
+            for kv in range(2):
+                ref = kv_pre[t, kv].reshape(d.n_kv_heads, d.head_dim).astype(np.float64)
+                got = g[layer, kv, page, :, slot, :].astype(np.float64)
+                rms = np.sqrt(np.mean(kv_pre[:, kv].astype(np.float64) ** 2))
+                bound = 2.0 ** -8 * np.abs(ref) + 1e-2 * rms
+                assert np.all(np.abs(got - ref) <= bound), (s, j, kv, float(np.max(np.abs(got - ref) / bound)))
+            t += 1
+    untouched = ~touched.reshape(-1)
+    assert np.array_equal(pool_gpu[untouched], pool_in[untouched]), "bytes outside the step's slots changed"
+
+
+# ----------------------------------------------------------------- GEMM op --
+@pytest.mark.parametrize("M,N,K,resid", [(128, 256, 64, False), (82, 520, 200, True), (300, 264, 72, True),
+                                         (2112, 1024, 3584, False), (1000, 2048, 1408, True), (16, 1536, 1024, True)])
+def test_gemm_op_matches_oracle_and_is_budget_invariant(orc, M, N, K, resid):
+    dev = torch.device("cuda:0")
+    g = torch.Generator().manual_seed(M * 7 + N)
+    a = torch.randn(M, K, generator=g).to(torch.bfloat16)
+    w = (torch.randn(N, K, generator=g) * 0.02).to(torch.bfloat16)
+    r = torch.randn(M, N, generator=g) if resid else None
+    want = orc.linear(a.float().numpy(), w.float().numpy())
+    if resid:
+        want = want + r.numpy()
+    outs = []
+    a_d, w_d = a.to(dev), w.to(dev)
+    for budget in (148, 74, 37, 8, 1):
+        if budget == 1 and M * N > 300 * 600:
+            continue
+        out = torch.full((M, N), float("nan"), device=dev)
+        status = torch.zeros(1, dtype=torch.int32, device=dev)
+        r_d = r.to(dev) if resid else None
+        B.hs_op_gemm_bf16(a_d.data_ptr(), w_d.data_ptr(), r_d.data_ptr() if resid else 0, out.data_ptr(), M, N, K,
+                          budget, status.data_ptr())
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        outs.append(out.cpu())
+    assert rel_err(outs[0].numpy(), want) < 1e-4          # fp32 accumulation of exact bf16 products
+    for o in outs[1:]:
+        assert torch.equal(o, outs[0])
+
+
+def test_gemm_op_in_place_residual(orc):
+    dev = torch.device("cuda:0")
+    g = torch.Generator().manual_seed(5)
+    a = torch.randn(200, 320, generator=g).to(torch.bfloat16)
+    w = torch.randn(264, 320, generator=g).to(torch.bfloat16)
+    x = torch.randn(200, 264, generator=g)
+    want = x.numpy() + orc.linear(a.float().numpy(), w.float().numpy())
+    x_d, a_d, w_d = x.to(dev), a.to(dev), w.to(dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    B.hs_op_gemm_bf16(a_d.data_ptr(), w_d.data_ptr(), x_d.data_ptr(), x_d.data_ptr(), 200, 264, 320, 148,
+                      status.data_ptr())
+    torch.cuda.synchronize()
+    assert rel_err(x_d.cpu().numpy(), want) < 1e-4
+
+
+def test_gemm_op_argument_errors():
+    dev = torch.device("cuda:0")
+    buf = torch.zeros(1 << 16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    p = buf.data_ptr()
+    for args, code in (((p, p, 0, p, 16, 20, 64, 148), B.HS_ERR_UNSUPPORTED_SHAPE),      # N % 8
+                       ((p, p, 0, p, 16, 64, 60, 148), B.HS_ERR_UNSUPPORTED_SHAPE),      # K % 8
+                       ((p, p, 0, p, 16, 64, 64, 0), B.HS_ERR_INVALID_BUDGET),
+                       ((p, p, 0, p, 16, 64, 64, 149), B.HS_ERR_INVALID_BUDGET),
+                       ((0, p, 0, p, 16, 64, 64, 148), B.HS_ERR_INVALID_ARG)):
+        with pytest.raises(B.HsError) as e:
+            B.hs_op_gemm_bf16(*args, status.data_ptr())
+        assert e.value.status == code
+
+
+# ---------------------------------------------------------------- config 1 --
+def config1_case(orc):
+    """Config 1 with a self-consistent cache: the decode sequences' context (40 and 64 tokens) is written
+    by an oracle prefill step, and that pool is what both sides start the step under test from."""
+    dims = wl.DIMS["c1_tiny"]
+    batch = wl.make_batch("c1_tiny", 0)
+    case = make_case(dims, batch, seed=0)
+    pre = wl.BatchSpec([40, 64], [0, 0])
+    x_pre = wl.to_f32_numpy(wl.make_x(pre.n_tokens, dims.d_model, 0, index=1))
+    orc.step(case.cfg, case.weights, case.kv_pool, pre.q_len, pre.ctx_len, case.block_tables[2:], x_pre)
+    return case
+
+
+def test_config1_step_matches_oracle_at_budgets_148_and_8(orc):
+    case = config1_case(orc)
+    assert case.block_tables[:, :5].tolist() == [[0, 1, -1, -1, -1], [2, 3, 4, -1, -1], [5, 6, 7, -1, -1],
+                                                 [8, 9, 10, 11, 12]]
+    pool_ref = case.kv_pool.copy()
+    y_ref, kv_pre = orc.layer(case.cfg, case.weights[0], 0, pool_ref, case.batch.q_len, case.batch.ctx_len,
+                              case.block_tables, case.x, want_kv_pre=True)
+    results = []
+    for budget in (148, 8):
+        st = make_stage(case)
+        y, pool = run_step(st, case, budget)
+        st.close()
+        err = rel_err(y, y_ref)
+        print(f"config 1, sm_budget {budget}: max|err|/RMS = {err:.2e}")
+        assert err <= TOL
+        check_kv_written(case, case.kv_pool, pool, kv_pre)
+        results.append((y, pool))
+    assert np.array_equal(results[0][0], results[1][0]) and np.array_equal(results[0][1], results[1][1])
+
+
+def test_budget_errors_and_idempotence(orc):
+    case = config1_case(orc)
+    st = make_stage(case)
+    try:
+        y1, pool1 = run_step(st, case, 148)
+        y2, pool2 = run_step(st, case, 3)            # same step again: same slots, same values
+        assert np.array_equal(y1, y2) and np.array_equal(pool1, pool2)
+        x = case.x_t.to(st.device)
+        y = torch.empty(case.batch.n_tokens, case.dims.d_model, device=st.device)
+        b = st.make_batch(case.batch.q_len, case.batch.ctx_len, case.block_tables, x, y)
+        for budget in (0, -1, st.sm_count + 1):
+            with pytest.raises(B.HsError) as e:
+                st.step(b, budget)
+            assert e.value.status == B.HS_ERR_INVALID_BUDGET
+        bad = case.block_tables.copy(); bad[0, 0] = case.cfg.num_pages
+        with pytest.raises(B.HsError) as e:
+            st.step(st.make_batch(case.batch.q_len, case.batch.ctx_len, bad, x, y), 8)
+        assert e.value.status == B.HS_ERR_BAD_BLOCK_TABLE
+        torch.cuda.synchronize()
+        assert np.array_equal(wl.bf16_bits_numpy(st.kv_pool).reshape(-1), pool1)   # nothing was launched
+    finally:
+        st.close()
+
+
+# -------------------------------------------------------------- edge cases --
+EDGE = {
+    # name: (dims, q_len, ctx_len)
+    "single_token_prompt": (wl.StageDims(1, 256, 4, 2, 64, 688), [1], [0]),
+    "page_boundaries": (wl.StageDims(1, 256, 4, 2, 64, 688), [16, 17, 15, 1, 1, 1], [0, 16, 1, 15, 16, 31]),
+    "continuation_chunks": (wl.StageDims(2, 256, 4, 2, 64, 688), [40, 100, 7], [24, 60, 129]),
+    "head_dim_128_mha": (wl.StageDims(1, 256, 2, 2, 128, 512), [70, 1, 33], [0, 200, 5]),
+    "gqa_7_dh128": (wl.StageDims(1, 512, 7, 1, 128, 1024), [61, 1, 1, 19], [3, 90, 700, 64]),
+    "gqa_16_dh64": (wl.StageDims(1, 256, 32, 2, 64, 256), [24, 1], [9, 130]),
+    "long_decode_many_splits": (wl.StageDims(1, 256, 4, 2, 64, 688), [1, 1, 1], [511, 512, 2100]),
+    "long_prefill_dh128": (wl.StageDims(1, 256, 8, 1, 128, 640), [700, 1], [0, 1500]),
+    "many_sequences": (wl.StageDims(1, 256, 4, 2, 64, 688), [1] * 40 + [3] * 10, list(range(0, 400, 10)) + [5] * 10),
+    "two_layers_talker_like": (wl.StageDims(2, 1024, 16, 4, 64, 2816), [1] * 16, [128 + 57 * i for i in range(16)]),
+}
+
+
+@pytest.mark.parametrize("name", sorted(EDGE))
+def test_edge_cases_match_oracle(orc, name):
+    dims, q_len, ctx_len = EDGE[name]
+    batch = wl.BatchSpec(list(q_len), list(ctx_len))
+    case = make_case(dims, batch, seed=11, kv_fill=True)
+    # the tail of every sequence's last page (and every page nobody owns) holds NaN on entry: it must
+    # neither reach the output nor be written
+    pool6 = case.kv_pool.reshape(dims.n_layers, 2, case.cfg.num_pages, dims.n_kv_heads, 16, dims.head_dim)
+    owned = np.zeros((case.cfg.num_pages, 16), dtype=bool)
+    for s, c in enumerate(batch.ctx_len):
+        for p in range(c):
+            owned[case.block_tables[s, p // 16], p % 16] = True
+    pool6[:, :, ~owned] = 0x7fc0
+    pool_ref = case.kv_pool.copy()
+    y_ref = orc.step(case.cfg, case.weights, pool_ref, batch.q_len, batch.ctx_len, case.block_tables, case.x)
+    assert np.all(np.isfinite(y_ref))
+    outs = []
+    for budget in (148, 5):
+        st = make_stage(case)
+        y, pool = run_step(st, case, budget)
+        st.close()
+        err = rel_err(y, y_ref)
+        print(f"{name}, sm_budget {budget}: max|err|/RMS = {err:.2e}")
+        assert err <= TOL
+        outs.append((y, pool))
+        # canary slots that the step does not own are untouched
+        written = np.zeros_like(owned)
+        for s, (n, c) in enumerate(zip(batch.q_len, batch.ctx_len)):
+            for p in range(c, c + n):
+                written[case.block_tables[s, p // 16], p % 16] = True
+        g6 = pool.reshape(pool6.shape)
+        assert np.all(g6[:, :, ~(owned | written)] == 0x7fc0)
+        assert np.array_equal(g6[:, :, owned & ~written], pool6[:, :, owned & ~written])
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+
+
+def test_chunked_prefill_then_decode_on_the_gpu_cache(orc):
+    """A multi-step chain that lives on the GPU's own cache: prefill in two chunks, then two decode steps;
+    every step is compared with the oracle running the same chain on its own cache."""
+    dims = wl.StageDims(2, 256, 4, 2, 64, 688)
+    total = wl.BatchSpec([50], [0])
+    case = make_case(dims, total, seed=13)
+    x_all = wl.make_x(50, dims.d_model, 13)
+    st = make_stage(case, max_tokens=64, max_position=64)
+    pool_ref = case.kv_pool.copy()
+    done = 0
+    try:
+        for n in (31, 17, 1, 1):
+            xs = x_all[done:done + n]
+            y_ref = orc.step(case.cfg, case.weights, pool_ref, [n], [done], case.block_tables, wl.to_f32_numpy(xs))
+            y, _ = run_step(st, case, 148, q_len=[n], ctx_len=[done], x_t=xs)
+            err = rel_err(y, y_ref)
+            print(f"chain step n={n} ctx={done}: max|err|/RMS = {err:.2e}")
+            assert err <= TOL
+            done += n
+    finally:
+        st.close()
+
+
+# ------------------------------------------------------ co-run on 2 streams --
+def test_corun_on_two_streams_is_bit_identical_to_solo(orc):
+    dims_a = wl.StageDims(2, 512, 8, 2, 64, 1408)
+    dims_b = wl.StageDims(2, 256, 4, 2, 64, 688)
+    case_a = make_case(dims_a, wl.BatchSpec([300, 200, 1, 1], [0, 40, 300, 900]), seed=21, kv_fill=True)
+    case_b = make_case(dims_b, wl.BatchSpec([1] * 8, [100 + 90 * i for i in range(8)]), seed=22, kv_fill=True)
+    st_a, st_b = make_stage(case_a), make_stage(case_b)
+    try:
+        ya_solo, pa_solo = run_step(st_a, case_a, 100)
+        yb_solo, pb_solo = run_step(st_b, case_b, 48)
+        sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+        dev = st_a.device
+        xa, xb = case_a.x_t.to(dev), case_b.x_t.to(dev)
+        ya = torch.empty(case_a.batch.n_tokens, dims_a.d_model, device=dev)
+        yb = torch.empty(case_b.batch.n_tokens, dims_b.d_model, device=dev)
+        ba = st_a.make_batch(case_a.batch.q_len, case_a.batch.ctx_len, case_a.block_tables, xa, ya)
+        bb = st_b.make_batch(case_b.batch.q_len, case_b.batch.ctx_len, case_b.block_tables, xb, yb)
+        torch.cuda.synchronize()
+        for _ in range(3):
+            st_a.step(ba, 100, sa)
+            st_b.step(bb, 48, sb)
+        torch.cuda.synchronize()
+        assert st_a.status() == 0 and st_b.status() == 0
+        assert np.array_equal(ya.cpu().numpy(), ya_solo) and np.array_equal(yb.cpu().numpy(), yb_solo)
+        assert np.array_equal(wl.bf16_bits_numpy(st_a.kv_pool).reshape(-1), pa_solo)
+        assert np.array_equal(wl.bf16_bits_numpy(st_b.kv_pool).reshape(-1), pb_solo)
+        y_ref = orc.step(case_a.cfg, case_a.weights, case_a.kv_pool.copy(), case_a.batch.q_len, case_a.batch.ctx_len,
+                         case_a.block_tables, case_a.x)
+        assert rel_err(ya_solo, y_ref) <= TOL
+    finally:
+        st_a.close(); st_b.close()
