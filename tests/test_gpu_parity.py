@@ -194,12 +194,14 @@ def test_edge_cases_match_oracle(orc, name):
     case = make_case(dims, batch, seed=11, kv_fill=True)
     # the tail of every sequence's last page (and every page nobody owns) holds NaN on entry: it must
     # neither reach the output nor be written
-    pool6 = case.kv_pool.reshape(dims.n_layers, 2, case.cfg.num_pages, dims.n_kv_heads, 16, dims.head_dim)
+    # view [layer][K|V][kv_head][page][slot][Dh] so that a [page, slot] mask indexes it
+    pool6 = case.kv_pool.reshape(dims.n_layers, 2, case.cfg.num_pages, dims.n_kv_heads, 16,
+                                 dims.head_dim).transpose(0, 1, 3, 2, 4, 5)
     owned = np.zeros((case.cfg.num_pages, 16), dtype=bool)
     for s, c in enumerate(batch.ctx_len):
         for p in range(c):
             owned[case.block_tables[s, p // 16], p % 16] = True
-    pool6[:, :, ~owned] = 0x7fc0
+    pool6[:, :, :, ~owned] = 0x7fc0
     pool_ref = case.kv_pool.copy()
     y_ref = orc.step(case.cfg, case.weights, pool_ref, batch.q_len, batch.ctx_len, case.block_tables, case.x)
     assert np.all(np.isfinite(y_ref))
@@ -217,9 +219,10 @@ def test_edge_cases_match_oracle(orc, name):
         for s, (n, c) in enumerate(zip(batch.q_len, batch.ctx_len)):
             for p in range(c, c + n):
                 written[case.block_tables[s, p // 16], p % 16] = True
-        g6 = pool.reshape(pool6.shape)
-        assert np.all(g6[:, :, ~(owned | written)] == 0x7fc0)
-        assert np.array_equal(g6[:, :, owned & ~written], pool6[:, :, owned & ~written])
+        g6 = pool.reshape(dims.n_layers, 2, case.cfg.num_pages, dims.n_kv_heads, 16,
+                          dims.head_dim).transpose(0, 1, 3, 2, 4, 5)
+        assert np.all(g6[:, :, :, ~(owned | written)] == 0x7fc0)
+        assert np.array_equal(g6[:, :, :, owned & ~written], pool6[:, :, :, owned & ~written])
     assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
 
 
