@@ -176,6 +176,10 @@ int32_t hs_stage_sm_count(const hs_stage_t *stage);
 hs_status_t hs_stage_destroy(hs_stage_t *stage);
 const char *hs_status_str(hs_status_t status);
 
+/* Text of the CUDA error behind the calling thread's most recent HS_ERR_CUDA ("" if there was none).
+ * The string is owned by the library and valid until the thread's next failing call. */
+const char *hs_last_error(void);
+
 #if defined(__GNUC__)
 #pragma GCC visibility pop
 #endif

@@ -19,7 +19,8 @@ extern "C" {
 /*
  * The dense contraction of the step (the projections of the decoder layer; the paper prints no
  * formula for them): out[M,N] (fp32) = a[M,K] (bf16, row-major) * w[N,K]^T (bf16, row-major, i.e.
- * [out_features, in_features]) + resid[M,N] (fp32, nullable, may alias out), fp32 accumulation,
+ * [out_features, in_features]) + resid[M,N] (fp32, nullable, may alias out; when it is a different buffer it
+ * is first copied to out, and the product is then added in place), fp32 accumulation,
  * run as at most sm_budget persistent blocks.  K and N must be multiples of 8; a, w 16-byte aligned.
  * `status_dev` is a device int (zero on entry) that receives HS_ERR_TIMEOUT if a bounded wait inside
  * the kernel runs out; it may not be NULL.
@@ -31,7 +32,6 @@ hs_status_t hs_op_gemm_bf16(const void *a, const void *w, const float *resid, fl
 /*
  * Diagnosis: device address and size of one of the stage's private intermediates after a step
  * (contents of the LAST layer executed).  name is one of
- *   "x"   fp32 [max_tokens, d]      residual stream before the last down projection was added to y_out
  *   "h"   bf16 [max_tokens, d]      last RMSNorm output
  *   "q"   bf16 [max_tokens, Hq*Dh]  queries after RoPE
  *   "o"   bf16 [max_tokens, Hq*Dh]  attention output

@@ -22,7 +22,7 @@ HS_OK, HS_ERR_INVALID_ARG, HS_ERR_INVALID_BUDGET, HS_ERR_UNSUPPORTED_SHAPE, HS_E
 EXPORTS = ("hs_status_str", "hs_kv_pool_bytes", "hs_workspace_bytes", "hs_stage_create", "hs_stage_destroy",
            "hs_kv_alloc", "hs_kv_free", "hs_kv_free_pages", "hs_stage_plan", "hs_stage_step", "hs_stage_status",
            "hs_stage_sm_count", "hs_op_gemm_bf16", "hs_stage_debug_buffer", "hs_stage_profile_enable",
-           "hs_stage_profile_read")
+           "hs_stage_profile_read", "hs_last_error")
 PROFILE_CLASSES = ("rmsnorm", "gemm_qkv", "attn_prefill", "attn_decode", "attn_combine", "gemm_out", "gemm_gateup",
                    "gemm_down")
 
@@ -52,7 +52,8 @@ class hs_batch_t(C.Structure):
 class HsError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__(f"{where}: {status_str(status)}")
+        detail = lib().hs_last_error().decode() if status == HS_ERR_CUDA else ""
+        super().__init__(f"{where}: {status_str(status)}" + (f" [{detail}]" if detail else ""))
 
 
 _lib: Optional[C.CDLL] = None
@@ -87,6 +88,7 @@ def lib() -> C.CDLL:
         l.hs_op_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                       C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         l.hs_stage_debug_buffer.argtypes = [C.c_void_p, C.c_char_p, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
+        l.hs_last_error.restype = C.c_char_p
         l.hs_stage_profile_enable.argtypes = [C.c_void_p, C.c_int32]
         l.hs_stage_profile_read.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = l
@@ -218,5 +220,5 @@ def hs_stage_profile_read(stage: int):
     n = np.zeros(len(PROFILE_CLASSES), dtype=np.int32)
     st = lib().hs_stage_profile_read(C.c_void_p(stage), ms.ctypes.data, n.ctypes.data)
     if st != HS_OK:
-        raise HsError(st, "hs_stage_profile_read")
+        raise HsError(st, "hs_stage_profile_read", "hs_last_error")
     return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(PROFILE_CLASSES)}

@@ -17,7 +17,7 @@ namespace {
 constexpr int kRing = 4;   // pinned staging slots for step metadata
 
 struct WsLayout {
-  size_t rope, x, h, q, o, act, meta, part_o, part_ml, status, total;
+  size_t rope, h, q, o, act, meta, part_o, part_ml, status, total;
 };
 
 WsLayout make_ws_layout(const hs_stage_config_t& c, const MetaLayout& ml) {
@@ -30,7 +30,6 @@ WsLayout make_ws_layout(const hs_stage_config_t& c, const MetaLayout& ml) {
   };
   const size_t T = c.max_tokens, q_dim = size_t(c.n_q_heads) * c.head_dim;
   w.rope = take(size_t(c.max_position) * (c.head_dim / 2) * sizeof(float2));
-  w.x = take(T * c.d_model * 4);
   w.h = take(T * c.d_model * 2);
   w.q = take(T * q_dim * 2);
   w.o = take(T * q_dim * 2);
@@ -61,18 +60,19 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// bf16 matrix [rows, cols] with cols contiguous; box = 64 columns x box_rows rows, 128-byte swizzle,
-// out-of-range elements read as zero.
-bool encode_2d(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+// Row-major matrix [rows, cols] (cols contiguous) of bf16 or fp32; box = 128 bytes of columns x box_rows
+// rows, 128-byte swizzle; out-of-range elements read as zero and are clipped on stores.
+bool encode_2d(CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, bool f32 = false) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return false;
+  const uint64_t esz = f32 ? 4 : 2;
   cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 2};
-  cuuint32_t box[2] = {64, box_rows};
+  cuuint64_t strides[1] = {cols * esz};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(128 / esz), box_rows};
   cuuint32_t estr[2] = {1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return fn(m, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
+            dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 struct LayerMaps {
@@ -92,12 +92,20 @@ struct DeviceGuard {
   }
 };
 
+thread_local std::string g_last_error;
+// Records where a CUDA call failed; returns HS_ERR_CUDA so that it can be used in a return statement.
+hs_status_t cuda_fail(const char* where, cudaError_t e) {
+  g_last_error = std::string(where) + ": " + cudaGetErrorName(e) + " (" + cudaGetErrorString(e) + ")";
+  return HS_ERR_CUDA;
+}
+
 bool g_attrs_set[64] = {};
 hs_status_t ensure_attributes(int device) {
   if (device >= 0 && device < 64 && g_attrs_set[device]) return HS_OK;
-  if (gemm_set_attributes() != cudaSuccess || norm_set_attributes() != cudaSuccess ||
-      attention_set_attributes() != cudaSuccess)
-    return HS_ERR_CUDA;
+  cudaError_t e;
+  if ((e = gemm_set_attributes()) != cudaSuccess) return cuda_fail("gemm attributes", e);
+  if ((e = norm_set_attributes()) != cudaSuccess) return cuda_fail("rmsnorm attributes", e);
+  if ((e = attention_set_attributes()) != cudaSuccess) return cuda_fail("attention attributes", e);
   if (device >= 0 && device < 64) g_attrs_set[device] = true;
   return HS_OK;
 }
@@ -119,7 +127,8 @@ struct hs_stage {
   __nv_bfloat16* kv_pool = nullptr;
   std::vector<hs_layer_weights_t> layers;
   std::vector<LayerMaps> maps;
-  CUtensorMap tm_h, tm_o, tm_act, tm_kv;
+  CUtensorMap tm_h, tm_o, tm_act, tm_kv;   // operand loads
+  CUtensorMap tm_q_st, tm_act_st;          // epilogue stores (box 64 x 32)
   int32_t* pinned[kRing] = {};
   cudaEvent_t ev[kRing] = {};
   bool ev_pending[kRing] = {};
@@ -158,6 +167,8 @@ struct LaunchTimer {
 }  // namespace
 
 extern "C" {
+
+const char* hs_last_error(void) { return g_last_error.c_str(); }
 
 const char* hs_status_str(hs_status_t s) {
   switch (s) {
@@ -246,6 +257,8 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
   const uint64_t q_dim = uint64_t(cfg->n_q_heads) * cfg->head_dim, kv_dim = uint64_t(cfg->n_kv_heads) * cfg->head_dim;
   bool ok = encode_2d(&s->tm_h, s->ws_dev + s->ws.h, T, d, 128) && encode_2d(&s->tm_o, s->ws_dev + s->ws.o, T, q_dim, 128) &&
             encode_2d(&s->tm_act, s->ws_dev + s->ws.act, T, F, 128);
+  ok = ok && encode_2d(&s->tm_q_st, s->ws_dev + s->ws.q, T, q_dim, 32) &&
+       encode_2d(&s->tm_act_st, s->ws_dev + s->ws.act, T, F, 32);
   const uint64_t pool_rows = uint64_t(cfg->n_layers) * 2 * cfg->num_pages * cfg->n_kv_heads * kPage;
   ok = ok && encode_2d(&s->tm_kv, s->kv_pool, pool_rows, cfg->head_dim, 16);
   s->maps.resize(cfg->n_layers);
@@ -356,19 +369,22 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
 
   const int T = plan.n_tokens, d = c.d_model, F = c.d_ffn, Dh = c.head_dim;
   const int q_dim = c.n_q_heads * Dh, kv_dim = c.n_kv_heads * Dh;
-  float* x = reinterpret_cast<float*>(s->ws_dev + s->ws.x);
+  // The fp32 residual stream lives in the caller's y_out for the whole step: the first RMSNorm widens
+  // x_in into it and every projection back to d_model is added into it by a TMA reduction.
+  float* x = static_cast<float*>(b->y_out);
+  CUtensorMap tm_y;
+  if (!encode_2d(&tm_y, x, T, d, 32, true)) return HS_ERR_CUDA;
   __nv_bfloat16* h = reinterpret_cast<__nv_bfloat16*>(s->ws_dev + s->ws.h);
   __nv_bfloat16* q = reinterpret_cast<__nv_bfloat16*>(s->ws_dev + s->ws.q);
   __nv_bfloat16* o = reinterpret_cast<__nv_bfloat16*>(s->ws_dev + s->ws.o);
-  __nv_bfloat16* act = reinterpret_cast<__nv_bfloat16*>(s->ws_dev + s->ws.act);
   int* status = reinterpret_cast<int*>(s->ws_dev + s->ws.status);
   const size_t layer_kv_elems = size_t(c.num_pages) * c.n_kv_heads * kPage * Dh;
   cudaError_t e = cudaSuccess;
+  const char* where = "";
 
   for (int l = 0; l < c.n_layers && e == cudaSuccess; ++l) {
     const hs_layer_weights_t& w = s->layers[l];
     const LayerMaps& m = s->maps[l];
-    const bool last = l == c.n_layers - 1;
 
     NormParams np{};
     np.x_bf16 = l == 0 ? static_cast<const __nv_bfloat16*>(b->x_in) : nullptr;
@@ -379,7 +395,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     np.T = T;
     np.d = d;
     np.eps = c.rms_eps;
-    { LaunchTimer t(s, 0, stream); e = launch_rmsnorm(np, sm_budget, stream); }
+    { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
     GemmParams g{};
@@ -388,14 +404,14 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     g.M = T; g.N = q_dim + 2 * kv_dim; g.K = d;
     g.mode = kGemmQkv;
     g.q_dim = q_dim; g.kv_dim = kv_dim; g.head_dim = Dh; g.n_kv_heads = c.n_kv_heads;
-    g.q_out = q;
+    g.tm_q = s->tm_q_st;
     g.k_cache = s->kv_pool + (size_t(l) * 2 + 0) * layer_kv_elems;
     g.v_cache = s->kv_pool + (size_t(l) * 2 + 1) * layer_kv_elems;
     g.tok_pos = meta + s->ml.tok_pos;
     g.tok_slot = meta + s->ml.tok_slot;
     g.rope = reinterpret_cast<const float2*>(s->ws_dev + s->ws.rope);
     g.status = status;
-    { LaunchTimer t(s, 1, stream); e = launch_gemm(g, sm_budget, stream); }
+    { LaunchTimer t(s, 1, stream); where = "qkv gemm"; e = launch_gemm(g, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
     AttnParams a{};
@@ -416,11 +432,11 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     a.part_ml = reinterpret_cast<float*>(s->ws_dev + s->ws.part_ml);
     a.counters = meta + s->ml.counters + 2 * l;
     a.status = status;
-    if (a.n_prefill_items > 0) { LaunchTimer t(s, 2, stream); e = launch_attention_prefill(a, sm_budget, stream); }
+    if (a.n_prefill_items > 0) { LaunchTimer t(s, 2, stream); where = "prefill attention"; e = launch_attention_prefill(a, sm_budget, stream); }
     if (e != cudaSuccess) break;
-    if (a.n_decode_items > 0) { LaunchTimer t(s, 3, stream); e = launch_attention_decode(a, sm_budget, stream); }
+    if (a.n_decode_items > 0) { LaunchTimer t(s, 3, stream); where = "decode attention"; e = launch_attention_decode(a, sm_budget, stream); }
     if (e != cudaSuccess) break;
-    if (a.n_decode_rows > 0) { LaunchTimer t(s, 4, stream); e = launch_attention_combine(a, sm_budget, stream); }
+    if (a.n_decode_rows > 0) { LaunchTimer t(s, 4, stream); where = "decode combine"; e = launch_attention_combine(a, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
     GemmParams go{};
@@ -428,14 +444,14 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     go.tm_b[0] = m.wo; go.tm_b[1] = m.wo; go.tm_b[2] = m.wo;
     go.M = T; go.N = d; go.K = q_dim;
     go.mode = kGemmResid;
-    go.resid = x; go.out = x;
+    go.tm_out = tm_y; go.accumulate = 1;
     go.status = status;
-    { LaunchTimer t(s, 5, stream); e = launch_gemm(go, sm_budget, stream); }
+    { LaunchTimer t(s, 5, stream); where = "out-proj gemm"; e = launch_gemm(go, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
     np.x_bf16 = nullptr;
     np.gain = static_cast<const __nv_bfloat16*>(w.g_mlp);
-    { LaunchTimer t(s, 0, stream); e = launch_rmsnorm(np, sm_budget, stream); }
+    { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
     GemmParams gu{};
@@ -443,9 +459,9 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gu.tm_b[0] = m.wgate; gu.tm_b[1] = m.wup; gu.tm_b[2] = m.wup;
     gu.M = T; gu.N = F; gu.K = d;
     gu.mode = kGemmGateUp;
-    gu.act = act;
+    gu.tm_act = s->tm_act_st;
     gu.status = status;
-    { LaunchTimer t(s, 6, stream); e = launch_gemm(gu, sm_budget, stream); }
+    { LaunchTimer t(s, 6, stream); where = "gate/up gemm"; e = launch_gemm(gu, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
     GemmParams gd{};
@@ -453,13 +469,12 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gd.tm_b[0] = m.wdown; gd.tm_b[1] = m.wdown; gd.tm_b[2] = m.wdown;
     gd.M = T; gd.N = d; gd.K = F;
     gd.mode = kGemmResid;
-    gd.resid = x;
-    gd.out = last ? static_cast<float*>(b->y_out) : x;
+    gd.tm_out = tm_y; gd.accumulate = 1;
     gd.status = status;
-    { LaunchTimer t(s, 7, stream); e = launch_gemm(gd, sm_budget, stream); }
+    { LaunchTimer t(s, 7, stream); where = "down gemm"; e = launch_gemm(gd, sm_budget, stream); }
     if (e != cudaSuccess) break;
   }
-  return e == cudaSuccess ? HS_OK : HS_ERR_CUDA;
+  return e == cudaSuccess ? HS_OK : cuda_fail(where, e);
 }
 
 hs_status_t hs_stage_status(hs_stage_t* s) {
@@ -504,8 +519,7 @@ hs_status_t hs_stage_debug_buffer(hs_stage_t* s, const char* name, void** dev_pt
   const size_t T = c.max_tokens, q_dim = size_t(c.n_q_heads) * c.head_dim;
   const std::string n(name);
   size_t off, sz;
-  if (n == "x") { off = s->ws.x; sz = T * c.d_model * 4; }
-  else if (n == "h") { off = s->ws.h; sz = T * c.d_model * 2; }
+  if (n == "h") { off = s->ws.h; sz = T * c.d_model * 2; }
   else if (n == "q") { off = s->ws.q; sz = T * q_dim * 2; }
   else if (n == "o") { off = s->ws.o; sz = T * q_dim * 2; }
   else if (n == "act") { off = s->ws.act; sz = T * c.d_ffn * 2; }
@@ -528,16 +542,23 @@ hs_status_t hs_op_gemm_bf16(const void* a, const void* w, const float* resid, fl
   if (prop.major != 10) return HS_ERR_CUDA;
   if (sm_budget < 1 || sm_budget > prop.multiProcessorCount) return HS_ERR_INVALID_BUDGET;
   if (ensure_attributes(dev) != HS_OK) return HS_ERR_CUDA;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   GemmParams g{};
-  if (!encode_2d(&g.tm_a, a, M, K, 128) || !encode_2d(&g.tm_b[0], w, N, K, 128)) return HS_ERR_CUDA;
+  if (!encode_2d(&g.tm_a, a, M, K, 128) || !encode_2d(&g.tm_b[0], w, N, K, 128) ||
+      !encode_2d(&g.tm_out, out, M, N, 32, true))
+    return HS_ERR_CUDA;
   g.tm_b[1] = g.tm_b[0];
   g.tm_b[2] = g.tm_b[0];
   g.M = M; g.N = N; g.K = K;
   g.mode = kGemmResid;
-  g.resid = resid;
-  g.out = out;
+  g.accumulate = resid != nullptr;
+  // the kernel adds into `out`: a residual that lives elsewhere is copied there first
+  if (resid && resid != out &&
+      cudaMemcpyAsync(out, resid, size_t(M) * N * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+    return HS_ERR_CUDA;
   g.status = status_dev;
-  return launch_gemm(g, sm_budget, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess ? HS_OK : HS_ERR_CUDA;
+  const cudaError_t e = launch_gemm(g, sm_budget, stream);
+  return e == cudaSuccess ? HS_OK : cuda_fail("gemm", e);
 }
 
 }  // extern "C"

@@ -3,8 +3,8 @@
 //
 //   prefill kernel   work item = (sequence, KV head, tile of 128/G tokens); the G query heads that share
 //                    the KV head are stacked as rows, so K/V are streamed once per KV head.  8 compute
-//                    warps x 16 rows, key blocks of 64 keys (4 pages) in a 4-stage ring fed by one
-//                    producer thread.
+//                    warps x 16 rows, key blocks of 64 keys (4 pages) in a 5-stage ring fed by one
+//                    producer thread that runs ahead across work items.
 //   decode kernel    work item = (sequence, KV head, run of <= 512 keys); rows = the G query heads of the
 //                    single new token.  4 compute warps each take one page of every 4-page stage; their
 //                    partial (max, sum, output) triples are merged in shared memory in warp order and
@@ -64,12 +64,21 @@ __device__ __forceinline__ uint32_t mask_v(uint32_t r, int k, int n_valid) {
   return r;
 }
 
+// Work hand-out shared by both kernels: the producer thread owns the queue head.  It pulls the next item
+// index, publishes it to the compute warps through a two-slot ring guarded by mbarriers, and immediately
+// starts fetching that item's pages, so the pipeline never drains at an item boundary and the compute
+// warps never meet at a block-wide barrier.
+struct ItemRing {
+  uint64_t full[2], empty[2];
+  int item[2];
+};
+
 // =================================================================== prefill ==
-constexpr int PF_WARPS = 8, PF_THREADS = (PF_WARPS + 1) * 32, PF_STAGES = 4, PF_BLOCK_KEYS = 64;
+constexpr int PF_WARPS = 8, PF_THREADS = (PF_WARPS + 1) * 32, PF_STAGES = 5, PF_BLOCK_KEYS = 64;
 
 template <int DH>
 constexpr int pf_smem_bytes() {
-  int b = 1024 + Geom<DH>::HALVES * 16384 + PF_STAGES * 8 * Geom<DH>::PAGE_BYTES + 256;
+  int b = 1024 + PF_STAGES * 8 * Geom<DH>::PAGE_BYTES + 512;
   return b > kMinSmemBytes ? b : kMinSmemBytes;
 }
 
@@ -79,12 +88,11 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
   constexpr int STAGE_BYTES = 8 * G_::PAGE_BYTES;   // 4 K pages then 4 V pages
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* q_smem = smem;                                      // [HALVES][128 rows][128 B], swizzled
-  uint8_t* stages = smem + G_::HALVES * 16384;
+  uint8_t* stages = smem;
   uint64_t* full = reinterpret_cast<uint64_t*>(stages + PF_STAGES * STAGE_BYTES);
   uint64_t* empty = full + PF_STAGES;
-  int* s_item = reinterpret_cast<int*>(empty + PF_STAGES);   // two slots, used alternately
-  volatile int* abort_flag = s_item + 2;
+  ItemRing* ring = reinterpret_cast<ItemRing*>(empty + PF_STAGES);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ring + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = p.n_q_heads / p.n_kv_heads;
@@ -96,35 +104,37 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
       mbar_init(&full[i], 1);
       mbar_init(&empty[i], PF_WARPS);
     }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&ring->full[i], 1);
+      mbar_init(&ring->empty[i], PF_WARPS);
+    }
     *abort_flag = 0;
     fence_barrier_init();
     tma_prefetch_desc(&p.tm_kv);
   }
   __syncthreads();
 
-  int s = 0;
-  uint32_t ph = 0;
-  bool alive = true;
-  for (int round = 0;; round ^= 1) {
-    // one barrier per item: a thread is never more than one item ahead, so two slots suffice
-    if (threadIdx.x == 0) s_item[round] = atomicAdd(p.counters, 1);
-    __syncthreads();
-    const int item = s_item[round];
-    if (item >= p.n_prefill_items || *abort_flag) break;
-    const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
-    const int seq = it.x, hk = it.y, tok_begin = it.z, n_tok = it.w;
-    const int ctx = p.seq_ctx[seq];
-    const int tok0 = p.seq_tok0[seq] + tok_begin;
-    const int pos0 = ctx + tok_begin;                 // position of the tile's first token
-    const int n_keys = pos0 + n_tok;
-    const int n_kblocks = (n_keys + PF_BLOCK_KEYS - 1) / PF_BLOCK_KEYS;
-    const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq;
+  int s = 0, rs = 0;          // K/V stage, item-ring slot
+  uint32_t ph = 0, rph = 0;   // and their phases
 
-    if (warp == PF_WARPS) {
-      // ----------------------------------------------------------- producer --
-      if (lane == 0 && alive) {
+  if (warp == PF_WARPS) {
+    // ------------------------------------------------------------- producer --
+    if (lane == 0) {
+      for (;;) {
+        if (!mbar_wait(&ring->empty[rs], rph ^ 1, abort_flag, p.status)) break;
+        const int item = atomicAdd(p.counters, 1);
+        ring->item[rs] = item;
+        mbar_arrive(&ring->full[rs]);
+        if (++rs == 2) { rs = 0; rph ^= 1; }
+        if (item >= p.n_prefill_items) break;
+        const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
+        const int seq = it.x, hk = it.y;
+        const int n_keys = p.seq_ctx[seq] + it.z + it.w;
+        const int n_kblocks = (n_keys + PF_BLOCK_KEYS - 1) / PF_BLOCK_KEYS;
+        const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq;
+        bool ok = true;
         for (int kb = 0; kb < n_kblocks; ++kb) {
-          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status)) { alive = false; break; }
+          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status)) { ok = false; break; }
           const int rem = n_keys - kb * PF_BLOCK_KEYS;
           const int np = rem >= PF_BLOCK_KEYS ? 4 : (rem + 15) >> 4;
           uint8_t* st = stages + s * STAGE_BYTES;
@@ -136,33 +146,49 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
           }
           if (++s == PF_STAGES) { s = 0; ph ^= 1; }
         }
+        if (!ok) break;
       }
-    } else {
-      // ---------------------------------------------------------- consumers --
+    }
+  } else {
+    // ------------------------------------------------------------ consumers --
+    for (;;) {
+      bool ok = mbar_wait(&ring->full[rs], rph, abort_flag, p.status);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      const int item = ring->item[rs];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ring->empty[rs]);
+      if (++rs == 2) { rs = 0; rph ^= 1; }
+      if (item >= p.n_prefill_items) break;
+      const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
+      const int seq = it.x, hk = it.y, tok_begin = it.z, n_tok = it.w;
+      const int tok0 = p.seq_tok0[seq] + tok_begin;
+      const int pos0 = p.seq_ctx[seq] + tok_begin;        // position of the tile's first token
+      const int n_keys = pos0 + n_tok;
+      const int n_kblocks = (n_keys + PF_BLOCK_KEYS - 1) / PF_BLOCK_KEYS;
       const int n_rows = n_tok * G;
-      // stage the Q tile: row r = (token r / G, query head hk*G + r % G)
-      for (int idx = threadIdx.x; idx < 128 * G_::CHUNKS; idx += PF_WARPS * 32) {
-        const int r = idx / G_::CHUNKS, cc = idx % G_::CHUNKS;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (r < n_rows) {
-          const __nv_bfloat16* src = p.q + size_t(tok0 + r / G) * q_dim + (hk * G + r % G) * DH + cc * 8;
-          v = *reinterpret_cast<const uint4*>(src);
-        }
-        *reinterpret_cast<uint4*>(q_smem + (cc >> 3) * 16384 + r * 128 + (((cc & 7) ^ (r & 7)) << 4)) = v;
-      }
-      named_barrier_sync(1, PF_WARPS * 32);
-      uint32_t qf[DH / 16][4];
-#pragma unroll
-      for (int ks = 0; ks < DH / 16; ++ks) {
-        const int r = warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8, cc = 2 * ks + (lane >> 4);
-        ldmatrix_x4(qf[ks], smem_u32(q_smem + (cc >> 3) * 16384 + r * 128 + (((cc & 7) ^ (r & 7)) << 4)));
-      }
-      // positions of this thread's two rows (padding rows behave like the tile's last token)
+
+      // this thread's two rows: row r = (token r / G, query head hk*G + r % G); padding rows behave like
+      // the tile's last token and are never written
       const int row_a = warp * 16 + (lane >> 2), row_b = row_a + 8;
       const int pos_a = pos0 + min(row_a / G, n_tok - 1), pos_b = pos0 + min(row_b / G, n_tok - 1);
       const bool warp_has_rows = warp * 16 < n_rows;
       const int warp_min_pos = pos0 + min((warp * 16) / G, n_tok - 1);
       const int warp_max_pos = pos0 + min((warp * 16 + 15) / G, n_tok - 1);
+
+      // Q fragments straight from global memory (written by the QKV GEMM just before; L2 hits)
+      uint32_t qf[DH / 16][4];
+      {
+        const __nv_bfloat16* qa = p.q + size_t(tok0 + min(row_a / G, n_tok - 1)) * q_dim + (hk * G + row_a % G) * DH;
+        const __nv_bfloat16* qb = p.q + size_t(tok0 + min(row_b / G, n_tok - 1)) * q_dim + (hk * G + row_b % G) * DH;
+#pragma unroll
+        for (int ks = 0; ks < DH / 16; ++ks) {
+          const int c = ks * 16 + 2 * (lane & 3);
+          qf[ks][0] = *reinterpret_cast<const uint32_t*>(qa + c);
+          qf[ks][1] = *reinterpret_cast<const uint32_t*>(qb + c);
+          qf[ks][2] = *reinterpret_cast<const uint32_t*>(qa + c + 8);
+          qf[ks][3] = *reinterpret_cast<const uint32_t*>(qb + c + 8);
+        }
+      }
 
       float o_acc[DH / 8][4];
 #pragma unroll
@@ -170,8 +196,8 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
       float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
 
       for (int kb = 0; kb < n_kblocks; ++kb) {
-        const bool ok = alive && mbar_wait(&full[s], ph, abort_flag, p.status);
-        if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+        ok = mbar_wait(&full[s], ph, abort_flag, p.status);
+        if (!__all_sync(0xffffffffu, ok)) break;
         const int key0 = kb * PF_BLOCK_KEYS;
         if (warp_has_rows && key0 <= warp_max_pos) {
           const uint32_t k_base = smem_u32(stages + s * STAGE_BYTES);
@@ -264,7 +290,8 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         if (lane == 0) mbar_arrive(&empty[s]);
         if (++s == PF_STAGES) { s = 0; ph ^= 1; }
       }
-      if (alive && warp_has_rows) {
+      if (!__all_sync(0xffffffffu, ok)) break;
+      if (warp_has_rows) {
         l_a = quad_sum(l_a);
         l_b = quad_sum(l_b);
         const float inv_a = 1.f / l_a, inv_b = 1.f / l_b;
@@ -283,7 +310,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
       }
     }
   }
-  __syncwarp();
+  __syncthreads();
   if (*abort_flag) drain_after_abort();
 }
 
@@ -292,7 +319,7 @@ constexpr int DC_WARPS = 4, DC_THREADS = (DC_WARPS + 1) * 32, DC_STAGES = 5;
 
 template <int DH>
 constexpr int dc_smem_bytes() {
-  int b = 1024 + DC_STAGES * 8 * Geom<DH>::PAGE_BYTES + DC_WARPS * 16 * DH * 4 + DC_WARPS * 16 * 2 * 4 + 256;
+  int b = 1024 + DC_STAGES * 8 * Geom<DH>::PAGE_BYTES + DC_WARPS * 16 * DH * 4 + DC_WARPS * 16 * 2 * 4 + 512;
   return b > kMinSmemBytes ? b : kMinSmemBytes;
 }
 
@@ -307,8 +334,8 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
   float* sm_ml = sm_o + DC_WARPS * 16 * DH;                                   // [warp][16][2]
   uint64_t* full = reinterpret_cast<uint64_t*>(sm_ml + DC_WARPS * 16 * 2);
   uint64_t* empty = full + DC_STAGES;
-  int* s_item = reinterpret_cast<int*>(empty + DC_STAGES);   // two slots, used alternately
-  volatile int* abort_flag = s_item + 2;
+  ItemRing* ring = reinterpret_cast<ItemRing*>(empty + DC_STAGES);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(ring + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = p.n_q_heads / p.n_kv_heads;
@@ -320,30 +347,37 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
       mbar_init(&full[i], 1);
       mbar_init(&empty[i], DC_WARPS);
     }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&ring->full[i], 1);
+      mbar_init(&ring->empty[i], DC_WARPS);
+    }
     *abort_flag = 0;
     fence_barrier_init();
     tma_prefetch_desc(&p.tm_kv);
   }
   __syncthreads();
 
-  int s = 0;
-  uint32_t ph = 0;
-  bool alive = true;
-  for (int round = 0;; round ^= 1) {
-    if (threadIdx.x == 0) s_item[round] = atomicAdd(p.counters + 1, 1);
-    __syncthreads();
-    const int item = s_item[round];
-    if (item >= p.n_decode_items || *abort_flag) break;
-    const int4 it = reinterpret_cast<const int4*>(p.decode_items)[item];
-    const int seq = it.x, hk = it.y, k0 = it.z, k1 = it.w;
-    const int n_pages = (k1 - k0 + 15) >> 4, first_page = k0 >> 4;
-    const int n_iters = (n_pages + 3) >> 2;
-    const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq + first_page;
+  int s = 0, rs = 0;
+  uint32_t ph = 0, rph = 0;
 
-    if (warp == DC_WARPS) {
-      if (lane == 0 && alive) {
+  if (warp == DC_WARPS) {
+    // ------------------------------------------------------------- producer --
+    if (lane == 0) {
+      for (;;) {
+        if (!mbar_wait(&ring->empty[rs], rph ^ 1, abort_flag, p.status)) break;
+        const int item = atomicAdd(p.counters + 1, 1);
+        ring->item[rs] = item;
+        mbar_arrive(&ring->full[rs]);
+        if (++rs == 2) { rs = 0; rph ^= 1; }
+        if (item >= p.n_decode_items) break;
+        const int4 it = reinterpret_cast<const int4*>(p.decode_items)[item];
+        const int seq = it.x, hk = it.y, k0 = it.z, k1 = it.w;
+        const int n_pages = (k1 - k0 + 15) >> 4;
+        const int n_iters = (n_pages + 3) >> 2;
+        const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq + (k0 >> 4);
+        bool ok = true;
         for (int i = 0; i < n_iters; ++i) {
-          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status)) { alive = false; break; }
+          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status)) { ok = false; break; }
           const int np = min(4, n_pages - i * 4);
           uint8_t* st = stages + s * STAGE_BYTES;
           mbar_expect_tx(&full[s], np * 2 * G_::PAGE_BYTES);
@@ -354,8 +388,24 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
           }
           if (++s == DC_STAGES) { s = 0; ph ^= 1; }
         }
+        if (!ok) break;
       }
-    } else {
+    }
+  } else {
+    // ------------------------------------------------------------ consumers --
+    for (;;) {
+      bool ok = mbar_wait(&ring->full[rs], rph, abort_flag, p.status);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      const int item = ring->item[rs];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ring->empty[rs]);
+      if (++rs == 2) { rs = 0; rph ^= 1; }
+      if (item >= p.n_decode_items) break;
+      const int4 it = reinterpret_cast<const int4*>(p.decode_items)[item];
+      const int seq = it.x, hk = it.y, k0 = it.z, k1 = it.w;
+      const int n_pages = (k1 - k0 + 15) >> 4;
+      const int n_iters = (n_pages + 3) >> 2;
+
       // Q fragments straight from global memory: rows = query heads hk*G .. hk*G + G - 1 of the new token
       const int tok = p.seq_tok0[seq];
       const __nv_bfloat16* qrow = p.q + size_t(tok) * q_dim + size_t(hk) * G * DH;
@@ -375,8 +425,8 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
       float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
 
       for (int i = 0; i < n_iters; ++i) {
-        const bool ok = alive && mbar_wait(&full[s], ph, abort_flag, p.status);
-        if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }
+        ok = mbar_wait(&full[s], ph, abort_flag, p.status);
+        if (!__all_sync(0xffffffffu, ok)) break;
         const int pi = i * 4 + warp;
         if (pi < n_pages) {
           const uint32_t k_base = smem_u32(stages + s * STAGE_BYTES + warp * G_::PAGE_BYTES);
@@ -451,6 +501,7 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
         if (lane == 0) mbar_arrive(&empty[s]);
         if (++s == DC_STAGES) { s = 0; ph ^= 1; }
       }
+      const bool alive = __all_sync(0xffffffffu, ok);
       // merge the four warps' partials in warp order
       l_a = quad_sum(l_a);
       l_b = quad_sum(l_b);
@@ -490,9 +541,11 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
           }
         }
       }
+      named_barrier_sync(2, DC_WARPS * 32);     // the merge buffers are free again
+      if (!alive) break;
     }
   }
-  __syncwarp();
+  __syncthreads();
   if (*abort_flag) drain_after_abort();
 }
 

@@ -10,8 +10,10 @@
 //               tile is produced by exactly one block with a fixed K order, so results do not depend on
 //               the budget.
 //
-// Epilogues: residual add (fp32 in / out), QKV (rotate-half RoPE + bf16 q + scatter of k, v into the
-// paged cache), gate/up (silu(gate) * up -> bf16).
+// Epilogues: residual add (the fp32 tile is ADDED into the residual stream by a TMA reduction, so the
+// stream is never read by the SM), QKV (rotate-half RoPE; bf16 q by TMA store; k, v scattered into the
+// paged cache), gate/up (silu(gate) * up -> bf16 by TMA store).  Output blocks are staged in shared memory
+// in the 128-byte-swizzled layout the tensor maps expect (conflict-free for one-row-per-thread writes).
 #include "kernels.h"
 #include "ptx.cuh"
 
@@ -24,7 +26,10 @@ constexpr int BH_BYTES = 128 * BK * 2;          // one 128-row half of the B til
 constexpr int STAGE_BYTES = A_BYTES + 2 * BH_BYTES;
 constexpr int GEMM_THREADS = 192;
 constexpr int TMEM_COLS = 512;                  // two 128 x 256 fp32 accumulators
-constexpr int GEMM_SMEM = 1024 + STAGES * STAGE_BYTES + 256;
+constexpr int EPI_BUF_BYTES = 4096;             // 32 rows x 128 B: a 32 x 32 fp32 or 32 x 64 bf16 output block
+constexpr int EPI_WARP_BYTES = 2 * EPI_BUF_BYTES;   // two blocks per epilogue warp, filled alternately
+constexpr int GEMM_SMEM = 1024 + STAGES * STAGE_BYTES + 4 * EPI_WARP_BYTES + 256;
+static_assert(GEMM_SMEM <= 227 * 1024, "fits one SM");
 static_assert(GEMM_SMEM >= kMinSmemBytes, "one block per SM");
 
 struct BSource { int map, row; };
@@ -54,6 +59,27 @@ __device__ __forceinline__ void store_bf16x32(__nv_bfloat16* dst, const float (&
   }
 }
 
+// Staging layout of an output block: row r (one thread of the warp) is 128 bytes = 8 units of 16 B,
+// unit u stored at r * 128 + ((u ^ (r & 7)) << 4): the 128-byte swizzle of the output tensor maps.
+__device__ __forceinline__ void stage_f32x32(uint8_t* buf, int lane, const uint32_t (&r)[32]) {
+#pragma unroll
+  for (int u = 0; u < 8; ++u)
+    *reinterpret_cast<uint4*>(buf + lane * 128 + ((u ^ (lane & 7)) << 4)) =
+        make_uint4(r[4 * u], r[4 * u + 1], r[4 * u + 2], r[4 * u + 3]);
+}
+// 32 values -> bf16 into units u0 .. u0+3 of the thread's row (u0 = 0 or 4: which 32 of the 64 columns).
+__device__ __forceinline__ void stage_bf16x32(uint8_t* buf, int lane, int u0, const float (&v)[32]) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    uint4 w;
+    w.x = pack_bf16(v[i * 8 + 0], v[i * 8 + 1]);
+    w.y = pack_bf16(v[i * 8 + 2], v[i * 8 + 3]);
+    w.z = pack_bf16(v[i * 8 + 4], v[i * 8 + 5]);
+    w.w = pack_bf16(v[i * 8 + 6], v[i * 8 + 7]);
+    *reinterpret_cast<uint4*>(buf + lane * 128 + (((u0 + i) ^ (lane & 7)) << 4)) = w;
+  }
+}
+
 // Address of element e of (slot, kv head) in one layer's K or V pages.
 __device__ __forceinline__ __nv_bfloat16* cache_ptr(__nv_bfloat16* base, int slot, int hk, int n_kv_heads, int Dh,
                                                     int e) {
@@ -64,7 +90,8 @@ __device__ __forceinline__ __nv_bfloat16* cache_ptr(__nv_bfloat16* base, int slo
 __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  uint8_t* epi_smem = smem + STAGES * STAGE_BYTES;
+  uint64_t* full = reinterpret_cast<uint64_t*>(epi_smem + 4 * EPI_WARP_BYTES);
   uint64_t* empty = full + STAGES;
   uint64_t* tfull = empty + STAGES;
   uint64_t* tempty = tfull + 2;
@@ -90,6 +117,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     fence_barrier_init();
     tma_prefetch_desc(&p.tm_a);
     tma_prefetch_desc(&p.tm_b[0]);
+    tma_prefetch_desc(p.mode == kGemmResid ? &p.tm_out : p.mode == kGemmQkv ? &p.tm_q : &p.tm_act);
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, TMEM_COLS);
@@ -154,6 +182,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     int acc = 0;
     uint32_t acc_ph = 0;
     const int Dh = p.head_dim;
+    uint8_t* epi_buf = epi_smem + quarter * EPI_WARP_BYTES;
+    int epi_sel = 0;                          // staging block to fill next
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
       const int m = tile % n_m_tiles, n = tile / n_m_tiles;
       const bool ok = mbar_wait(&tfull[acc], acc_ph, abort_flag, p.status);
@@ -165,28 +195,26 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
       uint32_t r0[32], r1[32];
       float v0[32], v1[32];
 
+      const int row_base = m * BM + quarter * 32;          // first row of this warp's 32
+
       if (p.mode == kGemmResid) {
         for (int c = 0; c < BN / 32; ++c) {
           const int col0 = n * BN + c * 32;
           if (col0 >= p.N) break;
           tmem_ld32(taddr + c * 32, r0);
           tmem_ld_wait();
-          if (row_ok) {
-            float* o = p.out + size_t(row) * p.N + col0;
-            const float* rs = p.resid ? p.resid + size_t(row) * p.N + col0 : nullptr;
-#pragma unroll
-            for (int v = 0; v < 8; ++v) {
-              if (col0 + v * 4 < p.N) {
-                float4 a = make_float4(__uint_as_float(r0[4 * v]), __uint_as_float(r0[4 * v + 1]),
-                                       __uint_as_float(r0[4 * v + 2]), __uint_as_float(r0[4 * v + 3]));
-                if (rs) {
-                  const float4 b = ld4(rs + 4 * v);
-                  a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
-                }
-                *reinterpret_cast<float4*>(o + 4 * v) = a;
-              }
-            }
+          if (lane == 0) bulk_wait_read<1>();     // the block staged two chunks ago has been read
+          __syncwarp();
+          uint8_t* buf = epi_buf + epi_sel * EPI_BUF_BYTES;
+          stage_f32x32(buf, lane, r0);
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            if (p.accumulate) tma_reduce_add_2d(&p.tm_out, buf, col0, row_base);
+            else tma_store_2d(&p.tm_out, buf, col0, row_base);
+            bulk_commit();
           }
+          epi_sel ^= 1;
         }
       } else if (p.mode == kGemmGateUp) {
         for (int c = 0; c < 4; ++c) {
@@ -195,13 +223,26 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
           tmem_ld32(taddr + c * 32, r0);          // gate
           tmem_ld32(taddr + 128 + c * 32, r1);    // up
           tmem_ld_wait();
-          if (row_ok) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) {
-              const float g = __uint_as_float(r0[e]), u = __uint_as_float(r1[e]);
-              v0[e] = g / (1.f + __expf(-g)) * u;
+          for (int e = 0; e < 32; ++e) {
+            const float g = __uint_as_float(r0[e]), u = __uint_as_float(r1[e]);
+            v0[e] = __fdividef(g * u, 1.f + __expf(-g));   // silu(g) * u
+          }
+          uint8_t* buf = epi_buf + epi_sel * EPI_BUF_BYTES;
+          if ((c & 1) == 0) {
+            if (lane == 0) bulk_wait_read<1>();
+            __syncwarp();
+          }
+          stage_bf16x32(buf, lane, (c & 1) * 4, v0);
+          const bool block_done = (c & 1) || col0 + 32 >= p.N;
+          if (block_done) {                       // 64 columns staged (or the ragged end of the row)
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&p.tm_act, buf, n * 128 + (c >> 1) * 64, row_base);
+              bulk_commit();
             }
-            store_bf16x32(p.act + size_t(row) * p.N + col0, v0, p.N - col0);
+            epi_sel ^= 1;
           }
         }
       } else {
@@ -226,32 +267,44 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
               }
             }
           } else {
+            if (region == 0) {                    // both staging blocks are about to be refilled
+              if (lane == 0) bulk_wait_read<0>();
+              __syncwarp();
+            }
             for (int j = 0; j < 2; ++j) {
               const int lo = Dh == 128 ? j : 2 * j, hi = lo + (Dh == 128 ? 2 : 1);
               const int i0 = Dh == 128 ? 32 * j : 0;       // index of the first rotation pair
               tmem_ld32(taddr + half * 128 + lo * 32, r0);
               tmem_ld32(taddr + half * 128 + hi * 32, r1);
               tmem_ld_wait();
-              if (row_ok) {
-                const float2* cs = p.rope + size_t(pos) * half_dh + i0;
+              const float2* cs = p.rope + size_t(pos) * half_dh + i0;
 #pragma unroll
-                for (int e = 0; e < 32; e += 2) {
-                  const float4 t = *reinterpret_cast<const float4*>(cs + e);   // cos,sin of pairs e, e+1
-                  const float a0 = __uint_as_float(r0[e]), b0 = __uint_as_float(r1[e]);
-                  const float a1 = __uint_as_float(r0[e + 1]), b1 = __uint_as_float(r1[e + 1]);
-                  v0[e] = a0 * t.x - b0 * t.y;
-                  v1[e] = b0 * t.x + a0 * t.y;
-                  v0[e + 1] = a1 * t.z - b1 * t.w;
-                  v1[e + 1] = b1 * t.z + a1 * t.w;
-                }
+              for (int e = 0; e < 32; e += 2) {
+                const float4 t = *reinterpret_cast<const float4*>(cs + e);   // cos,sin of pairs e, e+1
+                const float a0 = __uint_as_float(r0[e]), b0 = __uint_as_float(r1[e]);
+                const float a1 = __uint_as_float(r0[e + 1]), b1 = __uint_as_float(r1[e + 1]);
+                v0[e] = a0 * t.x - b0 * t.y;
+                v1[e] = b0 * t.x + a0 * t.y;
+                v0[e + 1] = a1 * t.z - b1 * t.w;
+                v1[e + 1] = b1 * t.z + a1 * t.w;
+              }
+              if (region == 0) {
+                // chunk ch of the half belongs to 64-column block ch / 2, units 4 (ch % 2) ..
+                stage_bf16x32(epi_buf + (lo >> 1) * EPI_BUF_BYTES, lane, (lo & 1) * 4, v0);
+                stage_bf16x32(epi_buf + (hi >> 1) * EPI_BUF_BYTES, lane, (hi & 1) * 4, v1);
+              } else if (row_ok) {
                 const int col_lo = vcol + lo * 32, col_hi = vcol + hi * 32;
-                if (region == 0) {
-                  store_bf16x32(p.q_out + size_t(row) * p.q_dim + col_lo, v0, 32);
-                  store_bf16x32(p.q_out + size_t(row) * p.q_dim + col_hi, v1, 32);
-                } else {
-                  store_bf16x32(cache_ptr(p.k_cache, slot, col_lo / Dh, p.n_kv_heads, Dh, col_lo % Dh), v0, 32);
-                  store_bf16x32(cache_ptr(p.k_cache, slot, col_hi / Dh, p.n_kv_heads, Dh, col_hi % Dh), v1, 32);
-                }
+                store_bf16x32(cache_ptr(p.k_cache, slot, col_lo / Dh, p.n_kv_heads, Dh, col_lo % Dh), v0, 32);
+                store_bf16x32(cache_ptr(p.k_cache, slot, col_hi / Dh, p.n_kv_heads, Dh, col_hi % Dh), v1, 32);
+              }
+            }
+            if (region == 0) {
+              fence_proxy_async();
+              __syncwarp();
+              if (lane == 0) {
+                tma_store_2d(&p.tm_q, epi_buf, vcol, row_base);
+                tma_store_2d(&p.tm_q, epi_buf + EPI_BUF_BYTES, vcol + 64, row_base);
+                bulk_commit();
               }
             }
           }
@@ -262,6 +315,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
       acc ^= 1;
       if (acc == 0) acc_ph ^= 1;
     }
+    if (lane == 0) bulk_wait<0>();            // every output block has been written
   }
 
   // ------------------------------------------------------------- teardown --

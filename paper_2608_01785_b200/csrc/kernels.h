@@ -17,7 +17,7 @@ constexpr int kMinSmemBytes = 117 * 1024;
 // out = A[M,K] * W^T with W given as up to three row blocks [rows, K] (bf16, K contiguous).  The output
 // tile is 128 x 256 "virtual" columns; each 128-column half of a tile is fetched from one weight matrix.
 enum GemmMode : int {
-  kGemmResid = 0,   // out[M,N] fp32 = (resid ? resid : 0) + A W^T                     (out-proj, down)
+  kGemmResid = 0,   // out[M,N] fp32 (+)= A W^T: TMA store, or TMA add-reduction into out (out-proj, down)
   kGemmQkv = 1,     // virtual columns [q | k | v]; RoPE on q,k; q -> bf16 buffer, k,v -> paged cache
   kGemmGateUp = 2   // tile = 128 gate columns + the same 128 up columns; act = silu(gate) * up -> bf16
 };
@@ -28,18 +28,18 @@ struct GemmParams {
   int M, N, K;               // N: Resid output width; Qkv (Hq + 2 Hkv) * Dh; GateUp F (activation width)
   int mode;
   // Resid
-  const float* resid;        // nullable; may alias out
-  float* out;                // [M, N]
+  CUtensorMap tm_out;        // fp32 [M, N], box 32 x 32, 128-byte swizzle (rows past M are clipped)
+  int accumulate;            // 1: out += A W^T (the residual add), 0: out = A W^T
   // Qkv
   int q_dim, kv_dim, head_dim, n_kv_heads;
-  __nv_bfloat16* q_out;      // [M, q_dim]
+  CUtensorMap tm_q;          // bf16 q [M, q_dim], box 64 x 32, 128-byte swizzle
   __nv_bfloat16* k_cache;    // this layer's K pages: [page][kv_head][16][Dh]
   __nv_bfloat16* v_cache;
   const int32_t* tok_pos;    // [M]
   const int32_t* tok_slot;   // [M]
   const float2* rope;        // [max_position][Dh/2] (cos, sin)
   // GateUp
-  __nv_bfloat16* act;        // [M, N]
+  CUtensorMap tm_act;        // bf16 act [M, N], box 64 x 32, 128-byte swizzle
   int* status;               // device status word
 };
 cudaError_t launch_gemm(const GemmParams& p, int sm_budget, cudaStream_t stream);

@@ -67,12 +67,11 @@ class Stage:
         return B.hs_stage_status(self.handle)
 
     def debug_tensor(self, name: str) -> torch.Tensor:
-        """Copy of a private intermediate ("x" fp32; "h", "q", "o", "act" bf16), shaped [max_tokens, width]."""
+        """Copy of a private intermediate ("h", "q", "o", "act"; bf16), shaped [max_tokens, width]."""
         ptr, size = B.hs_stage_debug_buffer(self.handle, name)
         off = ptr - self.workspace.data_ptr()
         raw = self.workspace[off: off + size].clone()
-        dt = torch.float32 if name == "x" else torch.bfloat16
-        return raw.view(dt).view(self.cfg.max_tokens, -1)
+        return raw.view(torch.bfloat16).view(self.cfg.max_tokens, -1)
 
     def close(self) -> None:
         if self.handle:
