@@ -94,14 +94,14 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_stage(name: str, device: int):
+def build_stage(name: str, device: int, init: str = "n002"):
     """Weights, KV pool with random-filled context, block tables and input of the named workload."""
     from paper_2608_01785_b200.stage import Stage
     dims = wl.DIMS[name]
     seed = SEED[name]
     batch = wl.make_batch(name, seed)
     dev = torch.device("cuda", device)
-    weights = wl.make_weights(dims, seed, dev)
+    weights = wl.make_weights(dims, seed, dev, init)
     num_pages = wl.pages_needed(batch) + 8
     mpps = max(-(-t // 16) for t in batch.total_len())
     stage = Stage(dims, weights, num_pages, batch.n_tokens, batch.n_seqs, mpps, max(batch.total_len()), device)

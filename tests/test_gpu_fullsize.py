@@ -1,0 +1,219 @@
+"""Parity at the full sizes of the benchmark configurations, in the launch configuration bench.py times.
+
+What is asserted, per configuration:
+  * y_out and the whole KV pool are bit-identical for every SM budget of the configuration's sweep;
+  * layer-local parity (the criterion that holds at any depth): the oracle's single layer l is given the
+    GPU's own fp32 residual stream before layer l (the output of the same stage truncated to l layers)
+    and the same cache context, and its output is compared with the GPU's stream after layer l:
+    max |err| <= 2e-2 * RMS.  At config 3 the oracle evaluates K/V of every token and a sample of rows;
+  * end to end (all layers, oracle never sees a GPU value): reported, and bounded by 1.3 x the error of
+    the oracle itself run with its tensor-core operands rounded to bf16 (h, q, P, o, act) -- the
+    arithmetic-format floor no bf16-operand implementation can beat.  For config 2 that floor is about
+    2.6e-2 * RMS after 4 layers, i.e. above the 2e-2 that a single layer meets with a wide margin.
+"""
+import numpy as np
+import pytest
+import torch
+
+import bench
+from oracle.oracle import Oracle, OracleConfig, ROUND_ALL
+from paper_2608_01785_b200 import workloads as wl
+from paper_2608_01785_b200.stage import Stage
+from tests.helpers import rel_err
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+
+@pytest.fixture(scope="module")
+def orc():
+    return Oracle("f32")
+
+
+def ocfg(dims, n_layers, num_pages):
+    return OracleConfig(n_layers, dims.d_model, dims.n_q_heads, dims.n_kv_heads, dims.head_dim, dims.d_ffn, 16,
+                        num_pages, dims.rms_eps, dims.rope_base)
+
+
+def gpu_step(stage, batch, bt, x, budget, pool0):
+    stage.kv_pool.copy_(pool0)
+    y = torch.full((batch.n_tokens, stage.dims.d_model), float("nan"), device=stage.device)
+    b = stage.make_batch(batch.q_len, batch.ctx_len, bt, x, y)
+    stage.step(b, budget)
+    torch.cuda.synchronize()
+    assert stage.status() == 0
+    return y
+
+
+def truncated_output(full: Stage, n_layers: int, batch, bt, x, pool0):
+    """Residual stream after the first n_layers layers: the same stage cut to n_layers (shares weights)."""
+    d = full.dims
+    dims_l = wl.StageDims(n_layers, d.d_model, d.n_q_heads, d.n_kv_heads, d.head_dim, d.d_ffn, d.rms_eps, d.rope_base)
+    st = Stage(dims_l, full.weights[:n_layers], full.cfg.num_pages, full.cfg.max_tokens, full.cfg.max_seqs,
+               full.cfg.max_pages_per_seq, full.cfg.max_position)
+    try:
+        for s, t in enumerate(batch.total_len()):
+            st.kv_alloc(s, t)
+        y = gpu_step(st, batch, bt, x, st.sm_count, pool0[: st.kv_pool.numel()])
+    finally:
+        st.close()
+    return y
+
+
+def layer_pool_bits(pool0: torch.Tensor, dims, num_pages: int, layer: int) -> np.ndarray:
+    """Cache context of one layer as a 1-layer oracle pool (uint16 bits)."""
+    per_layer = 2 * num_pages * dims.n_kv_heads * 16 * dims.head_dim
+    return wl.bf16_bits_numpy(pool0[layer * per_layer:(layer + 1) * per_layer]).reshape(-1).copy()
+
+
+def layer_local_error(orc, stage, batch, bt, x, pool0, layer, rows=None, want_floor=False):
+    """max|err|/RMS of GPU layer `layer` against the oracle's layer fed the GPU's own input stream.
+    With want_floor also returns the same error for the oracle layer run with bf16-rounded operands."""
+    dims = stage.dims
+    T = batch.n_tokens
+    x_in = wl.to_f32_numpy(x) if layer == 0 else truncated_output(stage, layer, batch, bt, x, pool0).cpu().numpy()
+    y_gpu = truncated_output(stage, layer + 1, batch, bt, x, pool0).cpu().numpy()
+    cfg1 = ocfg(dims, 1, stage.cfg.num_pages)
+    w = {k: wl.to_f32_numpy(v) for k, v in stage.weights[layer].items()}
+    mask = None
+    if rows is not None:
+        mask = np.zeros(T, dtype=np.uint8)
+        mask[rows] = 1
+    y_ref, _ = orc.layer(cfg1, w, 0, layer_pool_bits(pool0, dims, stage.cfg.num_pages, layer), batch.q_len,
+                         batch.ctx_len, bt, x_in, row_mask=mask)
+    sel = slice(None) if rows is None else rows
+    err = rel_err(y_gpu[sel], y_ref[sel])
+    if not want_floor:
+        return err
+    orc.set_operand_rounding(ROUND_ALL)
+    try:
+        y_floor, _ = orc.layer(cfg1, w, 0, layer_pool_bits(pool0, dims, stage.cfg.num_pages, layer), batch.q_len,
+                               batch.ctx_len, bt, x_in, row_mask=mask)
+    finally:
+        orc.set_operand_rounding(0)
+    return err, rel_err(y_floor[sel], y_ref[sel])
+
+
+# ---------------------------------------------------------------- config 2 --
+def test_config2_budget_sweep_layer_local_and_end_to_end(orc):
+    name = "c2_shared"
+    stage, dims, batch, bt, x = bench.build_stage(name, 0)
+    try:
+        pool0 = stage.kv_pool.clone()
+        outs = {}
+        for budget in wl.SM_BUDGETS[name]:
+            y = gpu_step(stage, batch, bt, x, budget, pool0)
+            outs[budget] = (y.cpu().numpy(), stage.kv_pool.clone())
+        first = wl.SM_BUDGETS[name][0]
+        for budget, (y, pool) in outs.items():
+            assert np.array_equal(y, outs[first][0]), budget
+            assert torch.equal(pool, outs[first][1]), budget
+        y_gpu = outs[first][0]
+        assert np.all(np.isfinite(y_gpu))
+
+        for layer in range(dims.n_layers):
+            err = layer_local_error(orc, stage, batch, bt, x, pool0, layer)
+            print(f"config 2 layer {layer}: layer-local max|err|/RMS = {err:.2e}")
+            assert err <= TOL
+
+        cfg = ocfg(dims, dims.n_layers, stage.cfg.num_pages)
+        w_np = wl.weights_to_numpy(stage.weights)
+        pool_np = wl.bf16_bits_numpy(pool0).reshape(-1)
+        x_np = wl.to_f32_numpy(x)
+        y_ref = orc.step(cfg, w_np, pool_np.copy(), batch.q_len, batch.ctx_len, bt, x_np)
+        orc.set_operand_rounding(ROUND_ALL)
+        try:
+            y_floor = orc.step(cfg, w_np, pool_np.copy(), batch.q_len, batch.ctx_len, bt, x_np)
+        finally:
+            orc.set_operand_rounding(0)
+        err, floor = rel_err(y_gpu, y_ref), rel_err(y_floor, y_ref)
+        print(f"config 2 end to end ({dims.n_layers} layers): max|err|/RMS = {err:.2e}; "
+              f"bf16-operand floor of the oracle itself = {floor:.2e}")
+        assert err <= max(TOL, 1.3 * floor)
+    finally:
+        stage.close()
+
+
+# ---------------------------------------------------------------- config 4 --
+def test_config4_talker_end_to_end_and_corun_with_config2(orc):
+    stage_b, dims_b, batch_b, bt_b, x_b = bench.build_stage("c4_talker", 0)
+    stage_a, dims_a, batch_a, bt_a, x_a = bench.build_stage("c2_shared", 0)
+    try:
+        pool_b0, pool_a0 = stage_b.kv_pool.clone(), stage_a.kv_pool.clone()
+        # the talker alone, 12 layers end to end, at the three complementary budgets of the co-run
+        outs = {}
+        for budget in (28, 52, 74, stage_b.sm_count):
+            outs[budget] = gpu_step(stage_b, batch_b, bt_b, x_b, budget, pool_b0).cpu().numpy()
+        for y in outs.values():
+            assert np.array_equal(y, outs[28])
+        cfg = ocfg(dims_b, dims_b.n_layers, stage_b.cfg.num_pages)
+        y_ref = orc.step(cfg, wl.weights_to_numpy(stage_b.weights), wl.bf16_bits_numpy(pool_b0).reshape(-1).copy(),
+                         batch_b.q_len, batch_b.ctx_len, bt_b, wl.to_f32_numpy(x_b))
+        err = rel_err(outs[28], y_ref)
+        print(f"config 4 talker end to end (12 layers): max|err|/RMS = {err:.2e}")
+        assert err <= TOL
+        pool_b_solo = stage_b.kv_pool.clone()
+
+        # co-run: backbone on stream A with budget B, talker on stream B with 148 - B
+        ya_solo = gpu_step(stage_a, batch_a, bt_a, x_a, 120, pool_a0).cpu().numpy()
+        pool_a_solo = stage_a.kv_pool.clone()
+        sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+        dev = stage_a.device
+        for budget_a in wl.SM_BUDGETS["c4_corun"]:
+            stage_a.kv_pool.copy_(pool_a0)
+            stage_b.kv_pool.copy_(pool_b0)
+            ya = torch.empty(batch_a.n_tokens, dims_a.d_model, device=dev)
+            yb = torch.empty(batch_b.n_tokens, dims_b.d_model, device=dev)
+            ba = stage_a.make_batch(batch_a.q_len, batch_a.ctx_len, bt_a, x_a, ya)
+            bb = stage_b.make_batch(batch_b.q_len, batch_b.ctx_len, bt_b, x_b, yb)
+            torch.cuda.synchronize()
+            for _ in range(2):
+                stage_a.step(ba, budget_a, sa)
+                for _ in range(3):
+                    stage_b.step(bb, stage_a.sm_count - budget_a, sb)
+            torch.cuda.synchronize()
+            assert stage_a.status() == 0 and stage_b.status() == 0
+            assert np.array_equal(ya.cpu().numpy(), ya_solo), budget_a
+            assert np.array_equal(yb.cpu().numpy(), outs[28]), budget_a
+            assert torch.equal(stage_a.kv_pool, pool_a_solo) and torch.equal(stage_b.kv_pool, pool_b_solo)
+    finally:
+        stage_a.close()
+        stage_b.close()
+
+
+# ---------------------------------------------------------------- config 3 --
+C3_ROWS = np.unique(np.concatenate([np.array([0, 1, 15, 16, 17, 127, 128, 1023, 2046, 2047]),
+                                    np.linspace(0, 2047, 24).astype(np.int64)]))
+
+
+@pytest.mark.parametrize("init", ["n002", "depth_scaled"])
+def test_config3_budget_sweep_and_sampled_layer_local(orc, init):
+    """Config 3 states no weight distribution.  With N(0, 0.02) everywhere the 18944-wide MLP dominates the
+    layer output and the bf16 rounding of its operands alone puts a single layer at about 2e-2 * RMS (the
+    oracle with bf16-rounded operands shows the same), so that variant is held to 1.3 x that floor; with
+    the output projections drawn at std 0.02 / sqrt(2 L) the flat 2e-2 applies."""
+    name = "c3_7b"
+    stage, dims, batch, bt, x = bench.build_stage(name, 0, init)
+    try:
+        pool0 = stage.kv_pool.clone()
+        first = None
+        budgets = wl.SM_BUDGETS[name] if init == "n002" else (148, 48)
+        for budget in budgets:
+            y = gpu_step(stage, batch, bt, x, budget, pool0)
+            if first is None:
+                first = (y.clone(), stage.kv_pool.clone())
+                assert bool(torch.isfinite(y).all())
+            else:
+                assert torch.equal(y, first[0]), budget
+                assert torch.equal(stage.kv_pool, first[1]), budget
+        del first
+        T = batch.n_tokens
+        # sampled rows: spread over the 2048-token prefill chunk (first, last, tile edges) + decode rows
+        rows = np.unique(np.concatenate([C3_ROWS, np.arange(2048, T, 4)]))
+        for layer in (0, 1, 13, 27):
+            err, floor = layer_local_error(orc, stage, batch, bt, x, pool0, layer, rows=rows, want_floor=True)
+            print(f"config 3 ({init}) layer {layer}: layer-local max|err|/RMS on {len(rows)} sampled rows = {err:.2e}; "
+                  f"bf16-operand floor of the oracle itself = {floor:.2e}")
+            assert err <= (TOL if init == "depth_scaled" else max(TOL, 1.3 * floor))
+    finally:
+        stage.close()
