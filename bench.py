@@ -197,6 +197,7 @@ def main():
     ap.add_argument("--workload", default="c2_shared", choices=sorted(SEED))
     ap.add_argument("--sm-budget", type=int, default=0, help="0 = all SMs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the SM-budget sweep and the co-run section")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -279,6 +280,27 @@ def main():
     ms_e2e = timed_steps(args.steps, step_e2e) / args.steps
     e2e_value = world * T / (ms_e2e * 1e-3)
 
+    # ---- step latency vs SM budget, and the co-run with a downstream stage (rank 0, single GPU) ----
+    sweep, corun_rows = None, None
+    if rank == 0 and world == 1 and not args.no_sweep:
+        sweep = []
+        for bud in [x for x in wl.SM_BUDGETS.get(name, (148, 112, 74, 37)) if x <= stage.sm_count]:
+            fn = lambda: stage.step(b, bud, stream)
+            timed_steps(3, fn)
+            ms_b = timed_steps(args.steps, fn) / args.steps
+            sweep.append({"sm_budget": bud, "ms_per_step": ms_b, "tokens_per_s": T / (ms_b * 1e-3)})
+        for row in sweep:
+            row["speed_vs_full"] = sweep[0]["ms_per_step"] / row["ms_per_step"]
+            row["budget_fraction"] = row["sm_budget"] / sweep[0]["sm_budget"]
+        if name == "c2_shared":
+            from paper_2608_01785_b200.corun import corun
+            talker, tdims, tbatch, tbt, tx = build_stage("c4_talker", local_rank)
+            ty = torch.empty(tbatch.n_tokens, tdims.d_model, dtype=torch.float32, device=dev)
+            tb = talker.make_batch(tbatch.q_len, tbatch.ctx_len, tbt, tx, ty)
+            corun_rows = [corun(stage, b, talker, tb, bud, args.steps) for bud in wl.SM_BUDGETS["c4_corun"]]
+            assert talker.status() == 0
+            talker.close()
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -300,6 +322,18 @@ def main():
                 "avg_launch_ms": gu_avg_s * 1e3, "launches": gu_n,
                 "step_tflops": (gemm_flops + attn_flops) / (ms_step * 1e-3) / 1e12}
     kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps} for k, v in prof.items()}
+    # decode attention against HBM: K and V pages of every decode sequence once per layer
+    dec_ms, dec_n = prof["attn_decode"]
+    dec_bytes = sum((c + 1) * 2 * dims.kv_dim * 2 for q, c in zip(batch.q_len, batch.ctx_len) if q == 1)
+    decode_roofline = None
+    if dec_n:
+        gbs = dec_bytes / (dec_ms * 1e-3 / dec_n) / 1e9
+        decode_roofline = {"bound": "hbm", "kernel": "attn_decode_kernel", "achieved": gbs,
+                           "peak": peaks["hbm_gbs"] * budget / stage.sm_count, "unit": "GB/s",
+                           "frac": gbs / (peaks["hbm_gbs"] * budget / stage.sm_count),
+                           "bytes_per_launch": dec_bytes, "avg_launch_ms": dec_ms / dec_n,
+                           "note": "bytes below the 126 MB L2 are served from L2, not HBM" if dec_bytes < 126e6 else
+                                   "working set exceeds L2"}
 
     cpu = None
     if not args.no_cpu_baseline:
@@ -318,7 +352,8 @@ def main():
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e, "h2d_bytes_per_step": T * d * 2,
                     "d2h_bytes_per_step": T * d * 4},
             "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu}
+            "roofline": roofline, "roofline_decode_attention": decode_roofline, "kernels": kernels,
+            "budget_sweep": sweep, "corun": corun_rows, "cpu_baseline": cpu}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
