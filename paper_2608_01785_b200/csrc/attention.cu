@@ -5,10 +5,10 @@
 //                    the KV head are stacked as rows, so K/V are streamed once per KV head.  8 compute
 //                    warps x 16 rows, key blocks of 64 keys (4 pages) in a 5-stage ring fed by one
 //                    producer thread that runs ahead across work items.
-//   decode kernel    work item = (sequence, KV head, run of <= 512 keys); rows = the G query heads of the
-//                    single new token.  4 compute warps each take one page of every 4-page stage; their
-//                    partial (max, sum, output) triples are merged in shared memory in warp order and
-//                    written as one partial per item.  HBM-bound: 5 stages x 32 KB in flight per SM.
+//   decode kernel    work item = (sequence, KV head, run of <= 256 keys); rows = the G query heads of the
+//                    single new token.  Six autonomous warps per block, each streaming its own item's
+//                    pages through a private TMA ring and writing one partial (max, sum, output) per
+//                    item.  HBM-bound: 6 warps x 3 pages x 8 KB in flight per SM.
 //   combine kernel   merges the partials of a sequence's splits in split order.
 // Work items are listed on the host independently of the SM budget and handed out through an atomic
 // queue head; an item's result does not depend on which block ran it, and every reduction has a fixed
@@ -315,27 +315,27 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
 }
 
 // ==================================================================== decode ==
-constexpr int DC_WARPS = 4, DC_THREADS = (DC_WARPS + 1) * 32, DC_STAGES = 5;
+// Every warp is its own pipeline: it pulls a work item from the queue, streams the item's pages through
+// a private ring of DC_STAGES (K page, V page) slots that its lane 0 fills by TMA a few pages ahead, and
+// writes the item's partial (max, sum, output) straight from its registers.  There is no producer warp,
+// no "slot free" barrier (a slot is refilled by the warp that has just finished reading it) and no
+// block-level synchronisation after start-up, so an SM keeps DC_WARPS x (DC_STAGES - 1) pages in flight.
+constexpr int DC_WARPS = 6, DC_THREADS = DC_WARPS * 32, DC_STAGES = 4;
 
 template <int DH>
 constexpr int dc_smem_bytes() {
-  int b = 1024 + DC_STAGES * 8 * Geom<DH>::PAGE_BYTES + DC_WARPS * 16 * DH * 4 + DC_WARPS * 16 * 2 * 4 + 512;
+  int b = 1024 + DC_WARPS * DC_STAGES * 2 * Geom<DH>::PAGE_BYTES + 512;
   return b > kMinSmemBytes ? b : kMinSmemBytes;
 }
 
 template <int DH>
 __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid_constant__ AttnParams p) {
   using G_ = Geom<DH>;
-  constexpr int STAGE_BYTES = 8 * G_::PAGE_BYTES;
+  constexpr int SLOT_BYTES = 2 * G_::PAGE_BYTES;    // K page then V page
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* stages = smem;
-  float* sm_o = reinterpret_cast<float*>(stages + DC_STAGES * STAGE_BYTES);   // [warp][16][DH]
-  float* sm_ml = sm_o + DC_WARPS * 16 * DH;                                   // [warp][16][2]
-  uint64_t* full = reinterpret_cast<uint64_t*>(sm_ml + DC_WARPS * 16 * 2);
-  uint64_t* empty = full + DC_STAGES;
-  ItemRing* ring = reinterpret_cast<ItemRing*>(empty + DC_STAGES);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(ring + 1);
+  uint64_t* full_all = reinterpret_cast<uint64_t*>(smem + DC_WARPS * DC_STAGES * SLOT_BYTES);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(full_all + DC_WARPS * DC_STAGES);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = p.n_q_heads / p.n_kv_heads;
@@ -343,206 +343,153 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
   const float scale_log2 = kLog2e / sqrtf(float(DH));
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < DC_STAGES; ++i) {
-      mbar_init(&full[i], 1);
-      mbar_init(&empty[i], DC_WARPS);
-    }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&ring->full[i], 1);
-      mbar_init(&ring->empty[i], DC_WARPS);
-    }
+    for (int i = 0; i < DC_WARPS * DC_STAGES; ++i) mbar_init(&full_all[i], 1);
     *abort_flag = 0;
     fence_barrier_init();
     tma_prefetch_desc(&p.tm_kv);
   }
   __syncthreads();
 
-  int s = 0, rs = 0;
-  uint32_t ph = 0, rph = 0;
+  uint8_t* slots = smem + warp * DC_STAGES * SLOT_BYTES;
+  uint64_t* full = full_all + warp * DC_STAGES;
+  uint32_t issued = 0, consumed = 0;      // pages this warp has requested / finished, over all its items
 
-  if (warp == DC_WARPS) {
-    // ------------------------------------------------------------- producer --
-    if (lane == 0) {
-      for (;;) {
-        if (!mbar_wait(&ring->empty[rs], rph ^ 1, abort_flag, p.status)) break;
-        const int item = atomicAdd(p.counters + 1, 1);
-        ring->item[rs] = item;
-        mbar_arrive(&ring->full[rs]);
-        if (++rs == 2) { rs = 0; rph ^= 1; }
-        if (item >= p.n_decode_items) break;
-        const int4 it = reinterpret_cast<const int4*>(p.decode_items)[item];
-        const int seq = it.x, hk = it.y, k0 = it.z, k1 = it.w;
-        const int n_pages = (k1 - k0 + 15) >> 4;
-        const int n_iters = (n_pages + 3) >> 2;
-        const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq + (k0 >> 4);
-        bool ok = true;
-        for (int i = 0; i < n_iters; ++i) {
-          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-          const int np = min(4, n_pages - i * 4);
-          uint8_t* st = stages + s * STAGE_BYTES;
-          mbar_expect_tx(&full[s], np * 2 * G_::PAGE_BYTES);
-          for (int w = 0; w < np; ++w) {
-            const int page = table[i * 4 + w];
-            load_page<DH>(p, st + w * G_::PAGE_BYTES, &full[s], 0, page, hk);
-            load_page<DH>(p, st + (4 + w) * G_::PAGE_BYTES, &full[s], 1, page, hk);
-          }
-          if (++s == DC_STAGES) { s = 0; ph ^= 1; }
-        }
-        if (!ok) break;
-      }
+  for (;;) {
+    int item = 0;
+    if (lane == 0) item = atomicAdd(p.counters + 1, 1);
+    item = __shfl_sync(0xffffffffu, item, 0);
+    if (item >= p.n_decode_items || *abort_flag) break;
+    const int4 it = reinterpret_cast<const int4*>(p.decode_items)[item];
+    const int seq = it.x, hk = it.y, k0 = it.z, k1 = it.w;
+    const int n_pages = (k1 - k0 + 15) >> 4;
+    const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq + (k0 >> 4);
+
+    auto issue = [&](int pi) {              // lane 0: request page pi of this item
+      const uint32_t st = issued % DC_STAGES;
+      const int page = table[pi];
+      mbar_expect_tx(&full[st], SLOT_BYTES);
+      load_page<DH>(p, slots + st * SLOT_BYTES, &full[st], 0, page, hk);
+      load_page<DH>(p, slots + st * SLOT_BYTES + G_::PAGE_BYTES, &full[st], 1, page, hk);
+      ++issued;
+    };
+    if (lane == 0)
+      for (int pi = 0; pi < min(DC_STAGES - 1, n_pages); ++pi) issue(pi);
+
+    // Q fragments straight from global memory: rows = query heads hk*G .. hk*G + G - 1 of the new token
+    const int tok = p.seq_tok0[seq];
+    const __nv_bfloat16* qrow = p.q + size_t(tok) * q_dim + size_t(hk) * G * DH;
+    const int ra = lane >> 2, rb = ra + 8;
+    uint32_t qf[DH / 16][4];
+#pragma unroll
+    for (int ks = 0; ks < DH / 16; ++ks) {
+      const int c = ks * 16 + 2 * (lane & 3);
+      qf[ks][0] = ra < G ? *reinterpret_cast<const uint32_t*>(qrow + ra * DH + c) : 0u;
+      qf[ks][1] = rb < G ? *reinterpret_cast<const uint32_t*>(qrow + rb * DH + c) : 0u;
+      qf[ks][2] = ra < G ? *reinterpret_cast<const uint32_t*>(qrow + ra * DH + c + 8) : 0u;
+      qf[ks][3] = rb < G ? *reinterpret_cast<const uint32_t*>(qrow + rb * DH + c + 8) : 0u;
     }
-  } else {
-    // ------------------------------------------------------------ consumers --
-    for (;;) {
-      bool ok = mbar_wait(&ring->full[rs], rph, abort_flag, p.status);
-      if (!__all_sync(0xffffffffu, ok)) break;
-      const int item = ring->item[rs];
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&ring->empty[rs]);
-      if (++rs == 2) { rs = 0; rph ^= 1; }
-      if (item >= p.n_decode_items) break;
-      const int4 it = reinterpret_cast<const int4*>(p.decode_items)[item];
-      const int seq = it.x, hk = it.y, k0 = it.z, k1 = it.w;
-      const int n_pages = (k1 - k0 + 15) >> 4;
-      const int n_iters = (n_pages + 3) >> 2;
+    float o_acc[DH / 8][4];
+#pragma unroll
+    for (int j = 0; j < DH / 8; ++j) o_acc[j][0] = o_acc[j][1] = o_acc[j][2] = o_acc[j][3] = 0.f;
+    float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
+    bool ok = true;
 
-      // Q fragments straight from global memory: rows = query heads hk*G .. hk*G + G - 1 of the new token
-      const int tok = p.seq_tok0[seq];
-      const __nv_bfloat16* qrow = p.q + size_t(tok) * q_dim + size_t(hk) * G * DH;
-      const int ra = lane >> 2, rb = ra + 8;
-      uint32_t qf[DH / 16][4];
+    for (int pi = 0; pi < n_pages; ++pi) {
+      // the slot read in the previous iteration is free: keep DC_STAGES - 1 pages in flight
+      if (lane == 0 && pi + DC_STAGES - 1 < n_pages) issue(pi + DC_STAGES - 1);
+      const uint32_t st = consumed % DC_STAGES;
+      ok = mbar_wait(&full[st], (consumed / DC_STAGES) & 1, abort_flag, p.status);
+      if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+      ++consumed;
+      const uint32_t k_base = smem_u32(slots + st * SLOT_BYTES);
+      const uint32_t v_base = k_base + G_::PAGE_BYTES;
+      const int n_valid = k1 - (k0 + pi * 16);            // keys of this page that belong to the item
+      float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
 #pragma unroll
       for (int ks = 0; ks < DH / 16; ++ks) {
-        const int c = ks * 16 + 2 * (lane & 3);
-        qf[ks][0] = ra < G ? *reinterpret_cast<const uint32_t*>(qrow + ra * DH + c) : 0u;
-        qf[ks][1] = rb < G ? *reinterpret_cast<const uint32_t*>(qrow + rb * DH + c) : 0u;
-        qf[ks][2] = ra < G ? *reinterpret_cast<const uint32_t*>(qrow + ra * DH + c + 8) : 0u;
-        qf[ks][3] = rb < G ? *reinterpret_cast<const uint32_t*>(qrow + rb * DH + c + 8) : 0u;
+        uint32_t kf[4];
+        const int kk = (lane & 7) + (lane >> 4) * 8, cc = 2 * ks + ((lane >> 3) & 1);
+        ldmatrix_x4(kf, k_base + kv_off(kk, cc));
+        mma_bf16_16816(sc[0], qf[ks], kf[0], kf[1]);
+        mma_bf16_16816(sc[1], qf[ks], kf[2], kf[3]);
       }
-      float o_acc[DH / 8][4];
+      float mx_a = -INFINITY, mx_b = -INFINITY;
 #pragma unroll
-      for (int j = 0; j < DH / 8; ++j) o_acc[j][0] = o_acc[j][1] = o_acc[j][2] = o_acc[j][3] = 0.f;
-      float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
+      for (int j = 0; j < 2; ++j) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float v = sc[j][e] * scale_log2;
+          if (8 * j + 2 * (lane & 3) + (e & 1) >= n_valid) v = -INFINITY;
+          sc[j][e] = v;
+        }
+        mx_a = fmaxf(mx_a, fmaxf(sc[j][0], sc[j][1]));
+        mx_b = fmaxf(mx_b, fmaxf(sc[j][2], sc[j][3]));
+      }
+      mx_a = quad_max(mx_a);
+      mx_b = quad_max(mx_b);
+      const float mn_a = fmaxf(m_a, mx_a), mn_b = fmaxf(m_b, mx_b);
+      const float al_a = exp2f(m_a - mn_a), al_b = exp2f(m_b - mn_b);
+      // the running maxima settle after a few pages: skip the rescale of O when no row's maximum moved
+      const bool rescale = __any_sync(0xffffffffu, mn_a != m_a || mn_b != m_b);
+      m_a = mn_a;
+      m_b = mn_b;
+      float sum_a = 0.f, sum_b = 0.f;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        sc[j][0] = exp2f(sc[j][0] - mn_a);
+        sc[j][1] = exp2f(sc[j][1] - mn_a);
+        sc[j][2] = exp2f(sc[j][2] - mn_b);
+        sc[j][3] = exp2f(sc[j][3] - mn_b);
+        sum_a += sc[j][0] + sc[j][1];
+        sum_b += sc[j][2] + sc[j][3];
+      }
+      l_a = l_a * al_a + sum_a;
+      l_b = l_b * al_b + sum_b;
+      if (rescale) {
+#pragma unroll
+        for (int j = 0; j < DH / 8; ++j) {
+          o_acc[j][0] *= al_a; o_acc[j][1] *= al_a;
+          o_acc[j][2] *= al_b; o_acc[j][3] *= al_b;
+        }
+      }
+      uint32_t pf[4];
+      pf[0] = pack_bf16(sc[0][0], sc[0][1]);
+      pf[1] = pack_bf16(sc[0][2], sc[0][3]);
+      pf[2] = pack_bf16(sc[1][0], sc[1][1]);
+      pf[3] = pack_bf16(sc[1][2], sc[1][3]);
+#pragma unroll
+      for (int dp = 0; dp < DH / 16; ++dp) {
+        uint32_t vf[4];
+        const int kk = (lane & 7) + ((lane >> 3) & 1) * 8, cc = 2 * dp + (lane >> 4);
+        ldmatrix_x4_trans(vf, v_base + kv_off(kk, cc));
+        if (n_valid < 16) {
+          const int k = 2 * (lane & 3);
+          vf[0] = mask_v(vf[0], k, n_valid);
+          vf[1] = mask_v(vf[1], k + 8, n_valid);
+          vf[2] = mask_v(vf[2], k, n_valid);
+          vf[3] = mask_v(vf[3], k + 8, n_valid);
+        }
+        mma_bf16_16816(o_acc[2 * dp], pf, vf[0], vf[1]);
+        mma_bf16_16816(o_acc[2 * dp + 1], pf, vf[2], vf[3]);
+      }
+      __syncwarp();                         // every lane is done with this slot before lane 0 refills it
+    }
+    if (!ok) break;
 
-      for (int i = 0; i < n_iters; ++i) {
-        ok = mbar_wait(&full[s], ph, abort_flag, p.status);
-        if (!__all_sync(0xffffffffu, ok)) break;
-        const int pi = i * 4 + warp;
-        if (pi < n_pages) {
-          const uint32_t k_base = smem_u32(stages + s * STAGE_BYTES + warp * G_::PAGE_BYTES);
-          const uint32_t v_base = k_base + 4 * G_::PAGE_BYTES;
-          const int n_valid = k1 - (k0 + pi * 16);          // keys of this page that belong to the item
-          float sc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    // the item's partial: unnormalised output, running max (log2 domain) and sum, rows = query heads
+    l_a = quad_sum(l_a);
+    l_b = quad_sum(l_b);
+    float* po = p.part_o + size_t(item) * 16 * DH;
+    float* pml = p.part_ml + size_t(item) * 16 * 2;
 #pragma unroll
-          for (int ks = 0; ks < DH / 16; ++ks) {
-            uint32_t kf[4];
-            const int kk = (lane & 7) + (lane >> 4) * 8, cc = 2 * ks + ((lane >> 3) & 1);
-            ldmatrix_x4(kf, k_base + kv_off(kk, cc));
-            mma_bf16_16816(sc[0], qf[ks], kf[0], kf[1]);
-            mma_bf16_16816(sc[1], qf[ks], kf[2], kf[3]);
-          }
-          float mx_a = -INFINITY, mx_b = -INFINITY;
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              float v = sc[j][e] * scale_log2;
-              if (8 * j + 2 * (lane & 3) + (e & 1) >= n_valid) v = -INFINITY;
-              sc[j][e] = v;
-            }
-            mx_a = fmaxf(mx_a, fmaxf(sc[j][0], sc[j][1]));
-            mx_b = fmaxf(mx_b, fmaxf(sc[j][2], sc[j][3]));
-          }
-          mx_a = quad_max(mx_a);
-          mx_b = quad_max(mx_b);
-          const float mn_a = fmaxf(m_a, mx_a), mn_b = fmaxf(m_b, mx_b);
-          const float al_a = exp2f(m_a - mn_a), al_b = exp2f(m_b - mn_b);
-          m_a = mn_a;
-          m_b = mn_b;
-          float sum_a = 0.f, sum_b = 0.f;
-#pragma unroll
-          for (int j = 0; j < 2; ++j) {
-            sc[j][0] = exp2f(sc[j][0] - mn_a);
-            sc[j][1] = exp2f(sc[j][1] - mn_a);
-            sc[j][2] = exp2f(sc[j][2] - mn_b);
-            sc[j][3] = exp2f(sc[j][3] - mn_b);
-            sum_a += sc[j][0] + sc[j][1];
-            sum_b += sc[j][2] + sc[j][3];
-          }
-          l_a = l_a * al_a + sum_a;
-          l_b = l_b * al_b + sum_b;
-          uint32_t pf[4];
-          pf[0] = pack_bf16(sc[0][0], sc[0][1]);
-          pf[1] = pack_bf16(sc[0][2], sc[0][3]);
-          pf[2] = pack_bf16(sc[1][0], sc[1][1]);
-          pf[3] = pack_bf16(sc[1][2], sc[1][3]);
-#pragma unroll
-          for (int dp = 0; dp < DH / 16; ++dp) {
-            uint32_t vf[4];
-            const int kk = (lane & 7) + ((lane >> 3) & 1) * 8, cc = 2 * dp + (lane >> 4);
-            ldmatrix_x4_trans(vf, v_base + kv_off(kk, cc));
-            if (n_valid < 16) {
-              const int k = 2 * (lane & 3);
-              vf[0] = mask_v(vf[0], k, n_valid);
-              vf[1] = mask_v(vf[1], k + 8, n_valid);
-              vf[2] = mask_v(vf[2], k, n_valid);
-              vf[3] = mask_v(vf[3], k + 8, n_valid);
-            }
-#pragma unroll
-            for (int t = 0; t < 2; ++t) {
-              float* oc = o_acc[2 * dp + t];
-              oc[0] *= al_a; oc[1] *= al_a; oc[2] *= al_b; oc[3] *= al_b;
-            }
-            mma_bf16_16816(o_acc[2 * dp], pf, vf[0], vf[1]);
-            mma_bf16_16816(o_acc[2 * dp + 1], pf, vf[2], vf[3]);
-          }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty[s]);
-        if (++s == DC_STAGES) { s = 0; ph ^= 1; }
-      }
-      const bool alive = __all_sync(0xffffffffu, ok);
-      // merge the four warps' partials in warp order
-      l_a = quad_sum(l_a);
-      l_b = quad_sum(l_b);
-      float* my_o = sm_o + warp * 16 * DH;
-#pragma unroll
-      for (int j = 0; j < DH / 8; ++j) {
-        const int col = 8 * j + 2 * (lane & 3);
-        *reinterpret_cast<float2*>(my_o + ra * DH + col) = make_float2(o_acc[j][0], o_acc[j][1]);
-        *reinterpret_cast<float2*>(my_o + rb * DH + col) = make_float2(o_acc[j][2], o_acc[j][3]);
-      }
-      if ((lane & 3) == 0) {
-        sm_ml[(warp * 16 + ra) * 2] = m_a;
-        sm_ml[(warp * 16 + ra) * 2 + 1] = l_a;
-        sm_ml[(warp * 16 + rb) * 2] = m_b;
-        sm_ml[(warp * 16 + rb) * 2 + 1] = l_b;
-      }
-      named_barrier_sync(1, DC_WARPS * 32);
-      if (alive) {
-        float* po = p.part_o + size_t(item) * 16 * DH;
-        float* pml = p.part_ml + size_t(item) * 16 * 2;
-        for (int idx = threadIdx.x; idx < G * DH; idx += DC_WARPS * 32) {
-          const int r = idx / DH, e = idx % DH;
-          float mm = -INFINITY;
-#pragma unroll
-          for (int w = 0; w < DC_WARPS; ++w) mm = fmaxf(mm, sm_ml[(w * 16 + r) * 2]);
-          float acc = 0.f, ll = 0.f;
-#pragma unroll
-          for (int w = 0; w < DC_WARPS; ++w) {
-            const float f = exp2f(sm_ml[(w * 16 + r) * 2] - mm);
-            acc += f * sm_o[(w * 16 + r) * DH + e];
-            ll += f * sm_ml[(w * 16 + r) * 2 + 1];
-          }
-          po[r * DH + e] = acc;
-          if (e == 0) {
-            pml[r * 2] = mm;
-            pml[r * 2 + 1] = ll;
-          }
-        }
-      }
-      named_barrier_sync(2, DC_WARPS * 32);     // the merge buffers are free again
-      if (!alive) break;
+    for (int j = 0; j < DH / 8; ++j) {
+      const int col = 8 * j + 2 * (lane & 3);
+      if (ra < G) *reinterpret_cast<float2*>(po + ra * DH + col) = make_float2(o_acc[j][0], o_acc[j][1]);
+      if (rb < G) *reinterpret_cast<float2*>(po + rb * DH + col) = make_float2(o_acc[j][2], o_acc[j][3]);
+    }
+    if ((lane & 3) == 0) {
+      if (ra < G) { pml[ra * 2] = m_a; pml[ra * 2 + 1] = l_a; }
+      if (rb < G) { pml[rb * 2] = m_b; pml[rb * 2 + 1] = l_b; }
     }
   }
   __syncthreads();
