@@ -129,6 +129,7 @@ struct hs_stage {
   std::vector<LayerMaps> maps;
   CUtensorMap tm_h, tm_o, tm_act, tm_kv;   // operand loads
   CUtensorMap tm_q_st, tm_act_st;          // epilogue stores (box 64 x 32)
+  CUtensorMap tm_q_attn;                   // Q tiles of the prefill attention (box 64 x tokens per item)
   int32_t* pinned[kRing] = {};
   cudaEvent_t ev[kRing] = {};
   bool ev_pending[kRing] = {};
@@ -259,6 +260,8 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
             encode_2d(&s->tm_act, s->ws_dev + s->ws.act, T, F, 128);
   ok = ok && encode_2d(&s->tm_q_st, s->ws_dev + s->ws.q, T, q_dim, 32) &&
        encode_2d(&s->tm_act_st, s->ws_dev + s->ws.act, T, F, 32);
+  ok = ok && encode_2d(&s->tm_q_attn, s->ws_dev + s->ws.q, T, q_dim,
+                       prefill_tokens_per_item(cfg->n_q_heads / cfg->n_kv_heads));
   const uint64_t pool_rows = uint64_t(cfg->n_layers) * 2 * cfg->num_pages * cfg->n_kv_heads * kPage;
   ok = ok && encode_2d(&s->tm_kv, s->kv_pool, pool_rows, cfg->head_dim, 16);
   s->maps.resize(cfg->n_layers);
@@ -416,6 +419,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
 
     AttnParams a{};
     a.tm_kv = s->tm_kv;
+    a.tm_q = s->tm_q_attn;
+    a.prefill_tokens = prefill_tokens_per_item(c.n_q_heads / c.n_kv_heads);
     a.q = q; a.o = o;
     a.n_q_heads = c.n_q_heads; a.n_kv_heads = c.n_kv_heads; a.head_dim = Dh;
     a.num_pages = c.num_pages; a.max_pages_per_seq = c.max_pages_per_seq; a.layer = l;

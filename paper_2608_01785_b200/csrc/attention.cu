@@ -1,10 +1,7 @@
-// Causal GQA attention over the paged bf16 KV cache: TMA-staged K/V pages, warp-level tensor-core tiles
-// (mma.sync m16n8k16) and an fp32 online softmax in the log2 domain.
+// Decode-side causal GQA attention over the paged bf16 KV cache: TMA-staged K/V pages, warp-level
+// tensor-core tiles (mma.sync m16n8k16) and an fp32 online softmax in the log2 domain.  (The prefill
+// kernel lives in attention_prefill.cu.)
 //
-//   prefill kernel   work item = (sequence, KV head, tile of 128/G tokens); the G query heads that share
-//                    the KV head are stacked as rows, so K/V are streamed once per KV head.  8 compute
-//                    warps x 16 rows, key blocks of 64 keys (4 pages) in a 5-stage ring fed by one
-//                    producer thread that runs ahead across work items.
 //   decode kernel    work item = (sequence, KV head, run of <= 256 keys); rows = the G query heads of the
 //                    single new token.  Six autonomous warps per block, each streaming its own item's
 //                    pages through a private TMA ring and writing one partial (max, sum, output) per
@@ -62,256 +59,6 @@ __device__ __forceinline__ uint32_t mask_v(uint32_t r, int k, int n_valid) {
   if (k >= n_valid) return 0u;
   if (k + 1 >= n_valid) return r & 0x0000ffffu;
   return r;
-}
-
-// Work hand-out shared by both kernels: the producer thread owns the queue head.  It pulls the next item
-// index, publishes it to the compute warps through a two-slot ring guarded by mbarriers, and immediately
-// starts fetching that item's pages, so the pipeline never drains at an item boundary and the compute
-// warps never meet at a block-wide barrier.
-struct ItemRing {
-  uint64_t full[2], empty[2];
-  int item[2];
-};
-
-// =================================================================== prefill ==
-constexpr int PF_WARPS = 8, PF_THREADS = (PF_WARPS + 1) * 32, PF_STAGES = 5, PF_BLOCK_KEYS = 64;
-
-template <int DH>
-constexpr int pf_smem_bytes() {
-  int b = 1024 + PF_STAGES * 8 * Geom<DH>::PAGE_BYTES + 512;
-  return b > kMinSmemBytes ? b : kMinSmemBytes;
-}
-
-template <int DH>
-__global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __grid_constant__ AttnParams p) {
-  using G_ = Geom<DH>;
-  constexpr int STAGE_BYTES = 8 * G_::PAGE_BYTES;   // 4 K pages then 4 V pages
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* stages = smem;
-  uint64_t* full = reinterpret_cast<uint64_t*>(stages + PF_STAGES * STAGE_BYTES);
-  uint64_t* empty = full + PF_STAGES;
-  ItemRing* ring = reinterpret_cast<ItemRing*>(empty + PF_STAGES);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(ring + 1);
-
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int G = p.n_q_heads / p.n_kv_heads;
-  const int q_dim = p.n_q_heads * DH;
-  const float scale_log2 = kLog2e / sqrtf(float(DH));
-
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < PF_STAGES; ++i) {
-      mbar_init(&full[i], 1);
-      mbar_init(&empty[i], PF_WARPS);
-    }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&ring->full[i], 1);
-      mbar_init(&ring->empty[i], PF_WARPS);
-    }
-    *abort_flag = 0;
-    fence_barrier_init();
-    tma_prefetch_desc(&p.tm_kv);
-  }
-  __syncthreads();
-
-  int s = 0, rs = 0;          // K/V stage, item-ring slot
-  uint32_t ph = 0, rph = 0;   // and their phases
-
-  if (warp == PF_WARPS) {
-    // ------------------------------------------------------------- producer --
-    if (lane == 0) {
-      for (;;) {
-        if (!mbar_wait(&ring->empty[rs], rph ^ 1, abort_flag, p.status)) break;
-        const int item = atomicAdd(p.counters, 1);
-        ring->item[rs] = item;
-        mbar_arrive(&ring->full[rs]);
-        if (++rs == 2) { rs = 0; rph ^= 1; }
-        if (item >= p.n_prefill_items) break;
-        const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
-        const int seq = it.x, hk = it.y;
-        const int n_keys = p.seq_ctx[seq] + it.z + it.w;
-        const int n_kblocks = (n_keys + PF_BLOCK_KEYS - 1) / PF_BLOCK_KEYS;
-        const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq;
-        bool ok = true;
-        for (int kb = 0; kb < n_kblocks; ++kb) {
-          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-          const int rem = n_keys - kb * PF_BLOCK_KEYS;
-          const int np = rem >= PF_BLOCK_KEYS ? 4 : (rem + 15) >> 4;
-          uint8_t* st = stages + s * STAGE_BYTES;
-          mbar_expect_tx(&full[s], np * 2 * G_::PAGE_BYTES);
-          for (int w = 0; w < np; ++w) {
-            const int page = table[kb * 4 + w];
-            load_page<DH>(p, st + w * G_::PAGE_BYTES, &full[s], 0, page, hk);
-            load_page<DH>(p, st + (4 + w) * G_::PAGE_BYTES, &full[s], 1, page, hk);
-          }
-          if (++s == PF_STAGES) { s = 0; ph ^= 1; }
-        }
-        if (!ok) break;
-      }
-    }
-  } else {
-    // ------------------------------------------------------------ consumers --
-    for (;;) {
-      bool ok = mbar_wait(&ring->full[rs], rph, abort_flag, p.status);
-      if (!__all_sync(0xffffffffu, ok)) break;
-      const int item = ring->item[rs];
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&ring->empty[rs]);
-      if (++rs == 2) { rs = 0; rph ^= 1; }
-      if (item >= p.n_prefill_items) break;
-      const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
-      const int seq = it.x, hk = it.y, tok_begin = it.z, n_tok = it.w;
-      const int tok0 = p.seq_tok0[seq] + tok_begin;
-      const int pos0 = p.seq_ctx[seq] + tok_begin;        // position of the tile's first token
-      const int n_keys = pos0 + n_tok;
-      const int n_kblocks = (n_keys + PF_BLOCK_KEYS - 1) / PF_BLOCK_KEYS;
-      const int n_rows = n_tok * G;
-
-      // this thread's two rows: row r = (token r / G, query head hk*G + r % G); padding rows behave like
-      // the tile's last token and are never written
-      const int row_a = warp * 16 + (lane >> 2), row_b = row_a + 8;
-      const int pos_a = pos0 + min(row_a / G, n_tok - 1), pos_b = pos0 + min(row_b / G, n_tok - 1);
-      const bool warp_has_rows = warp * 16 < n_rows;
-      const int warp_min_pos = pos0 + min((warp * 16) / G, n_tok - 1);
-      const int warp_max_pos = pos0 + min((warp * 16 + 15) / G, n_tok - 1);
-
-      // Q fragments straight from global memory (written by the QKV GEMM just before; L2 hits)
-      uint32_t qf[DH / 16][4];
-      {
-        const __nv_bfloat16* qa = p.q + size_t(tok0 + min(row_a / G, n_tok - 1)) * q_dim + (hk * G + row_a % G) * DH;
-        const __nv_bfloat16* qb = p.q + size_t(tok0 + min(row_b / G, n_tok - 1)) * q_dim + (hk * G + row_b % G) * DH;
-#pragma unroll
-        for (int ks = 0; ks < DH / 16; ++ks) {
-          const int c = ks * 16 + 2 * (lane & 3);
-          qf[ks][0] = *reinterpret_cast<const uint32_t*>(qa + c);
-          qf[ks][1] = *reinterpret_cast<const uint32_t*>(qb + c);
-          qf[ks][2] = *reinterpret_cast<const uint32_t*>(qa + c + 8);
-          qf[ks][3] = *reinterpret_cast<const uint32_t*>(qb + c + 8);
-        }
-      }
-
-      float o_acc[DH / 8][4];
-#pragma unroll
-      for (int j = 0; j < DH / 8; ++j) o_acc[j][0] = o_acc[j][1] = o_acc[j][2] = o_acc[j][3] = 0.f;
-      float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.f, l_b = 0.f;
-
-      for (int kb = 0; kb < n_kblocks; ++kb) {
-        ok = mbar_wait(&full[s], ph, abort_flag, p.status);
-        if (!__all_sync(0xffffffffu, ok)) break;
-        const int key0 = kb * PF_BLOCK_KEYS;
-        if (warp_has_rows && key0 <= warp_max_pos) {
-          const uint32_t k_base = smem_u32(stages + s * STAGE_BYTES);
-          const uint32_t v_base = k_base + 4 * G_::PAGE_BYTES;
-          const int rem = n_keys - key0;
-          const int np = rem >= PF_BLOCK_KEYS ? 4 : (rem + 15) >> 4;   // pages present in this stage
-          float sc[8][4];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f;
-#pragma unroll
-          for (int ks = 0; ks < DH / 16; ++ks) {
-#pragma unroll
-            for (int pg = 0; pg < 4; ++pg) {
-              uint32_t kf[4];
-              const int kk = (lane & 7) + (lane >> 4) * 8, cc = 2 * ks + ((lane >> 3) & 1);
-              ldmatrix_x4(kf, k_base + pg * G_::PAGE_BYTES + kv_off(kk, cc));
-              mma_bf16_16816(sc[2 * pg], qf[ks], kf[0], kf[1]);
-              mma_bf16_16816(sc[2 * pg + 1], qf[ks], kf[2], kf[3]);
-            }
-          }
-          // scale, causal mask (by selection), block max
-          const bool need_mask = key0 + PF_BLOCK_KEYS - 1 > warp_min_pos;
-          float mx_a = -INFINITY, mx_b = -INFINITY;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              float v = sc[j][e] * scale_log2;
-              if (need_mask) {
-                const int key = key0 + 8 * j + 2 * (lane & 3) + (e & 1);
-                if (key > (e < 2 ? pos_a : pos_b)) v = -INFINITY;
-              }
-              sc[j][e] = v;
-            }
-            mx_a = fmaxf(mx_a, fmaxf(sc[j][0], sc[j][1]));
-            mx_b = fmaxf(mx_b, fmaxf(sc[j][2], sc[j][3]));
-          }
-          mx_a = quad_max(mx_a);
-          mx_b = quad_max(mx_b);
-          const float mn_a = fmaxf(m_a, mx_a), mn_b = fmaxf(m_b, mx_b);
-          const float al_a = exp2f(m_a - mn_a), al_b = exp2f(m_b - mn_b);
-          m_a = mn_a;
-          m_b = mn_b;
-          float sum_a = 0.f, sum_b = 0.f;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            sc[j][0] = exp2f(sc[j][0] - mn_a);
-            sc[j][1] = exp2f(sc[j][1] - mn_a);
-            sc[j][2] = exp2f(sc[j][2] - mn_b);
-            sc[j][3] = exp2f(sc[j][3] - mn_b);
-            sum_a += sc[j][0] + sc[j][1];
-            sum_b += sc[j][2] + sc[j][3];
-          }
-          l_a = l_a * al_a + sum_a;
-          l_b = l_b * al_b + sum_b;
-#pragma unroll
-          for (int j = 0; j < DH / 8; ++j) {
-            o_acc[j][0] *= al_a; o_acc[j][1] *= al_a;
-            o_acc[j][2] *= al_b; o_acc[j][3] *= al_b;
-          }
-          // O += P V, one page (16 keys) per k-step
-#pragma unroll
-          for (int pg = 0; pg < 4; ++pg) {
-            if (pg < np) {
-              uint32_t pf[4];
-              pf[0] = pack_bf16(sc[2 * pg][0], sc[2 * pg][1]);
-              pf[1] = pack_bf16(sc[2 * pg][2], sc[2 * pg][3]);
-              pf[2] = pack_bf16(sc[2 * pg + 1][0], sc[2 * pg + 1][1]);
-              pf[3] = pack_bf16(sc[2 * pg + 1][2], sc[2 * pg + 1][3]);
-              const int n_valid = rem - pg * 16;      // keys of this page that exist
-#pragma unroll
-              for (int dp = 0; dp < DH / 16; ++dp) {
-                uint32_t vf[4];
-                const int kk = (lane & 7) + ((lane >> 3) & 1) * 8, cc = 2 * dp + (lane >> 4);
-                ldmatrix_x4_trans(vf, v_base + pg * G_::PAGE_BYTES + kv_off(kk, cc));
-                if (n_valid < 16) {
-                  const int k = 2 * (lane & 3);
-                  vf[0] = mask_v(vf[0], k, n_valid);
-                  vf[1] = mask_v(vf[1], k + 8, n_valid);
-                  vf[2] = mask_v(vf[2], k, n_valid);
-                  vf[3] = mask_v(vf[3], k + 8, n_valid);
-                }
-                mma_bf16_16816(o_acc[2 * dp], pf, vf[0], vf[1]);
-                mma_bf16_16816(o_acc[2 * dp + 1], pf, vf[2], vf[3]);
-              }
-            }
-          }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty[s]);
-        if (++s == PF_STAGES) { s = 0; ph ^= 1; }
-      }
-      if (!__all_sync(0xffffffffu, ok)) break;
-      if (warp_has_rows) {
-        l_a = quad_sum(l_a);
-        l_b = quad_sum(l_b);
-        const float inv_a = 1.f / l_a, inv_b = 1.f / l_b;
-#pragma unroll
-        for (int j = 0; j < DH / 8; ++j) {
-          const int col = 8 * j + 2 * (lane & 3);
-          if (row_a < n_rows) {
-            __nv_bfloat16* dst = p.o + size_t(tok0 + row_a / G) * q_dim + (hk * G + row_a % G) * DH + col;
-            *reinterpret_cast<uint32_t*>(dst) = pack_bf16(o_acc[j][0] * inv_a, o_acc[j][1] * inv_a);
-          }
-          if (row_b < n_rows) {
-            __nv_bfloat16* dst = p.o + size_t(tok0 + row_b / G) * q_dim + (hk * G + row_b % G) * DH + col;
-            *reinterpret_cast<uint32_t*>(dst) = pack_bf16(o_acc[j][2] * inv_b, o_acc[j][3] * inv_b);
-          }
-        }
-      }
-    }
-  }
-  __syncthreads();
-  if (*abort_flag) drain_after_abort();
 }
 
 // ==================================================================== decode ==
@@ -540,22 +287,11 @@ cudaError_t set_smem(K kernel, int bytes) {
 
 cudaError_t attention_set_attributes() {
   cudaError_t e;
-  if ((e = set_smem(attn_prefill_kernel<64>, pf_smem_bytes<64>())) != cudaSuccess) return e;
-  if ((e = set_smem(attn_prefill_kernel<128>, pf_smem_bytes<128>())) != cudaSuccess) return e;
+  if ((e = attention_prefill_set_attributes()) != cudaSuccess) return e;
   if ((e = set_smem(attn_decode_kernel<64>, dc_smem_bytes<64>())) != cudaSuccess) return e;
   if ((e = set_smem(attn_decode_kernel<128>, dc_smem_bytes<128>())) != cudaSuccess) return e;
   if ((e = set_smem(attn_combine_kernel<64>, kMinSmemBytes)) != cudaSuccess) return e;
   return set_smem(attn_combine_kernel<128>, kMinSmemBytes);
-}
-
-cudaError_t launch_attention_prefill(const AttnParams& p, int sm_budget, cudaStream_t stream) {
-  if (p.n_prefill_items <= 0) return cudaSuccess;
-  const int grid = p.n_prefill_items < sm_budget ? p.n_prefill_items : sm_budget;
-  if (p.head_dim == 128)
-    attn_prefill_kernel<128><<<grid, PF_THREADS, pf_smem_bytes<128>(), stream>>>(p);
-  else
-    attn_prefill_kernel<64><<<grid, PF_THREADS, pf_smem_bytes<64>(), stream>>>(p);
-  return cudaGetLastError();
 }
 
 cudaError_t launch_attention_decode(const AttnParams& p, int sm_budget, cudaStream_t stream) {

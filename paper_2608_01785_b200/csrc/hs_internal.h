@@ -16,8 +16,13 @@ constexpr int kPrefillRows = 128;        // (token, query head of one KV head) r
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-// Tokens per prefill work item: the G query heads of one KV head are stacked as rows of the tile.
-inline int prefill_tokens_per_item(int G) { return kPrefillRows / G; }
+// Tokens per prefill work item: the G query heads of one KV head are stacked head-major as rows of the
+// 128-row tile (row = head * tokens + token).  A multiple of 8 so that every head's rows start on a
+// 1024-byte boundary of the 128-byte-swizzled shared-memory tile.
+inline int prefill_tokens_per_item(int G) {
+  const int t = (kPrefillRows / G) & ~7;
+  return t < 8 ? 8 : t;
+}
 
 // ------------------------------------------------------------------ pages --
 // LIFO page allocator: pops on a fresh pool give 0, 1, 2, ...; a freed sequence returns its pages in

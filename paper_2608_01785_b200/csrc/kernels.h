@@ -63,6 +63,8 @@ cudaError_t norm_set_attributes();
 // -------------------------------------------------------------- attention --
 struct AttnParams {
   CUtensorMap tm_kv;               // whole pool as rows of Dh bf16: box 64 x 16, 128-byte swizzle
+  CUtensorMap tm_q;                // q [max_tokens, q_dim]: box 64 x prefill_tokens, 128-byte swizzle
+  int prefill_tokens;              // tokens per prefill work item
   const __nv_bfloat16* q;          // [T, q_dim] (after RoPE)
   __nv_bfloat16* o;                // [T, q_dim]
   int n_q_heads, n_kv_heads, head_dim, num_pages, max_pages_per_seq, layer;
@@ -84,5 +86,6 @@ cudaError_t launch_attention_prefill(const AttnParams& p, int sm_budget, cudaStr
 cudaError_t launch_attention_decode(const AttnParams& p, int sm_budget, cudaStream_t stream);
 cudaError_t launch_attention_combine(const AttnParams& p, int sm_budget, cudaStream_t stream);
 cudaError_t attention_set_attributes();
+cudaError_t attention_prefill_set_attributes();
 
 }  // namespace hs
