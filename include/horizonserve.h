@@ -115,9 +115,9 @@ typedef struct {
 /*
  * Sizes of the two caller-provided device buffers.
  *  KV pool: bf16 [n_layers][2 (K,V)][num_pages][n_kv_heads][16][head_dim]; K is stored after RoPE.
- *           One (page, head) block is 16*head_dim*2 contiguous bytes.  Must be 1024-byte aligned.
+ *           One (page, head) block is 16*head_dim*2 contiguous bytes.  Must be 256-byte aligned (what cudaMalloc gives).
  *  Workspace: private scratch of the stage (activations, RoPE table, step metadata, attention
- *           partials).  Must be 1024-byte aligned.  Its contents are meaningless to the caller.
+ *           partials).  Must be 256-byte aligned (what cudaMalloc gives).  Its contents are meaningless to the caller.
  * Both return 0 for an invalid configuration.
  */
 size_t hs_kv_pool_bytes(const hs_stage_config_t *cfg);

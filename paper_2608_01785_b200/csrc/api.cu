@@ -206,7 +206,7 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
   const bool host_only = cfg->device < 0;
   if (!host_only) {
     if (!layers || !kv_pool_dev || !workspace_dev) return HS_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(kv_pool_dev) & 1023) || (reinterpret_cast<uintptr_t>(workspace_dev) & 1023))
+    if ((reinterpret_cast<uintptr_t>(kv_pool_dev) & 255) || (reinterpret_cast<uintptr_t>(workspace_dev) & 255))
       return HS_ERR_INVALID_ARG;
     for (int l = 0; l < cfg->n_layers; ++l) {
       const void* ptrs[9] = {layers[l].g_attn, layers[l].w_q,    layers[l].w_k,  layers[l].w_v,   layers[l].w_o,
