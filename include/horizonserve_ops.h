@@ -54,6 +54,44 @@ hs_status_t hs_stage_debug_buffer(hs_stage_t *stage, const char *name, void **de
 hs_status_t hs_stage_profile_enable(hs_stage_t *stage, int32_t enable);
 hs_status_t hs_stage_profile_read(hs_stage_t *stage, float *ms, int32_t *launches);
 
+/*
+ * Decode attention for callers that cannot allocate device memory.  (The paper has no counterpart
+ * to this call: it is a packaging variant of the decode-attention kernels of hs_stage_step.)
+ *
+ * Who needs it: a process that gave all free HBM to its KV pool at start-up, or a component that only
+ * receives device pointers from its host runtime, cannot provide the scratch workspace that the stage
+ * API expects -- an allocation at that point fails or stalls every stream of the GPU.  Here the
+ * scratch (split-KV partials, work-queue head, the call's integer metadata, about 4.3 MB) is a fixed
+ * array inside the library image; every GPU that loads the library carries it until the process
+ * ends.  The call itself allocates nothing, on the device or the host, directly or through a library.
+ *
+ * Computes, for each of n_seqs sequences, o[s] = softmax(q[s] K^T / sqrt(head_dim)) V over keys
+ * 0 .. kv_len[s]-1 of that sequence (grouped-query: query head h reads KV head h / (n_q_heads /
+ * n_kv_heads)), exactly as the decode part of hs_stage_step does.
+ *   q_dev, o_dev   device bf16 [n_seqs, n_q_heads * head_dim], 16-byte aligned; q is used as given
+ *                  (apply RoPE before); o is overwritten.
+ *   kv_pool_dev    device bf16 pool in the layout of hs_kv_pool_bytes, 256-byte aligned; `layer`
+ *                  selects the layer, n_layers / num_pages describe the pool.
+ *   kv_len         host [n_seqs], >= 1; block_tables: host [n_seqs * max_pages_per_seq].
+ * Limits (the size of the fixed scratch): n_seqs <= HS_NOALLOC_MAX_SEQS, max_pages_per_seq <=
+ * HS_NOALLOC_MAX_PAGES_PER_SEQ, and sum over sequences of n_kv_heads * ceil(kv_len / 256) <=
+ * HS_NOALLOC_MAX_ITEMS; anything larger is refused with HS_ERR_UNSUPPORTED_SHAPE and nothing runs.
+ * The first call on a device resolves the scratch array's device address and configures the kernels;
+ * make that first call before any stream capture begins.  All calls share the one scratch area: it
+ * keeps the previous call's contents, the parts that must start from zero are cleared by each call,
+ * and two calls whose kernels can overlap on the GPU (different streams, no ordering between them)
+ * race on it -- order them.  The work is enqueued on cuda_stream; the call does not synchronise.
+ * Errors: INVALID_ARG, INVALID_BUDGET, UNSUPPORTED_SHAPE, BAD_BLOCK_TABLE, CUDA.
+ */
+#define HS_NOALLOC_MAX_SEQS 64
+#define HS_NOALLOC_MAX_PAGES_PER_SEQ 256
+#define HS_NOALLOC_MAX_ITEMS 512
+hs_status_t hs_op_decode_attention_noalloc(const void *q_dev, const void *kv_pool_dev, int32_t n_layers, int32_t layer,
+                                           int32_t num_pages, int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                           int32_t n_seqs, const int32_t *kv_len, const int32_t *block_tables,
+                                           int32_t max_pages_per_seq, void *o_dev, int32_t sm_budget,
+                                           void *cuda_stream);
+
 #if defined(__GNUC__)
 #pragma GCC visibility pop
 #endif

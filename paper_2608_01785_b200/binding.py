@@ -22,7 +22,7 @@ HS_OK, HS_ERR_INVALID_ARG, HS_ERR_INVALID_BUDGET, HS_ERR_UNSUPPORTED_SHAPE, HS_E
 EXPORTS = ("hs_status_str", "hs_kv_pool_bytes", "hs_workspace_bytes", "hs_stage_create", "hs_stage_destroy",
            "hs_kv_alloc", "hs_kv_free", "hs_kv_free_pages", "hs_stage_plan", "hs_stage_step", "hs_stage_status",
            "hs_stage_sm_count", "hs_op_gemm_bf16", "hs_stage_debug_buffer", "hs_stage_profile_enable",
-           "hs_stage_profile_read", "hs_last_error")
+           "hs_stage_profile_read", "hs_last_error", "hs_op_decode_attention_noalloc")
 PROFILE_CLASSES = ("rmsnorm", "gemm_qkv", "attn_prefill", "attn_decode", "attn_combine", "gemm_out", "gemm_gateup",
                    "gemm_down")
 
@@ -89,6 +89,8 @@ def lib() -> C.CDLL:
                                       C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
         l.hs_stage_debug_buffer.argtypes = [C.c_void_p, C.c_char_p, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
         l.hs_last_error.restype = C.c_char_p
+        l.hs_op_decode_attention_noalloc.argtypes = [C.c_void_p, C.c_void_p] + [C.c_int32] * 7 + \
+            [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p]
         l.hs_stage_profile_enable.argtypes = [C.c_void_p, C.c_int32]
         l.hs_stage_profile_read.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = l
@@ -220,5 +222,20 @@ def hs_stage_profile_read(stage: int):
     n = np.zeros(len(PROFILE_CLASSES), dtype=np.int32)
     st = lib().hs_stage_profile_read(C.c_void_p(stage), ms.ctypes.data, n.ctypes.data)
     if st != HS_OK:
-        raise HsError(st, "hs_stage_profile_read", "hs_last_error")
+        raise HsError(st, "hs_stage_profile_read", "hs_last_error", "hs_op_decode_attention_noalloc")
     return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(PROFILE_CLASSES)}
+
+
+def hs_op_decode_attention_noalloc(q_ptr: int, kv_pool_ptr: int, n_layers: int, layer: int, num_pages: int,
+                                   n_q_heads: int, n_kv_heads: int, head_dim: int, kv_len, block_tables,
+                                   o_ptr: int, sm_budget: int, cuda_stream: int = 0) -> None:
+    """Decode attention on the library's built-in scratch area (for callers that cannot allocate device
+    memory).  kv_len: int32 [n_seqs] keys per sequence; block_tables: int32 [n_seqs, max_pages_per_seq]."""
+    kv_len = np.ascontiguousarray(kv_len, dtype=np.int32)
+    bt = np.ascontiguousarray(block_tables, dtype=np.int32)
+    st = lib().hs_op_decode_attention_noalloc(C.c_void_p(q_ptr), C.c_void_p(kv_pool_ptr), n_layers, layer, num_pages,
+                                              n_q_heads, n_kv_heads, head_dim, len(kv_len), kv_len.ctypes.data,
+                                              bt.ctypes.data, bt.shape[1], C.c_void_p(o_ptr), sm_budget,
+                                              C.c_void_p(cuda_stream))
+    if st != HS_OK:
+        raise HsError(st, "hs_op_decode_attention_noalloc")
