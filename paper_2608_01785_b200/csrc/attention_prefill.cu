@@ -26,7 +26,7 @@ namespace hs {
 namespace {
 
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int PF_THREADS = 192, PF_STAGES = 4, PF_KEYS = 64;
+constexpr int PF_THREADS = 192, PF_STAGES = 3, PF_KEYS = 64;
 constexpr int TMEM_COLS = 512;
 
 template <int DH>
@@ -36,13 +36,13 @@ struct Geom {
   static constexpr int KV_BYTES = HALVES * 8192;        // K (or V) of one stage: [half][4 pages][16 keys][128 B]
   static constexpr int STAGE_BYTES = 2 * KV_BYTES;
   static constexpr int P_BYTES = 16384;                 // [128 rows][64 keys] bf16
-  static constexpr int SMEM = 1024 + Q_BYTES + PF_STAGES * STAGE_BYTES + 2 * P_BYTES + 512;
+  static constexpr int SMEM = 1024 + 2 * Q_BYTES + PF_STAGES * STAGE_BYTES + 2 * P_BYTES + 512;
   // tensor-memory columns
   static constexpr int S0 = 0, O0 = 128;                // S buffers at 0 / 64, O_blk buffers at 128 / 128 + DH
 };
 
 struct Barriers {
-  uint64_t q_full, q_empty;
+  uint64_t q_full[2], q_empty[2];
   uint64_t kv_full[PF_STAGES], kv_empty[PF_STAGES];
   uint64_t s_full[2], s_empty[2], p_full[2], o_full[2], o_empty[2];
   uint64_t ring_full[2], ring_empty[2];
@@ -53,6 +53,12 @@ struct Barriers {
 
 __device__ __forceinline__ int pool_row(const AttnParams& p, int kv, int page, int hk) {
   return (((p.layer * 2 + kv) * p.num_pages + page) * p.n_kv_heads + hk) * 16;
+}
+// 2^x on the special-function unit (ex2.approx: exact 0 for -inf, relative error about 2^-22).
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 // MN-major bf16 operand with the 128-byte swizzle: atoms of 64 (MN, contiguous) x 8 (K) elements;
 // lbo = bytes between atoms along MN, sbo = bytes between atoms along K.
@@ -72,7 +78,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* q_smem = smem;
-  uint8_t* stages = q_smem + G_::Q_BYTES;
+  uint8_t* stages = q_smem + 2 * G_::Q_BYTES;       // two Q tiles: the next item's tile loads early
   uint8_t* p_smem = stages + PF_STAGES * G_::STAGE_BYTES;
   Barriers* bar = reinterpret_cast<Barriers*>(p_smem + 2 * G_::P_BYTES);
   volatile int* abort_flag = &bar->abort_flag;
@@ -84,8 +90,10 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
   const float scale_log2 = kLog2e / sqrtf(float(DH));
 
   if (threadIdx.x == 0) {
-    mbar_init(&bar->q_full, 1);
-    mbar_init(&bar->q_empty, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bar->q_full[i], 1);
+      mbar_init(&bar->q_empty[i], 1);
+    }
     for (int i = 0; i < PF_STAGES; ++i) {
       mbar_init(&bar->kv_full[i], 1);
       mbar_init(&bar->kv_empty[i], 1);
@@ -135,11 +143,13 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         const int n_kblocks = (n_keys + PF_KEYS - 1) / PF_KEYS;
         const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq;
         // Q tile: one box of Mt token rows x 64 columns per (head, half)
-        if (!mbar_wait(&bar->q_empty, (n_items_seen & 1) ^ 1, abort_flag, p.status)) break;
-        mbar_expect_tx(&bar->q_full, G * G_::HALVES * Mt * 128);
+        const uint32_t qb = n_items_seen & 1;
+        if (!mbar_wait(&bar->q_empty[qb], ((n_items_seen >> 1) & 1) ^ 1, abort_flag, p.status)) break;
+        mbar_expect_tx(&bar->q_full[qb], G * G_::HALVES * Mt * 128);
         for (int g = 0; g < G; ++g)
           for (int h = 0; h < G_::HALVES; ++h)
-            tma_load_2d(q_smem + h * 16384 + g * Mt * 128, &p.tm_q, &bar->q_full, (hk * G + g) * DH + h * 64, tok0);
+            tma_load_2d(q_smem + qb * G_::Q_BYTES + h * 16384 + g * Mt * 128, &p.tm_q, &bar->q_full[qb],
+                        (hk * G + g) * DH + h * 64, tok0);
         ++n_items_seen;
         bool ok = true;
         for (int kb = 0; kb < n_kblocks; ++kb, ++gblk) {
@@ -193,7 +203,8 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
         const int n_keys = p.seq_ctx[it.x] + it.z + it.w;
         const int n_kblocks = (n_keys + PF_KEYS - 1) / PF_KEYS;
-        if (!mbar_wait(&bar->q_full, n_items_seen & 1, abort_flag, p.status)) break;
+        const uint32_t qb = n_items_seen & 1;
+        if (!mbar_wait(&bar->q_full[qb], (n_items_seen >> 1) & 1, abort_flag, p.status)) break;
         ++n_items_seen;
         bool ok = true;
         for (int j = 0; j < n_kblocks && ok; ++j, ++gblk) {
@@ -204,12 +215,12 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
           const uint32_t k_addr = st_addr + s * G_::STAGE_BYTES;
 #pragma unroll
           for (int ks = 0; ks < DH / 16; ++ks) {
-            const uint64_t a = umma_desc_kmajor_sw128(q_addr + (ks >> 2) * 16384) + 2 * (ks & 3);
+            const uint64_t a = umma_desc_kmajor_sw128(q_addr + qb * G_::Q_BYTES + (ks >> 2) * 16384) + 2 * (ks & 3);
             const uint64_t b = umma_desc_kmajor_sw128(k_addr + (ks >> 2) * 8192) + 2 * (ks & 3);
             umma_bf16(tmem + G_::S0 + buf * PF_KEYS, a, b, idesc_s, ks != 0);
           }
           umma_commit(&bar->s_full[buf]);
-          if (j == n_kblocks - 1) umma_commit(&bar->q_empty);     // Q may be replaced once these are done
+          if (j == n_kblocks - 1) umma_commit(&bar->q_empty[qb]);   // this Q tile may be replaced once these are done
           if (j > 0) ok = issue_pv(gblk - 1);                      // overlaps the softmax of block j
         }
         if (!ok || !issue_pv(gblk - 1)) break;
@@ -241,7 +252,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
 #pragma unroll
       for (int e = 0; e < DH; ++e) o_reg[e] = 0.f;
       float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
-      uint32_t sreg[32];
+      uint32_t sreg[32], sreg2[32];
 
       // o = o * alpha + O_blk of block b
       auto correct = [&](uint32_t b, float alpha) -> bool {
@@ -250,11 +261,15 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         if (!__all_sync(0xffffffffu, w)) return false;
         tc_fence_after_sync();
 #pragma unroll
-        for (int c = 0; c < DH / 32; ++c) {
-          tmem_ld32(tmem + lane_base + G_::O0 + buf * DH + c * 32, sreg);
+        for (int c = 0; c < DH / 64; ++c) {
+          tmem_ld32(tmem + lane_base + G_::O0 + buf * DH + c * 64, sreg);
+          tmem_ld32(tmem + lane_base + G_::O0 + buf * DH + c * 64 + 32, sreg2);
           tmem_ld_wait();
 #pragma unroll
-          for (int e = 0; e < 32; ++e) o_reg[c * 32 + e] = o_reg[c * 32 + e] * alpha + __uint_as_float(sreg[e]);
+          for (int e = 0; e < 32; ++e) {
+            o_reg[c * 64 + e] = fmaf(o_reg[c * 64 + e], alpha, __uint_as_float(sreg[e]));
+            o_reg[c * 64 + 32 + e] = fmaf(o_reg[c * 64 + 32 + e], alpha, __uint_as_float(sreg2[e]));
+          }
         }
         tc_fence_before_sync();
         mbar_arrive(&bar->o_empty[buf]);
@@ -267,25 +282,26 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
         tc_fence_after_sync();
         const int key0 = j * PF_KEYS;
-        const bool need_mask = key0 + PF_KEYS - 1 > pos0;      // some row of the tile may not see every key
-        float sv[PF_KEYS];
-        float mx = -INFINITY;
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          tmem_ld32(tmem + lane_base + G_::S0 + buf * PF_KEYS + c * 32, sreg);
-          tmem_ld_wait();
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            float v = __uint_as_float(sreg[e]) * scale_log2;
-            if (need_mask && key0 + c * 32 + e > pos) v = -INFINITY;
-            sv[c * 32 + e] = v;
-            mx = fmaxf(mx, v);
-          }
-        }
+        // both halves of the row in flight, one wait
+        tmem_ld32(tmem + lane_base + G_::S0 + buf * PF_KEYS, sreg);
+        tmem_ld32(tmem + lane_base + G_::S0 + buf * PF_KEYS + 32, sreg2);
+        tmem_ld_wait();
         tc_fence_before_sync();
         mbar_arrive(&bar->s_empty[buf]);
+        if (key0 + PF_KEYS - 1 > pos) {               // this row does not see every key of the block
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            if (key0 + e > pos) sreg[e] = 0xff800000u;          // -inf
+            if (key0 + 32 + e > pos) sreg2[e] = 0xff800000u;
+          }
+        }
+        float mx = -INFINITY;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) mx = fmaxf(mx, fmaxf(__uint_as_float(sreg[e]), __uint_as_float(sreg2[e])));
+        // running max kept on the raw scores; the 1/sqrt(Dh) * log2(e) scale is folded into the exponent
         const float m_new = fmaxf(m_run, mx);
-        const float alpha = exp2f(m_run - m_new);
+        const float alpha = fast_exp2((m_run - m_new) * scale_log2);
+        const float neg_ms = -m_new * scale_log2;
         m_run = m_new;
         float sum = 0.f;
         uint8_t* prow = p_smem + buf * G_::P_BYTES + r * 128;
@@ -294,7 +310,8 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
           float e8[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
-            e8[e] = exp2f(sv[u * 8 + e] - m_new);
+            const uint32_t raw = u < 4 ? sreg[u * 8 + e] : sreg2[(u - 4) * 8 + e];
+            e8[e] = fast_exp2(fmaf(__uint_as_float(raw), scale_log2, neg_ms));
             sum += e8[e];
           }
           uint4 w;
