@@ -450,6 +450,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     go.M = T; go.N = d; go.K = q_dim;
     go.mode = kGemmResid;
     go.tm_out = tm_y; go.accumulate = 1;
+    go.bn = gemm_pick_bn(T, d, s->sm_count);
     go.status = status;
     { LaunchTimer t(s, 5, stream); where = "out-proj gemm"; e = launch_gemm(go, sm_budget, stream); }
     if (e != cudaSuccess) break;
@@ -475,6 +476,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gd.M = T; gd.N = d; gd.K = F;
     gd.mode = kGemmResid;
     gd.tm_out = tm_y; gd.accumulate = 1;
+    gd.bn = gemm_pick_bn(T, d, s->sm_count);
     gd.status = status;
     { LaunchTimer t(s, 7, stream); where = "down gemm"; e = launch_gemm(gd, sm_budget, stream); }
     if (e != cudaSuccess) break;
@@ -557,6 +559,7 @@ hs_status_t hs_op_gemm_bf16(const void* a, const void* w, const float* resid, fl
   g.M = M; g.N = N; g.K = K;
   g.mode = kGemmResid;
   g.accumulate = resid != nullptr;
+  g.bn = gemm_pick_bn(M, N, prop.multiProcessorCount);
   // the kernel adds into `out`: a residual that lives elsewhere is copied there first
   if (resid && resid != out &&
       cudaMemcpyAsync(out, resid, size_t(M) * N * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)

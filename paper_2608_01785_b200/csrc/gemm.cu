@@ -32,9 +32,17 @@ constexpr int GEMM_SMEM = 1024 + STAGES * STAGE_BYTES + 4 * EPI_WARP_BYTES + 256
 static_assert(GEMM_SMEM <= 227 * 1024, "fits one SM");
 static_assert(GEMM_SMEM >= kMinSmemBytes, "one block per SM");
 
+// Output-tile width: 256 virtual columns, except in Resid mode where the launcher picks p.bn (a multiple
+// of 32 in [128, 256]) from the problem shape so that the tile count fills whole waves of SMs.
+__host__ __device__ __forceinline__ int gemm_n_tiles(const GemmParams& p) {
+  if (p.mode == kGemmGateUp) return (p.N + 127) / 128;
+  const int bn = p.mode == kGemmResid ? p.bn : BN;
+  return (p.N + bn - 1) / bn;
+}
+
 struct BSource { int map, row; };
 __device__ __forceinline__ BSource b_source(const GemmParams& p, int n_tile, int half) {
-  if (p.mode == kGemmResid) return {0, n_tile * BN + half * 128};
+  if (p.mode == kGemmResid) return {0, n_tile * p.bn + half * 128};
   if (p.mode == kGemmGateUp) return {half, n_tile * 128};
   int v = n_tile * BN + half * 128;
   if (v < p.q_dim) return {0, v};
@@ -100,7 +108,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_m_tiles = (p.M + BM - 1) / BM;
-  const int n_n_tiles = p.mode == kGemmGateUp ? (p.N + 127) / 128 : (p.N + BN - 1) / BN;
+  const int n_n_tiles = gemm_n_tiles(p);
   const int n_tiles = n_m_tiles * n_n_tiles;
   const int k_blocks = (p.K + BK - 1) / BK;
 
@@ -134,16 +142,17 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
+      const bool two_halves = p.mode != kGemmResid || p.bn > 128;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
         const int m = tile % n_m_tiles, n = tile / n_m_tiles;
         const BSource b0 = b_source(p, n, 0), b1 = b_source(p, n, 1);
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status)) { ok = false; break; }
           uint8_t* st = smem + s * STAGE_BYTES;
-          mbar_expect_tx(&full[s], STAGE_BYTES);
+          mbar_expect_tx(&full[s], two_halves ? STAGE_BYTES : A_BYTES + BH_BYTES);
           tma_load_2d(st, &p.tm_a, &full[s], kb * BK, m * BM);
           tma_load_2d(st + A_BYTES, &p.tm_b[b0.map], &full[s], kb * BK, b0.row);
-          tma_load_2d(st + A_BYTES + BH_BYTES, &p.tm_b[b1.map], &full[s], kb * BK, b1.row);
+          if (two_halves) tma_load_2d(st + A_BYTES + BH_BYTES, &p.tm_b[b1.map], &full[s], kb * BK, b1.row);
           if (++s == STAGES) { s = 0; ph ^= 1; }
         }
       }
@@ -151,7 +160,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
   } else if (warp == 1) {
     // --------------------------------------------------------- MMA issuer --
     if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_bf16_f32(BM, BN);
+      const uint32_t idesc = umma_idesc_bf16_f32(BM, p.mode == kGemmResid ? p.bn : BN);
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
       bool ok = true;
@@ -198,8 +207,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
       const int row_base = m * BM + quarter * 32;          // first row of this warp's 32
 
       if (p.mode == kGemmResid) {
-        for (int c = 0; c < BN / 32; ++c) {
-          const int col0 = n * BN + c * 32;
+        for (int c = 0; c < p.bn / 32; ++c) {
+          const int col0 = n * p.bn + c * 32;
           if (col0 >= p.N) break;
           tmem_ld32(taddr + c * 32, r0);
           tmem_ld_wait();
@@ -335,9 +344,30 @@ cudaError_t gemm_set_attributes() {
   return cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
 }
 
+int gemm_pick_bn(int M, int N, int sm_count) {
+  // Time of a launch ~ waves x time of one tile.  A tile's MMA work is proportional to its width, but the
+  // operand feed is not (the 128-row A tile is fetched whatever the width, and narrow tiles leave less
+  // time to hide the fetch): measured on B200, a 224-wide tile takes 0.95 and a 128-wide tile 0.80 of a
+  // 256-wide one, i.e. about 0.6 + 0.4 * bn / 256.  The choice depends on the shape and on the device's
+  // SM count only -- never on the SM budget -- so that the same tiles are computed at every budget.
+  const int m_tiles = (M + BM - 1) / BM;
+  int best = BN;
+  double best_cost = 1e30;
+  for (int bn = 256; bn >= 128; bn -= 32) {
+    const int tiles = m_tiles * ((N + bn - 1) / bn);
+    const int waves = (tiles + sm_count - 1) / sm_count;
+    const double cost = double(waves) * (0.6 + 0.4 * bn / 256.0);
+    if (cost < best_cost - 1e-9) {
+      best_cost = cost;
+      best = bn;
+    }
+  }
+  return best;
+}
+
 cudaError_t launch_gemm(const GemmParams& p, int sm_budget, cudaStream_t stream) {
   const int n_m_tiles = (p.M + BM - 1) / BM;
-  const int n_n_tiles = p.mode == kGemmGateUp ? (p.N + 127) / 128 : (p.N + BN - 1) / BN;
+  const int n_n_tiles = gemm_n_tiles(p);
   const int n_tiles = n_m_tiles * n_n_tiles;
   if (n_tiles <= 0) return cudaSuccess;
   const int grid = n_tiles < sm_budget ? n_tiles : sm_budget;

@@ -30,6 +30,7 @@ struct GemmParams {
   // Resid
   CUtensorMap tm_out;        // fp32 [M, N], box 32 x 32, 128-byte swizzle (rows past M are clipped)
   int accumulate;            // 1: out += A W^T (the residual add), 0: out = A W^T
+  int bn;                    // tile width of this launch (gemm_pick_bn); 256 when unused
   // Qkv
   int q_dim, kv_dim, head_dim, n_kv_heads;
   CUtensorMap tm_q;          // bf16 q [M, q_dim], box 64 x 32, 128-byte swizzle
@@ -44,6 +45,8 @@ struct GemmParams {
 };
 cudaError_t launch_gemm(const GemmParams& p, int sm_budget, cudaStream_t stream);
 cudaError_t gemm_set_attributes();
+// Tile width for a Resid-mode GEMM of this shape on a device with sm_count SMs (budget independent).
+int gemm_pick_bn(int M, int N, int sm_count);
 
 // ---------------------------------------------------------------- RMSNorm --
 // h[t,:] = bf16(x[t,:] * rsqrt(mean(x[t,:]^2) + eps) * g).  x comes either as bf16 (x_bf16, first layer;
