@@ -436,12 +436,11 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     a.part_o = reinterpret_cast<float*>(s->ws_dev + s->ws.part_o);
     a.part_ml = reinterpret_cast<float*>(s->ws_dev + s->ws.part_ml);
     a.counters = meta + s->ml.counters + 2 * l;
+    a.group_done = meta + s->ml.group_done;
     a.status = status;
     if (a.n_prefill_items > 0) { LaunchTimer t(s, 2, stream); where = "prefill attention"; e = launch_attention_prefill(a, sm_budget, stream); }
     if (e != cudaSuccess) break;
     if (a.n_decode_items > 0) { LaunchTimer t(s, 3, stream); where = "decode attention"; e = launch_attention_decode(a, sm_budget, stream); }
-    if (e != cudaSuccess) break;
-    if (a.n_decode_rows > 0) { LaunchTimer t(s, 4, stream); where = "decode combine"; e = launch_attention_combine(a, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
     GemmParams go{};

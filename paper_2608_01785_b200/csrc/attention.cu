@@ -6,7 +6,8 @@
 //                    single new token.  Six autonomous warps per block, each streaming its own item's
 //                    pages through a private TMA ring and writing one partial (max, sum, output) per
 //                    item.  HBM-bound: 6 warps x 3 pages x 8 KB in flight per SM.
-//   combine kernel   merges the partials of a sequence's splits in split order.
+//                    The warp that finishes the last split of a (sequence, KV head) merges that group's
+//                    partials in split order (a group with a single split writes its output directly).
 // Work items are listed on the host independently of the SM budget and handed out through an atomic
 // queue head; an item's result does not depend on which block ran it, and every reduction has a fixed
 // order, so outputs are bit-identical across budgets.
@@ -107,7 +108,9 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
     item = __shfl_sync(0xffffffffu, item, 0);
     if (item >= p.n_decode_items || *abort_flag) break;
     const int4 it = reinterpret_cast<const int4*>(p.decode_items)[item];
-    const int seq = it.x, hk = it.y, k0 = it.z, k1 = it.w;
+    const int drow = it.x, hk = it.y, k0 = it.z, k1 = it.w;
+    const int4 dr = reinterpret_cast<const int4*>(p.decode_rows)[drow];   // {seq, token row, first item, splits}
+    const int seq = dr.x, tok = dr.y, splits = dr.w;
     const int n_pages = (k1 - k0 + 15) >> 4;
     const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq + (k0 >> 4);
 
@@ -123,7 +126,6 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
       for (int pi = 0; pi < min(DC_STAGES - 1, n_pages); ++pi) issue(pi);
 
     // Q fragments straight from global memory: rows = query heads hk*G .. hk*G + G - 1 of the new token
-    const int tok = p.seq_tok0[seq];
     const __nv_bfloat16* qrow = p.q + size_t(tok) * q_dim + size_t(hk) * G * DH;
     const int ra = lane >> 2, rb = ra + 8;
     uint32_t qf[DH / 16][4];
@@ -223,9 +225,21 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
     }
     if (!ok) break;
 
-    // the item's partial: unnormalised output, running max (log2 domain) and sum, rows = query heads
     l_a = quad_sum(l_a);
     l_b = quad_sum(l_b);
+    __nv_bfloat16* orow = p.o + size_t(tok) * q_dim + size_t(hk) * G * DH;
+    if (splits == 1) {
+      // the whole key range was this item: normalise and write the output rows directly
+      const float inv_a = 1.f / l_a, inv_b = 1.f / l_b;
+#pragma unroll
+      for (int j = 0; j < DH / 8; ++j) {
+        const int col = 8 * j + 2 * (lane & 3);
+        if (ra < G) *reinterpret_cast<uint32_t*>(orow + ra * DH + col) = pack_bf16(o_acc[j][0] * inv_a, o_acc[j][1] * inv_a);
+        if (rb < G) *reinterpret_cast<uint32_t*>(orow + rb * DH + col) = pack_bf16(o_acc[j][2] * inv_b, o_acc[j][3] * inv_b);
+      }
+      continue;
+    }
+    // the item's partial: unnormalised output, running max (log2 domain) and sum, rows = query heads
     float* po = p.part_o + size_t(item) * 16 * DH;
     float* pml = p.part_ml + size_t(item) * 16 * 2;
 #pragma unroll
@@ -238,44 +252,56 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
       if (ra < G) { pml[ra * 2] = m_a; pml[ra * 2 + 1] = l_a; }
       if (rb < G) { pml[rb * 2] = m_b; pml[rb * 2 + 1] = l_b; }
     }
+    // The warp that completes the last split of a (sequence, KV head) merges all of its splits, always in
+    // split order, so the result does not depend on which warp that is.
+    __threadfence();
+    __syncwarp();
+    int* done = p.group_done + drow * p.n_kv_heads + hk;
+    int last = 0;
+    if (lane == 0) last = atomicAdd(done, 1) == splits - 1;
+    last = __shfl_sync(0xffffffffu, last, 0);
+    if (last) {
+      __threadfence();
+      // lanes_per_head lanes share one query head; each owns DH / lanes_per_head contiguous columns
+      const int lanes_per_head = G <= 8 ? 4 : 2;
+      const int g = lane / lanes_per_head, part = lane % lanes_per_head;
+      const int first = dr.z + hk * splits;
+      if (g < G) {
+        float mm = -INFINITY;
+        for (int j = 0; j < splits; ++j) mm = fmaxf(mm, __ldcg(p.part_ml + (size_t(first + j) * 16 + g) * 2));
+        float ll = 0.f;
+        constexpr int MAXV = DH / 8;               // float4 per lane when two lanes share a head
+        float4 acc[MAXV];
+        const int nv = DH / 4 / lanes_per_head;    // float4 per lane
+#pragma unroll
+        for (int i = 0; i < MAXV; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int j = 0; j < splits; ++j) {
+          const float* ml = p.part_ml + (size_t(first + j) * 16 + g) * 2;
+          const float f = exp2f(__ldcg(ml) - mm);
+          ll += f * __ldcg(ml + 1);
+          const float4* src = reinterpret_cast<const float4*>(p.part_o + (size_t(first + j) * 16 + g) * DH) + part * nv;
+#pragma unroll
+          for (int i = 0; i < MAXV; ++i) {
+            if (i < nv) {
+              const float4 v = __ldcg(src + i);
+              acc[i].x += f * v.x; acc[i].y += f * v.y; acc[i].z += f * v.z; acc[i].w += f * v.w;
+            }
+          }
+        }
+        const float inv = 1.f / ll;
+        __nv_bfloat16* dst = orow + g * DH + part * nv * 4;
+#pragma unroll
+        for (int i = 0; i < MAXV; ++i) {
+          if (i < nv)
+            *reinterpret_cast<uint2*>(dst + 4 * i) =
+                make_uint2(pack_bf16(acc[i].x * inv, acc[i].y * inv), pack_bf16(acc[i].z * inv, acc[i].w * inv));
+        }
+      }
+      if (lane == 0) *done = 0;             // ready for the next launch
+    }
   }
   __syncthreads();
   if (*abort_flag) drain_after_abort();
-}
-
-// =================================================================== combine ==
-constexpr int CB_THREADS = 256;
-
-template <int DH>
-__global__ void __launch_bounds__(CB_THREADS, 1) attn_combine_kernel(const AttnParams p) {
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int G = p.n_q_heads / p.n_kv_heads;
-  const int q_dim = p.n_q_heads * DH;
-  constexpr int PER = DH / 32;
-  const int total = p.n_decode_rows * p.n_q_heads;
-  for (int w = blockIdx.x * (CB_THREADS / 32) + warp; w < total; w += gridDim.x * (CB_THREADS / 32)) {
-    const int4 row = reinterpret_cast<const int4*>(p.decode_rows)[w / p.n_q_heads];
-    const int hq = w % p.n_q_heads, hk = hq / G, g = hq % G;
-    const int tok = row.y, first = row.z + hk * row.w, splits = row.w;
-    float mm = -INFINITY;
-    for (int j = 0; j < splits; ++j) mm = fmaxf(mm, p.part_ml[(size_t(first + j) * 16 + g) * 2]);
-    float acc[PER];
-#pragma unroll
-    for (int i = 0; i < PER; ++i) acc[i] = 0.f;
-    float ll = 0.f;
-    for (int j = 0; j < splits; ++j) {
-      const float* ml = p.part_ml + (size_t(first + j) * 16 + g) * 2;
-      const float f = exp2f(ml[0] - mm);
-      ll += f * ml[1];
-      const float* po = p.part_o + (size_t(first + j) * 16 + g) * DH + lane * PER;
-#pragma unroll
-      for (int i = 0; i < PER; ++i) acc[i] += f * po[i];
-    }
-    const float inv = 1.f / ll;
-    __nv_bfloat16* dst = p.o + size_t(tok) * q_dim + hq * DH + lane * PER;
-#pragma unroll
-    for (int i = 0; i < PER; i += 2) *reinterpret_cast<uint32_t*>(dst + i) = pack_bf16(acc[i] * inv, acc[i + 1] * inv);
-  }
 }
 
 template <typename K>
@@ -290,8 +316,7 @@ cudaError_t attention_set_attributes() {
   if ((e = attention_prefill_set_attributes()) != cudaSuccess) return e;
   if ((e = set_smem(attn_decode_kernel<64>, dc_smem_bytes<64>())) != cudaSuccess) return e;
   if ((e = set_smem(attn_decode_kernel<128>, dc_smem_bytes<128>())) != cudaSuccess) return e;
-  if ((e = set_smem(attn_combine_kernel<64>, kMinSmemBytes)) != cudaSuccess) return e;
-  return set_smem(attn_combine_kernel<128>, kMinSmemBytes);
+  return cudaSuccess;
 }
 
 cudaError_t launch_attention_decode(const AttnParams& p, int sm_budget, cudaStream_t stream) {
@@ -301,18 +326,6 @@ cudaError_t launch_attention_decode(const AttnParams& p, int sm_budget, cudaStre
     attn_decode_kernel<128><<<grid, DC_THREADS, dc_smem_bytes<128>(), stream>>>(p);
   else
     attn_decode_kernel<64><<<grid, DC_THREADS, dc_smem_bytes<64>(), stream>>>(p);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_attention_combine(const AttnParams& p, int sm_budget, cudaStream_t stream) {
-  if (p.n_decode_rows <= 0) return cudaSuccess;
-  const int total = p.n_decode_rows * p.n_q_heads;
-  const int blocks = (total + CB_THREADS / 32 - 1) / (CB_THREADS / 32);
-  const int grid = blocks < sm_budget ? blocks : sm_budget;
-  if (p.head_dim == 128)
-    attn_combine_kernel<128><<<grid, CB_THREADS, kMinSmemBytes, stream>>>(p);
-  else
-    attn_combine_kernel<64><<<grid, CB_THREADS, kMinSmemBytes, stream>>>(p);
   return cudaGetLastError();
 }
 

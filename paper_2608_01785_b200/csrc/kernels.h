@@ -76,18 +76,19 @@ struct AttnParams {
   const int32_t* block_tables;
   const int32_t* prefill_items;    // int4 per item
   int n_prefill_items;
-  const int32_t* decode_items;     // int4 per item
+  const int32_t* decode_items;     // int4 per item: {decode row, kv head, first key, end key}
   int n_decode_items;
   const int32_t* decode_rows;      // int4 per decode sequence
   int n_decode_rows;
   float* part_o;                   // [max_decode_items][16][Dh] unnormalised partial outputs
   float* part_ml;                  // [max_decode_items][16][2]  running max (log2 domain) and sum
   int* counters;                   // two work-queue heads of this layer (prefill, decode), zero at entry
+  int* group_done;                 // [n_decode_rows * n_kv_heads] finished splits per group, zero at entry
+                                   // and left at zero by the kernel
   int* status;
 };
 cudaError_t launch_attention_prefill(const AttnParams& p, int sm_budget, cudaStream_t stream);
 cudaError_t launch_attention_decode(const AttnParams& p, int sm_budget, cudaStream_t stream);
-cudaError_t launch_attention_combine(const AttnParams& p, int sm_budget, cudaStream_t stream);
 cudaError_t attention_set_attributes();
 cudaError_t attention_prefill_set_attributes();
 

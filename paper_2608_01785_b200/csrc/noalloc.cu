@@ -6,7 +6,7 @@
 // later (the allocation fails, or succeeds only by stalling every stream of the device while the
 // driver maps memory), and a plug-in that is handed raw device pointers by a host runtime may simply
 // not be allowed to call the allocator.  For them this file carries a fixed scratch area in a
-// file-scope __device__ array; the entry point below runs the same decode and combine kernels on it
+// file-scope __device__ array; the entry point below runs the same decode kernel on it
 // and allocates nothing, on the device or through any library.
 //
 // The array is a device symbol.  In host code its name is only a stand-in, not a device address, so
@@ -33,7 +33,8 @@ constexpr int kMaxItems = HS_NOALLOC_MAX_ITEMS;
 // fully rewritten for the items of the call before they are read.
 constexpr int kOffCounters = 0;                                   // [4]  work-queue heads, must start at 0
 constexpr int kOffStatus = 4;                                     // [4]  device status word
-constexpr int kOffSeqTok0 = 8;                                    // [kMaxSeqs]
+constexpr int kOffGroupDone = 8;                                  // [kMaxSeqs * 16] finished splits per group, 0
+constexpr int kOffSeqTok0 = kOffGroupDone + kMaxSeqs * 16;        // [kMaxSeqs]
 constexpr int kOffSeqCtx = kOffSeqTok0 + kMaxSeqs;                // [kMaxSeqs]
 constexpr int kOffTables = kOffSeqCtx + kMaxSeqs;                 // [kMaxSeqs * kMaxPagesPerSeq]
 constexpr int kOffItems = kOffTables + kMaxSeqs * kMaxPagesPerSeq;   // [kMaxItems * 4]
@@ -100,7 +101,7 @@ extern "C" hs_status_t hs_op_decode_attention_noalloc(const void* q_dev, const v
   if (n_layers < 1 || layer < 0 || layer >= n_layers || num_pages < 1 || n_seqs < 1 || max_pages_per_seq < 1)
     return HS_ERR_INVALID_ARG;
   if ((head_dim != 64 && head_dim != 128) || n_kv_heads < 1 || n_q_heads % n_kv_heads != 0 ||
-      n_q_heads / n_kv_heads > 16)
+      n_q_heads / n_kv_heads > 16 || n_kv_heads > 16)
     return HS_ERR_UNSUPPORTED_SHAPE;
   // the fixed scratch area bounds the problem size
   if (n_seqs > kMaxSeqs || max_pages_per_seq > kMaxPagesPerSeq) return HS_ERR_UNSUPPORTED_SHAPE;
@@ -166,8 +167,8 @@ extern "C" hs_status_t hs_op_decode_attention_noalloc(const void* q_dev, const v
   a.part_o = reinterpret_cast<float*>(scratch + kOffPartO);
   a.part_ml = reinterpret_cast<float*>(scratch + kOffPartMl);
   a.counters = words + kOffCounters;
+  a.group_done = words + kOffGroupDone;
   a.status = words + kOffStatus;
   if (launch_attention_decode(a, sm_budget, stream) != cudaSuccess) return HS_ERR_CUDA;
-  if (launch_attention_combine(a, sm_budget, stream) != cudaSuccess) return HS_ERR_CUDA;
   return HS_OK;
 }

@@ -80,6 +80,7 @@ MetaLayout make_meta_layout(const hs_stage_config_t& c) {
   m.decode_items = take(m.max_decode_items * 4);
   m.decode_rows = take(c.max_seqs * 4);
   m.counters = take(c.n_layers * 2);
+  m.group_done = take(c.max_seqs * c.n_kv_heads);
   m.total = off;
   return m;
 }
@@ -145,7 +146,7 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
         for (int hk = 0; hk < c.n_kv_heads; ++hk)
           for (int j = 0; j < splits; ++j) {
             int32_t* it = meta + ml.decode_items + (n_dec_items + hk * splits + j) * 4;
-            it[0] = s; it[1] = hk; it[2] = j * kDecodeSplit; it[3] = std::min(keys, (j + 1) * kDecodeSplit);
+            it[0] = n_dec_rows; it[1] = hk; it[2] = j * kDecodeSplit; it[3] = std::min(keys, (j + 1) * kDecodeSplit);
           }
       }
       n_dec_items += c.n_kv_heads * splits;
@@ -166,6 +167,7 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
     for (size_t i = 0; i < pre.size(); ++i)
       for (int k = 0; k < 4; ++k) meta[ml.prefill_items + int(i) * 4 + k] = pre[i].v[k];
     for (int i = 0; i < c.n_layers * 2; ++i) meta[ml.counters + i] = 0;
+    for (int i = 0; i < c.max_seqs * c.n_kv_heads; ++i) meta[ml.group_done + i] = 0;
   }
   p.n_prefill_items = int(pre.size());
   p.n_decode_items = n_dec_items;
