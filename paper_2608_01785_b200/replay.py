@@ -1,0 +1,306 @@
+"""Replay of a downstream-heavy request trace on the two stages (backbone + talker) of one GPU.
+
+Each scheduler tick issues one backbone step (every sequence in its decode phase, at most `max_decode`, plus
+one first-come-first-served prefill chunk of at most `max_prefill_chunk` tokens) and, when downstream work
+exists, one talker step (at most `max_talker` sequences) on a second stream with the complementary SM
+budget -- the co-running regime whose SM split the paper's spatial controller chooses per step (Sec. 4.3,
+Algorithm 1 steps 3-4).  The per-tick backbone budget comes from a seeded stand-in policy: all SMs when
+the talker is idle, otherwise a uniform draw from the ladder.  Time is virtual: the clock advances by the
+measured latency of each tick and idle gaps are skipped, so a long trace replays in GPU time only.
+
+The engine is pluggable: `GpuEngine` drives real stages through the C ABI; `ModelEngine` is a latency
+model used by the CPU tests of the scheduling logic (it runs the same page accounting on host-only
+stages, so allocator pressure is exercised without a GPU).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import statistics
+from collections import deque
+from dataclasses import dataclass, field
+from typing import Deque, Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+from . import binding as B
+from . import workloads as wl
+
+
+@dataclass
+class ReplayConfig:
+    max_decode: int = 64
+    max_prefill_chunk: int = 2048
+    max_talker: int = 16
+    talker_ctx0: int = 128          # conditioning tokens a talker sequence starts from
+    ladder: Tuple[int, ...] = (120, 96, 74, 48)
+    policy_seed: int = 5
+
+
+@dataclass
+class _Seq:
+    req: wl.Request
+    prefilled: int = 0              # prompt tokens already in the cache
+    decoded: int = 0                # backbone tokens generated
+    talker_done: int = 0
+    t_first: Optional[float] = None       # first backbone token (end of the tick that finished prefill)
+    t_first_down: Optional[float] = None  # first downstream token
+    t_done: Optional[float] = None
+
+
+class Engine:
+    """Runs one tick; returns (backbone ms or None, talker ms or None)."""
+    sm_count = 148
+
+    def tick(self, a_batch, b_batch, budget_a: int) -> Tuple[Optional[float], Optional[float]]:
+        raise NotImplementedError
+
+    def alloc(self, which: str, seq_id: int, total: int) -> None:
+        raise NotImplementedError
+
+    def free(self, which: str, seq_id: int) -> None:
+        raise NotImplementedError
+
+
+class ModelEngine(Engine):
+    """Latency model + real page accounting on host-only stages (no GPU)."""
+
+    def __init__(self, dims_a, dims_b, pages_a: int, pages_b: int, mpps_a: int, mpps_b: int):
+        self.h = {}
+        for name, dims, pages, mpps in (("a", dims_a, pages_a, mpps_a), ("b", dims_b, pages_b, mpps_b)):
+            cfg = B.make_config(dims, pages, 4096, 128, mpps, mpps * 16, device=-1)
+            self.h[name] = (B.hs_stage_create(cfg, None, 0, 0), mpps)
+
+    def alloc(self, which, seq_id, total):
+        h, mpps = self.h[which]
+        B.hs_kv_alloc(h, seq_id, total, mpps)
+
+    def free(self, which, seq_id):
+        B.hs_kv_free(self.h[which][0], seq_id)
+
+    def free_pages(self, which):
+        return B.hs_kv_free_pages(self.h[which][0])
+
+    def tick(self, a_batch, b_batch, budget_a):
+        la = lb = None
+        if a_batch:
+            toks = sum(q for _, q, _ in a_batch)
+            la = (2.0 + 0.012 * toks) * self.sm_count / budget_a
+        if b_batch:
+            lb = 1.2 * self.sm_count / max(self.sm_count - budget_a, 1) ** 0.3 / 4.0
+        return la, lb
+
+    def close(self):
+        for h, _ in self.h.values():
+            B.hs_stage_destroy(h)
+
+
+class GpuEngine(Engine):
+    """Two real stages on one GPU, stepped on two streams with complementary budgets."""
+
+    def __init__(self, dims_a, dims_b, pages_a: int, pages_b: int, mpps_a: int, mpps_b: int, cfg: ReplayConfig,
+                 seed: int = 4, device: int = 0):
+        import torch
+        from .stage import Stage
+        self.torch = torch
+        dev = torch.device("cuda", device)
+        max_tok_a = cfg.max_decode + cfg.max_prefill_chunk
+        self.sa = Stage(dims_a, wl.make_weights(dims_a, seed, dev), pages_a, max_tok_a, cfg.max_decode + 1, mpps_a,
+                        mpps_a * 16, device)
+        self.sb = Stage(dims_b, wl.make_weights(dims_b, seed + 1, dev), pages_b, cfg.max_talker, cfg.max_talker, mpps_b,
+                        mpps_b * 16, device)
+        self.sm_count = self.sa.sm_count
+        self.xa = wl.make_x(max_tok_a, dims_a.d_model, seed, dev)
+        self.xb = wl.make_x(cfg.max_talker, dims_b.d_model, seed + 1, dev)
+        self.ya = torch.empty(max_tok_a, dims_a.d_model, dtype=torch.float32, device=dev)
+        self.yb = torch.empty(cfg.max_talker, dims_b.d_model, dtype=torch.float32, device=dev)
+        self.stream_a, self.stream_b = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        self.tables = {"a": {}, "b": {}}
+
+    def _stage(self, which):
+        return self.sa if which == "a" else self.sb
+
+    def alloc(self, which, seq_id, total):
+        self.tables[which][seq_id] = self._stage(which).kv_alloc(seq_id, total)
+
+    def free(self, which, seq_id):
+        self._stage(which).kv_free(seq_id)
+        del self.tables[which][seq_id]
+
+    def free_pages(self, which):
+        return B.hs_kv_free_pages(self._stage(which).handle)
+
+    def _launch(self, which, batch, budget, stream, x, y):
+        st = self._stage(which)
+        bt = st.block_table_array([self.tables[which][sid] for sid, _, _ in batch])
+        n = sum(q for _, q, _ in batch)
+        b = st.make_batch([q for _, q, _ in batch], [c for _, _, c in batch], bt, x[:n], y[:n])
+        e0, e1 = self.torch.cuda.Event(enable_timing=True), self.torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        st.step(b, budget, stream)
+        e1.record(stream)
+        return e0, e1, b
+
+    def tick(self, a_batch, b_batch, budget_a):
+        ev = []
+        if a_batch:
+            ev.append(("a",) + self._launch("a", a_batch, budget_a, self.stream_a, self.xa, self.ya))
+        if b_batch:
+            ev.append(("b",) + self._launch("b", b_batch, self.sm_count - budget_a if a_batch else self.sm_count,
+                                            self.stream_b, self.xb, self.yb))
+        self.torch.cuda.synchronize()
+        out = {"a": None, "b": None}
+        for which, e0, e1, _ in ev:
+            out[which] = e0.elapsed_time(e1)
+        assert self.sa.status() == 0 and self.sb.status() == 0
+        return out["a"], out["b"]
+
+    def close(self):
+        self.sa.close()
+        self.sb.close()
+
+
+def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = ReplayConfig()) -> Dict:
+    """Runs the whole trace; returns aggregate metrics (virtual seconds)."""
+    rng = np.random.Generator(np.random.PCG64(cfg.policy_seed))
+    waiting: Deque[_Seq] = deque()
+    prefilling: Optional[_Seq] = None
+    decoding: List[_Seq] = []
+    talker_wait: Deque[_Seq] = deque()
+    talking: List[_Seq] = []
+    done: List[_Seq] = []
+    t = 0.0
+    nxt = 0
+    ticks_by_budget: Dict[int, List[float]] = {}
+    talker_lat: List[float] = []
+    backbone_tokens = talker_tokens = 0
+    busy_s = 0.0
+
+    def admit(now):
+        nonlocal nxt
+        while nxt < len(trace) and trace[nxt].arrival_s <= now:
+            waiting.append(_Seq(trace[nxt]))
+            nxt += 1
+
+    while len(done) < len(trace):
+        admit(t)
+        if prefilling is None and waiting and len(decoding) < cfg.max_decode:
+            prefilling = waiting.popleft()
+        while talker_wait and len(talking) < cfg.max_talker:
+            s = talker_wait.popleft()
+            talking.append(s)
+        if prefilling is None and not decoding and not talking:
+            if nxt >= len(trace):
+                break
+            t = max(t, trace[nxt].arrival_s)          # idle: jump to the next arrival
+            continue
+
+        # ---- build the tick's batches: (seq id, new tokens, cached tokens) ----
+        a_batch = []
+        if prefilling is not None:
+            n = min(cfg.max_prefill_chunk, prefilling.req.prompt_len - prefilling.prefilled)
+            engine.alloc("a", prefilling.req.rid, prefilling.prefilled + n)
+            a_batch.append((prefilling.req.rid, n, prefilling.prefilled))
+        stepped = list(decoding)                       # sequences that decode one token in this tick
+        for s in stepped:
+            ctx = s.req.prompt_len + s.decoded
+            engine.alloc("a", s.req.rid, ctx + 1)
+            a_batch.append((s.req.rid, 1, ctx))
+        b_batch = []
+        for s in talking:
+            ctx = cfg.talker_ctx0 + s.talker_done
+            engine.alloc("b", s.req.rid, ctx + 1)
+            b_batch.append((s.req.rid, 1, ctx))
+        budget = engine.sm_count if not b_batch else int(rng.choice(cfg.ladder))
+        lat_a, lat_b = engine.tick(a_batch, b_batch, budget)
+        tick_ms = max(lat_a or 0.0, lat_b or 0.0)
+        t += tick_ms * 1e-3
+        busy_s += tick_ms * 1e-3
+        if lat_a is not None:
+            ticks_by_budget.setdefault(budget, []).append(lat_a)
+            backbone_tokens += sum(q for _, q, _ in a_batch)
+        if lat_b is not None:
+            talker_lat.append(lat_b)
+            talker_tokens += len(b_batch)
+
+        # ---- advance request state ----
+        if prefilling is not None:
+            prefilling.prefilled += a_batch[0][1]
+            if prefilling.prefilled == prefilling.req.prompt_len:
+                prefilling.t_first = t
+                decoding.append(prefilling)
+                if prefilling.req.talker_out > 0:
+                    talker_wait.append(prefilling)
+                prefilling = None
+        for s in stepped:
+            s.decoded += 1
+        still = []
+        for s in decoding:
+            if s.decoded >= s.req.backbone_out:
+                engine.free("a", s.req.rid)
+                if s.req.talker_out == 0 or s.talker_done >= s.req.talker_out:
+                    s.t_done = t
+                    done.append(s)
+            else:
+                still.append(s)
+        decoding = still
+        still = []
+        for s in talking:
+            s.talker_done += 1
+            if s.t_first_down is None:
+                s.t_first_down = t
+            if s.talker_done >= s.req.talker_out:
+                engine.free("b", s.req.rid)
+                if s.decoded >= s.req.backbone_out:
+                    s.t_done = t
+                    done.append(s)
+            else:
+                still.append(s)
+        talking = still
+
+    def pct(v, q):
+        return float(np.percentile(v, q)) if v else None
+
+    by_class = {}
+    for cls in ("text", "speech", "image"):
+        sel = [s for s in done if s.req.out_class == cls]
+        ttft = [(s.t_first - s.req.arrival_s) * 1e3 for s in sel if s.t_first is not None]
+        ttfo = [(s.t_first_down - s.req.arrival_s) * 1e3 for s in sel if s.t_first_down is not None]
+        by_class[cls] = {"requests": len(sel), "ttft_ms_p50": pct(ttft, 50), "ttft_ms_p95": pct(ttft, 95),
+                         "first_downstream_ms_p50": pct(ttfo, 50), "first_downstream_ms_p95": pct(ttfo, 95)}
+    return {"requests_done": len(done), "virtual_seconds": t, "busy_seconds": busy_s,
+            "backbone_tokens": backbone_tokens, "talker_tokens": talker_tokens,
+            "backbone_tokens_per_s": backbone_tokens / busy_s if busy_s else None,
+            "tick_ms_by_budget": {str(b): {"n": len(v), "mean": statistics.fmean(v), "p50": pct(v, 50), "p95": pct(v, 95)}
+                                  for b, v in sorted(ticks_by_budget.items(), reverse=True)},
+            "talker_ms": {"n": len(talker_lat), "mean": statistics.fmean(talker_lat) if talker_lat else None,
+                          "p95": pct(talker_lat, 95)},
+            "by_class": by_class}
+
+
+def pool_sizes(cfg: ReplayConfig, max_prompt: int = 4096, max_out: int = 512, max_talker_out: int = 1500):
+    mpps_a = -(-(max_prompt + max_out + 1) // 16)
+    mpps_b = -(-(cfg.talker_ctx0 + max_talker_out + 1) // 16)
+    return (cfg.max_decode + 1) * mpps_a, cfg.max_talker * mpps_b, mpps_a, mpps_b
+
+
+def main():
+    ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
+    ap.add_argument("--rate", type=float, default=8.0, help="Poisson arrival rate, requests per second")
+    ap.add_argument("--requests", type=int, default=2000)
+    ap.add_argument("--backbone", default="c3_7b")
+    ap.add_argument("--talker", default="c4_talker")
+    args = ap.parse_args()
+    cfg = ReplayConfig()
+    pa, pb, ma, mb = pool_sizes(cfg)
+    eng = GpuEngine(wl.DIMS[args.backbone], wl.DIMS[args.talker], pa, pb, ma, mb, cfg)
+    try:
+        res = replay(wl.make_trace(args.rate, args.requests), eng, cfg)
+    finally:
+        eng.close()
+    res.update({"rate_per_s": args.rate, "backbone": args.backbone, "talker": args.talker})
+    print(json.dumps(res))
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,28 @@
+"""Trace replay on real stages (small dimensions): the backbone and the talker are stepped through the C
+ABI on two streams with complementary SM budgets, tick after tick, with sequences joining and leaving."""
+import pytest
+
+from paper_2608_01785_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def test_replay_small_trace_on_gpu():
+    from paper_2608_01785_b200.replay import GpuEngine, ReplayConfig, pool_sizes, replay
+    cfg = ReplayConfig(max_decode=12, max_prefill_chunk=512, max_talker=4, ladder=(120, 96, 74, 48))
+    trace = [wl.Request(r.rid, r.arrival_s, r.out_class, min(r.prompt_len, 900), min(r.backbone_out, 40),
+                        min(r.talker_out, 60)) for r in wl.make_trace(16.0, 30, seed=4)]
+    pa, pb, ma, mb = pool_sizes(cfg, max_prompt=900, max_out=40, max_talker_out=60)
+    backbone = wl.StageDims(2, 512, 8, 2, 64, 1408)
+    talker = wl.StageDims(2, 256, 4, 2, 64, 688)
+    eng = GpuEngine(backbone, talker, pa, pb, ma, mb, cfg)
+    try:
+        res = replay(trace, eng, cfg)
+        assert res["requests_done"] == 30
+        assert res["backbone_tokens"] == sum(r.prompt_len + r.backbone_out for r in trace)
+        assert res["talker_tokens"] == sum(r.talker_out for r in trace)
+        assert eng.free_pages("a") == pa and eng.free_pages("b") == pb
+        assert res["backbone_tokens_per_s"] > 0
+        assert set(res["tick_ms_by_budget"]) <= {"148", "120", "96", "74", "48"}
+    finally:
+        eng.close()

@@ -1,0 +1,46 @@
+"""Scheduling logic of the trace replay, on the latency-model engine (no GPU): every request finishes,
+token counts are conserved, the page allocators of both stages return to empty, budgets come from the
+ladder only while the talker has work."""
+import numpy as np
+
+from paper_2608_01785_b200 import workloads as wl
+from paper_2608_01785_b200.replay import ModelEngine, ReplayConfig, pool_sizes, replay
+
+
+def test_trace_statistics():
+    tr = wl.make_trace(8.0, 2000, seed=4)
+    assert len(tr) == 2000
+    gaps = np.diff([0.0] + [r.arrival_s for r in tr])
+    assert abs(gaps.mean() - 1 / 8.0) < 0.01                       # Poisson arrivals at the stated rate
+    frac = {c: sum(r.out_class == c for r in tr) / 2000 for c in ("text", "speech", "image")}
+    assert abs(frac["text"] - 0.3) < 0.04 and abs(frac["speech"] - 0.5) < 0.04 and abs(frac["image"] - 0.2) < 0.04
+    p = np.array([r.prompt_len for r in tr])
+    assert p.min() >= 64 and p.max() <= 4096 and 520 < np.median(p) < 690
+    assert all(64 <= r.backbone_out <= 512 for r in tr)
+    assert all((r.talker_out == 0) == (r.out_class == "text") for r in tr)
+    assert all(200 <= r.talker_out <= 1500 for r in tr if r.out_class != "text")
+    assert wl.make_trace(8.0, 50, seed=4)[:50] == tr[:50]           # seeded
+
+
+def test_replay_conserves_tokens_and_pages():
+    cfg = ReplayConfig(max_decode=8, max_prefill_chunk=256, max_talker=4)
+    trace = wl.make_trace(16.0, 60, seed=4)
+    pa, pb, ma, mb = pool_sizes(cfg)
+    eng = ModelEngine(wl.DIMS["c1_tiny"], wl.DIMS["c1_tiny"], pa, pb, ma, mb)
+    try:
+        res = replay(trace, eng, cfg)
+        assert res["requests_done"] == 60
+        assert res["backbone_tokens"] == sum(r.prompt_len + r.backbone_out for r in trace)
+        assert res["talker_tokens"] == sum(r.talker_out for r in trace)
+        assert eng.free_pages("a") == pa and eng.free_pages("b") == pb      # everything was returned
+        budgets = {int(b) for b in res["tick_ms_by_budget"]}
+        assert budgets <= {148, *cfg.ladder} and 148 in budgets and budgets & set(cfg.ladder)
+        for cls in ("text", "speech", "image"):
+            c = res["by_class"][cls]
+            assert c["requests"] == sum(r.out_class == cls for r in trace)
+            assert c["ttft_ms_p50"] is not None and c["ttft_ms_p50"] > 0
+        assert res["by_class"]["text"]["first_downstream_ms_p50"] is None
+        assert res["by_class"]["speech"]["first_downstream_ms_p50"] >= res["by_class"]["speech"]["ttft_ms_p50"]
+        assert res["virtual_seconds"] >= res["busy_seconds"] > 0
+    finally:
+        eng.close()
