@@ -17,7 +17,7 @@ namespace {
 constexpr int kRing = 4;   // pinned staging slots for step metadata
 
 struct WsLayout {
-  size_t rope, h, q, o, act, meta, part_o, part_ml, status, total;
+  size_t rope, h, q, o, act, meta, part_o, part_ml, status, turn, total;
 };
 
 WsLayout make_ws_layout(const hs_stage_config_t& c, const MetaLayout& ml) {
@@ -38,6 +38,7 @@ WsLayout make_ws_layout(const hs_stage_config_t& c, const MetaLayout& ml) {
   w.part_o = take(size_t(ml.max_decode_items) * 16 * c.head_dim * 4);
   w.part_ml = take(size_t(ml.max_decode_items) * 16 * 2 * 4);
   w.status = take(256);
+  w.turn = take(kGemmTurnWords * 4);
   w.total = off;
   return w;
 }
@@ -97,6 +98,13 @@ thread_local std::string g_last_error;
 hs_status_t cuda_fail(const char* where, cudaError_t e) {
   g_last_error = std::string(where) + ": " + cudaGetErrorName(e) + " (" + cudaGetErrorString(e) + ")";
   return HS_ERR_CUDA;
+}
+
+// K splits for a residual GEMM, or 1 when the whose-turn array could not hold its tiles.
+int pick_ksplit(int M, int N, int K, int bn, int sm_count) {
+  const int tiles = ceil_div(M, 128) * ceil_div(N, bn);
+  if (tiles * 4 > kGemmTurnWords) return 1;
+  return gemm_pick_ksplit(M, N, K, bn, sm_count);
 }
 
 bool g_attrs_set[64] = {};
@@ -250,7 +258,8 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
   }
   if (cudaMemcpy(s->ws_dev + s->ws.rope, rope.data(), rope.size() * sizeof(float2), cudaMemcpyHostToDevice) !=
           cudaSuccess ||
-      cudaMemset(s->ws_dev + s->ws.status, 0, 256) != cudaSuccess)
+      cudaMemset(s->ws_dev + s->ws.status, 0, 256) != cudaSuccess ||
+      cudaMemset(s->ws_dev + s->ws.turn, 0, kGemmTurnWords * 4) != cudaSuccess)
     return HS_ERR_CUDA;
 
   // tensor maps
@@ -450,6 +459,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     go.mode = kGemmResid;
     go.tm_out = tm_y; go.accumulate = 1;
     go.bn = gemm_pick_bn(T, d, s->sm_count);
+    go.ksplit = pick_ksplit(T, d, q_dim, go.bn, s->sm_count);
+    go.tile_turn = reinterpret_cast<int*>(s->ws_dev + s->ws.turn);
     go.status = status;
     { LaunchTimer t(s, 5, stream); where = "out-proj gemm"; e = launch_gemm(go, sm_budget, stream); }
     if (e != cudaSuccess) break;
@@ -476,6 +487,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gd.mode = kGemmResid;
     gd.tm_out = tm_y; gd.accumulate = 1;
     gd.bn = gemm_pick_bn(T, d, s->sm_count);
+    gd.ksplit = pick_ksplit(T, d, F, gd.bn, s->sm_count);
+    gd.tile_turn = reinterpret_cast<int*>(s->ws_dev + s->ws.turn);
     gd.status = status;
     { LaunchTimer t(s, 7, stream); where = "down gemm"; e = launch_gemm(gd, sm_budget, stream); }
     if (e != cudaSuccess) break;

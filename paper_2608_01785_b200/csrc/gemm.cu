@@ -88,6 +88,31 @@ __device__ __forceinline__ void stage_bf16x32(uint8_t* buf, int lane, int u0, co
   }
 }
 
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(int* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+// Bounded spin on a global word written by another block (same limits as the mbarrier waits).
+__device__ __forceinline__ bool spin_until_equal(const int* word, int value, volatile int* abort_flag, int* status) {
+  const unsigned long long t0 = globaltimer_ns();
+  for (uint32_t spins = 0;; ++spins) {
+    if (ld_acquire(word) == value) return true;
+    if ((spins & 0x3f) == 0x3f) {
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicExch(status, kErrTimeout);
+        return false;
+      }
+      __nanosleep(100);
+    }
+  }
+}
+
 // Address of element e of (slot, kv head) in one layer's K or V pages.
 __device__ __forceinline__ __nv_bfloat16* cache_ptr(__nv_bfloat16* base, int slot, int hk, int n_kv_heads, int Dh,
                                                     int e) {
@@ -111,6 +136,11 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
   const int n_n_tiles = gemm_n_tiles(p);
   const int n_tiles = n_m_tiles * n_n_tiles;
   const int k_blocks = (p.K + BK - 1) / BK;
+  // Work unit = (output tile, K split).  Splits exist only in Resid mode with few tiles; units are ordered
+  // split-major, so the units a split has to wait for always have smaller indices.
+  const int ksplit = p.mode == kGemmResid && p.ksplit > 1 ? p.ksplit : 1;
+  const int kb_per = (k_blocks + ksplit - 1) / ksplit;
+  const int n_units = n_tiles * ksplit;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) {
@@ -143,10 +173,12 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
       uint32_t ph = 0;
       bool ok = true;
       const bool two_halves = p.mode != kGemmResid || p.bn > 128;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        const int tile = u % n_tiles, ks = u / n_tiles;
         const int m = tile % n_m_tiles, n = tile / n_m_tiles;
         const BSource b0 = b_source(p, n, 0), b1 = b_source(p, n, 1);
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        const int kb_end = min(k_blocks, (ks + 1) * kb_per);
+        for (int kb = ks * kb_per; kb < kb_end; ++kb) {
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status)) { ok = false; break; }
           uint8_t* st = smem + s * STAGE_BYTES;
           mbar_expect_tx(&full[s], two_halves ? STAGE_BYTES : A_BYTES + BH_BYTES);
@@ -164,11 +196,12 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
         if (!mbar_wait(&tempty[acc], acc_ph ^ 1, abort_flag, p.status)) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int kb = 0; kb < k_blocks; ++kb) {
+        const int kb_begin = (u / n_tiles) * kb_per, kb_end = min(k_blocks, kb_begin + kb_per);
+        for (int kb = kb_begin; kb < kb_end; ++kb) {
           if (!mbar_wait(&full[s], ph, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after_sync();
           const uint32_t a_addr = smem_u32(smem + s * STAGE_BYTES);
@@ -176,7 +209,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
           const uint64_t b_desc = umma_desc_kmajor_sw128(a_addr + A_BYTES);
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)   // 16 bf16 = 32 B along K: +2 in the (address / 16) field
-            umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0);
+            umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, ((kb - kb_begin) | k) != 0);
           umma_commit(&empty[s]);             // frees the stage once these MMAs have read it
           if (++s == STAGES) { s = 0; ph ^= 1; }
         }
@@ -193,7 +226,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     const int Dh = p.head_dim;
     uint8_t* epi_buf = epi_smem + quarter * EPI_WARP_BYTES;
     int epi_sel = 0;                          // staging block to fill next
-    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+    for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+      const int tile = u % n_tiles, ks = u / n_tiles;
       const int m = tile % n_m_tiles, n = tile / n_m_tiles;
       const bool ok = mbar_wait(&tfull[acc], acc_ph, abort_flag, p.status);
       if (!__all_sync(0xffffffffu, ok)) break;
@@ -207,6 +241,16 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
       const int row_base = m * BM + quarter * 32;          // first row of this warp's 32
 
       if (p.mode == kGemmResid) {
+        // Ordered split-K: the partial sums of a tile are added into the output in split order, so the
+        // result is the same fixed sum whatever block computed which split.  This warp owns 32 rows of the
+        // tile; it waits until the previous split's add of those rows has been performed.
+        int* turn = p.tile_turn + tile * 4 + quarter;
+        if (ksplit > 1 && ks > 0) {
+          bool go = true;
+          if (lane == 0) go = spin_until_equal(turn, ks, abort_flag, p.status);
+          if (!__shfl_sync(0xffffffffu, go, 0)) break;
+        }
+        const bool add = p.accumulate || ks > 0;
         for (int c = 0; c < p.bn / 32; ++c) {
           const int col0 = n * p.bn + c * 32;
           if (col0 >= p.N) break;
@@ -219,11 +263,16 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
           fence_proxy_async();
           __syncwarp();
           if (lane == 0) {
-            if (p.accumulate) tma_reduce_add_2d(&p.tm_out, buf, col0, row_base);
+            if (add) tma_reduce_add_2d(&p.tm_out, buf, col0, row_base);
             else tma_store_2d(&p.tm_out, buf, col0, row_base);
             bulk_commit();
           }
           epi_sel ^= 1;
+        }
+        if (ksplit > 1 && lane == 0) {
+          bulk_wait<0>();                     // this split's adds have been performed
+          __threadfence();
+          st_release(turn, ks == ksplit - 1 ? 0 : ks + 1);   // the last split leaves the word at zero
         }
       } else if (p.mode == kGemmGateUp) {
         for (int c = 0; c < 4; ++c) {
@@ -365,10 +414,23 @@ int gemm_pick_bn(int M, int N, int sm_count) {
   return best;
 }
 
+int gemm_pick_ksplit(int M, int N, int K, int bn, int sm_count) {
+  // Few tiles (small M): split K so that about every SM streams a share of the weights.  Each split keeps
+  // at least 8 K-blocks.  Depends on the shape and the device only, never on the SM budget.
+  const int tiles = ((M + BM - 1) / BM) * ((N + bn - 1) / bn);
+  const int k_blocks = (K + BK - 1) / BK;
+  int ks = sm_count / tiles;
+  if (ks > 8) ks = 8;
+  if (ks > k_blocks / 8) ks = k_blocks / 8;
+  if (ks < 2) return 1;
+  const int per = (k_blocks + ks - 1) / ks;
+  return (k_blocks + per - 1) / per;          // no empty split
+}
+
 cudaError_t launch_gemm(const GemmParams& p, int sm_budget, cudaStream_t stream) {
   const int n_m_tiles = (p.M + BM - 1) / BM;
   const int n_n_tiles = gemm_n_tiles(p);
-  const int n_tiles = n_m_tiles * n_n_tiles;
+  const int n_tiles = n_m_tiles * n_n_tiles * (p.mode == kGemmResid && p.ksplit > 1 ? p.ksplit : 1);
   if (n_tiles <= 0) return cudaSuccess;
   const int grid = n_tiles < sm_budget ? n_tiles : sm_budget;
   gemm_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(p);

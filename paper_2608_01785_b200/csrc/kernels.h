@@ -31,6 +31,8 @@ struct GemmParams {
   CUtensorMap tm_out;        // fp32 [M, N], box 32 x 32, 128-byte swizzle (rows past M are clipped)
   int accumulate;            // 1: out += A W^T (the residual add), 0: out = A W^T
   int bn;                    // tile width of this launch (gemm_pick_bn); 256 when unused
+  int ksplit;                // K splits per output tile, added in split order (gemm_pick_ksplit); 0/1 = none
+  int* tile_turn;            // [tiles * 4] whose-turn words for the ordered adds; zero at entry and at exit
   // Qkv
   int q_dim, kv_dim, head_dim, n_kv_heads;
   CUtensorMap tm_q;          // bf16 q [M, q_dim], box 64 x 32, 128-byte swizzle
@@ -47,6 +49,8 @@ cudaError_t launch_gemm(const GemmParams& p, int sm_budget, cudaStream_t stream)
 cudaError_t gemm_set_attributes();
 // Tile width for a Resid-mode GEMM of this shape on a device with sm_count SMs (budget independent).
 int gemm_pick_bn(int M, int N, int sm_count);
+int gemm_pick_ksplit(int M, int N, int K, int bn, int sm_count);
+constexpr int kGemmTurnWords = 4096;   // capacity of the whose-turn array: splits are used only when tiles * 4 fits
 
 // ---------------------------------------------------------------- RMSNorm --
 // h[t,:] = bf16(x[t,:] * rsqrt(mean(x[t,:]^2) + eps) * g).  x comes either as bf16 (x_bf16, first layer;

@@ -62,6 +62,7 @@ DIMS = {
     "c3_7b": StageDims(28, 3584, 28, 4, 128, 18944),
     "c4_talker": StageDims(12, 1024, 16, 4, 64, 2816),
 }
+DIMS["c3_decode"] = DIMS["c3_7b"]
 SM_BUDGETS = {
     "c1_tiny": (148, 8),
     "c2_shared": (148, 112, 74, 37),
@@ -108,6 +109,9 @@ def make_batch(name: str, seed: int) -> BatchSpec:
     if name == "c3_7b":
         dec = r.integers(512, 4097, size=64).tolist()
         return BatchSpec([2048] + [1] * 64, [0] + dec)
+    if name == "c3_decode":          # config 3 without its prefill chunk: a decode-only tick of the trace replay
+        dec = r.integers(512, 4097, size=64).tolist()
+        return BatchSpec([1] * 64, dec)
     if name == "c4_talker":
         dec = r.integers(128, 1025, size=16).tolist()
         return BatchSpec([1] * 16, dec)
