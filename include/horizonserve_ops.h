@@ -36,6 +36,11 @@ hs_status_t hs_op_gemm_bf16(const void *a, const void *w, const float *resid, fl
  *   "q"   bf16 [max_tokens, Hq*Dh]  queries after RoPE
  *   "o"   bf16 [max_tokens, Hq*Dh]  attention output
  *   "act" bf16 [max_tokens, F]      silu(gate) * up
+ *   "smid" int32 [8 classes][160]   SM census: asking for this buffer switches the census on for the
+ *                                   following steps; entry [class][b] is then 1 + the SM on which block b
+ *                                   of the last layer's launch of that kernel class ran (0 = no such
+ *                                   block).  Classes as in hs_stage_profile_read.  It shows that a step
+ *                                   with sm_budget B never occupies more than B SMs at a time.
  * Errors: INVALID_ARG (unknown name), NO_DEVICE.
  */
 hs_status_t hs_stage_debug_buffer(hs_stage_t *stage, const char *name, void **dev_ptr, size_t *bytes);

@@ -10,6 +10,7 @@
 #include "../../include/horizonserve_ops.h"
 #include "hs_internal.h"
 #include "kernels.h"
+#include "ptx.cuh"
 
 namespace hs {
 namespace {
@@ -17,7 +18,7 @@ namespace {
 constexpr int kRing = 4;   // pinned staging slots for step metadata
 
 struct WsLayout {
-  size_t rope, h, q, o, act, meta, part_o, part_ml, status, turn, total;
+  size_t rope, h, q, o, act, meta, part_o, part_ml, status, turn, smid, total;
 };
 
 WsLayout make_ws_layout(const hs_stage_config_t& c, const MetaLayout& ml) {
@@ -39,6 +40,7 @@ WsLayout make_ws_layout(const hs_stage_config_t& c, const MetaLayout& ml) {
   w.part_ml = take(size_t(ml.max_decode_items) * 16 * 2 * 4);
   w.status = take(256);
   w.turn = take(kGemmTurnWords * 4);
+  w.smid = take(size_t(HS_PROFILE_CLASSES) * kSmidSlots * 4);
   w.total = off;
   return w;
 }
@@ -143,6 +145,7 @@ struct hs_stage {
   bool ev_pending[kRing] = {};
   int ring_pos = 0;
   // optional per-kernel timing
+  bool census = false;      // record SM placement of the last step's launches
   bool profile = false;
   struct Timed { int cls; cudaEvent_t a, b; };
   std::vector<Timed> timed;
@@ -393,6 +396,10 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
   const size_t layer_kv_elems = size_t(c.num_pages) * c.n_kv_heads * kPage * Dh;
   cudaError_t e = cudaSuccess;
   const char* where = "";
+  int* census = s->census ? reinterpret_cast<int*>(s->ws_dev + s->ws.smid) : nullptr;
+  if (census && cudaMemsetAsync(census, 0, size_t(HS_PROFILE_CLASSES) * kSmidSlots * 4, stream) != cudaSuccess)
+    return HS_ERR_CUDA;
+  auto slots = [&](int cls) { return census ? census + cls * kSmidSlots : nullptr; };
 
   for (int l = 0; l < c.n_layers && e == cudaSuccess; ++l) {
     const hs_layer_weights_t& w = s->layers[l];
@@ -407,6 +414,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     np.T = T;
     np.d = d;
     np.eps = c.rms_eps;
+    np.smid_log = slots(0);
     { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
@@ -423,6 +431,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     g.tok_slot = meta + s->ml.tok_slot;
     g.rope = reinterpret_cast<const float2*>(s->ws_dev + s->ws.rope);
     g.status = status;
+    g.smid_log = slots(1);
     { LaunchTimer t(s, 1, stream); where = "qkv gemm"; e = launch_gemm(g, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
@@ -447,6 +456,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     a.counters = meta + s->ml.counters + 2 * l;
     a.group_done = meta + s->ml.group_done;
     a.status = status;
+    a.smid_log = slots(2);       // prefill in class 2, decode in class 3 (the next slots)
     if (a.n_prefill_items > 0) { LaunchTimer t(s, 2, stream); where = "prefill attention"; e = launch_attention_prefill(a, sm_budget, stream); }
     if (e != cudaSuccess) break;
     if (a.n_decode_items > 0) { LaunchTimer t(s, 3, stream); where = "decode attention"; e = launch_attention_decode(a, sm_budget, stream); }
@@ -462,6 +472,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     go.ksplit = pick_ksplit(T, d, q_dim, go.bn, s->sm_count);
     go.tile_turn = reinterpret_cast<int*>(s->ws_dev + s->ws.turn);
     go.status = status;
+    go.smid_log = slots(5);
     { LaunchTimer t(s, 5, stream); where = "out-proj gemm"; e = launch_gemm(go, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
@@ -477,6 +488,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gu.mode = kGemmGateUp;
     gu.tm_act = s->tm_act_st;
     gu.status = status;
+    gu.smid_log = slots(6);
     { LaunchTimer t(s, 6, stream); where = "gate/up gemm"; e = launch_gemm(gu, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
@@ -490,6 +502,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gd.ksplit = pick_ksplit(T, d, F, gd.bn, s->sm_count);
     gd.tile_turn = reinterpret_cast<int*>(s->ws_dev + s->ws.turn);
     gd.status = status;
+    gd.smid_log = slots(7);
     { LaunchTimer t(s, 7, stream); where = "down gemm"; e = launch_gemm(gd, sm_budget, stream); }
     if (e != cudaSuccess) break;
   }
@@ -542,6 +555,12 @@ hs_status_t hs_stage_debug_buffer(hs_stage_t* s, const char* name, void** dev_pt
   else if (n == "q") { off = s->ws.q; sz = T * q_dim * 2; }
   else if (n == "o") { off = s->ws.o; sz = T * q_dim * 2; }
   else if (n == "act") { off = s->ws.act; sz = T * c.d_ffn * 2; }
+  else if (n == "smid") {
+    // asking for the census switches it on for the following steps
+    s->census = true;
+    off = s->ws.smid;
+    sz = size_t(HS_PROFILE_CLASSES) * kSmidSlots * 4;
+  }
   else return HS_ERR_INVALID_ARG;
   *dev_ptr = s->ws_dev + off;
   *bytes = sz;

@@ -86,6 +86,7 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
   volatile int* abort_flag = reinterpret_cast<volatile int*>(full_all + DC_WARPS * DC_STAGES);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  log_smid(p.smid_log ? p.smid_log + kSmidSlots : nullptr);
   const int G = p.n_q_heads / p.n_kv_heads;
   const int q_dim = p.n_q_heads * DH;
   const float scale_log2 = kLog2e / sqrtf(float(DH));

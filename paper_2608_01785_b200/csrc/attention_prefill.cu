@@ -84,6 +84,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
   volatile int* abort_flag = &bar->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  log_smid(p.smid_log);
   const int G = p.n_q_heads / p.n_kv_heads;
   const int Mt = p.prefill_tokens;
   const int q_dim = p.n_q_heads * DH;

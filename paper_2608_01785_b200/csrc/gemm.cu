@@ -132,6 +132,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  log_smid(p.smid_log);
   const int n_m_tiles = (p.M + BM - 1) / BM;
   const int n_n_tiles = gemm_n_tiles(p);
   const int n_tiles = n_m_tiles * n_n_tiles;

@@ -44,6 +44,7 @@ struct GemmParams {
   // GateUp
   CUtensorMap tm_act;        // bf16 act [M, N], box 64 x 32, 128-byte swizzle
   int* status;               // device status word
+  int* smid_log;             // nullable: SM census slots of this launch (see log_smid)
 };
 cudaError_t launch_gemm(const GemmParams& p, int sm_budget, cudaStream_t stream);
 cudaError_t gemm_set_attributes();
@@ -63,6 +64,7 @@ struct NormParams {
   __nv_bfloat16* h;
   int T, d;
   float eps;
+  int* smid_log;             // nullable: SM census slots of this launch
 };
 cudaError_t launch_rmsnorm(const NormParams& p, int sm_budget, cudaStream_t stream);
 cudaError_t norm_set_attributes();
@@ -90,6 +92,7 @@ struct AttnParams {
   int* group_done;                 // [n_decode_rows * n_kv_heads] finished splits per group, zero at entry
                                    // and left at zero by the kernel
   int* status;
+  int* smid_log;                   // nullable: SM census slots; prefill uses [0, 160), decode [160, 320)
 };
 cudaError_t launch_attention_prefill(const AttnParams& p, int sm_budget, cudaStream_t stream);
 cudaError_t launch_attention_decode(const AttnParams& p, int sm_budget, cudaStream_t stream);

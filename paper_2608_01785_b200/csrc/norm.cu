@@ -34,6 +34,7 @@ __device__ __forceinline__ void unpack8(const uint4& w, float (&f)[8]) {
 __global__ void __launch_bounds__(NORM_THREADS, 1) rmsnorm_kernel(const NormParams p) {
   extern __shared__ float norm_smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  log_smid(p.smid_log);
   float4* cache = reinterpret_cast<float4*>(norm_smem + warp * NORM_STAGE_FLOATS);
   const int d8 = p.d >> 3;                         // groups of 8 elements
   const int cached8 = min(d8, NORM_STAGE_FLOATS / 8);

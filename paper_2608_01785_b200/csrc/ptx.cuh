@@ -20,6 +20,16 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
   asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
   return t;
 }
+// Census of SM placement (diagnosis): block b of a launch records the SM it runs on, plus one, in
+// log[b]; a null log disables it.  kSmidSlots entries per kernel class.
+constexpr int kSmidSlots = 160;
+__device__ __forceinline__ void log_smid(int* log) {
+  if (log != nullptr && threadIdx.x == 0 && blockIdx.x < kSmidSlots) {
+    unsigned smid;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    log[blockIdx.x] = int(smid) + 1;
+  }
+}
 __device__ __forceinline__ bool elect_one() {
   uint32_t pred;
   asm volatile(

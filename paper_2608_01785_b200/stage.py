@@ -67,10 +67,13 @@ class Stage:
         return B.hs_stage_status(self.handle)
 
     def debug_tensor(self, name: str) -> torch.Tensor:
-        """Copy of a private intermediate ("h", "q", "o", "act"; bf16), shaped [max_tokens, width]."""
+        """Copy of a private intermediate ("h", "q", "o", "act"; bf16), shaped [max_tokens, width], or of the
+        SM census ("smid"; int32 [kernel class, block]; the first request switches the census on)."""
         ptr, size = B.hs_stage_debug_buffer(self.handle, name)
         off = ptr - self.workspace.data_ptr()
         raw = self.workspace[off: off + size].clone()
+        if name == "smid":
+            return raw.view(torch.int32).view(len(B.PROFILE_CLASSES), -1)
         return raw.view(torch.bfloat16).view(self.cfg.max_tokens, -1)
 
     def close(self) -> None:

@@ -280,3 +280,32 @@ def test_corun_on_two_streams_is_bit_identical_to_solo(orc):
         assert rel_err(ya_solo, y_ref) <= TOL
     finally:
         st_a.close(); st_b.close()
+
+
+# ------------------------------------------------------------- SM census --
+def test_every_kernel_of_a_step_stays_within_the_sm_budget(orc):
+    """Each block records the SM it runs on.  With sm_budget B no kernel class may show more than B
+    blocks, and blocks of one launch sit on pairwise different SMs (one block per SM)."""
+    dims = wl.StageDims(2, 512, 8, 2, 64, 1408)
+    case = make_case(dims, wl.BatchSpec([700, 333, 1, 1, 1, 1], [0, 100, 900, 300, 40, 2000]), seed=41, kv_fill=True)
+    st = make_stage(case)
+    try:
+        st.debug_tensor("smid")                              # switches the census on
+        y_ref = None
+        for budget in (148, 37, 5, 1):
+            y, _ = run_step(st, case, budget)
+            census = st.debug_tensor("smid").cpu().numpy()
+            used = set()
+            for cls, name in enumerate(B.PROFILE_CLASSES):
+                sms = census[cls][census[cls] > 0] - 1
+                if name == "attn_combine":
+                    assert len(sms) == 0
+                    continue
+                assert 1 <= len(sms) <= budget, (name, budget, len(sms))
+                assert len(set(sms.tolist())) == len(sms), (name, budget)      # one block per SM
+                used |= set(sms.tolist())
+            assert max(used) < st.sm_count
+            y_ref = y if y_ref is None else y_ref
+            assert np.array_equal(y, y_ref)
+    finally:
+        st.close()
