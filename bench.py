@@ -94,10 +94,13 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_stage(name: str, device: int, init: str = "n002"):
+def build_stage(name: str, device: int, init: str = "n002", layers: int = 0):
     """Weights, KV pool with random-filled context, block tables and input of the named workload."""
     from paper_2608_01785_b200.stage import Stage
     dims = wl.DIMS[name]
+    if layers:
+        dims = wl.StageDims(layers, dims.d_model, dims.n_q_heads, dims.n_kv_heads, dims.head_dim, dims.d_ffn,
+                            dims.rms_eps, dims.rope_base)
     seed = SEED[name]
     batch = wl.make_batch(name, seed)
     dev = torch.device("cuda", device)
@@ -198,6 +201,8 @@ def main():
     ap.add_argument("--sm-budget", type=int, default=0, help="0 = all SMs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sweep", action="store_true", help="skip the SM-budget sweep and the co-run section")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="profiling aid: cut the workload's stage to this many layers (not a benchmark configuration)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -223,7 +228,7 @@ def main():
         torch.cuda.synchronize()
 
     name = args.workload
-    stage, dims, batch, bt, x = build_stage(name, local_rank)
+    stage, dims, batch, bt, x = build_stage(name, local_rank, layers=args.layers)
     budget = args.sm_budget or stage.sm_count
     T, d = batch.n_tokens, dims.d_model
     dev = stage.device
@@ -373,7 +378,8 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": name, "n_layers": dims.n_layers, "d_model": d, "n_tokens": T,
+            "config": {"workload": name + (f" (cut to {args.layers} layers: profiling only)" if args.layers else ""),
+                       "n_layers": dims.n_layers, "d_model": d, "n_tokens": T,
                        "n_seqs": batch.n_seqs, "prefill_tokens": int(sum(q for q in batch.q_len if q > 1)),
                        "decode_seqs": int(sum(1 for q in batch.q_len if q == 1)), "sm_budget": budget,
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
