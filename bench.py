@@ -34,9 +34,9 @@ from paper_2608_01785_b200 import workloads as wl  # noqa: E402
 METRIC = "shared_stage_tokens_per_s"
 UNIT = "tokens/s"
 SEED = {"c1_tiny": 0, "c2_shared": 1, "c3_7b": 2, "c4_talker": 3, "c3_decode": 2}
-# DRAM bytes (read + write) of one gate/up GEMM launch, from the ncu capture summarised under profiles/
-# (None until a capture of this workload's launch exists).
-GATEUP_DRAM_TRAFFIC_BYTES = {"c2_shared": None}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one gate/up GEMM launch, from the ncu
+# capture summarised in profiles/gemm_gateup_c2_shared.md (None where no capture of that launch exists).
+GATEUP_DRAM_TRAFFIC_BYTES = {"c2_shared": 69852928 + 40344320}
 
 
 def measured_peaks():
