@@ -61,7 +61,7 @@ hs_status_t hs_stage_profile_read(hs_stage_t *stage, float *ms, int32_t *launche
 
 /*
  * Decode attention for callers that cannot allocate device memory.  (The paper has no counterpart
- * to this call: it is a packaging variant of the decode-attention kernels of hs_stage_step.)
+ * to this call: it is a packaging variant of the decode-attention kernel of hs_stage_step.)
  *
  * Who needs it: a process that gave all free HBM to its KV pool at start-up, or a component that only
  * receives device pointers from its host runtime, cannot provide the scratch workspace that the stage
