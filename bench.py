@@ -123,6 +123,21 @@ def build_stage(name: str, device: int, init: str = "n002", layers: int = 0):
     return stage, dims, batch, bt, x
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The slowest rank's device-timed duration: replicas are independent, the job is as slow as its slowest."""
+    if world <= 1:
+        return ms
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tokens_per_s(tokens_per_rank: int, world: int, ms_step_max: float) -> float:
+    """Whole-job throughput of `world` replicas that each process tokens_per_rank tokens per step."""
+    return world * tokens_per_rank / (ms_step_max * 1e-3)
+
+
 def flops_per_step(dims: wl.StageDims, batch: wl.BatchSpec):
     T = batch.n_tokens
     gemm = 2.0 * T * dims.params_per_layer() * dims.n_layers
@@ -245,10 +260,7 @@ def main():
                 fn()
             e1.record(stream)
         barrier()
-        ms = torch.tensor([e0.elapsed_time(e1)], device=dev)
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
+        return max_over_ranks(e0.elapsed_time(e1), world, dev)
 
     step_dev = lambda: stage.step(b, budget, stream)
 
@@ -261,7 +273,7 @@ def main():
     clocks = sampler.stop() if rank == 0 else None
     assert stage.status() == 0, "device status word is set"
     ms_step = ms_total / args.steps
-    value = world * T / (ms_step * 1e-3)
+    value = aggregate_tokens_per_s(T, world, ms_step)
 
     # ---- per-kernel timing (same launches, events around each kernel) ----
     B.hs_stage_profile_enable(stage.handle, True)
@@ -306,14 +318,11 @@ def main():
                 out_done[i].record(s_out)
         e1.record(s_out)
         barrier()
-        ms = torch.tensor([e0.elapsed_time(e1)], device=dev)
-        if world > 1:
-            dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-        return float(ms.item())
+        return max_over_ranks(e0.elapsed_time(e1), world, dev)
 
     e2e_steps(3)
     ms_e2e = e2e_steps(args.steps) / args.steps
-    e2e_value = world * T / (ms_e2e * 1e-3)
+    e2e_value = aggregate_tokens_per_s(T, world, ms_e2e)
 
     # ---- step latency vs SM budget, and the co-run with a downstream stage (rank 0, single GPU) ----
     sweep, corun_rows = None, None
