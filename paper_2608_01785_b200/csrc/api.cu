@@ -396,6 +396,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
   const size_t layer_kv_elems = size_t(c.num_pages) * c.n_kv_heads * kPage * Dh;
   cudaError_t e = cudaSuccess;
   const char* where = "";
+  // More than one 128-row tile of tokens: the GEMMs run on pairs of SMs (a choice by shape, not by budget).
+  const bool use_pair = T > 128;
   int* census = s->census ? reinterpret_cast<int*>(s->ws_dev + s->ws.smid) : nullptr;
   if (census && cudaMemsetAsync(census, 0, size_t(HS_PROFILE_CLASSES) * kSmidSlots * 4, stream) != cudaSuccess)
     return HS_ERR_CUDA;
@@ -423,6 +425,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     g.tm_b[0] = m.wq; g.tm_b[1] = m.wk; g.tm_b[2] = m.wv;
     g.M = T; g.N = q_dim + 2 * kv_dim; g.K = d;
     g.mode = kGemmQkv;
+    g.pair = use_pair;
     g.q_dim = q_dim; g.kv_dim = kv_dim; g.head_dim = Dh; g.n_kv_heads = c.n_kv_heads;
     g.tm_q = s->tm_q_st;
     g.k_cache = s->kv_pool + (size_t(l) * 2 + 0) * layer_kv_elems;
@@ -468,8 +471,9 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     go.M = T; go.N = d; go.K = q_dim;
     go.mode = kGemmResid;
     go.tm_out = tm_y; go.accumulate = 1;
-    go.bn = gemm_pick_bn(T, d, s->sm_count);
-    go.ksplit = pick_ksplit(T, d, q_dim, go.bn, s->sm_count);
+    go.pair = use_pair;
+    go.bn = use_pair ? 256 : gemm_pick_bn(T, d, s->sm_count);
+    go.ksplit = use_pair ? 1 : pick_ksplit(T, d, q_dim, go.bn, s->sm_count);
     go.tile_turn = reinterpret_cast<int*>(s->ws_dev + s->ws.turn);
     go.status = status;
     go.smid_log = slots(5);
@@ -486,6 +490,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gu.tm_b[0] = m.wgate; gu.tm_b[1] = m.wup; gu.tm_b[2] = m.wup;
     gu.M = T; gu.N = F; gu.K = d;
     gu.mode = kGemmGateUp;
+    gu.pair = use_pair;
     gu.tm_act = s->tm_act_st;
     gu.status = status;
     gu.smid_log = slots(6);
@@ -498,8 +503,9 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gd.M = T; gd.N = d; gd.K = F;
     gd.mode = kGemmResid;
     gd.tm_out = tm_y; gd.accumulate = 1;
-    gd.bn = gemm_pick_bn(T, d, s->sm_count);
-    gd.ksplit = pick_ksplit(T, d, F, gd.bn, s->sm_count);
+    gd.pair = use_pair;
+    gd.bn = use_pair ? 256 : gemm_pick_bn(T, d, s->sm_count);
+    gd.ksplit = use_pair ? 1 : pick_ksplit(T, d, F, gd.bn, s->sm_count);
     gd.tile_turn = reinterpret_cast<int*>(s->ws_dev + s->ws.turn);
     gd.status = status;
     gd.smid_log = slots(7);
@@ -590,7 +596,8 @@ hs_status_t hs_op_gemm_bf16(const void* a, const void* w, const float* resid, fl
   g.M = M; g.N = N; g.K = K;
   g.mode = kGemmResid;
   g.accumulate = resid != nullptr;
-  g.bn = gemm_pick_bn(M, N, prop.multiProcessorCount);
+  g.pair = M > 128;
+  g.bn = g.pair ? 256 : gemm_pick_bn(M, N, prop.multiProcessorCount);
   // the kernel adds into `out`: a residual that lives elsewhere is copied there first
   if (resid && resid != out &&
       cudaMemcpyAsync(out, resid, size_t(M) * N * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)

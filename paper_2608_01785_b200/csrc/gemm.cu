@@ -20,15 +20,22 @@
 namespace hs {
 namespace {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int BM = 128, BN = 256, BK = 64;
 constexpr int A_BYTES = BM * BK * 2;            // 16 KB
 constexpr int BH_BYTES = 128 * BK * 2;          // one 128-row half of the B tile, 16 KB
-constexpr int STAGE_BYTES = A_BYTES + 2 * BH_BYTES;
+// One block per tile: a stage holds A and both halves of B, 4 stages.  Block pair per 256 x 256 tile: every
+// block stages A and ONE half of B (the MMA reads the other half from the other block), 6 stages.
+template <bool PAIR> struct Ring {
+  static constexpr int STAGE_BYTES = PAIR ? A_BYTES + BH_BYTES : A_BYTES + 2 * BH_BYTES;
+  static constexpr int STAGES = PAIR ? 6 : 4;
+};
+constexpr int RING_BYTES = 4 * (A_BYTES + 2 * BH_BYTES);
+static_assert(Ring<true>::STAGES * Ring<true>::STAGE_BYTES == RING_BYTES, "both rings fill the same space");
 constexpr int GEMM_THREADS = 192;
 constexpr int TMEM_COLS = 512;                  // two 128 x 256 fp32 accumulators
 constexpr int EPI_BUF_BYTES = 4096;             // 32 rows x 128 B: a 32 x 32 fp32 or 32 x 64 bf16 output block
 constexpr int EPI_WARP_BYTES = 2 * EPI_BUF_BYTES;   // two blocks per epilogue warp, filled alternately
-constexpr int GEMM_SMEM = 1024 + STAGES * STAGE_BYTES + 4 * EPI_WARP_BYTES + 256;
+constexpr int GEMM_SMEM = 1024 + RING_BYTES + 4 * EPI_WARP_BYTES + 256;
 static_assert(GEMM_SMEM <= 227 * 1024, "fits one SM");
 static_assert(GEMM_SMEM >= kMinSmemBytes, "one block per SM");
 
@@ -120,26 +127,33 @@ __device__ __forceinline__ __nv_bfloat16* cache_ptr(__nv_bfloat16* base, int slo
   return base + row * Dh + e;
 }
 
-__global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+template <bool PAIR>
+__device__ __forceinline__ void gemm_body(const GemmParams& p) {
+  constexpr int STAGES = Ring<PAIR>::STAGES, STAGE_BYTES = Ring<PAIR>::STAGE_BYTES;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* epi_smem = smem + STAGES * STAGE_BYTES;
+  uint8_t* epi_smem = smem + RING_BYTES;
   uint64_t* full = reinterpret_cast<uint64_t*>(epi_smem + 4 * EPI_WARP_BYTES);
-  uint64_t* empty = full + STAGES;
-  uint64_t* tfull = empty + STAGES;
+  uint64_t* empty = full + 6;
+  uint64_t* tfull = empty + 6;
   uint64_t* tempty = tfull + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   log_smid(p.smid_log);
-  const int n_m_tiles = (p.M + BM - 1) / BM;
+  // In pair mode the two blocks of a cluster share every work unit: a unit's tile is 256 rows tall and
+  // block `rank` owns rows 128 * rank .. 128 * rank + 127 of it.
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0;
+  const int worker = PAIR ? int(blockIdx.x >> 1) : int(blockIdx.x);
+  const int n_workers = PAIR ? int(gridDim.x >> 1) : int(gridDim.x);
+  const int n_m_tiles = PAIR ? (p.M + 2 * BM - 1) / (2 * BM) : (p.M + BM - 1) / BM;
   const int n_n_tiles = gemm_n_tiles(p);
   const int n_tiles = n_m_tiles * n_n_tiles;
   const int k_blocks = (p.K + BK - 1) / BK;
   // Work unit = (output tile, K split).  Splits exist only in Resid mode with few tiles; units are ordered
   // split-major, so the units a split has to wait for always have smaller indices.
-  const int ksplit = p.mode == kGemmResid && p.ksplit > 1 ? p.ksplit : 1;
+  const int ksplit = !PAIR && p.mode == kGemmResid && p.ksplit > 1 ? p.ksplit : 1;
   const int kb_per = (k_blocks + ksplit - 1) / ksplit;
   const int n_units = n_tiles * ksplit;
 
@@ -150,7 +164,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&tfull[i], 1);
-      mbar_init(&tempty[i], 128);
+      mbar_init(&tempty[i], PAIR ? 8 : 4);      // one arrival per epilogue warp (of both blocks)
     }
     *abort_flag = 0;
     fence_barrier_init();
@@ -159,11 +173,17 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     tma_prefetch_desc(p.mode == kGemmResid ? &p.tm_out : p.mode == kGemmQkv ? &p.tm_q : &p.tm_act);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, TMEM_COLS);
-    tmem_relinquish();
+    if (PAIR) {
+      tmem_alloc_pair(tmem_slot, TMEM_COLS);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc(tmem_slot, TMEM_COLS);
+      tmem_relinquish();
+    }
   }
   tc_fence_before_sync();
   __syncthreads();
+  if (PAIR) cluster_sync_all();               // the other block's barriers exist before anything targets them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -174,30 +194,38 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
       uint32_t ph = 0;
       bool ok = true;
       const bool two_halves = p.mode != kGemmResid || p.bn > 128;
-      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+      for (int u = worker; u < n_units && ok; u += n_workers) {
         const int tile = u % n_tiles, ks = u / n_tiles;
         const int m = tile % n_m_tiles, n = tile / n_m_tiles;
-        const BSource b0 = b_source(p, n, 0), b1 = b_source(p, n, 1);
+        const BSource b0 = b_source(p, n, PAIR ? int(rank) : 0), b1 = b_source(p, n, 1);
         const int kb_end = min(k_blocks, (ks + 1) * kb_per);
         for (int kb = ks * kb_per; kb < kb_end; ++kb) {
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status)) { ok = false; break; }
           uint8_t* st = smem + s * STAGE_BYTES;
-          mbar_expect_tx(&full[s], two_halves ? STAGE_BYTES : A_BYTES + BH_BYTES);
-          tma_load_2d(st, &p.tm_a, &full[s], kb * BK, m * BM);
-          tma_load_2d(st + A_BYTES, &p.tm_b[b0.map], &full[s], kb * BK, b0.row);
-          if (two_halves) tma_load_2d(st + A_BYTES + BH_BYTES, &p.tm_b[b1.map], &full[s], kb * BK, b1.row);
+          if (PAIR) {
+            // both blocks' bytes are counted on the leader's barrier, which the leader arms for both
+            const uint32_t bar = mapa_u32(smem_u32(&full[s]), 0);
+            if (rank == 0) mbar_expect_tx(&full[s], 2 * STAGE_BYTES);
+            tma_load_2d_pair(st, &p.tm_a, bar, kb * BK, (2 * m + int(rank)) * BM);
+            tma_load_2d_pair(st + A_BYTES, &p.tm_b[b0.map], bar, kb * BK, b0.row);
+          } else {
+            mbar_expect_tx(&full[s], two_halves ? STAGE_BYTES : A_BYTES + BH_BYTES);
+            tma_load_2d(st, &p.tm_a, &full[s], kb * BK, m * BM);
+            tma_load_2d(st + A_BYTES, &p.tm_b[b0.map], &full[s], kb * BK, b0.row);
+            if (two_halves) tma_load_2d(st + A_BYTES + BH_BYTES, &p.tm_b[b1.map], &full[s], kb * BK, b1.row);
+          }
           if (++s == STAGES) { s = 0; ph ^= 1; }
         }
       }
     }
   } else if (warp == 1) {
     // --------------------------------------------------------- MMA issuer --
-    if (lane == 0) {
-      const uint32_t idesc = umma_idesc_bf16_f32(BM, p.mode == kGemmResid ? p.bn : BN);
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = umma_idesc_bf16_f32(PAIR ? 2 * BM : BM, p.mode == kGemmResid && !PAIR ? p.bn : BN);
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+      for (int u = worker; u < n_units && ok; u += n_workers) {
         if (!mbar_wait(&tempty[acc], acc_ph ^ 1, abort_flag, p.status)) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
@@ -209,12 +237,27 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
           const uint64_t a_desc = umma_desc_kmajor_sw128(a_addr);
           const uint64_t b_desc = umma_desc_kmajor_sw128(a_addr + A_BYTES);
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)   // 16 bf16 = 32 B along K: +2 in the (address / 16) field
-            umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, ((kb - kb_begin) | k) != 0);
-          umma_commit(&empty[s]);             // frees the stage once these MMAs have read it
+          for (int k = 0; k < BK / 16; ++k) {  // 16 bf16 = 32 B along K: +2 in the (address / 16) field
+            if (PAIR) umma_bf16_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, ((kb - kb_begin) | k) != 0);
+            else umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, ((kb - kb_begin) | k) != 0);
+          }
+          // frees the stage (in both blocks) once these MMAs have read it
+          if (PAIR) {
+            umma_commit_pair(mapa_u32(smem_u32(&empty[s]), 0));
+            umma_commit_pair(mapa_u32(smem_u32(&empty[s]), 1));
+          } else {
+            umma_commit(&empty[s]);
+          }
           if (++s == STAGES) { s = 0; ph ^= 1; }
         }
-        if (ok) umma_commit(&tfull[acc]);
+        if (ok) {
+          if (PAIR) {
+            umma_commit_pair(mapa_u32(smem_u32(&tfull[acc]), 0));
+            umma_commit_pair(mapa_u32(smem_u32(&tfull[acc]), 1));
+          } else {
+            umma_commit(&tfull[acc]);
+          }
+        }
         acc ^= 1;
         if (acc == 0) acc_ph ^= 1;
       }
@@ -227,9 +270,9 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
     const int Dh = p.head_dim;
     uint8_t* epi_buf = epi_smem + quarter * EPI_WARP_BYTES;
     int epi_sel = 0;                          // staging block to fill next
-    for (int u = blockIdx.x; u < n_units; u += gridDim.x) {
+    for (int u = worker; u < n_units; u += n_workers) {
       const int tile = u % n_tiles, ks = u / n_tiles;
-      const int m = tile % n_m_tiles, n = tile / n_m_tiles;
+      const int m = PAIR ? 2 * (tile % n_m_tiles) + int(rank) : tile % n_m_tiles, n = tile / n_m_tiles;
       const bool ok = mbar_wait(&tfull[acc], acc_ph, abort_flag, p.status);
       if (!__all_sync(0xffffffffu, ok)) break;
       tc_fence_after_sync();
@@ -369,8 +412,13 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
           }
         }
       }
+      // this warp has drained its rows of the accumulator: tell the MMA issuer (in the leader block)
       tc_fence_before_sync();
-      mbar_arrive(&tempty[acc]);
+      __syncwarp();
+      if (lane == 0) {
+        if (PAIR) mbar_arrive_cluster(mapa_u32(smem_u32(&tempty[acc]), 0));
+        else mbar_arrive(&tempty[acc]);
+      }
       acc ^= 1;
       if (acc == 0) acc_ph ^= 1;
     }
@@ -382,15 +430,28 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_cons
   if (*abort_flag) drain_after_abort();
   tc_fence_before_sync();
   __syncthreads();
+  if (PAIR) cluster_sync_all();               // neither block leaves while the other may still reach into it
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, TMEM_COLS);
+    if (PAIR) tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    else tmem_dealloc(tmem_base, TMEM_COLS);
   }
+}
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1) gemm_kernel(const __grid_constant__ GemmParams p) {
+  gemm_body<false>(p);
+}
+// Two blocks per cluster, one 256 x 256 tile per pair.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
+    gemm_pair_kernel(const __grid_constant__ GemmParams p) {
+  gemm_body<true>(p);
 }
 
 }  // namespace
 
 cudaError_t gemm_set_attributes() {
+  cudaError_t e = cudaFuncSetAttribute(gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
+  if (e != cudaSuccess) return e;
   return cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
 }
 
@@ -433,6 +494,13 @@ cudaError_t launch_gemm(const GemmParams& p, int sm_budget, cudaStream_t stream)
   const int n_n_tiles = gemm_n_tiles(p);
   const int n_tiles = n_m_tiles * n_n_tiles * (p.mode == kGemmResid && p.ksplit > 1 ? p.ksplit : 1);
   if (n_tiles <= 0) return cudaSuccess;
+  if (p.pair && sm_budget >= 2) {
+    // pairs of blocks (clusters of two SMs) on 256 x 256 tiles; an odd budget leaves one SM unused
+    const int pairs = ((p.M + 2 * BM - 1) / (2 * BM)) * n_n_tiles;
+    const int grid = 2 * (pairs < sm_budget / 2 ? pairs : sm_budget / 2);
+    gemm_pair_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(p);
+    return cudaGetLastError();
+  }
   const int grid = n_tiles < sm_budget ? n_tiles : sm_budget;
   gemm_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(p);
   return cudaGetLastError();

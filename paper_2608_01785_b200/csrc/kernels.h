@@ -27,6 +27,7 @@ struct GemmParams {
   CUtensorMap tm_b[3];       // weights, box 64 x 128: Resid {W}, Qkv {Wq, Wk, Wv}, GateUp {Wgate, Wup}
   int M, N, K;               // N: Resid output width; Qkv (Hq + 2 Hkv) * Dh; GateUp F (activation width)
   int mode;
+  int pair;                  // 1: run on pairs of SMs (256 x 256 tiles, bn = 256, no K split) when the budget allows
   // Resid
   CUtensorMap tm_out;        // fp32 [M, N], box 32 x 32, 128-byte swizzle (rows past M are clipped)
   int accumulate;            // 1: out += A W^T (the residual add), 0: out = A W^T
