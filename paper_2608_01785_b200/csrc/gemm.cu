@@ -1,14 +1,23 @@
 // Persistent, SM-budgeted bf16 GEMM on the 5th-generation tensor cores (tcgen05) with the step's
 // element-wise work fused into its epilogues.
 //
-//   tile        128 (tokens) x 256 (output columns), K consumed in blocks of 64
-//   operands    TMA (128-byte swizzle) -> 4-stage shared-memory ring -> tcgen05.mma, fp32 accumulators
-//               in tensor memory, two accumulator buffers so the epilogue of tile i overlaps the main
-//               loop of tile i+1
-//   roles       warp 0: TMA producer, warp 1: MMA issuer (one thread), warps 2..5: epilogue
-//   schedule    tile = blockIdx.x + i * gridDim.x, gridDim.x <= sm_budget, one block per SM.  Each output
-//               tile is produced by exactly one block with a fixed K order, so results do not depend on
-//               the budget.
+//   tile        pair kernel (more than 128 tokens): 256 x 256 per PAIR of blocks (a cluster of two SMs,
+//               tcgen05.mma.cta_group::2): each block stages its 128 token rows of A and ONE 128-row half
+//               of B per 64-wide K block (32 KB, 6-stage ring), the leader block issues M256 N256 K16 MMAs
+//               that read both blocks' shared memory, and each block owns the accumulator rows of its
+//               SM's tensor memory.  Halving the B bytes per SM is what lifts the operand-feed limit of the
+//               single-block kernel (128 x 256 tile, 48 KB per K block, 4-stage ring), which remains for
+//               small token counts, for sm_budget 1 and for the K-split path; both produce the same bits.
+//   operands    TMA (128-byte swizzle) -> shared-memory ring -> tcgen05.mma, fp32 accumulators in tensor
+//               memory, two accumulator buffers so the epilogue of tile i overlaps the main loop of i+1
+//   roles       warp 0: TMA producer, warp 1: MMA issuer (one thread, leader block only), warps 2..5:
+//               epilogue.  Cross-block signalling in a pair: both blocks' TMA bytes are counted on the
+//               leader's "full" barrier; the leader's tcgen05.commit arrives on the "empty" and
+//               "accumulator full" barriers of both blocks; epilogue warps of both blocks arrive on the
+//               leader's "accumulator empty" barrier.
+//   schedule    unit = worker + i * workers, workers <= sm_budget (pairs: sm_budget / 2), one block per
+//               SM.  Each output tile is produced by one block (pair) with a fixed K order, so results do
+//               not depend on the budget.
 //
 // Epilogues: residual add (the fp32 tile is ADDED into the residual stream by a TMA reduction, so the
 // stream is never read by the SM), QKV (rotate-half RoPE; bf16 q by TMA store; k, v scattered into the
