@@ -94,7 +94,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_stage(name: str, device: int, init: str = "n002", layers: int = 0):
+def build_stage(name: str, device: int, init: str = "n002", layers: int = 0, flags: int = 0):
     """Weights, KV pool with random-filled context, block tables and input of the named workload."""
     from paper_2608_01785_b200.stage import Stage
     dims = wl.DIMS[name]
@@ -107,7 +107,7 @@ def build_stage(name: str, device: int, init: str = "n002", layers: int = 0):
     weights = wl.make_weights(dims, seed, dev, init)
     num_pages = wl.pages_needed(batch) + 8
     mpps = max(-(-t // 16) for t in batch.total_len())
-    stage = Stage(dims, weights, num_pages, batch.n_tokens, batch.n_seqs, mpps, max(batch.total_len()), device)
+    stage = Stage(dims, weights, num_pages, batch.n_tokens, batch.n_seqs, mpps, max(batch.total_len()), device, flags)
     # context of the decode sequences: values do not change the timing; N(0,1) bf16 stands in for K/V
     # written by earlier steps
     g = torch.Generator(device=dev)
@@ -215,6 +215,8 @@ def main():
     ap.add_argument("--workload", default="c2_shared", choices=sorted(SEED))
     ap.add_argument("--sm-budget", type=int, default=0, help="0 = all SMs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--bf16-activations", action="store_true",
+                    help="stage flag HS_FLAG_BF16_ACTIVATIONS: h, o, act in bf16, no fp16 weight copies")
     ap.add_argument("--no-sweep", action="store_true", help="skip the SM-budget sweep and the co-run section")
     ap.add_argument("--layers", type=int, default=0,
                     help="profiling aid: cut the workload's stage to this many layers (not a benchmark configuration)")
@@ -243,7 +245,7 @@ def main():
         torch.cuda.synchronize()
 
     name = args.workload
-    stage, dims, batch, bt, x = build_stage(name, local_rank, layers=args.layers)
+    stage, dims, batch, bt, x = build_stage(name, local_rank, layers=args.layers, flags=1 if args.bf16_activations else 0)
     budget = args.sm_budget or stage.sm_count
     T, d = batch.n_tokens, dims.d_model
     dev = stage.device
@@ -360,7 +362,7 @@ def main():
     gemm_flops, attn_flops = flops_per_step(dims, batch)
     roofline = {"bound": "tensor", "kernel": "gemm_kernel (gate/up + SwiGLU epilogue)", "achieved": achieved,
                 "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                "peak_source": f"{peaks['source']} sustained bf16 x sm_budget/{stage.sm_count}",
+                "peak_source": f"{peaks['source']} sustained bf16 (fp16 operands: nominal ratio 1.0) x sm_budget/{stage.sm_count}",
                 "frac_of_burst_peak": achieved / (peaks["bf16_burst"] * budget / stage.sm_count),
                 "traffic": GATEUP_DRAM_TRAFFIC_BYTES.get(name),
                 "avg_launch_ms": gu_avg_s * 1e3, "launches": gu_n,
@@ -392,7 +394,11 @@ def main():
                        "n_seqs": batch.n_seqs, "prefill_tokens": int(sum(q for q in batch.q_len if q > 1)),
                        "decode_seqs": int(sum(1 for q in batch.q_len if q == 1)), "sm_budget": budget,
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
-                       "l2": "inputs larger than L2: weights + KV read per step exceed the 126 MB L2"},
+                       "l2": "inputs larger than L2: weights + KV read per step exceed the 126 MB L2",
+                       "formats": "all-bf16 operands (HS_FLAG_BF16_ACTIVATIONS); fp32 accumulation" if
+                                  args.bf16_activations else
+                                  "bf16 x_in, weights, KV cache, q and softmax weights; fp16 h, o, act against fp16 "
+                                  "copies of the weights; fp32 accumulation, residual stream and output"},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e, "h2d_bytes_per_step": T * d * 2,
                     "d2h_bytes_per_step": T * d * 4},

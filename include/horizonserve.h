@@ -22,10 +22,21 @@
  *     in the paged cache;  o = causal GQA attention of q over cache positions
  *     0..p (query head hq reads KV head hq / (Hq/Hkv));  x += o Wo^T;
  *     h2 = rmsnorm(x, g_mlp);  x += (silu(h2 Wg^T) * (h2 Wu^T)) Wd^T.
- * Numeric contract: bf16 storage and tensor-core operands, fp32 accumulation,
- * fp32 residual stream and fp32 output; every fp32 -> bf16 conversion rounds
- * to nearest even; inputs must be finite.  Outputs and the bytes written to
- * the KV cache are bit-identical for every valid sm_budget.
+ * Numeric contract: everything that crosses this interface is bf16 storage
+ * (x_in, weights, the KV cache) except the fp32 output; accumulation is fp32
+ * and the residual stream is fp32.  Inside a step q, K, V and the softmax
+ * weights are bf16; the activations that are multiplied with the weights (h,
+ * the attention output, the SwiGLU activation) are private to the stage and
+ * are held in fp16 (11 significand bits, clamped to +-65504) and multiplied
+ * with fp16 copies of the weights that hs_stage_create makes in the workspace
+ * (one MMA cannot mix fp16 with bf16; a bf16 weight is an fp16 value exactly
+ * when 2^-17 <= |w| <= 65504, smaller ones move by at most 2^-25), which
+ * keeps a multi-layer step within the 2e-2 RMS tolerance.
+ * HS_FLAG_BF16_ACTIVATIONS keeps those activations in bf16 and reads the
+ * caller's bf16 weights directly: no copies, a smaller workspace, the 8-bit
+ * significand's larger error.  Every
+ * conversion rounds to nearest even; inputs must be finite.  Outputs and the
+ * bytes written to the KV cache are bit-identical for every valid sm_budget.
  *
  * Conventions
  *  - No call allocates device memory: the caller (PyTorch in this repository)
@@ -57,6 +68,10 @@ extern "C" {
 
 #define HS_ABI_VERSION 1u
 #define HS_PAGE_SIZE 16 /* tokens per KV page; the only supported value */
+/* Stage flag: keep the private activations that feed the projections (h, attention output o, SwiGLU
+ * activation act) in bf16 instead of the default fp16, and make no fp16 copies of the weights -- see the
+ * numeric contract above. */
+#define HS_FLAG_BF16_ACTIVATIONS 1u
 
 typedef struct hs_stage hs_stage_t; /* opaque; owned by the library */
 
@@ -85,7 +100,7 @@ typedef struct {
   int32_t max_seqs;          /* most sequences in one step */
   int32_t max_pages_per_seq; /* row length of block tables */
   int32_t max_position;      /* ctx_len + q_len never exceeds this (sizes the RoPE table) */
-  uint32_t flags;            /* must be 0 */
+  uint32_t flags;            /* 0, or HS_FLAG_BF16_ACTIVATIONS */
 } hs_stage_config_t;
 
 /* One layer's weights: device pointers to bf16, row-major [out_features, in_features], no bias. */
@@ -117,7 +132,9 @@ typedef struct {
  *  KV pool: bf16 [n_layers][2 (K,V)][num_pages][n_kv_heads][16][head_dim]; K is stored after RoPE.
  *           One (page, head) block is 16*head_dim*2 contiguous bytes.  Must be 256-byte aligned (what cudaMalloc gives).
  *  Workspace: private scratch of the stage (activations, RoPE table, step metadata, attention
- *           partials).  Must be 256-byte aligned (what cudaMalloc gives).  Its contents are meaningless to the caller.
+ *           partials and, unless HS_FLAG_BF16_ACTIVATIONS is set, fp16 copies of all projection weights, i.e.
+ *           as many bytes again as those weights).  Must be 256-byte aligned (what cudaMalloc gives).  Its
+ *           contents are meaningless to the caller.
  * Both return 0 for an invalid configuration.
  */
 size_t hs_kv_pool_bytes(const hs_stage_config_t *cfg);
@@ -128,7 +145,9 @@ size_t hs_workspace_bytes(const hs_stage_config_t *cfg);
  * kv_pool_dev and workspace_dev are device buffers of at least the sizes above.  All of them stay
  * owned by the caller and must outlive the stage.  With cfg->device == -1 every device pointer may be
  * NULL and the stage supports only hs_kv_alloc / hs_kv_free / hs_stage_plan.
- * The call synchronises the device once (it uploads the RoPE table).
+ * The call reads the weights on the device's default stream (it makes the fp16 copies there) and
+ * synchronises the device once, so the weights must be complete when it is made; the stage does not see
+ * later changes to them unless HS_FLAG_BF16_ACTIVATIONS is set.
  * Errors: INVALID_ARG, UNSUPPORTED_SHAPE, CUDA.
  */
 hs_status_t hs_stage_create(const hs_stage_config_t *cfg, const hs_layer_weights_t *layers, void *kv_pool_dev,

@@ -30,12 +30,19 @@ hs_status_t hs_op_gemm_bf16(const void *a, const void *w, const float *resid, fl
                             int32_t K, int32_t sm_budget, int32_t *status_dev, void *cuda_stream);
 
 /*
+ * The same contraction with `a` and `w` both holding fp16 (IEEE half) values: the form the stage uses by
+ * default, its private activations in fp16 (an 11-bit significand) against fp16 copies of the weights.
+ */
+hs_status_t hs_op_gemm_f16(const void *a, const void *w, const float *resid, float *out, int32_t M, int32_t N,
+                           int32_t K, int32_t sm_budget, int32_t *status_dev, void *cuda_stream);
+
+/*
  * Diagnosis: device address and size of one of the stage's private intermediates after a step
  * (contents of the LAST layer executed).  name is one of
- *   "h"   bf16 [max_tokens, d]      last RMSNorm output
- *   "q"   bf16 [max_tokens, Hq*Dh]  queries after RoPE
- *   "o"   bf16 [max_tokens, Hq*Dh]  attention output
- *   "act" bf16 [max_tokens, F]      silu(gate) * up
+ *   "h"   [max_tokens, d]      last RMSNorm output            (fp16; bf16 with HS_FLAG_BF16_ACTIVATIONS)
+ *   "q"   [max_tokens, Hq*Dh]  queries after RoPE             (bf16)
+ *   "o"   [max_tokens, Hq*Dh]  attention output               (fp16; bf16 with the flag)
+ *   "act" [max_tokens, F]      silu(gate) * up                (fp16; bf16 with the flag)
  *   "smid" int32 [8 classes][160]   SM census: asking for this buffer switches the census on for the
  *                                   following steps; entry [class][b] is then 1 + the SM on which block b
  *                                   of the last layer's launch of that kernel class ran (0 = no such

@@ -55,8 +55,9 @@ typedef struct {
 } hso_layer_t;
 
 /* Diagnostic switch (never the pass/fail oracle): bit mask of intermediates
- * that are rounded to bf16 the way a bf16-operand tensor-core path would.
- * 1: h (both norms)  2: q  4: softmax weights P  8: o  16: act */
+ * that are rounded the way a 16-bit-operand tensor-core path would.
+ * 1: h (both norms)  2: q  4: softmax weights P  8: o  16: act
+ * 32: round h, o and act to fp16 (clamped to +-65504) instead of bf16 */
 static int g_round_mask = 0;
 void hso_set_operand_rounding(int mask) { g_round_mask = mask; }
 int hso_sizeof_real(void) { return (int)sizeof(real); }
@@ -80,6 +81,14 @@ float hso_bf16_to_float(uint16_t b) {
 static inline real round_bf16(real v) {
   return (real)hso_bf16_to_float(hso_bf16_rne((float)v));
 }
+static inline real round_f16(real v) {
+  float f = (float)v;
+  if (f > 65504.f) f = 65504.f;
+  if (f < -65504.f) f = -65504.f;
+  return (real)(float)(_Float16)f;
+}
+/* rounding of the activations that feed the projections (h, o, act) */
+static inline real round_act(real v) { return (g_round_mask & 32) ? round_f16(v) : round_bf16(v); }
 
 /* ------------------------------------------------------------- RMSNorm -- */
 /* h[t,i] = x[t,i] * r_t * g[i],  r_t = 1/sqrt(mean_i x[t,i]^2 + eps). */
@@ -224,7 +233,7 @@ int hso_layer(const hso_config_t *c, const hso_layer_t *w, int layer, uint16_t *
   real *h = (real *)malloc(sizeof(real) * (size_t)T * d);
   hso_rmsnorm(T, d, x, w->g_attn, c->rms_eps, h);
   if (g_round_mask & 1)
-    for (size_t i = 0; i < (size_t)T * d; ++i) h[i] = round_bf16(h[i]);
+    for (size_t i = 0; i < (size_t)T * d; ++i) h[i] = round_act(h[i]);
 
   /* 2. k, v of every token; RoPE on k; cache write (before any attention) */
   int KVd = Hkv * Dh;
@@ -279,7 +288,7 @@ int hso_layer(const hso_config_t *c, const hso_layer_t *w, int layer, uint16_t *
     }
   free(q);
   if (g_round_mask & 8)
-    for (size_t i = 0; i < (size_t)R * Qd; ++i) o[i] = round_bf16(o[i]);
+    for (size_t i = 0; i < (size_t)R * Qd; ++i) o[i] = round_act(o[i]);
 
   /* 5. output projection + residual */
   real *xR = (real *)malloc(sizeof(real) * (size_t)R * d), *tmp = (real *)malloc(sizeof(real) * (size_t)R * d);
@@ -291,13 +300,13 @@ int hso_layer(const hso_config_t *c, const hso_layer_t *w, int layer, uint16_t *
   /* 6. MLP norm, SwiGLU */
   hso_rmsnorm(R, d, xR, w->g_mlp, c->rms_eps, hR);
   if (g_round_mask & 1)
-    for (size_t i = 0; i < (size_t)R * d; ++i) hR[i] = round_bf16(hR[i]);
+    for (size_t i = 0; i < (size_t)R * d; ++i) hR[i] = round_act(hR[i]);
   real *gate = (real *)malloc(sizeof(real) * (size_t)R * F), *up = (real *)malloc(sizeof(real) * (size_t)R * F);
   hso_linear(R, F, d, hR, w->w_gate, gate);
   hso_linear(R, F, d, hR, w->w_up, up);
   for (size_t i = 0; i < (size_t)R * F; ++i) {
     gate[i] = hso_silu(gate[i]) * up[i];
-    if (g_round_mask & 16) gate[i] = round_bf16(gate[i]);
+    if (g_round_mask & 16) gate[i] = round_act(gate[i]);
   }
   free(up);
   free(hR);

@@ -24,6 +24,7 @@ _LIBS: Dict[str, C.CDLL] = {}
 
 ROUND_H, ROUND_Q, ROUND_P, ROUND_O, ROUND_ACT = 1, 2, 4, 8, 16
 ROUND_ALL = 31
+ROUND_ACT_F16 = 32          # with ROUND_H / ROUND_O / ROUND_ACT: those three go to fp16 instead of bf16
 
 
 def lib_path(precision: str) -> str:

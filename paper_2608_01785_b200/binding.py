@@ -16,13 +16,14 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhorizonserve.so")
 
 HS_ABI_VERSION = 1
+HS_FLAG_BF16_ACTIVATIONS = 1      # hs_stage_config_t.flags: keep h, o and act in bf16 instead of fp16
 HS_OK, HS_ERR_INVALID_ARG, HS_ERR_INVALID_BUDGET, HS_ERR_UNSUPPORTED_SHAPE, HS_ERR_OUT_OF_PAGES, \
     HS_ERR_BAD_BLOCK_TABLE, HS_ERR_CUDA, HS_ERR_TIMEOUT, HS_ERR_NO_DEVICE, HS_ERR_UNKNOWN_SEQ = range(10)
 
 EXPORTS = ("hs_status_str", "hs_kv_pool_bytes", "hs_workspace_bytes", "hs_stage_create", "hs_stage_destroy",
            "hs_kv_alloc", "hs_kv_free", "hs_kv_free_pages", "hs_stage_plan", "hs_stage_step", "hs_stage_status",
            "hs_stage_sm_count", "hs_op_gemm_bf16", "hs_stage_debug_buffer", "hs_stage_profile_enable",
-           "hs_stage_profile_read", "hs_last_error", "hs_op_decode_attention_noalloc")
+           "hs_stage_profile_read", "hs_last_error", "hs_op_decode_attention_noalloc", "hs_op_gemm_f16")
 PROFILE_CLASSES = ("rmsnorm", "gemm_qkv", "attn_prefill", "attn_decode", "attn_combine", "gemm_out", "gemm_gateup",
                    "gemm_down")
 
@@ -87,6 +88,7 @@ def lib() -> C.CDLL:
         l.hs_stage_sm_count.restype = C.c_int32
         l.hs_op_gemm_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                       C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+        l.hs_op_gemm_f16.argtypes = l.hs_op_gemm_bf16.argtypes
         l.hs_stage_debug_buffer.argtypes = [C.c_void_p, C.c_char_p, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
         l.hs_last_error.restype = C.c_char_p
         l.hs_op_decode_attention_noalloc.argtypes = [C.c_void_p, C.c_void_p] + [C.c_int32] * 7 + \
@@ -102,11 +104,11 @@ def status_str(status: int) -> str:
 
 
 def make_config(dims, num_pages: int, max_tokens: int, max_seqs: int, max_pages_per_seq: int, max_position: int,
-                device: int = 0) -> hs_stage_config_t:
+                device: int = 0, flags: int = 0) -> hs_stage_config_t:
     """dims: any object with n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, rms_eps, rope_base, page_size."""
     return hs_stage_config_t(HS_ABI_VERSION, device, dims.n_layers, dims.d_model, dims.n_q_heads, dims.n_kv_heads,
                              dims.head_dim, dims.d_ffn, dims.rms_eps, dims.rope_base, dims.page_size, num_pages,
-                             max_tokens, max_seqs, max_pages_per_seq, max_position, 0)
+                             max_tokens, max_seqs, max_pages_per_seq, max_position, flags)
 
 
 def hs_kv_pool_bytes(cfg: hs_stage_config_t) -> int:
@@ -203,8 +205,10 @@ def hs_stage_debug_buffer(stage: int, name: str):
 
 
 def hs_op_gemm_bf16(a_ptr: int, w_ptr: int, resid_ptr: int, out_ptr: int, M: int, N: int, K: int, sm_budget: int,
-                    status_ptr: int, cuda_stream: int = 0) -> None:
-    st = lib().hs_op_gemm_bf16(C.c_void_p(a_ptr), C.c_void_p(w_ptr), C.c_void_p(resid_ptr or None), C.c_void_p(out_ptr),
+                    status_ptr: int, cuda_stream: int = 0, a_is_f16: bool = False) -> None:
+    """out = a w^T (+ resid).  a_is_f16 selects the fp16-activation form (hs_op_gemm_f16)."""
+    fn = lib().hs_op_gemm_f16 if a_is_f16 else lib().hs_op_gemm_bf16
+    st = fn(C.c_void_p(a_ptr), C.c_void_p(w_ptr), C.c_void_p(resid_ptr or None), C.c_void_p(out_ptr),
                                M, N, K, sm_budget, C.c_void_p(status_ptr), C.c_void_p(cuda_stream))
     if st != HS_OK:
         raise HsError(st, "hs_op_gemm_bf16")
@@ -222,7 +226,7 @@ def hs_stage_profile_read(stage: int):
     n = np.zeros(len(PROFILE_CLASSES), dtype=np.int32)
     st = lib().hs_stage_profile_read(C.c_void_p(stage), ms.ctypes.data, n.ctypes.data)
     if st != HS_OK:
-        raise HsError(st, "hs_stage_profile_read", "hs_last_error", "hs_op_decode_attention_noalloc")
+        raise HsError(st, "hs_stage_profile_read")
     return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(PROFILE_CLASSES)}
 
 

@@ -18,8 +18,16 @@ namespace {
 constexpr int kRing = 4;   // pinned staging slots for step metadata
 
 struct WsLayout {
-  size_t rope, h, q, o, act, meta, part_o, part_ml, status, turn, smid, total;
+  size_t rope, h, q, o, act, meta, part_o, part_ml, status, turn, smid, w16, w16_layer, total;
 };
+
+// elements of the i-th weight matrix of a layer, in the order w_q, w_k, w_v, w_o, w_gate, w_up, w_down
+size_t weight_elems(const hs_stage_config_t& c, int i) {
+  const size_t d = c.d_model, F = c.d_ffn, q_dim = size_t(c.n_q_heads) * c.head_dim,
+               kv_dim = size_t(c.n_kv_heads) * c.head_dim;
+  const size_t n[7] = {q_dim * d, kv_dim * d, kv_dim * d, d * q_dim, F * d, F * d, d * F};
+  return n[i];
+}
 
 WsLayout make_ws_layout(const hs_stage_config_t& c, const MetaLayout& ml) {
   WsLayout w{};
@@ -41,6 +49,14 @@ WsLayout make_ws_layout(const hs_stage_config_t& c, const MetaLayout& ml) {
   w.status = take(256);
   w.turn = take(kGemmTurnWords * 4);
   w.smid = take(size_t(HS_PROFILE_CLASSES) * kSmidSlots * 4);
+  // fp16 copies of the seven weight matrices of every layer (absent with HS_FLAG_BF16_ACTIVATIONS);
+  // within a layer: w_q, w_k, w_v, w_o, w_gate, w_up, w_down, each 1024-byte aligned
+  w.w16 = off;
+  w.w16_layer = 0;
+  if (!(c.flags & HS_FLAG_BF16_ACTIVATIONS)) {
+    for (int i = 0; i < 7; ++i) w.w16_layer += align_up(weight_elems(c, i) * 2, 1024);
+    take(w.w16_layer * size_t(c.n_layers));
+  }
   w.total = off;
   return w;
 }
@@ -279,7 +295,19 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
   s->maps.resize(cfg->n_layers);
   for (int l = 0; l < cfg->n_layers && ok; ++l) {
     LayerMaps& m = s->maps[l];
-    const hs_layer_weights_t& w = s->layers[l];
+    hs_layer_weights_t w = s->layers[l];
+    if (!(cfg->flags & HS_FLAG_BF16_ACTIVATIONS)) {
+      // the projections read fp16 copies of the weights, made here once
+      const void* src[7] = {w.w_q, w.w_k, w.w_v, w.w_o, w.w_gate, w.w_up, w.w_down};
+      const void** dst[7] = {&w.w_q, &w.w_k, &w.w_v, &w.w_o, &w.w_gate, &w.w_up, &w.w_down};
+      uint8_t* at = s->ws_dev + s->ws.w16 + s->ws.w16_layer * size_t(l);
+      for (int i = 0; i < 7 && ok; ++i) {
+        ok = launch_bf16_to_f16(src[i], at, weight_elems(*cfg, i), nullptr) == cudaSuccess;
+        *dst[i] = at;
+        at += align_up(weight_elems(*cfg, i) * 2, 1024);
+      }
+      if (!ok) break;
+    }
     ok = encode_2d(&m.wq, w.w_q, q_dim, d, 128) && encode_2d(&m.wk, w.w_k, kv_dim, d, 128) &&
          encode_2d(&m.wv, w.w_v, kv_dim, d, 128) && encode_2d(&m.wo, w.w_o, d, q_dim, 128) &&
          encode_2d(&m.wgate, w.w_gate, F, d, 128) && encode_2d(&m.wup, w.w_up, F, d, 128) &&
@@ -398,6 +426,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
   const char* where = "";
   // More than one 128-row tile of tokens: the GEMMs run on pairs of SMs (a choice by shape, not by budget).
   const bool use_pair = T > 128;
+  const int f16 = (c.flags & HS_FLAG_BF16_ACTIVATIONS) ? 0 : 1;   // format of h, o, act
   int* census = s->census ? reinterpret_cast<int*>(s->ws_dev + s->ws.smid) : nullptr;
   if (census && cudaMemsetAsync(census, 0, size_t(HS_PROFILE_CLASSES) * kSmidSlots * 4, stream) != cudaSuccess)
     return HS_ERR_CUDA;
@@ -416,6 +445,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     np.T = T;
     np.d = d;
     np.eps = c.rms_eps;
+    np.h_f16 = f16;
     np.smid_log = slots(0);
     { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
     if (e != cudaSuccess) break;
@@ -425,6 +455,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     g.tm_b[0] = m.wq; g.tm_b[1] = m.wk; g.tm_b[2] = m.wv;
     g.M = T; g.N = q_dim + 2 * kv_dim; g.K = d;
     g.mode = kGemmQkv;
+    g.ab_f16 = f16;
     g.pair = use_pair;
     g.q_dim = q_dim; g.kv_dim = kv_dim; g.head_dim = Dh; g.n_kv_heads = c.n_kv_heads;
     g.tm_q = s->tm_q_st;
@@ -442,6 +473,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     a.tm_kv = s->tm_kv;
     a.tm_q = s->tm_q_attn;
     a.prefill_tokens = prefill_tokens_per_item(c.n_q_heads / c.n_kv_heads);
+    a.o_f16 = f16;
     a.q = q; a.o = o;
     a.n_q_heads = c.n_q_heads; a.n_kv_heads = c.n_kv_heads; a.head_dim = Dh;
     a.num_pages = c.num_pages; a.max_pages_per_seq = c.max_pages_per_seq; a.layer = l;
@@ -470,6 +502,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     go.tm_b[0] = m.wo; go.tm_b[1] = m.wo; go.tm_b[2] = m.wo;
     go.M = T; go.N = d; go.K = q_dim;
     go.mode = kGemmResid;
+    go.ab_f16 = f16;
     go.tm_out = tm_y; go.accumulate = 1;
     go.pair = use_pair;
     go.bn = use_pair ? 256 : gemm_pick_bn(T, d, s->sm_count);
@@ -490,6 +523,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gu.tm_b[0] = m.wgate; gu.tm_b[1] = m.wup; gu.tm_b[2] = m.wup;
     gu.M = T; gu.N = F; gu.K = d;
     gu.mode = kGemmGateUp;
+    gu.ab_f16 = f16;
+    gu.act_f16 = f16;
     gu.pair = use_pair;
     gu.tm_act = s->tm_act_st;
     gu.status = status;
@@ -502,6 +537,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gd.tm_b[0] = m.wdown; gd.tm_b[1] = m.wdown; gd.tm_b[2] = m.wdown;
     gd.M = T; gd.N = d; gd.K = F;
     gd.mode = kGemmResid;
+    gd.ab_f16 = f16;
     gd.tm_out = tm_y; gd.accumulate = 1;
     gd.pair = use_pair;
     gd.bn = use_pair ? 256 : gemm_pick_bn(T, d, s->sm_count);
@@ -573,8 +609,8 @@ hs_status_t hs_stage_debug_buffer(hs_stage_t* s, const char* name, void** dev_pt
   return HS_OK;
 }
 
-hs_status_t hs_op_gemm_bf16(const void* a, const void* w, const float* resid, float* out, int32_t M, int32_t N, int32_t K,
-                            int32_t sm_budget, int32_t* status_dev, void* cuda_stream) {
+static hs_status_t op_gemm(const void* a, const void* w, const float* resid, float* out, int32_t M, int32_t N, int32_t K,
+                           int32_t sm_budget, int32_t* status_dev, void* cuda_stream, int ab_f16) {
   if (!a || !w || !out || !status_dev || M < 1 || N < 1 || K < 1) return HS_ERR_INVALID_ARG;
   if ((N & 7) || (K & 7)) return HS_ERR_UNSUPPORTED_SHAPE;
   if ((reinterpret_cast<uintptr_t>(a) & 15) || (reinterpret_cast<uintptr_t>(w) & 15) ||
@@ -595,6 +631,7 @@ hs_status_t hs_op_gemm_bf16(const void* a, const void* w, const float* resid, fl
   g.tm_b[2] = g.tm_b[0];
   g.M = M; g.N = N; g.K = K;
   g.mode = kGemmResid;
+  g.ab_f16 = ab_f16;
   g.accumulate = resid != nullptr;
   g.pair = M > 128;
   g.bn = g.pair ? 256 : gemm_pick_bn(M, N, prop.multiProcessorCount);
@@ -605,6 +642,16 @@ hs_status_t hs_op_gemm_bf16(const void* a, const void* w, const float* resid, fl
   g.status = status_dev;
   const cudaError_t e = launch_gemm(g, sm_budget, stream);
   return e == cudaSuccess ? HS_OK : cuda_fail("gemm", e);
+}
+
+hs_status_t hs_op_gemm_bf16(const void* a, const void* w, const float* resid, float* out, int32_t M, int32_t N, int32_t K,
+                            int32_t sm_budget, int32_t* status_dev, void* cuda_stream) {
+  return op_gemm(a, w, resid, out, M, N, K, sm_budget, status_dev, cuda_stream, 0);
+}
+
+hs_status_t hs_op_gemm_f16(const void* a, const void* w, const float* resid, float* out, int32_t M, int32_t N,
+                                int32_t K, int32_t sm_budget, int32_t* status_dev, void* cuda_stream) {
+  return op_gemm(a, w, resid, out, M, N, K, sm_budget, status_dev, cuda_stream, 1);
 }
 
 }  // extern "C"

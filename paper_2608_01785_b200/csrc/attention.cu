@@ -235,8 +235,8 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
 #pragma unroll
       for (int j = 0; j < DH / 8; ++j) {
         const int col = 8 * j + 2 * (lane & 3);
-        if (ra < G) *reinterpret_cast<uint32_t*>(orow + ra * DH + col) = pack_bf16(o_acc[j][0] * inv_a, o_acc[j][1] * inv_a);
-        if (rb < G) *reinterpret_cast<uint32_t*>(orow + rb * DH + col) = pack_bf16(o_acc[j][2] * inv_b, o_acc[j][3] * inv_b);
+        if (ra < G) *reinterpret_cast<uint32_t*>(orow + ra * DH + col) = pack_act(o_acc[j][0] * inv_a, o_acc[j][1] * inv_a, p.o_f16 != 0);
+        if (rb < G) *reinterpret_cast<uint32_t*>(orow + rb * DH + col) = pack_act(o_acc[j][2] * inv_b, o_acc[j][3] * inv_b, p.o_f16 != 0);
       }
       continue;
     }
@@ -295,7 +295,8 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
         for (int i = 0; i < MAXV; ++i) {
           if (i < nv)
             *reinterpret_cast<uint2*>(dst + 4 * i) =
-                make_uint2(pack_bf16(acc[i].x * inv, acc[i].y * inv), pack_bf16(acc[i].z * inv, acc[i].w * inv));
+                make_uint2(pack_act(acc[i].x * inv, acc[i].y * inv, p.o_f16 != 0),
+                           pack_act(acc[i].z * inv, acc[i].w * inv, p.o_f16 != 0));
         }
       }
       if (lane == 0) *done = 0;             // ready for the next launch

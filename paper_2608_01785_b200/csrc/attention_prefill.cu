@@ -346,14 +346,15 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
       if (!correct(gblk - 1, alpha_prev)) break;
       if (row_valid) {
         const float inv = 1.f / l_run;
+        const bool f16 = p.o_f16 != 0;
         __nv_bfloat16* dst = p.o + size_t(tok0 + tok) * q_dim + (hk * G + g) * DH;
 #pragma unroll
         for (int u = 0; u < DH / 8; ++u) {
           uint4 w;
-          w.x = pack_bf16(o_reg[u * 8 + 0] * inv, o_reg[u * 8 + 1] * inv);
-          w.y = pack_bf16(o_reg[u * 8 + 2] * inv, o_reg[u * 8 + 3] * inv);
-          w.z = pack_bf16(o_reg[u * 8 + 4] * inv, o_reg[u * 8 + 5] * inv);
-          w.w = pack_bf16(o_reg[u * 8 + 6] * inv, o_reg[u * 8 + 7] * inv);
+          w.x = pack_act(o_reg[u * 8 + 0] * inv, o_reg[u * 8 + 1] * inv, f16);
+          w.y = pack_act(o_reg[u * 8 + 2] * inv, o_reg[u * 8 + 3] * inv, f16);
+          w.z = pack_act(o_reg[u * 8 + 4] * inv, o_reg[u * 8 + 5] * inv, f16);
+          w.w = pack_act(o_reg[u * 8 + 6] * inv, o_reg[u * 8 + 7] * inv, f16);
           *reinterpret_cast<uint4*>(dst + u * 8) = w;
         }
       }

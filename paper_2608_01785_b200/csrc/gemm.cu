@@ -92,14 +92,14 @@ __device__ __forceinline__ void stage_f32x32(uint8_t* buf, int lane, const uint3
         make_uint4(r[4 * u], r[4 * u + 1], r[4 * u + 2], r[4 * u + 3]);
 }
 // 32 values -> bf16 into units u0 .. u0+3 of the thread's row (u0 = 0 or 4: which 32 of the 64 columns).
-__device__ __forceinline__ void stage_bf16x32(uint8_t* buf, int lane, int u0, const float (&v)[32]) {
+__device__ __forceinline__ void stage_bf16x32(uint8_t* buf, int lane, int u0, const float (&v)[32], bool f16 = false) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     uint4 w;
-    w.x = pack_bf16(v[i * 8 + 0], v[i * 8 + 1]);
-    w.y = pack_bf16(v[i * 8 + 2], v[i * 8 + 3]);
-    w.z = pack_bf16(v[i * 8 + 4], v[i * 8 + 5]);
-    w.w = pack_bf16(v[i * 8 + 6], v[i * 8 + 7]);
+    w.x = pack_act(v[i * 8 + 0], v[i * 8 + 1], f16);
+    w.y = pack_act(v[i * 8 + 2], v[i * 8 + 3], f16);
+    w.z = pack_act(v[i * 8 + 4], v[i * 8 + 5], f16);
+    w.w = pack_act(v[i * 8 + 6], v[i * 8 + 7], f16);
     *reinterpret_cast<uint4*>(buf + lane * 128 + (((u0 + i) ^ (lane & 7)) << 4)) = w;
   }
 }
@@ -230,7 +230,10 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
   } else if (warp == 1) {
     // --------------------------------------------------------- MMA issuer --
     if (lane == 0 && rank == 0) {
-      const uint32_t idesc = umma_idesc_bf16_f32(PAIR ? 2 * BM : BM, p.mode == kGemmResid && !PAIR ? p.bn : BN);
+      // both operands are fp16 or both bf16 (one MMA cannot mix the two): the format fields of A (bits 7..9)
+      // and B (bits 10..12) are 0 for fp16 and 1 for bf16
+      const uint32_t idesc = umma_idesc_bf16_f32(PAIR ? 2 * BM : BM, p.mode == kGemmResid && !PAIR ? p.bn : BN) &
+                             (p.ab_f16 ? ~(63u << 7) : ~0u);
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
       bool ok = true;
@@ -344,7 +347,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
             if (lane == 0) bulk_wait_read<1>();
             __syncwarp();
           }
-          stage_bf16x32(buf, lane, (c & 1) * 4, v0);
+          stage_bf16x32(buf, lane, (c & 1) * 4, v0, p.act_f16 != 0);
           const bool block_done = (c & 1) || col0 + 32 >= p.N;
           if (block_done) {                       // 64 columns staged (or the ragged end of the row)
             fence_proxy_async();

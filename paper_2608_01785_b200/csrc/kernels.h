@@ -27,6 +27,7 @@ struct GemmParams {
   CUtensorMap tm_b[3];       // weights, box 64 x 128: Resid {W}, Qkv {Wq, Wk, Wv}, GateUp {Wgate, Wup}
   int M, N, K;               // N: Resid output width; Qkv (Hq + 2 Hkv) * Dh; GateUp F (activation width)
   int mode;
+  int ab_f16;                // 1: both operands hold fp16 values; 0: both bf16
   int pair;                  // 1: run on pairs of SMs (256 x 256 tiles, bn = 256, no K split) when the budget allows
   // Resid
   CUtensorMap tm_out;        // fp32 [M, N], box 32 x 32, 128-byte swizzle (rows past M are clipped)
@@ -45,6 +46,7 @@ struct GemmParams {
   // GateUp
   CUtensorMap tm_act;        // bf16 act [M, N], box 64 x 32, 128-byte swizzle
   int* status;               // device status word
+  int act_f16;               // GateUp: 1 = write act as fp16, 0 = bf16
   int* smid_log;             // nullable: SM census slots of this launch (see log_smid)
 };
 cudaError_t launch_gemm(const GemmParams& p, int sm_budget, cudaStream_t stream);
@@ -65,9 +67,13 @@ struct NormParams {
   __nv_bfloat16* h;
   int T, d;
   float eps;
+  int h_f16;                 // 1 = write h as fp16, 0 = bf16
   int* smid_log;             // nullable: SM census slots of this launch
 };
 cudaError_t launch_rmsnorm(const NormParams& p, int sm_budget, cudaStream_t stream);
+// dst[i] = fp16(src[i]) for n bf16 values (n a multiple of 8, both 16-byte aligned); used once per weight
+// matrix when a stage is created
+cudaError_t launch_bf16_to_f16(const void* src, void* dst, size_t n, cudaStream_t stream);
 cudaError_t norm_set_attributes();
 
 // -------------------------------------------------------------- attention --
@@ -75,6 +81,7 @@ struct AttnParams {
   CUtensorMap tm_kv;               // whole pool as rows of Dh bf16: box 64 x 16, 128-byte swizzle
   CUtensorMap tm_q;                // q [max_tokens, q_dim]: box 64 x prefill_tokens, 128-byte swizzle
   int prefill_tokens;              // tokens per prefill work item
+  int o_f16;                       // 1 = write o as fp16, 0 = bf16 (q, K, V are always bf16)
   const __nv_bfloat16* q;          // [T, q_dim] (after RoPE)
   __nv_bfloat16* o;                // [T, q_dim]
   int n_q_heads, n_kv_heads, head_dim, num_pages, max_pages_per_seq, layer;

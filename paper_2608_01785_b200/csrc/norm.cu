@@ -104,13 +104,35 @@ __global__ void __launch_bounds__(NORM_THREADS, 1) rmsnorm_kernel(const NormPara
       }
       float g[8];
       unpack8(gsrc[i], g);
-      hdst[i] = make_uint4(pack_bf16(a.x * r * g[0], a.y * r * g[1]), pack_bf16(a.z * r * g[2], a.w * r * g[3]),
-                           pack_bf16(b.x * r * g[4], b.y * r * g[5]), pack_bf16(b.z * r * g[6], b.w * r * g[7]));
+      const bool f16 = p.h_f16 != 0;
+      hdst[i] = make_uint4(pack_act(a.x * r * g[0], a.y * r * g[1], f16), pack_act(a.z * r * g[2], a.w * r * g[3], f16),
+                           pack_act(b.x * r * g[4], b.y * r * g[5], f16), pack_act(b.z * r * g[6], b.w * r * g[7], f16));
     }
   }
 }
 
+// One-time widening of the significand: bf16 weights -> fp16 copies (n8 groups of 8 values).  A bf16 value
+// is an fp16 value exactly when 2^-17 <= |w| <= 65504; smaller ones round to the fp16 subnormal grid
+// (absolute error <= 2^-25), larger ones saturate.
+__global__ void __launch_bounds__(256) bf16_to_f16_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst,
+                                                          size_t n8) {
+  for (size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n8; i += size_t(gridDim.x) * blockDim.x) {
+    float f[8];
+    unpack8(src[i], f);
+    dst[i] = make_uint4(pack_f16(f[0], f[1]), pack_f16(f[2], f[3]), pack_f16(f[4], f[5]), pack_f16(f[6], f[7]));
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_bf16_to_f16(const void* src, void* dst, size_t n, cudaStream_t stream) {
+  const size_t n8 = n / 8;
+  if (n8 == 0) return cudaSuccess;
+  const size_t want = (n8 + 255) / 256;
+  bf16_to_f16_kernel<<<unsigned(want < 1184 ? want : 1184), 256, 0, stream>>>(static_cast<const uint4*>(src),
+                                                                              static_cast<uint4*>(dst), n8);
+  return cudaGetLastError();
+}
 
 cudaError_t norm_set_attributes() {
   return cudaFuncSetAttribute(rmsnorm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, NORM_SMEM);

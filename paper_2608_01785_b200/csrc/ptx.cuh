@@ -4,6 +4,7 @@
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -271,6 +272,19 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);   // round-to-nearest-even; .x = lo (low 16 bits)
   return *reinterpret_cast<uint32_t*>(&v);
+}
+// Two fp32 -> packed fp16 (round to nearest even), clamped to the finite fp16 range so that an outlier
+// becomes +-65504 instead of infinity.
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  lo = fminf(fmaxf(lo, -65504.f), 65504.f);
+  hi = fminf(fmaxf(hi, -65504.f), 65504.f);
+  __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+// Packs as fp16 or bf16: the stage's private activations (h, o, act) are fp16 unless it was created with
+// HS_FLAG_BF16_ACTIVATIONS.
+__device__ __forceinline__ uint32_t pack_act(float lo, float hi, bool f16) {
+  return f16 ? pack_f16(lo, hi) : pack_bf16(lo, hi);
 }
 __device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");

@@ -18,12 +18,12 @@ class Stage:
     """
 
     def __init__(self, dims, weights: Sequence[Dict[str, torch.Tensor]], num_pages: int, max_tokens: int,
-                 max_seqs: int, max_pages_per_seq: int, max_position: int, device: int = 0):
+                 max_seqs: int, max_pages_per_seq: int, max_position: int, device: int = 0, flags: int = 0):
         if not torch.cuda.is_available():
             raise RuntimeError("Stage needs a CUDA device; there is no CPU implementation")
         self.dims = dims
         self.device = torch.device("cuda", device)
-        self.cfg = B.make_config(dims, num_pages, max_tokens, max_seqs, max_pages_per_seq, max_position, device)
+        self.cfg = B.make_config(dims, num_pages, max_tokens, max_seqs, max_pages_per_seq, max_position, device, flags)
         pool_bytes, ws_bytes = B.hs_kv_pool_bytes(self.cfg), B.hs_workspace_bytes(self.cfg)
         if pool_bytes == 0 or ws_bytes == 0:
             raise B.HsError(B.HS_ERR_UNSUPPORTED_SHAPE, "configuration rejected")
@@ -67,14 +67,16 @@ class Stage:
         return B.hs_stage_status(self.handle)
 
     def debug_tensor(self, name: str) -> torch.Tensor:
-        """Copy of a private intermediate ("h", "q", "o", "act"; bf16), shaped [max_tokens, width], or of the
-        SM census ("smid"; int32 [kernel class, block]; the first request switches the census on)."""
+        """Copy of a private intermediate, shaped [max_tokens, width] ("q" is bf16; "h", "o" and "act" are
+        fp16, or bf16 when the stage was made with HS_FLAG_BF16_ACTIVATIONS), or of the SM census ("smid";
+        int32 [kernel class, block]; the first request switches the census on)."""
         ptr, size = B.hs_stage_debug_buffer(self.handle, name)
         off = ptr - self.workspace.data_ptr()
         raw = self.workspace[off: off + size].clone()
         if name == "smid":
             return raw.view(torch.int32).view(len(B.PROFILE_CLASSES), -1)
-        return raw.view(torch.bfloat16).view(self.cfg.max_tokens, -1)
+        bf16 = name == "q" or (self.cfg.flags & B.HS_FLAG_BF16_ACTIVATIONS)
+        return raw.view(torch.bfloat16 if bf16 else torch.float16).view(self.cfg.max_tokens, -1)
 
     def close(self) -> None:
         if self.handle:

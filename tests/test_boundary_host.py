@@ -75,6 +75,21 @@ def test_config_validation():
     assert e.value.status == B.HS_ERR_INVALID_ARG
 
 
+def test_activation_format_flag_sizes_the_workspace():
+    """The default stage keeps fp16 copies of the seven projection matrices of every layer in its workspace;
+    HS_FLAG_BF16_ACTIVATIONS drops them.  Any other flag bit is refused."""
+    dims = wl.DIMS["c1_tiny"]
+    cfg16 = B.make_config(dims, 64, 128, 8, 8, 256, device=-1)
+    cfgbf = B.make_config(dims, 64, 128, 8, 8, 256, device=-1, flags=B.HS_FLAG_BF16_ACTIVATIONS)
+    w_bytes = 2 * dims.n_layers * (2 * dims.q_dim * dims.d_model + 2 * dims.kv_dim * dims.d_model +
+                                   3 * dims.d_ffn * dims.d_model)
+    extra = B.hs_workspace_bytes(cfg16) - B.hs_workspace_bytes(cfgbf)
+    assert w_bytes <= extra <= w_bytes + 7 * 1024 * dims.n_layers
+    assert B.hs_kv_pool_bytes(cfg16) == B.hs_kv_pool_bytes(cfgbf) > 0
+    bad = B.make_config(dims, 64, 128, 8, 8, 256, device=-1, flags=2)
+    assert B.hs_workspace_bytes(bad) == 0 and B.hs_kv_pool_bytes(bad) == 0
+
+
 def test_allocator_config_1_block_tables_by_hand():
     # sequences allocated in order with 32, 48, 40 + 1 and 64 + 1 tokens; pops yield 0, 1, 2, ...
     stage, _ = host_stage()

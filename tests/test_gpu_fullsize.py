@@ -6,23 +6,25 @@ What is asserted, per configuration:
     GPU's own fp32 residual stream before layer l (the output of the same stage truncated to l layers)
     and the same cache context, and its output is compared with the GPU's stream after layer l:
     max |err| <= 2e-2 * RMS.  At config 3 the oracle evaluates K/V of every token and a sample of rows;
-  * end to end (all layers, oracle never sees a GPU value): reported, and bounded by 1.3 x the error of
-    the oracle itself run with its tensor-core operands rounded to bf16 (h, q, P, o, act) -- the
-    arithmetic-format floor no bf16-operand implementation can beat.  For config 2 that floor is about
-    2.6e-2 * RMS after 4 layers, i.e. above the 2e-2 that a single layer meets with a wide margin.
+  * end to end (all layers, the oracle never sees a GPU value): max |err| <= 2e-2 * RMS as well.  Beside it
+    the test prints the error of the oracle itself run with its tensor-core operands rounded to the
+    stage's formats (q and P to bf16; h, o and act to fp16) -- the floor that the operand formats set.
+    (With h, o and act in bf16 that floor is 2.4e-2 * RMS for config 2, above the tolerance: the reason
+    why the stage keeps those three in fp16.)
 """
 import numpy as np
 import pytest
 import torch
 
 import bench
-from oracle.oracle import Oracle, OracleConfig, ROUND_ALL
+from oracle.oracle import Oracle, OracleConfig, ROUND_ALL, ROUND_ACT_F16
 from paper_2608_01785_b200 import workloads as wl
 from paper_2608_01785_b200.stage import Stage
 from tests.helpers import rel_err
 
 pytestmark = pytest.mark.gpu
 TOL = 2e-2
+ROUND_AS_GPU = ROUND_ALL | ROUND_ACT_F16     # q and P to bf16; h, o and act to fp16: the stage's default formats
 
 
 @pytest.fixture(scope="module")
@@ -68,7 +70,7 @@ def layer_pool_bits(pool0: torch.Tensor, dims, num_pages: int, layer: int) -> np
 
 def layer_local_error(orc, stage, batch, bt, x, pool0, layer, rows=None, want_floor=False):
     """max|err|/RMS of GPU layer `layer` against the oracle's layer fed the GPU's own input stream.
-    With want_floor also returns the same error for the oracle layer run with bf16-rounded operands."""
+    With want_floor also returns the same error for the oracle layer run with operands rounded as the GPU's."""
     dims = stage.dims
     T = batch.n_tokens
     x_in = wl.to_f32_numpy(x) if layer == 0 else truncated_output(stage, layer, batch, bt, x, pool0).cpu().numpy()
@@ -85,7 +87,7 @@ def layer_local_error(orc, stage, batch, bt, x, pool0, layer, rows=None, want_fl
     err = rel_err(y_gpu[sel], y_ref[sel])
     if not want_floor:
         return err
-    orc.set_operand_rounding(ROUND_ALL)
+    orc.set_operand_rounding(ROUND_AS_GPU)
     try:
         y_floor, _ = orc.layer(cfg1, w, 0, layer_pool_bits(pool0, dims, stage.cfg.num_pages, layer), batch.q_len,
                                batch.ctx_len, bt, x_in, row_mask=mask)
@@ -121,15 +123,15 @@ def test_config2_budget_sweep_layer_local_and_end_to_end(orc):
         pool_np = wl.bf16_bits_numpy(pool0).reshape(-1)
         x_np = wl.to_f32_numpy(x)
         y_ref = orc.step(cfg, w_np, pool_np.copy(), batch.q_len, batch.ctx_len, bt, x_np)
-        orc.set_operand_rounding(ROUND_ALL)
+        orc.set_operand_rounding(ROUND_AS_GPU)
         try:
             y_floor = orc.step(cfg, w_np, pool_np.copy(), batch.q_len, batch.ctx_len, bt, x_np)
         finally:
             orc.set_operand_rounding(0)
         err, floor = rel_err(y_gpu, y_ref), rel_err(y_floor, y_ref)
         print(f"config 2 end to end ({dims.n_layers} layers): max|err|/RMS = {err:.2e}; "
-              f"bf16-operand floor of the oracle itself = {floor:.2e}")
-        assert err <= max(TOL, 1.3 * floor)
+              f"operand-format floor of the oracle itself = {floor:.2e}")
+        assert err <= TOL
     finally:
         stage.close()
 
@@ -188,10 +190,9 @@ C3_ROWS = np.unique(np.concatenate([np.array([0, 1, 15, 16, 17, 127, 128, 1023, 
 
 @pytest.mark.parametrize("init", ["n002", "depth_scaled"])
 def test_config3_budget_sweep_and_sampled_layer_local(orc, init):
-    """Config 3 states no weight distribution.  With N(0, 0.02) everywhere the 18944-wide MLP dominates the
-    layer output and the bf16 rounding of its operands alone puts a single layer at about 2e-2 * RMS (the
-    oracle with bf16-rounded operands shows the same), so that variant is held to 1.3 x that floor; with
-    the output projections drawn at std 0.02 / sqrt(2 L) the flat 2e-2 applies."""
+    """Config 3 states no weight distribution, so two are run: N(0, 0.02) everywhere (the 18944-wide MLP
+    then dominates the layer output, the hardest case for 16-bit operands) and the output projections drawn
+    at std 0.02 / sqrt(2 L).  Both are held to the flat 2e-2."""
     name = "c3_7b"
     stage, dims, batch, bt, x = bench.build_stage(name, 0, init)
     try:
@@ -213,7 +214,7 @@ def test_config3_budget_sweep_and_sampled_layer_local(orc, init):
         for layer in (0, 1, 13, 27):
             err, floor = layer_local_error(orc, stage, batch, bt, x, pool0, layer, rows=rows, want_floor=True)
             print(f"config 3 ({init}) layer {layer}: layer-local max|err|/RMS on {len(rows)} sampled rows = {err:.2e}; "
-                  f"bf16-operand floor of the oracle itself = {floor:.2e}")
-            assert err <= (TOL if init == "depth_scaled" else max(TOL, 1.3 * floor))
+                  f"operand-format floor of the oracle itself = {floor:.2e}")
+            assert err <= TOL
     finally:
         stage.close()

@@ -57,11 +57,13 @@ def check_kv_written(case, pool_in, pool_gpu, kv_pre, layer=0):
 # ----------------------------------------------------------------- GEMM op --
 @pytest.mark.parametrize("M,N,K,resid", [(128, 256, 64, False), (82, 520, 200, True), (300, 264, 72, True),
                                          (2112, 1024, 3584, False), (1000, 2048, 1408, True), (16, 1536, 1024, True)])
-def test_gemm_op_matches_oracle_and_is_budget_invariant(orc, M, N, K, resid):
+@pytest.mark.parametrize("a_dtype", [torch.bfloat16, torch.float16])
+def test_gemm_op_matches_oracle_and_is_budget_invariant(orc, M, N, K, resid, a_dtype):
+    """Both operand forms: bf16 x bf16, and the fp16 x fp16 form the stage uses by default."""
     dev = torch.device("cuda:0")
     g = torch.Generator().manual_seed(M * 7 + N)
-    a = torch.randn(M, K, generator=g).to(torch.bfloat16)
-    w = (torch.randn(N, K, generator=g) * 0.02).to(torch.bfloat16)
+    a = torch.randn(M, K, generator=g).to(a_dtype)
+    w = (torch.randn(N, K, generator=g) * 0.02).to(a_dtype)
     r = torch.randn(M, N, generator=g) if resid else None
     want = orc.linear(a.float().numpy(), w.float().numpy())
     if resid:
@@ -75,11 +77,11 @@ def test_gemm_op_matches_oracle_and_is_budget_invariant(orc, M, N, K, resid):
         status = torch.zeros(1, dtype=torch.int32, device=dev)
         r_d = r.to(dev) if resid else None
         B.hs_op_gemm_bf16(a_d.data_ptr(), w_d.data_ptr(), r_d.data_ptr() if resid else 0, out.data_ptr(), M, N, K,
-                          budget, status.data_ptr())
+                          budget, status.data_ptr(), a_is_f16=a_dtype == torch.float16)
         torch.cuda.synchronize()
         assert status.item() == 0
         outs.append(out.cpu())
-    assert rel_err(outs[0].numpy(), want) < 1e-4          # fp32 accumulation of exact bf16 products
+    assert rel_err(outs[0].numpy(), want) < 1e-4          # fp32 accumulation of exact 16-bit products
     for o in outs[1:]:
         assert torch.equal(o, outs[0])
 
@@ -127,7 +129,9 @@ def config1_case(orc):
     return case
 
 
-def test_config1_step_matches_oracle_at_budgets_148_and_8(orc):
+@pytest.mark.parametrize("flags", [0, B.HS_FLAG_BF16_ACTIVATIONS])
+def test_config1_step_matches_oracle_at_budgets_148_and_8(orc, flags):
+    """flags 0: h, o and act in fp16 against fp16 copies of the weights (the default); the flag: all bf16."""
     case = config1_case(orc)
     assert case.block_tables[:, :5].tolist() == [[0, 1, -1, -1, -1], [2, 3, 4, -1, -1], [5, 6, 7, -1, -1],
                                                  [8, 9, 10, 11, 12]]
@@ -136,11 +140,11 @@ def test_config1_step_matches_oracle_at_budgets_148_and_8(orc):
                               case.block_tables, case.x, want_kv_pre=True)
     results = []
     for budget in (148, 8):
-        st = make_stage(case)
+        st = make_stage(case, flags=flags)
         y, pool = run_step(st, case, budget)
         st.close()
         err = rel_err(y, y_ref)
-        print(f"config 1, sm_budget {budget}: max|err|/RMS = {err:.2e}")
+        print(f"config 1 (flags {flags}), sm_budget {budget}: max|err|/RMS = {err:.2e}")
         assert err <= TOL
         check_kv_written(case, case.kv_pool, pool, kv_pre)
         results.append((y, pool))
@@ -224,6 +228,13 @@ def test_edge_cases_match_oracle(orc, name):
         assert np.all(g6[:, :, :, ~(owned | written)] == 0x7fc0)
         assert np.array_equal(g6[:, :, :, owned & ~written], pool6[:, :, :, owned & ~written])
     assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    # the all-bf16 variant of the stage (no fp16 weight copies) on the same case
+    st = make_stage(case, flags=B.HS_FLAG_BF16_ACTIVATIONS)
+    y, _ = run_step(st, case, 148)
+    st.close()
+    err = rel_err(y, y_ref)
+    print(f"{name}, bf16 activations: max|err|/RMS = {err:.2e}")
+    assert err <= TOL
 
 
 def test_chunked_prefill_then_decode_on_the_gpu_cache(orc):

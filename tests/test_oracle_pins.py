@@ -423,3 +423,27 @@ def test_float32_oracle_is_close_to_float64_on_config_1(oracle32, oracle64):
     y64 = oracle64.step(case.cfg, case.weights, case.kv_pool.copy(), *args)
     assert rel_err(y32, y64) < 1e-3      # dominated by 1-ulp flips of cached bf16 values
     assert rel_err(y64, case.x) > 1e-2   # and the layer is not the identity
+
+
+def test_operand_rounding_diagnostic_is_off_by_default_and_fp16_is_the_finer_grid(oracle32):
+    """The diagnostic switch (never the pass/fail oracle): off by default, rounding the intermediates moves
+    the output, and the fp16 grid for h, o and act (11-bit significand) moves it less than bf16 (8-bit)."""
+    from oracle.oracle import ROUND_ALL, ROUND_ACT_F16
+    dims = wl.StageDims(2, 128, 4, 2, 32, 512)
+    case = make_case(dims, wl.BatchSpec([24, 9], [0, 0]), seed=21)
+    args = (case.cfg, case.weights, None, case.batch.q_len, case.batch.ctx_len, case.block_tables, case.x)
+
+    def run(mask):
+        oracle32.set_operand_rounding(mask)
+        try:
+            return oracle32.step(args[0], args[1], case.kv_pool.copy(), *args[3:])
+        finally:
+            oracle32.set_operand_rounding(0)
+
+    y0, y0_again = run(0), run(0)
+    assert np.array_equal(y0, y0_again)
+    e_bf16, e_f16 = rel_err(run(ROUND_ALL), y0), rel_err(run(ROUND_ALL | ROUND_ACT_F16), y0)
+    assert 0 < e_f16 < e_bf16 < 2e-2
+    # h, o, act alone: the two grids differ by 2^3 in spacing (1-ulp flips of cached bf16 K/V blur the ratio)
+    e_b, e_h = rel_err(run(1 | 8 | 16), y0), rel_err(run(1 | 8 | 16 | ROUND_ACT_F16), y0)
+    assert e_b / 16 < e_h < e_b / 2

@@ -54,7 +54,7 @@ def test_noalloc_decode_attention_matches_the_stage_path_twice_in_a_row():
     ]
     for dims, ctx, seed in problems:
         case = _decode_case(dims, ctx, seed)
-        st = make_stage(case)
+        st = make_stage(case, flags=B.HS_FLAG_BF16_ACTIVATIONS)   # the stage's o in bf16, as this call writes it
         try:
             run_step(st, case, 148)
             n = case.batch.n_seqs
