@@ -446,6 +446,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     np.d = d;
     np.eps = c.rms_eps;
     np.h_f16 = f16;
+    np.status = status;
     np.smid_log = slots(0);
     { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
     if (e != cudaSuccess) break;

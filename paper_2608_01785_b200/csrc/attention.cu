@@ -62,6 +62,91 @@ __device__ __forceinline__ uint32_t mask_v(uint32_t r, int k, int n_valid) {
   return r;
 }
 
+// Merges the partials of one (sequence, KV head) group -- items first .. first + splits - 1 -- in split
+// order and writes the normalised output rows.  LPH lanes share one query head, each owning DH / LPH
+// contiguous columns.  A lone warp does this at the tail of the kernel, so what counts is latency: the
+// partial outputs travel by asynchronous copies into the warp's own (now idle) page ring, used as two
+// halves of PS splits each -- while one half is folded into the running sum the other is in flight -- laid
+// out [split][float4 index][lane] so that every lane reads back only what it copied itself, conflict-free.
+// The running maximum is updated per half (online rescaling); the order of all operations is fixed.
+template <int DH, int LPH, int RING_BYTES>
+__device__ __forceinline__ void merge_group(const float* part_o, const float* part_ml, uint8_t* ring, int first,
+                                            int splits, int G, int lane, __nv_bfloat16* orow, bool f16) {
+  constexpr int NV = DH / 4 / LPH;                 // float4 per lane and split
+  constexpr int PS = RING_BYTES / 2 / (NV * 512) < 4 ? RING_BYTES / 2 / (NV * 512) : 4;   // splits per half
+  static_assert(PS >= 1, "half a ring holds one split");
+  const int g = lane / LPH, part = lane % LPH;
+  if (g < G) {
+    const float2* ml_g = reinterpret_cast<const float2*>(part_ml) + size_t(first) * 16 + g;   // + j * 16
+    const uint32_t ring_u32 = smem_u32(ring) + lane * 16;
+    const float4* ring_f4 = reinterpret_cast<const float4*>(ring) + lane;
+    float2 mlv[2][PS];
+    auto request = [&](int j0, int half) {         // splits j0 .. j0 + PS - 1 into one half of the ring
+#pragma unroll
+      for (int u = 0; u < PS; ++u) {
+        if (j0 + u < splits) {
+          const float4* src = reinterpret_cast<const float4*>(part_o + (size_t(first + j0 + u) * 16 + g) * DH) + part * NV;
+#pragma unroll
+          for (int i = 0; i < NV; ++i)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ring_u32 + ((half * PS + u) * NV + i) * 512),
+                         "l"(src + i)
+                         : "memory");
+          mlv[half][u] = __ldcg(&ml_g[size_t(j0 + u) * 16]);
+        }
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    float mm = -INFINITY, ll = 0.f;
+    float4 acc[NV];
+#pragma unroll
+    for (int i = 0; i < NV; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    request(0, 0);
+    request(PS, 1);
+    int half = 0;
+    for (int j0 = 0; j0 < splits; j0 += PS, half ^= 1) {
+      asm volatile("cp.async.wait_group 1;" ::: "memory");     // the older of the two halves has landed
+      float pm = mm;
+      if (half == 0) {
+#pragma unroll
+        for (int u = 0; u < PS; ++u) if (j0 + u < splits) pm = fmaxf(pm, mlv[0][u].x);
+      } else {
+#pragma unroll
+        for (int u = 0; u < PS; ++u) if (j0 + u < splits) pm = fmaxf(pm, mlv[1][u].x);
+      }
+      const float sc = exp2f(mm - pm);                         // 0 on the first half (mm = -inf)
+      mm = pm;
+      ll *= sc;
+#pragma unroll
+      for (int i = 0; i < NV; ++i) { acc[i].x *= sc; acc[i].y *= sc; acc[i].z *= sc; acc[i].w *= sc; }
+#pragma unroll
+      for (int u = 0; u < PS; ++u) {
+        if (j0 + u < splits) {
+          const float2 ml = half == 0 ? mlv[0][u] : mlv[1][u];
+          const float f = exp2f(ml.x - mm);
+          ll += f * ml.y;
+#pragma unroll
+          for (int i = 0; i < NV; ++i) {
+            const float4 v = ring_f4[((half * PS + u) * NV + i) * 32];
+            acc[i].x += f * v.x; acc[i].y += f * v.y; acc[i].z += f * v.z; acc[i].w += f * v.w;
+          }
+        }
+      }
+      if (half == 0) request(j0 + 2 * PS, 0);                  // refill the half just read (may be empty)
+      else request(j0 + 2 * PS, 1);
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    const float inv = 1.f / ll;
+    __nv_bfloat16* dst = orow + g * DH + part * NV * 4;
+#pragma unroll
+    for (int i = 0; i < NV; ++i)
+      *reinterpret_cast<uint2*>(dst + 4 * i) =
+          make_uint2(pack_act(acc[i].x * inv, acc[i].y * inv, f16), pack_act(acc[i].z * inv, acc[i].w * inv, f16));
+  }
+  // the ring goes back to the copy engine for the next item: order these generic-proxy accesses before it
+  fence_proxy_async();
+  __syncwarp();
+}
+
 // ==================================================================== decode ==
 // Every warp is its own pipeline: it pulls a work item from the queue, streams the item's pages through
 // a private ring of DC_STAGES (K page, V page) slots that its lane 0 fills by TMA a few pages ahead, and
@@ -103,10 +188,16 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
   uint64_t* full = full_all + warp * DC_STAGES;
   uint32_t issued = 0, consumed = 0;      // pages this warp has requested / finished, over all its items
 
+  // a warp's first item is its own index in the grid (no round trip to the queue head before the first
+  // page request); the queue hands out the items after those
+  bool first_round = true;
   for (;;) {
-    int item = 0;
-    if (lane == 0) item = atomicAdd(p.counters + 1, 1);
-    item = __shfl_sync(0xffffffffu, item, 0);
+    int item = blockIdx.x * DC_WARPS + warp;
+    if (!first_round) {
+      if (lane == 0) item = int(gridDim.x) * DC_WARPS + atomicAdd(p.counters + 1, 1);
+      item = __shfl_sync(0xffffffffu, item, 0);
+    }
+    first_round = false;
     if (item >= p.n_decode_items || *abort_flag) break;
     const int4 it = reinterpret_cast<const int4*>(p.decode_items)[item];
     const int drow = it.x, hk = it.y, k0 = it.z, k1 = it.w;
@@ -115,16 +206,21 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
     const int n_pages = (k1 - k0 + 15) >> 4;
     const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq + (k0 >> 4);
 
-    auto issue = [&](int pi) {              // lane 0: request page pi of this item
+    // the item's page ids, one per lane, fetched with a single load: reading the block table page by page
+    // would put one dependent round trip to memory in front of every request
+    const int my_page = lane < n_pages ? table[lane] : 0;      // the planner keeps items within 32 pages
+    auto issue = [&](int page) {            // lane 0: request one page of this item
       const uint32_t st = issued % DC_STAGES;
-      const int page = table[pi];
       mbar_expect_tx(&full[st], SLOT_BYTES);
       load_page<DH>(p, slots + st * SLOT_BYTES, &full[st], 0, page, hk);
       load_page<DH>(p, slots + st * SLOT_BYTES + G_::PAGE_BYTES, &full[st], 1, page, hk);
       ++issued;
     };
-    if (lane == 0)
-      for (int pi = 0; pi < min(DC_STAGES - 1, n_pages); ++pi) issue(pi);
+#pragma unroll
+    for (int pi = 0; pi < DC_STAGES - 1; ++pi) {
+      const int page = __shfl_sync(0xffffffffu, my_page, pi);
+      if (lane == 0 && pi < n_pages) issue(page);
+    }
 
     // Q fragments straight from global memory: rows = query heads hk*G .. hk*G + G - 1 of the new token
     const __nv_bfloat16* qrow = p.q + size_t(tok) * q_dim + size_t(hk) * G * DH;
@@ -146,7 +242,8 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
 
     for (int pi = 0; pi < n_pages; ++pi) {
       // the slot read in the previous iteration is free: keep DC_STAGES - 1 pages in flight
-      if (lane == 0 && pi + DC_STAGES - 1 < n_pages) issue(pi + DC_STAGES - 1);
+      const int page_ahead = __shfl_sync(0xffffffffu, my_page, (pi + DC_STAGES - 1) & 31);
+      if (lane == 0 && pi + DC_STAGES - 1 < n_pages) issue(page_ahead);
       const uint32_t st = consumed % DC_STAGES;
       ok = mbar_wait(&full[st], (consumed / DC_STAGES) & 1, abort_flag, p.status);
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
@@ -263,42 +360,9 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
     last = __shfl_sync(0xffffffffu, last, 0);
     if (last) {
       __threadfence();
-      // lanes_per_head lanes share one query head; each owns DH / lanes_per_head contiguous columns
-      const int lanes_per_head = G <= 8 ? 4 : 2;
-      const int g = lane / lanes_per_head, part = lane % lanes_per_head;
       const int first = dr.z + hk * splits;
-      if (g < G) {
-        float mm = -INFINITY;
-        for (int j = 0; j < splits; ++j) mm = fmaxf(mm, __ldcg(p.part_ml + (size_t(first + j) * 16 + g) * 2));
-        float ll = 0.f;
-        constexpr int MAXV = DH / 8;               // float4 per lane when two lanes share a head
-        float4 acc[MAXV];
-        const int nv = DH / 4 / lanes_per_head;    // float4 per lane
-#pragma unroll
-        for (int i = 0; i < MAXV; ++i) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int j = 0; j < splits; ++j) {
-          const float* ml = p.part_ml + (size_t(first + j) * 16 + g) * 2;
-          const float f = exp2f(__ldcg(ml) - mm);
-          ll += f * __ldcg(ml + 1);
-          const float4* src = reinterpret_cast<const float4*>(p.part_o + (size_t(first + j) * 16 + g) * DH) + part * nv;
-#pragma unroll
-          for (int i = 0; i < MAXV; ++i) {
-            if (i < nv) {
-              const float4 v = __ldcg(src + i);
-              acc[i].x += f * v.x; acc[i].y += f * v.y; acc[i].z += f * v.z; acc[i].w += f * v.w;
-            }
-          }
-        }
-        const float inv = 1.f / ll;
-        __nv_bfloat16* dst = orow + g * DH + part * nv * 4;
-#pragma unroll
-        for (int i = 0; i < MAXV; ++i) {
-          if (i < nv)
-            *reinterpret_cast<uint2*>(dst + 4 * i) =
-                make_uint2(pack_act(acc[i].x * inv, acc[i].y * inv, p.o_f16 != 0),
-                           pack_act(acc[i].z * inv, acc[i].w * inv, p.o_f16 != 0));
-        }
-      }
+      if (G <= 8) merge_group<DH, 4, DC_STAGES * SLOT_BYTES>(p.part_o, p.part_ml, slots, first, splits, G, lane, orow, p.o_f16 != 0);
+      else merge_group<DH, 2, DC_STAGES * SLOT_BYTES>(p.part_o, p.part_ml, slots, first, splits, G, lane, orow, p.o_f16 != 0);
       if (lane == 0) *done = 0;             // ready for the next launch
     }
   }

@@ -11,6 +11,7 @@ namespace hs {
 
 constexpr int kPage = HS_PAGE_SIZE;      // tokens per KV page
 constexpr int kDecodeSplit = 256;        // keys per decode split-KV work item (budget independent)
+static_assert(kDecodeSplit % 16 == 0 && kDecodeSplit / 16 <= 32, "the decode kernel keeps one page id per lane");
 constexpr int kPrefillRows = 128;        // (token, query head of one KV head) rows per prefill work item
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }

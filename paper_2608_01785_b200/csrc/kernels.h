@@ -68,6 +68,7 @@ struct NormParams {
   int T, d;
   float eps;
   int h_f16;                 // 1 = write h as fp16, 0 = bf16
+  int* status;               // device status word (bounded waits report HS_ERR_TIMEOUT here)
   int* smid_log;             // nullable: SM census slots of this launch
 };
 cudaError_t launch_rmsnorm(const NormParams& p, int sm_budget, cudaStream_t stream);

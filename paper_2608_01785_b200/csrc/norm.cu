@@ -111,6 +111,116 @@ __global__ void __launch_bounds__(NORM_THREADS, 1) rmsnorm_kernel(const NormPara
   }
 }
 
+// The same operation with rows staged by bulk copies (the variant the launcher uses whenever two rows per
+// warp fit in shared memory).  Every warp owns two row buffers and an mbarrier for each; its lane 0 asks
+// the copy engine for row k + 2 as soon as the warp is done with row k, so an SM keeps up to
+// 2 x warps rows (about 200 KB) in flight instead of what its threads can hold in registers.  Rows are
+// handed out in the same fixed order and each row's arithmetic is the same fixed sequence (a per-lane
+// serial sum over groups lane, lane + 32, ... then a butterfly), whatever the grid.
+constexpr int BULK_SMEM_BUDGET = 200 * 1024;   // row buffers of one block
+constexpr int BULK_MAX_WARPS = 16, BULK_MIN_WARPS = 4;
+
+__device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(smem_dst)),
+               "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
+__global__ void __launch_bounds__(BULK_MAX_WARPS * 32, 1) rmsnorm_bulk_kernel(const NormParams p) {
+  extern __shared__ __align__(128) uint8_t bulk_smem[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+  log_smid(p.smid_log);
+  const bool in_bf16 = p.x_bf16 != nullptr;
+  const uint32_t row_bytes = uint32_t(p.d) * (in_bf16 ? 2u : 4u);
+  const uint32_t buf_bytes = uint32_t(p.d) * 4u;             // buffers are sized for fp32 rows
+  uint64_t* bars = reinterpret_cast<uint64_t*>(bulk_smem);    // [n_warps][2]
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * BULK_MAX_WARPS);
+  uint8_t* bufs = bulk_smem + 512 + size_t(warp) * 2 * buf_bytes;
+  uint2* gains = reinterpret_cast<uint2*>(bulk_smem + 512 + size_t(n_warps) * 2 * buf_bytes);   // [d] bf16
+  for (int i = threadIdx.x; i < (p.d >> 2); i += blockDim.x) gains[i] = reinterpret_cast<const uint2*>(p.gain)[i];
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 2 * n_warps; ++i) mbar_init(&bars[i], 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  __syncthreads();
+  uint64_t* full = bars + 2 * warp;
+  const int stride = gridDim.x * n_warps, first = blockIdx.x * n_warps + warp;
+  const char* src = in_bf16 ? reinterpret_cast<const char*>(p.x_bf16) : reinterpret_cast<const char*>(p.x_f32);
+  auto request = [&](int k) {                                 // lane 0: row number k of this warp
+    const int row = first + k * stride;
+    if (row < p.T) {
+      mbar_expect_tx(&full[k & 1], row_bytes);
+      bulk_load_1d(bufs + (k & 1) * buf_bytes, src + size_t(row) * row_bytes, row_bytes, &full[k & 1]);
+    }
+  };
+  if (lane == 0) {
+    request(0);
+    request(1);
+  }
+  const int d4 = p.d >> 2;
+  const bool f16 = p.h_f16 != 0;
+  bool ok = true;
+  int k = 0;
+  for (int row = first; row < p.T; row += stride, ++k) {
+    ok = mbar_wait(&full[k & 1], (k >> 1) & 1, abort_flag, p.status);
+    if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+    const uint8_t* buf = bufs + (k & 1) * buf_bytes;
+    const float4* bf = reinterpret_cast<const float4*>(buf);
+    const uint2* bb = reinterpret_cast<const uint2*>(buf);
+    auto group = [&](int i) {                                 // elements 4i .. 4i + 3 of the row
+      if (!in_bf16) return bf[i];
+      const uint2 w = bb[i];
+      return make_float4(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xffff0000u),
+                         __uint_as_float(w.y << 16), __uint_as_float(w.y & 0xffff0000u));
+    };
+    // four independent partial sums per lane (groups i, i + 32, i + 64, i + 96 of every 128), combined in
+    // a fixed order: enough independent work per lane to cover the shared-memory latency
+    float s4[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int i0 = lane; i0 < d4; i0 += 128) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + 32 * u;
+        if (i < d4) {
+          const float4 a = group(i);
+          s4[u] += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+        }
+      }
+    }
+    const float ss = warp_sum((s4[0] + s4[1]) + (s4[2] + s4[3]));
+    const float r = rsqrtf(ss / float(p.d) + p.eps);
+    uint2* hdst = reinterpret_cast<uint2*>(p.h + size_t(row) * p.d);
+    float4* xo = reinterpret_cast<float4*>(p.x_f32_out + size_t(row) * p.d);
+    for (int i0 = lane; i0 < d4; i0 += 128) {
+      float4 a[4];
+      uint2 gw[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + 32 * u;
+        if (i < d4) {
+          a[u] = group(i);
+          gw[u] = gains[i];
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + 32 * u;
+        if (i < d4) {
+          const float g0 = __uint_as_float(gw[u].x << 16), g1 = __uint_as_float(gw[u].x & 0xffff0000u);
+          const float g2 = __uint_as_float(gw[u].y << 16), g3 = __uint_as_float(gw[u].y & 0xffff0000u);
+          hdst[i] = make_uint2(pack_act(a[u].x * r * g0, a[u].y * r * g1, f16),
+                               pack_act(a[u].z * r * g2, a[u].w * r * g3, f16));
+          if (in_bf16) xo[i] = a[u];                          // the widened copy that starts the residual stream
+        }
+      }
+    }
+    __syncwarp();                                             // every lane has read the buffer
+    if (lane == 0) request(k + 2);
+  }
+  if (!ok) drain_after_abort();
+}
+
 // One-time widening of the significand: bf16 weights -> fp16 copies (n8 groups of 8 values).  A bf16 value
 // is an fp16 value exactly when 2^-17 <= |w| <= 65504; smaller ones round to the fp16 subnormal grid
 // (absolute error <= 2^-25), larger ones saturate.
@@ -135,11 +245,26 @@ cudaError_t launch_bf16_to_f16(const void* src, void* dst, size_t n, cudaStream_
 }
 
 cudaError_t norm_set_attributes() {
-  return cudaFuncSetAttribute(rmsnorm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, NORM_SMEM);
+  cudaError_t e = cudaFuncSetAttribute(rmsnorm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, NORM_SMEM);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(rmsnorm_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              512 + BULK_SMEM_BUDGET);
 }
 
 cudaError_t launch_rmsnorm(const NormParams& p, int sm_budget, cudaStream_t stream) {
   if (p.T <= 0) return cudaSuccess;
+  // bulk-staged variant: as many warps as have room for two fp32 rows each (a function of d alone, never of
+  // the budget); rows too wide for four warps fall back to the register-staged kernel
+  const size_t pair_bytes = size_t(p.d) * 4 * 2, gain_bytes = size_t(p.d) * 2;
+  int warps = int((BULK_SMEM_BUDGET - gain_bytes) / pair_bytes);
+  if (warps > BULK_MAX_WARPS) warps = BULK_MAX_WARPS;
+  if (warps >= BULK_MIN_WARPS && p.status) {
+    const int blocks = (p.T + warps - 1) / warps;
+    const int grid = blocks < sm_budget ? blocks : sm_budget;
+    const size_t smem = 512 + size_t(warps) * pair_bytes + gain_bytes;
+    rmsnorm_bulk_kernel<<<grid, warps * 32, smem < size_t(kMinSmemBytes) ? size_t(kMinSmemBytes) : smem, stream>>>(p);
+    return cudaGetLastError();
+  }
   const int blocks = (p.T + NORM_WARPS - 1) / NORM_WARPS;
   const int grid = blocks < sm_budget ? blocks : sm_budget;
   rmsnorm_kernel<<<grid, NORM_THREADS, NORM_SMEM, stream>>>(p);
