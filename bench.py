@@ -35,8 +35,8 @@ METRIC = "shared_stage_tokens_per_s"
 UNIT = "tokens/s"
 SEED = {"c1_tiny": 0, "c2_shared": 1, "c3_7b": 2, "c4_talker": 3, "c3_decode": 2}
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one gate/up GEMM launch, from the ncu
-# capture summarised in profiles/gemm_gateup_c2_shared.md (None where no capture of that launch exists).
-GATEUP_DRAM_TRAFFIC_BYTES = {"c2_shared": 69852928 + 40344320}
+# capture summarised in profiles/gemm_pair_gateup_c2_shared.md (None where no capture of that launch exists).
+GATEUP_DRAM_TRAFFIC_BYTES = {"c2_shared": 69989376 + 39707904}
 
 
 def measured_peaks():
@@ -360,7 +360,8 @@ def main():
     achieved = gu_flops / gu_avg_s / 1e12
     peak = peaks["bf16_sustained"] * budget / stage.sm_count
     gemm_flops, attn_flops = flops_per_step(dims, batch)
-    roofline = {"bound": "tensor", "kernel": "gemm_kernel (gate/up + SwiGLU epilogue)", "achieved": achieved,
+    roofline = {"bound": "tensor", "kernel": "gemm_pair_kernel (gate/up + SwiGLU epilogue)" if T > 128 and budget >= 2 else
+                          "gemm_kernel (gate/up + SwiGLU epilogue)", "achieved": achieved,
                 "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                 "peak_source": f"{peaks['source']} sustained bf16 (fp16 operands: nominal ratio 1.0) x sm_budget/{stage.sm_count}",
                 "frac_of_burst_peak": achieved / (peaks["bf16_burst"] * budget / stage.sm_count),
