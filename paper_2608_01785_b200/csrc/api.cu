@@ -427,6 +427,11 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
   // More than one 128-row tile of tokens: the GEMMs run on pairs of SMs (a choice by shape, not by budget).
   const bool use_pair = T > 128;
   const int f16 = (c.flags & HS_FLAG_BF16_ACTIVATIONS) ? 0 : 1;   // format of h, o, act
+  // With the whole device as its budget a step has no neighbour to take SMs from, so each kernel is launched
+  // such that its set-up overlaps the previous kernel's drain.  With a smaller budget the blocks of the next
+  // kernel would wait on SMs outside the budget, so the launches stay strictly serial.  (Not while the
+  // per-kernel timers run: an event between two kernels serialises them anyway.)
+  const int overlap = (sm_budget == s->sm_count && !s->profile) ? 1 : 0;
   int* census = s->census ? reinterpret_cast<int*>(s->ws_dev + s->ws.smid) : nullptr;
   if (census && cudaMemsetAsync(census, 0, size_t(HS_PROFILE_CLASSES) * kSmidSlots * 4, stream) != cudaSuccess)
     return HS_ERR_CUDA;
@@ -447,6 +452,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     np.eps = c.rms_eps;
     np.h_f16 = f16;
     np.status = status;
+    np.overlap = overlap;
     np.smid_log = slots(0);
     { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
     if (e != cudaSuccess) break;
@@ -457,6 +463,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     g.M = T; g.N = q_dim + 2 * kv_dim; g.K = d;
     g.mode = kGemmQkv;
     g.ab_f16 = f16;
+    g.overlap = overlap;
     g.pair = use_pair;
     g.q_dim = q_dim; g.kv_dim = kv_dim; g.head_dim = Dh; g.n_kv_heads = c.n_kv_heads;
     g.tm_q = s->tm_q_st;
@@ -475,6 +482,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     a.tm_q = s->tm_q_attn;
     a.prefill_tokens = prefill_tokens_per_item(c.n_q_heads / c.n_kv_heads);
     a.o_f16 = f16;
+    a.overlap = overlap;
     a.q = q; a.o = o;
     a.n_q_heads = c.n_q_heads; a.n_kv_heads = c.n_kv_heads; a.head_dim = Dh;
     a.num_pages = c.num_pages; a.max_pages_per_seq = c.max_pages_per_seq; a.layer = l;
@@ -504,6 +512,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     go.M = T; go.N = d; go.K = q_dim;
     go.mode = kGemmResid;
     go.ab_f16 = f16;
+    go.overlap = overlap;
     go.tm_out = tm_y; go.accumulate = 1;
     go.pair = use_pair;
     go.bn = use_pair ? 256 : gemm_pick_bn(T, d, s->sm_count);
@@ -525,6 +534,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gu.M = T; gu.N = F; gu.K = d;
     gu.mode = kGemmGateUp;
     gu.ab_f16 = f16;
+    gu.overlap = overlap;
     gu.act_f16 = f16;
     gu.pair = use_pair;
     gu.tm_act = s->tm_act_st;
@@ -539,6 +549,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gd.M = T; gd.N = d; gd.K = F;
     gd.mode = kGemmResid;
     gd.ab_f16 = f16;
+    gd.overlap = overlap;
     gd.tm_out = tm_y; gd.accumulate = 1;
     gd.pair = use_pair;
     gd.bn = use_pair ? 256 : gemm_pick_bn(T, d, s->sm_count);

@@ -183,6 +183,8 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
     tma_prefetch_desc(&p.tm_kv);
   }
   __syncthreads();
+  griddep_wait();
+  griddep_launch_dependents();
 
   uint8_t* slots = smem + warp * DC_STAGES * SLOT_BYTES;
   uint64_t* full = full_all + warp * DC_STAGES;
@@ -372,7 +374,7 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
 
 template <typename K>
 cudaError_t set_smem(K kernel, int bytes) {
-  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  return set_kernel_smem(kernel, bytes);
 }
 
 }  // namespace
@@ -389,10 +391,9 @@ cudaError_t launch_attention_decode(const AttnParams& p, int sm_budget, cudaStre
   if (p.n_decode_items <= 0) return cudaSuccess;
   const int grid = p.n_decode_items < sm_budget ? p.n_decode_items : sm_budget;
   if (p.head_dim == 128)
-    attn_decode_kernel<128><<<grid, DC_THREADS, dc_smem_bytes<128>(), stream>>>(p);
+    return launch_step_kernel(attn_decode_kernel<128>, grid, DC_THREADS, dc_smem_bytes<128>(), stream, p.overlap != 0, p);
   else
-    attn_decode_kernel<64><<<grid, DC_THREADS, dc_smem_bytes<64>(), stream>>>(p);
-  return cudaGetLastError();
+    return launch_step_kernel(attn_decode_kernel<64>, grid, DC_THREADS, dc_smem_bytes<64>(), stream, p.overlap != 0, p);
 }
 
 }  // namespace hs

@@ -121,6 +121,8 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = bar->tmem_base;
+  griddep_wait();
+  griddep_launch_dependents();
 
   int rs = 0;
   uint32_t rph = 0;       // item ring slot / phase
@@ -380,21 +382,18 @@ constexpr int pf_smem_bytes() {
 }  // namespace
 
 cudaError_t attention_prefill_set_attributes() {
-  cudaError_t e = cudaFuncSetAttribute(attn_prefill_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       pf_smem_bytes<64>());
+  cudaError_t e = set_kernel_smem(attn_prefill_kernel<64>, pf_smem_bytes<64>());
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(attn_prefill_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              pf_smem_bytes<128>());
+  return set_kernel_smem(attn_prefill_kernel<128>, pf_smem_bytes<128>());
 }
 
 cudaError_t launch_attention_prefill(const AttnParams& p, int sm_budget, cudaStream_t stream) {
   if (p.n_prefill_items <= 0) return cudaSuccess;
   const int grid = p.n_prefill_items < sm_budget ? p.n_prefill_items : sm_budget;
   if (p.head_dim == 128)
-    attn_prefill_kernel<128><<<grid, PF_THREADS, pf_smem_bytes<128>(), stream>>>(p);
+    return launch_step_kernel(attn_prefill_kernel<128>, grid, PF_THREADS, pf_smem_bytes<128>(), stream, p.overlap != 0, p);
   else
-    attn_prefill_kernel<64><<<grid, PF_THREADS, pf_smem_bytes<64>(), stream>>>(p);
-  return cudaGetLastError();
+    return launch_step_kernel(attn_prefill_kernel<64>, grid, PF_THREADS, pf_smem_bytes<64>(), stream, p.overlap != 0, p);
 }
 
 }  // namespace hs

@@ -195,6 +195,8 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
   if (PAIR) cluster_sync_all();               // the other block's barriers exist before anything targets them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();                 // everything above is set-up; the operands belong to the previous kernel until here
+  griddep_launch_dependents();
 
   if (warp == 0) {
     // ------------------------------------------------------- TMA producer --
@@ -462,9 +464,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(GEMM_THREADS, 1)
 }  // namespace
 
 cudaError_t gemm_set_attributes() {
-  cudaError_t e = cudaFuncSetAttribute(gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
+  cudaError_t e = set_kernel_smem(gemm_pair_kernel, GEMM_SMEM);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM);
+  return set_kernel_smem(gemm_kernel, GEMM_SMEM);
 }
 
 int gemm_pick_bn(int M, int N, int sm_count) {
@@ -510,12 +512,10 @@ cudaError_t launch_gemm(const GemmParams& p, int sm_budget, cudaStream_t stream)
     // pairs of blocks (clusters of two SMs) on 256 x 256 tiles; an odd budget leaves one SM unused
     const int pairs = ((p.M + 2 * BM - 1) / (2 * BM)) * n_n_tiles;
     const int grid = 2 * (pairs < sm_budget / 2 ? pairs : sm_budget / 2);
-    gemm_pair_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(p);
-    return cudaGetLastError();
+    return launch_step_kernel(gemm_pair_kernel, grid, GEMM_THREADS, GEMM_SMEM, stream, p.overlap != 0, p);
   }
   const int grid = n_tiles < sm_budget ? n_tiles : sm_budget;
-  gemm_kernel<<<grid, GEMM_THREADS, GEMM_SMEM, stream>>>(p);
-  return cudaGetLastError();
+  return launch_step_kernel(gemm_kernel, grid, GEMM_THREADS, GEMM_SMEM, stream, p.overlap != 0, p);
 }
 
 }  // namespace hs

@@ -28,6 +28,7 @@ struct GemmParams {
   int M, N, K;               // N: Resid output width; Qkv (Hq + 2 Hkv) * Dh; GateUp F (activation width)
   int mode;
   int ab_f16;                // 1: both operands hold fp16 values; 0: both bf16
+  int overlap;               // 1: launch so that the set-up overlaps the previous kernel's drain
   int pair;                  // 1: run on pairs of SMs (256 x 256 tiles, bn = 256, no K split) when the budget allows
   // Resid
   CUtensorMap tm_out;        // fp32 [M, N], box 32 x 32, 128-byte swizzle (rows past M are clipped)
@@ -68,6 +69,7 @@ struct NormParams {
   int T, d;
   float eps;
   int h_f16;                 // 1 = write h as fp16, 0 = bf16
+  int overlap;               // 1: launch so that the set-up overlaps the previous kernel's drain
   int* status;               // device status word (bounded waits report HS_ERR_TIMEOUT here)
   int* smid_log;             // nullable: SM census slots of this launch
 };
@@ -83,6 +85,7 @@ struct AttnParams {
   CUtensorMap tm_q;                // q [max_tokens, q_dim]: box 64 x prefill_tokens, 128-byte swizzle
   int prefill_tokens;              // tokens per prefill work item
   int o_f16;                       // 1 = write o as fp16, 0 = bf16 (q, K, V are always bf16)
+  int overlap;               // 1: launch so that the set-up overlaps the previous kernel's drain
   const __nv_bfloat16* q;          // [T, q_dim] (after RoPE)
   __nv_bfloat16* o;                // [T, q_dim]
   int n_q_heads, n_kv_heads, head_dim, num_pages, max_pages_per_seq, layer;

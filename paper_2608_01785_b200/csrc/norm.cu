@@ -36,6 +36,8 @@ __global__ void __launch_bounds__(NORM_THREADS, 1) rmsnorm_kernel(const NormPara
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   log_smid(p.smid_log);
   float4* cache = reinterpret_cast<float4*>(norm_smem + warp * NORM_STAGE_FLOATS);
+  griddep_wait();
+  griddep_launch_dependents();
   const int d8 = p.d >> 3;                         // groups of 8 elements
   const int cached8 = min(d8, NORM_STAGE_FLOATS / 8);
   const uint4* gsrc = reinterpret_cast<const uint4*>(p.gain);
@@ -145,6 +147,8 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32, 1) rmsnorm_bulk_kernel(co
     fence_barrier_init();
   }
   __syncthreads();
+  griddep_wait();                 // the gains above are weights; the rows belong to the previous kernel until here
+  griddep_launch_dependents();
   uint64_t* full = bars + 2 * warp;
   const int stride = gridDim.x * n_warps, first = blockIdx.x * n_warps + warp;
   const char* src = in_bf16 ? reinterpret_cast<const char*>(p.x_bf16) : reinterpret_cast<const char*>(p.x_f32);
@@ -245,10 +249,9 @@ cudaError_t launch_bf16_to_f16(const void* src, void* dst, size_t n, cudaStream_
 }
 
 cudaError_t norm_set_attributes() {
-  cudaError_t e = cudaFuncSetAttribute(rmsnorm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, NORM_SMEM);
+  cudaError_t e = set_kernel_smem(rmsnorm_kernel, NORM_SMEM);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(rmsnorm_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              512 + BULK_SMEM_BUDGET);
+  return set_kernel_smem(rmsnorm_bulk_kernel, 512 + BULK_SMEM_BUDGET);
 }
 
 cudaError_t launch_rmsnorm(const NormParams& p, int sm_budget, cudaStream_t stream) {
@@ -262,13 +265,12 @@ cudaError_t launch_rmsnorm(const NormParams& p, int sm_budget, cudaStream_t stre
     const int blocks = (p.T + warps - 1) / warps;
     const int grid = blocks < sm_budget ? blocks : sm_budget;
     const size_t smem = 512 + size_t(warps) * pair_bytes + gain_bytes;
-    rmsnorm_bulk_kernel<<<grid, warps * 32, smem < size_t(kMinSmemBytes) ? size_t(kMinSmemBytes) : smem, stream>>>(p);
-    return cudaGetLastError();
+    return launch_step_kernel(rmsnorm_bulk_kernel, grid, warps * 32,
+                              smem < size_t(kMinSmemBytes) ? size_t(kMinSmemBytes) : smem, stream, p.overlap != 0, p);
   }
   const int blocks = (p.T + NORM_WARPS - 1) / NORM_WARPS;
   const int grid = blocks < sm_budget ? blocks : sm_budget;
-  rmsnorm_kernel<<<grid, NORM_THREADS, NORM_SMEM, stream>>>(p);
-  return cudaGetLastError();
+  return launch_step_kernel(rmsnorm_kernel, grid, NORM_THREADS, NORM_SMEM, stream, p.overlap != 0, p);
 }
 
 }  // namespace hs

@@ -290,4 +290,44 @@ __device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
+// ------------------------------------------------- programmatic dependent launch --
+// A kernel of a step may be launched while its predecessor in the stream is still running (see
+// launch_step_kernel).  It must then call griddep_wait() after its set-up (barrier initialisation, TMEM
+// allocation, descriptor prefetch: nothing that touches data of the step) and before its first access to
+// memory the predecessor reads or writes: the call returns once the predecessor has completed and its
+// writes are visible (at once when the kernel was launched the ordinary way).
+// griddep_launch_dependents() lets the successor be launched; it is issued right after the wait, so at
+// most two kernels of a step are ever in flight.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Host side: launches `kernel`; with `overlap` set, the launch carries the programmatic-stream-serialisation
+// attribute, i.e. its blocks may become resident (and run up to griddep_wait()) while the previous kernel of
+// the stream drains.
+template <typename P>
+inline cudaError_t launch_step_kernel(void (*kernel)(P), int grid, int block, size_t smem, cudaStream_t stream,
+                                      bool overlap, const P& params) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(grid), 1, 1);
+  cfg.blockDim = dim3(unsigned(block), 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = overlap ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, params);
+}
+
+// Host side: lets `kernel` use `bytes` of dynamic shared memory and asks for the largest shared-memory
+// carve-out.  Every kernel of a step asks for the same carve-out, so that no SM has to be reconfigured (and
+// drained for it) between two kernels of a step.
+template <typename K>
+inline cudaError_t set_kernel_smem(K kernel, int bytes) {
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+}
+
 }  // namespace hs
