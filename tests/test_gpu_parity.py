@@ -188,6 +188,10 @@ EDGE = {
     "long_prefill_dh128": (wl.StageDims(1, 256, 8, 1, 128, 640), [700, 1], [0, 1500]),
     "many_sequences": (wl.StageDims(1, 256, 4, 2, 64, 688), [1] * 40 + [3] * 10, list(range(0, 400, 10)) + [5] * 10),
     "two_layers_talker_like": (wl.StageDims(2, 1024, 16, 4, 64, 2816), [1] * 16, [128 + 57 * i for i in range(16)]),
+    # few tokens against a long K: the QKV and gate/up GEMMs split K four ways through the scratch tile
+    "small_step_split_k": (wl.StageDims(1, 2048, 8, 2, 128, 1024), [20, 1, 1], [0, 300, 17]),
+    # rows too wide for the bulk-staged RMSNorm (register-staged fallback), K split eight ways
+    "wide_rows_d8192": (wl.StageDims(1, 8192, 2, 2, 64, 128), [20, 1], [0, 37]),
 }
 
 
