@@ -23,7 +23,9 @@ HS_OK, HS_ERR_INVALID_ARG, HS_ERR_INVALID_BUDGET, HS_ERR_UNSUPPORTED_SHAPE, HS_E
 EXPORTS = ("hs_status_str", "hs_kv_pool_bytes", "hs_workspace_bytes", "hs_stage_create", "hs_stage_destroy",
            "hs_kv_alloc", "hs_kv_free", "hs_kv_free_pages", "hs_stage_plan", "hs_stage_step", "hs_stage_status",
            "hs_stage_sm_count", "hs_op_gemm_bf16", "hs_stage_debug_buffer", "hs_stage_profile_enable",
-           "hs_stage_profile_read", "hs_last_error", "hs_op_decode_attention_noalloc", "hs_op_gemm_f16")
+           "hs_stage_profile_read", "hs_last_error", "hs_op_decode_attention_noalloc", "hs_op_gemm_f16",
+           "hs_spatial_create", "hs_spatial_update", "hs_spatial_state", "hs_spatial_destroy",
+           "hs_spatial_derive_cap")
 PROFILE_CLASSES = ("rmsnorm", "gemm_qkv", "attn_prefill", "attn_decode", "attn_combine", "gemm_out", "gemm_gateup",
                    "gemm_down")
 
@@ -48,6 +50,12 @@ class hs_layer_weights_t(C.Structure):
 class hs_batch_t(C.Structure):
     _fields_ = [("n_seqs", C.c_int32), ("n_tokens", C.c_int32), ("q_len", C.c_void_p), ("ctx_len", C.c_void_p),
                 ("block_tables", C.c_void_p), ("x_in", C.c_void_p), ("y_out", C.c_void_p)]
+
+
+class hs_spatial_config_t(C.Structure):
+    _fields_ = [("abi_version", C.c_uint32), ("s_total", C.c_int32), ("s_aggr", C.c_int32), ("n_levels", C.c_int32),
+                ("ladder", C.POINTER(C.c_int32)), ("b_sat", C.c_double), ("gamma", C.c_double),
+                ("delta_step", C.c_int32)]
 
 
 class HsError(RuntimeError):
@@ -91,6 +99,12 @@ def lib() -> C.CDLL:
         l.hs_op_gemm_f16.argtypes = l.hs_op_gemm_bf16.argtypes
         l.hs_stage_debug_buffer.argtypes = [C.c_void_p, C.c_char_p, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
         l.hs_last_error.restype = C.c_char_p
+        l.hs_spatial_create.argtypes = [C.POINTER(hs_spatial_config_t), C.POINTER(C.c_void_p)]
+        l.hs_spatial_update.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        l.hs_spatial_state.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int32)]
+        l.hs_spatial_destroy.argtypes = [C.c_void_p]
+        l.hs_spatial_derive_cap.argtypes = [C.POINTER(C.c_int32), C.POINTER(C.c_double), C.c_int32, C.c_int32,
+                                            C.c_double, C.POINTER(C.c_int32)]
         l.hs_op_decode_attention_noalloc.argtypes = [C.c_void_p, C.c_void_p] + [C.c_int32] * 7 + \
             [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p]
         l.hs_stage_profile_enable.argtypes = [C.c_void_p, C.c_int32]
@@ -243,3 +257,55 @@ def hs_op_decode_attention_noalloc(q_ptr: int, kv_pool_ptr: int, n_layers: int, 
                                               C.c_void_p(cuda_stream))
     if st != HS_OK:
         raise HsError(st, "hs_op_decode_attention_noalloc")
+
+
+class SpatialController:
+    """The library's spatial controller (hs_spatial_*): per step, the shared stage's SM budget from downstream
+    activity and a memory-pressure sample (Sec. 4.3, Eq. 1 of the paper).  Marshalling only."""
+
+    def __init__(self, s_total: int, s_aggr: int, ladder: Sequence[int], b_sat: float, gamma: float, delta_step: int):
+        arr = (C.c_int32 * max(len(ladder), 1))(*ladder)
+        cfg = hs_spatial_config_t(HS_ABI_VERSION, s_total, s_aggr, len(ladder), arr, b_sat, gamma, delta_step)
+        h = C.c_void_p()
+        st = lib().hs_spatial_create(C.byref(cfg), C.byref(h))
+        if st != HS_OK:
+            raise HsError(st, "hs_spatial_create")
+        self.handle = h
+
+    def update(self, downstream_active: bool, pressure: float):
+        """Returns (s_shared, s_down) for the next step."""
+        a, b = C.c_int32(), C.c_int32()
+        st = lib().hs_spatial_update(self.handle, int(bool(downstream_active)), float(pressure), C.byref(a), C.byref(b))
+        if st != HS_OK:
+            raise HsError(st, "hs_spatial_update")
+        return a.value, b.value
+
+    def state(self):
+        """(moving average of the pressure, cap in force)."""
+        bhat, s = C.c_double(), C.c_int32()
+        st = lib().hs_spatial_state(self.handle, C.byref(bhat), C.byref(s))
+        if st != HS_OK:
+            raise HsError(st, "hs_spatial_state")
+        return bhat.value, s.value
+
+    def close(self) -> None:
+        if self.handle:
+            lib().hs_spatial_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def hs_spatial_derive_cap(budgets: Sequence[int], latency: Sequence[float], s_total: int, tolerance: float) -> int:
+    n = len(budgets)
+    b = (C.c_int32 * max(n, 1))(*budgets)
+    t = (C.c_double * max(n, 1))(*latency)
+    out = C.c_int32()
+    st = lib().hs_spatial_derive_cap(b, t, n, s_total, float(tolerance), C.byref(out))
+    if st != HS_OK:
+        raise HsError(st, "hs_spatial_derive_cap")
+    return out.value

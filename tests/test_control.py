@@ -83,3 +83,66 @@ def test_derive_cap_smallest_near_best_budget_below_full_allocation():
     assert derive_cap(budgets, lat, 142, 0.0) == 96
     assert derive_cap(budgets, lat, 142, 10.0) == 16
     assert derive_cap([148, 74], [1.0, 5.0], 148, 0.05) == 74      # only one candidate below the total
+
+
+# ------------------------------------------------------------- library vs oracle --
+def test_library_controller_matches_the_oracle_decision_by_decision():
+    from paper_2608_01785_b200 import binding as B
+    rng = np.random.default_rng(7)
+    for trial in range(40):
+        n = int(rng.integers(1, 9))
+        ladder = sorted(rng.choice(np.arange(1, 140), size=n, replace=False).tolist())
+        s_aggr = int(rng.integers(ladder[-1] + 1, 149))
+        gamma = float(rng.uniform(0.05, 1.0))
+        b_sat = float(rng.uniform(0.2, 2.0))
+        delta = int(rng.integers(0, 40))
+        orc = SpatialOracle(148, s_aggr, ladder, b_sat, gamma, delta)
+        ctl = B.SpatialController(148, s_aggr, ladder, b_sat, gamma, delta)
+        assert ctl.state() == (0.0, s_aggr)
+        active = False
+        for step in range(400):
+            if rng.uniform() < 0.1:
+                active = not active
+            b = float(rng.choice([rng.uniform(0, 2.5), 0.0, b_sat, b_sat / 2]))
+            assert ctl.update(active, b) == orc.update(active, b), (trial, step)
+            bhat, s = ctl.state()
+            assert bhat == orc.bhat and s == orc.s_shared          # same double arithmetic, same order
+        ctl.close()
+
+
+def test_library_controller_argument_errors():
+    from paper_2608_01785_b200 import binding as B
+    bad = [dict(ladder=[]), dict(ladder=[74, 48]), dict(ladder=[48, 48]), dict(ladder=[0, 48]), dict(ladder=[48, 148]),
+           dict(s_aggr=120), dict(s_aggr=149), dict(b_sat=0.0), dict(b_sat=float("nan")), dict(gamma=0.0),
+           dict(gamma=1.5), dict(delta_step=-1)]
+    for kw in bad:
+        args = dict(s_total=148, s_aggr=148, ladder=LADDER, b_sat=0.9, gamma=0.4, delta_step=1)
+        args.update(kw)
+        with pytest.raises(B.HsError) as e:
+            B.SpatialController(**args)
+        assert e.value.status == B.HS_ERR_INVALID_ARG, kw
+    ctl = B.SpatialController(148, 148, LADDER, 0.9, 0.4, 1)
+    ctl.update(True, 0.5)
+    before = ctl.state()
+    for b in (-0.1, float("inf"), float("nan")):
+        with pytest.raises(B.HsError):
+            ctl.update(True, b)
+    assert ctl.state() == before                                   # a refused sample changes nothing
+    ctl.close()
+
+
+def test_library_derive_cap_matches_the_oracle():
+    from paper_2608_01785_b200 import binding as B
+    rng = np.random.default_rng(3)
+    for _ in range(200):
+        n = int(rng.integers(2, 10))
+        budgets = rng.choice(np.arange(1, 149), size=n, replace=False).tolist()
+        if min(budgets) == 148:
+            continue
+        lat = rng.uniform(1.0, 20.0, size=n).tolist()
+        tol = float(rng.choice([0.0, 0.05, 0.2, 3.0]))
+        assert B.hs_spatial_derive_cap(budgets, lat, 148, tol) == derive_cap(budgets, lat, 148, tol)
+    with pytest.raises(B.HsError):
+        B.hs_spatial_derive_cap([148], [1.0], 148, 0.05)           # nothing below the full allocation
+    with pytest.raises(B.HsError):
+        B.hs_spatial_derive_cap([74, 74], [1.0, 2.0], 148, 0.05)   # budgets must be distinct
