@@ -4,8 +4,12 @@ Each scheduler tick issues one backbone step (every sequence in its decode phase
 one first-come-first-served prefill chunk of at most `max_prefill_chunk` tokens) and, when downstream work
 exists, one talker step (at most `max_talker` sequences) on a second stream with the complementary SM
 budget -- the co-running regime whose SM split the paper's spatial controller chooses per step (Sec. 4.3,
-Algorithm 1 steps 3-4).  The per-tick backbone budget comes from a seeded stand-in policy: all SMs when
-the talker is idle, otherwise a uniform draw from the ladder.  Time is virtual: the clock advances by the
+Algorithm 1 steps 3-4).  The per-tick backbone budget comes from one of two policies: "seeded" (all SMs when
+the talker is idle, otherwise a uniform draw from the ladder: it visits every budget equally often, which is
+what the latency-by-budget tables want) or "controller" (the library's spatial controller, Eq. 1 of the
+paper, driven by a measured pressure sample per tick: the bytes the two steps of the previous tick had to
+read -- weights once per step, the KV pages of every sequence -- divided by the tick's duration and by the
+GPU's measured copy bandwidth).  Time is virtual: the clock advances by the
 measured latency of each tick and idle gaps are skipped, so a long trace replays in GPU time only.
 
 The engine is pluggable: `GpuEngine` drives real stages through the C ABI; `ModelEngine` is a latency
@@ -35,6 +39,11 @@ class ReplayConfig:
     talker_ctx0: int = 128          # conditioning tokens a talker sequence starts from
     ladder: Tuple[int, ...] = (120, 96, 74, 48)
     policy_seed: int = 5
+    policy: str = "seeded"          # "seeded" | "controller"
+    hbm_gbs: float = 6547.2         # measured copy bandwidth: normalises the controller's pressure samples
+    b_sat: float = 0.5              # pressure (fraction of hbm_gbs) at which the cap reaches the top of the ladder
+    gamma: float = 0.4              # weight of the newest pressure sample (the value of the paper's Fig. 10)
+    delta_step: int = 20            # smallest change of the cap that is applied while co-running (SMs)
 
 
 @dataclass
@@ -66,6 +75,7 @@ class ModelEngine(Engine):
     """Latency model + real page accounting on host-only stages (no GPU)."""
 
     def __init__(self, dims_a, dims_b, pages_a: int, pages_b: int, mpps_a: int, mpps_b: int):
+        self.dims_a, self.dims_b = dims_a, dims_b
         self.h = {}
         for name, dims, pages, mpps in (("a", dims_a, pages_a, mpps_a), ("b", dims_b, pages_b, mpps_b)):
             cfg = B.make_config(dims, pages, 4096, 128, mpps, mpps * 16, device=-1)
@@ -103,6 +113,7 @@ class GpuEngine(Engine):
         import torch
         from .stage import Stage
         self.torch = torch
+        self.dims_a, self.dims_b = dims_a, dims_b
         dev = torch.device("cuda", device)
         max_tok_a = cfg.max_decode + cfg.max_prefill_chunk
         self.sa = Stage(dims_a, wl.make_weights(dims_a, seed, dev), pages_a, max_tok_a, cfg.max_decode + 1, mpps_a,
@@ -160,9 +171,25 @@ class GpuEngine(Engine):
         self.sb.close()
 
 
+def step_bytes(dims, batch) -> float:
+    """Bytes one step of a stage has to read: its weights once, and the cached K/V of every sequence."""
+    if not batch:
+        return 0.0
+    kv = sum(ctx + q for _, q, ctx in batch) * 2 * dims.kv_dim * 2 * dims.n_layers
+    return float(dims.params_per_layer() * dims.n_layers * 2 + kv)
+
+
 def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = ReplayConfig()) -> Dict:
     """Runs the whole trace; returns aggregate metrics (virtual seconds)."""
     rng = np.random.Generator(np.random.PCG64(cfg.policy_seed))
+    ctl = None
+    if cfg.policy == "controller":
+        ctl = B.SpatialController(engine.sm_count, engine.sm_count, sorted(cfg.ladder), cfg.b_sat, cfg.gamma,
+                                  cfg.delta_step)
+    pressure = 0.0                  # sample of the previous tick
+    pressures: List[float] = []
+    cap_changes = 0
+    prev_budget = None
     waiting: Deque[_Seq] = deque()
     prefilling: Optional[_Seq] = None
     decoding: List[_Seq] = []
@@ -211,9 +238,18 @@ def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = Repl
             ctx = cfg.talker_ctx0 + s.talker_done
             engine.alloc("b", s.req.rid, ctx + 1)
             b_batch.append((s.req.rid, 1, ctx))
-        budget = engine.sm_count if not b_batch else int(rng.choice(cfg.ladder))
+        if ctl is not None:
+            budget, _ = ctl.update(bool(b_batch), pressure)
+        else:
+            budget = engine.sm_count if not b_batch else int(rng.choice(cfg.ladder))
+        if prev_budget is not None and budget != prev_budget:
+            cap_changes += 1
+        prev_budget = budget
         lat_a, lat_b = engine.tick(a_batch, b_batch, budget)
         tick_ms = max(lat_a or 0.0, lat_b or 0.0)
+        moved = step_bytes(engine.dims_a, a_batch) + step_bytes(engine.dims_b, b_batch)
+        pressure = moved / (tick_ms * 1e-3) / (cfg.hbm_gbs * 1e9) if tick_ms > 0 else 0.0
+        pressures.append(pressure)
         t += tick_ms * 1e-3
         busy_s += tick_ms * 1e-3
         if lat_a is not None:
@@ -268,7 +304,11 @@ def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = Repl
         ttfo = [(s.t_first_down - s.req.arrival_s) * 1e3 for s in sel if s.t_first_down is not None]
         by_class[cls] = {"requests": len(sel), "ttft_ms_p50": pct(ttft, 50), "ttft_ms_p95": pct(ttft, 95),
                          "first_downstream_ms_p50": pct(ttfo, 50), "first_downstream_ms_p95": pct(ttfo, 95)}
-    return {"requests_done": len(done), "virtual_seconds": t, "busy_seconds": busy_s,
+    if ctl is not None:
+        ctl.close()
+    return {"requests_done": len(done), "virtual_seconds": t, "busy_seconds": busy_s, "policy": cfg.policy,
+            "pressure": {"mean": statistics.fmean(pressures) if pressures else None, "p95": pct(pressures, 95)},
+            "cap_changes": cap_changes,
             "backbone_tokens": backbone_tokens, "talker_tokens": talker_tokens,
             "backbone_tokens_per_s": backbone_tokens / busy_s if busy_s else None,
             "tick_ms_by_budget": {str(b): {"n": len(v), "mean": statistics.fmean(v), "p50": pct(v, 50), "p95": pct(v, 95)}
@@ -290,8 +330,10 @@ def main():
     ap.add_argument("--requests", type=int, default=2000)
     ap.add_argument("--backbone", default="c3_7b")
     ap.add_argument("--talker", default="c4_talker")
+    ap.add_argument("--policy", default="seeded", choices=["seeded", "controller"])
+    ap.add_argument("--b-sat", type=float, default=ReplayConfig.b_sat)
     args = ap.parse_args()
-    cfg = ReplayConfig()
+    cfg = ReplayConfig(policy=args.policy, b_sat=args.b_sat)
     pa, pb, ma, mb = pool_sizes(cfg)
     eng = GpuEngine(wl.DIMS[args.backbone], wl.DIMS[args.talker], pa, pb, ma, mb, cfg)
     try:

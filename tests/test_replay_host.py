@@ -44,3 +44,30 @@ def test_replay_conserves_tokens_and_pages():
         assert res["virtual_seconds"] >= res["busy_seconds"] > 0
     finally:
         eng.close()
+
+
+def test_replay_under_the_spatial_controller():
+    """The same replay with the library's controller choosing the budget: while the talker has work the
+    backbone never gets more than the top of the ladder, it gets all SMs when the talker is idle, the cap
+    follows the pressure (higher b_sat -> lower caps), and tokens and pages are conserved as before."""
+    trace = wl.make_trace(16.0, 60, seed=4)
+    seen = {}
+    for b_sat in (0.05, 1e6):
+        cfg = ReplayConfig(max_decode=8, max_prefill_chunk=256, max_talker=4, policy="controller", b_sat=b_sat,
+                           hbm_gbs=0.01)                 # a tiny "peak" so that the model engine's ticks register
+        pa, pb, ma, mb = pool_sizes(cfg)
+        eng = ModelEngine(wl.DIMS["c1_tiny"], wl.DIMS["c1_tiny"], pa, pb, ma, mb)
+        try:
+            res = replay(trace, eng, cfg)
+            assert res["requests_done"] == 60 and res["policy"] == "controller"
+            assert res["backbone_tokens"] == sum(r.prompt_len + r.backbone_out for r in trace)
+            assert eng.free_pages("a") == pa and eng.free_pages("b") == pb
+            budgets = {int(b): v["n"] for b, v in res["tick_ms_by_budget"].items()}
+            assert set(budgets) <= {148, *cfg.ladder} and 148 in budgets
+            assert res["pressure"]["mean"] > 0
+            seen[b_sat] = budgets
+        finally:
+            eng.close()
+    co = lambda d: {b: n for b, n in d.items() if b != 148}
+    assert max(co(seen[0.05])) == 120            # saturated pressure: the top of the ladder, never beyond it
+    assert set(co(seen[1e6])) == {48}            # negligible pressure: the bottom of the ladder
