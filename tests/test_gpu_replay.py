@@ -7,9 +7,11 @@ from paper_2608_01785_b200 import workloads as wl
 pytestmark = pytest.mark.gpu
 
 
-def test_replay_small_trace_on_gpu():
+@pytest.mark.parametrize("policy", ["seeded", "controller"])
+def test_replay_small_trace_on_gpu(policy):
     from paper_2608_01785_b200.replay import GpuEngine, ReplayConfig, pool_sizes, replay
-    cfg = ReplayConfig(max_decode=12, max_prefill_chunk=512, max_talker=4, ladder=(120, 96, 74, 48))
+    cfg = ReplayConfig(max_decode=12, max_prefill_chunk=512, max_talker=4, ladder=(120, 96, 74, 48), policy=policy,
+                       b_sat=0.02)          # small stages move few bytes: a low saturation point makes the cap move
     trace = [wl.Request(r.rid, r.arrival_s, r.out_class, min(r.prompt_len, 900), min(r.backbone_out, 40),
                         min(r.talker_out, 60)) for r in wl.make_trace(16.0, 30, seed=4)]
     pa, pb, ma, mb = pool_sizes(cfg, max_prompt=900, max_out=40, max_talker_out=60)
