@@ -201,9 +201,10 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
     }
     first_round = false;
     if (item >= p.n_decode_items || *abort_flag) break;
-    const int4 it = reinterpret_cast<const int4*>(p.decode_items)[item];
+    // one 32-byte record: {decode row, kv head, first key, end key} {seq, token row, group's first item, splits}
+    const int4 it = reinterpret_cast<const int4*>(p.decode_items)[2 * item];
+    const int4 dr = reinterpret_cast<const int4*>(p.decode_items)[2 * item + 1];
     const int drow = it.x, hk = it.y, k0 = it.z, k1 = it.w;
-    const int4 dr = reinterpret_cast<const int4*>(p.decode_rows)[drow];   // {seq, token row, first item, splits}
     const int seq = dr.x, tok = dr.y, splits = dr.w;
     const int n_pages = (k1 - k0 + 15) >> 4;
     const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq + (k0 >> 4);
@@ -362,7 +363,7 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
     last = __shfl_sync(0xffffffffu, last, 0);
     if (last) {
       __threadfence();
-      const int first = dr.z + hk * splits;
+      const int first = dr.z;
       if (G <= 8) merge_group<DH, 4, DC_STAGES * SLOT_BYTES>(p.part_o, p.part_ml, slots, first, splits, G, lane, orow, p.o_f16 != 0);
       else merge_group<DH, 2, DC_STAGES * SLOT_BYTES>(p.part_o, p.part_ml, slots, first, splits, G, lane, orow, p.o_f16 != 0);
       if (lane == 0) *done = 0;             // ready for the next launch

@@ -49,7 +49,8 @@ struct MetaLayout {
   int seq_tok0, seq_ctx, seq_qlen;   // [max_seqs]        first token row, cached tokens, new tokens
   int block_tables;                  // [max_seqs * max_pages_per_seq]
   int prefill_items;                 // [max_prefill_items * 4]  {seq, kv_head, first token of the tile, tokens}
-  int decode_items;                  // [max_decode_items * 4]   {decode row, kv_head, first key, end key}
+  int decode_items;                  // [max_decode_items * 8]   {decode row, kv_head, first key, end key,
+                                     //                           seq, token row, first item of the group, splits}
   int decode_rows;                   // [max_seqs * 4]           {seq, token row, first item, splits}
   int counters;                      // [n_layers * 2]           work-queue heads, zero at step start
   int group_done;                    // [max_seqs * n_kv_heads]  finished decode splits per group, zero

@@ -94,7 +94,8 @@ struct AttnParams {
   const int32_t* block_tables;
   const int32_t* prefill_items;    // int4 per item
   int n_prefill_items;
-  const int32_t* decode_items;     // int4 per item: {decode row, kv head, first key, end key}
+  const int32_t* decode_items;     // two int4 per item: {decode row, kv head, first key, end key}
+                                   //                    {seq, token row, first item of its group, splits}
   int n_decode_items;
   const int32_t* decode_rows;      // int4 per decode sequence
   int n_decode_rows;

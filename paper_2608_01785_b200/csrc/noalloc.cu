@@ -37,8 +37,8 @@ constexpr int kOffGroupDone = 8;                                  // [kMaxSeqs *
 constexpr int kOffSeqTok0 = kOffGroupDone + kMaxSeqs * 16;        // [kMaxSeqs]
 constexpr int kOffSeqCtx = kOffSeqTok0 + kMaxSeqs;                // [kMaxSeqs]
 constexpr int kOffTables = kOffSeqCtx + kMaxSeqs;                 // [kMaxSeqs * kMaxPagesPerSeq]
-constexpr int kOffItems = kOffTables + kMaxSeqs * kMaxPagesPerSeq;   // [kMaxItems * 4]
-constexpr int kOffRows = kOffItems + kMaxItems * 4;               // [kMaxSeqs * 4]
+constexpr int kOffItems = kOffTables + kMaxSeqs * kMaxPagesPerSeq;   // [kMaxItems * 8]
+constexpr int kOffRows = kOffItems + kMaxItems * 8;               // [kMaxSeqs * 4]
 constexpr int kMetaWords = kOffRows + kMaxSeqs * 4;
 constexpr int kOffPartMl = (kMetaWords + 63) & ~63;               // [kMaxItems * 16 * 2] floats
 constexpr int kOffPartO = kOffPartMl + kMaxItems * 32;            // [kMaxItems * 16 * 128] floats
@@ -130,9 +130,10 @@ extern "C" hs_status_t hs_op_decode_attention_noalloc(const void* q_dev, const v
     row[0] = s; row[1] = s; row[2] = n_items; row[3] = splits;
     for (int hk = 0; hk < n_kv_heads; ++hk)
       for (int j = 0; j < splits; ++j) {
-        int32_t* it = meta + kOffItems + (n_items + hk * splits + j) * 4;
+        int32_t* it = meta + kOffItems + (n_items + hk * splits + j) * 8;
         it[0] = s; it[1] = hk; it[2] = j * kDecodeSplit;
         it[3] = keys < (j + 1) * kDecodeSplit ? keys : (j + 1) * kDecodeSplit;
+        it[4] = s; it[5] = s; it[6] = n_items + hk * splits; it[7] = splits;   // one query row per sequence
       }
     n_items += n_kv_heads * splits;
   }

@@ -77,7 +77,7 @@ MetaLayout make_meta_layout(const hs_stage_config_t& c) {
   m.seq_qlen = take(c.max_seqs);
   m.block_tables = take(c.max_seqs * c.max_pages_per_seq);
   m.prefill_items = take(m.max_prefill_items * 4);
-  m.decode_items = take(m.max_decode_items * 4);
+  m.decode_items = take(m.max_decode_items * 8);
   m.decode_rows = take(c.max_seqs * 4);
   m.counters = take(c.n_layers * 2);
   m.group_done = take(c.max_seqs * c.n_kv_heads);
@@ -145,8 +145,9 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
         row[0] = s; row[1] = t; row[2] = n_dec_items; row[3] = splits;
         for (int hk = 0; hk < c.n_kv_heads; ++hk)
           for (int j = 0; j < splits; ++j) {
-            int32_t* it = meta + ml.decode_items + (n_dec_items + hk * splits + j) * 4;
+            int32_t* it = meta + ml.decode_items + (n_dec_items + hk * splits + j) * 8;
             it[0] = n_dec_rows; it[1] = hk; it[2] = j * kDecodeSplit; it[3] = std::min(keys, (j + 1) * kDecodeSplit);
+            it[4] = s; it[5] = t; it[6] = n_dec_items + hk * splits; it[7] = splits;
           }
       }
       n_dec_items += c.n_kv_heads * splits;
