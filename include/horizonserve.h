@@ -182,6 +182,9 @@ hs_status_t hs_stage_plan(hs_stage_t *stage, const hs_batch_t *batch, int32_t *t
  * ctx_len .. ctx_len + q_len - 1; their K/V are written to the cache pages named by the block table and
  * every new token attends causally to positions 0..p.  y_out receives all n_tokens rows.  Re-running
  * the same step rewrites the same slots with the same values.  The caller advances ctx_len itself.
+ * With sm_budget < the device's SM count every kernel of the step starts only after the previous one has
+ * ended, so that no block of the step ever sits on an SM outside the budget; with sm_budget == SM count
+ * (no co-running neighbour) each kernel's set-up overlaps the previous kernel's drain.
  * Errors (nothing launched): INVALID_ARG, INVALID_BUDGET, BAD_BLOCK_TABLE, NO_DEVICE, CUDA.
  */
 hs_status_t hs_stage_step(hs_stage_t *stage, const hs_batch_t *batch, int32_t sm_budget, void *cuda_stream);

@@ -58,7 +58,10 @@ hs_status_t hs_stage_debug_buffer(hs_stage_t *stage, const char *name, void **de
  * events on the step's stream.  hs_stage_profile_read synchronises those events and adds, per
  * kernel class, the elapsed milliseconds to ms[class] and the launch count to launches[class]
  * (host arrays of HS_PROFILE_CLASSES entries, accumulated since the last read), then forgets them.
- * Classes: 0 rmsnorm, 1 qkv gemm, 2 prefill attention, 3 decode attention, 4 decode combine,
+ * While enabled, the kernels of a step never overlap (the events between them serialise the stream), so the
+ * per-class times add up to slightly more than an unprofiled full-budget step takes.
+ * Classes: 0 rmsnorm, 1 qkv gemm, 2 prefill attention, 3 decode attention (with the merge of its split
+ * partials), 4 unused (always zero; kept so that the class numbers stay what they were),
  * 5 out-proj gemm, 6 gate/up gemm, 7 down gemm.
  * Errors: INVALID_ARG, NO_DEVICE, CUDA.
  */
