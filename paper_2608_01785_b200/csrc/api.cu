@@ -465,6 +465,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     g.ab_f16 = f16;
     g.overlap = overlap;
     g.pair = use_pair;
+    g.bn = use_pair ? 256 : 128;     // small steps: 128-column tiles, twice as many SMs stream the weights
     g.q_dim = q_dim; g.kv_dim = kv_dim; g.head_dim = Dh; g.n_kv_heads = c.n_kv_heads;
     g.tm_q = s->tm_q_st;
     g.k_cache = s->kv_pool + (size_t(l) * 2 + 0) * layer_kv_elems;

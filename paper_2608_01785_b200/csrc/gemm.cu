@@ -48,11 +48,16 @@ constexpr int GEMM_SMEM = 1024 + RING_BYTES + 4 * EPI_WARP_BYTES + 256;
 static_assert(GEMM_SMEM <= 227 * 1024, "fits one SM");
 static_assert(GEMM_SMEM >= kMinSmemBytes, "one block per SM");
 
+// Qkv mode, single blocks: tiles of 128 virtual columns (one B box) when p.bn says so -- the launcher asks for
+// them at small M, where the tile count decides how many SMs stream weights; 256 otherwise.  A 128-column
+// tile never straddles q | k | v (their widths are multiples of 128) and holds whole heads.
+__host__ __device__ __forceinline__ int gemm_qkv_width(const GemmParams& p) { return p.bn == 128 && !p.pair ? 128 : BN; }
+
 // Output-tile width: 256 virtual columns, except in Resid mode where the launcher picks p.bn (a multiple
 // of 32 in [128, 256]) from the problem shape so that the tile count fills whole waves of SMs.
 __host__ __device__ __forceinline__ int gemm_n_tiles(const GemmParams& p) {
   if (p.mode == kGemmGateUp) return (p.N + 127) / 128;
-  const int bn = p.mode == kGemmResid ? p.bn : BN;
+  const int bn = p.mode == kGemmResid ? p.bn : gemm_qkv_width(p);
   return (p.N + bn - 1) / bn;
 }
 
@@ -60,7 +65,7 @@ struct BSource { int map, row; };
 __device__ __forceinline__ BSource b_source(const GemmParams& p, int n_tile, int half) {
   if (p.mode == kGemmResid) return {0, n_tile * p.bn + half * 128};
   if (p.mode == kGemmGateUp) return {half, n_tile * 128};
-  int v = n_tile * BN + half * 128;
+  int v = n_tile * gemm_qkv_width(p) + half * 128;
   if (v < p.q_dim) return {0, v};
   v -= p.q_dim;
   if (v < p.kv_dim) return {1, v};
@@ -204,7 +209,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      const bool two_halves = p.mode != kGemmResid || p.bn > 128;
+      const bool two_halves = p.mode == kGemmGateUp || (p.mode == kGemmResid ? p.bn : gemm_qkv_width(p)) > 128;
       for (int u = worker; u < n_units && ok; u += n_workers) {
         const int tile = u % n_tiles, ks = u / n_tiles;
         const int m = tile % n_m_tiles, n = tile / n_m_tiles;
@@ -234,7 +239,8 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
     if (lane == 0 && rank == 0) {
       // both operands are fp16 or both bf16 (one MMA cannot mix the two): the format fields of A (bits 7..9)
       // and B (bits 10..12) are 0 for fp16 and 1 for bf16
-      const uint32_t idesc = umma_idesc_bf16_f32(PAIR ? 2 * BM : BM, p.mode == kGemmResid && !PAIR ? p.bn : BN) &
+      const uint32_t idesc = umma_idesc_bf16_f32(PAIR ? 2 * BM : BM,
+                                                 PAIR ? BN : p.mode == kGemmResid ? p.bn : p.mode == kGemmQkv ? gemm_qkv_width(p) : BN) &
                              (p.ab_f16 ? ~(63u << 7) : ~0u);
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
@@ -365,8 +371,9 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
         const int pos = row_ok ? p.tok_pos[row] : 0;
         const int slot = row_ok ? p.tok_slot[row] : 0;
         const int half_dh = Dh >> 1;
-        for (int half = 0; half < 2; ++half) {
-          int vcol = n * BN + half * 128;         // virtual column of this half in [q | k | v]
+        const int qkv_w = gemm_qkv_width(p);
+        for (int half = 0; half < qkv_w / 128; ++half) {
+          int vcol = n * qkv_w + half * 128;      // virtual column of this half in [q | k | v]
           if (vcol >= p.N) break;
           int region = 0;
           if (vcol >= p.q_dim) { region = 1; vcol -= p.q_dim; }
