@@ -25,7 +25,8 @@ EXPORTS = ("hs_status_str", "hs_kv_pool_bytes", "hs_workspace_bytes", "hs_stage_
            "hs_stage_sm_count", "hs_op_gemm_bf16", "hs_stage_debug_buffer", "hs_stage_profile_enable",
            "hs_stage_profile_read", "hs_last_error", "hs_op_decode_attention_noalloc", "hs_op_gemm_f16",
            "hs_spatial_create", "hs_spatial_update", "hs_spatial_state", "hs_spatial_destroy",
-           "hs_spatial_derive_cap")
+           "hs_spatial_derive_cap", "hs_head_workspace_bytes", "hs_head_create", "hs_head_step", "hs_head_status",
+           "hs_head_destroy", "hs_op_embed")
 PROFILE_CLASSES = ("rmsnorm", "gemm_qkv", "attn_prefill", "attn_decode", "attn_combine", "gemm_out", "gemm_gateup",
                    "gemm_down")
 
@@ -50,6 +51,11 @@ class hs_layer_weights_t(C.Structure):
 class hs_batch_t(C.Structure):
     _fields_ = [("n_seqs", C.c_int32), ("n_tokens", C.c_int32), ("q_len", C.c_void_p), ("ctx_len", C.c_void_p),
                 ("block_tables", C.c_void_p), ("x_in", C.c_void_p), ("y_out", C.c_void_p)]
+
+
+class hs_head_config_t(C.Structure):
+    _fields_ = [("abi_version", C.c_uint32), ("device", C.c_int32), ("d_model", C.c_int32), ("vocab", C.c_int32),
+                ("rms_eps", C.c_float), ("max_rows", C.c_int32)]
 
 
 class hs_spatial_config_t(C.Structure):
@@ -99,6 +105,16 @@ def lib() -> C.CDLL:
         l.hs_op_gemm_f16.argtypes = l.hs_op_gemm_bf16.argtypes
         l.hs_stage_debug_buffer.argtypes = [C.c_void_p, C.c_char_p, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]
         l.hs_last_error.restype = C.c_char_p
+        l.hs_head_workspace_bytes.restype = C.c_size_t
+        l.hs_head_workspace_bytes.argtypes = [C.POINTER(hs_head_config_t)]
+        l.hs_head_create.argtypes = [C.POINTER(hs_head_config_t), C.c_void_p, C.c_void_p, C.c_void_p,
+                                     C.POINTER(C.c_void_p)]
+        l.hs_head_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32,
+                                   C.c_void_p]
+        l.hs_head_status.argtypes = [C.c_void_p]
+        l.hs_head_destroy.argtypes = [C.c_void_p]
+        l.hs_op_embed.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32,
+                                  C.c_void_p, C.c_void_p]
         l.hs_spatial_create.argtypes = [C.POINTER(hs_spatial_config_t), C.POINTER(C.c_void_p)]
         l.hs_spatial_update.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         l.hs_spatial_state.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int32)]
@@ -309,3 +325,44 @@ def hs_spatial_derive_cap(budgets: Sequence[int], latency: Sequence[float], s_to
     if st != HS_OK:
         raise HsError(st, "hs_spatial_derive_cap")
     return out.value
+
+
+def make_head_config(d_model: int, vocab: int, rms_eps: float, max_rows: int, device: int = 0) -> hs_head_config_t:
+    return hs_head_config_t(HS_ABI_VERSION, device, d_model, vocab, rms_eps, max_rows)
+
+
+def hs_head_workspace_bytes(cfg: hs_head_config_t) -> int:
+    return int(lib().hs_head_workspace_bytes(C.byref(cfg)))
+
+
+def hs_head_create(cfg: hs_head_config_t, g_final_ptr: int, w_vocab_ptr: int, workspace_ptr: int) -> int:
+    h = C.c_void_p()
+    st = lib().hs_head_create(C.byref(cfg), C.c_void_p(g_final_ptr), C.c_void_p(w_vocab_ptr), C.c_void_p(workspace_ptr),
+                              C.byref(h))
+    if st != HS_OK:
+        raise HsError(st, "hs_head_create")
+    return h.value
+
+
+def hs_head_step(head: int, y_ptr: int, rows_ptr: int, n: int, logits_ptr: int, tokens_ptr: int, sm_budget: int,
+                 cuda_stream: int = 0) -> None:
+    st = lib().hs_head_step(C.c_void_p(head), C.c_void_p(y_ptr), C.c_void_p(rows_ptr), n, C.c_void_p(logits_ptr),
+                            C.c_void_p(tokens_ptr), sm_budget, C.c_void_p(cuda_stream))
+    if st != HS_OK:
+        raise HsError(st, "hs_head_step")
+
+
+def hs_head_status(head: int) -> int:
+    return int(lib().hs_head_status(C.c_void_p(head)))
+
+
+def hs_head_destroy(head: int) -> None:
+    lib().hs_head_destroy(C.c_void_p(head))
+
+
+def hs_op_embed(tokens_ptr: int, n: int, table_ptr: int, vocab: int, d_model: int, x_out_ptr: int, sm_budget: int,
+                status_ptr: int, cuda_stream: int = 0) -> None:
+    st = lib().hs_op_embed(C.c_void_p(tokens_ptr), n, C.c_void_p(table_ptr), vocab, d_model, C.c_void_p(x_out_ptr),
+                           sm_budget, C.c_void_p(status_ptr), C.c_void_p(cuda_stream))
+    if st != HS_OK:
+        raise HsError(st, "hs_op_embed")

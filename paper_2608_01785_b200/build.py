@@ -8,10 +8,11 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libhorizonserve.so")
-SOURCES = ["api.cu", "gemm.cu", "attention.cu", "attention_prefill.cu", "norm.cu", "noalloc.cu", "plan.cc", "control.cc"]
+SOURCES = ["api.cu", "gemm.cu", "attention.cu", "attention_prefill.cu", "norm.cu", "noalloc.cu", "head.cu", "plan.cc", "control.cc"]
 HEADERS = ["hs_internal.h", "kernels.h", "ptx.cuh", os.path.join("..", "..", "include", "horizonserve.h"),
            os.path.join("..", "..", "include", "horizonserve_ops.h"),
-           os.path.join("..", "..", "include", "horizonserve_control.h")]
+           os.path.join("..", "..", "include", "horizonserve_control.h"),
+           os.path.join("..", "..", "include", "horizonserve_head.h")]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr"]
 

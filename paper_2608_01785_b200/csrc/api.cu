@@ -7,6 +7,7 @@
 #include <string>
 #include <vector>
 
+#include "../../include/horizonserve_head.h"
 #include "../../include/horizonserve_ops.h"
 #include "hs_internal.h"
 #include "kernels.h"
@@ -132,6 +133,7 @@ hs_status_t ensure_attributes(int device) {
   if ((e = gemm_set_attributes()) != cudaSuccess) return cuda_fail("gemm attributes", e);
   if ((e = norm_set_attributes()) != cudaSuccess) return cuda_fail("rmsnorm attributes", e);
   if ((e = attention_set_attributes()) != cudaSuccess) return cuda_fail("attention attributes", e);
+  if ((e = head_set_attributes()) != cudaSuccess) return cuda_fail("head attributes", e);
   if (device >= 0 && device < 64) g_attrs_set[device] = true;
   return HS_OK;
 }
@@ -668,3 +670,140 @@ hs_status_t hs_op_gemm_f16(const void* a, const void* w, const float* resid, flo
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------ ends of the stage --
+struct hs_head {
+  hs_head_config_t cfg;
+  int sm_count = 0;
+  uint8_t* ws_dev = nullptr;       // [max_rows][d] bf16 h, then the status word
+  size_t off_status = 0;
+  const __nv_bfloat16* g_final = nullptr;
+  CUtensorMap tm_h, tm_w;
+};
+
+namespace {
+bool head_config_ok(const hs_head_config_t& c) {
+  return c.abi_version == HS_ABI_VERSION && c.device >= 0 && c.d_model >= 64 && c.d_model % 8 == 0 && c.vocab >= 8 &&
+         c.vocab % 8 == 0 && c.max_rows >= 1 && c.max_rows <= 128 && c.rms_eps > 0.f;
+}
+size_t head_status_offset(const hs_head_config_t& c) { return align_up(size_t(c.max_rows) * c.d_model * 2, 1024); }
+}  // namespace
+
+size_t hs_head_workspace_bytes(const hs_head_config_t* cfg) {
+  if (!cfg || !head_config_ok(*cfg)) return 0;
+  return head_status_offset(*cfg) + 1024;
+}
+
+hs_status_t hs_head_create(const hs_head_config_t* cfg, const void* g_final, const void* w_vocab, void* workspace_dev,
+                           hs_head_t** out) {
+  if (!cfg || !out) return HS_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!head_config_ok(*cfg)) return cfg->abi_version != HS_ABI_VERSION ? HS_ERR_INVALID_ARG : HS_ERR_UNSUPPORTED_SHAPE;
+  if (!g_final || !w_vocab || !workspace_dev) return HS_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(g_final) & 15) || (reinterpret_cast<uintptr_t>(w_vocab) & 15) ||
+      (reinterpret_cast<uintptr_t>(workspace_dev) & 255))
+    return HS_ERR_INVALID_ARG;
+  DeviceGuard guard(cfg->device);
+  if (!guard.ok) return HS_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess || prop.major != 10) return HS_ERR_CUDA;
+  hs_status_t st = ensure_attributes(cfg->device);
+  if (st != HS_OK) return st;
+  std::unique_ptr<hs_head> h(new (std::nothrow) hs_head());
+  if (!h) return HS_ERR_INVALID_ARG;
+  h->cfg = *cfg;
+  h->sm_count = prop.multiProcessorCount;
+  h->ws_dev = static_cast<uint8_t*>(workspace_dev);
+  h->off_status = head_status_offset(*cfg);
+  h->g_final = static_cast<const __nv_bfloat16*>(g_final);
+  if (!encode_2d(&h->tm_h, h->ws_dev, cfg->max_rows, cfg->d_model, 128) ||
+      !encode_2d(&h->tm_w, w_vocab, cfg->vocab, cfg->d_model, 128))
+    return HS_ERR_CUDA;
+  if (cudaMemset(h->ws_dev + h->off_status, 0, 256) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess)
+    return HS_ERR_CUDA;
+  *out = h.release();
+  return HS_OK;
+}
+
+hs_status_t hs_head_step(hs_head_t* h, const float* y, const int32_t* rows, int32_t n, float* logits, int32_t* tokens,
+                         int32_t sm_budget, void* cuda_stream) {
+  if (!h || !y || !rows || !logits || !tokens || n < 1 || n > h->cfg.max_rows) return HS_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(logits) & 15) return HS_ERR_INVALID_ARG;
+  if (sm_budget < 1 || sm_budget > h->sm_count) return HS_ERR_INVALID_BUDGET;
+  DeviceGuard guard(h->cfg.device);
+  if (!guard.ok) return HS_ERR_CUDA;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  int* status = reinterpret_cast<int*>(h->ws_dev + h->off_status);
+  const int d = h->cfg.d_model, V = h->cfg.vocab;
+
+  NormParams np{};
+  np.x_f32 = y;
+  np.gain = h->g_final;
+  np.h = reinterpret_cast<__nv_bfloat16*>(h->ws_dev);
+  np.T = n;
+  np.d = d;
+  np.eps = h->cfg.rms_eps;
+  np.row_index = rows;
+  np.status = status;
+  cudaError_t e = launch_rmsnorm(np, sm_budget, stream);
+  if (e != cudaSuccess) return cuda_fail("head rmsnorm", e);
+
+  GemmParams g{};
+  g.tm_a = h->tm_h;
+  g.tm_b[0] = g.tm_b[1] = g.tm_b[2] = h->tm_w;
+  if (!encode_2d(&g.tm_out, logits, n, V, 32, true)) return HS_ERR_CUDA;
+  g.M = n; g.N = V; g.K = d;
+  g.mode = kGemmResid;
+  g.accumulate = 0;                          // plain store of the logits
+  g.pair = 0;
+  g.bn = gemm_pick_bn(n, V, h->sm_count);
+  g.ksplit = 1;
+  g.status = status;
+  e = launch_gemm(g, sm_budget, stream);
+  if (e != cudaSuccess) return cuda_fail("head gemm", e);
+
+  ArgmaxParams a{};
+  a.logits = logits;
+  a.tokens = tokens;
+  a.n = n;
+  a.vocab = V;
+  e = launch_argmax(a, sm_budget, stream);
+  return e == cudaSuccess ? HS_OK : cuda_fail("head argmax", e);
+}
+
+hs_status_t hs_head_status(hs_head_t* h) {
+  if (!h) return HS_ERR_INVALID_ARG;
+  DeviceGuard guard(h->cfg.device);
+  int v = 0;
+  if (cudaMemcpy(&v, h->ws_dev + h->off_status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return HS_ERR_CUDA;
+  return v == 0 ? HS_OK : static_cast<hs_status_t>(v);
+}
+
+hs_status_t hs_head_destroy(hs_head_t* h) {
+  if (!h) return HS_ERR_INVALID_ARG;
+  delete h;
+  return HS_OK;
+}
+
+hs_status_t hs_op_embed(const int32_t* tokens, int32_t n, const void* table, int32_t vocab, int32_t d_model, void* x_out,
+                        int32_t sm_budget, int32_t* status_dev, void* cuda_stream) {
+  if (!tokens || !table || !x_out || !status_dev || n < 1 || vocab < 1) return HS_ERR_INVALID_ARG;
+  if (d_model < 8 || d_model % 8 != 0) return HS_ERR_UNSUPPORTED_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(table) & 15) || (reinterpret_cast<uintptr_t>(x_out) & 15)) return HS_ERR_INVALID_ARG;
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return HS_ERR_CUDA;
+  if (prop.major != 10) return HS_ERR_CUDA;
+  if (sm_budget < 1 || sm_budget > prop.multiProcessorCount) return HS_ERR_INVALID_BUDGET;
+  if (ensure_attributes(dev) != HS_OK) return HS_ERR_CUDA;
+  EmbedParams p{};
+  p.tokens = tokens;
+  p.table = static_cast<const __nv_bfloat16*>(table);
+  p.x_out = static_cast<__nv_bfloat16*>(x_out);
+  p.n = n;
+  p.vocab = vocab;
+  p.d = d_model;
+  p.status = status_dev;
+  const cudaError_t e = launch_embed(p, sm_budget, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? HS_OK : cuda_fail("embed", e);
+}

@@ -68,12 +68,30 @@ struct NormParams {
   __nv_bfloat16* h;
   int T, d;
   float eps;
+  const int* row_index;      // nullable: input row of output row t is row_index[t] (device int32 [T]); else t
   int h_f16;                 // 1 = write h as fp16, 0 = bf16
   int overlap;               // 1: launch so that the set-up overlaps the previous kernel's drain
   int* status;               // device status word (bounded waits report HS_ERR_TIMEOUT here)
   int* smid_log;             // nullable: SM census slots of this launch
 };
 cudaError_t launch_rmsnorm(const NormParams& p, int sm_budget, cudaStream_t stream);
+
+// Embedding lookup and greedy sampling (head.cu).
+struct EmbedParams {
+  const int32_t* tokens;           // device [n]
+  const __nv_bfloat16* table;      // [vocab, d]
+  __nv_bfloat16* x_out;            // [n, d]
+  int n, vocab, d;
+  int* status;                     // receives HS_ERR_INVALID_ARG for an id outside the table
+};
+struct ArgmaxParams {
+  const float* logits;             // [n, vocab]
+  int32_t* tokens;                 // [n]: lowest index of each row's maximum
+  int n, vocab;
+};
+cudaError_t head_set_attributes();
+cudaError_t launch_embed(const EmbedParams& p, int sm_budget, cudaStream_t stream);
+cudaError_t launch_argmax(const ArgmaxParams& p, int sm_budget, cudaStream_t stream);
 // dst[i] = fp16(src[i]) for n bf16 values (n a multiple of 8, both 16-byte aligned); used once per weight
 // matrix when a stage is created
 cudaError_t launch_bf16_to_f16(const void* src, void* dst, size_t n, cudaStream_t stream);

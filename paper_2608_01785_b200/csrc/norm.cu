@@ -43,8 +43,9 @@ __global__ void __launch_bounds__(NORM_THREADS, 1) rmsnorm_kernel(const NormPara
   const uint4* gsrc = reinterpret_cast<const uint4*>(p.gain);
   for (int row = blockIdx.x * NORM_WARPS + warp; row < p.T; row += gridDim.x * NORM_WARPS) {
     float ss = 0.f;
-    const uint4* xb = reinterpret_cast<const uint4*>(p.x_bf16 + size_t(row) * p.d);
-    const float4* xf = reinterpret_cast<const float4*>(p.x_f32 + size_t(row) * p.d);
+    const int src_row = p.row_index ? p.row_index[row] : row;
+    const uint4* xb = reinterpret_cast<const uint4*>(p.x_bf16 + size_t(src_row) * p.d);
+    const float4* xf = reinterpret_cast<const float4*>(p.x_f32 + size_t(src_row) * p.d);
     float4* xo = reinterpret_cast<float4*>(p.x_f32_out + size_t(row) * p.d);
     // four groups per lane are requested before any is used, to keep enough bytes in flight
     for (int i0 = lane; i0 < d8; i0 += 128) {
@@ -155,8 +156,9 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32, 1) rmsnorm_bulk_kernel(co
   auto request = [&](int k) {                                 // lane 0: row number k of this warp
     const int row = first + k * stride;
     if (row < p.T) {
+      const int src_row = p.row_index ? p.row_index[row] : row;
       mbar_expect_tx(&full[k & 1], row_bytes);
-      bulk_load_1d(bufs + (k & 1) * buf_bytes, src + size_t(row) * row_bytes, row_bytes, &full[k & 1]);
+      bulk_load_1d(bufs + (k & 1) * buf_bytes, src + size_t(src_row) * row_bytes, row_bytes, &full[k & 1]);
     }
   };
   if (lane == 0) {

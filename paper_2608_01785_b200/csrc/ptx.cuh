@@ -11,6 +11,7 @@
 namespace hs {
 
 constexpr int kErrTimeout = 7;                       // HS_ERR_TIMEOUT
+constexpr int kErrInvalidArg = 1;                    // HS_ERR_INVALID_ARG
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // a bounded wait gives up after 2 s
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

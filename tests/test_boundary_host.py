@@ -22,7 +22,7 @@ def host_stage(dims=wl.DIMS["c1_tiny"], num_pages=64, max_tokens=256, max_seqs=1
 
 def declared_functions():
     names = []
-    for header in ("horizonserve.h", "horizonserve_ops.h", "horizonserve_control.h"):
+    for header in ("horizonserve.h", "horizonserve_ops.h", "horizonserve_control.h", "horizonserve_head.h"):
         text = open(os.path.join(ROOT, "include", header)).read()
         text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
         names += re.findall(r"\b(hs_[a-z0-9_]+)\s*\(", text)
