@@ -206,13 +206,65 @@ def run_reference(args, rank: int):
     print(json.dumps(line))
 
 
+def run_head(args):
+    """Auxiliary measurement (not the headline metric): the sampling head behind a config-3 step -- final
+    RMSNorm on the last row of each of the 65 sequences, the 152064 x 3584 vocabulary projection and the
+    row-wise argmax -- and the embedding lookup in front of it.  HBM-bound: the vocabulary matrix is read once."""
+    from paper_2608_01785_b200 import binding as B
+    dev = torch.device("cuda", 0)
+    d, V, n, T = wl.DIMS["c3_7b"].d_model, 152064, 65, 2112
+    g = torch.Generator(device="cpu").manual_seed(11)
+    y = torch.randn(T, d, generator=g).to(dev)
+    gain = (1.0 + 0.02 * torch.randn(d, generator=g)).to(torch.bfloat16).to(dev)
+    w = (0.02 * torch.randn(V, d, device=dev)).to(torch.bfloat16)
+    rows = torch.arange(T - n, T, dtype=torch.int32, device=dev)
+    cfg = B.make_head_config(d, V, 1e-6, 128)
+    ws = torch.empty(B.hs_head_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
+    head = B.hs_head_create(cfg, gain.data_ptr(), w.data_ptr(), ws.data_ptr())
+    logits = torch.empty(n, V, device=dev)
+    tokens = torch.empty(n, dtype=torch.int32, device=dev)
+    x_emb = torch.empty(n, d, dtype=torch.bfloat16, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    budget = args.sm_budget or torch.cuda.get_device_properties(dev).multi_processor_count
+    stream = torch.cuda.Stream(device=dev)
+
+    def one():
+        B.hs_head_step(head, y.data_ptr(), rows.data_ptr(), n, logits.data_ptr(), tokens.data_ptr(), budget,
+                       stream.cuda_stream)
+        B.hs_op_embed(tokens.data_ptr(), n, w.data_ptr(), V, d, x_emb.data_ptr(), budget, status.data_ptr(),
+                      stream.cuda_stream)
+
+    with torch.cuda.stream(stream):
+        for _ in range(max(args.warmup, 3)):
+            one()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            one()
+        e1.record(stream)
+    torch.cuda.synchronize()
+    assert B.hs_head_status(head) == 0 and status.item() == 0
+    ms = e0.elapsed_time(e1) / args.steps
+    B.hs_head_destroy(head)
+    peaks = measured_peaks()
+    bytes_moved = V * d * 2 + n * V * 4 * 2                     # the matrix once, the logits written and read
+    print(json.dumps({"metric": "sampled_tokens_per_s", "value": n / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+                      "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms, "higher_is_better": True,
+                      "dtype": "bf16", "data": "synthetic",
+                      "config": {"workload": "c3_head", "d_model": d, "vocab": V, "rows": n, "sm_budget": budget,
+                                 "l2": "the 1.09 GB vocabulary matrix exceeds L2"},
+                      "roofline": {"bound": "hbm", "kernel": "head step (rmsnorm + vocabulary GEMM + argmax) + embed",
+                                   "achieved": bytes_moved / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": bytes_moved / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2_shared", choices=sorted(SEED))
+    ap.add_argument("--workload", default="c2_shared", choices=sorted(SEED) + ["c3_head"])
     ap.add_argument("--sm-budget", type=int, default=0, help="0 = all SMs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--bf16-activations", action="store_true",
@@ -231,6 +283,10 @@ def main():
         return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the CUDA library is the only implementation of the step")
+    if args.workload == "c3_head":
+        if rank == 0:
+            run_head(args)
+        return
 
     import torch.distributed as dist
     from paper_2608_01785_b200 import binding as B

@@ -126,6 +126,13 @@ int pick_ksplit(int M, int N, int K, int bn, int sm_count) {
   return gemm_pick_ksplit(M, N, K, bn, sm_count);
 }
 
+// SM count and compute-capability major of a device, through the attribute queries (cudaGetDeviceProperties
+// takes milliseconds, too slow for a per-call check).
+bool device_info(int dev, int* sm_count, int* major) {
+  return cudaDeviceGetAttribute(sm_count, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess &&
+         cudaDeviceGetAttribute(major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess;
+}
+
 bool g_attrs_set[64] = {};
 hs_status_t ensure_attributes(int device) {
   if (device >= 0 && device < 64 && g_attrs_set[device]) return HS_OK;
@@ -632,10 +639,10 @@ static hs_status_t op_gemm(const void* a, const void* w, const float* resid, flo
       (reinterpret_cast<uintptr_t>(out) & 15) || (reinterpret_cast<uintptr_t>(resid) & 15))
     return HS_ERR_INVALID_ARG;
   int dev = 0;
-  cudaDeviceProp prop;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return HS_ERR_CUDA;
-  if (prop.major != 10) return HS_ERR_CUDA;
-  if (sm_budget < 1 || sm_budget > prop.multiProcessorCount) return HS_ERR_INVALID_BUDGET;
+  int sm_count = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || !device_info(dev, &sm_count, &major)) return HS_ERR_CUDA;
+  if (major != 10) return HS_ERR_CUDA;
+  if (sm_budget < 1 || sm_budget > sm_count) return HS_ERR_INVALID_BUDGET;
   if (ensure_attributes(dev) != HS_OK) return HS_ERR_CUDA;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   GemmParams g{};
@@ -649,7 +656,7 @@ static hs_status_t op_gemm(const void* a, const void* w, const float* resid, flo
   g.ab_f16 = ab_f16;
   g.accumulate = resid != nullptr;
   g.pair = M > 128;
-  g.bn = g.pair ? 256 : gemm_pick_bn(M, N, prop.multiProcessorCount);
+  g.bn = g.pair ? 256 : gemm_pick_bn(M, N, sm_count);
   // the kernel adds into `out`: a residual that lives elsewhere is copied there first
   if (resid && resid != out &&
       cudaMemcpyAsync(out, resid, size_t(M) * N * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
@@ -791,10 +798,10 @@ hs_status_t hs_op_embed(const int32_t* tokens, int32_t n, const void* table, int
   if (d_model < 8 || d_model % 8 != 0) return HS_ERR_UNSUPPORTED_SHAPE;
   if ((reinterpret_cast<uintptr_t>(table) & 15) || (reinterpret_cast<uintptr_t>(x_out) & 15)) return HS_ERR_INVALID_ARG;
   int dev = 0;
-  cudaDeviceProp prop;
-  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return HS_ERR_CUDA;
-  if (prop.major != 10) return HS_ERR_CUDA;
-  if (sm_budget < 1 || sm_budget > prop.multiProcessorCount) return HS_ERR_INVALID_BUDGET;
+  int sm_count = 0, major = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || !device_info(dev, &sm_count, &major)) return HS_ERR_CUDA;
+  if (major != 10) return HS_ERR_CUDA;
+  if (sm_budget < 1 || sm_budget > sm_count) return HS_ERR_INVALID_BUDGET;
   if (ensure_attributes(dev) != HS_OK) return HS_ERR_CUDA;
   EmbedParams p{};
   p.tokens = tokens;
