@@ -163,6 +163,7 @@ struct hs_stage {
   std::vector<hs_layer_weights_t> layers;
   std::vector<LayerMaps> maps;
   CUtensorMap tm_h, tm_o, tm_act, tm_kv;   // operand loads
+  CUtensorMap tm_h_s[2], tm_o_s[2], tm_act_s[2];   // the same A operands with 64- and 32-row boxes (small steps)
   CUtensorMap tm_q_st, tm_act_st;          // epilogue stores (box 64 x 32)
   CUtensorMap tm_q_attn;                   // Q tiles of the prefill attention (box 64 x tokens per item)
   int32_t* pinned[kRing] = {};
@@ -295,6 +296,11 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
   const uint64_t q_dim = uint64_t(cfg->n_q_heads) * cfg->head_dim, kv_dim = uint64_t(cfg->n_kv_heads) * cfg->head_dim;
   bool ok = encode_2d(&s->tm_h, s->ws_dev + s->ws.h, T, d, 128) && encode_2d(&s->tm_o, s->ws_dev + s->ws.o, T, q_dim, 128) &&
             encode_2d(&s->tm_act, s->ws_dev + s->ws.act, T, F, 128);
+  for (int i = 0; i < 2 && ok; ++i) {
+    const uint32_t rows = i == 0 ? 64 : 32;
+    ok = encode_2d(&s->tm_h_s[i], s->ws_dev + s->ws.h, T, d, rows) && encode_2d(&s->tm_o_s[i], s->ws_dev + s->ws.o, T, q_dim, rows) &&
+         encode_2d(&s->tm_act_s[i], s->ws_dev + s->ws.act, T, F, rows);
+  }
   ok = ok && encode_2d(&s->tm_q_st, s->ws_dev + s->ws.q, T, q_dim, 32) &&
        encode_2d(&s->tm_act_st, s->ws_dev + s->ws.act, T, F, 32);
   ok = ok && encode_2d(&s->tm_q_attn, s->ws_dev + s->ws.q, T, q_dim,
@@ -441,6 +447,9 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
   // kernel would wait on SMs outside the budget, so the launches stay strictly serial.  (Not while the
   // per-kernel timers run: an event between two kernels serialises them anyway.)
   const int overlap = (sm_budget == s->sm_count && !s->profile) ? 1 : 0;
+  // A operands of a small step are fetched with boxes of 64 or 32 rows instead of 128
+  const int a_rows = use_pair ? 128 : (T <= 32 ? 32 : T <= 64 ? 64 : 128);
+  const int a_sel = a_rows == 64 ? 0 : 1;
   int* census = s->census ? reinterpret_cast<int*>(s->ws_dev + s->ws.smid) : nullptr;
   if (census && cudaMemsetAsync(census, 0, size_t(HS_PROFILE_CLASSES) * kSmidSlots * 4, stream) != cudaSuccess)
     return HS_ERR_CUDA;
@@ -467,7 +476,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     if (e != cudaSuccess) break;
 
     GemmParams g{};
-    g.tm_a = s->tm_h;
+    g.tm_a = a_rows == 128 ? s->tm_h : s->tm_h_s[a_sel];
+    g.a_box_rows = a_rows;
     g.tm_b[0] = m.wq; g.tm_b[1] = m.wk; g.tm_b[2] = m.wv;
     g.M = T; g.N = q_dim + 2 * kv_dim; g.K = d;
     g.mode = kGemmQkv;
@@ -517,7 +527,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     if (e != cudaSuccess) break;
 
     GemmParams go{};
-    go.tm_a = s->tm_o;
+    go.tm_a = a_rows == 128 ? s->tm_o : s->tm_o_s[a_sel];
+    go.a_box_rows = a_rows;
     go.tm_b[0] = m.wo; go.tm_b[1] = m.wo; go.tm_b[2] = m.wo;
     go.M = T; go.N = d; go.K = q_dim;
     go.mode = kGemmResid;
@@ -539,7 +550,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     if (e != cudaSuccess) break;
 
     GemmParams gu{};
-    gu.tm_a = s->tm_h;
+    gu.tm_a = a_rows == 128 ? s->tm_h : s->tm_h_s[a_sel];
+    gu.a_box_rows = a_rows;
     gu.tm_b[0] = m.wgate; gu.tm_b[1] = m.wup; gu.tm_b[2] = m.wup;
     gu.M = T; gu.N = F; gu.K = d;
     gu.mode = kGemmGateUp;
@@ -554,7 +566,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     if (e != cudaSuccess) break;
 
     GemmParams gd{};
-    gd.tm_a = s->tm_act;
+    gd.tm_a = a_rows == 128 ? s->tm_act : s->tm_act_s[a_sel];
+    gd.a_box_rows = a_rows;
     gd.tm_b[0] = m.wdown; gd.tm_b[1] = m.wdown; gd.tm_b[2] = m.wdown;
     gd.M = T; gd.N = d; gd.K = F;
     gd.mode = kGemmResid;

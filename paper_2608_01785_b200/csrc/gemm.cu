@@ -40,11 +40,12 @@ template <bool PAIR> struct Ring {
 };
 constexpr int RING_BYTES = 4 * (A_BYTES + 2 * BH_BYTES);
 static_assert(Ring<true>::STAGES * Ring<true>::STAGE_BYTES == RING_BYTES, "both rings fill the same space");
+constexpr int kMaxStages = 12;                  // barrier slots; the ring holds fewer when stages are large
 constexpr int GEMM_THREADS = 192;
 constexpr int TMEM_COLS = 512;                  // two 128 x 256 fp32 accumulators
 constexpr int EPI_BUF_BYTES = 4096;             // 32 rows x 128 B: a 32 x 32 fp32 or 32 x 64 bf16 output block
 constexpr int EPI_WARP_BYTES = 2 * EPI_BUF_BYTES;   // two blocks per epilogue warp, filled alternately
-constexpr int GEMM_SMEM = 1024 + RING_BYTES + 4 * EPI_WARP_BYTES + 256;
+constexpr int GEMM_SMEM = 1024 + RING_BYTES + 4 * EPI_WARP_BYTES + 384;
 static_assert(GEMM_SMEM <= 227 * 1024, "fits one SM");
 static_assert(GEMM_SMEM >= kMinSmemBytes, "one block per SM");
 
@@ -143,13 +144,22 @@ __device__ __forceinline__ __nv_bfloat16* cache_ptr(__nv_bfloat16* base, int slo
 
 template <bool PAIR>
 __device__ __forceinline__ void gemm_body(const GemmParams& p) {
-  constexpr int STAGES = Ring<PAIR>::STAGES, STAGE_BYTES = Ring<PAIR>::STAGE_BYTES;
+  // Ring geometry.  Pairs: 6 stages of 32 KB.  Single blocks: a stage holds the A box (128 rows, or only 64 / 32
+  // when the step is that small) and one or two 128-row B boxes, and the ring holds as many stages as fit (at
+  // most kMaxStages): a block's streaming rate is stages in flight / memory latency, so the small stages of a
+  // small step buy depth -- 8 or 9 stages instead of 4.
+  const bool b_two = p.mode == kGemmGateUp || (p.mode == kGemmResid ? p.bn : gemm_qkv_width(p)) > 128;
+  const int a_bytes = (p.a_box_rows > 0 && !PAIR ? p.a_box_rows : BM) * BK * 2;
+  const int STAGE_BYTES = PAIR ? Ring<true>::STAGE_BYTES : a_bytes + (b_two ? 2 : 1) * BH_BYTES;
+  const int STAGES = PAIR ? Ring<true>::STAGES
+                          : (RING_BYTES / STAGE_BYTES < kMaxStages ? RING_BYTES / STAGE_BYTES : kMaxStages);
+  const int b_off = PAIR ? A_BYTES : a_bytes;     // B boxes follow the A box inside a stage
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* epi_smem = smem + RING_BYTES;
   uint64_t* full = reinterpret_cast<uint64_t*>(epi_smem + 4 * EPI_WARP_BYTES);
-  uint64_t* empty = full + 6;
-  uint64_t* tfull = empty + 6;
+  uint64_t* empty = full + kMaxStages;
+  uint64_t* tfull = empty + kMaxStages;
   uint64_t* tempty = tfull + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -209,7 +219,10 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      const bool two_halves = p.mode == kGemmGateUp || (p.mode == kGemmResid ? p.bn : gemm_qkv_width(p)) > 128;
+      // A small step's A box holds only the rows that exist (32 or 64 instead of 128): the MMA still reads 128
+      // rows starting at the stage's base -- beyond the A box that is the B data of the stage, finite values
+      // that only reach accumulator rows no epilogue stores
+      const bool two_halves = b_two;
       for (int u = worker; u < n_units && ok; u += n_workers) {
         const int tile = u % n_tiles, ks = u / n_tiles;
         const int m = tile % n_m_tiles, n = tile / n_m_tiles;
@@ -223,12 +236,12 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
             const uint32_t bar = mapa_u32(smem_u32(&full[s]), 0);
             if (rank == 0) mbar_expect_tx(&full[s], 2 * STAGE_BYTES);
             tma_load_2d_pair(st, &p.tm_a, bar, kb * BK, (2 * m + int(rank)) * BM);
-            tma_load_2d_pair(st + A_BYTES, &p.tm_b[b0.map], bar, kb * BK, b0.row);
+            tma_load_2d_pair(st + b_off, &p.tm_b[b0.map], bar, kb * BK, b0.row);
           } else {
-            mbar_expect_tx(&full[s], two_halves ? STAGE_BYTES : A_BYTES + BH_BYTES);
+            mbar_expect_tx(&full[s], a_bytes + (two_halves ? 2 * BH_BYTES : BH_BYTES));
             tma_load_2d(st, &p.tm_a, &full[s], kb * BK, m * BM);
-            tma_load_2d(st + A_BYTES, &p.tm_b[b0.map], &full[s], kb * BK, b0.row);
-            if (two_halves) tma_load_2d(st + A_BYTES + BH_BYTES, &p.tm_b[b1.map], &full[s], kb * BK, b1.row);
+            tma_load_2d(st + b_off, &p.tm_b[b0.map], &full[s], kb * BK, b0.row);
+            if (two_halves) tma_load_2d(st + b_off + BH_BYTES, &p.tm_b[b1.map], &full[s], kb * BK, b1.row);
           }
           if (++s == STAGES) { s = 0; ph ^= 1; }
         }
@@ -255,7 +268,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
           tc_fence_after_sync();
           const uint32_t a_addr = smem_u32(smem + s * STAGE_BYTES);
           const uint64_t a_desc = umma_desc_kmajor_sw128(a_addr);
-          const uint64_t b_desc = umma_desc_kmajor_sw128(a_addr + A_BYTES);
+          const uint64_t b_desc = umma_desc_kmajor_sw128(a_addr + b_off);
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {  // 16 bf16 = 32 B along K: +2 in the (address / 16) field
             if (PAIR) umma_bf16_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, ((kb - kb_begin) | k) != 0);

@@ -28,6 +28,7 @@ struct GemmParams {
   int M, N, K;               // N: Resid output width; Qkv (Hq + 2 Hkv) * Dh; GateUp F (activation width)
   int mode;
   int ab_f16;                // 1: both operands hold fp16 values; 0: both bf16
+  int a_box_rows;            // rows of tm_a's box: 128, or 64 / 32 when M is that small (0 means 128); single blocks only
   int overlap;               // 1: launch so that the set-up overlaps the previous kernel's drain
   int pair;                  // 1: run on pairs of SMs (256 x 256 tiles, bn = 256, no K split) when the budget allows
   // Resid
