@@ -1,5 +1,6 @@
 /*
- * horizonserve_control.h -- the spatial controller that chooses hs_stage_step's sm_budget per step: the
+ * horizonserve_control.h -- the two host-side controllers around hs_stage_step.  First the spatial one, which
+ * chooses the step's sm_budget: the
  * bandwidth-guided SM throttling of the paper (Sec. 4.3, Eq. 1; Algorithm 1 step 3), and the offline choice
  * of the co-running cap from a fixed-SM sweep (Sec. 4.1, "SLO and SM-ladder construction").  Host-only: no
  * call touches a GPU or allocates device memory; all pointers are host pointers.
@@ -76,6 +77,57 @@ hs_status_t hs_spatial_destroy(hs_spatial_t *ctl);
  */
 hs_status_t hs_spatial_derive_cap(const int32_t *budgets, const double *latency, int32_t n, int32_t s_total,
                                   double tolerance, int32_t *s_cap);
+
+/*
+ * ---------------------------------------------------------------------------------------------------------
+ * The temporal scheduler's view: which requests the base scheduler may see in one scheduling step
+ * (Sec. 4.1 "Remaining-slack ratio", Sec. 4.2 "Shared-Stage Path Rotation"; Algorithm 1 steps 1-2).
+ *
+ * Per request the caller passes its path (0 short: ends after the shared stage; 1 long: activates a
+ * downstream stage), its stage (0 waiting for or in prefill; 1 decode continuation), its first-response
+ * deadline d and a coarse estimate rhat of the time it still needs.  One call is one scheduling step k:
+ *     u = (d - now) / rhat;  protected = u < u_guard      (rhat <= 0: protected iff d <= now)
+ *     when a cycle starts:  N = round(N_min + f (N_max - N_min)),  f = the protected fraction of the waiting
+ *                           short-path prefills (0 if there is none); halves round up
+ *     phase = short during the first N steps of the cycle, long during the following M
+ *     visible = decode continuations, protected requests, prefills whose path is the phase's
+ *     long-path cap: of the visible unprotected long-path prefills only the (long_cap - long_admitted) with
+ *                    the earliest deadlines stay visible (ties: the lower id)
+ * The caller runs its base scheduler on the visible requests and "restores" the hidden ones simply by
+ * passing them again at the next step.  The paper leaves open when N takes effect (here: at the start of a
+ * cycle), the rounding (nearest, halves up) and the tie rule of the cap.
+ */
+typedef struct hs_temporal hs_temporal_t; /* opaque, owned by the library */
+
+typedef struct {
+  uint32_t abi_version; /* HS_ABI_VERSION */
+  int32_t n_min, n_max; /* short-path steps per cycle, 1 <= n_min <= n_max <= 64 (the paper: 2 and 8) */
+  int32_t m;            /* long-path steps per cycle, >= 1 (the paper: 2) */
+  double u_guard;       /* guard band of the slack ratio, > 0 */
+  int32_t long_cap;     /* most ordinary long-path prefills that may hold shared-stage slots, >= 0 */
+} hs_temporal_config_t;
+
+typedef struct {
+  int64_t id;
+  int32_t path;     /* 0 short, 1 long */
+  int32_t stage;    /* 0 prefill (waiting or running), 1 decode continuation */
+  double deadline;  /* absolute time of the first-response deadline */
+  double remaining; /* estimate of the time the request still needs to its first response */
+} hs_request_view_t;
+
+hs_status_t hs_temporal_create(const hs_temporal_config_t *cfg, hs_temporal_t **out);
+
+/*
+ * One scheduling step.  reqs: host array of n requests (n >= 0; may be NULL when n == 0); long_admitted: how
+ * many ordinary long-path prefills already hold shared-stage slots; visible: host array of n bytes, receives
+ * 1 for visible and 0 for hidden; phase (nullable) receives 0 / 1 for a short- / long-path phase, n_short
+ * (nullable) the N in force.  Errors: INVALID_ARG (NULL, n < 0, a path or stage outside {0, 1}, non-finite
+ * numbers); the rotation does not advance then.
+ */
+hs_status_t hs_temporal_step(hs_temporal_t *ctl, double now, const hs_request_view_t *reqs, int32_t n,
+                             int32_t long_admitted, uint8_t *visible, int32_t *phase, int32_t *n_short);
+
+hs_status_t hs_temporal_destroy(hs_temporal_t *ctl);
 
 #if defined(__GNUC__)
 #pragma GCC visibility pop

@@ -26,7 +26,7 @@ EXPORTS = ("hs_status_str", "hs_kv_pool_bytes", "hs_workspace_bytes", "hs_stage_
            "hs_stage_profile_read", "hs_last_error", "hs_op_decode_attention_noalloc", "hs_op_gemm_f16",
            "hs_spatial_create", "hs_spatial_update", "hs_spatial_state", "hs_spatial_destroy",
            "hs_spatial_derive_cap", "hs_head_workspace_bytes", "hs_head_create", "hs_head_step", "hs_head_status",
-           "hs_head_destroy", "hs_op_embed")
+           "hs_head_destroy", "hs_op_embed", "hs_temporal_create", "hs_temporal_step", "hs_temporal_destroy")
 PROFILE_CLASSES = ("rmsnorm", "gemm_qkv", "attn_prefill", "attn_decode", "attn_combine", "gemm_out", "gemm_gateup",
                    "gemm_down")
 
@@ -56,6 +56,16 @@ class hs_batch_t(C.Structure):
 class hs_head_config_t(C.Structure):
     _fields_ = [("abi_version", C.c_uint32), ("device", C.c_int32), ("d_model", C.c_int32), ("vocab", C.c_int32),
                 ("rms_eps", C.c_float), ("max_rows", C.c_int32)]
+
+
+class hs_temporal_config_t(C.Structure):
+    _fields_ = [("abi_version", C.c_uint32), ("n_min", C.c_int32), ("n_max", C.c_int32), ("m", C.c_int32),
+                ("u_guard", C.c_double), ("long_cap", C.c_int32)]
+
+
+class hs_request_view_t(C.Structure):
+    _fields_ = [("id", C.c_int64), ("path", C.c_int32), ("stage", C.c_int32), ("deadline", C.c_double),
+                ("remaining", C.c_double)]
 
 
 class hs_spatial_config_t(C.Structure):
@@ -115,6 +125,10 @@ def lib() -> C.CDLL:
         l.hs_head_destroy.argtypes = [C.c_void_p]
         l.hs_op_embed.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_int32,
                                   C.c_void_p, C.c_void_p]
+        l.hs_temporal_create.argtypes = [C.POINTER(hs_temporal_config_t), C.POINTER(C.c_void_p)]
+        l.hs_temporal_step.argtypes = [C.c_void_p, C.c_double, C.POINTER(hs_request_view_t), C.c_int32, C.c_int32,
+                                       C.POINTER(C.c_uint8), C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+        l.hs_temporal_destroy.argtypes = [C.c_void_p]
         l.hs_spatial_create.argtypes = [C.POINTER(hs_spatial_config_t), C.POINTER(C.c_void_p)]
         l.hs_spatial_update.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
         l.hs_spatial_state.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int32)]
@@ -366,3 +380,40 @@ def hs_op_embed(tokens_ptr: int, n: int, table_ptr: int, vocab: int, d_model: in
                            sm_budget, C.c_void_p(status_ptr), C.c_void_p(cuda_stream))
     if st != HS_OK:
         raise HsError(st, "hs_op_embed")
+
+
+class TemporalView:
+    """The library's temporal scheduler view (hs_temporal_*): path rotation, slack guard, adaptive ratio and
+    long-path cap of the paper (Sec. 4.2).  Marshalling only."""
+
+    def __init__(self, n_min: int = 2, n_max: int = 8, m: int = 2, u_guard: float = 1.5, long_cap: int = 4):
+        cfg = hs_temporal_config_t(HS_ABI_VERSION, n_min, n_max, m, u_guard, long_cap)
+        h = C.c_void_p()
+        st = lib().hs_temporal_create(C.byref(cfg), C.byref(h))
+        if st != HS_OK:
+            raise HsError(st, "hs_temporal_create")
+        self.handle = h
+
+    def step(self, now: float, reqs, long_admitted: int):
+        """reqs: sequence of (id, path, stage, deadline, remaining).  Returns (visible flags, phase, N)."""
+        n = len(reqs)
+        arr = (hs_request_view_t * max(n, 1))()
+        for i, (rid, path, stage, deadline, remaining) in enumerate(reqs):
+            arr[i] = hs_request_view_t(rid, path, stage, deadline, remaining)
+        vis = (C.c_uint8 * max(n, 1))()
+        phase, ns = C.c_int32(), C.c_int32()
+        st = lib().hs_temporal_step(self.handle, float(now), arr, n, long_admitted, vis, C.byref(phase), C.byref(ns))
+        if st != HS_OK:
+            raise HsError(st, "hs_temporal_step")
+        return [bool(vis[i]) for i in range(n)], phase.value, ns.value
+
+    def close(self) -> None:
+        if self.handle:
+            lib().hs_temporal_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

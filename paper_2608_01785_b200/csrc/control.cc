@@ -1,6 +1,7 @@
 // Spatial controller: per-step choice of the shared stage's SM budget from downstream activity and a
 // smoothed memory-pressure signal (Sec. 4.3, Eq. 1; Algorithm 1 step 3 of the paper), and the offline choice
 // of the co-running cap from a fixed-SM sweep (Sec. 4.1).  Host-only.
+#include <algorithm>
 #include <cmath>
 #include <new>
 #include <vector>
@@ -113,6 +114,89 @@ hs_status_t hs_spatial_derive_cap(const int32_t* budgets, const double* latency,
     if (budgets[i] < s_total && latency[i] <= best * (1.0 + tolerance) && (cap == 0 || budgets[i] < cap))
       cap = budgets[i];
   *s_cap = cap;
+  return HS_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------ temporal view --
+struct hs_temporal {
+  int32_t n_min, n_max, m, long_cap;
+  double u_guard;
+  int32_t n;     // short-path steps of the current cycle
+  int32_t pos;   // position inside the current cycle
+};
+
+extern "C" {
+
+hs_status_t hs_temporal_create(const hs_temporal_config_t* cfg, hs_temporal_t** out) {
+  if (!cfg || !out) return HS_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cfg->abi_version != HS_ABI_VERSION || cfg->n_min < 1 || cfg->n_max < cfg->n_min || cfg->n_max > 64 ||
+      cfg->m < 1 || cfg->long_cap < 0 || !std::isfinite(cfg->u_guard) || !(cfg->u_guard > 0.0))
+    return HS_ERR_INVALID_ARG;
+  hs_temporal* c = new (std::nothrow) hs_temporal();
+  if (!c) return HS_ERR_INVALID_ARG;
+  c->n_min = cfg->n_min;
+  c->n_max = cfg->n_max;
+  c->m = cfg->m;
+  c->long_cap = cfg->long_cap;
+  c->u_guard = cfg->u_guard;
+  c->n = cfg->n_min;
+  c->pos = 0;
+  *out = c;
+  return HS_OK;
+}
+
+hs_status_t hs_temporal_step(hs_temporal_t* c, double now, const hs_request_view_t* reqs, int32_t n,
+                             int32_t long_admitted, uint8_t* visible, int32_t* phase_out, int32_t* n_short) {
+  if (!c || n < 0 || (n > 0 && (!reqs || !visible)) || !std::isfinite(now)) return HS_ERR_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    const hs_request_view_t& r = reqs[i];
+    if ((r.path != 0 && r.path != 1) || (r.stage != 0 && r.stage != 1) || !std::isfinite(r.deadline) ||
+        !std::isfinite(r.remaining))
+      return HS_ERR_INVALID_ARG;
+  }
+  std::vector<uint8_t> prot(size_t(n) > 0 ? size_t(n) : 1);
+  int short_wait = 0, short_prot = 0;
+  for (int i = 0; i < n; ++i) {
+    const hs_request_view_t& r = reqs[i];
+    const double slack = r.deadline - now;
+    prot[i] = r.remaining <= 0.0 ? slack <= 0.0 : slack / r.remaining < c->u_guard;
+    if (r.path == 0 && r.stage == 0) {
+      ++short_wait;
+      short_prot += prot[i];
+    }
+  }
+  if (c->pos == 0) {   // a cycle starts: the short-path share follows the protected fraction
+    const double f = short_wait > 0 ? double(short_prot) / double(short_wait) : 0.0;
+    c->n = int32_t(std::floor(double(c->n_min) + f * double(c->n_max - c->n_min) + 0.5));
+  }
+  const int32_t phase = c->pos < c->n ? 0 : 1;
+  c->pos = (c->pos + 1) % (c->n + c->m);
+  std::vector<int> cand;
+  for (int i = 0; i < n; ++i) {
+    const hs_request_view_t& r = reqs[i];
+    visible[i] = r.stage == 1 || prot[i] || r.path == phase;
+    if (visible[i] && r.stage == 0 && r.path == 1 && !prot[i]) cand.push_back(i);
+  }
+  // long-path admission cap: the earliest deadlines keep their place, ties go to the lower id
+  const int room = c->long_cap - long_admitted > 0 ? c->long_cap - long_admitted : 0;
+  if (int(cand.size()) > room) {
+    std::sort(cand.begin(), cand.end(), [&](int a, int b) {
+      if (reqs[a].deadline != reqs[b].deadline) return reqs[a].deadline < reqs[b].deadline;
+      return reqs[a].id < reqs[b].id;
+    });
+    for (size_t k = size_t(room); k < cand.size(); ++k) visible[cand[k]] = 0;
+  }
+  if (phase_out) *phase_out = phase;
+  if (n_short) *n_short = c->n;
+  return HS_OK;
+}
+
+hs_status_t hs_temporal_destroy(hs_temporal_t* c) {
+  if (!c) return HS_ERR_INVALID_ARG;
+  delete c;
   return HS_OK;
 }
 

@@ -76,3 +76,45 @@ def test_long_path_cap_keeps_the_earliest_deadlines():
     o2 = TemporalOracle(n_min=2, m=2, long_cap=3)
     o2.step(0.0, [], 0); o2.step(0.0, [], 0)
     assert o2.step(0.0, reqs, 5)[0] == [False, False, False, False, True, True, False]   # no room at all
+
+
+# ------------------------------------------------------------- library vs oracle --
+def test_library_view_matches_the_oracle_step_by_step():
+    from paper_2608_01785_b200 import binding as B
+    rng = np.random.default_rng(11)
+    for trial in range(30):
+        n_min = int(rng.integers(1, 4))
+        n_max = int(rng.integers(n_min, 10))
+        m = int(rng.integers(1, 4))
+        guard = float(rng.uniform(0.8, 3.0))
+        cap = int(rng.integers(0, 6))
+        orc = TemporalOracle(n_min, n_max, m, guard, cap)
+        lib = B.TemporalView(n_min, n_max, m, guard, cap)
+        now = 0.0
+        for step in range(200):
+            now += float(rng.uniform(0.0, 0.05))
+            n = int(rng.integers(0, 14))
+            reqs = [Req(int(rng.integers(0, 1000)), int(rng.integers(0, 2)), int(rng.integers(0, 2)),
+                        now + float(rng.choice([rng.uniform(-0.2, 3.0), 0.5, 1.0])),
+                        float(rng.choice([rng.uniform(0.0, 2.0), 0.0, 0.5]))) for _ in range(n)]
+            admitted = int(rng.integers(0, 7))
+            want = orc.step(now, reqs, admitted)
+            got = lib.step(now, [(r.rid, r.path, r.stage, r.deadline, r.remaining) for r in reqs], admitted)
+            assert got == (want[0], want[1], want[2]), (trial, step)
+        lib.close()
+
+
+def test_library_view_argument_errors():
+    from paper_2608_01785_b200 import binding as B
+    for kw in (dict(n_min=0), dict(n_min=5, n_max=4), dict(n_max=65), dict(m=0), dict(u_guard=0.0), dict(long_cap=-1)):
+        with pytest.raises(B.HsError):
+            B.TemporalView(**kw)
+    v = B.TemporalView()
+    assert v.step(0.0, [], 0) == ([], SHORT, 2)
+    with pytest.raises(B.HsError):
+        v.step(0.0, [(1, 2, 0, 1.0, 1.0)], 0)                   # path outside {0, 1}
+    with pytest.raises(B.HsError):
+        v.step(0.0, [(1, 0, 0, float("nan"), 1.0)], 0)
+    assert v.step(0.0, [], 0)[1] == SHORT                        # the refused steps did not advance the rotation
+    assert v.step(0.0, [], 0)[1] == LONG
+    v.close()
