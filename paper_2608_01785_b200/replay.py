@@ -39,11 +39,19 @@ class ReplayConfig:
     talker_ctx0: int = 128          # conditioning tokens a talker sequence starts from
     ladder: Tuple[int, ...] = (120, 96, 74, 48)
     policy_seed: int = 5
-    policy: str = "seeded"          # "seeded" | "controller"
+    policy: str = "seeded"          # "seeded" | "controller" | "horizon" (temporal view + spatial controller)
     hbm_gbs: float = 6547.2         # measured copy bandwidth: normalises the controller's pressure samples
     b_sat: float = 0.5              # pressure (fraction of hbm_gbs) at which the cap reaches the top of the ladder
     gamma: float = 0.4              # weight of the newest pressure sample (the value of the paper's Fig. 10)
     delta_step: int = 20            # smallest change of the cap that is applied while co-running (SMs)
+    # first-response deadlines per class (ms after arrival): text = first backbone token, speech / image = first
+    # downstream step.  Stand-ins for the paper's "solo p95 x multiplier" table (Sec. 4.1)
+    slo_ms: Tuple[Tuple[str, float], ...] = (("text", 120.0), ("speech", 1500.0), ("image", 1500.0))
+    u_guard: float = 1.5            # slack-ratio guard band
+    long_cap: int = 24              # most ordinary long-path requests holding backbone slots
+    est_fixed_ms: float = 8.0       # coarse remaining-time estimate: fixed part (one tick) ...
+    est_per_token_ms: float = 0.014 # ... + per prompt token still to prefill ...
+    est_down_ms: float = 8.0        # ... + one more tick for the first downstream step of a long-path request
 
 
 @dataclass
@@ -209,14 +217,46 @@ def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = Repl
             waiting.append(_Seq(trace[nxt]))
             nxt += 1
 
+    slo = dict(cfg.slo_ms)
+    view = B.TemporalView(2, 8, 2, cfg.u_guard, cfg.long_cap) if cfg.policy == "horizon" else None
+    if view is not None and ctl is None:
+        ctl = B.SpatialController(engine.sm_count, engine.sm_count, sorted(cfg.ladder), cfg.b_sat, cfg.gamma,
+                                  cfg.delta_step)
+
+    def is_long(s):
+        return s.req.talker_out > 0
+
+    def deadline(s):
+        return s.req.arrival_s + slo[s.req.out_class] * 1e-3
+
+    def remaining(s):
+        est = cfg.est_fixed_ms + cfg.est_per_token_ms * (s.req.prompt_len - s.prefilled)
+        return (est + (cfg.est_down_ms if is_long(s) else 0.0)) * 1e-3
+
+    def pick_next():
+        """The base scheduler (first come, first served) on the temporal view of this step."""
+        if view is None:
+            return waiting.popleft()
+        reqs = [(s.req.rid, int(is_long(s)), 0, deadline(s), remaining(s)) for s in waiting] + \
+               [(s.req.rid, int(is_long(s)), 1, deadline(s), 0.0) for s in decoding]
+        admitted = sum(1 for s in decoding if is_long(s))
+        visible, _, _ = view.step(t, reqs, admitted)
+        for i, s in enumerate(waiting):
+            if visible[i]:
+                del waiting[i]
+                return s
+        return None
+
     while len(done) < len(trace):
         admit(t)
         if prefilling is None and waiting and len(decoding) < cfg.max_decode:
-            prefilling = waiting.popleft()
+            prefilling = pick_next()
         while talker_wait and len(talking) < cfg.max_talker:
             s = talker_wait.popleft()
             talking.append(s)
         if prefilling is None and not decoding and not talking:
+            if waiting:
+                continue                              # everything waiting was hidden in this phase: next step
             if nxt >= len(trace):
                 break
             t = max(t, trace[nxt].arrival_s)          # idle: jump to the next arrival
@@ -302,10 +342,15 @@ def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = Repl
         sel = [s for s in done if s.req.out_class == cls]
         ttft = [(s.t_first - s.req.arrival_s) * 1e3 for s in sel if s.t_first is not None]
         ttfo = [(s.t_first_down - s.req.arrival_s) * 1e3 for s in sel if s.t_first_down is not None]
+        first = [(s.t_first if cls == "text" else s.t_first_down) for s in sel]
+        met = [f is not None and (f - s.req.arrival_s) * 1e3 <= slo[cls] for f, s in zip(first, sel)]
         by_class[cls] = {"requests": len(sel), "ttft_ms_p50": pct(ttft, 50), "ttft_ms_p95": pct(ttft, 95),
+                         "slo_ms": slo[cls], "slo_attainment": (sum(met) / len(met)) if met else None,
                          "first_downstream_ms_p50": pct(ttfo, 50), "first_downstream_ms_p95": pct(ttfo, 95)}
     if ctl is not None:
         ctl.close()
+    if view is not None:
+        view.close()
     return {"requests_done": len(done), "virtual_seconds": t, "busy_seconds": busy_s, "policy": cfg.policy,
             "pressure": {"mean": statistics.fmean(pressures) if pressures else None, "p95": pct(pressures, 95)},
             "cap_changes": cap_changes,
@@ -330,7 +375,7 @@ def main():
     ap.add_argument("--requests", type=int, default=2000)
     ap.add_argument("--backbone", default="c3_7b")
     ap.add_argument("--talker", default="c4_talker")
-    ap.add_argument("--policy", default="seeded", choices=["seeded", "controller"])
+    ap.add_argument("--policy", default="seeded", choices=["seeded", "controller", "horizon"])
     ap.add_argument("--b-sat", type=float, default=ReplayConfig.b_sat)
     args = ap.parse_args()
     cfg = ReplayConfig(policy=args.policy, b_sat=args.b_sat)

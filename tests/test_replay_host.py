@@ -71,3 +71,28 @@ def test_replay_under_the_spatial_controller():
     co = lambda d: {b: n for b, n in d.items() if b != 148}
     assert max(co(seen[0.05])) == 120            # saturated pressure: the top of the ladder, never beyond it
     assert set(co(seen[1e6])) == {48}            # negligible pressure: the bottom of the ladder
+
+
+def test_replay_with_the_temporal_view_protects_short_path_requests():
+    """"horizon" = temporal view (path rotation, slack guard, long-path cap) + spatial controller.  On the latency
+    model near saturation the short-path class reaches its first token sooner and meets its deadline more often
+    than under first-come-first-served admission; nothing is lost or leaked."""
+    trace = wl.make_trace(1.0, 200, seed=4)
+    out = {}
+    for policy in ("controller", "horizon"):
+        cfg = ReplayConfig(max_decode=8, max_prefill_chunk=256, max_talker=4, policy=policy, hbm_gbs=0.01, long_cap=3,
+                           slo_ms=(("text", 400.0), ("speech", 20000.0), ("image", 20000.0)))
+        pa, pb, ma, mb = pool_sizes(cfg)
+        eng = ModelEngine(wl.DIMS["c1_tiny"], wl.DIMS["c1_tiny"], pa, pb, ma, mb)
+        try:
+            res = replay(trace, eng, cfg)
+            assert res["requests_done"] == 200
+            assert res["backbone_tokens"] == sum(r.prompt_len + r.backbone_out for r in trace)
+            assert res["talker_tokens"] == sum(r.talker_out for r in trace)
+            assert eng.free_pages("a") == pa and eng.free_pages("b") == pb
+            out[policy] = res["by_class"]
+        finally:
+            eng.close()
+    assert out["horizon"]["text"]["ttft_ms_p95"] < out["controller"]["text"]["ttft_ms_p95"]
+    assert out["horizon"]["text"]["slo_attainment"] >= out["controller"]["text"]["slo_attainment"]
+    assert out["horizon"]["text"]["slo_attainment"] > 0.95
