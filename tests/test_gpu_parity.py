@@ -214,7 +214,9 @@ def test_edge_cases_match_oracle(orc, name):
     y_ref = orc.step(case.cfg, case.weights, pool_ref, batch.q_len, batch.ctx_len, case.block_tables, case.x)
     assert np.all(np.isfinite(y_ref))
     outs = []
-    for budget in (148, 5):
+    # more than 128 tokens put the GEMMs on pairs of SMs; a budget of one SM then has to fall back to single blocks
+    budgets = (148, 5, 1) if name == "continuation_chunks" else (148, 5)
+    for budget in budgets:
         st = make_stage(case)
         y, pool = run_step(st, case, budget)
         st.close()
@@ -231,7 +233,8 @@ def test_edge_cases_match_oracle(orc, name):
                           dims.head_dim).transpose(0, 1, 3, 2, 4, 5)
         assert np.all(g6[:, :, :, ~(owned | written)] == 0x7fc0)
         assert np.array_equal(g6[:, :, :, owned & ~written], pool6[:, :, :, owned & ~written])
-    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    for other in outs[1:]:
+        assert np.array_equal(outs[0][0], other[0]) and np.array_equal(outs[0][1], other[1])
     # the all-bf16 variant of the stage (no fp16 weight copies) on the same case
     st = make_stage(case, flags=B.HS_FLAG_BF16_ACTIVATIONS)
     y, _ = run_step(st, case, 148)

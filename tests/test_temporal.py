@@ -118,3 +118,25 @@ def test_library_view_argument_errors():
     assert v.step(0.0, [], 0)[1] == SHORT                        # the refused steps did not advance the rotation
     assert v.step(0.0, [], 0)[1] == LONG
     v.close()
+
+
+def _paper_constants():
+    import os
+    out = {}
+    for line in open(os.path.join(os.path.dirname(__file__), "golden", "paper_scheduler_constants.txt")):
+        line = line.split("#")[0].split()
+        if len(line) == 2:
+            out[line[0]] = float(line[1])
+    return out
+
+
+def test_defaults_and_long_path_share_match_the_values_the_paper_prints():
+    """tests/golden/paper_scheduler_constants.txt holds what the paper states (Sec. 4.2, Sec. 6.4)."""
+    c = _paper_constants()
+    o = TemporalOracle()
+    assert (o.n_min, o.n_max, o.m) == (c["rotation_n_min"], c["rotation_n_max"], c["rotation_m"])
+    reqs = [R(0, SHORT, deadline=0.5, remaining=1.0), R(1, LONG)]       # every waiting short-path request protected
+    phases = [o.step(0.0, reqs, 0)[1] for _ in range(1000)]
+    assert abs(phases.count(LONG) / 1000 - c["long_share_at_max_pressure"]) < 1e-12
+    from paper_2608_01785_b200.replay import ReplayConfig
+    assert ReplayConfig().gamma == c["ewma_gamma"]
