@@ -94,15 +94,16 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_stage(name: str, device: int, init: str = "n002", layers: int = 0, flags: int = 0):
-    """Weights, KV pool with random-filled context, block tables and input of the named workload."""
+def build_stage(name: str, device: int, init: str = "n002", layers: int = 0, flags: int = 0, batch=None):
+    """Weights, KV pool with random-filled context, block tables and input of the named workload (or of the
+    workload's dimensions with another batch)."""
     from paper_2608_01785_b200.stage import Stage
     dims = wl.DIMS[name]
     if layers:
         dims = wl.StageDims(layers, dims.d_model, dims.n_q_heads, dims.n_kv_heads, dims.head_dim, dims.d_ffn,
                             dims.rms_eps, dims.rope_base)
     seed = SEED[name]
-    batch = wl.make_batch(name, seed)
+    batch = batch or wl.make_batch(name, seed)
     dev = torch.device("cuda", device)
     weights = wl.make_weights(dims, seed, dev, init)
     num_pages = wl.pages_needed(batch) + 8

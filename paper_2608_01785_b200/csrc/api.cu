@@ -141,6 +141,7 @@ hs_status_t ensure_attributes(int device) {
   if ((e = norm_set_attributes()) != cudaSuccess) return cuda_fail("rmsnorm attributes", e);
   if ((e = attention_set_attributes()) != cudaSuccess) return cuda_fail("attention attributes", e);
   if ((e = head_set_attributes()) != cudaSuccess) return cuda_fail("head attributes", e);
+  if ((e = gemm_skinny_set_attributes()) != cudaSuccess) return cuda_fail("small-step gemm attributes", e);
   if (device >= 0 && device < 64) g_attrs_set[device] = true;
   return HS_OK;
 }
@@ -161,6 +162,7 @@ struct hs_stage {
   uint8_t* ws_dev = nullptr;
   __nv_bfloat16* kv_pool = nullptr;
   std::vector<hs_layer_weights_t> layers;
+  std::vector<hs_layer_weights_t> operands;   // what the projections read: the fp16 copies, or `layers` itself
   std::vector<LayerMaps> maps;
   CUtensorMap tm_h, tm_o, tm_act, tm_kv;   // operand loads
   CUtensorMap tm_h_s[2], tm_o_s[2], tm_act_s[2];   // the same A operands with 64- and 32-row boxes (small steps)
@@ -308,6 +310,7 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
   const uint64_t pool_rows = uint64_t(cfg->n_layers) * 2 * cfg->num_pages * cfg->n_kv_heads * kPage;
   ok = ok && encode_2d(&s->tm_kv, s->kv_pool, pool_rows, cfg->head_dim, 16);
   s->maps.resize(cfg->n_layers);
+  s->operands = s->layers;
   for (int l = 0; l < cfg->n_layers && ok; ++l) {
     LayerMaps& m = s->maps[l];
     hs_layer_weights_t w = s->layers[l];
@@ -322,6 +325,7 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
         at += align_up(weight_elems(*cfg, i) * 2, 1024);
       }
       if (!ok) break;
+      s->operands[l] = w;
     }
     ok = encode_2d(&m.wq, w.w_q, q_dim, d, 128) && encode_2d(&m.wk, w.w_k, kv_dim, d, 128) &&
          encode_2d(&m.wv, w.w_v, kv_dim, d, 128) && encode_2d(&m.wo, w.w_o, d, q_dim, 128) &&
@@ -450,6 +454,15 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
   // A operands of a small step are fetched with boxes of 64 or 32 rows instead of 128
   const int a_rows = use_pair ? 128 : (T <= 32 ? 32 : T <= 64 ? 64 : 128);
   const int a_sel = a_rows == 64 ? 0 : 1;
+  // Steps of at most 64 rows: a projection runs on the weight-streaming kernel (no K split) where that is the
+  // faster one for its shape
+  auto skinny = [&](int K, int N, int mode) { return gemm_skinny_wins(T, K, N, mode, Dh, s->sm_count); };
+  auto skinny_base = [&](const void* a, int K, int N, int mode) {
+    SkinnyParams k{};
+    k.a = a; k.T = T; k.K = K; k.N = N; k.mode = mode;
+    k.ab_f16 = f16; k.overlap = overlap;
+    return k;
+  };
   int* census = s->census ? reinterpret_cast<int*>(s->ws_dev + s->ws.smid) : nullptr;
   if (census && cudaMemsetAsync(census, 0, size_t(HS_PROFILE_CLASSES) * kSmidSlots * 4, stream) != cudaSuccess)
     return HS_ERR_CUDA;
@@ -458,6 +471,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
   for (int l = 0; l < c.n_layers && e == cudaSuccess; ++l) {
     const hs_layer_weights_t& w = s->layers[l];
     const LayerMaps& m = s->maps[l];
+    const hs_layer_weights_t& wo = s->operands[l];
 
     NormParams np{};
     np.x_bf16 = l == 0 ? static_cast<const __nv_bfloat16*>(b->x_in) : nullptr;
@@ -494,7 +508,15 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     g.rope = reinterpret_cast<const float2*>(s->ws_dev + s->ws.rope);
     g.status = status;
     g.smid_log = slots(1);
-    { LaunchTimer t(s, 1, stream); where = "qkv gemm"; e = launch_gemm(g, sm_budget, stream); }
+    if (skinny(d, q_dim + 2 * kv_dim, kGemmQkv)) {
+      SkinnyParams k = skinny_base(h, d, q_dim + 2 * kv_dim, kGemmQkv);
+      k.w[0] = wo.w_q; k.w[1] = wo.w_k; k.w[2] = wo.w_v;
+      k.q_dim = q_dim; k.kv_dim = kv_dim; k.head_dim = Dh; k.n_kv_heads = c.n_kv_heads;
+      k.q_out = q; k.k_cache = g.k_cache; k.v_cache = g.v_cache;
+      k.tok_pos = g.tok_pos; k.tok_slot = g.tok_slot; k.rope = g.rope;
+      k.smid_log = slots(1);
+      LaunchTimer t(s, 1, stream); where = "qkv gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
+    } else { LaunchTimer t(s, 1, stream); where = "qkv gemm"; e = launch_gemm(g, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
     AttnParams a{};
@@ -541,7 +563,12 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     go.tile_turn = reinterpret_cast<int*>(s->ws_dev + s->ws.turn);
     go.status = status;
     go.smid_log = slots(5);
-    { LaunchTimer t(s, 5, stream); where = "out-proj gemm"; e = launch_gemm(go, sm_budget, stream); }
+    if (skinny(q_dim, d, kGemmResid)) {
+      SkinnyParams k = skinny_base(o, q_dim, d, kGemmResid);
+      k.w[0] = wo.w_o; k.y = x; k.accumulate = 1;
+      k.smid_log = slots(5);
+      LaunchTimer t(s, 5, stream); where = "out-proj gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
+    } else { LaunchTimer t(s, 5, stream); where = "out-proj gemm"; e = launch_gemm(go, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
     np.x_bf16 = nullptr;
@@ -562,7 +589,13 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gu.tm_act = s->tm_act_st;
     gu.status = status;
     gu.smid_log = slots(6);
-    { LaunchTimer t(s, 6, stream); where = "gate/up gemm"; e = launch_gemm(gu, sm_budget, stream); }
+    if (skinny(d, F, kGemmGateUp)) {
+      SkinnyParams k = skinny_base(h, d, F, kGemmGateUp);
+      k.w[0] = wo.w_gate; k.w[1] = wo.w_up;
+      k.act = reinterpret_cast<__nv_bfloat16*>(s->ws_dev + s->ws.act); k.act_f16 = f16;
+      k.smid_log = slots(6);
+      LaunchTimer t(s, 6, stream); where = "gate/up gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
+    } else { LaunchTimer t(s, 6, stream); where = "gate/up gemm"; e = launch_gemm(gu, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
     GemmParams gd{};
@@ -580,7 +613,12 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gd.tile_turn = reinterpret_cast<int*>(s->ws_dev + s->ws.turn);
     gd.status = status;
     gd.smid_log = slots(7);
-    { LaunchTimer t(s, 7, stream); where = "down gemm"; e = launch_gemm(gd, sm_budget, stream); }
+    if (skinny(F, d, kGemmResid)) {
+      SkinnyParams k = skinny_base(s->ws_dev + s->ws.act, F, d, kGemmResid);
+      k.w[0] = wo.w_down; k.y = x; k.accumulate = 1;
+      k.smid_log = slots(7);
+      LaunchTimer t(s, 7, stream); where = "down gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
+    } else { LaunchTimer t(s, 7, stream); where = "down gemm"; e = launch_gemm(gd, sm_budget, stream); }
     if (e != cudaSuccess) break;
   }
   return e == cudaSuccess ? HS_OK : cuda_fail(where, e);
@@ -658,6 +696,17 @@ static hs_status_t op_gemm(const void* a, const void* w, const float* resid, flo
   if (sm_budget < 1 || sm_budget > sm_count) return HS_ERR_INVALID_BUDGET;
   if (ensure_attributes(dev) != HS_OK) return HS_ERR_CUDA;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  // the kernels add into `out`: a residual that lives elsewhere is copied there first
+  if (resid && resid != out &&
+      cudaMemcpyAsync(out, resid, size_t(M) * N * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+    return HS_ERR_CUDA;
+  if (gemm_skinny_wins(M, K, N, kGemmResid, 0, sm_count)) {
+    SkinnyParams k{};
+    k.a = a; k.w[0] = w; k.T = M; k.K = K; k.N = N; k.mode = kGemmResid;
+    k.ab_f16 = ab_f16; k.y = out; k.accumulate = resid != nullptr;
+    const cudaError_t e = launch_gemm_skinny(k, sm_budget, stream);
+    return e == cudaSuccess ? HS_OK : cuda_fail("small-step gemm", e);
+  }
   GemmParams g{};
   if (!encode_2d(&g.tm_a, a, M, K, 128) || !encode_2d(&g.tm_b[0], w, N, K, 128) ||
       !encode_2d(&g.tm_out, out, M, N, 32, true))
@@ -670,10 +719,6 @@ static hs_status_t op_gemm(const void* a, const void* w, const float* resid, flo
   g.accumulate = resid != nullptr;
   g.pair = M > 128;
   g.bn = g.pair ? 256 : gemm_pick_bn(M, N, sm_count);
-  // the kernel adds into `out`: a residual that lives elsewhere is copied there first
-  if (resid && resid != out &&
-      cudaMemcpyAsync(out, resid, size_t(M) * N * 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
-    return HS_ERR_CUDA;
   g.status = status_dev;
   const cudaError_t e = launch_gemm(g, sm_budget, stream);
   return e == cudaSuccess ? HS_OK : cuda_fail("gemm", e);

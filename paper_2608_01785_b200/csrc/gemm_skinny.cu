@@ -1,0 +1,366 @@
+// The projections of a small step (at most 64 token rows).  With so few rows every GEMM of the layer is a
+// weight-streaming problem, and what counts is how many SMs pull weights and how directly.  The tcgen05 kernel
+// of gemm.cu feeds 128-row tiles through TMA boxes of 128-byte pieces and needs a K split with an ordered
+// chain of adds to occupy the GPU; this kernel does the opposite:
+//   * one block per unit of 32 output columns and the WHOLE K range: no K split across blocks, no chain;
+//   * inside the block the K range is dealt over 8 warps; every warp streams its K steps of the unit's 32 weight
+//     rows with 16-byte cp.async copies into a private ring of shared memory (every lane reads back exactly the
+//     16 bytes it copied, so the ring needs no barrier at all), the matching slice of the activations the same
+//     way, and feeds mma.sync m16n8k16 fragments from the ring -- no TMA, no TMEM, no mbarrier;
+//   * the 8 partial accumulators meet in shared memory and are summed in warp order, then the epilogue of the
+//     mode runs: residual add, RoPE + cache write + q store, or SwiGLU.
+// Units are listed independently of the SM budget and a unit's arithmetic is one fixed sequence, so the results
+// do not depend on the budget.  A unit's 32 columns are chosen per mode so that the epilogue finds its partner
+// columns in the same thread: Qkv units take columns c .. c+15 and c + Dh/2 .. c + Dh/2 + 15 of one head (the
+// rotation pairs), GateUp units 16 gate columns and the same 16 up columns.
+//
+// Fragment trick: a lane loads 8 consecutive K elements (16 bytes) of its weight row and of its two
+// activation rows; the two MMAs of a 32-wide K step use elements 0..3 and 4..7 of those.  That is a
+// permutation of the K index inside the step, applied to both operands alike, so the dot products are
+// unchanged and every load is a full 16 bytes.
+#include <cuda_fp16.h>
+
+#include "kernels.h"
+#include "ptx.cuh"
+
+namespace hs {
+namespace {
+
+constexpr int SK_WARPS = 8, SK_THREADS = SK_WARPS * 32;
+
+template <bool F16>
+__device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                          uint32_t b1) {
+  if (F16)
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+  else
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// cp.async.cg reads through the L2 only: right for weights that are used once and for activations that the
+// kernel before this one wrote (it may still be draining when this kernel starts).
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ uint4 lds16(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+
+// First element of (slot, kv head) in one layer's K or V pages: [page][kv_head][16][Dh].
+__device__ __forceinline__ __nv_bfloat16* cache_row(__nv_bfloat16* base, int slot, int hk, int n_kv_heads, int Dh) {
+  return base + ((size_t(slot >> 4) * n_kv_heads + hk) * 16 + (slot & 15)) * Dh;
+}
+
+constexpr int NT = 4;                  // n8 tiles of a unit: 32 output columns
+constexpr int PART_STRIDE = 40;        // floats between rows of a warp's partial tile (32 + padding)
+
+// Where tile j (0..3), column g (0..7) of unit `unit` lives: the weight row to read.
+__device__ __forceinline__ const uint8_t* unit_row(const SkinnyParams& p, int unit, int j, int g) {
+  const size_t row_bytes = size_t(p.K) * 2;
+  if (p.mode == kGemmResid) return static_cast<const uint8_t*>(p.w[0]) + size_t(unit * 32 + j * 8 + g) * row_bytes;
+  if (p.mode == kGemmGateUp) {
+    const int r = unit * 16 + (j & 1) * 8 + g;                       // tiles 0,1 gate; 2,3 the same rows of up
+    return static_cast<const uint8_t*>(p.w[j >> 1]) + size_t(r) * row_bytes;
+  }
+  const int upr = p.head_dim >> 5;                                   // units per head
+  const int head = unit / upr, sub = unit - head * upr;
+  int col = head * p.head_dim + sub * 16 + (j & 1) * 8 + g + (j >> 1) * (p.head_dim >> 1);
+  int which = 0;
+  if (col >= p.q_dim) { col -= p.q_dim; which = 1; }
+  if (which == 1 && col >= p.kv_dim) { col -= p.kv_dim; which = 2; }
+  return static_cast<const uint8_t*>(p.w[which]) + size_t(col) * row_bytes;
+}
+
+
+// MT: 16-row tiles of activations (T <= 16 MT); DB: depth of a warp's ring of K steps.
+template <int MT, int DB, bool F16>
+__global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const SkinnyParams p) {
+  extern __shared__ __align__(16) uint8_t sk_smem[];
+  constexpr int STAGE_BYTES = (NT + 2 * MT) * 512;          // per warp and K step: 4 weight tiles, 2 MT row groups
+  constexpr int RING_BYTES = DB * STAGE_BYTES;              // per warp
+  constexpr int PART_FLOATS = MT * 16 * PART_STRIDE;        // per warp
+  // The partial tiles of the reduction get their own shared memory when it fits; else they reuse the rings.
+  constexpr bool ALIAS = SK_WARPS * (RING_BYTES + PART_FLOATS * 4) > 227 * 1024;
+  static_assert(!ALIAS || PART_FLOATS * 4 <= RING_BYTES, "a warp's partial tile must fit its own ring");
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+  const uint32_t ring = smem_u32(sk_smem) + warp * RING_BYTES + lane * 16;
+  float* part_all = reinterpret_cast<float*>(sk_smem + (ALIAS ? 0 : SK_WARPS * RING_BYTES));
+  constexpr int PART_PITCH = ALIAS ? RING_BYTES / 4 : PART_FLOATS;   // floats between two warps' partial tiles
+  float* part = part_all + warp * PART_PITCH;
+  log_smid(p.smid_log);
+
+  const int units = p.mode == kGemmGateUp ? p.N >> 4 : p.N >> 5;
+  // 32-wide K steps, dealt to the warps in turn: warp w takes steps w, w + 8, ...  The eight warps move through
+  // the K range together, so at any moment the block reads 512 contiguous bytes of each weight row -- a run long
+  // enough for the DRAM pages it opens.  (Contiguous per-warp K slices would make 8 x 32 separate 64-byte streams.)
+  const int steps = p.K >> 5;
+  const int n = (steps - warp + SK_WARPS - 1) / SK_WARPS;
+  const size_t k_off = (size_t(warp) * 32 + t * 8) * 2;     // byte offset of this lane's first 16 bytes in a row
+  constexpr int STEP_BYTES = SK_WARPS * 64;                 // from one of the warp's steps to its next
+
+  const uint8_t* wrow[NT];
+  auto set_rows = [&](int unit) {
+#pragma unroll
+    for (int j = 0; j < NT; ++j) wrow[j] = unit_row(p, unit, j, g) + k_off;
+  };
+  // activation rows of this lane: rows 16 i + g and 16 i + g + 8 (clamped into the step)
+  const uint8_t* arow[MT][2];
+#pragma unroll
+  for (int i = 0; i < MT; ++i)
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      int r = 16 * i + 8 * h + g;
+      r = r < p.T ? r : p.T - 1;
+      arow[i][h] = static_cast<const uint8_t*>(p.a) + size_t(r) * p.K * 2 + k_off;
+    }
+  auto issue_b = [&](int s, int slot) {                     // weights of step s of this warp's slice
+#pragma unroll
+    for (int j = 0; j < NT; ++j) cp_async16(ring + slot * STAGE_BYTES + j * 512, wrow[j] + size_t(s) * STEP_BYTES);
+  };
+  auto issue_a = [&](int s, int slot) {                     // activations of the same step
+#pragma unroll
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+      for (int h = 0; h < 2; ++h)
+        cp_async16(ring + slot * STAGE_BYTES + (NT + 2 * i + h) * 512, arow[i][h] + size_t(s) * STEP_BYTES);
+  };
+  auto prologue = [&]() {
+#pragma unroll
+    for (int s = 0; s < DB - 1; ++s) {
+      if (s < n) {
+        issue_b(s, s);
+        issue_a(s, s);
+      }
+      cp_async_commit();
+    }
+  };
+
+  int unit = blockIdx.x;
+  if (unit < units) {                                       // weights never change: fetch them before the wait
+    set_rows(unit);
+#pragma unroll
+    for (int s = 0; s < DB - 1; ++s)
+      if (s < n) issue_b(s, s);
+  }
+  griddep_wait();
+  griddep_launch_dependents();
+  if (unit < units) {
+#pragma unroll
+    for (int s = 0; s < DB - 1; ++s) {
+      if (s < n) issue_a(s, s);
+      cp_async_commit();
+    }
+  }
+
+  for (; unit < units; unit += gridDim.x) {
+    float acc[MT][NT][4];
+#pragma unroll
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+      for (int j = 0; j < NT; ++j)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
+
+    int slot = 0, fill = DB - 1;                            // ring slot of step s / of step s + DB - 1
+    for (int s = 0; s < n; ++s) {
+      if (s + DB - 1 < n) {
+        issue_b(s + DB - 1, fill);
+        issue_a(s + DB - 1, fill);
+      }
+      cp_async_commit();
+      cp_async_wait<DB - 1>();
+      const uint32_t at = ring + slot * STAGE_BYTES;
+      uint4 b[NT];
+#pragma unroll
+      for (int j = 0; j < NT; ++j) b[j] = lds16(at + j * 512);
+#pragma unroll
+      for (int i = 0; i < MT; ++i) {
+        const uint4 lo = lds16(at + (NT + 2 * i) * 512), hi = lds16(at + (NT + 2 * i + 1) * 512);
+        // the two MMAs on one accumulator are kept apart: four independent ones run between them
+#pragma unroll
+        for (int j = 0; j < NT; ++j) mma_16816<F16>(acc[i][j], lo.x, hi.x, lo.y, hi.y, b[j].x, b[j].y);
+#pragma unroll
+        for (int j = 0; j < NT; ++j) mma_16816<F16>(acc[i][j], lo.z, hi.z, lo.w, hi.w, b[j].z, b[j].w);
+      }
+      slot = slot + 1 == DB ? 0 : slot + 1;
+      fill = fill + 1 == DB ? 0 : fill + 1;
+    }
+    cp_async_wait<0>();
+
+    // the next unit's first steps travel while this one is reduced and written (when the rings stay free)
+    const int next = unit + gridDim.x;
+    if (!ALIAS && next < units) {
+      set_rows(next);
+      prologue();
+    }
+
+    // partial tiles -> shared memory
+#pragma unroll
+    for (int i = 0; i < MT; ++i)
+#pragma unroll
+      for (int j = 0; j < NT; ++j) {
+        float* at = part + (16 * i + g) * PART_STRIDE + 8 * j + 2 * t;
+        *reinterpret_cast<float2*>(at) = make_float2(acc[i][j][0], acc[i][j][1]);
+        *reinterpret_cast<float2*>(at + 8 * PART_STRIDE) = make_float2(acc[i][j][2], acc[i][j][3]);
+      }
+    __syncthreads();
+
+    // sum of the 8 warps' partials in warp order, then the epilogue of the mode.  Thread -> row tid / 4 and the
+    // tile columns jq .. jq + 3 ("lo") and 16 + jq .. 16 + jq + 3 ("hi").
+    const int row = threadIdx.x >> 2, jq = (threadIdx.x & 3) * 4;
+    if (row < MT * 16 && row < p.T) {
+      const float* src = part_all + row * PART_STRIDE + jq;
+      float4 lo = *reinterpret_cast<const float4*>(src), hi = *reinterpret_cast<const float4*>(src + 16);
+#pragma unroll
+      for (int w = 1; w < SK_WARPS; ++w) {
+        const float4 l = *reinterpret_cast<const float4*>(src + w * PART_PITCH);
+        const float4 h = *reinterpret_cast<const float4*>(src + w * PART_PITCH + 16);
+        lo.x += l.x; lo.y += l.y; lo.z += l.z; lo.w += l.w;
+        hi.x += h.x; hi.y += h.y; hi.z += h.z; hi.w += h.w;
+      }
+      if (p.mode == kGemmResid) {
+        float4* y_lo = reinterpret_cast<float4*>(p.y + size_t(row) * p.N + unit * 32 + jq);
+        float4* y_hi = y_lo + 4;
+        if (p.accumulate) {
+          const float4 a = *y_lo, b = *y_hi;
+          lo.x += a.x; lo.y += a.y; lo.z += a.z; lo.w += a.w;
+          hi.x += b.x; hi.y += b.y; hi.z += b.z; hi.w += b.w;
+        }
+        *y_lo = lo;
+        *y_hi = hi;
+      } else if (p.mode == kGemmGateUp) {
+        const float gt[4] = {lo.x, lo.y, lo.z, lo.w}, up[4] = {hi.x, hi.y, hi.z, hi.w};
+        float v[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) v[e] = __fdividef(gt[e] * up[e], 1.f + __expf(-gt[e]));   // silu(gate) * up
+        uint2 out;
+        out.x = pack_act(v[0], v[1], p.act_f16 != 0);
+        out.y = pack_act(v[2], v[3], p.act_f16 != 0);
+        *reinterpret_cast<uint2*>(p.act + size_t(row) * p.N + unit * 16 + jq) = out;
+      } else {
+        const int Dh = p.head_dim, half = Dh >> 1, upr = Dh >> 5;
+        const int head = unit / upr, sub = unit - head * upr;
+        const int i0 = sub * 16 + jq;                        // first rotation pair / first element inside the head
+        const int n_q_heads = p.q_dim / Dh;
+        float a[4] = {lo.x, lo.y, lo.z, lo.w}, b[4] = {hi.x, hi.y, hi.z, hi.w};
+        if (head < n_q_heads + p.n_kv_heads) {               // q and k heads are rotated
+          const float4* cs = reinterpret_cast<const float4*>(p.rope + size_t(p.tok_pos[row]) * half + i0);
+          const float4 t0 = cs[0], t1 = cs[1];               // (cos, sin) of pairs i0 .. i0 + 3
+          const float c[4] = {t0.x, t0.z, t1.x, t1.z}, sn[4] = {t0.y, t0.w, t1.y, t1.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float x0 = a[e], x1 = b[e];
+            a[e] = x0 * c[e] - x1 * sn[e];
+            b[e] = x1 * c[e] + x0 * sn[e];
+          }
+        }
+        uint2 o_lo, o_hi;
+        o_lo.x = pack_act(a[0], a[1], false); o_lo.y = pack_act(a[2], a[3], false);
+        o_hi.x = pack_act(b[0], b[1], false); o_hi.y = pack_act(b[2], b[3], false);
+        __nv_bfloat16* dst;
+        if (head < n_q_heads) {
+          dst = p.q_out + size_t(row) * p.q_dim + head * Dh + i0;
+        } else {
+          const int hk = head - n_q_heads;
+          const int slot = p.tok_slot[row];
+          dst = hk < p.n_kv_heads ? cache_row(p.k_cache, slot, hk, p.n_kv_heads, Dh) + i0
+                                  : cache_row(p.v_cache, slot, hk - p.n_kv_heads, p.n_kv_heads, Dh) + i0;
+        }
+        *reinterpret_cast<uint2*>(dst) = o_lo;
+        *reinterpret_cast<uint2*>(dst + half) = o_hi;
+      }
+    }
+    __syncthreads();                                         // the partial tiles are free again
+    if (ALIAS && next < units) {
+      set_rows(next);
+      prologue();
+    }
+  }
+}
+
+template <int MT, int DB>
+constexpr int skinny_smem() {
+  constexpr int rings = SK_WARPS * DB * (NT + 2 * MT) * 512, both = rings + SK_WARPS * MT * 16 * PART_STRIDE * 4;
+  return both > 227 * 1024 ? rings : both;
+}
+constexpr int DB1 = 8, DB2 = 6, DB4 = 4;                     // ring depths by row-tile count
+static_assert(skinny_smem<1, DB1>() <= 227 * 1024 && skinny_smem<2, DB2>() <= 227 * 1024 && skinny_smem<4, DB4>() <= 227 * 1024,
+              "rings and partial tiles must fit one SM");
+
+template <int MT, int DB>
+cudaError_t launch_one(const SkinnyParams& p, int grid, cudaStream_t stream) {
+  constexpr int smem = skinny_smem<MT, DB>() < kMinSmemBytes ? kMinSmemBytes : skinny_smem<MT, DB>();
+  if (p.ab_f16) return launch_step_kernel(gemm_skinny_kernel<MT, DB, true>, grid, SK_THREADS, smem, stream, p.overlap != 0, p);
+  return launch_step_kernel(gemm_skinny_kernel<MT, DB, false>, grid, SK_THREADS, smem, stream, p.overlap != 0, p);
+}
+template <int MT, int DB>
+cudaError_t set_one() {
+  constexpr int smem = skinny_smem<MT, DB>() < kMinSmemBytes ? kMinSmemBytes : skinny_smem<MT, DB>();
+  cudaError_t e = set_kernel_smem(gemm_skinny_kernel<MT, DB, true>, smem);
+  if (e != cudaSuccess) return e;
+  return set_kernel_smem(gemm_skinny_kernel<MT, DB, false>, smem);
+}
+
+}  // namespace
+
+bool gemm_skinny_supports(int T, int K, int N, int mode, int head_dim) {
+  if (T < 1 || T > 64 || K < 32 || K % 32 != 0) return false;
+  if (mode == kGemmResid) return N % 32 == 0;
+  if (mode == kGemmGateUp) return N % 16 == 0;
+  return head_dim % 32 == 0 && N % head_dim == 0;
+}
+
+// Which kernel is faster for this shape, from measurements on B200 (config-3 and talker dimensions, 8 .. 64 rows).
+// A block of this kernel takes in about 70 KB/us and reads, per unit, 32 weight rows plus all (16 MT) activation
+// rows of width K, with about 1.5 us per unit for set-up, reduction and epilogue; units run in rounds of one per SM.
+// The tiled kernel streams a 64-wide K block in about 0.36 us (0.8 us with two weight boxes per stage, gate/up)
+// and pays 3.5 us per link of a K-split chain.  So this kernel wins where the tiled one has too few tiles to
+// occupy the device or needs a long chain (QKV, out-projection, down at few rows), and loses where there are
+// tiles enough (gate/up of a wide FFN), because here every 32 columns re-read the activations.
+// Depends on the shape and the device only, never on the SM budget.
+bool gemm_skinny_wins(int T, int K, int N, int mode, int head_dim, int sm_count) {
+  if (!gemm_skinny_supports(T, K, N, mode, head_dim)) return false;
+  const int mt = T <= 16 ? 1 : T <= 32 ? 2 : 4;
+  const int units = mode == kGemmGateUp ? N / 16 : N / 32;
+  const int rounds = (units + sm_count - 1) / sm_count;
+  const double mine = rounds * (1.5 + double(32 + 16 * mt) * K * 2 / 70e3);
+  const int k_blocks = (K + 63) / 64;
+  double tiled;
+  if (mode == kGemmResid) {
+    const int bn = gemm_pick_bn(T, N, sm_count), ks = gemm_pick_ksplit(T, N, K, bn, sm_count);
+    const int tiles = (N + bn - 1) / bn, waves = (tiles * ks + sm_count - 1) / sm_count;
+    tiled = double(waves) * ((k_blocks + ks - 1) / ks) * 0.36 + (ks - 1) * 3.5;
+  } else {
+    const int tiles = (N + 127) / 128, waves = (tiles + sm_count - 1) / sm_count;
+    tiled = double(waves) * k_blocks * (mode == kGemmGateUp ? 0.8 : 0.36);
+  }
+  return mine < tiled;
+}
+
+cudaError_t gemm_skinny_set_attributes() {
+  cudaError_t e = set_one<1, DB1>();
+  if (e == cudaSuccess) e = set_one<2, DB2>();
+  if (e == cudaSuccess) e = set_one<4, DB4>();
+  return e;
+}
+
+cudaError_t launch_gemm_skinny(const SkinnyParams& p, int sm_budget, cudaStream_t stream) {
+  if (p.T <= 0) return cudaSuccess;
+  const int units = p.mode == kGemmGateUp ? p.N / 16 : p.N / 32;
+  const int grid = units < sm_budget ? units : sm_budget;
+  if (p.T <= 16) return launch_one<1, DB1>(p, grid, stream);
+  if (p.T <= 32) return launch_one<2, DB2>(p, grid, stream);
+  return launch_one<4, DB4>(p, grid, stream);
+}
+
+}  // namespace hs

@@ -56,6 +56,32 @@ cudaError_t gemm_set_attributes();
 // Tile width for a Resid-mode GEMM of this shape on a device with sm_count SMs (budget independent).
 int gemm_pick_bn(int M, int N, int sm_count);
 int gemm_pick_ksplit(int M, int N, int K, int bn, int sm_count);
+// The same three GEMMs for steps of at most 64 rows (gemm_skinny.cu): weight streaming on plain loads and
+// warp-level MMAs, one block per 32 output columns and the whole K range, no K split across blocks.
+struct SkinnyParams {
+  const void* a;             // activations [rows >= T, K], 16-bit (fp16 or bf16 as ab_f16 says), row-major
+  const void* w[3];          // Resid {W}, Qkv {Wq, Wk, Wv}, GateUp {Wgate, Wup}; 16-bit [out, K] row-major
+  int T, K, N;               // N: Resid output width; Qkv (Hq + 2 Hkv) * Dh; GateUp F
+  int mode, ab_f16, overlap;
+  float* y;                  // Resid: fp32 [T, N]
+  int accumulate;            // Resid: 1: y += A W^T, 0: y = A W^T
+  int q_dim, kv_dim, head_dim, n_kv_heads;      // Qkv
+  __nv_bfloat16* q_out;      // bf16 [T, q_dim]
+  __nv_bfloat16* k_cache;
+  __nv_bfloat16* v_cache;
+  const int32_t* tok_pos;
+  const int32_t* tok_slot;
+  const float2* rope;
+  __nv_bfloat16* act;        // GateUp: 16-bit [T, N]
+  int act_f16;
+  int* smid_log;
+};
+// True when the skinny kernel covers this shape (few rows, K a multiple of 32, widths it can tile).
+bool gemm_skinny_supports(int T, int K, int N, int mode, int head_dim);
+// True when it is also expected to be faster than the tiled kernel for this shape (budget independent).
+bool gemm_skinny_wins(int T, int K, int N, int mode, int head_dim, int sm_count);
+cudaError_t launch_gemm_skinny(const SkinnyParams& p, int sm_budget, cudaStream_t stream);
+cudaError_t gemm_skinny_set_attributes();
 constexpr int kGemmTurnWords = 4096;   // capacity of the whose-turn array: splits are used only when tiles * 4 fits
 
 // ---------------------------------------------------------------- RMSNorm --

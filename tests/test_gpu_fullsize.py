@@ -218,3 +218,42 @@ def test_config3_budget_sweep_and_sampled_layer_local(orc, init):
             assert err <= TOL
     finally:
         stage.close()
+
+
+# ------------------------------------------------- config 3 dimensions, decode-only ticks --
+@pytest.mark.parametrize("n_dec", [64, 24, 9])
+def test_config3_decode_only_tick(orc, n_dec):
+    """A decode-only tick of the trace replay at the 7B-class dimensions: every projection is a small-step GEMM
+    (64 rows: four 16-row tiles, 24: two, 9: one; the kernel behind each projection is chosen by shape).  One
+    layer against the oracle, and the budget sweep bit for bit."""
+    r = np.random.default_rng(100 + n_dec)
+    batch = wl.BatchSpec([1] * n_dec, r.integers(512, 4097, size=n_dec).tolist())
+    stage, dims, batch, bt, x = bench.build_stage("c3_decode", 0, layers=1, batch=batch)
+    try:
+        pool0 = stage.kv_pool.clone()
+        outs = {}
+        for budget in (stage.sm_count, 100, 48, 7):
+            y = gpu_step(stage, batch, bt, x, budget, pool0)
+            outs[budget] = (y.cpu().numpy(), stage.kv_pool.clone())
+        y_gpu, pool_gpu = outs[stage.sm_count]
+        for budget, (y, pool) in outs.items():
+            assert np.array_equal(y, y_gpu), budget
+            assert torch.equal(pool, pool_gpu), budget
+        cfg = ocfg(dims, 1, stage.cfg.num_pages)
+        pool_ref = wl.bf16_bits_numpy(pool0).reshape(-1).copy()
+        y_ref = orc.step(cfg, wl.weights_to_numpy(stage.weights), pool_ref, batch.q_len, batch.ctx_len, bt,
+                         wl.to_f32_numpy(x))
+        err = rel_err(y_gpu, y_ref)
+        print(f"config 3 dimensions, {n_dec} decode rows, 1 layer: max|err|/RMS = {err:.2e}")
+        assert err <= TOL
+        # the K/V this step appended: the oracle's pool against the GPU's, as bf16 values
+        got = wl.bf16_bits_numpy(pool_gpu).reshape(-1).view(np.uint16)
+        want = np.asarray(pool_ref).reshape(-1).view(np.uint16)
+        changed = np.flatnonzero(want != wl.bf16_bits_numpy(pool0).reshape(-1).view(np.uint16))
+        assert changed.size > 0
+        a = (got[changed].astype(np.uint32) << 16).view(np.float32)
+        b = (want[changed].astype(np.uint32) << 16).view(np.float32)
+        # a bf16 step is at most 2^-7 |value|: the two sides may round a value that lies between two codes apart
+        assert np.all(np.abs(a - b) <= 2.0 ** -7 * np.abs(b) + 1e-2 * np.sqrt(np.mean(b * b)))
+    finally:
+        stage.close()

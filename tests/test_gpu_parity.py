@@ -56,7 +56,11 @@ def check_kv_written(case, pool_in, pool_gpu, kv_pre, layer=0):
 
 # ----------------------------------------------------------------- GEMM op --
 @pytest.mark.parametrize("M,N,K,resid", [(128, 256, 64, False), (82, 520, 200, True), (300, 264, 72, True),
-                                         (2112, 1024, 3584, False), (1000, 2048, 1408, True), (16, 1536, 1024, True)])
+                                         (2112, 1024, 3584, False), (1000, 2048, 1408, True), (16, 1536, 1024, True),
+                                         # at most 64 rows and few output tiles: the weight-streaming kernel,
+                                         # with one, two and four 16-row tiles and a ragged last tile
+                                         (1, 256, 1024, True), (33, 512, 2048, True), (48, 1024, 4096, False),
+                                         (64, 3584, 3584, True)])
 @pytest.mark.parametrize("a_dtype", [torch.bfloat16, torch.float16])
 def test_gemm_op_matches_oracle_and_is_budget_invariant(orc, M, N, K, resid, a_dtype):
     """Both operand forms: bf16 x bf16, and the fp16 x fp16 form the stage uses by default."""
