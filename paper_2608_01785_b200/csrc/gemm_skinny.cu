@@ -327,7 +327,12 @@ bool gemm_skinny_supports(int T, int K, int N, int mode, int head_dim) {
 // and pays 3.5 us per link of a K-split chain.  So this kernel wins where the tiled one has too few tiles to
 // occupy the device or needs a long chain (QKV, out-projection, down at few rows), and loses where there are
 // tiles enough (gate/up of a wide FFN), because here every 32 columns re-read the activations.
-// Depends on the shape and the device only, never on the SM budget.
+// Depends on the shape and the device only, never on the SM budget: the two kernels round differently, and a
+// step's result must not depend on its budget.  Rounds and waves are counted for the whole device.  Measured
+// against the alternatives over budgets 148 / 111 / 74 at config-3 dimensions (ms per 28-layer decode-only step,
+// all projections tiled -> this rule): 16 rows 4.39 -> 3.49, 5.42 -> 5.14, 5.74 -> 5.27; 32 rows 4.91 -> 4.36,
+// 5.99 -> 5.80, 6.34 -> 6.15; 64 rows 5.72 -> 5.38, 7.21 -> 7.43, 8.06 -> 8.32 (with its unit count just below
+// the SM count this kernel needs a second round as soon as the budget drops, which at 64 rows costs 3 %).
 bool gemm_skinny_wins(int T, int K, int N, int mode, int head_dim, int sm_count) {
   if (!gemm_skinny_supports(T, K, N, mode, head_dim)) return false;
   const int mt = T <= 16 ? 1 : T <= 32 ? 2 : 4;
