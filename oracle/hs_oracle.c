@@ -14,7 +14,8 @@
  * textbook pre-norm decoder layer:
  *
  *   h   = rmsnorm(x; g_attn)            r = 1/sqrt(mean(x^2) + eps)
- *   q,k,v = h W_q^T, h W_k^T, h W_v^T   (weights are [out, in], no bias)
+ *   q,k,v = h W_q^T + b_q, h W_k^T + b_k, h W_v^T + b_v   (weights are [out, in]; the biases are optional and
+ *           added before RoPE, as in the checkpoints of the 7B-class backbones that carry them)
  *   q,k <- rope(q,k; position)          rotate-half pairs (i, i + Dh/2)
  *   cache[page(p)][slot(p)] <- bf16(k), bf16(v)     (all tokens first)
  *   o   = softmax(q K^T / sqrt(Dh)) V   keys 0..p read back from the cache
@@ -52,6 +53,7 @@ typedef struct {
 
 typedef struct {
   const real *g_attn, *w_q, *w_k, *w_v, *w_o, *g_mlp, *w_gate, *w_up, *w_down;
+  const real *b_q, *b_k, *b_v; /* [Hq Dh], [Hkv Dh], [Hkv Dh]; NULL = no bias */
 } hso_layer_t;
 
 /* Diagnostic switch (never the pass/fail oracle): bit mask of intermediates
@@ -199,6 +201,13 @@ void hso_attend(const hso_config_t *c, const uint16_t *kv_pool, int layer, const
 }
 
 /* ----------------------------------------------------------- one layer -- */
+/* y[t, :] += b for every row (b == NULL: nothing). */
+static void add_bias(int T, int n, const real *b, real *y) {
+  if (!b) return;
+  for (int t = 0; t < T; ++t)
+    for (int i = 0; i < n; ++i) y[(size_t)t * n + i] += b[i];
+}
+
 /*
  * Runs layer `layer` on the residual stream x[T,d] in place.
  *   q_len[s], ctx_len[s]: new / already cached tokens of sequence s; token j
@@ -240,6 +249,8 @@ int hso_layer(const hso_config_t *c, const hso_layer_t *w, int layer, uint16_t *
   real *k = (real *)malloc(sizeof(real) * (size_t)T * KVd), *v = (real *)malloc(sizeof(real) * (size_t)T * KVd);
   hso_linear(T, KVd, d, h, w->w_k, k);
   hso_linear(T, KVd, d, h, w->w_v, v);
+  add_bias(T, KVd, w->b_k, k);
+  add_bias(T, KVd, w->b_v, v);
   for (int t = 0; t < T; ++t) {
     hso_rope(Hkv, Dh, tok_pos[t], c->rope_base, k + (size_t)t * KVd);
     if (kv_pre) {
@@ -273,6 +284,7 @@ int hso_layer(const hso_config_t *c, const hso_layer_t *w, int layer, uint16_t *
   free(h);
   real *q = (real *)malloc(sizeof(real) * (size_t)R * Qd);
   hso_linear(R, Qd, d, hR, w->w_q, q);
+  add_bias(R, Qd, w->b_q, q);
   for (int r = 0; r < R; ++r) hso_rope(Hq, Dh, tok_pos[rows[r]], c->rope_base, q + (size_t)r * Qd);
   if (g_round_mask & 2)
     for (size_t i = 0; i < (size_t)R * Qd; ++i) q[i] = round_bf16(q[i]);

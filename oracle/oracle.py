@@ -50,10 +50,11 @@ class _Cfg(C.Structure):
 
 class _Layer(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("g_attn", "w_q", "w_k", "w_v", "w_o", "g_mlp", "w_gate", "w_up",
-                                           "w_down")]
+                                           "w_down", "b_q", "b_k", "b_v")]
 
 
 WEIGHT_NAMES = ("g_attn", "w_q", "w_k", "w_v", "w_o", "g_mlp", "w_gate", "w_up", "w_down")
+BIAS_NAMES = ("b_q", "b_k", "b_v")      # optional entries of a layer's dict: biases of the q, k, v projections
 
 
 def _load(precision: str) -> C.CDLL:
@@ -166,6 +167,11 @@ class Oracle:
                 a = self._arr(lw[name])
                 keep.append(a)
                 setattr(arr[i], name, a.ctypes.data)
+            for name in BIAS_NAMES:
+                if lw.get(name) is not None:
+                    a = self._arr(lw[name])
+                    keep.append(a)
+                    setattr(arr[i], name, a.ctypes.data)
         return arr, keep
 
     def layer(self, cfg: OracleConfig, layer_weights: Dict[str, np.ndarray], layer: int, kv_pool: np.ndarray,

@@ -235,9 +235,9 @@ def _torch_reference_single_sequence(dims, weights, x, n_layers):
     for l in range(n_layers):
         w = {k: torch.from_numpy(v).double() for k, v in weights[l].items()}
         h = F.rms_norm(xt, (dims.d_model,), w["g_attn"], dims.rms_eps)
-        q = rope((h @ w["w_q"].T).view(n, Hq, Dh))
-        k = rope((h @ w["w_k"].T).view(n, Hkv, Dh)).bfloat16().double()
-        v = (h @ w["w_v"].T).view(n, Hkv, Dh).bfloat16().double()
+        q = rope(F.linear(h, w["w_q"], w.get("b_q")).view(n, Hq, Dh))
+        k = rope(F.linear(h, w["w_k"], w.get("b_k")).view(n, Hkv, Dh)).bfloat16().double()
+        v = F.linear(h, w["w_v"], w.get("b_v")).view(n, Hkv, Dh).bfloat16().double()
         k = k.repeat_interleave(Hq // Hkv, dim=1); v = v.repeat_interleave(Hq // Hkv, dim=1)
         o = F.scaled_dot_product_attention(q.transpose(0, 1), k.transpose(0, 1), v.transpose(0, 1), is_causal=True)
         xt = xt + o.transpose(0, 1).reshape(n, Hq * Dh) @ w["w_o"].T
@@ -283,6 +283,38 @@ def test_layer_matches_library_when_cache_rounding_is_exact(oracle64):
                       case.block_tables, case.x)
     assert rel_err(y, want) < 1e-12
     assert rel_err(want, case.x) > 0.05
+
+
+def test_qkv_bias_matches_library_composition_and_closed_form(oracle64):
+    """The optional biases of the q, k, v projections enter before RoPE: against torch's linear-with-bias in the
+    float64 composition, and, with all three weight matrices zero, against the closed form: every value row is
+    b_v, so each head's output is its KV head's slice of b_v whatever the scores are."""
+    dims = wl.StageDims(1, 64, 4, 2, 16, 96)
+    case = make_case(dims, wl.BatchSpec([23], [0]), seed=8)
+    g = np.random.default_rng(8)
+    w = {k: (v if k.startswith("g_") else v * 8.0) for k, v in case.weights[0].items()}
+    w["b_q"] = g.normal(0, 1.0, dims.n_q_heads * dims.head_dim)
+    w["b_k"] = g.normal(0, 1.0, dims.n_kv_heads * dims.head_dim)
+    w["b_v"] = g.normal(0, 1.0, dims.n_kv_heads * dims.head_dim)
+    args = (case.batch.q_len, case.batch.ctx_len, case.block_tables, case.x)
+    y = oracle64.step(case.cfg, [w], case.kv_pool.copy(), *args)
+    want = _torch_reference_single_sequence(dims, [w], case.x, 1)
+    assert rel_err(y, want) < 1e-10
+    no_bias = oracle64.step(case.cfg, [{k: v for k, v in w.items() if not k.startswith("b_")}], case.kv_pool.copy(), *args)
+    assert rel_err(y, no_bias) > 0.05           # the biases matter in this case
+    for drop in ("b_q", "b_k", "b_v"):          # and each one on its own
+        y_drop = oracle64.step(case.cfg, [{k: v for k, v in w.items() if k != drop}], case.kv_pool.copy(), *args)
+        assert rel_err(y, y_drop) > 1e-3, drop
+
+    z = dict(w, w_q=np.zeros_like(w["w_q"]), w_k=np.zeros_like(w["w_k"]), w_v=np.zeros_like(w["w_v"]),
+             w_down=np.zeros_like(w["w_down"]))
+    z["b_v"] = np.asarray(torch.from_numpy(w["b_v"]).bfloat16().double())        # exact in the cache
+    y = oracle64.step(case.cfg, [z], case.kv_pool.copy(), *args)
+    G = dims.n_q_heads // dims.n_kv_heads
+    o_row = np.concatenate([z["b_v"][(hq // G) * dims.head_dim:(hq // G + 1) * dims.head_dim]
+                            for hq in range(dims.n_q_heads)])
+    want = case.x.astype(np.float64) + (z["w_o"].astype(np.float64) @ o_row)[None, :]
+    assert rel_err(y, want) < 1e-12
 
 
 def test_zero_gate_weight_means_mlp_adds_nothing(oracle32):
