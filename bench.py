@@ -417,8 +417,9 @@ def main():
     achieved = gu_flops / gu_avg_s / 1e12
     peak = peaks["bf16_sustained"] * budget / stage.sm_count
     gemm_flops, attn_flops = flops_per_step(dims, batch)
-    roofline = {"bound": "tensor", "kernel": "gemm_pair_kernel (gate/up + SwiGLU epilogue)" if T > 128 and budget >= 2 else
-                          "gemm_kernel (gate/up + SwiGLU epilogue)", "achieved": achieved,
+    gateup_kernel = ("gemm_pair_kernel" if T > 128 and budget >= 2 else
+                     "gemm_kernel" if T > 64 else "gemm_kernel or gemm_skinny_kernel (chosen by shape)")
+    roofline = {"bound": "tensor", "kernel": gateup_kernel + " (gate/up + SwiGLU epilogue)", "achieved": achieved,
                 "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                 "peak_source": f"{peaks['source']} sustained bf16 (fp16 operands: nominal ratio 1.0) x sm_budget/{stage.sm_count}",
                 "frac_of_burst_peak": achieved / (peaks["bf16_burst"] * budget / stage.sm_count),

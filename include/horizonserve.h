@@ -103,7 +103,7 @@ typedef struct {
   uint32_t flags;            /* 0, or HS_FLAG_BF16_ACTIVATIONS */
 } hs_stage_config_t;
 
-/* One layer's weights: device pointers to bf16, row-major [out_features, in_features], no bias. */
+/* One layer's weights: device pointers to bf16, row-major [out_features, in_features] (biases: hs_stage_set_qkv_bias). */
 typedef struct {
   const void *g_attn; /* [d]          gain of the attention RMSNorm */
   const void *w_q;    /* [Hq*Dh, d]   */
@@ -188,6 +188,16 @@ hs_status_t hs_stage_plan(hs_stage_t *stage, const hs_batch_t *batch, int32_t *t
  * Errors (nothing launched): INVALID_ARG, INVALID_BUDGET, BAD_BLOCK_TABLE, NO_DEVICE, CUDA.
  */
 hs_status_t hs_stage_step(hs_stage_t *stage, const hs_batch_t *batch, int32_t sm_budget, void *cuda_stream);
+
+/*
+ * Optional biases of one layer's q, k, v projections: q, k, v = h W^T + b, added before RoPE (the paper runs its
+ * backbones' model code unchanged, Sec. 5; the 7B-class backbones it serves carry these three biases).
+ *   b_q  device bf16 [n_q_heads * head_dim];  b_k, b_v  device bf16 [n_kv_heads * head_dim]
+ * 16-byte aligned, borrowed until the stage is destroyed or the layer's biases are set again; any of the three
+ * may be NULL (no bias on that projection; the state of a new stage).  Takes effect for steps enqueued after
+ * the call.  Errors: INVALID_ARG (NULL stage, layer out of range, misaligned pointer), NO_DEVICE.
+ */
+hs_status_t hs_stage_set_qkv_bias(hs_stage_t *stage, int32_t layer, const void *b_q, const void *b_k, const void *b_v);
 
 /* Device-side status of the steps run so far (HS_OK or HS_ERR_TIMEOUT); call after synchronising the stream. */
 hs_status_t hs_stage_status(hs_stage_t *stage);

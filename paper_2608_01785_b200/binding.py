@@ -26,7 +26,8 @@ EXPORTS = ("hs_status_str", "hs_kv_pool_bytes", "hs_workspace_bytes", "hs_stage_
            "hs_stage_profile_read", "hs_last_error", "hs_op_decode_attention_noalloc", "hs_op_gemm_f16",
            "hs_spatial_create", "hs_spatial_update", "hs_spatial_state", "hs_spatial_destroy",
            "hs_spatial_derive_cap", "hs_head_workspace_bytes", "hs_head_create", "hs_head_step", "hs_head_status",
-           "hs_head_destroy", "hs_op_embed", "hs_temporal_create", "hs_temporal_step", "hs_temporal_destroy")
+           "hs_head_destroy", "hs_op_embed", "hs_temporal_create", "hs_temporal_step", "hs_temporal_destroy",
+           "hs_stage_set_qkv_bias")
 PROFILE_CLASSES = ("rmsnorm", "gemm_qkv", "attn_prefill", "attn_decode", "attn_combine", "gemm_out", "gemm_gateup",
                    "gemm_down")
 
@@ -138,6 +139,7 @@ def lib() -> C.CDLL:
         l.hs_op_decode_attention_noalloc.argtypes = [C.c_void_p, C.c_void_p] + [C.c_int32] * 7 + \
             [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p]
         l.hs_stage_profile_enable.argtypes = [C.c_void_p, C.c_int32]
+        l.hs_stage_set_qkv_bias.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         l.hs_stage_profile_read.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = l
     return _lib
@@ -256,6 +258,14 @@ def hs_op_gemm_bf16(a_ptr: int, w_ptr: int, resid_ptr: int, out_ptr: int, M: int
                                M, N, K, sm_budget, C.c_void_p(status_ptr), C.c_void_p(cuda_stream))
     if st != HS_OK:
         raise HsError(st, "hs_op_gemm_bf16")
+
+
+def hs_stage_set_qkv_bias(stage: int, layer: int, b_q: int, b_k: int, b_v: int) -> None:
+    """Device pointers (0 = no bias) of the layer's q, k, v biases (bf16)."""
+    st = lib().hs_stage_set_qkv_bias(C.c_void_p(stage), int(layer), C.c_void_p(b_q or None), C.c_void_p(b_k or None),
+                                     C.c_void_p(b_v or None))
+    if st != HS_OK:
+        raise HsError(st, "hs_stage_set_qkv_bias")
 
 
 def hs_stage_profile_enable(stage: int, enable: bool) -> None:

@@ -162,6 +162,8 @@ struct hs_stage {
   uint8_t* ws_dev = nullptr;
   __nv_bfloat16* kv_pool = nullptr;
   std::vector<hs_layer_weights_t> layers;
+  struct QkvBias { const __nv_bfloat16* b[3] = {nullptr, nullptr, nullptr}; };
+  std::vector<QkvBias> qkv_bias;              // per layer, optional (hs_stage_set_qkv_bias)
   std::vector<hs_layer_weights_t> operands;   // what the projections read: the fp16 copies, or `layers` itself
   std::vector<LayerMaps> maps;
   CUtensorMap tm_h, tm_o, tm_act, tm_kv;   // operand loads
@@ -311,6 +313,7 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
   ok = ok && encode_2d(&s->tm_kv, s->kv_pool, pool_rows, cfg->head_dim, 16);
   s->maps.resize(cfg->n_layers);
   s->operands = s->layers;
+  s->qkv_bias.assign(cfg->n_layers, hs_stage::QkvBias());
   for (int l = 0; l < cfg->n_layers && ok; ++l) {
     LayerMaps& m = s->maps[l];
     hs_layer_weights_t w = s->layers[l];
@@ -506,6 +509,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     g.tok_pos = meta + s->ml.tok_pos;
     g.tok_slot = meta + s->ml.tok_slot;
     g.rope = reinterpret_cast<const float2*>(s->ws_dev + s->ws.rope);
+    for (int i = 0; i < 3; ++i) g.qkv_bias[i] = s->qkv_bias[l].b[i];
     g.status = status;
     g.smid_log = slots(1);
     if (skinny(d, q_dim + 2 * kv_dim, kGemmQkv)) {
@@ -514,6 +518,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
       k.q_dim = q_dim; k.kv_dim = kv_dim; k.head_dim = Dh; k.n_kv_heads = c.n_kv_heads;
       k.q_out = q; k.k_cache = g.k_cache; k.v_cache = g.v_cache;
       k.tok_pos = g.tok_pos; k.tok_slot = g.tok_slot; k.rope = g.rope;
+      for (int i = 0; i < 3; ++i) k.qkv_bias[i] = g.qkv_bias[i];
       k.smid_log = slots(1);
       LaunchTimer t(s, 1, stream); where = "qkv gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
     } else { LaunchTimer t(s, 1, stream); where = "qkv gemm"; e = launch_gemm(g, sm_budget, stream); }
@@ -622,6 +627,16 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     if (e != cudaSuccess) break;
   }
   return e == cudaSuccess ? HS_OK : cuda_fail(where, e);
+}
+
+hs_status_t hs_stage_set_qkv_bias(hs_stage_t* s, int32_t layer, const void* b_q, const void* b_k, const void* b_v) {
+  if (!s || layer < 0 || layer >= s->cfg.n_layers) return HS_ERR_INVALID_ARG;
+  if (s->cfg.device < 0) return HS_ERR_NO_DEVICE;
+  const void* b[3] = {b_q, b_k, b_v};
+  for (const void* ptr : b)
+    if (reinterpret_cast<uintptr_t>(ptr) & 15) return HS_ERR_INVALID_ARG;
+  for (int i = 0; i < 3; ++i) s->qkv_bias[layer].b[i] = static_cast<const __nv_bfloat16*>(b[i]);
+  return HS_OK;
 }
 
 hs_status_t hs_stage_status(hs_stage_t* s) {

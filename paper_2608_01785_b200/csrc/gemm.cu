@@ -135,6 +135,22 @@ __device__ __forceinline__ bool spin_until_equal(const int* word, int value, vol
   }
 }
 
+// r[0..31] += b[0..31]: fp32 values held as raw bits, bias in bf16 (64-byte aligned; the same for every row,
+// so the loads of a warp are broadcasts out of the L1).
+__device__ __forceinline__ void add_bias32(uint32_t (&r)[32], const __nv_bfloat16* b) {
+  const uint4* src = reinterpret_cast<const uint4*>(b);
+#pragma unroll
+  for (int u = 0; u < 4; ++u) {
+    const uint4 w = __ldg(src + u);
+    const uint32_t pk[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      r[u * 8 + 2 * e] = __float_as_uint(__uint_as_float(r[u * 8 + 2 * e]) + __uint_as_float(pk[e] << 16));
+      r[u * 8 + 2 * e + 1] = __float_as_uint(__uint_as_float(r[u * 8 + 2 * e + 1]) + __uint_as_float(pk[e] & 0xffff0000u));
+    }
+  }
+}
+
 // Address of element e of (slot, kv head) in one layer's K or V pages.
 __device__ __forceinline__ __nv_bfloat16* cache_ptr(__nv_bfloat16* base, int slot, int hk, int n_kv_heads, int Dh,
                                                     int e) {
@@ -391,10 +407,12 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
           int region = 0;
           if (vcol >= p.q_dim) { region = 1; vcol -= p.q_dim; }
           if (region == 1 && vcol >= p.kv_dim) { region = 2; vcol -= p.kv_dim; }
+          const __nv_bfloat16* bias = p.qkv_bias[region];      // of this region's projection, or null
           if (region == 2) {
             for (int c = 0; c < 4; ++c) {
               tmem_ld32(taddr + half * 128 + c * 32, r0);
               tmem_ld_wait();
+              if (bias) add_bias32(r0, bias + vcol + c * 32);
               if (row_ok) {
 #pragma unroll
                 for (int e = 0; e < 32; ++e) v0[e] = __uint_as_float(r0[e]);
@@ -413,6 +431,10 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
               tmem_ld32(taddr + half * 128 + lo * 32, r0);
               tmem_ld32(taddr + half * 128 + hi * 32, r1);
               tmem_ld_wait();
+              if (bias) {                                        // the bias comes before the rotation
+                add_bias32(r0, bias + vcol + lo * 32);
+                add_bias32(r1, bias + vcol + hi * 32);
+              }
               const float2* cs = p.rope + size_t(pos) * half_dh + i0;
 #pragma unroll
               for (int e = 0; e < 32; e += 2) {

@@ -253,6 +253,16 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
         const int i0 = sub * 16 + jq;                        // first rotation pair / first element inside the head
         const int n_q_heads = p.q_dim / Dh;
         float a[4] = {lo.x, lo.y, lo.z, lo.w}, b[4] = {hi.x, hi.y, hi.z, hi.w};
+        const int region = head < n_q_heads ? 0 : head < n_q_heads + p.n_kv_heads ? 1 : 2;
+        if (p.qkv_bias[region]) {                            // the bias comes before the rotation
+          const int col = (head - (region == 0 ? 0 : region == 1 ? n_q_heads : n_q_heads + p.n_kv_heads)) * Dh + i0;
+          const uint2 wl = __ldg(reinterpret_cast<const uint2*>(p.qkv_bias[region] + col));
+          const uint2 wh = __ldg(reinterpret_cast<const uint2*>(p.qkv_bias[region] + col + half));
+          a[0] += __uint_as_float(wl.x << 16); a[1] += __uint_as_float(wl.x & 0xffff0000u);
+          a[2] += __uint_as_float(wl.y << 16); a[3] += __uint_as_float(wl.y & 0xffff0000u);
+          b[0] += __uint_as_float(wh.x << 16); b[1] += __uint_as_float(wh.x & 0xffff0000u);
+          b[2] += __uint_as_float(wh.y << 16); b[3] += __uint_as_float(wh.y & 0xffff0000u);
+        }
         if (head < n_q_heads + p.n_kv_heads) {               // q and k heads are rotated
           const float4* cs = reinterpret_cast<const float4*>(p.rope + size_t(p.tok_pos[row]) * half + i0);
           const float4 t0 = cs[0], t1 = cs[1];               // (cos, sin) of pairs i0 .. i0 + 3

@@ -45,6 +45,7 @@ struct GemmParams {
   const int32_t* tok_pos;    // [M]
   const int32_t* tok_slot;   // [M]
   const float2* rope;        // [max_position][Dh/2] (cos, sin)
+  const __nv_bfloat16* qkv_bias[3];   // optional biases of the q, k, v projections ([q_dim], [kv_dim], [kv_dim]); null = none
   // GateUp
   CUtensorMap tm_act;        // bf16 act [M, N], box 64 x 32, 128-byte swizzle
   int* status;               // device status word
@@ -72,6 +73,7 @@ struct SkinnyParams {
   const int32_t* tok_pos;
   const int32_t* tok_slot;
   const float2* rope;
+  const __nv_bfloat16* qkv_bias[3];   // optional, as in GemmParams
   __nv_bfloat16* act;        // GateUp: 16-bit [T, N]
   int act_f16;
   int* smid_log;

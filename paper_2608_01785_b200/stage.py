@@ -66,6 +66,14 @@ class Stage:
     def status(self) -> int:
         return B.hs_stage_status(self.handle)
 
+    def set_qkv_bias(self, layer: int, b_q=None, b_k=None, b_v=None) -> None:
+        """bf16 device tensors (or None) added to the layer's q, k, v projections before RoPE; kept alive here."""
+        for t in (b_q, b_k, b_v):
+            assert t is None or (t.dtype == torch.bfloat16 and t.is_cuda and t.is_contiguous())
+        self._biases = getattr(self, "_biases", {})
+        self._biases[layer] = (b_q, b_k, b_v)
+        B.hs_stage_set_qkv_bias(self.handle, layer, *[0 if t is None else t.data_ptr() for t in (b_q, b_k, b_v)])
+
     def debug_tensor(self, name: str) -> torch.Tensor:
         """Copy of a private intermediate, shaped [max_tokens, width] ("q" is bf16; "h", "o" and "act" are
         fp16, or bf16 when the stage was made with HS_FLAG_BF16_ACTIVATIONS), or of the SM census ("smid";

@@ -194,6 +194,8 @@ EDGE = {
     "two_layers_talker_like": (wl.StageDims(2, 1024, 16, 4, 64, 2816), [1] * 16, [128 + 57 * i for i in range(16)]),
     # few tokens against a long K: the QKV and gate/up GEMMs split K four ways through the scratch tile
     "small_step_split_k": (wl.StageDims(1, 2048, 8, 2, 128, 1024), [20, 1, 1], [0, 300, 17]),
+    # the RoPE base of long-context checkpoints, positions up to 3000
+    "rope_base_1e6": (wl.StageDims(1, 256, 4, 2, 64, 688, rope_base=1.0e6), [90, 1, 1], [0, 2999, 1500]),
     # rows too wide for the bulk-staged RMSNorm (register-staged fallback), K split eight ways
     "wide_rows_d8192": (wl.StageDims(1, 8192, 2, 2, 64, 128), [20, 1], [0, 37]),
 }
@@ -246,6 +248,73 @@ def test_edge_cases_match_oracle(orc, name):
     err = rel_err(y, y_ref)
     print(f"{name}, bf16 activations: max|err|/RMS = {err:.2e}")
     assert err <= TOL
+
+
+BIAS_CASES = {
+    # name: (dims, q_len, ctx_len): which QKV epilogue adds the biases
+    "pair_tiles_dh64": (wl.StageDims(2, 256, 4, 2, 64, 688), [100, 60, 1, 1], [0, 37, 64, 200]),   # T > 128
+    "single_tile_dh128": (wl.StageDims(1, 256, 2, 2, 128, 512), [70, 1, 33], [0, 200, 5]),         # 64 < T <= 128
+    "streaming_kernel_dh64": (wl.StageDims(2, 1024, 16, 4, 64, 2816), [1] * 16, [128 + 57 * i for i in range(16)]),
+    "streaming_kernel_dh128": (wl.StageDims(1, 2048, 8, 2, 128, 1024), [20, 1, 1], [0, 300, 17]),
+}
+
+
+@pytest.mark.parametrize("name", sorted(BIAS_CASES))
+def test_qkv_bias_matches_oracle(orc, name):
+    """Biases on q, k and v (N(0, 0.5): as large as the projections themselves) in every variant of the QKV
+    epilogue; the same step with one bias missing follows the oracle with that bias missing, so none of the
+    three is dropped or attached to the wrong projection."""
+    dims, q_len, ctx_len = BIAS_CASES[name]
+    batch = wl.BatchSpec(list(q_len), list(ctx_len))
+    case = make_case(dims, batch, seed=21, kv_fill=True)
+    g = torch.Generator().manual_seed(77)
+    q_dim, kv_dim = dims.n_q_heads * dims.head_dim, dims.n_kv_heads * dims.head_dim
+    biases = [[(torch.randn(n, generator=g) * 0.5).to(torch.bfloat16) for n in (q_dim, kv_dim, kv_dim)]
+              for _ in range(dims.n_layers)]
+    weights = [dict(lw, b_q=b[0].float().numpy(), b_k=b[1].float().numpy(), b_v=b[2].float().numpy())
+               for lw, b in zip(case.weights, biases)]
+    y_ref = orc.step(case.cfg, weights, case.kv_pool.copy(), batch.q_len, batch.ctx_len, case.block_tables, case.x)
+    y_plain = orc.step(case.cfg, case.weights, case.kv_pool.copy(), batch.q_len, batch.ctx_len, case.block_tables,
+                       case.x)
+    assert rel_err(y_plain, y_ref) > 0.05
+    outs = []
+    for budget in (148, 5):
+        st = make_stage(case)
+        dev_b = [[t.to(st.device) for t in b] for b in biases]
+        for l, b in enumerate(dev_b):
+            st.set_qkv_bias(l, *b)
+        y, pool = run_step(st, case, budget)
+        err = rel_err(y, y_ref)
+        print(f"{name}, sm_budget {budget}: max|err|/RMS = {err:.2e}")
+        assert err <= TOL
+        outs.append((y, pool))
+        if budget == 148:
+            for drop, key in enumerate(("b_q", "b_k", "b_v")):
+                w_drop = [{k: v for k, v in weights[0].items() if k != key}] + weights[1:]
+                y_ref_drop = orc.step(case.cfg, w_drop, case.kv_pool.copy(), batch.q_len, batch.ctx_len,
+                                      case.block_tables, case.x)
+                assert rel_err(y_ref_drop, y_ref) > 5e-3, key      # the missing bias is visible in the oracle
+                st.kv_pool.copy_(wl.bits_to_bf16_tensor(case.kv_pool, st.device))
+                st.set_qkv_bias(0, *[None if i == drop else t for i, t in enumerate(dev_b[0])])
+                y_drop, _ = run_step(st, case, budget)
+                assert rel_err(y_drop, y_ref_drop) <= TOL, key     # and the GPU follows it
+        st.close()
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+
+
+def test_qkv_bias_argument_errors(orc):
+    case = config1_case(orc)
+    st = make_stage(case)
+    try:
+        buf = torch.zeros(1024, dtype=torch.bfloat16, device=st.device)
+        for args, code in (((-1, 0, 0, 0), B.HS_ERR_INVALID_ARG), ((1, 0, 0, 0), B.HS_ERR_INVALID_ARG),
+                           ((0, buf.data_ptr() + 2, 0, 0), B.HS_ERR_INVALID_ARG)):
+            with pytest.raises(B.HsError) as e:
+                B.hs_stage_set_qkv_bias(st.handle, *args)
+            assert e.value.status == code
+        B.hs_stage_set_qkv_bias(st.handle, 0, 0, 0, 0)       # clearing is allowed
+    finally:
+        st.close()
 
 
 def test_chunked_prefill_then_decode_on_the_gpu_cache(orc):
