@@ -49,6 +49,9 @@ typedef struct {
   int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn;
   int32_t page_size, num_pages;
   float rms_eps, rope_base;
+  int32_t bidirectional; /* 0: causal (a token sees the keys up to its own position); 1: every token of a
+                          * sequence sees all of the sequence's keys, the cached ones and all new ones (the
+                          * attention of a denoising / DiT-style block: no mask) */
 } hso_config_t;
 
 typedef struct {
@@ -295,7 +298,8 @@ int hso_layer(const hso_config_t *c, const hso_layer_t *w, int layer, uint16_t *
   for (int r = 0; r < R; ++r)
     for (int hq = 0; hq < Hq; ++hq) {
       int t = rows[r];
-      hso_attend(c, kv_pool, layer, block_tables + (size_t)tok_seq[t] * mpps, tok_pos[t], hq,
+      int last = c->bidirectional ? ctx_len[tok_seq[t]] + q_len[tok_seq[t]] - 1 : tok_pos[t];
+      hso_attend(c, kv_pool, layer, block_tables + (size_t)tok_seq[t] * mpps, last, hq,
                  q + (size_t)r * Qd + (size_t)hq * Dh, o + (size_t)r * Qd + (size_t)hq * Dh, NULL);
     }
   free(q);

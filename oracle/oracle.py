@@ -45,7 +45,7 @@ def build(force: bool = False) -> None:
 class _Cfg(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim",
                                           "d_ffn", "page_size", "num_pages")] + \
-               [("rms_eps", C.c_float), ("rope_base", C.c_float)]
+               [("rms_eps", C.c_float), ("rope_base", C.c_float), ("bidirectional", C.c_int32)]
 
 
 class _Layer(C.Structure):
@@ -85,10 +85,11 @@ class OracleConfig:
     num_pages: int
     rms_eps: float = 1e-6
     rope_base: float = 10000.0
+    bidirectional: bool = False      # no causal mask: every token sees all keys of its sequence
 
     def c(self) -> _Cfg:
         return _Cfg(self.n_layers, self.d_model, self.n_q_heads, self.n_kv_heads, self.head_dim, self.d_ffn,
-                    self.page_size, self.num_pages, self.rms_eps, self.rope_base)
+                    self.page_size, self.num_pages, self.rms_eps, self.rope_base, int(self.bidirectional))
 
     def kv_pool_elems(self) -> int:
         return self.n_layers * 2 * self.num_pages * self.n_kv_heads * self.page_size * self.head_dim

@@ -218,7 +218,7 @@ def test_causal_gqa_brute_force(oracle64, page_size):
 SMALL = wl.StageDims(2, 64, 4, 2, 16, 96)
 
 
-def _torch_reference_single_sequence(dims, weights, x, n_layers):
+def _torch_reference_single_sequence(dims, weights, x, n_layers, causal=True):
     """float64 composition of library routines for one non-paged sequence starting at position 0."""
     xt = torch.from_numpy(x).double()
     n = xt.shape[0]
@@ -239,7 +239,7 @@ def _torch_reference_single_sequence(dims, weights, x, n_layers):
         k = rope(F.linear(h, w["w_k"], w.get("b_k")).view(n, Hkv, Dh)).bfloat16().double()
         v = F.linear(h, w["w_v"], w.get("b_v")).view(n, Hkv, Dh).bfloat16().double()
         k = k.repeat_interleave(Hq // Hkv, dim=1); v = v.repeat_interleave(Hq // Hkv, dim=1)
-        o = F.scaled_dot_product_attention(q.transpose(0, 1), k.transpose(0, 1), v.transpose(0, 1), is_causal=True)
+        o = F.scaled_dot_product_attention(q.transpose(0, 1), k.transpose(0, 1), v.transpose(0, 1), is_causal=causal)
         xt = xt + o.transpose(0, 1).reshape(n, Hq * Dh) @ w["w_o"].T
         h2 = F.rms_norm(xt, (dims.d_model,), w["g_mlp"], dims.rms_eps)
         xt = xt + (F.silu(h2 @ w["w_gate"].T) * (h2 @ w["w_up"].T)) @ w["w_down"].T
@@ -315,6 +315,40 @@ def test_qkv_bias_matches_library_composition_and_closed_form(oracle64):
                             for hq in range(dims.n_q_heads)])
     want = case.x.astype(np.float64) + (z["w_o"].astype(np.float64) @ o_row)[None, :]
     assert rel_err(y, want) < 1e-12
+
+
+def test_bidirectional_attention_matches_library_and_invariants(oracle64):
+    """The unmasked attention of a denoising-style block: against torch's attention without a causal mask in the
+    float64 composition; it differs from the causal result on every row but the last (which sees all keys either
+    way); and the mean-pooling closed form: with W_q = 0 every score is 0, so every row's attention output is
+    the plain mean of all value rows of the sequence."""
+    import dataclasses
+    dims = wl.StageDims(2, 64, 4, 2, 16, 96)
+    case = make_case(dims, wl.BatchSpec([29], [0]), seed=9)
+    weights = [{k: (v if k.startswith("g_") else v * 8.0) for k, v in lw.items()} for lw in case.weights]
+    cfg = dataclasses.replace(case.cfg, bidirectional=True)
+    args = (case.batch.q_len, case.batch.ctx_len, case.block_tables, case.x)
+    y = oracle64.step(cfg, weights, case.kv_pool.copy(), *args)
+    want = _torch_reference_single_sequence(dims, weights, case.x, dims.n_layers, causal=False)
+    assert rel_err(y, want) < 1e-10
+    y_causal = oracle64.step(case.cfg, weights, case.kv_pool.copy(), *args)
+    one = dataclasses.replace(cfg, n_layers=1)
+    pool1 = case.kv_pool[: one.kv_pool_elems()]
+    y1 = oracle64.step(one, weights[:1], pool1.copy(), *args)
+    y1c = oracle64.step(dataclasses.replace(one, bidirectional=False), weights[:1], pool1.copy(), *args)
+    row_diff = np.max(np.abs(y1 - y1c), axis=1)
+    assert row_diff[-1] == 0.0 and np.all(row_diff[:-1] > 1e-6)      # one layer: only the last row sees the same keys
+    assert rel_err(y, y_causal) > 0.05
+
+    z = dict(weights[0], w_q=np.zeros_like(weights[0]["w_q"]), w_down=np.zeros_like(weights[0]["w_down"]))
+    y0 = oracle64.step(one, [z], pool1.copy(), *args)
+    xt = torch.from_numpy(case.x).double()
+    h = F.rms_norm(xt, (dims.d_model,), torch.from_numpy(z["g_attn"]).double(), dims.rms_eps)
+    v = (h @ torch.from_numpy(z["w_v"]).double().T).bfloat16().double()          # [n, Hkv * Dh], as cached
+    G = dims.n_q_heads // dims.n_kv_heads
+    o_row = v.mean(dim=0).view(dims.n_kv_heads, dims.head_dim).repeat_interleave(G, dim=0).reshape(-1)
+    want0 = xt + (torch.from_numpy(z["w_o"]).double() @ o_row)[None, :]
+    assert rel_err(y0, want0.numpy()) < 1e-12
 
 
 def test_zero_gate_weight_means_mlp_adds_nothing(oracle32):
