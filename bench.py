@@ -3,7 +3,7 @@
 the tensor-core roofline reached by the dominant kernel and the CPU oracle timed beside it.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload c2_shared|c3_7b|c4_talker|c1_tiny] [--sm-budget B]
+                    [--workload c2_shared|c3_7b|c4_talker|c6_dit|c1_tiny] [--sm-budget B]
 
 A "step" is one hs_stage_step over the whole batch (every layer: RMSNorm, QKV GEMM + RoPE + cache write,
 paged attention, out-proj, gate/up + SwiGLU, down).  Inputs are seeded and synthetic.  With N > 1 (one
@@ -33,7 +33,7 @@ from paper_2608_01785_b200 import workloads as wl  # noqa: E402
 
 METRIC = "shared_stage_tokens_per_s"
 UNIT = "tokens/s"
-SEED = {"c1_tiny": 0, "c2_shared": 1, "c3_7b": 2, "c4_talker": 3, "c3_decode": 2}
+SEED = {"c1_tiny": 0, "c2_shared": 1, "c3_7b": 2, "c4_talker": 3, "c3_decode": 2, "c6_dit": 5}
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one gate/up GEMM launch, from the ncu
 # capture summarised in profiles/gemm_pair_gateup_c2_shared.md (None where no capture of that launch exists).
 GATEUP_DRAM_TRAFFIC_BYTES = {"c2_shared": 69989376 + 39707904}
@@ -108,7 +108,8 @@ def build_stage(name: str, device: int, init: str = "n002", layers: int = 0, fla
     weights = wl.make_weights(dims, seed, dev, init)
     num_pages = wl.pages_needed(batch) + 8
     mpps = max(-(-t // 16) for t in batch.total_len())
-    stage = Stage(dims, weights, num_pages, batch.n_tokens, batch.n_seqs, mpps, max(batch.total_len()), device, flags)
+    stage = Stage(dims, weights, num_pages, batch.n_tokens, batch.n_seqs, mpps, max(batch.total_len()), device,
+                  flags | wl.STAGE_FLAGS.get(name, 0))
     # context of the decode sequences: values do not change the timing; N(0,1) bf16 stands in for K/V
     # written by earlier steps
     g = torch.Generator(device=dev)
@@ -162,7 +163,7 @@ def cpu_oracle_sample(name: str, target_s: float):
     tables = [alloc.alloc(s, t) for s, t in enumerate(batch.total_len())]
     bt = block_table_array(tables, max(len(t) for t in tables))
     cfg = OracleConfig(1, dims.d_model, dims.n_q_heads, dims.n_kv_heads, dims.head_dim, dims.d_ffn, 16, num_pages,
-                       dims.rms_eps, dims.rope_base)
+                       dims.rms_eps, dims.rope_base, bool(wl.STAGE_FLAGS.get(name, 0) & 2))
     w = wl.weights_to_numpy([wl.make_layer_weights(one, seed, 0)])
     pool = wl.bf16_bits_numpy(wl.make_kv_fill(one, num_pages, seed)).reshape(-1).copy()
     x = wl.to_f32_numpy(wl.make_x(batch.n_tokens, dims.d_model, seed))
@@ -384,7 +385,7 @@ def main():
     e2e_value = aggregate_tokens_per_s(T, world, ms_e2e)
 
     # ---- step latency vs SM budget, and the co-run with a downstream stage (rank 0, single GPU) ----
-    sweep, corun_rows = None, None
+    sweep, corun_rows, corun_dit_rows = None, None, None
     if rank == 0 and world == 1 and not args.no_sweep:
         sweep = []
         for bud in [x for x in wl.SM_BUDGETS.get(name, (148, 112, 74, 37)) if x <= stage.sm_count]:
@@ -403,6 +404,13 @@ def main():
             corun_rows = [corun(stage, b, talker, tb, bud, args.steps) for bud in wl.SM_BUDGETS["c4_corun"]]
             assert talker.status() == 0
             talker.close()
+            # the same co-run with the denoising-style stage (the image path's downstream partner)
+            dit, ddims, dbatch, dbt, dx = build_stage("c6_dit", local_rank)
+            dy = torch.empty(dbatch.n_tokens, ddims.d_model, dtype=torch.float32, device=dev)
+            db = dit.make_batch(dbatch.q_len, dbatch.ctx_len, dbt, dx, dy)
+            corun_dit_rows = [corun(stage, b, dit, db, bud, max(args.steps // 4, 5)) for bud in wl.SM_BUDGETS["c4_corun"]]
+            assert dit.status() == 0
+            dit.close()
 
     if rank != 0:
         if world > 1:
@@ -463,7 +471,7 @@ def main():
                     "d2h_bytes_per_step": T * d * 4},
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "roofline_decode_attention": decode_roofline, "kernels": kernels,
-            "budget_sweep": sweep, "corun": corun_rows, "cpu_baseline": cpu}
+            "budget_sweep": sweep, "corun": corun_rows, "corun_dit": corun_dit_rows, "cpu_baseline": cpu}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -72,6 +72,13 @@ extern "C" {
  * activation act) in bf16 instead of the default fp16, and make no fp16 copies of the weights -- see the
  * numeric contract above. */
 #define HS_FLAG_BF16_ACTIVATIONS 1u
+/*
+ * No causal mask: every token of a sequence attends to all of the sequence's keys, the cached ones and all new
+ * ones of the step (K/V of the whole step are written before any attention runs).  This is the attention of a
+ * denoising (DiT-style) block, the kind of downstream visual generator the paper co-locates with the shared stage
+ * (Sec. 2.1, Sec. 3.1); such a stage normally runs every step with ctx_len = 0 and frees nothing in between.
+ */
+#define HS_FLAG_BIDIRECTIONAL 2u
 
 typedef struct hs_stage hs_stage_t; /* opaque; owned by the library */
 
@@ -100,7 +107,7 @@ typedef struct {
   int32_t max_seqs;          /* most sequences in one step */
   int32_t max_pages_per_seq; /* row length of block tables */
   int32_t max_position;      /* ctx_len + q_len never exceeds this (sizes the RoPE table) */
-  uint32_t flags;            /* 0, or HS_FLAG_BF16_ACTIVATIONS */
+  uint32_t flags;            /* 0, or an OR of HS_FLAG_BF16_ACTIVATIONS, HS_FLAG_BIDIRECTIONAL */
 } hs_stage_config_t;
 
 /* One layer's weights: device pointers to bf16, row-major [out_features, in_features] (biases: hs_stage_set_qkv_bias). */

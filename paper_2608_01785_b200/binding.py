@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libhorizonserve.so")
 
 HS_ABI_VERSION = 1
 HS_FLAG_BF16_ACTIVATIONS = 1      # hs_stage_config_t.flags: keep h, o and act in bf16 instead of fp16
+HS_FLAG_BIDIRECTIONAL = 2         # hs_stage_config_t.flags: attention without the causal mask (denoising-style block)
 HS_OK, HS_ERR_INVALID_ARG, HS_ERR_INVALID_BUDGET, HS_ERR_UNSUPPORTED_SHAPE, HS_ERR_OUT_OF_PAGES, \
     HS_ERR_BAD_BLOCK_TABLE, HS_ERR_CUDA, HS_ERR_TIMEOUT, HS_ERR_NO_DEVICE, HS_ERR_UNKNOWN_SEQ = range(10)
 

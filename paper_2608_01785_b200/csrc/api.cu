@@ -535,6 +535,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     a.num_pages = c.num_pages; a.max_pages_per_seq = c.max_pages_per_seq; a.layer = l;
     a.seq_tok0 = meta + s->ml.seq_tok0;
     a.seq_ctx = meta + s->ml.seq_ctx;
+    a.seq_qlen = meta + s->ml.seq_qlen;
+    a.bidirectional = (c.flags & HS_FLAG_BIDIRECTIONAL) ? 1 : 0;
     a.block_tables = meta + s->ml.block_tables;
     a.prefill_items = meta + s->ml.prefill_items;
     a.n_prefill_items = plan.n_prefill_items;

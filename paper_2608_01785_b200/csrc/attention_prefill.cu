@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
         const int seq = it.x, hk = it.y, tok_begin = it.z, n_tok = it.w;
         const int tok0 = p.seq_tok0[seq] + tok_begin;
-        const int n_keys = p.seq_ctx[seq] + tok_begin + n_tok;
+        const int n_keys = p.seq_ctx[seq] + (p.bidirectional ? p.seq_qlen[seq] : tok_begin + n_tok);
         const int n_kblocks = (n_keys + PF_KEYS - 1) / PF_KEYS;
         const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq;
         // Q tile: one box of Mt token rows x 64 columns per (head, half)
@@ -204,7 +204,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         if (++rs == 2) { rs = 0; rph ^= 1; }
         if (item >= p.n_prefill_items) break;
         const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
-        const int n_keys = p.seq_ctx[it.x] + it.z + it.w;
+        const int n_keys = p.seq_ctx[it.x] + (p.bidirectional ? p.seq_qlen[it.x] : it.z + it.w);
         const int n_kblocks = (n_keys + PF_KEYS - 1) / PF_KEYS;
         const uint32_t qb = n_items_seen & 1;
         if (!mbar_wait(&bar->q_full[qb], (n_items_seen >> 1) & 1, abort_flag, p.status)) break;
@@ -245,11 +245,12 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
       const int seq = it.x, hk = it.y, tok_begin = it.z, n_tok = it.w;
       const int tok0 = p.seq_tok0[seq] + tok_begin;
       const int pos0 = p.seq_ctx[seq] + tok_begin;
-      const int n_keys = pos0 + n_tok;
+      const int n_keys = p.bidirectional ? p.seq_ctx[seq] + p.seq_qlen[seq] : pos0 + n_tok;
       const int n_kblocks = (n_keys + PF_KEYS - 1) / PF_KEYS;
       const int g = r / Mt, tok = r - g * Mt;
       const bool row_valid = g < G && tok < n_tok;
-      const int pos = pos0 + min(tok, n_tok - 1);          // padding rows behave like the last token
+      // last key a row sees: its own position (padding rows behave like the last token), or the sequence's last key
+      const int pos = p.bidirectional ? n_keys - 1 : pos0 + min(tok, n_tok - 1);
 
       float o_reg[DH];
 #pragma unroll

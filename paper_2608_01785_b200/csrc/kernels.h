@@ -138,6 +138,8 @@ struct AttnParams {
   int n_q_heads, n_kv_heads, head_dim, num_pages, max_pages_per_seq, layer;
   const int32_t* seq_tok0;
   const int32_t* seq_ctx;
+  const int32_t* seq_qlen;   // new tokens per sequence (prefill kernel, bidirectional only)
+  int bidirectional;         // prefill kernel: 1 = no causal mask, a row sees every key of its sequence
   const int32_t* block_tables;
   const int32_t* prefill_items;    // int4 per item
   int n_prefill_items;

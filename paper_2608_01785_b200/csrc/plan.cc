@@ -9,7 +9,7 @@
 namespace hs {
 
 hs_status_t validate_config(const hs_stage_config_t& c) {
-  if (c.abi_version != HS_ABI_VERSION || (c.flags & ~HS_FLAG_BF16_ACTIVATIONS) != 0) return HS_ERR_INVALID_ARG;
+  if (c.abi_version != HS_ABI_VERSION || (c.flags & ~(HS_FLAG_BF16_ACTIVATIONS | HS_FLAG_BIDIRECTIONAL)) != 0) return HS_ERR_INVALID_ARG;
   if (c.n_layers < 1 || c.d_model < 64 || c.n_q_heads < 1 || c.n_kv_heads < 1 || c.d_ffn < 64) return HS_ERR_INVALID_ARG;
   if (c.num_pages < 1 || c.max_tokens < 1 || c.max_seqs < 1 || c.max_pages_per_seq < 1 || c.max_position < 1)
     return HS_ERR_INVALID_ARG;

@@ -63,6 +63,10 @@ DIMS = {
     "c4_talker": StageDims(12, 1024, 16, 4, 64, 2816),
 }
 DIMS["c3_decode"] = DIMS["c3_7b"]
+# A denoising-style (DiT-like) downstream stage, the visual generator kind of the paper's Sec. 2.1: the talker's
+# width and depth with multi-head attention and no causal mask; a step denoises 4 images of 256 latent tokens.
+DIMS["c6_dit"] = StageDims(12, 1024, 16, 16, 64, 2816)
+STAGE_FLAGS = {"c6_dit": 2}      # hs_stage_config_t.flags by workload (2 = no causal mask)
 SM_BUDGETS = {
     "c1_tiny": (148, 8),
     "c2_shared": (148, 112, 74, 37),
@@ -115,6 +119,8 @@ def make_batch(name: str, seed: int) -> BatchSpec:
     if name == "c4_talker":
         dec = r.integers(128, 1025, size=16).tolist()
         return BatchSpec([1] * 16, dec)
+    if name == "c6_dit":
+        return BatchSpec([256] * 4, [0] * 4)
     raise KeyError(name)
 
 

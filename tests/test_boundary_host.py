@@ -86,7 +86,9 @@ def test_activation_format_flag_sizes_the_workspace():
     extra = B.hs_workspace_bytes(cfg16) - B.hs_workspace_bytes(cfgbf)
     assert w_bytes <= extra <= w_bytes + 7 * 1024 * dims.n_layers
     assert B.hs_kv_pool_bytes(cfg16) == B.hs_kv_pool_bytes(cfgbf) > 0
-    bad = B.make_config(dims, 64, 128, 8, 8, 256, device=-1, flags=2)
+    bidir = B.make_config(dims, 64, 128, 8, 8, 256, device=-1, flags=B.HS_FLAG_BIDIRECTIONAL)
+    assert B.hs_workspace_bytes(bidir) == B.hs_workspace_bytes(cfg16)      # the mask changes no buffer
+    bad = B.make_config(dims, 64, 128, 8, 8, 256, device=-1, flags=4)
     assert B.hs_workspace_bytes(bad) == 0 and B.hs_kv_pool_bytes(bad) == 0
 
 

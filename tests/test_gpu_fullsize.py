@@ -220,6 +220,35 @@ def test_config3_budget_sweep_and_sampled_layer_local(orc, init):
         stage.close()
 
 
+# ------------------------------------------------- denoising-style stage (no causal mask) --
+def test_denoising_stage_budget_sweep_and_two_layer_parity(orc):
+    """The c6_dit workload (4 images x 256 latent tokens, multi-head attention without a mask): the 12-layer
+    step bit for bit over budgets, and its first two layers end to end against the oracle."""
+    import dataclasses
+    stage, dims, batch, bt, x = bench.build_stage("c6_dit", 0)
+    try:
+        assert stage.cfg.flags & 2
+        pool0 = stage.kv_pool.clone()
+        outs = [gpu_step(stage, batch, bt, x, budget, pool0).cpu().numpy() for budget in (stage.sm_count, 74, 28)]
+        assert np.all(np.isfinite(outs[0]))
+        for y in outs[1:]:
+            assert np.array_equal(y, outs[0])
+    finally:
+        stage.close()
+    stage2, dims2, batch, bt, x = bench.build_stage("c6_dit", 0, layers=2)
+    try:
+        pool0 = stage2.kv_pool.clone()
+        y_gpu = gpu_step(stage2, batch, bt, x, stage2.sm_count, pool0).cpu().numpy()
+        cfg = dataclasses.replace(ocfg(dims2, 2, stage2.cfg.num_pages), bidirectional=True)
+        y_ref = orc.step(cfg, wl.weights_to_numpy(stage2.weights), wl.bf16_bits_numpy(pool0).reshape(-1).copy(),
+                         batch.q_len, batch.ctx_len, bt, wl.to_f32_numpy(x))
+        err = rel_err(y_gpu, y_ref)
+        print(f"denoising-style stage, 2 layers end to end: max|err|/RMS = {err:.2e}")
+        assert err <= TOL
+    finally:
+        stage2.close()
+
+
 # ------------------------------------------------- config 3 dimensions, decode-only ticks --
 @pytest.mark.parametrize("n_dec", [64, 24, 9])
 def test_config3_decode_only_tick(orc, n_dec):

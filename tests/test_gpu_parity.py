@@ -302,6 +302,39 @@ def test_qkv_bias_matches_oracle(orc, name):
     assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
 
 
+BIDIR_CASES = {
+    # name: (dims, q_len, ctx_len)
+    "dh64_several_sequences": (wl.StageDims(2, 256, 4, 2, 64, 688), [100, 37, 1, 64], [0, 0, 0, 0]),
+    "dh128_with_cached_context": (wl.StageDims(1, 256, 2, 2, 128, 512), [70, 20, 1], [0, 33, 40]),
+    "gqa_8_long": (wl.StageDims(1, 256, 8, 1, 128, 640), [300], [0]),
+}
+
+
+@pytest.mark.parametrize("name", sorted(BIDIR_CASES))
+def test_bidirectional_attention_matches_oracle(orc, name):
+    """HS_FLAG_BIDIRECTIONAL: no causal mask (the attention of a denoising-style block).  Early rows now depend on
+    later tokens of their sequence, so the result must differ from the causal one on those rows."""
+    import dataclasses
+    dims, q_len, ctx_len = BIDIR_CASES[name]
+    batch = wl.BatchSpec(list(q_len), list(ctx_len))
+    case = make_case(dims, batch, seed=31, kv_fill=True)
+    cfg = dataclasses.replace(case.cfg, bidirectional=True)
+    y_ref = orc.step(cfg, case.weights, case.kv_pool.copy(), batch.q_len, batch.ctx_len, case.block_tables, case.x)
+    y_causal = orc.step(case.cfg, case.weights, case.kv_pool.copy(), batch.q_len, batch.ctx_len, case.block_tables,
+                        case.x)
+    assert rel_err(y_causal, y_ref) > 5 * TOL
+    outs = []
+    for budget in (148, 5):
+        st = make_stage(case, flags=B.HS_FLAG_BIDIRECTIONAL)
+        y, pool = run_step(st, case, budget)
+        st.close()
+        err = rel_err(y, y_ref)
+        print(f"{name}, sm_budget {budget}: max|err|/RMS = {err:.2e}")
+        assert err <= TOL
+        outs.append((y, pool))
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+
+
 def test_qkv_bias_argument_errors(orc):
     case = config1_case(orc)
     st = make_stage(case)
