@@ -150,6 +150,7 @@ hs_status_t ensure_attributes(int device) {
 }  // namespace hs
 
 using namespace hs;
+static_assert(kDecodeWarps == kDecodeKernelWarps, "the planner sizes decode items for the kernel's warp count");
 
 struct hs_stage {
   hs_stage_config_t cfg;
@@ -397,7 +398,7 @@ hs_status_t hs_stage_plan(hs_stage_t* s, const hs_batch_t* b, int32_t* tok_seq, 
   if (!s || !b) return HS_ERR_INVALID_ARG;
   std::vector<int32_t> meta(s->ml.total);
   StepPlan plan;
-  const hs_status_t st = plan_step(s->cfg, s->ml, *b, s->page_stamp, ++s->stamp, meta.data(), tok_seq, &plan);
+  const hs_status_t st = plan_step(s->cfg, s->ml, *b, s->sm_count, s->page_stamp, ++s->stamp, meta.data(), tok_seq, &plan);
   if (st != HS_OK) return st;
   if (tok_pos) memcpy(tok_pos, meta.data() + s->ml.tok_pos, size_t(plan.n_tokens) * 4);
   if (tok_slot) memcpy(tok_slot, meta.data() + s->ml.tok_slot, size_t(plan.n_tokens) * 4);
@@ -422,7 +423,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     s->ev_pending[slot] = false;
   }
   StepPlan plan;
-  hs_status_t st = plan_step(c, s->ml, *b, s->page_stamp, ++s->stamp, s->pinned[slot], nullptr, &plan);
+  hs_status_t st = plan_step(c, s->ml, *b, s->sm_count, s->page_stamp, ++s->stamp, s->pinned[slot], nullptr, &plan);
   if (st != HS_OK) return st;
   s->ring_pos = (slot + 1) % kRing;
 

@@ -153,7 +153,7 @@ __device__ __forceinline__ void merge_group(const float* part_o, const float* pa
 // writes the item's partial (max, sum, output) straight from its registers.  There is no producer warp,
 // no "slot free" barrier (a slot is refilled by the warp that has just finished reading it) and no
 // block-level synchronisation after start-up, so an SM keeps DC_WARPS x (DC_STAGES - 1) pages in flight.
-constexpr int DC_WARPS = 6, DC_THREADS = DC_WARPS * 32, DC_STAGES = 4;
+constexpr int DC_WARPS = kDecodeKernelWarps, DC_THREADS = DC_WARPS * 32, DC_STAGES = 4;
 
 template <int DH>
 constexpr int dc_smem_bytes() {

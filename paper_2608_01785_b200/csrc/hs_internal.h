@@ -10,8 +10,10 @@
 namespace hs {
 
 constexpr int kPage = HS_PAGE_SIZE;      // tokens per KV page
-constexpr int kDecodeSplit = 256;        // keys per decode split-KV work item (budget independent)
-static_assert(kDecodeSplit % 16 == 0 && kDecodeSplit / 16 <= 32, "the decode kernel keeps one page id per lane");
+constexpr int kDecodeSplit = 256;        // smallest number of keys per decode split-KV work item (sizes the buffers)
+constexpr int kDecodeWarps = 6;            // warps per block of the decode attention kernel (kernels.h: kDecodeKernelWarps)
+constexpr int kDecodeSplitMax = 512;     // largest number of keys per item the planner may choose
+static_assert(kDecodeSplit % 16 == 0 && kDecodeSplitMax / 16 <= 32, "the decode kernel keeps one page id per lane");
 constexpr int kPrefillRows = 128;        // (token, query head of one KV head) rows per prefill work item
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -68,7 +70,10 @@ struct StepPlan {
 // `page_stamp` is scratch of num_pages entries used to detect a page named by two sequences; `stamp`
 // must be a value not used by an earlier call.  tok_seq (nullable) receives the owning sequence of each
 // token.  Returns HS_OK, HS_ERR_INVALID_ARG or HS_ERR_BAD_BLOCK_TABLE.
-hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs_batch_t& b,
+// Keys per decode work item for this batch: 256, 384 or 512, whichever lets the device's warps finish the items in
+// the fewest, shortest rounds.  A function of the batch and of the device's SM count only (never of the budget).
+int pick_decode_split(const hs_stage_config_t& c, const hs_batch_t& b, int sm_count);
+hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs_batch_t& b, int sm_count,
                       std::vector<int32_t>& page_stamp, int32_t stamp, int32_t* meta, int32_t* tok_seq,
                       StepPlan* plan);
 

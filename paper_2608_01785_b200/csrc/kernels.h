@@ -12,6 +12,9 @@ namespace hs {
 // Dynamic shared memory every kernel requests at least, so that two blocks (of this or of a co-running
 // stage's kernel) never share an SM: more than half of the 227 KB an SM offers.
 constexpr int kMinSmemBytes = 117 * 1024;
+// Warps per block of the decode attention kernel (each works through one item at a time); the planner sizes its
+// work items for sm_count x this many warps.
+constexpr int kDecodeKernelWarps = 6;
 
 // ------------------------------------------------------------------ GEMM --
 // out = A[M,K] * W^T with W given as up to three row blocks [rows, K] (bf16, K contiguous).  The output

@@ -85,7 +85,32 @@ MetaLayout make_meta_layout(const hs_stage_config_t& c) {
   return m;
 }
 
-hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs_batch_t& b,
+int pick_decode_split(const hs_stage_config_t& c, const hs_batch_t& b, int sm_count) {
+  // Every warp of the decode kernel works through whole items, so the kernel lasts about
+  //   rounds x (pages per item + 8),   rounds = ceil(items / (0.97 x warps of the device)),
+  // in units of the time a warp needs for one page: the items are handed out in rounds (a short last round leaves
+  // most warps idle for a whole item), and an item costs about 8 page times on top of its pages (queue, record,
+  // page ids, first bytes, partial result, its share of the merge).  Measured on B200, 64 sequences of 512..4096
+  // keys, 4 KV heads: 256 keys 72 us, 384 keys 68 us, 512 keys 76 us per launch; 32 sequences: 49 / 39 / 44 us.
+  const int warps = (sm_count > 0 ? sm_count : 148) * kDecodeWarps;
+  int best = kDecodeSplit;
+  double best_cost = 1e30;
+  for (int split = kDecodeSplit; split <= kDecodeSplitMax; split += 128) {
+    int64_t items = 0;
+    for (int s = 0; s < b.n_seqs; ++s)
+      if (b.q_len[s] == 1) items += int64_t(c.n_kv_heads) * ceil_div(b.ctx_len[s] + 1, split);
+    if (items == 0) return kDecodeSplit;
+    const double rounds = double((items * 100 + int64_t(warps) * 97 - 1) / (int64_t(warps) * 97));
+    const double cost = rounds * (split / kPage + 8);
+    if (cost < best_cost - 1e-9) {
+      best_cost = cost;
+      best = split;
+    }
+  }
+  return best;
+}
+
+hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs_batch_t& b, int sm_count,
                       std::vector<int32_t>& page_stamp, int32_t stamp, int32_t* meta, int32_t* tok_seq,
                       StepPlan* plan) {
   if (!b.q_len || !b.ctx_len || !b.block_tables) return HS_ERR_INVALID_ARG;
@@ -112,6 +137,7 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
 
   const int G = c.n_q_heads / c.n_kv_heads;
   const int Mt = prefill_tokens_per_item(G);
+  const int split = pick_decode_split(c, b, sm_count);
   StepPlan p;
   p.n_tokens = b.n_tokens;
   p.n_seqs = b.n_seqs;
@@ -138,15 +164,15 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
       if (tok_seq) tok_seq[t + j] = s;
     }
     if (n == 1) {
-      // decode: keys 0..ctx split into fixed runs of kDecodeSplit
-      const int keys = ctx + 1, splits = ceil_div(keys, kDecodeSplit);
+      // decode: keys 0..ctx split into fixed runs of `split` keys
+      const int keys = ctx + 1, splits = ceil_div(keys, split);
       if (meta) {
         int32_t* row = meta + ml.decode_rows + n_dec_rows * 4;
         row[0] = s; row[1] = t; row[2] = n_dec_items; row[3] = splits;
         for (int hk = 0; hk < c.n_kv_heads; ++hk)
           for (int j = 0; j < splits; ++j) {
             int32_t* it = meta + ml.decode_items + (n_dec_items + hk * splits + j) * 8;
-            it[0] = n_dec_rows; it[1] = hk; it[2] = j * kDecodeSplit; it[3] = std::min(keys, (j + 1) * kDecodeSplit);
+            it[0] = n_dec_rows; it[1] = hk; it[2] = j * split; it[3] = std::min(keys, (j + 1) * split);
             it[4] = s; it[5] = t; it[6] = n_dec_items + hk * splits; it[7] = splits;
           }
       }
