@@ -57,6 +57,12 @@ typedef struct {
 typedef struct {
   const real *g_attn, *w_q, *w_k, *w_v, *w_o, *g_mlp, *w_gate, *w_up, *w_down;
   const real *b_q, *b_k, *b_v; /* [Hq Dh], [Hkv Dh], [Hkv Dh]; NULL = no bias */
+  /* Per-sequence modulation of a conditioned (DiT-style, "adaLN-Zero") block, [n_seqs][6][d], NULL = none:
+   * rows 0..5 of sequence s are shift_a, scale_a, gate_a, shift_m, scale_m, gate_m and
+   *   h_a = rmsnorm(x) g_attn (1 + scale_a) + shift_a,   x += gate_a * (attention output W_o^T),
+   *   h_m = rmsnorm(x) g_mlp  (1 + scale_m) + shift_m,   x += gate_m * (MLP output),
+   * all products element-wise over the d_model axis. */
+  const real *mod;
 } hso_layer_t;
 
 /* Diagnostic switch (never the pass/fail oracle): bit mask of intermediates
@@ -204,6 +210,23 @@ void hso_attend(const hso_config_t *c, const uint16_t *kv_pool, int layer, const
 }
 
 /* ----------------------------------------------------------- one layer -- */
+/* h[r, :] = h[r, :] * (1 + scale) + shift with the vectors of row r's sequence (mod == NULL: nothing).
+ * seq_of[r] is the sequence of row r; `which` = 0 for the attention branch, 3 for the MLP branch. */
+static void modulate(int R, int d, const real *mod, const int *seq_of, int which, real *h) {
+  if (!mod) return;
+  for (int r = 0; r < R; ++r) {
+    const real *shift = mod + ((size_t)seq_of[r] * 6 + which) * d, *scale = shift + d;
+    for (int i = 0; i < d; ++i) h[(size_t)r * d + i] = h[(size_t)r * d + i] * ((real)1 + scale[i]) + shift[i];
+  }
+}
+/* x[r, :] += gate * t[r, :] (mod == NULL: gate = 1); `which` = 2 for the attention branch, 5 for the MLP. */
+static void gated_add(int R, int d, const real *mod, const int *seq_of, int which, const real *t, real *x) {
+  for (int r = 0; r < R; ++r) {
+    const real *gate = mod ? mod + ((size_t)seq_of[r] * 6 + which) * d : NULL;
+    for (int i = 0; i < d; ++i) x[(size_t)r * d + i] += (gate ? gate[i] : (real)1) * t[(size_t)r * d + i];
+  }
+}
+
 /* y[t, :] += b for every row (b == NULL: nothing). */
 static void add_bias(int T, int n, const real *b, real *y) {
   if (!b) return;
@@ -244,6 +267,7 @@ int hso_layer(const hso_config_t *c, const hso_layer_t *w, int layer, uint16_t *
   /* 1. attention norm */
   real *h = (real *)malloc(sizeof(real) * (size_t)T * d);
   hso_rmsnorm(T, d, x, w->g_attn, c->rms_eps, h);
+  modulate(T, d, w->mod, tok_seq, 0, h);
   if (g_round_mask & 1)
     for (size_t i = 0; i < (size_t)T * d; ++i) h[i] = round_act(h[i]);
 
@@ -310,11 +334,14 @@ int hso_layer(const hso_config_t *c, const hso_layer_t *w, int layer, uint16_t *
   real *xR = (real *)malloc(sizeof(real) * (size_t)R * d), *tmp = (real *)malloc(sizeof(real) * (size_t)R * d);
   for (int r = 0; r < R; ++r) memcpy(xR + (size_t)r * d, x + (size_t)rows[r] * d, sizeof(real) * (size_t)d);
   hso_linear(R, d, Qd, o, w->w_o, tmp);
-  for (size_t i = 0; i < (size_t)R * d; ++i) xR[i] += tmp[i];
+  int *seqR = (int *)malloc(sizeof(int) * (size_t)(R > 0 ? R : 1));
+  for (int r = 0; r < R; ++r) seqR[r] = tok_seq[rows[r]];
+  gated_add(R, d, w->mod, seqR, 2, tmp, xR);
   free(o);
 
   /* 6. MLP norm, SwiGLU */
   hso_rmsnorm(R, d, xR, w->g_mlp, c->rms_eps, hR);
+  modulate(R, d, w->mod, seqR, 3, hR);
   if (g_round_mask & 1)
     for (size_t i = 0; i < (size_t)R * d; ++i) hR[i] = round_act(hR[i]);
   real *gate = (real *)malloc(sizeof(real) * (size_t)R * F), *up = (real *)malloc(sizeof(real) * (size_t)R * F);
@@ -329,7 +356,8 @@ int hso_layer(const hso_config_t *c, const hso_layer_t *w, int layer, uint16_t *
 
   /* 7. down projection + residual */
   hso_linear(R, d, F, gate, w->w_down, tmp);
-  for (size_t i = 0; i < (size_t)R * d; ++i) xR[i] += tmp[i];
+  gated_add(R, d, w->mod, seqR, 5, tmp, xR);
+  free(seqR);
   free(gate);
   free(tmp);
   for (int r = 0; r < R; ++r) memcpy(x + (size_t)rows[r] * d, xR + (size_t)r * d, sizeof(real) * (size_t)d);

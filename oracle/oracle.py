@@ -50,11 +50,13 @@ class _Cfg(C.Structure):
 
 class _Layer(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in ("g_attn", "w_q", "w_k", "w_v", "w_o", "g_mlp", "w_gate", "w_up",
-                                           "w_down", "b_q", "b_k", "b_v")]
+                                           "w_down", "b_q", "b_k", "b_v", "mod")]
 
 
 WEIGHT_NAMES = ("g_attn", "w_q", "w_k", "w_v", "w_o", "g_mlp", "w_gate", "w_up", "w_down")
-BIAS_NAMES = ("b_q", "b_k", "b_v")      # optional entries of a layer's dict: biases of the q, k, v projections
+# optional entries of a layer's dict: biases of the q, k, v projections; "mod" [n_seqs, 6, d]: per-sequence
+# shift / scale / gate vectors of a conditioned (adaLN-Zero) block for the attention and the MLP branch
+BIAS_NAMES = ("b_q", "b_k", "b_v", "mod")
 
 
 def _load(precision: str) -> C.CDLL:

@@ -234,15 +234,17 @@ def _torch_reference_single_sequence(dims, weights, x, n_layers, causal=True):
 
     for l in range(n_layers):
         w = {k: torch.from_numpy(v).double() for k, v in weights[l].items()}
-        h = F.rms_norm(xt, (dims.d_model,), w["g_attn"], dims.rms_eps)
+        mod = w.get("mod")                                   # [1, 6, d]: one sequence
+        sh_a, sc_a, g_a, sh_m, sc_m, g_m = (mod[0, i] for i in range(6)) if mod is not None else (0, 0, 1, 0, 0, 1)
+        h = F.rms_norm(xt, (dims.d_model,), w["g_attn"], dims.rms_eps) * (1 + sc_a) + sh_a
         q = rope(F.linear(h, w["w_q"], w.get("b_q")).view(n, Hq, Dh))
         k = rope(F.linear(h, w["w_k"], w.get("b_k")).view(n, Hkv, Dh)).bfloat16().double()
         v = F.linear(h, w["w_v"], w.get("b_v")).view(n, Hkv, Dh).bfloat16().double()
         k = k.repeat_interleave(Hq // Hkv, dim=1); v = v.repeat_interleave(Hq // Hkv, dim=1)
         o = F.scaled_dot_product_attention(q.transpose(0, 1), k.transpose(0, 1), v.transpose(0, 1), is_causal=causal)
-        xt = xt + o.transpose(0, 1).reshape(n, Hq * Dh) @ w["w_o"].T
-        h2 = F.rms_norm(xt, (dims.d_model,), w["g_mlp"], dims.rms_eps)
-        xt = xt + (F.silu(h2 @ w["w_gate"].T) * (h2 @ w["w_up"].T)) @ w["w_down"].T
+        xt = xt + g_a * (o.transpose(0, 1).reshape(n, Hq * Dh) @ w["w_o"].T)
+        h2 = F.rms_norm(xt, (dims.d_model,), w["g_mlp"], dims.rms_eps) * (1 + sc_m) + sh_m
+        xt = xt + g_m * ((F.silu(h2 @ w["w_gate"].T) * (h2 @ w["w_up"].T)) @ w["w_down"].T)
     return xt.numpy()
 
 
@@ -349,6 +351,48 @@ def test_bidirectional_attention_matches_library_and_invariants(oracle64):
     o_row = v.mean(dim=0).view(dims.n_kv_heads, dims.head_dim).repeat_interleave(G, dim=0).reshape(-1)
     want0 = xt + (torch.from_numpy(z["w_o"]).double() @ o_row)[None, :]
     assert rel_err(y0, want0.numpy()) < 1e-12
+
+
+def test_modulation_matches_library_composition_and_special_cases(oracle64):
+    """Per-sequence shift / scale / gate vectors of a conditioned block (adaLN-Zero with RMSNorm): against the
+    float64 library composition; scale = shift = 0 with gate = 1 is the plain layer, bit for bit; gate = 0 on both
+    branches returns the input; and two sequences of one batch each follow their own vectors."""
+    dims = wl.StageDims(2, 64, 4, 2, 16, 96)
+    case = make_case(dims, wl.BatchSpec([26], [0]), seed=10)
+    g = np.random.default_rng(10)
+    weights = [{k: (v if k.startswith("g_") else v * 8.0) for k, v in lw.items()} for lw in case.weights]
+    mods = [g.normal(0, 0.5, (1, 6, dims.d_model)) for _ in range(dims.n_layers)]
+    wm = [dict(lw, mod=m) for lw, m in zip(weights, mods)]
+    args = (case.batch.q_len, case.batch.ctx_len, case.block_tables, case.x)
+    y = oracle64.step(case.cfg, wm, case.kv_pool.copy(), *args)
+    want = _torch_reference_single_sequence(dims, wm, case.x, dims.n_layers)
+    assert rel_err(y, want) < 1e-10
+    y_plain = oracle64.step(case.cfg, weights, case.kv_pool.copy(), *args)
+    assert rel_err(y, y_plain) > 0.05
+    ident = np.zeros((1, 6, dims.d_model)); ident[0, 2] = 1.0; ident[0, 5] = 1.0
+    assert np.array_equal(oracle64.step(case.cfg, [dict(lw, mod=ident) for lw in weights], case.kv_pool.copy(), *args),
+                          y_plain)
+    closed = np.array(mods[0]); closed[0, 2] = 0.0; closed[0, 5] = 0.0
+    y0 = oracle64.step(case.cfg, [dict(lw, mod=closed) for lw in weights], case.kv_pool.copy(), *args)
+    assert np.array_equal(y0, case.x.astype(y0.dtype))
+    for drop in range(6):                        # every one of the six vectors matters on its own
+        m2 = [np.array(m) for m in mods]
+        m2[0][0, drop] = 1.0 if drop in (2, 5) else 0.0
+        y2 = oracle64.step(case.cfg, [dict(lw, mod=m) for lw, m in zip(weights, m2)], case.kv_pool.copy(), *args)
+        assert rel_err(y2, y) > 1e-3, drop
+
+    # two sequences in one batch: each equals the single-sequence run with its own vectors
+    one = wl.StageDims(1, 64, 4, 2, 16, 96)
+    both = make_case(one, wl.BatchSpec([13, 21], [0, 0]), seed=12)
+    m_both = g.normal(0, 0.5, (2, 6, one.d_model))
+    w1 = {k: (v if k.startswith("g_") else v * 8.0) for k, v in both.weights[0].items()}
+    y_both = oracle64.step(both.cfg, [dict(w1, mod=m_both)], both.kv_pool.copy(), both.batch.q_len, both.batch.ctx_len,
+                           both.block_tables, both.x)
+    t0 = 0
+    for s_i, n in enumerate([13, 21]):
+        want_s = _torch_reference_single_sequence(one, [dict(w1, mod=m_both[s_i:s_i + 1])], both.x[t0:t0 + n], 1)
+        assert rel_err(y_both[t0:t0 + n], want_s) < 1e-10
+        t0 += n
 
 
 def test_zero_gate_weight_means_mlp_adds_nothing(oracle32):
