@@ -122,6 +122,8 @@ def build_stage(name: str, device: int, init: str = "n002", layers: int = 0, fla
     tables = [stage.kv_alloc(s, t) for s, t in enumerate(batch.total_len())]
     bt = stage.block_table_array(tables)
     x = wl.make_x(batch.n_tokens, dims.d_model, seed, dev)
+    if name in wl.CONDITIONED:
+        stage.set_modulation(wl.make_modulation(dims, batch.n_seqs, seed, dev))
     return stage, dims, batch, bt, x
 
 
@@ -165,6 +167,8 @@ def cpu_oracle_sample(name: str, target_s: float):
     cfg = OracleConfig(1, dims.d_model, dims.n_q_heads, dims.n_kv_heads, dims.head_dim, dims.d_ffn, 16, num_pages,
                        dims.rms_eps, dims.rope_base, bool(wl.STAGE_FLAGS.get(name, 0) & 2))
     w = wl.weights_to_numpy([wl.make_layer_weights(one, seed, 0)])
+    if name in wl.CONDITIONED:
+        w[0]["mod"] = wl.make_modulation(one, batch.n_seqs, seed)[0].numpy()
     pool = wl.bf16_bits_numpy(wl.make_kv_fill(one, num_pages, seed)).reshape(-1).copy()
     x = wl.to_f32_numpy(wl.make_x(batch.n_tokens, dims.d_model, seed))
     orc = Oracle("f32")

@@ -206,6 +206,20 @@ hs_status_t hs_stage_step(hs_stage_t *stage, const hs_batch_t *batch, int32_t sm
  */
 hs_status_t hs_stage_set_qkv_bias(hs_stage_t *stage, int32_t layer, const void *b_q, const void *b_k, const void *b_v);
 
+/*
+ * Optional per-sequence modulation of a conditioned block (the adaLN-Zero block of diffusion transformers, with
+ * this stage's RMSNorm; the paper names such generators as downstream stages, Sec. 2.1, and gives no arithmetic).
+ *   mod  device fp32 [n_layers][max_seqs][6][d_model], 16-byte aligned, borrowed until replaced or the stage is
+ *        destroyed; NULL switches the modulation off (the state of a new stage).
+ * Rows 0..5 of (layer, sequence s) are shift_a, scale_a, gate_a, shift_m, scale_m, gate_m, and the layer computes
+ *   h_a = rmsnorm(x) g_attn (1 + scale_a) + shift_a,   x += gate_a * (attention output W_o^T),
+ *   h_m = rmsnorm(x) g_mlp  (1 + scale_m) + shift_m,   x += gate_m * (MLP output),
+ * element-wise over d_model, where s is the index of the token's sequence in the step's batch.  The vectors are
+ * read when a step runs, so they may be rewritten between steps (a new timestep) without another call.
+ * Errors: INVALID_ARG (NULL stage, misaligned pointer), NO_DEVICE.
+ */
+hs_status_t hs_stage_set_modulation(hs_stage_t *stage, const void *mod);
+
 /* Device-side status of the steps run so far (HS_OK or HS_ERR_TIMEOUT); call after synchronising the stream. */
 hs_status_t hs_stage_status(hs_stage_t *stage);
 

@@ -28,7 +28,7 @@ EXPORTS = ("hs_status_str", "hs_kv_pool_bytes", "hs_workspace_bytes", "hs_stage_
            "hs_spatial_create", "hs_spatial_update", "hs_spatial_state", "hs_spatial_destroy",
            "hs_spatial_derive_cap", "hs_head_workspace_bytes", "hs_head_create", "hs_head_step", "hs_head_status",
            "hs_head_destroy", "hs_op_embed", "hs_temporal_create", "hs_temporal_step", "hs_temporal_destroy",
-           "hs_stage_set_qkv_bias")
+           "hs_stage_set_qkv_bias", "hs_stage_set_modulation")
 PROFILE_CLASSES = ("rmsnorm", "gemm_qkv", "attn_prefill", "attn_decode", "attn_combine", "gemm_out", "gemm_gateup",
                    "gemm_down")
 
@@ -141,6 +141,7 @@ def lib() -> C.CDLL:
             [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p]
         l.hs_stage_profile_enable.argtypes = [C.c_void_p, C.c_int32]
         l.hs_stage_set_qkv_bias.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+        l.hs_stage_set_modulation.argtypes = [C.c_void_p, C.c_void_p]
         l.hs_stage_profile_read.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = l
     return _lib
@@ -267,6 +268,13 @@ def hs_stage_set_qkv_bias(stage: int, layer: int, b_q: int, b_k: int, b_v: int) 
                                      C.c_void_p(b_v or None))
     if st != HS_OK:
         raise HsError(st, "hs_stage_set_qkv_bias")
+
+
+def hs_stage_set_modulation(stage: int, mod: int) -> None:
+    """Device pointer (0 = off) of the fp32 [n_layers, max_seqs, 6, d_model] shift / scale / gate vectors."""
+    st = lib().hs_stage_set_modulation(C.c_void_p(stage), C.c_void_p(mod or None))
+    if st != HS_OK:
+        raise HsError(st, "hs_stage_set_modulation")
 
 
 def hs_stage_profile_enable(stage: int, enable: bool) -> None:

@@ -165,6 +165,7 @@ struct hs_stage {
   std::vector<hs_layer_weights_t> layers;
   struct QkvBias { const __nv_bfloat16* b[3] = {nullptr, nullptr, nullptr}; };
   std::vector<QkvBias> qkv_bias;              // per layer, optional (hs_stage_set_qkv_bias)
+  const float* modulation = nullptr;          // optional [n_layers][max_seqs][6][d_model] (hs_stage_set_modulation)
   std::vector<hs_layer_weights_t> operands;   // what the projections read: the fp16 copies, or `layers` itself
   std::vector<LayerMaps> maps;
   CUtensorMap tm_h, tm_o, tm_act, tm_kv;   // operand loads
@@ -490,6 +491,10 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     np.status = status;
     np.overlap = overlap;
     np.smid_log = slots(0);
+    const float* mod_l = s->modulation ? s->modulation + size_t(l) * c.max_seqs * 6 * d : nullptr;
+    np.mod = mod_l;
+    np.tok_seq = meta + s->ml.tok_seq;
+    np.mod_which = 0;
     { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
@@ -565,6 +570,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     go.ab_f16 = f16;
     go.overlap = overlap;
     go.tm_out = tm_y; go.accumulate = 1;
+    go.gate_mod = mod_l; go.tok_seq = meta + s->ml.tok_seq; go.gate_which = 2;
     go.pair = use_pair;
     go.bn = use_pair ? 256 : gemm_pick_bn(T, d, s->sm_count);
     go.ksplit = use_pair ? 1 : pick_ksplit(T, d, q_dim, go.bn, s->sm_count);
@@ -574,6 +580,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     if (skinny(q_dim, d, kGemmResid)) {
       SkinnyParams k = skinny_base(o, q_dim, d, kGemmResid);
       k.w[0] = wo.w_o; k.y = x; k.accumulate = 1;
+      k.gate_mod = go.gate_mod; k.tok_seq = go.tok_seq; k.gate_which = 2;
       k.smid_log = slots(5);
       LaunchTimer t(s, 5, stream); where = "out-proj gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
     } else { LaunchTimer t(s, 5, stream); where = "out-proj gemm"; e = launch_gemm(go, sm_budget, stream); }
@@ -581,6 +588,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
 
     np.x_bf16 = nullptr;
     np.gain = static_cast<const __nv_bfloat16*>(w.g_mlp);
+    np.mod_which = 3;
     { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
@@ -615,6 +623,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gd.ab_f16 = f16;
     gd.overlap = overlap;
     gd.tm_out = tm_y; gd.accumulate = 1;
+    gd.gate_mod = mod_l; gd.tok_seq = meta + s->ml.tok_seq; gd.gate_which = 5;
     gd.pair = use_pair;
     gd.bn = use_pair ? 256 : gemm_pick_bn(T, d, s->sm_count);
     gd.ksplit = use_pair ? 1 : pick_ksplit(T, d, F, gd.bn, s->sm_count);
@@ -624,6 +633,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     if (skinny(F, d, kGemmResid)) {
       SkinnyParams k = skinny_base(s->ws_dev + s->ws.act, F, d, kGemmResid);
       k.w[0] = wo.w_down; k.y = x; k.accumulate = 1;
+      k.gate_mod = gd.gate_mod; k.tok_seq = gd.tok_seq; k.gate_which = 5;
       k.smid_log = slots(7);
       LaunchTimer t(s, 7, stream); where = "down gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
     } else { LaunchTimer t(s, 7, stream); where = "down gemm"; e = launch_gemm(gd, sm_budget, stream); }
@@ -639,6 +649,13 @@ hs_status_t hs_stage_set_qkv_bias(hs_stage_t* s, int32_t layer, const void* b_q,
   for (const void* ptr : b)
     if (reinterpret_cast<uintptr_t>(ptr) & 15) return HS_ERR_INVALID_ARG;
   for (int i = 0; i < 3; ++i) s->qkv_bias[layer].b[i] = static_cast<const __nv_bfloat16*>(b[i]);
+  return HS_OK;
+}
+
+hs_status_t hs_stage_set_modulation(hs_stage_t* s, const void* mod) {
+  if (!s || (reinterpret_cast<uintptr_t>(mod) & 15)) return HS_ERR_INVALID_ARG;
+  if (s->cfg.device < 0) return HS_ERR_NO_DEVICE;
+  s->modulation = static_cast<const float*>(mod);
   return HS_OK;
 }
 

@@ -344,11 +344,32 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
           if (!__shfl_sync(0xffffffffu, go, 0)) break;
         }
         const bool add = p.accumulate || ks > 0;
+        // conditioned block: the product is scaled by the gate vector of the row's sequence before it is added
+        const float* gate = p.gate_mod && row_ok ? p.gate_mod + (size_t(p.tok_seq[row]) * 6 + p.gate_which) * p.N : nullptr;
+        if (gate) {   // pull this tile's part of the gate vector into the L1 before the chunk loop needs it
+          const int chunk = lane % (p.bn / 32), col = n * p.bn + chunk * 32;
+          if (col < p.N) asm volatile("prefetch.global.L1 [%0];" ::"l"(gate + col));
+        }
         for (int c = 0; c < p.bn / 32; ++c) {
           const int col0 = n * p.bn + c * 32;
           if (col0 >= p.N) break;
           tmem_ld32(taddr + c * 32, r0);
+          float4 gv[8];
+          const int nv = p.N - col0 >= 32 ? 8 : (p.N - col0) >> 2;          // float4s of the chunk inside the row
+          if (gate) {                              // requested while the accumulator chunk is on its way
+#pragma unroll
+            for (int e = 0; e < 8; ++e) gv[e] = e < nv ? __ldg(reinterpret_cast<const float4*>(gate + col0) + e) : make_float4(1.f, 1.f, 1.f, 1.f);
+          }
           tmem_ld_wait();
+          if (gate) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              r0[4 * e] = __float_as_uint(__uint_as_float(r0[4 * e]) * gv[e].x);
+              r0[4 * e + 1] = __float_as_uint(__uint_as_float(r0[4 * e + 1]) * gv[e].y);
+              r0[4 * e + 2] = __float_as_uint(__uint_as_float(r0[4 * e + 2]) * gv[e].z);
+              r0[4 * e + 3] = __float_as_uint(__uint_as_float(r0[4 * e + 3]) * gv[e].w);
+            }
+          }
           if (lane == 0) bulk_wait_read<1>();     // the block staged two chunks ago has been read
           __syncwarp();
           uint8_t* buf = epi_buf + epi_sel * EPI_BUF_BYTES;

@@ -231,6 +231,13 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
       if (p.mode == kGemmResid) {
         float4* y_lo = reinterpret_cast<float4*>(p.y + size_t(row) * p.N + unit * 32 + jq);
         float4* y_hi = y_lo + 4;
+        if (p.gate_mod) {                                    // conditioned block: gate vector of the row's sequence
+          const float4* gate = reinterpret_cast<const float4*>(p.gate_mod + (size_t(p.tok_seq[row]) * 6 + p.gate_which) * p.N +
+                                                               unit * 32 + jq);
+          const float4 g_lo = __ldg(gate), g_hi = __ldg(gate + 4);
+          lo.x *= g_lo.x; lo.y *= g_lo.y; lo.z *= g_lo.z; lo.w *= g_lo.w;
+          hi.x *= g_hi.x; hi.y *= g_hi.y; hi.z *= g_hi.z; hi.w *= g_hi.w;
+        }
         if (p.accumulate) {
           const float4 a = *y_lo, b = *y_hi;
           lo.x += a.x; lo.y += a.y; lo.z += a.z; lo.w += a.w;

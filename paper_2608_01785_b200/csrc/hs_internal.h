@@ -47,7 +47,7 @@ class PageAllocator {
 // Offsets (in int32 units) of the arrays inside the per-step metadata block that is copied to the
 // device once per step.  Fixed at stage creation from the configuration's maxima.
 struct MetaLayout {
-  int tok_pos, tok_slot;             // [max_tokens]      absolute position / cache slot of each new token
+  int tok_pos, tok_slot, tok_seq;    // [max_tokens]      absolute position / cache slot / sequence index of each new token
   int seq_tok0, seq_ctx, seq_qlen;   // [max_seqs]        first token row, cached tokens, new tokens
   int block_tables;                  // [max_seqs * max_pages_per_seq]
   int prefill_items;                 // [max_prefill_items * 4]  {seq, kv_head, first token of the tile, tokens}

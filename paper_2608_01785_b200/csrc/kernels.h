@@ -49,6 +49,11 @@ struct GemmParams {
   const int32_t* tok_slot;   // [M]
   const float2* rope;        // [max_position][Dh/2] (cos, sin)
   const __nv_bfloat16* qkv_bias[3];   // optional biases of the q, k, v projections ([q_dim], [kv_dim], [kv_dim]); null = none
+  // Resid, optional: out += gate * (A W^T) with the gate vector of the row's sequence: gate_mod is this layer's
+  // fp32 [max_seqs][6][N], gate_which the row of the gate vector (2 or 5), tok_seq the sequence of every row
+  const float* gate_mod;
+  const int32_t* tok_seq;
+  int gate_which;
   // GateUp
   CUtensorMap tm_act;        // bf16 act [M, N], box 64 x 32, 128-byte swizzle
   int* status;               // device status word
@@ -77,6 +82,9 @@ struct SkinnyParams {
   const int32_t* tok_slot;
   const float2* rope;
   const __nv_bfloat16* qkv_bias[3];   // optional, as in GemmParams
+  const float* gate_mod;     // Resid, optional, as in GemmParams
+  const int32_t* tok_seq;
+  int gate_which;
   __nv_bfloat16* act;        // GateUp: 16-bit [T, N]
   int act_f16;
   int* smid_log;
@@ -101,6 +109,12 @@ struct NormParams {
   int T, d;
   float eps;
   const int* row_index;      // nullable: input row of output row t is row_index[t] (device int32 [T]); else t
+  // optional modulation of a conditioned block: h = rmsnorm(x) g (1 + scale) + shift with the vectors of the
+  // row's sequence; mod is this layer's fp32 [max_seqs][6][d], mod_which the row of the shift vector (0 or 3,
+  // the scale follows it), tok_seq the sequence of every row.  mod null = none.
+  const float* mod;
+  const int32_t* tok_seq;
+  int mod_which;
   int h_f16;                 // 1 = write h as fp16, 0 = bf16
   int overlap;               // 1: launch so that the set-up overlaps the previous kernel's drain
   int* status;               // device status word (bounded waits report HS_ERR_TIMEOUT here)

@@ -91,6 +91,8 @@ __global__ void __launch_bounds__(NORM_THREADS, 1) rmsnorm_kernel(const NormPara
     ss = warp_sum(ss);
     const float r = rsqrtf(ss / float(p.d) + p.eps);
     uint4* hdst = reinterpret_cast<uint4*>(p.h + size_t(row) * p.d);
+    // shift vector of the row's sequence (the scale vector follows it), or null
+    const float* shift = p.mod ? p.mod + (size_t(p.tok_seq[row]) * 6 + p.mod_which) * p.d : nullptr;
     for (int i = lane; i < d8; i += 32) {
       float4 a, b;
       if (i < cached8) {                            // written by this same lane above
@@ -108,8 +110,18 @@ __global__ void __launch_bounds__(NORM_THREADS, 1) rmsnorm_kernel(const NormPara
       float g[8];
       unpack8(gsrc[i], g);
       const bool f16 = p.h_f16 != 0;
-      hdst[i] = make_uint4(pack_act(a.x * r * g[0], a.y * r * g[1], f16), pack_act(a.z * r * g[2], a.w * r * g[3], f16),
-                           pack_act(b.x * r * g[4], b.y * r * g[5], f16), pack_act(b.z * r * g[6], b.w * r * g[7], f16));
+      float v[8] = {a.x * r * g[0], a.y * r * g[1], a.z * r * g[2], a.w * r * g[3],
+                    b.x * r * g[4], b.y * r * g[5], b.z * r * g[6], b.w * r * g[7]};
+      if (shift) {                                   // conditioned block: (1 + scale) and shift of the row's sequence
+        const float4 s0 = reinterpret_cast<const float4*>(shift)[2 * i], s1 = reinterpret_cast<const float4*>(shift)[2 * i + 1];
+        const float4 c0 = reinterpret_cast<const float4*>(shift + p.d)[2 * i], c1 = reinterpret_cast<const float4*>(shift + p.d)[2 * i + 1];
+        const float sh[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+        const float sc[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = fmaf(v[e], 1.f + sc[e], sh[e]);
+      }
+      hdst[i] = make_uint4(pack_act(v[0], v[1], f16), pack_act(v[2], v[3], f16), pack_act(v[4], v[5], f16),
+                           pack_act(v[6], v[7], f16));
     }
   }
 }
@@ -170,6 +182,12 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32, 1) rmsnorm_bulk_kernel(co
   bool ok = true;
   int k = 0;
   for (int row = first; row < p.T; row += stride, ++k) {
+    if (p.mod) {
+      // conditioned block: pull the row's shift and scale vectors (2 d floats, one after the other) into the L1
+      // while the row itself is still on its way, so that the write pass below does not wait on the L2
+      const char* v = reinterpret_cast<const char*>(p.mod + (size_t(p.tok_seq[row]) * 6 + p.mod_which) * p.d);
+      for (int off = lane * 128; off < 2 * p.d * 4; off += 32 * 128) asm volatile("prefetch.global.L1 [%0];" ::"l"(v + off));
+    }
     ok = mbar_wait(&full[k & 1], (k >> 1) & 1, abort_flag, p.status);
     if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
     const uint8_t* buf = bufs + (k & 1) * buf_bytes;
@@ -197,6 +215,8 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32, 1) rmsnorm_bulk_kernel(co
     const float ss = warp_sum((s4[0] + s4[1]) + (s4[2] + s4[3]));
     const float r = rsqrtf(ss / float(p.d) + p.eps);
     uint2* hdst = reinterpret_cast<uint2*>(p.h + size_t(row) * p.d);
+    // shift vector of the row's sequence (the scale vector follows it), or null
+    const float* shift = p.mod ? p.mod + (size_t(p.tok_seq[row]) * 6 + p.mod_which) * p.d : nullptr;
     float4* xo = reinterpret_cast<float4*>(p.x_f32_out + size_t(row) * p.d);
     for (int i0 = lane; i0 < d4; i0 += 128) {
       float4 a[4];
@@ -215,8 +235,13 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32, 1) rmsnorm_bulk_kernel(co
         if (i < d4) {
           const float g0 = __uint_as_float(gw[u].x << 16), g1 = __uint_as_float(gw[u].x & 0xffff0000u);
           const float g2 = __uint_as_float(gw[u].y << 16), g3 = __uint_as_float(gw[u].y & 0xffff0000u);
-          hdst[i] = make_uint2(pack_act(a[u].x * r * g0, a[u].y * r * g1, f16),
-                               pack_act(a[u].z * r * g2, a[u].w * r * g3, f16));
+          float4 v = make_float4(a[u].x * r * g0, a[u].y * r * g1, a[u].z * r * g2, a[u].w * r * g3);
+          if (shift) {                               // conditioned block: (1 + scale) and shift of the row's sequence
+            const float4 sh = reinterpret_cast<const float4*>(shift)[i], sc = reinterpret_cast<const float4*>(shift + p.d)[i];
+            v = make_float4(fmaf(v.x, 1.f + sc.x, sh.x), fmaf(v.y, 1.f + sc.y, sh.y), fmaf(v.z, 1.f + sc.z, sh.z),
+                            fmaf(v.w, 1.f + sc.w, sh.w));
+          }
+          hdst[i] = make_uint2(pack_act(v.x, v.y, f16), pack_act(v.z, v.w, f16));
           if (in_bf16) xo[i] = a[u];                          // the widened copy that starts the residual stream
         }
       }

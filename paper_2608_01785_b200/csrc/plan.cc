@@ -72,6 +72,7 @@ MetaLayout make_meta_layout(const hs_stage_config_t& c) {
   };
   m.tok_pos = take(c.max_tokens);
   m.tok_slot = take(c.max_tokens);
+  m.tok_seq = take(c.max_tokens);
   m.seq_tok0 = take(c.max_seqs);
   m.seq_ctx = take(c.max_seqs);
   m.seq_qlen = take(c.max_seqs);
@@ -160,6 +161,7 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
       if (meta) {
         meta[ml.tok_pos + t + j] = pos;
         meta[ml.tok_slot + t + j] = slot;
+        meta[ml.tok_seq + t + j] = s;
       }
       if (tok_seq) tok_seq[t + j] = s;
     }

@@ -66,6 +66,14 @@ class Stage:
     def status(self) -> int:
         return B.hs_stage_status(self.handle)
 
+    def set_modulation(self, mod) -> None:
+        """fp32 device tensor [n_layers, max_seqs, 6, d_model] (or None): per-sequence shift / scale / gate vectors
+        of a conditioned block; kept alive here, read at every step."""
+        assert mod is None or (mod.dtype == torch.float32 and mod.is_cuda and mod.is_contiguous() and
+                               tuple(mod.shape) == (self.cfg.n_layers, self.cfg.max_seqs, 6, self.cfg.d_model))
+        self._mod = mod
+        B.hs_stage_set_modulation(self.handle, 0 if mod is None else mod.data_ptr())
+
     def set_qkv_bias(self, layer: int, b_q=None, b_k=None, b_v=None) -> None:
         """bf16 device tensors (or None) added to the layer's q, k, v projections before RoPE; kept alive here."""
         for t in (b_q, b_k, b_v):

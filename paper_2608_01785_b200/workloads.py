@@ -23,7 +23,7 @@ import numpy as np
 import torch
 
 WEIGHT_NAMES = ("g_attn", "w_q", "w_k", "w_v", "w_o", "g_mlp", "w_gate", "w_up", "w_down")
-_STREAM = {"weights": 1, "x": 2, "lengths": 3, "kv": 4, "trace": 5, "policy": 6}
+_STREAM = {"weights": 1, "x": 2, "lengths": 3, "kv": 4, "trace": 5, "policy": 6, "modulation": 7}
 
 
 @dataclass(frozen=True)
@@ -64,9 +64,11 @@ DIMS = {
 }
 DIMS["c3_decode"] = DIMS["c3_7b"]
 # A denoising-style (DiT-like) downstream stage, the visual generator kind of the paper's Sec. 2.1: the talker's
-# width and depth with multi-head attention and no causal mask; a step denoises 4 images of 256 latent tokens.
+# width and depth with multi-head attention, no causal mask and per-image shift / scale / gate conditioning; a step
+# denoises 4 images of 256 latent tokens.
 DIMS["c6_dit"] = StageDims(12, 1024, 16, 16, 64, 2816)
 STAGE_FLAGS = {"c6_dit": 2}      # hs_stage_config_t.flags by workload (2 = no causal mask)
+CONDITIONED = {"c6_dit"}         # workloads whose stage runs with per-sequence shift / scale / gate vectors
 SM_BUDGETS = {
     "c1_tiny": (148, 8),
     "c2_shared": (148, 112, 74, 37),
@@ -157,6 +159,19 @@ def make_x(n_tokens: int, d_model: int, seed: int, device="cpu", index: int = 0)
     gen = torch.Generator(device=device)
     gen.manual_seed(_subseed(seed, "x", index))
     return _normal_bf16((n_tokens, d_model), 1.0, 0.0, gen, device)
+
+
+def make_modulation(dims: StageDims, n_seqs: int, seed: int, device="cpu") -> torch.Tensor:
+    """Shift / scale / gate vectors of a conditioned block, fp32 [n_layers, n_seqs, 6, d_model]: shift and scale
+    ~ N(0, 0.1), gates ~ N(1, 0.1) (the magnitudes of a trained conditioning path are not public; these keep the
+    residual stream's scale)."""
+    gen = torch.Generator(device=device)
+    gen.manual_seed(_subseed(seed, "modulation", 0))
+    m = torch.empty((dims.n_layers, n_seqs, 6, dims.d_model), dtype=torch.float32, device=device)
+    m.normal_(0.0, 0.1, generator=gen)
+    m[:, :, 2] += 1.0
+    m[:, :, 5] += 1.0
+    return m
 
 
 def kv_pool_shape(dims: StageDims, num_pages: int) -> Tuple[int, ...]:

@@ -222,8 +222,9 @@ def test_config3_budget_sweep_and_sampled_layer_local(orc, init):
 
 # ------------------------------------------------- denoising-style stage (no causal mask) --
 def test_denoising_stage_budget_sweep_and_two_layer_parity(orc):
-    """The c6_dit workload (4 images x 256 latent tokens, multi-head attention without a mask): the 12-layer
-    step bit for bit over budgets, and its first two layers end to end against the oracle."""
+    """The c6_dit workload (4 images x 256 latent tokens, multi-head attention without a mask, per-image shift /
+    scale / gate vectors): the 12-layer step bit for bit over budgets, and its first two layers end to end
+    against the oracle."""
     import dataclasses
     stage, dims, batch, bt, x = bench.build_stage("c6_dit", 0)
     try:
@@ -240,9 +241,14 @@ def test_denoising_stage_budget_sweep_and_two_layer_parity(orc):
         pool0 = stage2.kv_pool.clone()
         y_gpu = gpu_step(stage2, batch, bt, x, stage2.sm_count, pool0).cpu().numpy()
         cfg = dataclasses.replace(ocfg(dims2, 2, stage2.cfg.num_pages), bidirectional=True)
-        y_ref = orc.step(cfg, wl.weights_to_numpy(stage2.weights), wl.bf16_bits_numpy(pool0).reshape(-1).copy(),
+        mod = stage2._mod.cpu().numpy()                       # the conditioning vectors the bench runs with
+        w_np = [dict(lw, mod=mod[l]) for l, lw in enumerate(wl.weights_to_numpy(stage2.weights))]
+        y_ref = orc.step(cfg, w_np, wl.bf16_bits_numpy(pool0).reshape(-1).copy(),
                          batch.q_len, batch.ctx_len, bt, wl.to_f32_numpy(x))
         err = rel_err(y_gpu, y_ref)
+        y_uncond = orc.step(cfg, wl.weights_to_numpy(stage2.weights), wl.bf16_bits_numpy(pool0).reshape(-1).copy(),
+                            batch.q_len, batch.ctx_len, bt, wl.to_f32_numpy(x))
+        assert rel_err(y_uncond, y_ref) > 5 * TOL             # the conditioning is visible
         print(f"denoising-style stage, 2 layers end to end: max|err|/RMS = {err:.2e}")
         assert err <= TOL
     finally:

@@ -335,6 +335,49 @@ def test_bidirectional_attention_matches_oracle(orc, name):
     assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
 
 
+MOD_CASES = {
+    # name: (dims, q_len, ctx_len, flags)
+    "pair_tiles_bidirectional": (wl.StageDims(2, 256, 4, 4, 64, 688), [150, 60, 9], [0, 0, 0], B.HS_FLAG_BIDIRECTIONAL),
+    "single_tile_causal": (wl.StageDims(1, 256, 2, 2, 128, 512), [70, 1, 33], [0, 200, 5], 0),
+    "streaming_kernel_16_rows": (wl.StageDims(2, 1024, 16, 4, 64, 2816), [1] * 16, [128 + 57 * i for i in range(16)], 0),
+    "streaming_kernel_22_rows": (wl.StageDims(1, 2048, 8, 2, 128, 1024), [20, 1, 1], [0, 300, 17], 0),
+    "wide_rows_d8192": (wl.StageDims(1, 8192, 2, 2, 64, 128), [20, 1], [0, 37], 0),
+}
+
+
+@pytest.mark.parametrize("name", sorted(MOD_CASES))
+def test_modulation_matches_oracle(orc, name):
+    """Per-sequence shift / scale / gate vectors (hs_stage_set_modulation) through both RMSNorm kernels and every
+    variant of the residual GEMM epilogue; switching the modulation off again restores the plain step."""
+    import dataclasses
+    dims, q_len, ctx_len, flags = MOD_CASES[name]
+    batch = wl.BatchSpec(list(q_len), list(ctx_len))
+    case = make_case(dims, batch, seed=41, kv_fill=True)
+    cfg = dataclasses.replace(case.cfg, bidirectional=bool(flags & B.HS_FLAG_BIDIRECTIONAL))
+    g = torch.Generator().manual_seed(99)
+    mod = torch.randn(dims.n_layers, batch.n_seqs, 6, dims.d_model, generator=g) * 0.5
+    weights = [dict(lw, mod=mod[l].numpy()) for l, lw in enumerate(case.weights)]
+    y_ref = orc.step(cfg, weights, case.kv_pool.copy(), batch.q_len, batch.ctx_len, case.block_tables, case.x)
+    y_plain = orc.step(cfg, case.weights, case.kv_pool.copy(), batch.q_len, batch.ctx_len, case.block_tables, case.x)
+    assert rel_err(y_plain, y_ref) > 5 * TOL
+    outs = []
+    for budget in (148, 5):
+        st = make_stage(case, flags=flags)
+        st.set_modulation(mod.to(st.device).contiguous())
+        y, pool = run_step(st, case, budget)
+        err = rel_err(y, y_ref)
+        print(f"{name}, sm_budget {budget}: max|err|/RMS = {err:.2e}")
+        assert err <= TOL
+        outs.append((y, pool))
+        if budget == 148:
+            st.kv_pool.copy_(wl.bits_to_bf16_tensor(case.kv_pool, st.device))
+            st.set_modulation(None)
+            y_off, _ = run_step(st, case, budget)
+            assert rel_err(y_off, y_plain) <= TOL
+        st.close()
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+
+
 def test_qkv_bias_argument_errors(orc):
     case = config1_case(orc)
     st = make_stage(case)
