@@ -142,6 +142,8 @@ __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, u
                : "memory");
 }
 
+// MOD: the conditioned form (shift / scale vectors per sequence); the plain form carries none of its code.
+template <bool MOD>
 __global__ void __launch_bounds__(BULK_MAX_WARPS * 32, 1) rmsnorm_bulk_kernel(const NormParams p) {
   extern __shared__ __align__(128) uint8_t bulk_smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
@@ -182,7 +184,7 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32, 1) rmsnorm_bulk_kernel(co
   bool ok = true;
   int k = 0;
   for (int row = first; row < p.T; row += stride, ++k) {
-    if (p.mod) {
+    if (MOD) {
       // conditioned block: pull the row's shift and scale vectors (2 d floats, one after the other) into the L1
       // while the row itself is still on its way, so that the write pass below does not wait on the L2
       const char* v = reinterpret_cast<const char*>(p.mod + (size_t(p.tok_seq[row]) * 6 + p.mod_which) * p.d);
@@ -216,7 +218,7 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32, 1) rmsnorm_bulk_kernel(co
     const float r = rsqrtf(ss / float(p.d) + p.eps);
     uint2* hdst = reinterpret_cast<uint2*>(p.h + size_t(row) * p.d);
     // shift vector of the row's sequence (the scale vector follows it), or null
-    const float* shift = p.mod ? p.mod + (size_t(p.tok_seq[row]) * 6 + p.mod_which) * p.d : nullptr;
+    const float* shift = MOD ? p.mod + (size_t(p.tok_seq[row]) * 6 + p.mod_which) * p.d : nullptr;
     float4* xo = reinterpret_cast<float4*>(p.x_f32_out + size_t(row) * p.d);
     for (int i0 = lane; i0 < d4; i0 += 128) {
       float4 a[4];
@@ -236,7 +238,7 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32, 1) rmsnorm_bulk_kernel(co
           const float g0 = __uint_as_float(gw[u].x << 16), g1 = __uint_as_float(gw[u].x & 0xffff0000u);
           const float g2 = __uint_as_float(gw[u].y << 16), g3 = __uint_as_float(gw[u].y & 0xffff0000u);
           float4 v = make_float4(a[u].x * r * g0, a[u].y * r * g1, a[u].z * r * g2, a[u].w * r * g3);
-          if (shift) {                               // conditioned block: (1 + scale) and shift of the row's sequence
+          if (MOD) {                                 // conditioned block: (1 + scale) and shift of the row's sequence
             const float4 sh = reinterpret_cast<const float4*>(shift)[i], sc = reinterpret_cast<const float4*>(shift + p.d)[i];
             v = make_float4(fmaf(v.x, 1.f + sc.x, sh.x), fmaf(v.y, 1.f + sc.y, sh.y), fmaf(v.z, 1.f + sc.z, sh.z),
                             fmaf(v.w, 1.f + sc.w, sh.w));
@@ -278,7 +280,8 @@ cudaError_t launch_bf16_to_f16(const void* src, void* dst, size_t n, cudaStream_
 cudaError_t norm_set_attributes() {
   cudaError_t e = set_kernel_smem(rmsnorm_kernel, NORM_SMEM);
   if (e != cudaSuccess) return e;
-  return set_kernel_smem(rmsnorm_bulk_kernel, 512 + BULK_SMEM_BUDGET);
+  if ((e = set_kernel_smem(rmsnorm_bulk_kernel<false>, 512 + BULK_SMEM_BUDGET)) != cudaSuccess) return e;
+  return set_kernel_smem(rmsnorm_bulk_kernel<true>, 512 + BULK_SMEM_BUDGET);
 }
 
 cudaError_t launch_rmsnorm(const NormParams& p, int sm_budget, cudaStream_t stream) {
@@ -292,8 +295,9 @@ cudaError_t launch_rmsnorm(const NormParams& p, int sm_budget, cudaStream_t stre
     const int blocks = (p.T + warps - 1) / warps;
     const int grid = blocks < sm_budget ? blocks : sm_budget;
     const size_t smem = 512 + size_t(warps) * pair_bytes + gain_bytes;
-    return launch_step_kernel(rmsnorm_bulk_kernel, grid, warps * 32,
-                              smem < size_t(kMinSmemBytes) ? size_t(kMinSmemBytes) : smem, stream, p.overlap != 0, p);
+    const size_t bytes = smem < size_t(kMinSmemBytes) ? size_t(kMinSmemBytes) : smem;
+    if (p.mod) return launch_step_kernel(rmsnorm_bulk_kernel<true>, grid, warps * 32, bytes, stream, p.overlap != 0, p);
+    return launch_step_kernel(rmsnorm_bulk_kernel<false>, grid, warps * 32, bytes, stream, p.overlap != 0, p);
   }
   const int blocks = (p.T + NORM_WARPS - 1) / NORM_WARPS;
   const int grid = blocks < sm_budget ? blocks : sm_budget;
