@@ -12,6 +12,10 @@ read -- weights once per step, the KV pages of every sequence -- divided by the 
 GPU's measured copy bandwidth).  Time is virtual: the clock advances by the
 measured latency of each tick and idle gaps are skipped, so a long trace replays in GPU time only.
 
+With `image_stage = "dit"` the image class's downstream stage is a third stage, the conditioned denoising
+stage without a causal mask (workload c6_dit): an image runs `dit_steps` steps over its `dit_tokens` latent
+tokens, at most `max_dit` images per step, each step behind the talker's on the downstream stream.
+
 The engine is pluggable: `GpuEngine` drives real stages through the C ABI; `ModelEngine` is a latency
 model used by the CPU tests of the scheduling logic (it runs the same page accounting on host-only
 stages, so allocator pressure is exercised without a GPU).
@@ -52,6 +56,13 @@ class ReplayConfig:
     est_fixed_ms: float = 8.0       # coarse remaining-time estimate: fixed part (one tick) ...
     est_per_token_ms: float = 0.014 # ... + per prompt token still to prefill ...
     est_down_ms: float = 8.0        # ... + one more tick for the first downstream step of a long-path request
+    # downstream stage of the image class: "talker" (talker-shaped steps, the stand-in) or "dit": a conditioned
+    # denoising stage without a causal mask that runs dit_steps steps over dit_tokens latent tokens per image,
+    # at most max_dit images per step, after the talker's step on the downstream stream
+    image_stage: str = "talker"
+    dit_steps: int = 20
+    dit_tokens: int = 256
+    max_dit: int = 4
 
 
 @dataclass
@@ -60,16 +71,18 @@ class _Seq:
     prefilled: int = 0              # prompt tokens already in the cache
     decoded: int = 0                # backbone tokens generated
     talker_done: int = 0
+    dit_done: int = 0
     t_first: Optional[float] = None       # first backbone token (end of the tick that finished prefill)
     t_first_down: Optional[float] = None  # first downstream token
     t_done: Optional[float] = None
 
 
 class Engine:
-    """Runs one tick; returns (backbone ms or None, talker ms or None)."""
+    """Runs one tick; returns (backbone ms, talker ms, denoising-stage ms), None where a stage had no batch."""
     sm_count = 148
+    dims_c = None
 
-    def tick(self, a_batch, b_batch, budget_a: int) -> Tuple[Optional[float], Optional[float]]:
+    def tick(self, a_batch, b_batch, budget_a: int, c_batch=None):
         raise NotImplementedError
 
     def alloc(self, which: str, seq_id: int, total: int) -> None:
@@ -82,10 +95,14 @@ class Engine:
 class ModelEngine(Engine):
     """Latency model + real page accounting on host-only stages (no GPU)."""
 
-    def __init__(self, dims_a, dims_b, pages_a: int, pages_b: int, mpps_a: int, mpps_b: int):
-        self.dims_a, self.dims_b = dims_a, dims_b
+    def __init__(self, dims_a, dims_b, pages_a: int, pages_b: int, mpps_a: int, mpps_b: int, dims_c=None,
+                 pages_c: int = 0, mpps_c: int = 0):
+        self.dims_a, self.dims_b, self.dims_c = dims_a, dims_b, dims_c
         self.h = {}
-        for name, dims, pages, mpps in (("a", dims_a, pages_a, mpps_a), ("b", dims_b, pages_b, mpps_b)):
+        stages = [("a", dims_a, pages_a, mpps_a), ("b", dims_b, pages_b, mpps_b)]
+        if dims_c is not None:
+            stages.append(("c", dims_c, pages_c, mpps_c))
+        for name, dims, pages, mpps in stages:
             cfg = B.make_config(dims, pages, 4096, 128, mpps, mpps * 16, device=-1)
             self.h[name] = (B.hs_stage_create(cfg, None, 0, 0), mpps)
 
@@ -99,14 +116,16 @@ class ModelEngine(Engine):
     def free_pages(self, which):
         return B.hs_kv_free_pages(self.h[which][0])
 
-    def tick(self, a_batch, b_batch, budget_a):
-        la = lb = None
+    def tick(self, a_batch, b_batch, budget_a, c_batch=None):
+        la = lb = lc = None
         if a_batch:
             toks = sum(q for _, q, _ in a_batch)
             la = (2.0 + 0.012 * toks) * self.sm_count / budget_a
         if b_batch:
             lb = 1.2 * self.sm_count / max(self.sm_count - budget_a, 1) ** 0.3 / 4.0
-        return la, lb
+        if c_batch:
+            lc = (0.6 + 0.0006 * sum(q for _, q, _ in c_batch)) * (self.sm_count / max(self.sm_count - budget_a, 28)) ** 0.5
+        return la, lb, lc
 
     def close(self):
         for h, _ in self.h.values():
@@ -117,7 +136,7 @@ class GpuEngine(Engine):
     """Two real stages on one GPU, stepped on two streams with complementary budgets."""
 
     def __init__(self, dims_a, dims_b, pages_a: int, pages_b: int, mpps_a: int, mpps_b: int, cfg: ReplayConfig,
-                 seed: int = 4, device: int = 0):
+                 seed: int = 4, device: int = 0, dims_c=None):
         import torch
         from .stage import Stage
         self.torch = torch
@@ -134,10 +153,19 @@ class GpuEngine(Engine):
         self.ya = torch.empty(max_tok_a, dims_a.d_model, dtype=torch.float32, device=dev)
         self.yb = torch.empty(cfg.max_talker, dims_b.d_model, dtype=torch.float32, device=dev)
         self.stream_a, self.stream_b = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
-        self.tables = {"a": {}, "b": {}}
+        self.tables = {"a": {}, "b": {}, "c": {}}
+        self.dims_c, self.sc = dims_c, None
+        if dims_c is not None:      # the denoising stage: no causal mask, conditioned, an image's pages live for its steps
+            mpps_c = -(-cfg.dit_tokens // 16)
+            max_tok_c = cfg.max_dit * cfg.dit_tokens
+            self.sc = Stage(dims_c, wl.make_weights(dims_c, seed + 2, dev), cfg.max_dit * mpps_c, max_tok_c, cfg.max_dit,
+                            mpps_c, cfg.dit_tokens, device, B.HS_FLAG_BIDIRECTIONAL)
+            self.sc.set_modulation(wl.make_modulation(dims_c, cfg.max_dit, seed + 2, dev))
+            self.xc = wl.make_x(max_tok_c, dims_c.d_model, seed + 2, dev)
+            self.yc = torch.empty(max_tok_c, dims_c.d_model, dtype=torch.float32, device=dev)
 
     def _stage(self, which):
-        return self.sa if which == "a" else self.sb
+        return {"a": self.sa, "b": self.sb, "c": self.sc}[which]
 
     def alloc(self, which, seq_id, total):
         self.tables[which][seq_id] = self._stage(which).kv_alloc(seq_id, total)
@@ -160,23 +188,27 @@ class GpuEngine(Engine):
         e1.record(stream)
         return e0, e1, b
 
-    def tick(self, a_batch, b_batch, budget_a):
+    def tick(self, a_batch, b_batch, budget_a, c_batch=None):
         ev = []
+        down = self.sm_count - budget_a if a_batch else self.sm_count
         if a_batch:
             ev.append(("a",) + self._launch("a", a_batch, budget_a, self.stream_a, self.xa, self.ya))
         if b_batch:
-            ev.append(("b",) + self._launch("b", b_batch, self.sm_count - budget_a if a_batch else self.sm_count,
-                                            self.stream_b, self.xb, self.yb))
+            ev.append(("b",) + self._launch("b", b_batch, down, self.stream_b, self.xb, self.yb))
+        if c_batch:                 # behind the talker's step on the downstream stream, same SM share
+            ev.append(("c",) + self._launch("c", c_batch, down, self.stream_b, self.xc, self.yc))
         self.torch.cuda.synchronize()
-        out = {"a": None, "b": None}
+        out = {"a": None, "b": None, "c": None}
         for which, e0, e1, _ in ev:
             out[which] = e0.elapsed_time(e1)
-        assert self.sa.status() == 0 and self.sb.status() == 0
-        return out["a"], out["b"]
+        assert self.sa.status() == 0 and self.sb.status() == 0 and (self.sc is None or self.sc.status() == 0)
+        return out["a"], out["b"], out["c"]
 
     def close(self):
         self.sa.close()
         self.sb.close()
+        if self.sc is not None:
+            self.sc.close()
 
 
 def step_bytes(dims, batch) -> float:
@@ -203,6 +235,11 @@ def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = Repl
     decoding: List[_Seq] = []
     talker_wait: Deque[_Seq] = deque()
     talking: List[_Seq] = []
+    use_dit = cfg.image_stage == "dit" and engine.dims_c is not None
+    dit_wait: Deque[_Seq] = deque()
+    denoising: List[_Seq] = []
+    dit_lat: List[float] = []
+    dit_tokens = 0
     done: List[_Seq] = []
     t = 0.0
     nxt = 0
@@ -225,6 +262,11 @@ def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = Repl
 
     def is_long(s):
         return s.req.talker_out > 0
+
+    def down_finished(s):
+        if use_dit and s.req.out_class == "image":
+            return s.dit_done >= cfg.dit_steps
+        return s.req.talker_out == 0 or s.talker_done >= s.req.talker_out
 
     def deadline(s):
         return s.req.arrival_s + slo[s.req.out_class] * 1e-3
@@ -254,7 +296,9 @@ def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = Repl
         while talker_wait and len(talking) < cfg.max_talker:
             s = talker_wait.popleft()
             talking.append(s)
-        if prefilling is None and not decoding and not talking:
+        while dit_wait and len(denoising) < cfg.max_dit:
+            denoising.append(dit_wait.popleft())
+        if prefilling is None and not decoding and not talking and not denoising:
             if waiting:
                 continue                              # everything waiting was hidden in this phase: next step
             if nxt >= len(trace):
@@ -278,16 +322,23 @@ def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = Repl
             ctx = cfg.talker_ctx0 + s.talker_done
             engine.alloc("b", s.req.rid, ctx + 1)
             b_batch.append((s.req.rid, 1, ctx))
+        c_batch = []
+        for s in denoising:                            # a denoising step sees the whole image, nothing is cached
+            engine.alloc("c", s.req.rid, cfg.dit_tokens)
+            c_batch.append((s.req.rid, cfg.dit_tokens, 0))
+        down_active = bool(b_batch) or bool(c_batch)
         if ctl is not None:
-            budget, _ = ctl.update(bool(b_batch), pressure)
+            budget, _ = ctl.update(down_active, pressure)
         else:
-            budget = engine.sm_count if not b_batch else int(rng.choice(cfg.ladder))
+            budget = engine.sm_count if not down_active else int(rng.choice(cfg.ladder))
         if prev_budget is not None and budget != prev_budget:
             cap_changes += 1
         prev_budget = budget
-        lat_a, lat_b = engine.tick(a_batch, b_batch, budget)
-        tick_ms = max(lat_a or 0.0, lat_b or 0.0)
+        lat_a, lat_b, lat_c = engine.tick(a_batch, b_batch, budget, c_batch)
+        tick_ms = max(lat_a or 0.0, (lat_b or 0.0) + (lat_c or 0.0))     # the two downstream steps share a stream
         moved = step_bytes(engine.dims_a, a_batch) + step_bytes(engine.dims_b, b_batch)
+        if c_batch:
+            moved += step_bytes(engine.dims_c, c_batch)
         pressure = moved / (tick_ms * 1e-3) / (cfg.hbm_gbs * 1e9) if tick_ms > 0 else 0.0
         pressures.append(pressure)
         t += tick_ms * 1e-3
@@ -298,6 +349,9 @@ def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = Repl
         if lat_b is not None:
             talker_lat.append(lat_b)
             talker_tokens += len(b_batch)
+        if lat_c is not None:
+            dit_lat.append(lat_c)
+            dit_tokens += cfg.dit_tokens * len(c_batch)
 
         # ---- advance request state ----
         if prefilling is not None:
@@ -305,7 +359,9 @@ def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = Repl
             if prefilling.prefilled == prefilling.req.prompt_len:
                 prefilling.t_first = t
                 decoding.append(prefilling)
-                if prefilling.req.talker_out > 0:
+                if use_dit and prefilling.req.out_class == "image":
+                    dit_wait.append(prefilling)
+                elif prefilling.req.talker_out > 0:
                     talker_wait.append(prefilling)
                 prefilling = None
         for s in stepped:
@@ -314,7 +370,7 @@ def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = Repl
         for s in decoding:
             if s.decoded >= s.req.backbone_out:
                 engine.free("a", s.req.rid)
-                if s.req.talker_out == 0 or s.talker_done >= s.req.talker_out:
+                if down_finished(s):
                     s.t_done = t
                     done.append(s)
             else:
@@ -333,6 +389,19 @@ def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = Repl
             else:
                 still.append(s)
         talking = still
+        still = []
+        for s in denoising:
+            s.dit_done += 1
+            if s.t_first_down is None:
+                s.t_first_down = t
+            if s.dit_done >= cfg.dit_steps:
+                engine.free("c", s.req.rid)
+                if s.decoded >= s.req.backbone_out:
+                    s.t_done = t
+                    done.append(s)
+            else:
+                still.append(s)
+        denoising = still
 
     def pct(v, q):
         return float(np.percentile(v, q)) if v else None
@@ -360,6 +429,8 @@ def replay(trace: Sequence[wl.Request], engine: Engine, cfg: ReplayConfig = Repl
                                   for b, v in sorted(ticks_by_budget.items(), reverse=True)},
             "talker_ms": {"n": len(talker_lat), "mean": statistics.fmean(talker_lat) if talker_lat else None,
                           "p95": pct(talker_lat, 95)},
+            "image_stage": cfg.image_stage if use_dit else "talker", "dit_tokens": dit_tokens,
+            "dit_ms": {"n": len(dit_lat), "mean": statistics.fmean(dit_lat) if dit_lat else None, "p95": pct(dit_lat, 95)},
             "by_class": by_class}
 
 
@@ -377,10 +448,13 @@ def main():
     ap.add_argument("--talker", default="c4_talker")
     ap.add_argument("--policy", default="seeded", choices=["seeded", "controller", "horizon"])
     ap.add_argument("--b-sat", type=float, default=ReplayConfig.b_sat)
+    ap.add_argument("--image-stage", default="talker", choices=["talker", "dit"],
+                    help="downstream stage of the image class: talker-shaped steps, or the denoising stage (c6_dit)")
     args = ap.parse_args()
-    cfg = ReplayConfig(policy=args.policy, b_sat=args.b_sat)
+    cfg = ReplayConfig(policy=args.policy, b_sat=args.b_sat, image_stage=args.image_stage)
     pa, pb, ma, mb = pool_sizes(cfg)
-    eng = GpuEngine(wl.DIMS[args.backbone], wl.DIMS[args.talker], pa, pb, ma, mb, cfg)
+    eng = GpuEngine(wl.DIMS[args.backbone], wl.DIMS[args.talker], pa, pb, ma, mb, cfg,
+                    dims_c=wl.DIMS["c6_dit"] if args.image_stage == "dit" else None)
     try:
         res = replay(wl.make_trace(args.rate, args.requests), eng, cfg)
     finally:

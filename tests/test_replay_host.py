@@ -46,6 +46,38 @@ def test_replay_conserves_tokens_and_pages():
         eng.close()
 
 
+def test_replay_with_the_denoising_stage_for_images():
+    """image_stage = "dit": images leave the talker's queue and run a fixed number of denoising steps on a third
+    stage; talker tokens are then those of the speech class only, every image gets exactly dit_steps steps of
+    dit_tokens tokens, and all three page pools return to empty."""
+    cfg = ReplayConfig(max_decode=8, max_prefill_chunk=256, max_talker=4, image_stage="dit", dit_steps=7, dit_tokens=48,
+                       max_dit=2)
+    trace = wl.make_trace(16.0, 60, seed=4)
+    pa, pb, ma, mb = pool_sizes(cfg)
+    mc = -(-cfg.dit_tokens // 16)
+    pc = cfg.max_dit * mc
+    eng = ModelEngine(wl.DIMS["c1_tiny"], wl.DIMS["c1_tiny"], pa, pb, ma, mb, wl.DIMS["c1_tiny"], pc, mc)
+    try:
+        res = replay(trace, eng, cfg)
+        n_img = sum(r.out_class == "image" for r in trace)
+        assert n_img > 0 and res["requests_done"] == 60 and res["image_stage"] == "dit"
+        assert res["talker_tokens"] == sum(r.talker_out for r in trace if r.out_class == "speech")
+        assert res["dit_tokens"] == n_img * cfg.dit_steps * cfg.dit_tokens
+        assert res["dit_ms"]["n"] >= n_img * cfg.dit_steps / cfg.max_dit
+        assert eng.free_pages("a") == pa and eng.free_pages("b") == pb and eng.free_pages("c") == pc
+        img = res["by_class"]["image"]
+        assert img["first_downstream_ms_p50"] >= img["ttft_ms_p50"] > 0
+    finally:
+        eng.close()
+    # without a third stage in the engine the option falls back to talker-shaped steps
+    eng = ModelEngine(wl.DIMS["c1_tiny"], wl.DIMS["c1_tiny"], pa, pb, ma, mb)
+    try:
+        res = replay(trace, eng, cfg)
+        assert res["image_stage"] == "talker" and res["talker_tokens"] == sum(r.talker_out for r in trace)
+    finally:
+        eng.close()
+
+
 def test_replay_under_the_spatial_controller():
     """The same replay with the library's controller choosing the budget: while the talker has work the
     backbone never gets more than the top of the ladder, it gets all SMs when the talker is idle, the cap
