@@ -448,8 +448,22 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
   const size_t layer_kv_elems = size_t(c.num_pages) * c.n_kv_heads * kPage * Dh;
   cudaError_t e = cudaSuccess;
   const char* where = "";
-  // More than one 128-row tile of tokens: the GEMMs run on pairs of SMs (a choice by shape, not by budget).
+  // More than one 128-row tile of tokens: a GEMM runs on pairs of SMs (256 x 256 tiles), unless such tiles would
+  // occupy less than half of the device's pairs AND its 128-row tiles for single blocks fit one wave: then single
+  // blocks occupy more SMs (and a residual GEMM may split K).  A choice by shape, never by budget; the two
+  // kernels give the same bits.  Measured at config-3 dimensions, one prefill chunk + decodes (ms per step, all
+  // pairs -> this rule): 220 rows 7.41 -> 5.60, 440 rows 9.23 -> 8.63; at 650 rows and more (pair tiles on 57 %
+  // of the pairs and up) pairs are the faster form again, a pair tile moving two thirds of the operand bytes of
+  // two single tiles.
   const bool use_pair = T > 128;
+  auto pair_for = [&](int n_cols, int single_bn) {
+    if (!use_pair) return false;
+    const bool few_pair_tiles = ceil_div(T, 256) * ceil_div(n_cols, 256) < s->sm_count / 4;
+    const bool singles_fit = ceil_div(T, 128) * ceil_div(n_cols, single_bn) <= s->sm_count;
+    return !(few_pair_tiles && singles_fit);
+  };
+  const bool pair_qkv = pair_for(q_dim + 2 * kv_dim, 128), pair_gu = pair_for(2 * F, 256);
+  const bool pair_d = pair_for(d, gemm_pick_bn(T, d, s->sm_count));
   const int f16 = (c.flags & HS_FLAG_BF16_ACTIVATIONS) ? 0 : 1;   // format of h, o, act
   // With the whole device as its budget a step has no neighbour to take SMs from, so each kernel is launched
   // such that its set-up overlaps the previous kernel's drain.  With a smaller budget the blocks of the next
@@ -506,8 +520,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     g.mode = kGemmQkv;
     g.ab_f16 = f16;
     g.overlap = overlap;
-    g.pair = use_pair;
-    g.bn = use_pair ? 256 : 128;     // small steps: 128-column tiles, twice as many SMs stream the weights
+    g.pair = pair_qkv;
+    g.bn = pair_qkv ? 256 : 128;     // small steps: 128-column tiles, twice as many SMs stream the weights
     g.q_dim = q_dim; g.kv_dim = kv_dim; g.head_dim = Dh; g.n_kv_heads = c.n_kv_heads;
     g.tm_q = s->tm_q_st;
     g.k_cache = s->kv_pool + (size_t(l) * 2 + 0) * layer_kv_elems;
@@ -571,9 +585,9 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     go.overlap = overlap;
     go.tm_out = tm_y; go.accumulate = 1;
     go.gate_mod = mod_l; go.tok_seq = meta + s->ml.tok_seq; go.gate_which = 2;
-    go.pair = use_pair;
-    go.bn = use_pair ? 256 : gemm_pick_bn(T, d, s->sm_count);
-    go.ksplit = use_pair ? 1 : pick_ksplit(T, d, q_dim, go.bn, s->sm_count);
+    go.pair = pair_d;
+    go.bn = pair_d ? 256 : gemm_pick_bn(T, d, s->sm_count);
+    go.ksplit = pair_d ? 1 : pick_ksplit(T, d, q_dim, go.bn, s->sm_count);
     go.tile_turn = reinterpret_cast<int*>(s->ws_dev + s->ws.turn);
     go.status = status;
     go.smid_log = slots(5);
@@ -601,7 +615,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gu.ab_f16 = f16;
     gu.overlap = overlap;
     gu.act_f16 = f16;
-    gu.pair = use_pair;
+    gu.pair = pair_gu;
     gu.tm_act = s->tm_act_st;
     gu.status = status;
     gu.smid_log = slots(6);
@@ -624,9 +638,9 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gd.overlap = overlap;
     gd.tm_out = tm_y; gd.accumulate = 1;
     gd.gate_mod = mod_l; gd.tok_seq = meta + s->ml.tok_seq; gd.gate_which = 5;
-    gd.pair = use_pair;
-    gd.bn = use_pair ? 256 : gemm_pick_bn(T, d, s->sm_count);
-    gd.ksplit = use_pair ? 1 : pick_ksplit(T, d, F, gd.bn, s->sm_count);
+    gd.pair = pair_d;
+    gd.bn = pair_d ? 256 : gemm_pick_bn(T, d, s->sm_count);
+    gd.ksplit = pair_d ? 1 : pick_ksplit(T, d, F, gd.bn, s->sm_count);
     gd.tile_turn = reinterpret_cast<int*>(s->ws_dev + s->ws.turn);
     gd.status = status;
     gd.smid_log = slots(7);
