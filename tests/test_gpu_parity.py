@@ -220,7 +220,7 @@ def test_edge_cases_match_oracle(orc, name):
     y_ref = orc.step(case.cfg, case.weights, pool_ref, batch.q_len, batch.ctx_len, case.block_tables, case.x)
     assert np.all(np.isfinite(y_ref))
     outs = []
-    # more than 128 tokens put the GEMMs on pairs of SMs; a budget of one SM then has to fall back to single blocks
+    # more than one 128-row tile per GEMM (two m-tiles, K splits over several tiles); also run on a single SM
     budgets = (148, 5, 1) if name == "continuation_chunks" else (148, 5)
     for budget in budgets:
         st = make_stage(case)
@@ -252,8 +252,8 @@ def test_edge_cases_match_oracle(orc, name):
 
 BIAS_CASES = {
     # name: (dims, q_len, ctx_len): which QKV epilogue adds the biases
-    "pair_tiles_dh64": (wl.StageDims(2, 256, 4, 2, 64, 688), [100, 60, 1, 1], [0, 37, 64, 200]),   # T > 128
-    "single_tile_dh128": (wl.StageDims(1, 256, 2, 2, 128, 512), [70, 1, 33], [0, 200, 5]),         # 64 < T <= 128
+    "two_row_tiles_dh64": (wl.StageDims(2, 256, 4, 2, 64, 688), [100, 60, 1, 1], [0, 37, 64, 200]),   # T > 128
+    "single_tile_dh128": (wl.StageDims(1, 256, 2, 2, 128, 512), [70, 1, 33], [0, 200, 5]),          # 64 < T <= 128
     "streaming_kernel_dh64": (wl.StageDims(2, 1024, 16, 4, 64, 2816), [1] * 16, [128 + 57 * i for i in range(16)]),
     "streaming_kernel_dh128": (wl.StageDims(1, 2048, 8, 2, 128, 1024), [20, 1, 1], [0, 300, 17]),
 }
@@ -337,7 +337,7 @@ def test_bidirectional_attention_matches_oracle(orc, name):
 
 MOD_CASES = {
     # name: (dims, q_len, ctx_len, flags)
-    "pair_tiles_bidirectional": (wl.StageDims(2, 256, 4, 4, 64, 688), [150, 60, 9], [0, 0, 0], B.HS_FLAG_BIDIRECTIONAL),
+    "two_row_tiles_bidirectional": (wl.StageDims(2, 256, 4, 4, 64, 688), [150, 60, 9], [0, 0, 0], B.HS_FLAG_BIDIRECTIONAL),
     "single_tile_causal": (wl.StageDims(1, 256, 2, 2, 128, 512), [70, 1, 33], [0, 200, 5], 0),
     "streaming_kernel_16_rows": (wl.StageDims(2, 1024, 16, 4, 64, 2816), [1] * 16, [128 + 57 * i for i in range(16)], 0),
     "streaming_kernel_22_rows": (wl.StageDims(1, 2048, 8, 2, 128, 1024), [20, 1, 1], [0, 300, 17], 0),
