@@ -292,3 +292,44 @@ def test_config3_decode_only_tick(orc, n_dec):
         assert np.all(np.abs(a - b) <= 2.0 ** -7 * np.abs(b) + 1e-2 * np.sqrt(np.mean(b * b)))
     finally:
         stage.close()
+
+
+# ------------------------------------------------- optional features on SM pairs --
+def test_bias_and_modulation_on_pair_tiles(orc):
+    """Config-2 dimensions, one layer, 1300 rows: every projection has enough 256 x 256 tiles to run on pairs of
+    SMs, so the q / k / v biases and the shift / scale / gate vectors go through the pair form of the epilogues.
+    The oracle evaluates K/V of all tokens and a sample of rows."""
+    r = np.random.default_rng(7)
+    batch = wl.BatchSpec([700, 500] + [1] * 100, [0, 300] + r.integers(64, 1500, size=100).tolist())
+    stage, dims, batch, bt, x = bench.build_stage("c2_shared", 0, layers=1, batch=batch)
+    try:
+        dev = stage.device
+        g = torch.Generator().manual_seed(3)
+        biases = [(torch.randn(n, generator=g) * 0.5).to(torch.bfloat16) for n in (dims.q_dim, dims.kv_dim, dims.kv_dim)]
+        dev_b = [t.to(dev) for t in biases]
+        stage.set_qkv_bias(0, *dev_b)
+        mod = wl.make_modulation(dims, stage.cfg.max_seqs, 9)
+        mod[:, :, [0, 1, 3, 4]] *= 3.0                       # larger shifts and scales than the bench's
+        stage.set_modulation(mod.to(dev).contiguous())
+        pool0 = stage.kv_pool.clone()
+        y_gpu = gpu_step(stage, batch, bt, x, stage.sm_count, pool0).cpu().numpy()
+        y_74 = gpu_step(stage, batch, bt, x, 74, pool0).cpu().numpy()
+        assert np.array_equal(y_gpu, y_74)
+        rows = np.unique(np.concatenate([np.array([0, 1, 255, 256, 699, 700, 1199, 1200, 1299]),
+                                         np.linspace(0, batch.n_tokens - 1, 40).astype(np.int64)]))
+        mask = np.zeros(batch.n_tokens, dtype=np.uint8)
+        mask[rows] = 1
+        w = {k: wl.to_f32_numpy(v) for k, v in stage.weights[0].items()}
+        w.update(b_q=biases[0].float().numpy(), b_k=biases[1].float().numpy(), b_v=biases[2].float().numpy(),
+                 mod=mod[0, :batch.n_seqs].numpy())
+        y_ref, _ = orc.layer(ocfg(dims, 1, stage.cfg.num_pages), w, 0, wl.bf16_bits_numpy(pool0).reshape(-1).copy(),
+                             batch.q_len, batch.ctx_len, bt, wl.to_f32_numpy(x), row_mask=mask)
+        err = rel_err(y_gpu[rows], y_ref[rows])
+        print(f"config-2 dimensions, 1300 rows, biases + modulation on pair tiles: max|err|/RMS = {err:.2e}")
+        assert err <= TOL
+        plain = {k: v for k, v in w.items() if k not in ("b_q", "b_k", "b_v", "mod")}
+        y_plain, _ = orc.layer(ocfg(dims, 1, stage.cfg.num_pages), plain, 0, wl.bf16_bits_numpy(pool0).reshape(-1).copy(),
+                               batch.q_len, batch.ctx_len, bt, wl.to_f32_numpy(x), row_mask=mask)
+        assert rel_err(y_plain[rows], y_ref[rows]) > 5 * TOL
+    finally:
+        stage.close()
