@@ -17,8 +17,10 @@
  * where ladder[0] = S_min < ... < ladder[n-1] = S_cap < s_aggr <= s_total, and snap returns the ladder value
  * nearest to its argument (the lower one on a tie).  Hysteresis (Sec. 4.3, last paragraph; Algorithm 1
  * step 3): while the downstream stage is active the cap changes only if s* differs from the previous cap by
- * at least delta_step SMs; when the downstream stage is inactive s* = s_aggr is applied at once.  The
- * downstream stage receives s_down = max(0, s_total - s_shared).
+ * at least delta_step SMs -- except that a previous cap above S_cap (the aggressive allocation of the steps
+ * without downstream work) is always replaced by s*, so that a co-running step never runs above S_cap (Eq. 1:
+ * S_cap < S_aggr) and the downstream stage is never left without SMs; when the downstream stage is inactive
+ * s* = s_aggr is applied at once.  The downstream stage receives s_down = max(0, s_total - s_shared).
  * The paper leaves open: the form of the moving average and its start, the tie rule of snap, whether
  * delta_step counts SMs or ladder levels (SMs here; use the ladder's spacing for "one ladder step"), and
  * whether Bhat is updated while A == 0 (it is).

@@ -44,8 +44,11 @@ class SpatialOracle:
             rho = min(max(self.bhat / self.b_sat, 0.0), 1.0)
             s_min, s_cap = self.ladder[0], self.ladder[-1]
             s_star = self.snap(s_min + rho * (s_cap - s_min))
-            # hysteresis: keep the previous cap unless the level moves by at least delta_step
-            if abs(s_star - self.s_shared) >= self.delta_step:
+            # Sec. 4.3: during co-running the cap stays within the ladder, "never back to full allocation"
+            # (S_cap < S_aggr), so a cap above S_cap left by the inactive case is replaced at once; the
+            # hysteresis (keep the previous cap unless the level moves by at least delta_step) acts only
+            # between ladder levels
+            if self.s_shared > s_cap or abs(s_star - self.s_shared) >= self.delta_step:
                 self.s_shared = s_star
         # "Complementary downstream headroom"
         return self.s_shared, max(0, self.s_total - self.s_shared)

@@ -72,7 +72,10 @@ hs_status_t hs_spatial_update(hs_spatial_t* c, int32_t downstream_active, double
     const int32_t s_min = c->ladder.front(), s_cap = c->ladder.back();
     const int32_t s_star = snap(c->ladder, double(s_min) + rho * double(s_cap - s_min));
     const int32_t diff = s_star > c->s_shared ? s_star - c->s_shared : c->s_shared - s_star;
-    if (diff >= c->delta_step) c->s_shared = s_star;       // hysteresis: smaller moves are not applied
+    // Hysteresis holds a cap only between ladder levels: a cap above S_cap (the aggressive allocation left over
+    // from the steps without downstream work) is never kept while the downstream stage runs, because Eq. 1 bounds
+    // the co-running cap by S_cap < S_aggr whatever the distance to the new level.
+    if (c->s_shared > s_cap || diff >= c->delta_step) c->s_shared = s_star;
   }
   if (s_shared) *s_shared = c->s_shared;
   if (s_down) *s_down = c->s_total - c->s_shared > 0 ? c->s_total - c->s_shared : 0;

@@ -75,6 +75,32 @@ def test_hysteresis_holds_the_cap_until_the_level_moves_far_enough():
     assert o.update(True, 0.33)[0] == 74
 
 
+def test_active_downstream_never_keeps_the_aggressive_cap_whatever_the_hysteresis():
+    """Eq. 1 / Sec. 4.3: S_cap < S_aggr bounds the cap of every co-running step.  The case a hysteresis taken
+    literally gets wrong: coming from the inactive case at 148 with maximum pressure, s* = 120 lies only 28 SMs
+    away, less than delta_step = 30 -- the cap must still drop to 120 at once (and the downstream stage must be
+    left with SMs)."""
+    o = make(gamma=1.0, delta=30)
+    assert o.update(False, 0.9) == (148, 0)
+    assert o.update(True, 0.9) == (120, 28)
+    rng = np.random.default_rng(11)
+    for trial in range(60):
+        n = int(rng.integers(1, 7))
+        ladder = sorted(rng.choice(np.arange(8, 140), size=n, replace=False).tolist())
+        s_aggr = int(rng.integers(ladder[-1] + 1, 149))
+        o = SpatialOracle(148, s_aggr, ladder, float(rng.uniform(0.2, 2.0)), float(rng.uniform(0.05, 1.0)),
+                          int(rng.integers(0, 60)))
+        active = False
+        for _ in range(300):
+            if rng.uniform() < 0.15:
+                active = not active
+            s, d = o.update(active, float(rng.uniform(0, 2.5)))
+            if active:
+                assert s in ladder and s <= ladder[-1] < s_aggr and d == 148 - s and d > 0, (trial, s)
+            else:
+                assert s == s_aggr
+
+
 def test_derive_cap_smallest_near_best_budget_below_full_allocation():
     # decode latency saturates at 80 SMs and gets worse at full allocation (the shape of the paper's Fig. 4)
     budgets = [16, 32, 48, 64, 80, 96, 120, 142]
