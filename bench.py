@@ -34,9 +34,13 @@ from paper_2608_01785_b200 import workloads as wl  # noqa: E402
 METRIC = "shared_stage_tokens_per_s"
 UNIT = "tokens/s"
 SEED = {"c1_tiny": 0, "c2_shared": 1, "c3_7b": 2, "c4_talker": 3, "c3_decode": 2, "c6_dit": 5}
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one gate/up GEMM launch, from the ncu
-# capture summarised in profiles/gemm_pair_gateup_c2_shared.md (None where no capture of that launch exists).
-GATEUP_DRAM_TRAFFIC_BYTES = {"c2_shared": 69989376 + 39707904}
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one gate/up GEMM launch per workload, each from one
+# ncu capture of that launch (the config-3 launch was captured on a 2-layer cut of the stage: a layer's launch
+# reads its own weights and the step's activations whatever the depth).  None where no capture exists.
+GATEUP_DRAM_TRAFFIC_BYTES = {"c2_shared": 69989376 + 39707904, "c3_7b": None}
+# Below this length of the timed region a kernel runs at burst clocks and is held against the burst peak; a longer
+# region settles under the power cap and is held against the sustained peak.
+BURST_REGION_MS = 1000.0
 
 
 def measured_peaks():
@@ -61,7 +65,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -264,18 +268,186 @@ def run_head(args):
                                    "frac": bytes_moved / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "traffic": None}}))
 
 
+def gemm_classes(dims: wl.StageDims, T: int):
+    """flops = 2 M K N of the four projection launches of one layer."""
+    d, F = dims.d_model, dims.d_ffn
+    return {"gemm_qkv": 2.0 * T * d * (dims.q_dim + 2 * dims.kv_dim), "gemm_out": 2.0 * T * dims.q_dim * d,
+            "gemm_gateup": 2.0 * T * d * 2 * F, "gemm_down": 2.0 * T * F * d}
+
+
+def rooflines(name, dims, batch, prof, steps, ms_step, clocks, budget, sm_count, peaks):
+    """Roofline entries from the per-class event timing: one per GEMM class, prefill attention (tensor), decode
+    attention and RMSNorm (HBM).  The tensor peak is the burst figure when the timed region is short, the
+    sustained one otherwise; both fractions are printed, and time x median SM clock lets a reader normalise."""
+    T = batch.n_tokens
+    region_ms = ms_step * steps
+    use_burst = region_ms < BURST_REGION_MS
+    peak_t = (peaks["bf16_burst"] if use_burst else peaks["bf16_sustained"]) * budget / sm_count
+    mhz = (clocks or {}).get("sm_mhz")
+    out = {}
+    for cls, flops in gemm_classes(dims, T).items():
+        ms, n = prof[cls]
+        if not n:
+            continue
+        avg_s = ms * 1e-3 / n
+        ach = flops / avg_s / 1e12
+        out[cls] = {"bound": "tensor", "achieved": ach, "peak": peak_t, "unit": "TFLOP/s", "frac": ach / peak_t,
+                    "frac_of_burst_peak": ach / (peaks["bf16_burst"] * budget / sm_count),
+                    "frac_of_sustained_peak": ach / (peaks["bf16_sustained"] * budget / sm_count),
+                    "flops_per_launch": flops, "avg_launch_ms": avg_s * 1e3, "launches": n,
+                    "ms_x_sm_mhz": avg_s * 1e3 * mhz if mhz else None}
+    _, attn_flops = flops_per_step(dims, batch)
+    ms, n = prof["attn_prefill"]
+    if n:
+        fl = attn_flops / dims.n_layers - sum(4.0 * dims.n_q_heads * dims.head_dim * (c + 1)
+                                              for q, c in zip(batch.q_len, batch.ctx_len) if q == 1)
+        ach = fl / (ms * 1e-3 / n) / 1e12
+        out["attn_prefill"] = {"bound": "tensor", "achieved": ach, "peak": peak_t, "unit": "TFLOP/s", "frac": ach / peak_t,
+                               "flops_per_launch": fl, "avg_launch_ms": ms / n, "launches": n,
+                               "note": "causal flops 4 Hq Dh sum(c n + n (n + 1) / 2); bound by the exponentials "
+                                       "as much as by the tensor pipe"}
+    ms, n = prof["attn_decode"]
+    if n:
+        dec_bytes = sum((c + 1) * 2 * dims.kv_dim * 2 for q, c in zip(batch.q_len, batch.ctx_len) if q == 1)
+        gbs = dec_bytes / (ms * 1e-3 / n) / 1e9
+        out["attn_decode"] = {"bound": "hbm", "kernel": "attn_decode_kernel", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                              "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "bytes_per_launch": dec_bytes,
+                              "avg_launch_ms": ms / n, "launches": n,
+                              "note": ("K and V pages of every decode sequence once per layer; " +
+                                       ("bytes below the 126 MB L2 are served from L2, not HBM" if dec_bytes < 126e6
+                                        else "working set exceeds L2") + "; the HBM peak is not scaled by the budget")}
+    ms, n = prof["rmsnorm"]
+    if n:
+        nbytes = T * dims.d_model * (4 + 2)
+        gbs = nbytes / (ms * 1e-3 / n) / 1e9
+        out["rmsnorm"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                          "frac": gbs / peaks["hbm_gbs"], "bytes_per_launch": nbytes, "avg_launch_ms": ms / n, "launches": n}
+    meta = {"timed_region_ms": region_ms, "tensor_peak_used": "burst" if use_burst else "sustained",
+            "rule": f"burst peak when the timed region is under {BURST_REGION_MS:.0f} ms, sustained otherwise",
+            "peaks": {"bf16_burst_tflops": peaks["bf16_burst"], "bf16_sustained_tflops": peaks["bf16_sustained"],
+                      "hbm_gbs": peaks["hbm_gbs"], "source": peaks["source"]},
+            "operands": "fp16 x fp16 (nominal rate equals bf16 x bf16: ratio 1.0)", "median_sm_mhz": mhz}
+    return out, meta
+
+
+class Measured:
+    """Device-resident timing, per-class timing and the end-to-end leg of one workload on one stage."""
+
+    def __init__(self, name, args, local_rank, rank, world, barrier, flags=0):
+        self.name, self.args, self.rank, self.world, self.barrier = name, args, rank, world, barrier
+        self.stage, self.dims, self.batch, self.bt, self.x = build_stage(name, local_rank, layers=args.layers, flags=flags)
+        self.dev = self.stage.device
+        self.T, self.d = self.batch.n_tokens, self.dims.d_model
+        self.y = torch.empty(self.T, self.d, dtype=torch.float32, device=self.dev)
+        self.b = self.stage.make_batch(self.batch.q_len, self.batch.ctx_len, self.bt, self.x, self.y)
+        self.stream = torch.cuda.Stream(device=self.dev)
+        self.budget = args.sm_budget or self.stage.sm_count
+
+    def timed_steps(self, k, fn):
+        self.barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(self.stream):
+            e0.record(self.stream)
+            for _ in range(k):
+                fn()
+            e1.record(self.stream)
+        self.barrier()
+        return max_over_ranks(e0.elapsed_time(e1), self.world, self.dev)
+
+    def step_fn(self, budget=None):
+        bud = budget or self.budget
+        return lambda: self.stage.step(self.b, bud, self.stream)
+
+    def device_resident(self, steps, warmup, sample_clocks):
+        self.timed_steps(warmup, self.step_fn())
+        sampler = ClockSampler(self.dev.index or 0)
+        if sample_clocks:
+            sampler.start()
+        ms_total = self.timed_steps(steps, self.step_fn())
+        clocks = sampler.stop() if sample_clocks else None
+        assert self.stage.status() == 0, "device status word is set"
+        assert self.stage.saturation_count() == 0, "fp16 activations were clamped"
+        return ms_total / steps, clocks
+
+    def per_class(self, steps):
+        from paper_2608_01785_b200 import binding as B
+        B.hs_stage_profile_enable(self.stage.handle, True)
+        self.timed_steps(steps, self.step_fn())
+        prof = B.hs_stage_profile_read(self.stage.handle)
+        B.hs_stage_profile_enable(self.stage.handle, False)
+        return prof
+
+    def e2e(self, steps):
+        """Every step's x_in comes from pinned host memory and its y_out goes back to pinned host memory, all inside
+        the timed region.  The copies of step i+1 / i-1 run on their own streams beside the kernels of step i (two
+        device buffers each way), as a serving loop would do it."""
+        stage, batch, bt, x, dev, T, d = self.stage, self.batch, self.bt, self.x, self.dev, self.T, self.d
+        x_host = x.cpu().pin_memory()
+        y_host = torch.empty(T, d, dtype=torch.float32).pin_memory()
+        x_dev2 = [torch.empty_like(x) for _ in range(2)]
+        y_dev2 = [torch.empty(T, d, dtype=torch.float32, device=dev) for _ in range(2)]
+        b2 = [stage.make_batch(batch.q_len, batch.ctx_len, bt, x_dev2[i], y_dev2[i]) for i in range(2)]
+        s_in, s_out, stream = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev), self.stream
+
+        def run(k):
+            self.barrier()
+            in_done = [torch.cuda.Event() for _ in range(k)]
+            cmp_done = [torch.cuda.Event() for _ in range(k)]
+            out_done = [torch.cuda.Event() for _ in range(k)]
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(s_in)
+            for i in range(k):
+                j = i & 1
+                with torch.cuda.stream(s_in):
+                    if i >= 2:
+                        s_in.wait_event(cmp_done[i - 2])        # x_dev2[j] was read by step i-2
+                    x_dev2[j].copy_(x_host, non_blocking=True)
+                    in_done[i].record(s_in)
+                stream.wait_event(in_done[i])
+                if i >= 2:
+                    stream.wait_event(out_done[i - 2])          # y_dev2[j] has been copied out
+                stage.step(b2[j], self.budget, stream)
+                cmp_done[i].record(stream)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(cmp_done[i])
+                    y_host.copy_(y_dev2[j], non_blocking=True)
+                    out_done[i].record(s_out)
+            e1.record(s_out)
+            self.barrier()
+            return max_over_ranks(e0.elapsed_time(e1), self.world, dev)
+
+        run(3)
+        return run(steps) / steps
+
+    def sweep(self, steps):
+        rows = []
+        for bud in [x for x in wl.SM_BUDGETS.get(self.name, (148, 112, 74, 37)) if x <= self.stage.sm_count]:
+            fn = self.step_fn(bud)
+            self.timed_steps(3, fn)
+            ms_b = self.timed_steps(steps, fn) / steps
+            rows.append({"sm_budget": bud, "ms_per_step": ms_b, "tokens_per_s": self.T / (ms_b * 1e-3)})
+        for row in rows:
+            row["speed_vs_full"] = rows[0]["ms_per_step"] / row["ms_per_step"]
+            row["budget_fraction"] = row["sm_budget"] / rows[0]["sm_budget"]
+        return rows
+
+    def close(self):
+        self.stage.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c2_shared", choices=sorted(SEED) + ["c3_head"])
+    ap.add_argument("--workload", default="c3_7b", choices=sorted(SEED) + ["c3_head"])
     ap.add_argument("--sm-budget", type=int, default=0, help="0 = all SMs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--bf16-activations", action="store_true",
                     help="stage flag HS_FLAG_BF16_ACTIVATIONS: h, o, act in bf16, no fp16 weight copies")
-    ap.add_argument("--no-sweep", action="store_true", help="skip the SM-budget sweep and the co-run section")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="skip the SM-budget sweep, the all-bf16 leg and the config-2 / co-run section")
     ap.add_argument("--layers", type=int, default=0,
                     help="profiling aid: cut the workload's stage to this many layers (not a benchmark configuration)")
     args = ap.parse_args()
@@ -295,7 +467,6 @@ def main():
         return
 
     import torch.distributed as dist
-    from paper_2608_01785_b200 import binding as B
     torch.cuda.set_device(local_rank)
     if world > 1:
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
@@ -307,150 +478,78 @@ def main():
         torch.cuda.synchronize()
 
     name = args.workload
-    stage, dims, batch, bt, x = build_stage(name, local_rank, layers=args.layers, flags=1 if args.bf16_activations else 0)
-    budget = args.sm_budget or stage.sm_count
-    T, d = batch.n_tokens, dims.d_model
-    dev = stage.device
-    y = torch.empty(T, d, dtype=torch.float32, device=dev)
-    b = stage.make_batch(batch.q_len, batch.ctx_len, bt, x, y)
-    stream = torch.cuda.Stream(device=dev)
+    peaks = measured_peaks()
+    m = Measured(name, args, local_rank, rank, world, barrier, flags=1 if args.bf16_activations else 0)
+    dims, batch, T, d, budget, stage = m.dims, m.batch, m.T, m.d, m.budget, m.stage
 
-    def timed_steps(k: int, fn):
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        with torch.cuda.stream(stream):
-            e0.record(stream)
-            for _ in range(k):
-                fn()
-            e1.record(stream)
-        barrier()
-        return max_over_ranks(e0.elapsed_time(e1), world, dev)
-
-    step_dev = lambda: stage.step(b, budget, stream)
-
-    # ---- device-resident throughput -------------------------------------
-    timed_steps(args.warmup, step_dev)
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    ms_total = timed_steps(args.steps, step_dev)
-    clocks = sampler.stop() if rank == 0 else None
-    assert stage.status() == 0, "device status word is set"
-    ms_step = ms_total / args.steps
+    # ---- device-resident throughput, per-kernel timing, end to end -----------
+    ms_step, clocks = m.device_resident(args.steps, args.warmup, rank == 0)
     value = aggregate_tokens_per_s(T, world, ms_step)
-
-    # ---- per-kernel timing (same launches, events around each kernel) ----
-    B.hs_stage_profile_enable(stage.handle, True)
-    timed_steps(args.steps, step_dev)
-    prof = B.hs_stage_profile_read(stage.handle)
-    B.hs_stage_profile_enable(stage.handle, False)
+    prof = m.per_class(args.steps)
     launches_per_step = sum(n for _, n in prof.values()) // args.steps
-
-    # ---- end to end: host buffers in, host buffers out -------------------
-    # Every step's x_in comes from pinned host memory and its y_out goes back to pinned host memory, all
-    # inside the timed region.  The copies of step i+1 / i-1 run on their own streams beside the kernels of
-    # step i (two device buffers each way), as a serving loop would do it.
-    x_host = x.cpu().pin_memory()
-    y_host = torch.empty(T, d, dtype=torch.float32).pin_memory()
-    x_dev2 = [torch.empty_like(x) for _ in range(2)]
-    y_dev2 = [torch.empty(T, d, dtype=torch.float32, device=dev) for _ in range(2)]
-    b2 = [stage.make_batch(batch.q_len, batch.ctx_len, bt, x_dev2[i], y_dev2[i]) for i in range(2)]
-    s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
-
-    def e2e_steps(k: int) -> float:
-        barrier()
-        in_done = [torch.cuda.Event() for _ in range(k)]
-        cmp_done = [torch.cuda.Event() for _ in range(k)]
-        out_done = [torch.cuda.Event() for _ in range(k)]
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(s_in)
-        for i in range(k):
-            j = i & 1
-            with torch.cuda.stream(s_in):
-                if i >= 2:
-                    s_in.wait_event(cmp_done[i - 2])        # x_dev2[j] was read by step i-2
-                x_dev2[j].copy_(x_host, non_blocking=True)
-                in_done[i].record(s_in)
-            stream.wait_event(in_done[i])
-            if i >= 2:
-                stream.wait_event(out_done[i - 2])          # y_dev2[j] has been copied out
-            stage.step(b2[j], budget, stream)
-            cmp_done[i].record(stream)
-            with torch.cuda.stream(s_out):
-                s_out.wait_event(cmp_done[i])
-                y_host.copy_(y_dev2[j], non_blocking=True)
-                out_done[i].record(s_out)
-        e1.record(s_out)
-        barrier()
-        return max_over_ranks(e0.elapsed_time(e1), world, dev)
-
-    e2e_steps(3)
-    ms_e2e = e2e_steps(args.steps) / args.steps
+    ms_e2e = m.e2e(args.steps)
     e2e_value = aggregate_tokens_per_s(T, world, ms_e2e)
 
-    # ---- step latency vs SM budget, and the co-run with a downstream stage (rank 0, single GPU) ----
-    sweep, corun_rows, corun_dit_rows = None, None, None
+    # ---- rank 0, single GPU: budget sweep, the all-bf16 form, config 2 and the co-runs ----
+    sweep, bf16_leg, c2_obj, corun_rows, corun_dit_rows = None, None, None, None, None
+    small = max(args.steps // 2, 5)
     if rank == 0 and world == 1 and not args.no_sweep:
-        sweep = []
-        for bud in [x for x in wl.SM_BUDGETS.get(name, (148, 112, 74, 37)) if x <= stage.sm_count]:
-            fn = lambda: stage.step(b, bud, stream)
-            timed_steps(3, fn)
-            ms_b = timed_steps(args.steps, fn) / args.steps
-            sweep.append({"sm_budget": bud, "ms_per_step": ms_b, "tokens_per_s": T / (ms_b * 1e-3)})
-        for row in sweep:
-            row["speed_vs_full"] = sweep[0]["ms_per_step"] / row["ms_per_step"]
-            row["budget_fraction"] = row["sm_budget"] / sweep[0]["sm_budget"]
-        if name == "c2_shared":
+        sweep = m.sweep(args.steps)
+        if not args.bf16_activations and name in ("c3_7b", "c2_shared"):
+            # the same step with every operand in bf16 (HS_FLAG_BF16_ACTIVATIONS: no fp16 copies of the weights)
+            mb = Measured(name, args, local_rank, rank, world, barrier, flags=1)
+            ms_b, _ = mb.device_resident(small, 3, False)
+            bf16_leg = {"ms_per_step": ms_b, "tokens_per_s": T / (ms_b * 1e-3), "steps": small,
+                        "formats": "all-bf16 operands (HS_FLAG_BF16_ACTIVATIONS); fp32 accumulation"}
+            mb.close()
+            del mb
+        if name == "c3_7b":
+            # config 2 (shared backbone, 4 layers) with its own sweep, per-class rooflines and the co-runs of config 4
             from paper_2608_01785_b200.corun import corun
+            steps2 = max(args.steps, 20)
+            m2 = Measured("c2_shared", args, local_rank, rank, world, barrier)
+            ms2, clocks2 = m2.device_resident(steps2, 3, True)
+            prof2 = m2.per_class(steps2)
+            roof2, roof2_meta = rooflines("c2_shared", m2.dims, m2.batch, prof2, steps2, ms2, clocks2, m2.budget,
+                                          m2.stage.sm_count, peaks)
+            c2_obj = {"workload": "c2_shared", "n_tokens": m2.T, "n_layers": m2.dims.n_layers, "steps": steps2,
+                      "ms_per_step": ms2, "tokens_per_s": m2.T / (ms2 * 1e-3), "e2e_ms_per_step": m2.e2e(steps2),
+                      "clocks": clocks2, "rooflines": roof2, "roofline_basis": roof2_meta,
+                      "kernels": {k: {"ms_per_step": v[0] / steps2, "launches_per_step": v[1] / steps2} for k, v in prof2.items()},
+                      "budget_sweep": m2.sweep(steps2)}
             talker, tdims, tbatch, tbt, tx = build_stage("c4_talker", local_rank)
-            ty = torch.empty(tbatch.n_tokens, tdims.d_model, dtype=torch.float32, device=dev)
+            ty = torch.empty(tbatch.n_tokens, tdims.d_model, dtype=torch.float32, device=m2.dev)
             tb = talker.make_batch(tbatch.q_len, tbatch.ctx_len, tbt, tx, ty)
-            corun_rows = [corun(stage, b, talker, tb, bud, args.steps) for bud in wl.SM_BUDGETS["c4_corun"]]
+            corun_rows = [corun(m2.stage, m2.b, talker, tb, bud, steps2) for bud in wl.SM_BUDGETS["c4_corun"]]
             assert talker.status() == 0
             talker.close()
-            # the same co-run with the denoising-style stage (the image path's downstream partner)
             dit, ddims, dbatch, dbt, dx = build_stage("c6_dit", local_rank)
-            dy = torch.empty(dbatch.n_tokens, ddims.d_model, dtype=torch.float32, device=dev)
+            dy = torch.empty(dbatch.n_tokens, ddims.d_model, dtype=torch.float32, device=m2.dev)
             db = dit.make_batch(dbatch.q_len, dbatch.ctx_len, dbt, dx, dy)
-            corun_dit_rows = [corun(stage, b, dit, db, bud, max(args.steps // 4, 5)) for bud in wl.SM_BUDGETS["c4_corun"]]
+            corun_dit_rows = [corun(m2.stage, m2.b, dit, db, bud, max(steps2 // 4, 5)) for bud in wl.SM_BUDGETS["c4_corun"]]
             assert dit.status() == 0
             dit.close()
+            m2.close()
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the dominant kernel (gate/up GEMM) -------------------
-    peaks = measured_peaks()
-    gu_ms, gu_n = prof["gemm_gateup"]
-    gu_flops = 2.0 * T * dims.d_model * 2 * dims.d_ffn
-    gu_avg_s = gu_ms * 1e-3 / max(gu_n, 1)
-    achieved = gu_flops / gu_avg_s / 1e12
-    peak = peaks["bf16_sustained"] * budget / stage.sm_count
+    # ---- rooflines ---------------------------------------------------------
+    roofs, roof_meta = rooflines(name, dims, batch, prof, args.steps, ms_step, clocks, budget, stage.sm_count, peaks)
     gemm_flops, attn_flops = flops_per_step(dims, batch)
     gateup_kernel = ("gemm_pair_kernel" if T > 128 and budget >= 2 else
                      "gemm_kernel" if T > 64 else "gemm_kernel or gemm_skinny_kernel (chosen by shape)")
-    roofline = {"bound": "tensor", "kernel": gateup_kernel + " (gate/up + SwiGLU epilogue)", "achieved": achieved,
-                "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                "peak_source": f"{peaks['source']} sustained bf16 (fp16 operands: nominal ratio 1.0) x sm_budget/{stage.sm_count}",
-                "frac_of_burst_peak": achieved / (peaks["bf16_burst"] * budget / stage.sm_count),
-                "traffic": GATEUP_DRAM_TRAFFIC_BYTES.get(name),
-                "avg_launch_ms": gu_avg_s * 1e3, "launches": gu_n,
-                "step_tflops": (gemm_flops + attn_flops) / (ms_step * 1e-3) / 1e12}
+    roofline = dict(roofs.get("gemm_gateup", {}))
+    roofline.update({"kernel": gateup_kernel + " (gate/up + SwiGLU epilogue), the dominant kernel of the step",
+                     "peak_source": f"{peaks['source']} {roof_meta['tensor_peak_used']} bf16 (timed region "
+                                    f"{roof_meta['timed_region_ms']:.0f} ms; fp16 operands: nominal ratio 1.0) "
+                                    f"x sm_budget/{stage.sm_count}",
+                     "traffic": GATEUP_DRAM_TRAFFIC_BYTES.get(name) if not args.layers else None,
+                     "algorithmic_bytes": T * d * 2 + 2 * dims.d_ffn * d * 2 + T * dims.d_ffn * 2,
+                     "step_tflops": (gemm_flops + attn_flops) / (ms_step * 1e-3) / 1e12})
     kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps} for k, v in prof.items()}
-    # decode attention against HBM: K and V pages of every decode sequence once per layer
-    dec_ms, dec_n = prof["attn_decode"]
-    dec_bytes = sum((c + 1) * 2 * dims.kv_dim * 2 for q, c in zip(batch.q_len, batch.ctx_len) if q == 1)
-    decode_roofline = None
-    if dec_n:
-        gbs = dec_bytes / (dec_ms * 1e-3 / dec_n) / 1e9
-        decode_roofline = {"bound": "hbm", "kernel": "attn_decode_kernel", "achieved": gbs,
-                           "peak": peaks["hbm_gbs"] * budget / stage.sm_count, "unit": "GB/s",
-                           "frac": gbs / (peaks["hbm_gbs"] * budget / stage.sm_count),
-                           "bytes_per_launch": dec_bytes, "avg_launch_ms": dec_ms / dec_n,
-                           "note": "bytes below the 126 MB L2 are served from L2, not HBM" if dec_bytes < 126e6 else
-                                   "working set exceeds L2"}
 
     cpu = None
     if not args.no_cpu_baseline:
@@ -459,24 +558,28 @@ def main():
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "vs_baseline": None, "dtype": "bf16" if args.bf16_activations else "f16", "data": "synthetic",
+            "dtype_detail": "all-bf16 operands (HS_FLAG_BF16_ACTIVATIONS); fp32 accumulation" if args.bf16_activations else
+                            "projections: fp16 x fp16 -> fp32 (h, o, act in fp16 against fp16 copies of the bf16 weights); "
+                            "attention: bf16 x bf16 -> fp32 (q, K, V, softmax weights in bf16); fp32 residual stream and "
+                            "output; bf16 x_in, weights and KV cache at the interface",
             "config": {"workload": name + (f" (cut to {args.layers} layers: profiling only)" if args.layers else ""),
                        "n_layers": dims.n_layers, "d_model": d, "n_tokens": T,
                        "n_seqs": batch.n_seqs, "prefill_tokens": int(sum(q for q in batch.q_len if q > 1)),
                        "decode_seqs": int(sum(1 for q in batch.q_len if q == 1)), "sm_budget": budget,
                        "parallelism": f"replicas x{world}" if world > 1 else "single GPU",
-                       "l2": "inputs larger than L2: weights + KV read per step exceed the 126 MB L2",
-                       "formats": "all-bf16 operands (HS_FLAG_BF16_ACTIVATIONS); fp32 accumulation" if
-                                  args.bf16_activations else
-                                  "bf16 x_in, weights, KV cache, q and softmax weights; fp16 h, o, act against fp16 "
-                                  "copies of the weights; fp32 accumulation, residual stream and output"},
+                       "l2": "inputs larger than L2: weights + KV read per step exceed the 126 MB L2"},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e, "h2d_bytes_per_step": T * d * 2,
                     "d2h_bytes_per_step": T * d * 4},
             "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "roofline_decode_attention": decode_roofline, "kernels": kernels,
-            "budget_sweep": sweep, "corun": corun_rows, "corun_dit": corun_dit_rows, "cpu_baseline": cpu}
+            "roofline": roofline, "rooflines": roofs, "roofline_basis": roof_meta,
+            "roofline_decode_attention": roofs.get("attn_decode"), "kernels": kernels,
+            "budget_sweep": sweep, "bf16_path": bf16_leg,
+            "bf16_path_ms_per_step": bf16_leg["ms_per_step"] if bf16_leg else None,
+            "c2_shared": c2_obj, "corun": corun_rows, "corun_dit": corun_dit_rows, "cpu_baseline": cpu}
     print(json.dumps(line))
+    m.close()
     if world > 1:
         dist.destroy_process_group()
 

@@ -223,6 +223,16 @@ hs_status_t hs_stage_set_modulation(hs_stage_t *stage, const void *mod);
 /* Device-side status of the steps run so far (HS_OK or HS_ERR_TIMEOUT); call after synchronising the stream. */
 hs_status_t hs_stage_status(hs_stage_t *stage);
 
+/*
+ * Saturation report of the stage's private fp16 activations.  h, the attention output and the SwiGLU activation
+ * are clamped to +-65504 when they are stored (numeric contract above); *count receives how many stored values
+ * were clamped since the stage was created -- 0 for every well-scaled model, and a signal that the step's output
+ * is no longer within tolerance otherwise (rerun the stage with HS_FLAG_BF16_ACTIVATIONS, whose range is that of
+ * fp32).  Always 0 with that flag.  Call after synchronising the stream.
+ * Errors: INVALID_ARG, NO_DEVICE, CUDA.
+ */
+hs_status_t hs_stage_saturation_count(hs_stage_t *stage, int64_t *count);
+
 /* SM count of the stage's device (S_tot of Eq. 1); 0 for a host-only stage. */
 int32_t hs_stage_sm_count(const hs_stage_t *stage);
 

@@ -70,6 +70,19 @@ hs_status_t hs_stage_profile_enable(hs_stage_t *stage, int32_t enable);
 hs_status_t hs_stage_profile_read(hs_stage_t *stage, float *ms, int32_t *launches);
 
 /*
+ * Diagnosis of the bounded waits (the paper has no counterpart; it concerns this library's kernels only).  Every
+ * wait inside the step's kernels gives up after a time limit, records HS_ERR_TIMEOUT in the device status word
+ * and lets its block wind down in order -- roles leave their loops, copies in flight are given time to land,
+ * tensor memory is freed -- so a lost signal ends as an error code, never as a hung GPU.  This call runs that
+ * sequence on purpose: one small block waits on a barrier that nobody signals, with the caller's limit
+ * (limit_ns nanoseconds, 1 us .. 100 ms) in place of the kernels' 2 s.  After the stream has been synchronised
+ * *status_dev (a device int, zero on entry) holds HS_ERR_TIMEOUT and *waited_ns_dev (device uint64, nullable) the
+ * time the first waiter spent; the context remains usable.
+ * Errors: INVALID_ARG (NULL status, limit out of range), CUDA.
+ */
+hs_status_t hs_op_wait_probe(uint64_t limit_ns, int32_t *status_dev, uint64_t *waited_ns_dev, void *cuda_stream);
+
+/*
  * Decode attention for callers that cannot allocate device memory.  (The paper has no counterpart
  * to this call: it is a packaging variant of the decode-attention kernel of hs_stage_step.)
  *
@@ -78,7 +91,8 @@ hs_status_t hs_stage_profile_read(hs_stage_t *stage, float *ms, int32_t *launche
  * API expects -- an allocation at that point fails or stalls every stream of the GPU.  Here the
  * scratch (split-KV partials, work-queue head, the call's integer metadata, about 4.3 MB) is a fixed
  * array inside the library image; every GPU that loads the library carries it until the process
- * ends.  The call itself allocates nothing, on the device or the host, directly or through a library.
+ * ends.  The call itself calls no allocating routine: no cudaMalloc, cudaFree or cudaHostAlloc, no heap, and no
+ * library that allocates; its host-side metadata lives in a fixed array of the library image.
  *
  * Computes, for each of n_seqs sequences, o[s] = softmax(q[s] K^T / sqrt(head_dim)) V over keys
  * 0 .. kv_len[s]-1 of that sequence (grouped-query: query head h reads KV head h / (n_q_heads /
@@ -95,7 +109,12 @@ hs_status_t hs_stage_profile_read(hs_stage_t *stage, float *ms, int32_t *launche
  * make that first call before any stream capture begins.  All calls share the one scratch area: it
  * keeps the previous call's contents, the parts that must start from zero are cleared by each call,
  * and two calls whose kernels can overlap on the GPU (different streams, no ordering between them)
- * race on it -- order them.  The work is enqueued on cuda_stream; the call does not synchronise.
+ * race on it -- order them.  The work is enqueued on cuda_stream.  The metadata travels by an asynchronous copy
+ * from ordinary (pageable) host memory, so the call may wait on the host until earlier work of that stream has
+ * finished; it does not wait for its own kernel.  Calls from several host threads are serialised inside.
+ * If a bounded wait inside the kernel runs out, the kernel ends in order and records HS_ERR_TIMEOUT in a status
+ * word of the scratch area; hs_op_decode_attention_noalloc_status (after synchronising the stream) copies the
+ * status word of the most recent call to *status_out (HS_OK = 0 when nothing went wrong).
  * Errors: INVALID_ARG, INVALID_BUDGET, UNSUPPORTED_SHAPE, BAD_BLOCK_TABLE, CUDA.
  */
 #define HS_NOALLOC_MAX_SEQS 64
@@ -106,6 +125,7 @@ hs_status_t hs_op_decode_attention_noalloc(const void *q_dev, const void *kv_poo
                                            int32_t n_seqs, const int32_t *kv_len, const int32_t *block_tables,
                                            int32_t max_pages_per_seq, void *o_dev, int32_t sm_budget,
                                            void *cuda_stream);
+hs_status_t hs_op_decode_attention_noalloc_status(int32_t *status_out);
 
 #if defined(__GNUC__)
 #pragma GCC visibility pop

@@ -117,7 +117,11 @@ void hso_rmsnorm(int T, int d, const real *x, const real *g, float eps, real *h)
 /* -------------------------------------------------------------- linear -- */
 /* y[t,n] = sum_i a[t,i] * w[n,i]   (a: [T,K], w: [N,K], y: [T,N]).
  * The token loop is cut into groups of TB rows only so that one weight row
- * is reused from cache; every dot product is the same plain i-loop. */
+ * is reused from cache.  Every dot product is one i-loop over the whole K
+ * range, but not a strictly sequential sum: the simd reduction lets the
+ * compiler keep one partial sum per vector lane and add the lanes at the
+ * end, so the order of the additions is the compiler's (a reassociation
+ * of the same K terms; the float64 build bounds its effect at 1e-6). */
 void hso_linear(int T, int N, int K, const real *a, const real *w, real *y) {
   enum { TB = 16 };
   int n_groups = (T + TB - 1) / TB;

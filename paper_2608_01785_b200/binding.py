@@ -28,7 +28,8 @@ EXPORTS = ("hs_status_str", "hs_kv_pool_bytes", "hs_workspace_bytes", "hs_stage_
            "hs_spatial_create", "hs_spatial_update", "hs_spatial_state", "hs_spatial_destroy",
            "hs_spatial_derive_cap", "hs_head_workspace_bytes", "hs_head_create", "hs_head_step", "hs_head_status",
            "hs_head_destroy", "hs_op_embed", "hs_temporal_create", "hs_temporal_step", "hs_temporal_destroy",
-           "hs_stage_set_qkv_bias", "hs_stage_set_modulation")
+           "hs_stage_set_qkv_bias", "hs_stage_set_modulation", "hs_stage_saturation_count", "hs_op_wait_probe",
+           "hs_op_decode_attention_noalloc_status")
 PROFILE_CLASSES = ("rmsnorm", "gemm_qkv", "attn_prefill", "attn_decode", "attn_combine", "gemm_out", "gemm_gateup",
                    "gemm_down")
 
@@ -139,6 +140,9 @@ def lib() -> C.CDLL:
                                             C.c_double, C.POINTER(C.c_int32)]
         l.hs_op_decode_attention_noalloc.argtypes = [C.c_void_p, C.c_void_p] + [C.c_int32] * 7 + \
             [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p]
+        l.hs_op_decode_attention_noalloc_status.argtypes = [C.POINTER(C.c_int32)]
+        l.hs_stage_saturation_count.argtypes = [C.c_void_p, C.POINTER(C.c_int64)]
+        l.hs_op_wait_probe.argtypes = [C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p]
         l.hs_stage_profile_enable.argtypes = [C.c_void_p, C.c_int32]
         l.hs_stage_set_qkv_bias.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
         l.hs_stage_set_modulation.argtypes = [C.c_void_p, C.c_void_p]
@@ -306,6 +310,32 @@ def hs_op_decode_attention_noalloc(q_ptr: int, kv_pool_ptr: int, n_layers: int, 
                                               C.c_void_p(cuda_stream))
     if st != HS_OK:
         raise HsError(st, "hs_op_decode_attention_noalloc")
+
+
+def hs_op_decode_attention_noalloc_status() -> int:
+    """Device status word of the most recent hs_op_decode_attention_noalloc call (synchronise its stream first)."""
+    v = C.c_int32(-1)
+    st = lib().hs_op_decode_attention_noalloc_status(C.byref(v))
+    if st != HS_OK:
+        raise HsError(st, "hs_op_decode_attention_noalloc_status")
+    return v.value
+
+
+def hs_stage_saturation_count(stage: int) -> int:
+    """How many fp16 activation values the stage has clamped to +-65504 since it was created."""
+    v = C.c_int64(-1)
+    st = lib().hs_stage_saturation_count(C.c_void_p(stage), C.byref(v))
+    if st != HS_OK:
+        raise HsError(st, "hs_stage_saturation_count")
+    return v.value
+
+
+def hs_op_wait_probe(limit_ns: int, status_ptr: int, waited_ns_ptr: int = 0, cuda_stream: int = 0) -> None:
+    """Launches the bounded-wait probe: one block waits limit_ns on a barrier nobody signals, then winds down."""
+    st = lib().hs_op_wait_probe(int(limit_ns), C.c_void_p(status_ptr), C.c_void_p(waited_ns_ptr or None),
+                                C.c_void_p(cuda_stream))
+    if st != HS_OK:
+        raise HsError(st, "hs_op_wait_probe")
 
 
 class SpatialController:

@@ -8,7 +8,7 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libhorizonserve.so")
-SOURCES = ["api.cu", "gemm.cu", "gemm_skinny.cu", "attention.cu", "attention_prefill.cu", "norm.cu", "noalloc.cu", "head.cu", "plan.cc", "control.cc"]
+SOURCES = ["api.cu", "gemm.cu", "gemm_skinny.cu", "attention.cu", "attention_prefill.cu", "norm.cu", "noalloc.cu", "diag.cu", "head.cu", "plan.cc", "control.cc"]
 HEADERS = ["hs_internal.h", "kernels.h", "ptx.cuh", os.path.join("..", "..", "include", "horizonserve.h"),
            os.path.join("..", "..", "include", "horizonserve_ops.h"),
            os.path.join("..", "..", "include", "horizonserve_control.h"),

@@ -3,6 +3,7 @@
 #include <string.h>
 
 #include <memory>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -119,6 +120,12 @@ hs_status_t cuda_fail(const char* where, cudaError_t e) {
   return HS_ERR_CUDA;
 }
 
+// Records a failure that has no CUDA error code behind it; returns HS_ERR_CUDA.
+hs_status_t fail(const char* what) {
+  g_last_error = what;
+  return HS_ERR_CUDA;
+}
+
 // K splits for a residual GEMM, or 1 when the whose-turn array could not hold its tiles.
 int pick_ksplit(int M, int N, int K, int bn, int sm_count) {
   const int tiles = ceil_div(M, 128) * ceil_div(N, bn);
@@ -133,8 +140,12 @@ bool device_info(int dev, int* sm_count, int* major) {
          cudaDeviceGetAttribute(major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess;
 }
 
+// Stages may be created and ops called from several host threads (the co-run harness drives each stage from its
+// own thread): the table and the attribute calls behind it are serialised.
+std::mutex g_attrs_mutex;
 bool g_attrs_set[64] = {};
 hs_status_t ensure_attributes(int device) {
+  std::lock_guard<std::mutex> lock(g_attrs_mutex);
   if (device >= 0 && device < 64 && g_attrs_set[device]) return HS_OK;
   cudaError_t e;
   if ((e = gemm_set_attributes()) != cudaSuccess) return cuda_fail("gemm attributes", e);
@@ -271,11 +282,12 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
   }
 
   DeviceGuard guard(cfg->device);
-  if (!guard.ok) return HS_ERR_CUDA;
-  cudaDeviceProp prop;
-  if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return HS_ERR_CUDA;
-  if (prop.major != 10) return HS_ERR_CUDA;   // the kernels exist for sm_100a only
-  s->sm_count = prop.multiProcessorCount;
+  if (!guard.ok) return fail("hs_stage_create: cannot make the configured device current");
+  int sm_count = 0, major = 0;
+  if (!device_info(cfg->device, &sm_count, &major)) return fail("hs_stage_create: device attribute query failed");
+  if (major != 10)   // the kernels exist for sm_100a only
+    return fail("hs_stage_create: the device is not compute capability 10.x; the kernels are built for sm_100a only");
+  s->sm_count = sm_count;
   if ((st = ensure_attributes(cfg->device)) != HS_OK) return st;
   s->ws_dev = static_cast<uint8_t*>(workspace_dev);
   s->kv_pool = static_cast<__nv_bfloat16*>(kv_pool_dev);
@@ -295,7 +307,7 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
           cudaSuccess ||
       cudaMemset(s->ws_dev + s->ws.status, 0, 256) != cudaSuccess ||
       cudaMemset(s->ws_dev + s->ws.turn, 0, kGemmTurnWords * 4) != cudaSuccess)
-    return HS_ERR_CUDA;
+    return cuda_fail("hs_stage_create: workspace initialisation", cudaGetLastError());
 
   // tensor maps
   const uint64_t T = cfg->max_tokens, d = cfg->d_model, F = cfg->d_ffn;
@@ -337,19 +349,23 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
          encode_2d(&m.wgate, w.w_gate, F, d, 128) && encode_2d(&m.wup, w.w_up, F, d, 128) &&
          encode_2d(&m.wdown, w.w_down, d, F, 128);
   }
-  if (!ok) return HS_ERR_CUDA;
+  if (!ok)
+    return fail("hs_stage_create: fp16 weight copy or tensor-map encoding failed (cuTensorMapEncodeTiled unavailable, or "
+                "a matrix whose row pitch is not a multiple of 16 bytes)");
 
   for (int i = 0; i < kRing; ++i) {
     if (cudaHostAlloc(reinterpret_cast<void**>(&s->pinned[i]), size_t(s->ml.total) * 4, cudaHostAllocDefault) !=
             cudaSuccess ||
         cudaEventCreateWithFlags(&s->ev[i], cudaEventDisableTiming) != cudaSuccess) {
+      const cudaError_t e = cudaGetLastError();
       hs_stage_destroy(s.release());
-      return HS_ERR_CUDA;
+      return cuda_fail("hs_stage_create: pinned staging or event creation", e);
     }
   }
-  if (cudaDeviceSynchronize() != cudaSuccess) {
+  const cudaError_t sync_err = cudaDeviceSynchronize();
+  if (sync_err != cudaSuccess) {
     hs_stage_destroy(s.release());
-    return HS_ERR_CUDA;
+    return cuda_fail("hs_stage_create: device synchronisation", sync_err);
   }
   *out = s.release();
   return HS_OK;
@@ -480,6 +496,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     SkinnyParams k{};
     k.a = a; k.T = T; k.K = K; k.N = N; k.mode = mode;
     k.ab_f16 = f16; k.overlap = overlap;
+    k.status = status;
     return k;
   };
   int* census = s->census ? reinterpret_cast<int*>(s->ws_dev + s->ws.smid) : nullptr;
@@ -682,6 +699,16 @@ hs_status_t hs_stage_status(hs_stage_t* s) {
   return v == 0 ? HS_OK : static_cast<hs_status_t>(v);
 }
 
+hs_status_t hs_stage_saturation_count(hs_stage_t* s, int64_t* count) {
+  if (!s || !count) return HS_ERR_INVALID_ARG;
+  if (s->cfg.device < 0) return HS_ERR_NO_DEVICE;
+  DeviceGuard guard(s->cfg.device);
+  int v = 0;
+  if (cudaMemcpy(&v, s->ws_dev + s->ws.status + 4, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return HS_ERR_CUDA;
+  *count = int64_t(uint32_t(v));
+  return HS_OK;
+}
+
 hs_status_t hs_stage_profile_enable(hs_stage_t* s, int32_t enable) {
   if (!s) return HS_ERR_INVALID_ARG;
   if (s->cfg.device < 0) return HS_ERR_NO_DEVICE;
@@ -819,14 +846,15 @@ hs_status_t hs_head_create(const hs_head_config_t* cfg, const void* g_final, con
     return HS_ERR_INVALID_ARG;
   DeviceGuard guard(cfg->device);
   if (!guard.ok) return HS_ERR_CUDA;
-  cudaDeviceProp prop;
-  if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess || prop.major != 10) return HS_ERR_CUDA;
+  int sm_count = 0, major = 0;
+  if (!device_info(cfg->device, &sm_count, &major)) return fail("hs_head_create: device attribute query failed");
+  if (major != 10) return fail("hs_head_create: the device is not compute capability 10.x");
   hs_status_t st = ensure_attributes(cfg->device);
   if (st != HS_OK) return st;
   std::unique_ptr<hs_head> h(new (std::nothrow) hs_head());
   if (!h) return HS_ERR_INVALID_ARG;
   h->cfg = *cfg;
-  h->sm_count = prop.multiProcessorCount;
+  h->sm_count = sm_count;
   h->ws_dev = static_cast<uint8_t*>(workspace_dev);
   h->off_status = head_status_offset(*cfg);
   h->g_final = static_cast<const __nv_bfloat16*>(g_final);

@@ -71,7 +71,7 @@ __device__ __forceinline__ uint32_t mask_v(uint32_t r, int k, int n_valid) {
 // The running maximum is updated per half (online rescaling); the order of all operations is fixed.
 template <int DH, int LPH, int RING_BYTES>
 __device__ __forceinline__ void merge_group(const float* part_o, const float* part_ml, uint8_t* ring, int first,
-                                            int splits, int G, int lane, __nv_bfloat16* orow, bool f16) {
+                                            int splits, int G, int lane, __nv_bfloat16* orow, bool f16, int* status) {
   constexpr int NV = DH / 4 / LPH;                 // float4 per lane and split
   constexpr int PS = RING_BYTES / 2 / (NV * 512) < 4 ? RING_BYTES / 2 / (NV * 512) : 4;   // splits per half
   static_assert(PS >= 1, "half a ring holds one split");
@@ -136,6 +136,13 @@ __device__ __forceinline__ void merge_group(const float* part_o, const float* pa
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     const float inv = 1.f / ll;
+    if (f16) {
+#pragma unroll
+      for (int i = 0; i < NV; ++i) {
+        const float v4[4] = {acc[i].x, acc[i].y, acc[i].z, acc[i].w};
+        note_f16_saturation(v4, status, inv);
+      }
+    }
     __nv_bfloat16* dst = orow + g * DH + part * NV * 4;
 #pragma unroll
     for (int i = 0; i < NV; ++i)
@@ -332,6 +339,23 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
     if (splits == 1) {
       // the whole key range was this item: normalise and write the output rows directly
       const float inv_a = 1.f / l_a, inv_b = 1.f / l_b;
+      if (p.o_f16) {                        // saturation report of the fp16 output (see note_f16_saturation)
+        float mx_oa = 0.f, mx_ob = 0.f;
+#pragma unroll
+        for (int j = 0; j < DH / 8; ++j) {
+          mx_oa = fmaxf(mx_oa, fmaxf(fabsf(o_acc[j][0]), fabsf(o_acc[j][1])));
+          mx_ob = fmaxf(mx_ob, fmaxf(fabsf(o_acc[j][2]), fabsf(o_acc[j][3])));
+        }
+        if ((ra < G && mx_oa * inv_a > 65504.f) || (rb < G && mx_ob * inv_b > 65504.f)) {
+          int c = 0;
+#pragma unroll
+          for (int j = 0; j < DH / 8; ++j) {
+            if (ra < G) c += (fabsf(o_acc[j][0] * inv_a) > 65504.f) + (fabsf(o_acc[j][1] * inv_a) > 65504.f);
+            if (rb < G) c += (fabsf(o_acc[j][2] * inv_b) > 65504.f) + (fabsf(o_acc[j][3] * inv_b) > 65504.f);
+          }
+          atomicAdd(p.status + 1, c);
+        }
+      }
 #pragma unroll
       for (int j = 0; j < DH / 8; ++j) {
         const int col = 8 * j + 2 * (lane & 3);
@@ -364,8 +388,8 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
     if (last) {
       __threadfence();
       const int first = dr.z;
-      if (G <= 8) merge_group<DH, 4, DC_STAGES * SLOT_BYTES>(p.part_o, p.part_ml, slots, first, splits, G, lane, orow, p.o_f16 != 0);
-      else merge_group<DH, 2, DC_STAGES * SLOT_BYTES>(p.part_o, p.part_ml, slots, first, splits, G, lane, orow, p.o_f16 != 0);
+      if (G <= 8) merge_group<DH, 4, DC_STAGES * SLOT_BYTES>(p.part_o, p.part_ml, slots, first, splits, G, lane, orow, p.o_f16 != 0, p.status);
+      else merge_group<DH, 2, DC_STAGES * SLOT_BYTES>(p.part_o, p.part_ml, slots, first, splits, G, lane, orow, p.o_f16 != 0, p.status);
       if (lane == 0) *done = 0;             // ready for the next launch
     }
   }

@@ -1,19 +1,26 @@
 // Causal GQA attention for prefill chunks on the 5th-generation tensor cores.
 //
-//   work item   (sequence, KV head, tile of Mt tokens), Mt = 128 / G rounded down to a multiple of 8.  The G
-//               query heads that share the KV head are stacked head-major as rows of one 128-row tile
-//               (row = head * Mt + token), so K and V are streamed once per KV head.
-//   per block   of 64 keys:  S = Q K^T (tcgen05.mma, M128 N64, fp32 in tensor memory)  ->  softmax warps
-//               (one thread per row: no shuffles) read S, scale, mask by selection, keep the running max and
-//               sum in the log2 domain, write P as bf16 into a swizzled shared-memory tile  ->  O_blk = P V
-//               (tcgen05.mma, M128 N=Dh, V used in place as an MN-major operand)  ->  the same threads fold
-//               O_blk into fp32 registers: o = o * exp2(m_old - m_new) + O_blk.
-//   pipeline    S, P and O_blk are double buffered, so the MMA warp computes S of block j+1 while the
-//               softmax warps work on block j; K/V pages arrive by TMA in a 4-stage ring ([half][page][16][64]
-//               tiles with the 128-byte swizzle, the K tile being a K-major and the V tile an MN-major
-//               operand); the producer owns the work queue and runs ahead across items.
-//   roles       warps 0..3 softmax / correction (thread = row = TMEM lane), warp 4 TMA producer, warp 5 MMA
-//               issuer and TMEM owner.
+//   work item   (sequence, KV head, up to 2 Mt consecutive tokens), Mt = 128 / G rounded down to a multiple of 8.
+//               The item is two Q tiles: tile A holds its first Mt tokens, tile B the rest.  In a tile the G query
+//               heads that share the KV head are stacked head-major as rows of a 128-row tile (row = head * Mt +
+//               token).  Both tiles read the same K / V blocks, which are staged once for the two of them.
+//   per block   of 64 keys and per tile:  S = Q K^T (tcgen05.mma, M128 N64, fp32 in tensor memory)  ->  the tile's
+//               softmax warp group (one thread per row: no shuffles) reads S, masks by selection, exponentiates
+//               in the log2 domain against a per-row reference maximum, writes P as bf16 into a swizzled
+//               shared-memory tile  ->  O += P V (tcgen05.mma, M128 N = Dh, V used in place as an MN-major
+//               operand).  O stays in tensor memory for the whole item; it is read once, at the item's end.
+//   reference   A row's reference maximum follows its running maximum lazily: it moves only when the running
+//   maximum     maximum exceeds it by more than 8 (in log2 units, a factor of 256), and only then is the row of O
+//               rescaled (tcgen05.ld / multiply / tcgen05.st by the softmax threads, while no P V product of the
+//               tile is in flight).  P and the running sum use the same reference, so the quotient O / l at the
+//               end is exact whatever reference was used; values stay far inside the range of bf16 and fp32.
+//   pipeline    two tiles x two S buffers x two P buffers: while one tile's warp group exponentiates, the tensor
+//               core works on the other tile's products.  K and V blocks arrive by TMA in two rings of their own
+//               ([half][page][16][64] tiles with the 128-byte swizzle, the K tile being a K-major and the V tile an
+//               MN-major operand): a K slot is free again as soon as the block's scores are computed, a V slot
+//               after its P V products.  The producer owns the work queue and runs ahead across items.
+//   roles       warps 0..3 softmax of tile A, warps 4..7 softmax of tile B (thread = row = TMEM lane), warp 8 TMA
+//               producer, warp 9 MMA issuer and TMEM owner.
 // Keys past the end of a sequence are masked by selection on the key index, and the matching V rows are
 // zeroed in shared memory before the P V product, so arbitrary bytes in unused cache slots cannot reach
 // the output.  An item's result does not depend on which block ran it: outputs are budget independent.
@@ -26,30 +33,33 @@ namespace hs {
 namespace {
 
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int PF_THREADS = 192, PF_STAGES = 3, PF_KEYS = 64;
+constexpr int PF_THREADS = 320, PF_KEYS = 64;
+constexpr int PF_KSTAGES = 3, PF_VSTAGES = 3;
 constexpr int TMEM_COLS = 512;
+constexpr float kRefSlack = 8.f;   // log2 units by which a row's running maximum may exceed its reference
 
 template <int DH>
 struct Geom {
   static constexpr int HALVES = DH / 64;
-  static constexpr int Q_BYTES = HALVES * 16384;        // [half][128 rows][128 B]
-  static constexpr int KV_BYTES = HALVES * 8192;        // K (or V) of one stage: [half][4 pages][16 keys][128 B]
-  static constexpr int STAGE_BYTES = 2 * KV_BYTES;
+  static constexpr int Q_BYTES = HALVES * 16384;        // one tile: [half][128 rows][128 B]
+  static constexpr int KV_BYTES = HALVES * 8192;        // K (or V) of one block: [half][4 pages][16 keys][128 B]
   static constexpr int P_BYTES = 16384;                 // [128 rows][64 keys] bf16
-  static constexpr int SMEM = 1024 + 2 * Q_BYTES + PF_STAGES * STAGE_BYTES + 2 * P_BYTES + 512;
-  // tensor-memory columns
-  static constexpr int S0 = 0, O0 = 128;                // S buffers at 0 / 64, O_blk buffers at 128 / 128 + DH
+  static constexpr int SMEM = 1024 + 2 * Q_BYTES + (PF_KSTAGES + PF_VSTAGES) * KV_BYTES + 4 * P_BYTES + 1024;
+  // tensor-memory columns: S(tile, buffer) at tile * 128 + buffer * 64; O(tile) at 256 + tile * DH
+  static constexpr int S0 = 0, O0 = 256;
 };
+static_assert(Geom<128>::SMEM <= 227 * 1024, "fits one SM");
 
 struct Barriers {
-  uint64_t q_full[2], q_empty[2];
-  uint64_t kv_full[PF_STAGES], kv_empty[PF_STAGES];
-  uint64_t s_full[2], s_empty[2], p_full[2], o_full[2], o_empty[2];
+  uint64_t q_full, q_empty;
+  uint64_t k_full[PF_KSTAGES], k_empty[PF_KSTAGES], v_full[PF_VSTAGES], v_empty[PF_VSTAGES];
+  uint64_t s_full[2][2], s_empty[2][2], p_full[2][2], o_full[2];
   uint64_t ring_full[2], ring_empty[2];
   int ring_item[2];
   uint32_t tmem_base;
   int abort_flag;
 };
+static_assert(sizeof(Barriers) <= 1024, "barrier block");
 
 __device__ __forceinline__ int pool_row(const AttnParams& p, int kv, int page, int hk) {
   return (((p.layer * 2 + kv) * p.num_pages + page) * p.n_kv_heads + hk) * 16;
@@ -71,16 +81,56 @@ __device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t smem_addr, 
   d |= static_cast<uint64_t>(2) << 61;
   return d;
 }
+// 32 lanes x 32 consecutive 32-bit columns, registers -> tensor memory (the inverse of tmem_ld32).
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Geometry of one item, the same in every role.
+struct ItemView {
+  int seq, hk, tok_begin, n_tok;     // the item record
+  int tok0, pos0, ctx;               // first token row of tile A, its absolute position, cached tokens
+  int n_tok_t[2];                    // tokens of tile A / B (0 = tile absent)
+  int n_keys;                        // keys the item's K / V blocks cover (valid cache rows)
+  int nblk_t[2], nblk;               // key blocks per tile and of the item
+};
+__device__ __forceinline__ ItemView view_item(const AttnParams& p, int item, int Mt) {
+  const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
+  ItemView v;
+  v.seq = it.x; v.hk = it.y; v.tok_begin = it.z; v.n_tok = it.w;
+  v.ctx = p.seq_ctx[v.seq];
+  v.tok0 = p.seq_tok0[v.seq] + v.tok_begin;
+  v.pos0 = v.ctx + v.tok_begin;
+  v.n_tok_t[0] = min(v.n_tok, Mt);
+  v.n_tok_t[1] = v.n_tok - v.n_tok_t[0];
+  const int all = v.ctx + p.seq_qlen[v.seq];
+  v.n_keys = p.bidirectional ? all : v.pos0 + v.n_tok;
+  const int keys_a = p.bidirectional ? all : v.pos0 + v.n_tok_t[0];
+  v.nblk_t[0] = (keys_a + PF_KEYS - 1) / PF_KEYS;
+  v.nblk_t[1] = v.n_tok_t[1] > 0 ? (v.n_keys + PF_KEYS - 1) / PF_KEYS : 0;
+  v.nblk = max(v.nblk_t[0], v.nblk_t[1]);
+  return v;
+}
 
 template <int DH>
 __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __grid_constant__ AttnParams p) {
   using G_ = Geom<DH>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* q_smem = smem;
-  uint8_t* stages = q_smem + 2 * G_::Q_BYTES;       // two Q tiles: the next item's tile loads early
-  uint8_t* p_smem = stages + PF_STAGES * G_::STAGE_BYTES;
-  Barriers* bar = reinterpret_cast<Barriers*>(p_smem + 2 * G_::P_BYTES);
+  uint8_t* q_smem = smem;                                   // tile A then tile B
+  uint8_t* k_smem = q_smem + 2 * G_::Q_BYTES;
+  uint8_t* v_smem = k_smem + PF_KSTAGES * G_::KV_BYTES;
+  uint8_t* p_smem = v_smem + PF_VSTAGES * G_::KV_BYTES;     // [tile][buffer]
+  Barriers* bar = reinterpret_cast<Barriers*>(p_smem + 4 * G_::P_BYTES);
   volatile int* abort_flag = &bar->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -91,29 +141,28 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
   const float scale_log2 = kLog2e / sqrtf(float(DH));
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&bar->q_full[i], 1);
-      mbar_init(&bar->q_empty[i], 1);
+    mbar_init(&bar->q_full, 1);
+    mbar_init(&bar->q_empty, 1);
+    for (int i = 0; i < PF_KSTAGES; ++i) { mbar_init(&bar->k_full[i], 1); mbar_init(&bar->k_empty[i], 1); }
+    for (int i = 0; i < PF_VSTAGES; ++i) { mbar_init(&bar->v_full[i], 1); mbar_init(&bar->v_empty[i], 1); }
+    for (int t = 0; t < 2; ++t) {
+      for (int i = 0; i < 2; ++i) {
+        mbar_init(&bar->s_full[t][i], 1);
+        mbar_init(&bar->s_empty[t][i], 128);
+        mbar_init(&bar->p_full[t][i], 128);
+      }
+      mbar_init(&bar->o_full[t], 1);
     }
-    for (int i = 0; i < PF_STAGES; ++i) {
-      mbar_init(&bar->kv_full[i], 1);
-      mbar_init(&bar->kv_empty[i], 1);
-    }
     for (int i = 0; i < 2; ++i) {
-      mbar_init(&bar->s_full[i], 1);
-      mbar_init(&bar->s_empty[i], 128);
-      mbar_init(&bar->p_full[i], 128);
-      mbar_init(&bar->o_full[i], 1);
-      mbar_init(&bar->o_empty[i], 128);
       mbar_init(&bar->ring_full[i], 1);
-      mbar_init(&bar->ring_empty[i], 5);    // four softmax warps + the MMA warp
+      mbar_init(&bar->ring_empty[i], 9);      // eight softmax warps + the MMA warp
     }
     bar->abort_flag = 0;
     fence_barrier_init();
     tma_prefetch_desc(&p.tm_kv);
     tma_prefetch_desc(&p.tm_q);
   }
-  if (warp == 5) {
+  if (warp == 9) {
     tmem_alloc(&bar->tmem_base, TMEM_COLS);
     tmem_relinquish();
   }
@@ -126,10 +175,10 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
 
   int rs = 0;
   uint32_t rph = 0;       // item ring slot / phase
-  uint32_t gblk = 0;      // key blocks processed so far by this thread's role, over all items
   uint32_t n_items_seen = 0;
+  uint32_t blk_base = 0;  // key blocks of all earlier items of this thread block (K / V ring position)
 
-  if (warp == 4) {
+  if (warp == 8) {
     // =========================================================== TMA producer ==
     if (lane == 0) {
       for (;;) {
@@ -139,62 +188,72 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         mbar_arrive(&bar->ring_full[rs]);
         if (++rs == 2) { rs = 0; rph ^= 1; }
         if (item >= p.n_prefill_items) break;
-        const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
-        const int seq = it.x, hk = it.y, tok_begin = it.z, n_tok = it.w;
-        const int tok0 = p.seq_tok0[seq] + tok_begin;
-        const int n_keys = p.seq_ctx[seq] + (p.bidirectional ? p.seq_qlen[seq] : tok_begin + n_tok);
-        const int n_kblocks = (n_keys + PF_KEYS - 1) / PF_KEYS;
-        const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq;
-        // Q tile: one box of Mt token rows x 64 columns per (head, half)
-        const uint32_t qb = n_items_seen & 1;
-        if (!mbar_wait(&bar->q_empty[qb], ((n_items_seen >> 1) & 1) ^ 1, abort_flag, p.status)) break;
-        mbar_expect_tx(&bar->q_full[qb], G * G_::HALVES * Mt * 128);
-        for (int g = 0; g < G; ++g)
-          for (int h = 0; h < G_::HALVES; ++h)
-            tma_load_2d(q_smem + qb * G_::Q_BYTES + h * 16384 + g * Mt * 128, &p.tm_q, &bar->q_full[qb],
-                        (hk * G + g) * DH + h * 64, tok0);
+        const ItemView v = view_item(p, item, Mt);
+        const int32_t* table = p.block_tables + size_t(v.seq) * p.max_pages_per_seq;
+        // Q tiles: one box of Mt token rows x 64 columns per (tile, head, half)
+        if (!mbar_wait(&bar->q_empty, (n_items_seen & 1) ^ 1, abort_flag, p.status)) break;
+        const int n_tiles = v.n_tok_t[1] > 0 ? 2 : 1;
+        mbar_expect_tx(&bar->q_full, n_tiles * G * G_::HALVES * Mt * 128);
+        for (int t = 0; t < n_tiles; ++t)
+          for (int g = 0; g < G; ++g)
+            for (int h = 0; h < G_::HALVES; ++h)
+              tma_load_2d(q_smem + t * G_::Q_BYTES + h * 16384 + g * Mt * 128, &p.tm_q, &bar->q_full,
+                          (v.hk * G + g) * DH + h * 64, v.tok0 + t * Mt);
         ++n_items_seen;
         bool ok = true;
-        for (int kb = 0; kb < n_kblocks; ++kb, ++gblk) {
-          const int s = gblk % PF_STAGES;
-          if (!mbar_wait(&bar->kv_empty[s], ((gblk / PF_STAGES) & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
-          const int rem = n_keys - kb * PF_KEYS;
+        for (int kb = 0; kb < v.nblk && ok; ++kb) {
+          const uint32_t gb = blk_base + kb;
+          const int rem = v.n_keys - kb * PF_KEYS;
           const int np = rem >= PF_KEYS ? 4 : (rem + 15) >> 4;
-          uint8_t* st = stages + s * G_::STAGE_BYTES;
-          mbar_expect_tx(&bar->kv_full[s], np * 2 * G_::HALVES * 2048);
-          for (int w = 0; w < np; ++w) {
-            const int page = table[kb * 4 + w];
-            const int krow = pool_row(p, 0, page, hk), vrow = pool_row(p, 1, page, hk);
-            for (int h = 0; h < G_::HALVES; ++h) {
-              tma_load_2d(st + h * 8192 + w * 2048, &p.tm_kv, &bar->kv_full[s], h * 64, krow);
-              tma_load_2d(st + G_::KV_BYTES + h * 8192 + w * 2048, &p.tm_kv, &bar->kv_full[s], h * 64, vrow);
+          for (int kv = 0; kv < 2 && ok; ++kv) {
+            const uint32_t st = gb % (kv ? PF_VSTAGES : PF_KSTAGES), ph = (gb / (kv ? PF_VSTAGES : PF_KSTAGES)) & 1;
+            uint64_t* full = kv ? &bar->v_full[st] : &bar->k_full[st];
+            if (!mbar_wait(kv ? &bar->v_empty[st] : &bar->k_empty[st], ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+            uint8_t* dst = (kv ? v_smem : k_smem) + st * G_::KV_BYTES;
+            mbar_expect_tx(full, np * G_::HALVES * 2048);
+            for (int w = 0; w < np; ++w) {
+              const int row = pool_row(p, kv, table[kb * 4 + w], v.hk);
+              for (int h = 0; h < G_::HALVES; ++h) tma_load_2d(dst + h * 8192 + w * 2048, &p.tm_kv, full, h * 64, row);
             }
           }
         }
         if (!ok) break;
+        blk_base += v.nblk;
       }
     }
-  } else if (warp == 5) {
+  } else if (warp == 9) {
     // ============================================================= MMA issuer ==
     if (lane == 0) {
       constexpr uint32_t idesc_s = umma_idesc_bf16_f32(128, PF_KEYS);
       constexpr uint32_t idesc_pv = umma_idesc_bf16_f32(128, DH) | (1u << 16);   // B (= V) is MN-major
-      const uint32_t q_addr = smem_u32(q_smem), st_addr = smem_u32(stages), p_addr = smem_u32(p_smem);
-      // O_blk(buffer of block b) = P(buffer) * V(stage of block b)
-      auto issue_pv = [&](uint32_t b) -> bool {
-        const uint32_t buf = b & 1, bph = (b >> 1) & 1, s = b % PF_STAGES;
-        if (!mbar_wait(&bar->p_full[buf], bph, abort_flag, p.status)) return false;
-        if (!mbar_wait(&bar->o_empty[buf], bph ^ 1, abort_flag, p.status)) return false;
+      const uint32_t q_addr = smem_u32(q_smem), k_addr0 = smem_u32(k_smem), v_addr0 = smem_u32(v_smem),
+                     p_addr = smem_u32(p_smem);
+      uint32_t g_t[2] = {0, 0};          // blocks of each tile whose S has been issued, over all items
+      uint32_t pv_t[2] = {0, 0};         // blocks of each tile whose P V has been issued
+      bool ok = true;
+      // O(tile) (+)= P(tile, buffer) * V(block gb); `first` = first block of the item (overwrites O)
+      auto issue_pv = [&](int t, uint32_t gb, bool first) -> bool {
+        const uint32_t c = pv_t[t], buf = c & 1, bph = (c >> 1) & 1;
+        if (!mbar_wait(&bar->p_full[t][buf], bph, abort_flag, p.status)) return false;
         tc_fence_after_sync();
-        const uint32_t v_addr = st_addr + s * G_::STAGE_BYTES + G_::KV_BYTES;
+        const uint32_t v_addr = v_addr0 + (gb % PF_VSTAGES) * G_::KV_BYTES;
 #pragma unroll
         for (int pg = 0; pg < 4; ++pg) {      // 16 keys (one page) per MMA
-          const uint64_t a = umma_desc_kmajor_sw128(p_addr + buf * G_::P_BYTES) + 2 * pg;
+          const uint64_t a = umma_desc_kmajor_sw128(p_addr + (t * 2 + buf) * G_::P_BYTES) + 2 * pg;
           const uint64_t bdesc = umma_desc_mnmajor_sw128(v_addr + pg * 2048, 8192, 1024);
-          umma_bf16(tmem + G_::O0 + buf * DH, a, bdesc, idesc_pv, pg != 0);
+          umma_bf16(tmem + G_::O0 + t * DH, a, bdesc, idesc_pv, (pg != 0 || !first) ? 1u : 0u);
         }
-        umma_commit(&bar->o_full[buf]);
-        umma_commit(&bar->kv_empty[s]);
+        umma_commit(&bar->o_full[t]);
+        ++pv_t[t];
+        return true;
+      };
+      // P V products of block j of the current item, both tiles, then the V slot goes back to the producer
+      auto issue_pv_block = [&](const ItemView& v, int j) -> bool {
+        const uint32_t gb = blk_base + j;
+        if (!mbar_wait(&bar->v_full[gb % PF_VSTAGES], (gb / PF_VSTAGES) & 1, abort_flag, p.status)) return false;
+        for (int t = 0; t < 2; ++t)
+          if (j < v.nblk_t[t] && !issue_pv(t, gb, j == 0)) return false;
+        umma_commit(&bar->v_empty[gb % PF_VSTAGES]);
         return true;
       };
       for (;;) {
@@ -203,36 +262,44 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         mbar_arrive(&bar->ring_empty[rs]);
         if (++rs == 2) { rs = 0; rph ^= 1; }
         if (item >= p.n_prefill_items) break;
-        const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
-        const int n_keys = p.seq_ctx[it.x] + (p.bidirectional ? p.seq_qlen[it.x] : it.z + it.w);
-        const int n_kblocks = (n_keys + PF_KEYS - 1) / PF_KEYS;
-        const uint32_t qb = n_items_seen & 1;
-        if (!mbar_wait(&bar->q_full[qb], (n_items_seen >> 1) & 1, abort_flag, p.status)) break;
+        const ItemView v = view_item(p, item, Mt);
+        if (!mbar_wait(&bar->q_full, n_items_seen & 1, abort_flag, p.status)) break;
         ++n_items_seen;
-        bool ok = true;
-        for (int j = 0; j < n_kblocks && ok; ++j, ++gblk) {
-          const uint32_t buf = gblk & 1, bph = (gblk >> 1) & 1, s = gblk % PF_STAGES;
-          if (!mbar_wait(&bar->kv_full[s], (gblk / PF_STAGES) & 1, abort_flag, p.status)) { ok = false; break; }
-          if (!mbar_wait(&bar->s_empty[buf], bph ^ 1, abort_flag, p.status)) { ok = false; break; }
-          tc_fence_after_sync();
-          const uint32_t k_addr = st_addr + s * G_::STAGE_BYTES;
+        for (int j = 0; j < v.nblk && ok; ++j) {
+          const uint32_t gb = blk_base + j, kst = gb % PF_KSTAGES;
+          if (!mbar_wait(&bar->k_full[kst], (gb / PF_KSTAGES) & 1, abort_flag, p.status)) { ok = false; break; }
+          for (int t = 0; t < 2 && ok; ++t) {
+            if (j >= v.nblk_t[t]) continue;
+            const uint32_t buf = g_t[t] & 1, bph = (g_t[t] >> 1) & 1;
+            if (!mbar_wait(&bar->s_empty[t][buf], bph ^ 1, abort_flag, p.status)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t k_addr = k_addr0 + kst * G_::KV_BYTES;
 #pragma unroll
-          for (int ks = 0; ks < DH / 16; ++ks) {
-            const uint64_t a = umma_desc_kmajor_sw128(q_addr + qb * G_::Q_BYTES + (ks >> 2) * 16384) + 2 * (ks & 3);
-            const uint64_t b = umma_desc_kmajor_sw128(k_addr + (ks >> 2) * 8192) + 2 * (ks & 3);
-            umma_bf16(tmem + G_::S0 + buf * PF_KEYS, a, b, idesc_s, ks != 0);
+            for (int ks = 0; ks < DH / 16; ++ks) {
+              const uint64_t a = umma_desc_kmajor_sw128(q_addr + t * G_::Q_BYTES + (ks >> 2) * 16384) + 2 * (ks & 3);
+              const uint64_t b = umma_desc_kmajor_sw128(k_addr + (ks >> 2) * 8192) + 2 * (ks & 3);
+              umma_bf16(tmem + G_::S0 + t * 128 + buf * PF_KEYS, a, b, idesc_s, ks != 0);
+            }
+            umma_commit(&bar->s_full[t][buf]);
+            ++g_t[t];
           }
-          umma_commit(&bar->s_full[buf]);
-          if (j == n_kblocks - 1) umma_commit(&bar->q_empty[qb]);   // this Q tile may be replaced once these are done
-          if (j > 0) ok = issue_pv(gblk - 1);                      // overlaps the softmax of block j
+          if (!ok) break;
+          umma_commit(&bar->k_empty[kst]);                          // the K slot, once these scores are computed
+          if (j == v.nblk - 1) umma_commit(&bar->q_empty);          // and the Q tiles after the item's last scores
+          if (j > 0) ok = issue_pv_block(v, j - 1);                 // overlaps the softmax of block j
         }
-        if (!ok || !issue_pv(gblk - 1)) break;
+        if (!ok || !issue_pv_block(v, v.nblk - 1)) break;
+        blk_base += v.nblk;
       }
     }
   } else {
-    // ================================================= softmax and correction ==
-    const int r = threadIdx.x;                    // row of the tile = TMEM lane
-    const uint32_t lane_base = uint32_t(warp * 32) << 16;
+    // ================================================================ softmax ==
+    const int t = warp >> 2;                      // tile of this warp group
+    const int r = threadIdx.x & 127;              // row of the tile = TMEM lane
+    const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
+    const uint32_t s_col = G_::S0 + t * 128, o_col = G_::O0 + t * DH;
+    uint8_t* p_tile = p_smem + t * 2 * G_::P_BYTES;
+    uint32_t g = 0;                               // blocks this tile has processed, over all items
     for (;;) {
       bool ok = mbar_wait(&bar->ring_full[rs], rph, abort_flag, p.status);
       if (!__all_sync(0xffffffffu, ok)) break;
@@ -241,57 +308,27 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
       if (lane == 0) mbar_arrive(&bar->ring_empty[rs]);
       if (++rs == 2) { rs = 0; rph ^= 1; }
       if (item >= p.n_prefill_items) break;
-      const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
-      const int seq = it.x, hk = it.y, tok_begin = it.z, n_tok = it.w;
-      const int tok0 = p.seq_tok0[seq] + tok_begin;
-      const int pos0 = p.seq_ctx[seq] + tok_begin;
-      const int n_keys = p.bidirectional ? p.seq_ctx[seq] + p.seq_qlen[seq] : pos0 + n_tok;
-      const int n_kblocks = (n_keys + PF_KEYS - 1) / PF_KEYS;
-      const int g = r / Mt, tok = r - g * Mt;
-      const bool row_valid = g < G && tok < n_tok;
-      // last key a row sees: its own position (padding rows behave like the last token), or the sequence's last key
-      const int pos = p.bidirectional ? n_keys - 1 : pos0 + min(tok, n_tok - 1);
+      const ItemView v = view_item(p, item, Mt);
+      const int nblk = v.nblk_t[t], n_tok = v.n_tok_t[t];
+      if (nblk == 0) { blk_base += v.nblk; continue; }            // the item has no tile for this warp group
+      const int hg = r / Mt, tok = r - hg * Mt;
+      const bool row_valid = hg < G && tok < n_tok;
+      // last key a row sees: its own position (padding rows behave like the tile's last token), or the sequence's last key
+      const int pos = p.bidirectional ? v.n_keys - 1 : v.pos0 + t * Mt + min(tok, n_tok - 1);
 
-      float o_reg[DH];
-#pragma unroll
-      for (int e = 0; e < DH; ++e) o_reg[e] = 0.f;
-      float m_run = -INFINITY, l_run = 0.f, alpha_prev = 0.f;
+      float m_ref = -INFINITY, l_run = 0.f;
       uint32_t sreg[32], sreg2[32];
-
-      // o = o * alpha + O_blk of block b
-      auto correct = [&](uint32_t b, float alpha) -> bool {
-        const uint32_t buf = b & 1, bph = (b >> 1) & 1;
-        const bool w = mbar_wait(&bar->o_full[buf], bph, abort_flag, p.status);
-        if (!__all_sync(0xffffffffu, w)) return false;
-        tc_fence_after_sync();
-#pragma unroll
-        for (int c = 0; c < DH / 64; ++c) {
-          tmem_ld32(tmem + lane_base + G_::O0 + buf * DH + c * 64, sreg);
-          tmem_ld32(tmem + lane_base + G_::O0 + buf * DH + c * 64 + 32, sreg2);
-          tmem_ld_wait();
-#pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            o_reg[c * 64 + e] = fmaf(o_reg[c * 64 + e], alpha, __uint_as_float(sreg[e]));
-            o_reg[c * 64 + 32 + e] = fmaf(o_reg[c * 64 + 32 + e], alpha, __uint_as_float(sreg2[e]));
-          }
-        }
-        tc_fence_before_sync();
-        mbar_arrive(&bar->o_empty[buf]);
-        return true;
-      };
-
-      for (int j = 0; j < n_kblocks; ++j, ++gblk) {
-        const uint32_t buf = gblk & 1, bph = (gblk >> 1) & 1;
-        ok = mbar_wait(&bar->s_full[buf], bph, abort_flag, p.status);
+      for (int j = 0; j < nblk; ++j, ++g) {
+        const uint32_t buf = g & 1, bph = (g >> 1) & 1;
+        ok = mbar_wait(&bar->s_full[t][buf], bph, abort_flag, p.status);
         if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
         tc_fence_after_sync();
         const int key0 = j * PF_KEYS;
-        // both halves of the row in flight, one wait
-        tmem_ld32(tmem + lane_base + G_::S0 + buf * PF_KEYS, sreg);
-        tmem_ld32(tmem + lane_base + G_::S0 + buf * PF_KEYS + 32, sreg2);
+        tmem_ld32(tmem + lane_base + s_col + buf * PF_KEYS, sreg);
+        tmem_ld32(tmem + lane_base + s_col + buf * PF_KEYS + 32, sreg2);
         tmem_ld_wait();
         tc_fence_before_sync();
-        mbar_arrive(&bar->s_empty[buf]);
+        mbar_arrive(&bar->s_empty[t][buf]);
         if (key0 + PF_KEYS - 1 > pos) {               // this row does not see every key of the block
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
@@ -302,37 +339,59 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         float mx = -INFINITY;
 #pragma unroll
         for (int e = 0; e < 32; ++e) mx = fmaxf(mx, fmaxf(__uint_as_float(sreg[e]), __uint_as_float(sreg2[e])));
-        // running max kept on the raw scores; the 1/sqrt(Dh) * log2(e) scale is folded into the exponent
-        const float m_new = fmaxf(m_run, mx);
-        const float alpha = fast_exp2((m_run - m_new) * scale_log2);
-        const float neg_ms = -m_new * scale_log2;
-        m_run = m_new;
+        // the reference maximum (kept on the raw scores; the 1/sqrt(Dh) * log2(e) scale is folded into the
+        // exponent) moves only when the block's maximum is far above it
+        float alpha = 1.f;
+        const bool move = row_valid && (j == 0 || (mx - m_ref) * scale_log2 > kRefSlack);
+        if (j == 0) m_ref = mx;
+        else if (move) {
+          alpha = fast_exp2((m_ref - mx) * scale_log2);
+          m_ref = mx;
+        }
+        const bool rescale = j > 0 && __any_sync(0xffffffffu, move);
+        const float neg_ms = -m_ref * scale_log2;
         float sum = 0.f;
-        uint8_t* prow = p_smem + buf * G_::P_BYTES + r * 128;
+        uint32_t pk[32];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          float e8[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-            const uint32_t raw = u < 4 ? sreg[u * 8 + e] : sreg2[(u - 4) * 8 + e];
-            e8[e] = fast_exp2(fmaf(__uint_as_float(raw), scale_log2, neg_ms));
-            sum += e8[e];
-          }
-          uint4 w;
-          w.x = pack_bf16(e8[0], e8[1]);
-          w.y = pack_bf16(e8[2], e8[3]);
-          w.z = pack_bf16(e8[4], e8[5]);
-          w.w = pack_bf16(e8[6], e8[7]);
-          *reinterpret_cast<uint4*>(prow + ((u ^ (r & 7)) << 4)) = w;
+        for (int e = 0; e < 32; e += 2) {
+          const float a0 = fast_exp2(fmaf(__uint_as_float(sreg[e]), scale_log2, neg_ms));
+          const float a1 = fast_exp2(fmaf(__uint_as_float(sreg[e + 1]), scale_log2, neg_ms));
+          const float b0 = fast_exp2(fmaf(__uint_as_float(sreg2[e]), scale_log2, neg_ms));
+          const float b1 = fast_exp2(fmaf(__uint_as_float(sreg2[e + 1]), scale_log2, neg_ms));
+          sum += (a0 + a1) + (b0 + b1);
+          pk[e >> 1] = pack_bf16(a0, a1);
+          pk[16 + (e >> 1)] = pack_bf16(b0, b1);
         }
         l_run = l_run * alpha + sum;
-        // ragged last block: V rows of keys that do not exist must not carry stray NaN / Inf bits
-        const int n_valid = n_keys - key0;
+        // every earlier P V product of this tile has completed from here on: the P buffer written below (read by
+        // the product two blocks back) is free, and O is at rest for the rescale
+        if (g > 0) {
+          ok = mbar_wait(&bar->o_full[t], (g - 1) & 1, abort_flag, p.status);
+          if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+        }
+        if (rescale) {
+          tc_fence_after_sync();
+#pragma unroll
+          for (int c = 0; c < DH / 32; ++c) {
+            tmem_ld32(tmem + lane_base + o_col + c * 32, sreg);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) sreg[e] = __float_as_uint(__uint_as_float(sreg[e]) * alpha);
+            tmem_st32(tmem + lane_base + o_col + c * 32, sreg);
+          }
+          tmem_st_wait();
+        }
+        uint8_t* prow = p_tile + buf * G_::P_BYTES + r * 128;
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          *reinterpret_cast<uint4*>(prow + ((u ^ (r & 7)) << 4)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
+        // ragged last block of the item: V rows of keys that do not exist must not carry stray NaN / Inf bits
+        const int n_valid = v.n_keys - key0;
         if (n_valid < PF_KEYS) {
-          const uint32_t s = gblk % PF_STAGES;
-          const bool w = mbar_wait(&bar->kv_full[s], (gblk / PF_STAGES) & 1, abort_flag, p.status);
+          const uint32_t gb = blk_base + j, s = gb % PF_VSTAGES;
+          const bool w = mbar_wait(&bar->v_full[s], (gb / PF_VSTAGES) & 1, abort_flag, p.status);
           if (!__all_sync(0xffffffffu, w)) { ok = false; break; }
-          uint8_t* vst = stages + s * G_::STAGE_BYTES + G_::KV_BYTES;
+          uint8_t* vst = v_smem + s * G_::KV_BYTES;
           const int n_units = (PF_KEYS - n_valid) * G_::HALVES * 8;
           for (int idx = r; idx < n_units; idx += 128) {
             const int u = idx & 7, h = (idx >> 3) % G_::HALVES, k = n_valid + (idx >> 3) / G_::HALVES;
@@ -341,26 +400,39 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
           }
         }
         fence_proxy_async();
-        mbar_arrive(&bar->p_full[buf]);
-        if (j > 0 && !correct(gblk - 1, alpha_prev)) { ok = false; break; }
-        alpha_prev = alpha;
+        tc_fence_before_sync();
+        mbar_arrive(&bar->p_full[t][buf]);
       }
       if (!ok) break;
-      if (!correct(gblk - 1, alpha_prev)) break;
-      if (row_valid) {
-        const float inv = 1.f / l_run;
-        const bool f16 = p.o_f16 != 0;
-        __nv_bfloat16* dst = p.o + size_t(tok0 + tok) * q_dim + (hk * G + g) * DH;
+      // the item's last P V product, then the tile's rows of O leave through registers
+      ok = mbar_wait(&bar->o_full[t], (g - 1) & 1, abort_flag, p.status);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      tc_fence_after_sync();
+      const float inv = 1.f / l_run;
+      const bool f16 = p.o_f16 != 0;
+      __nv_bfloat16* dst = p.o + size_t(v.tok0 + t * Mt + tok) * q_dim + (v.hk * G + hg) * DH;
 #pragma unroll
-        for (int u = 0; u < DH / 8; ++u) {
-          uint4 w;
-          w.x = pack_act(o_reg[u * 8 + 0] * inv, o_reg[u * 8 + 1] * inv, f16);
-          w.y = pack_act(o_reg[u * 8 + 2] * inv, o_reg[u * 8 + 3] * inv, f16);
-          w.z = pack_act(o_reg[u * 8 + 4] * inv, o_reg[u * 8 + 5] * inv, f16);
-          w.w = pack_act(o_reg[u * 8 + 6] * inv, o_reg[u * 8 + 7] * inv, f16);
-          *reinterpret_cast<uint4*>(dst + u * 8) = w;
+      for (int c = 0; c < DH / 32; ++c) {
+        tmem_ld32(tmem + lane_base + o_col + c * 32, sreg);
+        tmem_ld_wait();
+        if (row_valid) {
+          float o32[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e) o32[e] = __uint_as_float(sreg[e]) * inv;
+          if (f16) note_f16_saturation(o32, p.status);
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            uint4 w;
+            w.x = pack_act(o32[u * 8 + 0], o32[u * 8 + 1], f16);
+            w.y = pack_act(o32[u * 8 + 2], o32[u * 8 + 3], f16);
+            w.z = pack_act(o32[u * 8 + 4], o32[u * 8 + 5], f16);
+            w.w = pack_act(o32[u * 8 + 6], o32[u * 8 + 7], f16);
+            *reinterpret_cast<uint4*>(dst + c * 32 + u * 8) = w;
+          }
         }
       }
+      tc_fence_before_sync();
+      blk_base += v.nblk;
     }
   }
 
@@ -369,7 +441,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
   if (*abort_flag) drain_after_abort();
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 5) {
+  if (warp == 9) {
     tc_fence_after_sync();
     tmem_dealloc(tmem, TMEM_COLS);
   }

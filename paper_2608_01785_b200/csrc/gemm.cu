@@ -400,6 +400,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
             const float g = __uint_as_float(r0[e]), u = __uint_as_float(r1[e]);
             v0[e] = __fdividef(g * u, 1.f + __expf(-g));   // silu(g) * u
           }
+          if (p.act_f16) note_f16_saturation(v0, p.status);
           uint8_t* buf = epi_buf + epi_sel * EPI_BUF_BYTES;
           if ((c & 1) == 0) {
             if (lane == 0) bulk_wait_read<1>();

@@ -250,6 +250,7 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
         float v[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) v[e] = __fdividef(gt[e] * up[e], 1.f + __expf(-gt[e]));   // silu(gate) * up
+        if (p.act_f16 && p.status) note_f16_saturation(v, p.status);
         uint2 out;
         out.x = pack_act(v[0], v[1], p.act_f16 != 0);
         out.y = pack_act(v[2], v[3], p.act_f16 != 0);

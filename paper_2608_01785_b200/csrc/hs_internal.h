@@ -50,7 +50,7 @@ struct MetaLayout {
   int tok_pos, tok_slot, tok_seq;    // [max_tokens]      absolute position / cache slot / sequence index of each new token
   int seq_tok0, seq_ctx, seq_qlen;   // [max_seqs]        first token row, cached tokens, new tokens
   int block_tables;                  // [max_seqs * max_pages_per_seq]
-  int prefill_items;                 // [max_prefill_items * 4]  {seq, kv_head, first token of the tile, tokens}
+  int prefill_items;                 // [max_prefill_items * 4]  {seq, kv_head, first token, tokens (at most two tiles)}
   int decode_items;                  // [max_decode_items * 8]   {decode row, kv_head, first key, end key,
                                      //                           seq, token row, first item of the group, splits}
   int decode_rows;                   // [max_seqs * 4]           {seq, token row, first item, splits}

@@ -56,7 +56,7 @@ struct GemmParams {
   int gate_which;
   // GateUp
   CUtensorMap tm_act;        // bf16 act [M, N], box 64 x 32, 128-byte swizzle
-  int* status;               // device status word
+  int* status;               // device status word; with act_f16 the word after it counts saturated act values
   int act_f16;               // GateUp: 1 = write act as fp16, 0 = bf16
   int* smid_log;             // nullable: SM census slots of this launch (see log_smid)
 };
@@ -87,6 +87,7 @@ struct SkinnyParams {
   int gate_which;
   __nv_bfloat16* act;        // GateUp: 16-bit [T, N]
   int act_f16;
+  int* status;               // nullable: the stage's device status words (the second one counts fp16 saturations)
   int* smid_log;
 };
 // True when the skinny kernel covers this shape (few rows, K a multiple of 32, widths it can tile).

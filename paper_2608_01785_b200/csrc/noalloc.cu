@@ -6,8 +6,9 @@
 // later (the allocation fails, or succeeds only by stalling every stream of the device while the
 // driver maps memory), and a plug-in that is handed raw device pointers by a host runtime may simply
 // not be allowed to call the allocator.  For them this file carries a fixed scratch area in a
-// file-scope __device__ array; the entry point below runs the same decode kernel on it
-// and allocates nothing, on the device or through any library.
+// file-scope __device__ array; the entry point below runs the same decode kernel on it and calls no
+// allocating routine: no cudaMalloc / cudaFree / cudaHostAlloc, no heap, no library that allocates.  The
+// call's integer metadata is assembled in a fixed host array of the library image (guarded by a mutex).
 //
 // The array is a device symbol.  In host code its name is only a stand-in, not a device address, so
 // the address is obtained once per device with cudaGetSymbolAddress (with that device current) and it
@@ -47,40 +48,60 @@ constexpr int kScratchWords = kOffPartO + kMaxItems * 16 * 128;   // about 4.3 M
 // Held by every GPU that loads the library, until the process exits.
 static __device__ __align__(256) uint32_t g_noalloc_scratch[kScratchWords];
 
-std::mutex g_setup_mutex;
-uint32_t* g_scratch_dev[64] = {};   // device address of the array, per device ordinal
-
-// First use on a device: resolve the symbol's device address and raise the kernels' shared-memory limit.
-hs_status_t setup_device(int dev, uint32_t** out) {
-  std::lock_guard<std::mutex> lock(g_setup_mutex);
-  if (!g_scratch_dev[dev]) {
-    void* ptr = nullptr;
-    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) return HS_ERR_CUDA;
-    if (attention_set_attributes() != cudaSuccess) return HS_ERR_CUDA;
-    g_scratch_dev[dev] = static_cast<uint32_t*>(ptr);
-  }
-  *out = g_scratch_dev[dev];
-  return HS_OK;
-}
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// What the first call on a device finds out once and every later call reuses.
+struct DeviceSetup {
+  uint32_t* scratch = nullptr;   // device address of g_noalloc_scratch on this device
+  int sm_count = 0, cc_major = 0;
+};
+std::mutex g_mutex;              // guards the set-up table, the encode entry point and the host metadata array
+DeviceSetup g_setup[64];
+EncodeTiledFn g_encode = nullptr;
+int32_t g_meta[kMetaWords];      // the call's integer metadata on the host: fixed, shared, filled under g_mutex
+int g_last_device = -1;          // device of the most recent call (for hs_op_decode_attention_noalloc_status)
+
+// First use on a device (that device current): resolve the symbol's device address, read the two device
+// attributes the argument checks need, raise the kernels' shared-memory limit and fetch the driver's tensor-map
+// encoder.  Called with g_mutex held.
+hs_status_t setup_device(int dev, const DeviceSetup** out) {
+  DeviceSetup& d = g_setup[dev];
+  if (!d.scratch) {
+    int sm = 0, major = 0;
+    if (cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+      return HS_ERR_CUDA;
+    if (major != 10) return HS_ERR_CUDA;            // the kernels exist for sm_100a only
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) return HS_ERR_CUDA;
+    if (attention_set_attributes() != cudaSuccess) return HS_ERR_CUDA;
+    if (!g_encode) {
+      void* fn = nullptr;
+      cudaDriverEntryPointQueryResult q;
+      if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
+          q != cudaDriverEntryPointSuccess)
+        return HS_ERR_CUDA;
+      g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    d.sm_count = sm;
+    d.cc_major = major;
+    d.scratch = static_cast<uint32_t*>(ptr);
+  }
+  *out = &d;
+  return HS_OK;
+}
+
 bool encode_pool_map(CUtensorMap* m, const void* pool, uint64_t rows, uint64_t head_dim) {
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult q;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q) != cudaSuccess ||
-      q != cudaDriverEntryPointSuccess)
-    return false;
+  EncodeTiledFn fn = g_encode;
   cuuint64_t dims[2] = {head_dim, rows};
   cuuint64_t strides[1] = {head_dim * 2};
   cuuint32_t box[2] = {64, 16};
   cuuint32_t estr[2] = {1, 1};
-  return reinterpret_cast<EncodeTiledFn>(fn)(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(pool), dims,
-                                             strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(pool), dims,
+            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace
@@ -108,8 +129,10 @@ extern "C" hs_status_t hs_op_decode_attention_noalloc(const void* q_dev, const v
   const int64_t pool_rows = int64_t(n_layers) * 2 * num_pages * n_kv_heads * kPage;
   if (pool_rows >= (int64_t(1) << 31)) return HS_ERR_UNSUPPORTED_SHAPE;
 
-  // integer metadata, assembled in a per-thread host buffer (no heap, no pinned allocation)
-  static thread_local int32_t meta[kMetaWords];
+  // integer metadata, assembled in the library's fixed host array (no heap, no pinned allocation); the lock is
+  // held until the copy below has taken the array's contents
+  std::lock_guard<std::mutex> lock(g_mutex);
+  int32_t* meta = g_meta;
   memset(meta, 0, sizeof(int32_t) * (kOffSeqTok0));
   int n_items = 0;
   for (int s = 0; s < n_seqs; ++s) {
@@ -139,19 +162,20 @@ extern "C" hs_status_t hs_op_decode_attention_noalloc(const void* q_dev, const v
   }
 
   int dev = 0;
-  cudaDeviceProp prop;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64 ||
-      cudaGetDeviceProperties(&prop, dev) != cudaSuccess || prop.major != 10)
-    return HS_ERR_CUDA;
-  if (sm_budget < 1 || sm_budget > prop.multiProcessorCount) return HS_ERR_INVALID_BUDGET;
-  uint32_t* scratch = nullptr;
-  hs_status_t st = setup_device(dev, &scratch);
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HS_ERR_CUDA;
+  const DeviceSetup* setup = nullptr;
+  hs_status_t st = setup_device(dev, &setup);
   if (st != HS_OK) return st;
+  if (sm_budget < 1 || sm_budget > setup->sm_count) return HS_ERR_INVALID_BUDGET;
+  uint32_t* scratch = setup->scratch;
+  g_last_device = dev;
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   AttnParams a{};
   if (!encode_pool_map(&a.tm_kv, kv_pool_dev, uint64_t(pool_rows), uint64_t(head_dim))) return HS_ERR_CUDA;
-  // The metadata copy also resets the queue heads and the status word left by the previous call.
+  // The metadata copy also resets the queue heads and the status word left by the previous call.  The source is
+  // ordinary (pageable) host memory: the runtime has taken its contents when the call returns, possibly after
+  // waiting for earlier work of the stream.
   if (cudaMemcpyAsync(scratch, meta, sizeof(int32_t) * kMetaWords, cudaMemcpyHostToDevice, stream) != cudaSuccess)
     return HS_ERR_CUDA;
   int32_t* words = reinterpret_cast<int32_t*>(scratch);
@@ -171,5 +195,20 @@ extern "C" hs_status_t hs_op_decode_attention_noalloc(const void* q_dev, const v
   a.group_done = words + kOffGroupDone;
   a.status = words + kOffStatus;
   if (launch_attention_decode(a, sm_budget, stream) != cudaSuccess) return HS_ERR_CUDA;
+  return HS_OK;
+}
+
+extern "C" hs_status_t hs_op_decode_attention_noalloc_status(int32_t* status_out) {
+  if (!status_out) return HS_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  if (g_last_device < 0 || !g_setup[g_last_device].scratch) return HS_ERR_INVALID_ARG;   // no call was made yet
+  int32_t v = 0;
+  int prev = -1;
+  if (cudaGetDevice(&prev) != cudaSuccess) return HS_ERR_CUDA;
+  if (prev != g_last_device && cudaSetDevice(g_last_device) != cudaSuccess) return HS_ERR_CUDA;
+  const cudaError_t e = cudaMemcpy(&v, g_setup[g_last_device].scratch + kOffStatus, 4, cudaMemcpyDeviceToHost);
+  if (prev != g_last_device) cudaSetDevice(prev);
+  if (e != cudaSuccess) return HS_ERR_CUDA;
+  *status_out = v;
   return HS_OK;
 }

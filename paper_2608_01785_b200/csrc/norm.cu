@@ -120,6 +120,7 @@ __global__ void __launch_bounds__(NORM_THREADS, 1) rmsnorm_kernel(const NormPara
 #pragma unroll
         for (int e = 0; e < 8; ++e) v[e] = fmaf(v[e], 1.f + sc[e], sh[e]);
       }
+      if (f16 && p.status) note_f16_saturation(v, p.status);
       hdst[i] = make_uint4(pack_act(v[0], v[1], f16), pack_act(v[2], v[3], f16), pack_act(v[4], v[5], f16),
                            pack_act(v[6], v[7], f16));
     }
@@ -242,6 +243,10 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32, 1) rmsnorm_bulk_kernel(co
             const float4 sh = reinterpret_cast<const float4*>(shift)[i], sc = reinterpret_cast<const float4*>(shift + p.d)[i];
             v = make_float4(fmaf(v.x, 1.f + sc.x, sh.x), fmaf(v.y, 1.f + sc.y, sh.y), fmaf(v.z, 1.f + sc.z, sh.z),
                             fmaf(v.w, 1.f + sc.w, sh.w));
+          }
+          if (f16) {
+            const float v4[4] = {v.x, v.y, v.z, v.w};
+            note_f16_saturation(v4, p.status);
           }
           hdst[i] = make_uint2(pack_act(v.x, v.y, f16), pack_act(v.z, v.w, f16));
           if (in_bf16) xo[i] = a[u];                          // the widened copy that starts the residual stream

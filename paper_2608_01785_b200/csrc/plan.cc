@@ -181,9 +181,10 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
       n_dec_items += c.n_kv_heads * splits;
       ++n_dec_rows;
     } else {
-      for (int t0 = 0; t0 < n; t0 += Mt)
+      // a prefill item covers two Q tiles of Mt tokens each (the second one may be short or absent)
+      for (int t0 = 0; t0 < n; t0 += 2 * Mt)
         for (int hk = 0; hk < c.n_kv_heads; ++hk) {
-          const int nt = std::min(Mt, n - t0);
+          const int nt = std::min(2 * Mt, n - t0);
           pre.push_back(Item{{s, hk, t0, nt}, ctx + t0 + nt});
         }
     }

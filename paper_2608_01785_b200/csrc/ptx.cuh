@@ -66,10 +66,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Waits for the phase with the given parity to complete.  Bounded: after kWaitLimitNs (or as soon as
+// Waits for the phase with the given parity to complete.  Bounded: after limit_ns (or as soon as
 // another thread of the block has given up) it raises the block's abort flag, records HS_ERR_TIMEOUT in
 // the global status word and returns false; the caller then leaves its role loop.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = globaltimer_ns();
   uint32_t spins = 0;
@@ -77,7 +78,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 0xffu) == 0) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      if (globaltimer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         atomicExch(status, kErrTimeout);
         return false;
@@ -286,6 +287,21 @@ __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
 // HS_FLAG_BF16_ACTIVATIONS.
 __device__ __forceinline__ uint32_t pack_act(float lo, float hi, bool f16) {
   return f16 ? pack_f16(lo, hi) : pack_bf16(lo, hi);
+}
+// Saturation report of the fp16 activations: the word after a stage's device status word counts the values that
+// pack_f16 had to clamp (|v| > 65504, infinities included).  Call with the values about to be packed; the common
+// case costs one max per value.
+template <int N>
+__device__ __forceinline__ void note_f16_saturation(const float (&v)[N], int* status, float scale = 1.f) {
+  float mx = 0.f;
+#pragma unroll
+  for (int e = 0; e < N; ++e) mx = fmaxf(mx, fabsf(v[e]));
+  if (mx * fabsf(scale) > 65504.f) {
+    int c = 0;
+#pragma unroll
+    for (int e = 0; e < N; ++e) c += fabsf(v[e] * scale) > 65504.f ? 1 : 0;
+    atomicAdd(status + 1, c);
+  }
 }
 __device__ __forceinline__ void named_barrier_sync(int id, int nthreads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");

@@ -66,6 +66,10 @@ class Stage:
     def status(self) -> int:
         return B.hs_stage_status(self.handle)
 
+    def saturation_count(self) -> int:
+        """fp16 activation values clamped to +-65504 since the stage was created (0 for a well-scaled model)."""
+        return B.hs_stage_saturation_count(self.handle)
+
     def set_modulation(self, mod) -> None:
         """fp32 device tensor [n_layers, max_seqs, 6, d_model] (or None): per-sequence shift / scale / gate vectors
         of a conditioned block; kept alive here, read at every step."""

@@ -187,6 +187,14 @@ def make_kv_fill(dims: StageDims, num_pages: int, seed: int, device="cpu") -> to
     return _normal_bf16(kv_pool_shape(dims, num_pages), 1.0, 0.0, gen, device)
 
 
+def make_kv_fill_layer(dims: StageDims, num_pages: int, seed: int, layer: int, device="cpu") -> torch.Tensor:
+    """One layer's [K or V][page][kv_head][slot][head_dim] block of such a fill, from a sub-stream of its own, for
+    stages too deep to draw the whole pool at once."""
+    gen = torch.Generator(device=device)
+    gen.manual_seed(_subseed(seed, "kv", layer + 1))
+    return _normal_bf16(kv_pool_shape(dims, num_pages)[1:], 1.0, 0.0, gen, device)
+
+
 def pages_needed(batch: BatchSpec, page_size: int = 16) -> int:
     return int(sum(-(-t // page_size) for t in batch.total_len()))
 

@@ -27,7 +27,7 @@ def make_stage(case: Case, max_tokens: Optional[int] = None, max_position: Optio
 
 
 def run_step(st: Stage, case: Case, budget: int, q_len=None, ctx_len=None, x_t=None, block_tables=None,
-             stream=None):
+             stream=None, expect_saturation: bool = False):
     """One hs_stage_step; returns (y float32 numpy [T, d], pool uint16 numpy, flat)."""
     q_len = case.batch.q_len if q_len is None else q_len
     ctx_len = case.batch.ctx_len if ctx_len is None else ctx_len
@@ -37,6 +37,8 @@ def run_step(st: Stage, case: Case, budget: int, q_len=None, ctx_len=None, x_t=N
     st.step(b, budget, stream)
     torch.cuda.synchronize()
     assert st.status() == 0
+    if not expect_saturation:
+        assert st.saturation_count() == 0, "a regular case clamped fp16 activations"
     return y.cpu().numpy(), wl.bf16_bits_numpy(st.kv_pool).reshape(-1)
 
 

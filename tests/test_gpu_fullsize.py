@@ -96,6 +96,24 @@ def layer_local_error(orc, stage, batch, bt, x, pool0, layer, rows=None, want_fl
     return err, rel_err(y_floor[sel], y_ref[sel])
 
 
+def kv_element_rule(stage, dims, batch, bt, pool_gpu, kv_pre, layer=0):
+    """Largest |k_gpu - k_ref| / (2^-8 |k_ref| + 1e-2 RMS(k_ref)) over the K and V elements that the step wrote for
+    `layer` (k_ref: the oracle's value before its bf16 rounding; one bf16 rounding plus operand noise is allowed)."""
+    pool = pool_gpu.view(dims.n_layers, 2, stage.cfg.num_pages, dims.n_kv_heads, 16, dims.head_dim)[layer].float().cpu().numpy()
+    pages, slots = [], []
+    for s, (n, c) in enumerate(zip(batch.q_len, batch.ctx_len)):
+        pos = c + np.arange(n)
+        pages.append(bt[s, pos // 16]); slots.append(pos % 16)
+    pages, slots = np.concatenate(pages), np.concatenate(slots)
+    worst = 0.0
+    for kv in range(2):
+        ref = kv_pre[:, kv].reshape(-1, dims.n_kv_heads, dims.head_dim).astype(np.float64)
+        got = pool[kv][pages, :, slots, :].astype(np.float64)            # [T, kv heads, Dh]
+        bound = 2.0 ** -8 * np.abs(ref) + 1e-2 * np.sqrt(np.mean(ref ** 2))
+        worst = max(worst, float(np.max(np.abs(got - ref) / bound)))
+    return worst
+
+
 # ---------------------------------------------------------------- config 2 --
 def test_config2_budget_sweep_layer_local_and_end_to_end(orc):
     name = "c2_shared"
@@ -112,6 +130,17 @@ def test_config2_budget_sweep_layer_local_and_end_to_end(orc):
             assert torch.equal(pool, outs[first][1]), budget
         y_gpu = outs[first][0]
         assert np.all(np.isfinite(y_gpu))
+
+        # K / V written by layer 0 at full size, element by element against the oracle's values before their bf16
+        # rounding (the oracle forms K / V of every token and evaluates no row past the cache write)
+        cfg1 = ocfg(dims, 1, stage.cfg.num_pages)
+        w0 = {k: wl.to_f32_numpy(v) for k, v in stage.weights[0].items()}
+        _, kv_pre = orc.layer(cfg1, w0, 0, layer_pool_bits(pool0, dims, stage.cfg.num_pages, 0), batch.q_len,
+                              batch.ctx_len, bt, wl.to_f32_numpy(x), row_mask=np.zeros(batch.n_tokens, dtype=np.uint8),
+                              want_kv_pre=True)
+        worst = kv_element_rule(stage, dims, batch, bt, outs[first][1], kv_pre)
+        print(f"config 2 layer 0: K/V element rule over {batch.n_tokens} tokens, worst |err| / bound = {worst:.2f}")
+        assert worst <= 1.0
 
         for layer in range(dims.n_layers):
             err = layer_local_error(orc, stage, batch, bt, x, pool0, layer)
@@ -331,5 +360,61 @@ def test_bias_and_modulation_on_pair_tiles(orc):
         y_plain, _ = orc.layer(ocfg(dims, 1, stage.cfg.num_pages), plain, 0, wl.bf16_bits_numpy(pool0).reshape(-1).copy(),
                                batch.q_len, batch.ctx_len, bt, wl.to_f32_numpy(x), row_mask=mask)
         assert rel_err(y_plain[rows], y_ref[rows]) > 5 * TOL
+    finally:
+        stage.close()
+
+
+# ------------------------------------------------- config 3, all 28 layers against the stored oracle output --
+def test_config3_end_to_end_against_the_stored_oracle_output():
+    """The whole config-3 step (28 layers, 2048-token prefill chunk + 64 decode sequences) against the CPU oracle's
+    output of the same step on sampled rows (first / last rows, tile edges, decode rows).  The oracle's rows were
+    written once by tests/golden/make_c3_end_to_end.py (a quarter of an hour of CPU time), which calls only the
+    oracle and the seeded generators; here the same generators draw the same buffers on the CPU (checked by the
+    checksums stored with the rows) and upload them.  Weights: std 0.02, output projections 0.02 / sqrt(2 L)."""
+    import os
+    import zlib
+    from concurrent.futures import ThreadPoolExecutor
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "c3_end_to_end.npz")
+    gold = np.load(path)
+    rows, y_want = gold["rows"].astype(np.int64), gold["y"]
+    name, seed, init, num_pages = gold["recipe"][0], int(gold["recipe"][1]), gold["recipe"][2], int(gold["recipe"][3])
+    want_crc = {k: int(v) for k, v in gold["input_crc32"]}
+    dims, batch = wl.DIMS[str(name)], wl.make_batch(str(name), seed)
+    assert num_pages == wl.pages_needed(batch) + 8
+    crc = lambda t: zlib.crc32(wl.bf16_bits_numpy(t).reshape(-1).data) & 0xFFFFFFFF
+    dev = torch.device("cuda", 0)
+
+    def draw(layer):
+        return wl.make_layer_weights(dims, seed, layer, "cpu", str(init)), wl.make_kv_fill_layer(dims, num_pages, seed, layer)
+
+    weights, fills = [], []
+    with ThreadPoolExecutor(max_workers=8) as pool:
+        for layer, (w, kv) in enumerate(pool.map(draw, range(dims.n_layers))):
+            if layer in (0, dims.n_layers - 1):
+                assert crc(w["w_down"]) == want_crc[f"w_down_{layer}"], "the weight generator drew other values here"
+                assert crc(kv) == want_crc[f"kv_{layer}"], "the cache-fill generator drew other values here"
+            weights.append({k: v.to(dev) for k, v in w.items()})
+            fills.append(kv.to(dev))
+    x = wl.make_x(batch.n_tokens, dims.d_model, seed)
+    assert crc(x) == want_crc["x"]
+    mpps = max(-(-t // 16) for t in batch.total_len())
+    stage = Stage(dims, weights, num_pages, batch.n_tokens, batch.n_seqs, mpps, max(batch.total_len()))
+    try:
+        view = stage.kv_pool_view()
+        for layer, kv in enumerate(fills):
+            view[layer].copy_(kv)
+        del fills
+        bt = stage.block_table_array([stage.kv_alloc(s, t) for s, t in enumerate(batch.total_len())])
+        y = torch.full((batch.n_tokens, dims.d_model), float("nan"), device=dev)
+        b = stage.make_batch(batch.q_len, batch.ctx_len, bt, x.to(dev), y)
+        stage.step(b, stage.sm_count)
+        torch.cuda.synchronize()
+        assert stage.status() == 0 and stage.saturation_count() == 0
+        y_gpu = y.cpu().numpy()
+        assert np.all(np.isfinite(y_gpu))
+        err = rel_err(y_gpu[rows], y_want)
+        print(f"config 3 end to end (28 layers, depth-scaled init), {len(rows)} sampled rows against the stored "
+              f"oracle output: max|err|/RMS = {err:.2e}")
+        assert err <= TOL
     finally:
         stage.close()

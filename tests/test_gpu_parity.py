@@ -476,3 +476,75 @@ def test_every_kernel_of_a_step_stays_within_the_sm_budget(orc):
             assert np.array_equal(y, y_ref)
     finally:
         st.close()
+
+
+# ------------------------------------------------- fp16 range of the private activations --
+@pytest.mark.parametrize("T", [40, 300])
+def test_fp16_saturation_is_counted_and_the_output_stays_finite(orc, T):
+    """h, o and act are stored as fp16, clamped to +-65504.  A stage whose SwiGLU activations leave that range
+    (gate and up projections scaled x300 here; nothing faults, clamping is defined behaviour) must say so through
+    hs_stage_saturation_count and still return finite numbers; the bf16 form of the same stage reports nothing and
+    stays within the tolerance.  T = 40 goes through the weight-streaming GEMM, T = 300 through the tiled one."""
+    dims = wl.StageDims(1, 512, 8, 2, 64, 1024)
+    case = make_case(dims, wl.BatchSpec([T], [0]), seed=41)
+    big = [dict(lw) for lw in case.weights_t]
+    for k in ("w_gate", "w_up"):
+        big[0][k] = (big[0][k].float() * 300.0).to(torch.bfloat16)
+    w_np = wl.weights_to_numpy(big)
+    y_ref = orc.step(case.cfg, w_np, case.kv_pool.copy(), case.batch.q_len, case.batch.ctx_len, case.block_tables, case.x)
+    # the scaled projections of a unit-RMS row have a standard deviation of 0.02 * 300 * sqrt(512) = 136, so
+    # silu(gate) * up passes 65504 in the tails; checked on the input rows as a stand-in for the MLP's input
+    h_like = orc.rmsnorm(case.x, w_np[0]["g_mlp"], dims.rms_eps)
+    assert float(np.max(np.abs(orc.linear(h_like, w_np[0]["w_gate"])))) > 400.0
+    st = make_stage(case, weights=big)
+    try:
+        assert st.saturation_count() == 0
+        y, _ = run_step(st, case, st.sm_count, expect_saturation=True)
+        n_sat = st.saturation_count()
+        assert n_sat > 0, "clamped activations went unreported"
+        assert np.all(np.isfinite(y))
+        y2, _ = run_step(st, case, 8, expect_saturation=True)
+        assert np.array_equal(y, y2)
+        assert st.saturation_count() == 2 * n_sat           # the count accumulates, and is the same at every budget
+    finally:
+        st.close()
+    st = make_stage(case, weights=big, flags=B.HS_FLAG_BF16_ACTIVATIONS)
+    try:
+        y, _ = run_step(st, case, st.sm_count)
+        assert st.saturation_count() == 0
+        assert rel_err(y, y_ref) <= 3e-2                    # all-bf16 operands: within the format's own floor
+    finally:
+        st.close()
+
+
+# ------------------------------------------------- bounded waits --
+def test_a_wait_that_nothing_satisfies_gives_up_with_a_timeout_status():
+    """The wind-down every kernel runs when a wait exceeds its limit (abort flag, status word, roles leaving, drain,
+    tensor memory freed), run on purpose by the probe with a 1 ms limit: it must return by itself with
+    HS_ERR_TIMEOUT in the status word, quickly, and leave the context usable for a regular step."""
+    import time
+    dev = torch.device("cuda:0")
+    status = torch.zeros(2, dtype=torch.int32, device=dev)
+    waited = torch.zeros(1, dtype=torch.int64, device=dev)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    B.hs_op_wait_probe(1_000_000, status.data_ptr(), waited.data_ptr())
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    assert status[0].item() == B.HS_ERR_TIMEOUT
+    assert 1_000_000 <= waited.item() < 50_000_000          # gave up after the limit, not long after
+    assert dt < 1.0
+    for bad in (0, 10, 10**9):
+        with pytest.raises(B.HsError):
+            B.hs_op_wait_probe(bad, status.data_ptr())
+    with pytest.raises(B.HsError):
+        B.hs_op_wait_probe(1_000_000, 0)
+    # the context is intact: a GEMM runs and is right
+    a = torch.randn(64, 128, device=dev).to(torch.bfloat16)
+    w = torch.randn(256, 128, device=dev).to(torch.bfloat16)
+    out = torch.empty(64, 256, device=dev)
+    st2 = torch.zeros(1, dtype=torch.int32, device=dev)
+    B.hs_op_gemm_bf16(a.data_ptr(), w.data_ptr(), 0, out.data_ptr(), 64, 256, 128, 148, st2.data_ptr())
+    torch.cuda.synchronize()
+    assert st2.item() == 0
+    assert torch.allclose(out, a.float() @ w.float().T, rtol=1e-3, atol=1e-2)

@@ -524,6 +524,44 @@ def test_row_mask_matches_full_evaluation(oracle32):
     assert np.array_equal(pool_a, pool_b)
 
 
+def test_kv_pre_is_k_after_rope_and_v_before_the_cache_rounding(oracle32, oracle64):
+    """kv_pre, the layer's side output that the GPU tests hold the written K / V against: slot 0 must be
+    rope(h W_k^T + b_k) and slot 1 h W_v^T + b_v, formed here from the separately pinned primitives (rmsnorm,
+    linear, rope), and its bf16 rounding must be the very bits the same call wrote into the cache -- a copy taken
+    before RoPE, K and V swapped, or a wrong page / slot fails one of the two."""
+    batch = wl.make_batch("c1_tiny", 0)                    # prefill 32, 48 + decode with ctx 40, 64
+    for orc, tol in ((oracle32, 0.0), (oracle64, 0.0)):
+        case = make_case(TINY, batch, seed=0, kv_fill=True)
+        w = dict(case.weights[0])
+        g = np.random.default_rng(4)
+        w["b_k"] = g.normal(0, 0.5, TINY.kv_dim).astype(np.float32)
+        w["b_v"] = g.normal(0, 0.5, TINY.kv_dim).astype(np.float32)
+        pool = case.kv_pool.copy()
+        _, kv_pre = orc.layer(case.cfg, w, 0, pool, batch.q_len, batch.ctx_len, case.block_tables, case.x,
+                              want_kv_pre=True)
+        assert kv_pre.shape == (batch.n_tokens, 2, TINY.kv_dim)
+        h = orc.rmsnorm(case.x, w["g_attn"], TINY.rms_eps)
+        k_lin = orc.linear(h, w["w_k"]) + w["b_k"].astype(orc.dtype)
+        v_lin = orc.linear(h, w["w_v"]) + w["b_v"].astype(orc.dtype)
+        pool5 = pool.reshape(TINY.n_layers, 2, case.cfg.num_pages, TINY.n_kv_heads, 16, TINY.head_dim)
+        t = 0
+        moved = 0.0
+        for s in range(batch.n_seqs):
+            for j in range(batch.q_len[s]):
+                pos = batch.ctx_len[s] + j
+                k_rot = orc.rope(k_lin[t].reshape(TINY.n_kv_heads, TINY.head_dim), pos, TINY.rope_base)
+                assert np.array_equal(kv_pre[t, 0], k_rot.reshape(-1)), (s, j)
+                assert np.array_equal(kv_pre[t, 1], v_lin[t]), (s, j)
+                moved = max(moved, float(np.max(np.abs(k_rot.reshape(-1) - k_lin[t]))))
+                page, slot = case.block_tables[s, pos // 16], pos % 16
+                for kv in (0, 1):
+                    want = np.array([orc.bf16_rne(float(v)) for v in kv_pre[t, kv]], dtype=np.uint16)
+                    assert np.array_equal(pool5[0, kv, page, :, slot, :].reshape(-1), want), (s, j, kv)
+                t += 1
+        assert moved > 0.1                                  # the rotation is visible: "before RoPE" would fail
+        assert float(np.max(np.abs(kv_pre[:, 0] - kv_pre[:, 1]))) > 0.1   # and K is not V
+
+
 # --------------------------------------------------- float32 vs float64 --
 def test_float32_oracle_is_close_to_float64_on_config_1(oracle32, oracle64):
     batch = wl.make_batch("c1_tiny", 0)
