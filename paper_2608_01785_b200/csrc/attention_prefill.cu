@@ -6,16 +6,21 @@
 //               token).  Both tiles read the same K / V blocks, which are staged once for the two of them.
 //   per block   of 64 keys and per tile:  S = Q K^T (tcgen05.mma, M128 N64, fp32 in tensor memory)  ->  the tile's
 //               softmax warp group (one thread per row: no shuffles) reads S, masks by selection, exponentiates
-//               in the log2 domain against a per-row reference maximum, writes P as bf16 into a swizzled
-//               shared-memory tile  ->  O += P V (tcgen05.mma, M128 N = Dh, V used in place as an MN-major
-//               operand).  O stays in tensor memory for the whole item; it is read once, at the item's end.
+//               in the log2 domain against a per-row reference maximum, writes P as bf16 back into tensor memory,
+//               over the first half of the S buffer it has just read (tcgen05.st: row = lane, two keys per
+//               32-bit column)  ->  O += P V (tcgen05.mma with the A operand in tensor memory, M128 N = Dh, V used
+//               in place as an MN-major operand from shared memory).  An MMA whose operands both come from shared
+//               memory is bound by the operand fetch (about 64 bytes per clock and SM); taking P from tensor
+//               memory halves the bytes of the P V product.  O stays in tensor memory for the whole item; it is
+//               read once, at the item's end.
 //   reference   A row's reference maximum follows its running maximum lazily: it moves only when the running
 //   maximum     maximum exceeds it by more than 8 (in log2 units, a factor of 256), and only then is the row of O
 //               rescaled (tcgen05.ld / multiply / tcgen05.st by the softmax threads, while no P V product of the
 //               tile is in flight).  P and the running sum use the same reference, so the quotient O / l at the
 //               end is exact whatever reference was used; values stay far inside the range of bf16 and fp32.
-//   pipeline    two tiles x two S buffers x two P buffers: while one tile's warp group exponentiates, the tensor
-//               core works on the other tile's products.  K and V blocks arrive by TMA in two rings of their own
+//   pipeline    two tiles x two S buffers: while one tile's warp group exponentiates, the tensor core works on the
+//               other tile's products.  The tensor core runs its instructions in issue order, which is what makes
+//               the overlay safe: S of block j + 2 is issued after the P V product of block j, whose P it replaces.  K and V blocks arrive by TMA in two rings of their own
 //               ([half][page][16][64] tiles with the 128-byte swizzle, the K tile being a K-major and the V tile an
 //               MN-major operand): a K slot is free again as soon as the block's scores are computed, a V slot
 //               after its P V products.  The producer owns the work queue and runs ahead across items.
@@ -34,7 +39,7 @@ namespace {
 
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int PF_THREADS = 320, PF_KEYS = 64;
-constexpr int PF_KSTAGES = 3, PF_VSTAGES = 3;
+constexpr int PF_KSTAGES = 4, PF_VSTAGES = 4;
 constexpr int TMEM_COLS = 512;
 constexpr float kRefSlack = 8.f;   // log2 units by which a row's running maximum may exceed its reference
 
@@ -43,19 +48,28 @@ struct Geom {
   static constexpr int HALVES = DH / 64;
   static constexpr int Q_BYTES = HALVES * 16384;        // one tile: [half][128 rows][128 B]
   static constexpr int KV_BYTES = HALVES * 8192;        // K (or V) of one block: [half][4 pages][16 keys][128 B]
-  static constexpr int P_BYTES = 16384;                 // [128 rows][64 keys] bf16
-  static constexpr int SMEM = 1024 + 2 * Q_BYTES + (PF_KSTAGES + PF_VSTAGES) * KV_BYTES + 4 * P_BYTES + 1024;
-  // tensor-memory columns: S(tile, buffer) at tile * 128 + buffer * 64; O(tile) at 256 + tile * DH
+  static constexpr int SMEM = 1024 + 2 * Q_BYTES + (PF_KSTAGES + PF_VSTAGES) * KV_BYTES + 1024;
+  // tensor-memory columns: S(tile, buffer) at tile * 128 + buffer * 64, P(tile, buffer) over its first 32 columns;
+  // O(tile) at 256 + tile * DH
   static constexpr int S0 = 0, O0 = 256;
 };
 static_assert(Geom<128>::SMEM <= 227 * 1024, "fits one SM");
 
+// Geometry of one item, the same in every role.
+struct ItemView {
+  int seq, hk, tok_begin, n_tok;     // the item record
+  int tok0, pos0, ctx;               // first token row of tile A, its absolute position, cached tokens
+  int n_tok_t[2];                    // tokens of tile A / B (0 = tile absent)
+  int n_keys;                        // keys the item's K / V blocks cover (valid cache rows)
+  int nblk_t[2], nblk;               // key blocks per tile and of the item
+};
 struct Barriers {
   uint64_t q_full, q_empty;
   uint64_t k_full[PF_KSTAGES], k_empty[PF_KSTAGES], v_full[PF_VSTAGES], v_empty[PF_VSTAGES];
-  uint64_t s_full[2][2], s_empty[2][2], p_full[2][2], o_full[2];
+  uint64_t s_full[2][2], p_full[2][2], o_full[2][2];
   uint64_t ring_full[2], ring_empty[2];
   int ring_item[2];
+  ItemView ring_view[2];          // the item's geometry, worked out once by the producer
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -93,16 +107,18 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
         "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
+// D[tmem] (+)= A[tmem] * B[smem]^T: the A operand (M rows = lanes, 16 K elements = 8 columns of packed pairs) is read
+// from tensor memory; one thread issues for the block.
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}\n"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// Geometry of one item, the same in every role.
-struct ItemView {
-  int seq, hk, tok_begin, n_tok;     // the item record
-  int tok0, pos0, ctx;               // first token row of tile A, its absolute position, cached tokens
-  int n_tok_t[2];                    // tokens of tile A / B (0 = tile absent)
-  int n_keys;                        // keys the item's K / V blocks cover (valid cache rows)
-  int nblk_t[2], nblk;               // key blocks per tile and of the item
-};
 __device__ __forceinline__ ItemView view_item(const AttnParams& p, int item, int Mt) {
   const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
   ItemView v;
@@ -129,8 +145,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
   uint8_t* q_smem = smem;                                   // tile A then tile B
   uint8_t* k_smem = q_smem + 2 * G_::Q_BYTES;
   uint8_t* v_smem = k_smem + PF_KSTAGES * G_::KV_BYTES;
-  uint8_t* p_smem = v_smem + PF_VSTAGES * G_::KV_BYTES;     // [tile][buffer]
-  Barriers* bar = reinterpret_cast<Barriers*>(p_smem + 4 * G_::P_BYTES);
+  Barriers* bar = reinterpret_cast<Barriers*>(v_smem + PF_VSTAGES * G_::KV_BYTES);
   volatile int* abort_flag = &bar->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -148,10 +163,9 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
     for (int t = 0; t < 2; ++t) {
       for (int i = 0; i < 2; ++i) {
         mbar_init(&bar->s_full[t][i], 1);
-        mbar_init(&bar->s_empty[t][i], 128);
         mbar_init(&bar->p_full[t][i], 128);
+        mbar_init(&bar->o_full[t][i], 1);
       }
-      mbar_init(&bar->o_full[t], 1);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bar->ring_full[i], 1);
@@ -180,54 +194,83 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
 
   if (warp == 8) {
     // =========================================================== TMA producer ==
-    if (lane == 0) {
-      for (;;) {
-        if (!mbar_wait(&bar->ring_empty[rs], rph ^ 1, abort_flag, p.status)) break;
-        const int item = atomicAdd(p.counters, 1);
+    // Lane 0 waits and issues; the whole warp fetches page ids: lane l holds the id of page 32 c + l of the item
+    // for the current chunk c of 8 key blocks (one coalesced load per chunk, requested a chunk ahead), so that no
+    // round trip to the block table stands in front of a page request.
+    for (;;) {
+      int item = 0;
+      bool ok = true;
+      if (lane == 0) {
+        ok = mbar_wait(&bar->ring_empty[rs], rph ^ 1, abort_flag, p.status);
+        if (ok) item = atomicAdd(p.counters, 1);
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      item = __shfl_sync(0xffffffffu, item, 0);
+      ItemView v{};
+      if (item < p.n_prefill_items) v = view_item(p, item, Mt);
+      if (lane == 0) {
         bar->ring_item[rs] = item;
+        bar->ring_view[rs] = v;
         mbar_arrive(&bar->ring_full[rs]);
-        if (++rs == 2) { rs = 0; rph ^= 1; }
-        if (item >= p.n_prefill_items) break;
-        const ItemView v = view_item(p, item, Mt);
-        const int32_t* table = p.block_tables + size_t(v.seq) * p.max_pages_per_seq;
+      }
+      if (++rs == 2) { rs = 0; rph ^= 1; }
+      if (item >= p.n_prefill_items) break;
+      const int32_t* table = p.block_tables + size_t(v.seq) * p.max_pages_per_seq;
+      const int n_pages = (v.n_keys + 15) >> 4;
+      int pg_next = lane < n_pages ? table[lane] : 0, pg_cur = 0;
+      if (lane == 0) {
         // Q tiles: one box of Mt token rows x 64 columns per (tile, head, half)
-        if (!mbar_wait(&bar->q_empty, (n_items_seen & 1) ^ 1, abort_flag, p.status)) break;
-        const int n_tiles = v.n_tok_t[1] > 0 ? 2 : 1;
-        mbar_expect_tx(&bar->q_full, n_tiles * G * G_::HALVES * Mt * 128);
-        for (int t = 0; t < n_tiles; ++t)
-          for (int g = 0; g < G; ++g)
-            for (int h = 0; h < G_::HALVES; ++h)
-              tma_load_2d(q_smem + t * G_::Q_BYTES + h * 16384 + g * Mt * 128, &p.tm_q, &bar->q_full,
-                          (v.hk * G + g) * DH + h * 64, v.tok0 + t * Mt);
-        ++n_items_seen;
-        bool ok = true;
-        for (int kb = 0; kb < v.nblk && ok; ++kb) {
-          const uint32_t gb = blk_base + kb;
-          const int rem = v.n_keys - kb * PF_KEYS;
-          const int np = rem >= PF_KEYS ? 4 : (rem + 15) >> 4;
-          for (int kv = 0; kv < 2 && ok; ++kv) {
-            const uint32_t st = gb % (kv ? PF_VSTAGES : PF_KSTAGES), ph = (gb / (kv ? PF_VSTAGES : PF_KSTAGES)) & 1;
-            uint64_t* full = kv ? &bar->v_full[st] : &bar->k_full[st];
-            if (!mbar_wait(kv ? &bar->v_empty[st] : &bar->k_empty[st], ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-            uint8_t* dst = (kv ? v_smem : k_smem) + st * G_::KV_BYTES;
-            mbar_expect_tx(full, np * G_::HALVES * 2048);
-            for (int w = 0; w < np; ++w) {
-              const int row = pool_row(p, kv, table[kb * 4 + w], v.hk);
+        ok = mbar_wait(&bar->q_empty, (n_items_seen & 1) ^ 1, abort_flag, p.status);
+        if (ok) {
+          const int n_tiles = v.n_tok_t[1] > 0 ? 2 : 1;
+          mbar_expect_tx(&bar->q_full, n_tiles * G * G_::HALVES * Mt * 128);
+          for (int t = 0; t < n_tiles; ++t)
+            for (int g = 0; g < G; ++g)
+              for (int h = 0; h < G_::HALVES; ++h)
+                tma_load_2d(q_smem + t * G_::Q_BYTES + h * 16384 + g * Mt * 128, &p.tm_q, &bar->q_full,
+                            (v.hk * G + g) * DH + h * 64, v.tok0 + t * Mt);
+        }
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      ++n_items_seen;
+      for (int kb = 0; kb < v.nblk && ok; ++kb) {
+        if ((kb & 7) == 0) {
+          pg_cur = pg_next;
+          const int idx = (kb + 8) * 4 + lane;
+          pg_next = idx < n_pages ? table[idx] : 0;
+        }
+        const uint32_t gb = blk_base + kb;
+        const int rem = v.n_keys - kb * PF_KEYS;
+        const int np = rem >= PF_KEYS ? 4 : (rem + 15) >> 4;
+        for (int kv = 0; kv < 2 && ok; ++kv) {
+          const uint32_t st = gb % (kv ? PF_VSTAGES : PF_KSTAGES), ph = (gb / (kv ? PF_VSTAGES : PF_KSTAGES)) & 1;
+          uint64_t* full = kv ? &bar->v_full[st] : &bar->k_full[st];
+          uint8_t* dst = (kv ? v_smem : k_smem) + st * G_::KV_BYTES;
+          if (lane == 0) {
+            ok = mbar_wait(kv ? &bar->v_empty[st] : &bar->k_empty[st], ph ^ 1, abort_flag, p.status);
+            if (ok) mbar_expect_tx(full, np * G_::HALVES * 2048);
+          }
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+          if (!ok) break;
+          for (int w = 0; w < np; ++w) {
+            const int page = __shfl_sync(0xffffffffu, pg_cur, (kb & 7) * 4 + w);
+            if (lane == 0) {
+              const int row = pool_row(p, kv, page, v.hk);
               for (int h = 0; h < G_::HALVES; ++h) tma_load_2d(dst + h * 8192 + w * 2048, &p.tm_kv, full, h * 64, row);
             }
           }
         }
-        if (!ok) break;
-        blk_base += v.nblk;
       }
+      if (!ok) break;
+      blk_base += v.nblk;
     }
   } else if (warp == 9) {
     // ============================================================= MMA issuer ==
     if (lane == 0) {
       constexpr uint32_t idesc_s = umma_idesc_bf16_f32(128, PF_KEYS);
       constexpr uint32_t idesc_pv = umma_idesc_bf16_f32(128, DH) | (1u << 16);   // B (= V) is MN-major
-      const uint32_t q_addr = smem_u32(q_smem), k_addr0 = smem_u32(k_smem), v_addr0 = smem_u32(v_smem),
-                     p_addr = smem_u32(p_smem);
+      const uint32_t q_addr = smem_u32(q_smem), k_addr0 = smem_u32(k_smem), v_addr0 = smem_u32(v_smem);
       uint32_t g_t[2] = {0, 0};          // blocks of each tile whose S has been issued, over all items
       uint32_t pv_t[2] = {0, 0};         // blocks of each tile whose P V has been issued
       bool ok = true;
@@ -238,12 +281,15 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         tc_fence_after_sync();
         const uint32_t v_addr = v_addr0 + (gb % PF_VSTAGES) * G_::KV_BYTES;
 #pragma unroll
-        for (int pg = 0; pg < 4; ++pg) {      // 16 keys (one page) per MMA
-          const uint64_t a = umma_desc_kmajor_sw128(p_addr + (t * 2 + buf) * G_::P_BYTES) + 2 * pg;
+        for (int pg = 0; pg < 4; ++pg) {      // 16 keys (one page) per MMA: 8 columns of P
           const uint64_t bdesc = umma_desc_mnmajor_sw128(v_addr + pg * 2048, 8192, 1024);
-          umma_bf16(tmem + G_::O0 + t * DH, a, bdesc, idesc_pv, (pg != 0 || !first) ? 1u : 0u);
+          umma_bf16_ts(tmem + G_::O0 + t * DH, tmem + G_::S0 + t * 128 + buf * PF_KEYS + 8 * pg, bdesc, idesc_pv,
+                       (pg != 0 || !first) ? 1u : 0u);
         }
-        umma_commit(&bar->o_full[t]);
+        // "P V of block c has completed" alternates between two barriers: a waiter that does not look at every block
+        // is then never more than one phase of a barrier away from it (the scores of block c + 2, which it waits for
+        // first, complete after the product of block c), so a parity wait cannot mistake one phase for another
+        umma_commit(&bar->o_full[t][buf]);
         ++pv_t[t];
         return true;
       };
@@ -259,10 +305,10 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
       for (;;) {
         if (!mbar_wait(&bar->ring_full[rs], rph, abort_flag, p.status)) break;
         const int item = bar->ring_item[rs];
+        const ItemView v = bar->ring_view[rs];
         mbar_arrive(&bar->ring_empty[rs]);
         if (++rs == 2) { rs = 0; rph ^= 1; }
         if (item >= p.n_prefill_items) break;
-        const ItemView v = view_item(p, item, Mt);
         if (!mbar_wait(&bar->q_full, n_items_seen & 1, abort_flag, p.status)) break;
         ++n_items_seen;
         for (int j = 0; j < v.nblk && ok; ++j) {
@@ -270,9 +316,8 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
           if (!mbar_wait(&bar->k_full[kst], (gb / PF_KSTAGES) & 1, abort_flag, p.status)) { ok = false; break; }
           for (int t = 0; t < 2 && ok; ++t) {
             if (j >= v.nblk_t[t]) continue;
-            const uint32_t buf = g_t[t] & 1, bph = (g_t[t] >> 1) & 1;
-            if (!mbar_wait(&bar->s_empty[t][buf], bph ^ 1, abort_flag, p.status)) { ok = false; break; }
-            tc_fence_after_sync();
+            // the buffer held S and then P of block j - 2, whose P V product was issued in the previous round
+            const uint32_t buf = g_t[t] & 1;
             const uint32_t k_addr = k_addr0 + kst * G_::KV_BYTES;
 #pragma unroll
             for (int ks = 0; ks < DH / 16; ++ks) {
@@ -298,17 +343,16 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
     const int r = threadIdx.x & 127;              // row of the tile = TMEM lane
     const uint32_t lane_base = uint32_t((warp & 3) * 32) << 16;
     const uint32_t s_col = G_::S0 + t * 128, o_col = G_::O0 + t * DH;
-    uint8_t* p_tile = p_smem + t * 2 * G_::P_BYTES;
     uint32_t g = 0;                               // blocks this tile has processed, over all items
     for (;;) {
       bool ok = mbar_wait(&bar->ring_full[rs], rph, abort_flag, p.status);
       if (!__all_sync(0xffffffffu, ok)) break;
       const int item = bar->ring_item[rs];
+      const ItemView v = bar->ring_view[rs];
       __syncwarp();
       if (lane == 0) mbar_arrive(&bar->ring_empty[rs]);
       if (++rs == 2) { rs = 0; rph ^= 1; }
       if (item >= p.n_prefill_items) break;
-      const ItemView v = view_item(p, item, Mt);
       const int nblk = v.nblk_t[t], n_tok = v.n_tok_t[t];
       if (nblk == 0) { blk_base += v.nblk; continue; }            // the item has no tile for this warp group
       const int hg = r / Mt, tok = r - hg * Mt;
@@ -327,8 +371,6 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         tmem_ld32(tmem + lane_base + s_col + buf * PF_KEYS, sreg);
         tmem_ld32(tmem + lane_base + s_col + buf * PF_KEYS + 32, sreg2);
         tmem_ld_wait();
-        tc_fence_before_sync();
-        mbar_arrive(&bar->s_empty[t][buf]);
         if (key0 + PF_KEYS - 1 > pos) {               // this row does not see every key of the block
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
@@ -363,13 +405,11 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
           pk[16 + (e >> 1)] = pack_bf16(b0, b1);
         }
         l_run = l_run * alpha + sum;
-        // every earlier P V product of this tile has completed from here on: the P buffer written below (read by
-        // the product two blocks back) is free, and O is at rest for the rescale
-        if (g > 0) {
-          ok = mbar_wait(&bar->o_full[t], (g - 1) & 1, abort_flag, p.status);
-          if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
-        }
         if (rescale) {
+          // O must be at rest: the P V product of the previous block has completed (its successor cannot be issued
+          // before this warp group hands over P)
+          ok = mbar_wait(&bar->o_full[t][(g - 1) & 1], ((g - 1) >> 1) & 1, abort_flag, p.status);
+          if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
           tc_fence_after_sync();
 #pragma unroll
           for (int c = 0; c < DH / 32; ++c) {
@@ -381,10 +421,8 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
           }
           tmem_st_wait();
         }
-        uint8_t* prow = p_tile + buf * G_::P_BYTES + r * 128;
-#pragma unroll
-        for (int u = 0; u < 8; ++u)
-          *reinterpret_cast<uint4*>(prow + ((u ^ (r & 7)) << 4)) = make_uint4(pk[4 * u], pk[4 * u + 1], pk[4 * u + 2], pk[4 * u + 3]);
+        // P over the first 32 columns of the S buffer just read: column c of row r = keys 2 c, 2 c + 1
+        tmem_st32(tmem + lane_base + s_col + buf * PF_KEYS, pk);
         // ragged last block of the item: V rows of keys that do not exist must not carry stray NaN / Inf bits
         const int n_valid = v.n_keys - key0;
         if (n_valid < PF_KEYS) {
@@ -398,14 +436,15 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
             *reinterpret_cast<uint4*>(vst + h * 8192 + (k >> 4) * 2048 + (k & 15) * 128 + (u << 4)) =
                 make_uint4(0, 0, 0, 0);
           }
+          fence_proxy_async();
         }
-        fence_proxy_async();
+        tmem_st_wait();
         tc_fence_before_sync();
         mbar_arrive(&bar->p_full[t][buf]);
       }
       if (!ok) break;
       // the item's last P V product, then the tile's rows of O leave through registers
-      ok = mbar_wait(&bar->o_full[t], (g - 1) & 1, abort_flag, p.status);
+      ok = mbar_wait(&bar->o_full[t][(g - 1) & 1], ((g - 1) >> 1) & 1, abort_flag, p.status);
       if (!__all_sync(0xffffffffu, ok)) break;
       tc_fence_after_sync();
       const float inv = 1.f / l_run;
