@@ -23,9 +23,9 @@
 //               the overlay safe: S of block j + 2 is issued after the P V product of block j, whose P it replaces.  K and V blocks arrive by TMA in two rings of their own
 //               ([half][page][16][64] tiles with the 128-byte swizzle, the K tile being a K-major and the V tile an
 //               MN-major operand): a K slot is free again as soon as the block's scores are computed, a V slot
-//               after its P V products.  The producer owns the work queue and runs ahead across items.
-//   roles       warps 0..3 softmax of tile A, warps 4..7 softmax of tile B (thread = row = TMEM lane), warp 8 TMA
-//               producer, warp 9 MMA issuer and TMEM owner.
+//               after its P V products.  The producers own the work queue and run ahead across items.
+//   roles       warps 0..3 softmax of tile A, warps 4..7 softmax of tile B (thread = row = TMEM lane), warp 8 and
+//               warps 11..13 TMA producers, warp 9 MMA issuer of tile A and TMEM owner, warp 10 MMA issuer of tile B.
 // Keys past the end of a sequence are masked by selection on the key index, and the matching V rows are
 // zeroed in shared memory before the P V product, so arbitrary bytes in unused cache slots cannot reach
 // the output.  An item's result does not depend on which block ran it: outputs are budget independent.
@@ -38,7 +38,7 @@ namespace hs {
 namespace {
 
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int PF_THREADS = 320, PF_KEYS = 64;
+constexpr int PF_THREADS = 448, PF_KEYS = 64;
 constexpr int PF_KSTAGES = 4, PF_VSTAGES = 4;
 constexpr int TMEM_COLS = 512;
 constexpr float kRefSlack = 8.f;   // log2 units by which a row's running maximum may exceed its reference
@@ -157,9 +157,9 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
 
   if (threadIdx.x == 0) {
     mbar_init(&bar->q_full, 1);
-    mbar_init(&bar->q_empty, 1);
-    for (int i = 0; i < PF_KSTAGES; ++i) { mbar_init(&bar->k_full[i], 1); mbar_init(&bar->k_empty[i], 1); }
-    for (int i = 0; i < PF_VSTAGES; ++i) { mbar_init(&bar->v_full[i], 1); mbar_init(&bar->v_empty[i], 1); }
+    mbar_init(&bar->q_empty, 2);              // one arrival per MMA thread
+    for (int i = 0; i < PF_KSTAGES; ++i) { mbar_init(&bar->k_full[i], 2); mbar_init(&bar->k_empty[i], 2); }
+    for (int i = 0; i < PF_VSTAGES; ++i) { mbar_init(&bar->v_full[i], 2); mbar_init(&bar->v_empty[i], 2); }
     for (int t = 0; t < 2; ++t) {
       for (int i = 0; i < 2; ++i) {
         mbar_init(&bar->s_full[t][i], 1);
@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bar->ring_full[i], 1);
-      mbar_init(&bar->ring_empty[i], 9);      // eight softmax warps + the MMA warp
+      mbar_init(&bar->ring_empty[i], 13);     // eight softmax warps, two MMA warps, three further producers
     }
     bar->abort_flag = 0;
     fence_barrier_init();
@@ -192,34 +192,48 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
   uint32_t n_items_seen = 0;
   uint32_t blk_base = 0;  // key blocks of all earlier items of this thread block (K / V ring position)
 
-  if (warp == 8) {
-    // =========================================================== TMA producer ==
-    // Lane 0 waits and issues; the whole warp fetches page ids: lane l holds the id of page 32 c + l of the item
-    // for the current chunk c of 8 key blocks (one coalesced load per chunk, requested a chunk ahead), so that no
-    // round trip to the block table stands in front of a page request.
+  if (warp == 8 || warp >= 11) {
+    // ========================================================== TMA producers ==
+    // Four warps share the page requests (a bulk tensor copy costs its issuing thread well over a hundred cycles,
+    // and a 64-key block needs sixteen of them: one thread could not keep up with the tensor core): producer 0
+    // (warp 8) owns the work queue, loads the Q tiles and pages 0, 1 of every K block; producer 1 pages 2, 3 of K;
+    // producers 2 and 3 the same halves of V.  Lane 0 of each waits and issues; the whole warp fetches page ids:
+    // lane l holds the id of page 32 c + l of the item for the current chunk c of 8 key blocks (one coalesced load per
+    // chunk, requested a chunk ahead), so that no round trip to the block table stands in front of a page request.
+    const int pi = warp == 8 ? 0 : warp - 10;           // producer index 0..3
+    const int kv = pi >> 1, w0 = (pi & 1) * 2;          // K or V; first of its two pages in a block
     for (;;) {
       int item = 0;
       bool ok = true;
-      if (lane == 0) {
-        ok = mbar_wait(&bar->ring_empty[rs], rph ^ 1, abort_flag, p.status);
-        if (ok) item = atomicAdd(p.counters, 1);
-      }
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      item = __shfl_sync(0xffffffffu, item, 0);
       ItemView v{};
-      if (item < p.n_prefill_items) v = view_item(p, item, Mt);
-      if (lane == 0) {
-        bar->ring_item[rs] = item;
-        bar->ring_view[rs] = v;
-        mbar_arrive(&bar->ring_full[rs]);
+      if (pi == 0) {
+        if (lane == 0) {
+          ok = mbar_wait(&bar->ring_empty[rs], rph ^ 1, abort_flag, p.status);
+          if (ok) item = atomicAdd(p.counters, 1);
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        item = __shfl_sync(0xffffffffu, item, 0);
+        if (item < p.n_prefill_items) v = view_item(p, item, Mt);
+        if (lane == 0) {
+          bar->ring_item[rs] = item;
+          bar->ring_view[rs] = v;
+          mbar_arrive(&bar->ring_full[rs]);
+        }
+      } else {
+        ok = mbar_wait(&bar->ring_full[rs], rph, abort_flag, p.status);
+        if (!__all_sync(0xffffffffu, ok)) break;
+        item = bar->ring_item[rs];
+        v = bar->ring_view[rs];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bar->ring_empty[rs]);
       }
       if (++rs == 2) { rs = 0; rph ^= 1; }
       if (item >= p.n_prefill_items) break;
       const int32_t* table = p.block_tables + size_t(v.seq) * p.max_pages_per_seq;
       const int n_pages = (v.n_keys + 15) >> 4;
       int pg_next = lane < n_pages ? table[lane] : 0, pg_cur = 0;
-      if (lane == 0) {
+      if (pi == 0 && lane == 0) {
         // Q tiles: one box of Mt token rows x 64 columns per (tile, head, half)
         ok = mbar_wait(&bar->q_empty, (n_items_seen & 1) ^ 1, abort_flag, p.status);
         if (ok) {
@@ -242,64 +256,74 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         }
         const uint32_t gb = blk_base + kb;
         const int rem = v.n_keys - kb * PF_KEYS;
-        const int np = rem >= PF_KEYS ? 4 : (rem + 15) >> 4;
-        for (int kv = 0; kv < 2 && ok; ++kv) {
-          const uint32_t st = gb % (kv ? PF_VSTAGES : PF_KSTAGES), ph = (gb / (kv ? PF_VSTAGES : PF_KSTAGES)) & 1;
-          uint64_t* full = kv ? &bar->v_full[st] : &bar->k_full[st];
-          uint8_t* dst = (kv ? v_smem : k_smem) + st * G_::KV_BYTES;
-          if (lane == 0) {
-            ok = mbar_wait(kv ? &bar->v_empty[st] : &bar->k_empty[st], ph ^ 1, abort_flag, p.status);
-            if (ok) mbar_expect_tx(full, np * G_::HALVES * 2048);
+        const int np = rem >= PF_KEYS ? 4 : (rem + 15) >> 4;        // pages of the block that exist
+        const int mine = np - w0 >= 2 ? 2 : (np - w0 > 0 ? np - w0 : 0);
+        const uint32_t st = gb % (kv ? PF_VSTAGES : PF_KSTAGES), ph = (gb / (kv ? PF_VSTAGES : PF_KSTAGES)) & 1;
+        uint64_t* full = kv ? &bar->v_full[st] : &bar->k_full[st];
+        uint8_t* dst = (kv ? v_smem : k_smem) + st * G_::KV_BYTES;
+        if (lane == 0) {
+          ok = mbar_wait(kv ? &bar->v_empty[st] : &bar->k_empty[st], ph ^ 1, abort_flag, p.status);
+          if (ok) {
+            if (mine > 0) mbar_expect_tx(full, mine * G_::HALVES * 2048);
+            else mbar_arrive(full);                                  // nothing to fetch, but the block counts on two arrivals
           }
-          ok = __shfl_sync(0xffffffffu, ok, 0);
-          if (!ok) break;
-          for (int w = 0; w < np; ++w) {
-            const int page = __shfl_sync(0xffffffffu, pg_cur, (kb & 7) * 4 + w);
-            if (lane == 0) {
-              const int row = pool_row(p, kv, page, v.hk);
-              for (int h = 0; h < G_::HALVES; ++h) tma_load_2d(dst + h * 8192 + w * 2048, &p.tm_kv, full, h * 64, row);
-            }
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        for (int w = w0; w < w0 + mine; ++w) {
+          const int page = __shfl_sync(0xffffffffu, pg_cur, (kb & 7) * 4 + w);
+          if (lane == 0) {
+            const int row = pool_row(p, kv, page, v.hk);
+            for (int h = 0; h < G_::HALVES; ++h) tma_load_2d(dst + h * 8192 + w * 2048, &p.tm_kv, full, h * 64, row);
           }
         }
       }
       if (!ok) break;
       blk_base += v.nblk;
     }
-  } else if (warp == 9) {
-    // ============================================================= MMA issuer ==
+  } else if (warp == 9 || warp == 10) {
+    // ============================================================ MMA issuers ==
+    // One issuing thread per tile (warp 9: tile A, warp 10: tile B).  Every wait and every commit costs its thread
+    // on the order of a hundred cycles even when nothing has to be waited for; with a thread per tile those sit
+    // beside the other tile's MMAs instead of between them (the tensor core takes the instructions of both threads
+    // in the order they arrive; each thread's own order is all that the overlay of P on S relies on).
+    // The K and V slots and the Q tiles are released by both threads (barriers of two arrivals): a thread with
+    // no block to compute -- its tile is absent or shorter -- arrives without a commit, but only after it has seen
+    // the slot filled, so that its arrival cannot fall into an earlier phase of the barrier.
     if (lane == 0) {
+      const int t = warp - 9;
       constexpr uint32_t idesc_s = umma_idesc_bf16_f32(128, PF_KEYS);
       constexpr uint32_t idesc_pv = umma_idesc_bf16_f32(128, DH) | (1u << 16);   // B (= V) is MN-major
-      const uint32_t q_addr = smem_u32(q_smem), k_addr0 = smem_u32(k_smem), v_addr0 = smem_u32(v_smem);
-      uint32_t g_t[2] = {0, 0};          // blocks of each tile whose S has been issued, over all items
-      uint32_t pv_t[2] = {0, 0};         // blocks of each tile whose P V has been issued
+      // descriptors of this tile's Q / the first K slot / the first V slot (shared memory is below 256 KB, so adding
+      // byte offsets / 16 to a descriptor never carries out of its address field)
+      const uint64_t q_desc = umma_desc_kmajor_sw128(smem_u32(q_smem) + t * G_::Q_BYTES);
+      const uint64_t k_desc0 = umma_desc_kmajor_sw128(smem_u32(k_smem));
+      const uint64_t v_desc0 = umma_desc_mnmajor_sw128(smem_u32(v_smem), 8192, 1024);
+      const uint32_t d_o = tmem + G_::O0 + t * DH, s_base = tmem + G_::S0 + t * 128;
+      uint32_t g_s = 0, g_pv = 0;        // blocks of this tile whose S / whose P V has been issued, over all items
       bool ok = true;
-      // O(tile) (+)= P(tile, buffer) * V(block gb); `first` = first block of the item (overwrites O)
-      auto issue_pv = [&](int t, uint32_t gb, bool first) -> bool {
-        const uint32_t c = pv_t[t], buf = c & 1, bph = (c >> 1) & 1;
+      // O (+)= P(buffer) * V(block gb) for block j of the item, then the V slot goes back to the producer
+      auto pv_block = [&](const ItemView& v, int j) -> bool {
+        const uint32_t gb = blk_base + j, vst = gb % PF_VSTAGES;
+        if (!mbar_wait(&bar->v_full[vst], (gb / PF_VSTAGES) & 1, abort_flag, p.status)) return false;
+        if (j >= v.nblk_t[t]) {                                     // nothing of this tile in the block
+          mbar_arrive(&bar->v_empty[vst]);
+          return true;
+        }
+        const uint32_t buf = g_pv & 1, bph = (g_pv >> 1) & 1;
         if (!mbar_wait(&bar->p_full[t][buf], bph, abort_flag, p.status)) return false;
         tc_fence_after_sync();
-        const uint32_t v_addr = v_addr0 + (gb % PF_VSTAGES) * G_::KV_BYTES;
+        const uint64_t vdesc = v_desc0 + uint64_t(vst * (G_::KV_BYTES >> 4));
+        const uint32_t a_p = s_base + buf * PF_KEYS, acc0 = j == 0 ? 0u : 1u;    // the item's first block overwrites O
 #pragma unroll
-        for (int pg = 0; pg < 4; ++pg) {      // 16 keys (one page) per MMA: 8 columns of P
-          const uint64_t bdesc = umma_desc_mnmajor_sw128(v_addr + pg * 2048, 8192, 1024);
-          umma_bf16_ts(tmem + G_::O0 + t * DH, tmem + G_::S0 + t * 128 + buf * PF_KEYS + 8 * pg, bdesc, idesc_pv,
-                       (pg != 0 || !first) ? 1u : 0u);
-        }
+        for (int pg = 0; pg < 4; ++pg)        // 16 keys (one page) per MMA: 8 columns of P
+          umma_bf16_ts(d_o, a_p + 8 * pg, vdesc + uint64_t(pg * (2048 >> 4)), idesc_pv, pg != 0 ? 1u : acc0);
         // "P V of block c has completed" alternates between two barriers: a waiter that does not look at every block
         // is then never more than one phase of a barrier away from it (the scores of block c + 2, which it waits for
         // first, complete after the product of block c), so a parity wait cannot mistake one phase for another
         umma_commit(&bar->o_full[t][buf]);
-        ++pv_t[t];
-        return true;
-      };
-      // P V products of block j of the current item, both tiles, then the V slot goes back to the producer
-      auto issue_pv_block = [&](const ItemView& v, int j) -> bool {
-        const uint32_t gb = blk_base + j;
-        if (!mbar_wait(&bar->v_full[gb % PF_VSTAGES], (gb / PF_VSTAGES) & 1, abort_flag, p.status)) return false;
-        for (int t = 0; t < 2; ++t)
-          if (j < v.nblk_t[t] && !issue_pv(t, gb, j == 0)) return false;
-        umma_commit(&bar->v_empty[gb % PF_VSTAGES]);
+        umma_commit(&bar->v_empty[vst]);
+        ++g_pv;
         return true;
       };
       for (;;) {
@@ -309,31 +333,32 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         mbar_arrive(&bar->ring_empty[rs]);
         if (++rs == 2) { rs = 0; rph ^= 1; }
         if (item >= p.n_prefill_items) break;
+        const int nblk = v.nblk_t[t];
         if (!mbar_wait(&bar->q_full, n_items_seen & 1, abort_flag, p.status)) break;
         ++n_items_seen;
+        if (nblk == 0) mbar_arrive(&bar->q_empty);
         for (int j = 0; j < v.nblk && ok; ++j) {
           const uint32_t gb = blk_base + j, kst = gb % PF_KSTAGES;
           if (!mbar_wait(&bar->k_full[kst], (gb / PF_KSTAGES) & 1, abort_flag, p.status)) { ok = false; break; }
-          for (int t = 0; t < 2 && ok; ++t) {
-            if (j >= v.nblk_t[t]) continue;
-            // the buffer held S and then P of block j - 2, whose P V product was issued in the previous round
-            const uint32_t buf = g_t[t] & 1;
-            const uint32_t k_addr = k_addr0 + kst * G_::KV_BYTES;
+          if (j < nblk) {
+            tc_fence_after_sync();
+            // the buffer held S and then P of block j - 2, whose P V product this thread issued in the previous round
+            const uint32_t buf = g_s & 1;
+            const uint64_t kdesc = k_desc0 + uint64_t(kst * (G_::KV_BYTES >> 4));
 #pragma unroll
-            for (int ks = 0; ks < DH / 16; ++ks) {
-              const uint64_t a = umma_desc_kmajor_sw128(q_addr + t * G_::Q_BYTES + (ks >> 2) * 16384) + 2 * (ks & 3);
-              const uint64_t b = umma_desc_kmajor_sw128(k_addr + (ks >> 2) * 8192) + 2 * (ks & 3);
-              umma_bf16(tmem + G_::S0 + t * 128 + buf * PF_KEYS, a, b, idesc_s, ks != 0);
-            }
+            for (int ks = 0; ks < DH / 16; ++ks)
+              umma_bf16(s_base + buf * PF_KEYS, q_desc + uint64_t((ks >> 2) * (16384 >> 4) + 2 * (ks & 3)),
+                        kdesc + uint64_t((ks >> 2) * (8192 >> 4) + 2 * (ks & 3)), idesc_s, ks != 0);
             umma_commit(&bar->s_full[t][buf]);
-            ++g_t[t];
+            umma_commit(&bar->k_empty[kst]);                        // the K slot, once these scores are computed
+            if (j == nblk - 1) umma_commit(&bar->q_empty);          // and the Q tile after the tile's last scores
+            ++g_s;
+          } else {
+            mbar_arrive(&bar->k_empty[kst]);
           }
-          if (!ok) break;
-          umma_commit(&bar->k_empty[kst]);                          // the K slot, once these scores are computed
-          if (j == v.nblk - 1) umma_commit(&bar->q_empty);          // and the Q tiles after the item's last scores
-          if (j > 0) ok = issue_pv_block(v, j - 1);                 // overlaps the softmax of block j
+          if (j > 0) ok = pv_block(v, j - 1);                       // overlaps the softmax of block j
         }
-        if (!ok || !issue_pv_block(v, v.nblk - 1)) break;
+        if (!ok || !pv_block(v, v.nblk - 1)) break;
         blk_base += v.nblk;
       }
     }
