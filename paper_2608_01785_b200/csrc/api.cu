@@ -605,6 +605,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     go.pair = pair_d;
     go.bn = pair_d ? 256 : gemm_pick_bn(T, d, s->sm_count);
     go.ksplit = pair_d ? 1 : pick_ksplit(T, d, q_dim, go.bn, s->sm_count);
+    go.stream_k_slots = pair_d ? gemm_pick_stream_k(T, d, q_dim, s->sm_count) : 0;
     go.tile_turn = reinterpret_cast<int*>(s->ws_dev + s->ws.turn);
     go.status = status;
     go.smid_log = slots(5);
@@ -658,6 +659,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gd.pair = pair_d;
     gd.bn = pair_d ? 256 : gemm_pick_bn(T, d, s->sm_count);
     gd.ksplit = pair_d ? 1 : pick_ksplit(T, d, F, gd.bn, s->sm_count);
+    gd.stream_k_slots = pair_d ? gemm_pick_stream_k(T, d, F, s->sm_count) : 0;
     gd.tile_turn = reinterpret_cast<int*>(s->ws_dev + s->ws.turn);
     gd.status = status;
     gd.smid_log = slots(7);
@@ -758,6 +760,22 @@ hs_status_t hs_stage_debug_buffer(hs_stage_t* s, const char* name, void** dev_pt
   return HS_OK;
 }
 
+// Whose-turn words for bare GEMM calls: a zero-initialised array of the library image (device symbols start at zero and
+// the kernels leave the words at zero), its device address resolved once per device.
+static __device__ int g_op_turn[hs::kGemmTurnWords];
+static int* op_turn_words(int dev) {
+  static std::mutex m;
+  static int* ptr[64] = {};
+  if (dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(m);
+  if (!ptr[dev]) {
+    void* q = nullptr;
+    if (cudaGetSymbolAddress(&q, g_op_turn) != cudaSuccess) return nullptr;
+    ptr[dev] = static_cast<int*>(q);
+  }
+  return ptr[dev];
+}
+
 static hs_status_t op_gemm(const void* a, const void* w, const float* resid, float* out, int32_t M, int32_t N, int32_t K,
                            int32_t sm_budget, int32_t* status_dev, void* cuda_stream, int ab_f16) {
   if (!a || !w || !out || !status_dev || M < 1 || N < 1 || K < 1) return HS_ERR_INVALID_ARG;
@@ -796,6 +814,14 @@ static hs_status_t op_gemm(const void* a, const void* w, const float* resid, flo
   g.pair = M > 128;
   g.bn = g.pair ? 256 : gemm_pick_bn(M, N, sm_count);
   g.status = status_dev;
+  // The ordered adds of the stream-K form need whose-turn words that are zero between launches.  A bare GEMM call has
+  // no stage workspace, so it uses a word array of the library image (shared by all bare GEMM calls of the process:
+  // such calls must not overlap on the GPU when they take this form; the stage's GEMMs use the stage's own words).
+  g.stream_k_slots = g.pair ? gemm_pick_stream_k(M, N, K, sm_count) : 0;
+  if (g.stream_k_slots > 0) {
+    g.tile_turn = op_turn_words(dev);
+    if (!g.tile_turn) g.stream_k_slots = 0;
+  }
   const cudaError_t e = launch_gemm(g, sm_budget, stream);
   return e == cudaSuccess ? HS_OK : cuda_fail("gemm", e);
 }

@@ -158,6 +158,90 @@ __device__ __forceinline__ __nv_bfloat16* cache_ptr(__nv_bfloat16* base, int slo
   return base + row * Dh + e;
 }
 
+// One work unit of a block (pair): the K blocks [kb_begin, kb_end) of an output tile.  `seg` counts the earlier K
+// segments of the same tile (their sums are added into the output before this one's), `last` marks the tile's final
+// segment.
+struct Unit { int tile, kb_begin, kb_end, seg, last, half; };
+
+// Hands a worker its units, in the same order for the producer, the MMA issuer and the epilogue warps.
+//   plain / split-K   unit u = worker + i * workers over tiles x splits, split-major (a split's predecessors have
+//                     smaller unit numbers).
+//   stream-K          (Resid mode on pairs, chosen by shape) the tiles' K blocks, laid end to end tile after tile, are
+//                     cut into `n_slots` equal runs -- one per pair of the whole device, whatever the budget -- so that
+//                     no pair idles through a ragged last wave.  A run is a tail segment of one tile, whole tiles, and
+//                     a head segment of another; slot s is worked by worker s mod workers.  Within a slot the head
+//                     segment comes first and the tail segment last: the tail's predecessor is the head segment of
+//                     the previous slot, which that slot has done first, so the ordered add never waits long.
+//                     With sm_budget 1 there is no pair: the single block then works the same slots on the same
+//                     256-row tiles, each unit twice -- once per 128-row half (`half`) -- so that every output
+//                     element still receives the same partial sums in the same order.
+struct UnitWalk {
+  int stream_k, n_tiles, k_blocks, ksplit, kb_per, n_workers, n_slots;
+  int halves, n_m_tiles, M;  // halves = 2: a single block standing in for a pair
+  int cur;                 // unit (plain) or slot (stream-K) being handed out
+  int idx, n_seg, first_tile;
+  long long lo, hi;
+  __device__ __forceinline__ void init(const GemmParams& p, bool pair, bool emulate_pair, int n_m_tiles_, int n_tiles_,
+                                       int k_blocks_, int worker, int n_workers_) {
+    stream_k = (pair || emulate_pair) && p.mode == kGemmResid && p.stream_k_slots > 0;
+    halves = emulate_pair ? 2 : 1;
+    n_m_tiles = n_m_tiles_;
+    M = p.M;
+    n_tiles = n_tiles_; k_blocks = k_blocks_; n_workers = n_workers_;
+    ksplit = !pair && p.mode == kGemmResid && p.ksplit > 1 ? p.ksplit : 1;
+    kb_per = (k_blocks + ksplit - 1) / ksplit;
+    n_slots = stream_k ? p.stream_k_slots : n_tiles * ksplit;
+    cur = worker - n_workers;
+    idx = n_seg = 0; first_tile = 0; lo = hi = 0;
+  }
+  __device__ __forceinline__ bool next(Unit& u) {
+    if (halves == 2 && idx > 0 && u.half == 0) {   // the second half of the unit handed out last, if it has rows
+      if ((2 * (u.tile % n_m_tiles) + 1) * BM < M) {
+        u.half = 1;
+        return true;
+      }
+    }
+    u.half = 0;
+    if (!stream_k) {
+      cur += n_workers;
+      if (cur >= n_slots) return false;
+      const int ks = cur / n_tiles;
+      u.tile = cur - ks * n_tiles;
+      u.kb_begin = ks * kb_per;
+      u.kb_end = min(k_blocks, u.kb_begin + kb_per);
+      u.seg = ks;
+      u.last = ks == ksplit - 1;
+      return true;
+    }
+    const long long total = (long long)n_tiles * k_blocks;
+    while (idx == n_seg) {                         // next slot of this worker (empty slots are skipped)
+      cur += n_workers;
+      if (cur >= n_slots) return false;
+      lo = total * cur / n_slots;
+      hi = total * (cur + 1) / n_slots;
+      idx = 0;
+      n_seg = 0;
+      if (hi > lo) {
+        first_tile = int(lo / k_blocks);
+        n_seg = int((hi - 1) / k_blocks) - first_tile + 1;
+      }
+    }
+    const int nat = n_seg == 1 ? 0 : (idx == 0 ? n_seg - 1 : (idx == n_seg - 1 ? 0 : idx));
+    const int t = first_tile + nat;
+    const long long t0 = (long long)t * k_blocks;
+    const long long b = lo > t0 ? lo : t0, e = hi < t0 + k_blocks ? hi : t0 + k_blocks;
+    u.tile = t;
+    u.kb_begin = int(b - t0);
+    u.kb_end = int(e - t0);
+    // earlier segments of the tile = slot boundaries inside the tile before this segment; the slot that holds the
+    // tile's first K block is ceil((t0 + 1) n_slots / total) - 1
+    u.seg = u.kb_begin == 0 ? 0 : cur - (int(((t0 + 1) * n_slots + total - 1) / total) - 1);
+    u.last = u.kb_end == k_blocks;
+    ++idx;
+    return true;
+  }
+};
+
 template <bool PAIR>
 __device__ __forceinline__ void gemm_body(const GemmParams& p) {
   // Ring geometry.  Pairs: 6 stages of 32 KB.  Single blocks: a stage holds the A box (128 rows, or only 64 / 32
@@ -187,15 +271,18 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
   const uint32_t rank = PAIR ? cluster_ctarank() : 0;
   const int worker = PAIR ? int(blockIdx.x >> 1) : int(blockIdx.x);
   const int n_workers = PAIR ? int(gridDim.x >> 1) : int(gridDim.x);
-  const int n_m_tiles = PAIR ? (p.M + 2 * BM - 1) / (2 * BM) : (p.M + BM - 1) / BM;
+  // a single block that stands in for a pair (stream-K form at sm_budget 1) walks the pair's 256-row tiles
+  const bool emulate_pair = !PAIR && p.pair && p.mode == kGemmResid && p.stream_k_slots > 0;
+  const int n_m_tiles = PAIR || emulate_pair ? (p.M + 2 * BM - 1) / (2 * BM) : (p.M + BM - 1) / BM;
   const int n_n_tiles = gemm_n_tiles(p);
   const int n_tiles = n_m_tiles * n_n_tiles;
   const int k_blocks = (p.K + BK - 1) / BK;
-  // Work unit = (output tile, K split).  Splits exist only in Resid mode with few tiles; units are ordered
-  // split-major, so the units a split has to wait for always have smaller indices.
-  const int ksplit = !PAIR && p.mode == kGemmResid && p.ksplit > 1 ? p.ksplit : 1;
-  const int kb_per = (k_blocks + ksplit - 1) / ksplit;
-  const int n_units = n_tiles * ksplit;
+  // Work unit = (output tile, run of K blocks): see UnitWalk.  Runs shorter than the whole K range exist only in
+  // Resid mode, whose epilogue adds partial sums into the output in a fixed order.
+  UnitWalk walk;
+  walk.init(p, PAIR, emulate_pair, n_m_tiles, n_tiles, k_blocks, worker, n_workers);
+  const bool ordered = walk.stream_k || walk.ksplit > 1;
+  Unit un;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) {
@@ -239,12 +326,12 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
       // rows starting at the stage's base -- beyond the A box that is the B data of the stage, finite values
       // that only reach accumulator rows no epilogue stores
       const bool two_halves = b_two;
-      for (int u = worker; u < n_units && ok; u += n_workers) {
-        const int tile = u % n_tiles, ks = u / n_tiles;
+      while (ok && walk.next(un)) {
+        const int tile = un.tile;
         const int m = tile % n_m_tiles, n = tile / n_m_tiles;
         const BSource b0 = b_source(p, n, PAIR ? int(rank) : 0), b1 = b_source(p, n, 1);
-        const int kb_end = min(k_blocks, (ks + 1) * kb_per);
-        for (int kb = ks * kb_per; kb < kb_end; ++kb) {
+        const int kb_end = un.kb_end;
+        for (int kb = un.kb_begin; kb < kb_end; ++kb) {
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status)) { ok = false; break; }
           uint8_t* st = smem + s * STAGE_BYTES;
           if (PAIR) {
@@ -255,7 +342,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
             tma_load_2d_pair(st + b_off, &p.tm_b[b0.map], bar, kb * BK, b0.row);
           } else {
             mbar_expect_tx(&full[s], a_bytes + (two_halves ? 2 * BH_BYTES : BH_BYTES));
-            tma_load_2d(st, &p.tm_a, &full[s], kb * BK, m * BM);
+            tma_load_2d(st, &p.tm_a, &full[s], kb * BK, (emulate_pair ? 2 * m + un.half : m) * BM);
             tma_load_2d(st + b_off, &p.tm_b[b0.map], &full[s], kb * BK, b0.row);
             if (two_halves) tma_load_2d(st + b_off + BH_BYTES, &p.tm_b[b1.map], &full[s], kb * BK, b1.row);
           }
@@ -274,11 +361,11 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
       bool ok = true;
-      for (int u = worker; u < n_units && ok; u += n_workers) {
+      while (ok && walk.next(un)) {
         if (!mbar_wait(&tempty[acc], acc_ph ^ 1, abort_flag, p.status)) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        const int kb_begin = (u / n_tiles) * kb_per, kb_end = min(k_blocks, kb_begin + kb_per);
+        const int kb_begin = un.kb_begin, kb_end = un.kb_end;
         for (int kb = kb_begin; kb < kb_end; ++kb) {
           if (!mbar_wait(&full[s], ph, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after_sync();
@@ -319,9 +406,11 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
     const int Dh = p.head_dim;
     uint8_t* epi_buf = epi_smem + quarter * EPI_WARP_BYTES;
     int epi_sel = 0;                          // staging block to fill next
-    for (int u = worker; u < n_units; u += n_workers) {
-      const int tile = u % n_tiles, ks = u / n_tiles;
-      const int m = PAIR ? 2 * (tile % n_m_tiles) + int(rank) : tile % n_m_tiles, n = tile / n_m_tiles;
+    while (walk.next(un)) {
+      const int tile = un.tile, ks = un.seg;
+      const int m = PAIR ? 2 * (tile % n_m_tiles) + int(rank)
+                         : emulate_pair ? 2 * (tile % n_m_tiles) + un.half : tile % n_m_tiles,
+                n = tile / n_m_tiles;
       const bool ok = mbar_wait(&tfull[acc], acc_ph, abort_flag, p.status);
       if (!__all_sync(0xffffffffu, ok)) break;
       tc_fence_after_sync();
@@ -337,8 +426,8 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
         // Ordered split-K: the partial sums of a tile are added into the output in split order, so the
         // result is the same fixed sum whatever block computed which split.  This warp owns 32 rows of the
         // tile; it waits until the previous split's add of those rows has been performed.
-        int* turn = p.tile_turn + tile * 4 + quarter;
-        if (ksplit > 1 && ks > 0) {
+        int* turn = p.tile_turn + (PAIR ? tile * 2 + int(rank) : emulate_pair ? tile * 2 + un.half : tile) * 4 + quarter;
+        if (ordered && ks > 0) {
           bool go = true;
           if (lane == 0) go = spin_until_equal(turn, ks, abort_flag, p.status);
           if (!__shfl_sync(0xffffffffu, go, 0)) break;
@@ -383,10 +472,10 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
           }
           epi_sel ^= 1;
         }
-        if (ksplit > 1 && lane == 0) {
-          bulk_wait<0>();                     // this split's adds have been performed
+        if (ordered && !(ks == 0 && un.last) && lane == 0) {    // a tile with a single segment needs no turn
+          bulk_wait<0>();                     // this segment's adds have been performed
           __threadfence();
-          st_release(turn, ks == ksplit - 1 ? 0 : ks + 1);   // the last split leaves the word at zero
+          st_release(turn, un.last ? 0 : ks + 1);   // the last segment leaves the word at zero
         }
       } else if (p.mode == kGemmGateUp) {
         for (int c = 0; c < 4; ++c) {
@@ -579,6 +668,24 @@ int gemm_pick_ksplit(int M, int N, int K, int bn, int sm_count) {
   return (k_blocks + per - 1) / per;          // no empty split
 }
 
+int gemm_pick_stream_k(int M, int N, int K, int sm_count) {
+  // Whole 256 x 256 tiles on W pairs take ceil(tiles / W) rounds; cutting the K blocks of all tiles into W equal
+  // runs takes tiles / W rounds' worth, at the price of a second (ordered) add for the tiles that a cut falls into.
+  // Worth it when the last round would be under about 90 % full and K is long: a run that ends inside a tile costs
+  // that tile a second epilogue (the 256 x 256 fp32 block leaves by TMA add-reductions, about a third of the main
+  // loop's time at K = 3584), and a short head or tail segment cannot hide its epilogue behind the next main loop.
+  // Measured on B200 (per launch, whole tiles -> equal runs): 126 tiles of K = 18944 on 74 pairs (1.70 rounds run
+  // as 2) 254 -> 233 us at equal clocks; 184 tiles of K = 5632 (2.49 run as 3) 114 -> 104 us; but 126 tiles of
+  // K = 3584 62 -> 64 us and 184 tiles of K = 2048 53 -> 52 us: no gain below about 64 K blocks.
+  const int W = sm_count / 2;
+  const int tiles = ((M + 2 * BM - 1) / (2 * BM)) * ((N + BN - 1) / BN);
+  const int k_blocks = (K + BK - 1) / BK;
+  if (W < 1 || tiles * 8 > kGemmTurnWords || k_blocks < 64) return 0;
+  if (tiles * 2 < W) return 0;                       // few tiles: single blocks with a K split serve better
+  const int rounds = (tiles + W - 1) / W;
+  return double(tiles) / W < 0.92 * rounds ? W : 0;
+}
+
 cudaError_t launch_gemm(const GemmParams& p, int sm_budget, cudaStream_t stream) {
   const int n_m_tiles = (p.M + BM - 1) / BM;
   const int n_n_tiles = gemm_n_tiles(p);
@@ -586,7 +693,8 @@ cudaError_t launch_gemm(const GemmParams& p, int sm_budget, cudaStream_t stream)
   if (n_tiles <= 0) return cudaSuccess;
   if (p.pair && sm_budget >= 2) {
     // pairs of blocks (clusters of two SMs) on 256 x 256 tiles; an odd budget leaves one SM unused
-    const int pairs = ((p.M + 2 * BM - 1) / (2 * BM)) * n_n_tiles;
+    const int pair_tiles = ((p.M + 2 * BM - 1) / (2 * BM)) * n_n_tiles;
+    const int pairs = p.mode == kGemmResid && p.stream_k_slots > 0 ? p.stream_k_slots : pair_tiles;
     const int grid = 2 * (pairs < sm_budget / 2 ? pairs : sm_budget / 2);
     return launch_step_kernel(gemm_pair_kernel, grid, GEMM_THREADS, GEMM_SMEM, stream, p.overlap != 0, p);
   }

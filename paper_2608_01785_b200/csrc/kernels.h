@@ -39,7 +39,8 @@ struct GemmParams {
   int accumulate;            // 1: out += A W^T (the residual add), 0: out = A W^T
   int bn;                    // tile width of this launch (gemm_pick_bn); 256 when unused
   int ksplit;                // K splits per output tile, added in split order (gemm_pick_ksplit); 0/1 = none
-  int* tile_turn;            // [tiles * 4] whose-turn words for the ordered adds; zero at entry and at exit
+  int stream_k_slots;        // pairs only: > 0 = cut the tiles' K blocks into this many equal runs (gemm_pick_stream_k)
+  int* tile_turn;            // [tiles * 4] ([tiles * 8] on pairs) whose-turn words for the ordered adds; zero at entry and at exit
   // Qkv
   int q_dim, kv_dim, head_dim, n_kv_heads;
   CUtensorMap tm_q;          // bf16 q [M, q_dim], box 64 x 32, 128-byte swizzle
@@ -65,6 +66,9 @@ cudaError_t gemm_set_attributes();
 // Tile width for a Resid-mode GEMM of this shape on a device with sm_count SMs (budget independent).
 int gemm_pick_bn(int M, int N, int sm_count);
 int gemm_pick_ksplit(int M, int N, int K, int bn, int sm_count);
+// Runs for the stream-K form of a Resid-mode GEMM on pairs (one per pair of the device), or 0 when whole tiles
+// already fill their waves well enough (budget independent).
+int gemm_pick_stream_k(int M, int N, int K, int sm_count);
 // The same three GEMMs for steps of at most 64 rows (gemm_skinny.cu): weight streaming on plain loads and
 // warp-level MMAs, one block per 32 output columns and the whole K range, no K split across blocks.
 struct SkinnyParams {
