@@ -18,9 +18,10 @@ namespace hs {
 namespace {
 
 constexpr int kRing = 4;   // pinned staging slots for step metadata
+constexpr int kRowSsStride = 64;   // partial sums of x^2 kept per token: one per 128-column tile of d_model at most
 
 struct WsLayout {
-  size_t rope, h, q, o, act, meta, part_o, part_ml, status, turn, smid, w16, w16_layer, total;
+  size_t rope, h, q, o, act, meta, part_o, part_ml, status, turn, smid, row_ss, row_rs, row_done, w16, w16_layer, total;
 };
 
 // elements of the i-th weight matrix of a layer, in the order w_q, w_k, w_v, w_o, w_gate, w_up, w_down
@@ -51,6 +52,9 @@ WsLayout make_ws_layout(const hs_stage_config_t& c, const MetaLayout& ml) {
   w.status = take(256);
   w.turn = take(kGemmTurnWords * 4);
   w.smid = take(size_t(HS_PROFILE_CLASSES) * kSmidSlots * 4);
+  w.row_ss = take(T * kRowSsStride * 4);             // partial sums of x^2 per (token, tile column) of a folded RMSNorm
+  w.row_rs = take(T * 4);                            // r of every token
+  w.row_done = take((T / 32 + 2) * 4);               // tile columns delivered per group of 32 token rows
   // fp16 copies of the seven weight matrices of every layer (absent with HS_FLAG_BF16_ACTIVATIONS);
   // within a layer: w_q, w_k, w_v, w_o, w_gate, w_up, w_down, each 1024-byte aligned
   w.w16 = off;
@@ -181,7 +185,7 @@ struct hs_stage {
   std::vector<LayerMaps> maps;
   CUtensorMap tm_h, tm_o, tm_act, tm_kv;   // operand loads
   CUtensorMap tm_h_s[2], tm_o_s[2], tm_act_s[2];   // the same A operands with 64- and 32-row boxes (small steps)
-  CUtensorMap tm_q_st, tm_act_st;          // epilogue stores (box 64 x 32)
+  CUtensorMap tm_q_st, tm_act_st, tm_h_st; // epilogue stores (box 64 x 32)
   CUtensorMap tm_q_attn;                   // Q tiles of the prefill attention (box 64 x tokens per item)
   int32_t* pinned[kRing] = {};
   cudaEvent_t ev[kRing] = {};
@@ -306,7 +310,8 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
   if (cudaMemcpy(s->ws_dev + s->ws.rope, rope.data(), rope.size() * sizeof(float2), cudaMemcpyHostToDevice) !=
           cudaSuccess ||
       cudaMemset(s->ws_dev + s->ws.status, 0, 256) != cudaSuccess ||
-      cudaMemset(s->ws_dev + s->ws.turn, 0, kGemmTurnWords * 4) != cudaSuccess)
+      cudaMemset(s->ws_dev + s->ws.turn, 0, kGemmTurnWords * 4) != cudaSuccess ||
+      cudaMemset(s->ws_dev + s->ws.row_done, 0, (size_t(cfg->max_tokens) / 32 + 2) * 4) != cudaSuccess)
     return cuda_fail("hs_stage_create: workspace initialisation", cudaGetLastError());
 
   // tensor maps
@@ -320,7 +325,7 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
          encode_2d(&s->tm_act_s[i], s->ws_dev + s->ws.act, T, F, rows);
   }
   ok = ok && encode_2d(&s->tm_q_st, s->ws_dev + s->ws.q, T, q_dim, 32) &&
-       encode_2d(&s->tm_act_st, s->ws_dev + s->ws.act, T, F, 32);
+       encode_2d(&s->tm_act_st, s->ws_dev + s->ws.act, T, F, 32) && encode_2d(&s->tm_h_st, s->ws_dev + s->ws.h, T, d, 32);
   ok = ok && encode_2d(&s->tm_q_attn, s->ws_dev + s->ws.q, T, q_dim,
                        prefill_tokens_per_item(cfg->n_q_heads / cfg->n_kv_heads));
   const uint64_t pool_rows = uint64_t(cfg->n_layers) * 2 * cfg->num_pages * cfg->n_kv_heads * kPage;
@@ -499,6 +504,32 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     k.status = status;
     return k;
   };
+  // RMSNorm folded into the GEMMs around it (rmsnorm(x) W^T = diag(r) ((x o g) W^T)): the residual GEMM in front of a
+  // norm emits h = 16-bit(x o g) and the partial sums of x^2 from its epilogue, the GEMM behind it scales its
+  // accumulator rows by r.  Used when all four projections of the step run on pairs of SMs and the stage is not
+  // conditioned (a shift between norm and product breaks the factoring); the first norm of a step, which has no
+  // GEMM in front of it, stays a kernel.  A choice by shape and stage, never by budget.  Measured on B200 the fold
+  // costs each residual GEMM about what the RMSNorm launch it replaces cost (config 2 and 3 steps within 1 % either
+  // way, at the full budget and at partial ones); what it buys is two launches per layer.
+  const int n_ss_tiles = ceil_div(d, pair_d ? 256 : gemm_pick_bn(T, d, s->sm_count));
+  const bool fold_norm = !s->modulation && n_ss_tiles <= kRowSsStride && !skinny(d, q_dim + 2 * kv_dim, kGemmQkv) &&
+                         !skinny(q_dim, d, kGemmResid) && !skinny(d, F, kGemmGateUp) && !skinny(F, d, kGemmResid) &&
+                         pair_d && pair_qkv && pair_gu;
+  float* row_ss = reinterpret_cast<float*>(s->ws_dev + s->ws.row_ss);
+  auto fold_out = [&](GemmParams& gp, const void* gain) {      // producing side
+    gp.norm_gain = static_cast<const __nv_bfloat16*>(gain);
+    gp.tm_norm_h = s->tm_h_st;
+    gp.row_ss = row_ss;
+    gp.ss_stride = kRowSsStride;
+    gp.row_rs = reinterpret_cast<float*>(s->ws_dev + s->ws.row_rs);
+    gp.row_group_done = reinterpret_cast<int*>(s->ws_dev + s->ws.row_done);
+    gp.y_in = x;
+    gp.norm_h_f16 = f16;
+    gp.norm_eps = c.rms_eps;
+  };
+  auto fold_in = [&](GemmParams& gp) {                         // consuming side
+    gp.in_row_rs = reinterpret_cast<const float*>(s->ws_dev + s->ws.row_rs);
+  };
   int* census = s->census ? reinterpret_cast<int*>(s->ws_dev + s->ws.smid) : nullptr;
   if (census && cudaMemsetAsync(census, 0, size_t(HS_PROFILE_CLASSES) * kSmidSlots * 4, stream) != cudaSuccess)
     return HS_ERR_CUDA;
@@ -526,7 +557,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     np.mod = mod_l;
     np.tok_seq = meta + s->ml.tok_seq;
     np.mod_which = 0;
-    { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
+    const bool folded_attn_norm = fold_norm && l > 0;          // the previous layer's down-projection produced h and the sums
+    if (!folded_attn_norm) { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
     GemmParams g{};
@@ -549,6 +581,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     for (int i = 0; i < 3; ++i) g.qkv_bias[i] = s->qkv_bias[l].b[i];
     g.status = status;
     g.smid_log = slots(1);
+    if (folded_attn_norm) fold_in(g);
     if (skinny(d, q_dim + 2 * kv_dim, kGemmQkv)) {
       SkinnyParams k = skinny_base(h, d, q_dim + 2 * kv_dim, kGemmQkv);
       k.w[0] = wo.w_q; k.w[1] = wo.w_k; k.w[2] = wo.w_v;
@@ -609,6 +642,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     go.tile_turn = reinterpret_cast<int*>(s->ws_dev + s->ws.turn);
     go.status = status;
     go.smid_log = slots(5);
+    if (fold_norm) fold_out(go, w.g_mlp);
     if (skinny(q_dim, d, kGemmResid)) {
       SkinnyParams k = skinny_base(o, q_dim, d, kGemmResid);
       k.w[0] = wo.w_o; k.y = x; k.accumulate = 1;
@@ -621,7 +655,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     np.x_bf16 = nullptr;
     np.gain = static_cast<const __nv_bfloat16*>(w.g_mlp);
     np.mod_which = 3;
-    { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
+    if (!fold_norm) { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
     GemmParams gu{};
@@ -637,6 +671,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gu.tm_act = s->tm_act_st;
     gu.status = status;
     gu.smid_log = slots(6);
+    if (fold_norm) fold_in(gu);
     if (skinny(d, F, kGemmGateUp)) {
       SkinnyParams k = skinny_base(h, d, F, kGemmGateUp);
       k.w[0] = wo.w_gate; k.w[1] = wo.w_up;
@@ -663,6 +698,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gd.tile_turn = reinterpret_cast<int*>(s->ws_dev + s->ws.turn);
     gd.status = status;
     gd.smid_log = slots(7);
+    if (fold_norm && l + 1 < c.n_layers) fold_out(gd, s->layers[l + 1].g_attn);
     if (skinny(F, d, kGemmResid)) {
       SkinnyParams k = skinny_base(s->ws_dev + s->ws.act, F, d, kGemmResid);
       k.w[0] = wo.w_down; k.y = x; k.accumulate = 1;

@@ -151,6 +151,33 @@ __device__ __forceinline__ void add_bias32(uint32_t (&r)[32], const __nv_bfloat1
   }
 }
 
+// r[0..31] *= s (fp32 values held as raw bits)
+__device__ __forceinline__ void scale32(uint32_t (&r)[32], float s) {
+#pragma unroll
+  for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * s);
+}
+
+// Folded RMSNorm, producing side: a thread leaves the sum of x^2 of its row over one tile column; the warp that
+// delivers the last tile column of its 32 rows (counted per row group) adds each row's partials in tile-column order --
+// the same sum whoever comes last -- and writes r = rsqrt(mean(x^2) + eps) for the GEMM that follows.
+__device__ __forceinline__ void finish_row_norm(const GemmParams& p, int row, bool row_ok, int row_group, int n,
+                                                int n_n_tiles, float ss, int lane) {
+  if (row_ok) p.row_ss[size_t(row) * p.ss_stride + n] = ss;
+  __threadfence();
+  __syncwarp();
+  int last = 0;
+  if (lane == 0) last = atomicAdd(p.row_group_done + row_group, 1) == n_n_tiles - 1;
+  last = __shfl_sync(0xffffffffu, last, 0);
+  if (!last) return;
+  __threadfence();
+  if (row_ok) {
+    float sum = 0.f;
+    for (int i = 0; i < n_n_tiles; ++i) sum += __ldcg(p.row_ss + size_t(row) * p.ss_stride + i);
+    p.row_rs[row] = rsqrtf(sum / float(p.N) + p.norm_eps);
+  }
+  if (lane == 0) p.row_group_done[row_group] = 0;      // ready for the next launch
+}
+
 // Address of element e of (slot, kv head) in one layer's K or V pages.
 __device__ __forceinline__ __nv_bfloat16* cache_ptr(__nv_bfloat16* base, int slot, int hk, int n_kv_heads, int Dh,
                                                     int e) {
@@ -251,7 +278,10 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
   const bool b_two = p.mode == kGemmGateUp || (p.mode == kGemmResid ? p.bn : gemm_qkv_width(p)) > 128;
   const int a_bytes = (p.a_box_rows > 0 && !PAIR ? p.a_box_rows : BM) * BK * 2;
   const int STAGE_BYTES = PAIR ? Ring<true>::STAGE_BYTES : a_bytes + (b_two ? 2 : 1) * BH_BYTES;
-  const int STAGES = PAIR ? Ring<true>::STAGES
+  // (a pair kernel that folds the following RMSNorm into its epilogue runs its ring one stage short and uses the last
+  // stage's 32 KB as landing blocks for the residual stream: see the epilogue)
+  const bool fold_pair = PAIR && p.mode == kGemmResid && p.norm_gain != nullptr;
+  const int STAGES = PAIR ? Ring<true>::STAGES - (fold_pair ? 1 : 0)
                           : (RING_BYTES / STAGE_BYTES < kMaxStages ? RING_BYTES / STAGE_BYTES : kMaxStages);
   const int b_off = PAIR ? A_BYTES : a_bytes;     // B boxes follow the A box inside a stage
   extern __shared__ uint8_t smem_raw[];
@@ -263,6 +293,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
   uint64_t* tempty = tfull + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  uint64_t* xbar = reinterpret_cast<uint64_t*>(epi_smem + 4 * EPI_WARP_BYTES + 256);   // [4 warps][4] landing-block barriers (three used)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   log_smid(p.smid_log);
@@ -293,6 +324,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
       mbar_init(&tfull[i], 1);
       mbar_init(&tempty[i], PAIR ? 8 : 4);      // one arrival per epilogue warp (of both blocks)
     }
+    for (int i = 0; i < 16; ++i) mbar_init(&xbar[i], 1);
     *abort_flag = 0;
     fence_barrier_init();
     tma_prefetch_desc(&p.tm_a);
@@ -406,28 +438,55 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
     const int Dh = p.head_dim;
     uint8_t* epi_buf = epi_smem + quarter * EPI_WARP_BYTES;
     int epi_sel = 0;                          // staging block to fill next
+    uint32_t xph = 0;                         // phase bits of this warp's landing-block barriers
     while (walk.next(un)) {
       const int tile = un.tile, ks = un.seg;
       const int m = PAIR ? 2 * (tile % n_m_tiles) + int(rank)
                          : emulate_pair ? 2 * (tile % n_m_tiles) + un.half : tile % n_m_tiles,
                 n = tile / n_m_tiles;
+      const int row = m * BM + quarter * 32 + lane;
+      const bool row_ok = row < p.M;
+      const int row_base = m * BM + quarter * 32;          // first row of this warp's 32
+      // folded RMSNorm, consuming side: r of this thread's row, requested before the wait for the accumulator
+      float rs = 1.f;
+      if (p.in_row_rs != nullptr && p.mode != kGemmResid && row_ok) rs = __ldcg(p.in_row_rs + row);
+      // folded RMSNorm, producing side: the first two blocks of this warp's rows of y are on their way before the
+      // tile's products are complete
+      const bool fold_now = fold_pair && un.last;
+      // three landing blocks per warp: two in the ring's unused last stage, the third is the warp's second staging block
+      uint8_t* xb_stage = smem + (Ring<true>::STAGES - 1) * Ring<true>::STAGE_BYTES + quarter * 2 * EPI_BUF_BYTES;
+      auto landing = [&](int i) -> uint8_t* { return i < 2 ? xb_stage + i * EPI_BUF_BYTES : epi_buf + EPI_BUF_BYTES; };
+      uint64_t* xb_bar = xbar + quarter * 4;
+      const int n_chunks = min(p.bn / 32, (p.N - n * p.bn + 31) / 32);
+      if (fold_now) {
+        if (ordered && ks > 0) {              // every earlier segment of the tile must be in y before y is read
+          int* turn = p.tile_turn + (tile * 2 + int(rank)) * 4 + quarter;
+          bool go = true;
+          if (lane == 0) go = spin_until_equal(turn, ks, abort_flag, p.status);
+          if (!__shfl_sync(0xffffffffu, go, 0)) break;
+        }
+        if (lane == 0) {
+          bulk_wait_read<0>();                // nothing of an earlier unit still reads the staging blocks
+          for (int c = 0; c < 3 && c < n_chunks; ++c) {
+            mbar_expect_tx(&xb_bar[c], EPI_BUF_BYTES);
+            tma_load_2d(landing(c), &p.tm_out, &xb_bar[c], n * p.bn + c * 32, row_base);
+          }
+        }
+      }
       const bool ok = mbar_wait(&tfull[acc], acc_ph, abort_flag, p.status);
       if (!__all_sync(0xffffffffu, ok)) break;
       tc_fence_after_sync();
       const uint32_t taddr = tmem_base + acc * BN + (uint32_t(quarter * 32) << 16);
-      const int row = m * BM + quarter * 32 + lane;
-      const bool row_ok = row < p.M;
       uint32_t r0[32], r1[32];
       float v0[32], v1[32];
 
-      const int row_base = m * BM + quarter * 32;          // first row of this warp's 32
 
       if (p.mode == kGemmResid) {
         // Ordered split-K: the partial sums of a tile are added into the output in split order, so the
         // result is the same fixed sum whatever block computed which split.  This warp owns 32 rows of the
         // tile; it waits until the previous split's add of those rows has been performed.
         int* turn = p.tile_turn + (PAIR ? tile * 2 + int(rank) : emulate_pair ? tile * 2 + un.half : tile) * 4 + quarter;
-        if (ordered && ks > 0) {
+        if (ordered && ks > 0 && !fold_now) {
           bool go = true;
           if (lane == 0) go = spin_until_equal(turn, ks, abort_flag, p.status);
           if (!__shfl_sync(0xffffffffu, go, 0)) break;
@@ -439,6 +498,130 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
           const int chunk = lane % (p.bn / 32), col = n * p.bn + chunk * 32;
           if (col < p.N) asm volatile("prefetch.global.L1 [%0];" ::"l"(gate + col));
         }
+        if (fold_now) {
+          // Final segment of the tile with the following RMSNorm folded in: x = y + acc is formed here (every
+          // earlier segment has been added into y), written back, and reused for h = 16-bit(x o g) and sum x^2.
+          // The 32 x 32 blocks of y come in by TMA, one chunk ahead, into two landing blocks per warp (the ring's
+          // unused last stage), are updated in place and leave by TMA stores; the 16-bit block of a pair of chunks
+          // is staged beside them.
+          const bool h16 = p.norm_h_f16 != 0;
+          float ss = 0.f;
+          uint8_t* buf_h = epi_buf;
+          bool okx = true;
+          for (int c = 0; c < n_chunks; ++c) {
+            const int col0 = n * p.bn + c * 32;
+            const int xi = c % 3;
+            uint8_t* bx = landing(xi);
+            if (lane == 0 && c > 0) {
+              bulk_wait_read<0>();                         // the stores of the previous chunk have read their blocks
+              if (c + 2 < n_chunks) {                      // ... so its landing block can take the chunk two further on
+                const int xn = (c + 2) % 3;
+                mbar_expect_tx(&xb_bar[xn], EPI_BUF_BYTES);
+                tma_load_2d(landing(xn), &p.tm_out, &xb_bar[xn], col0 + 64, row_base);
+              }
+            }
+            tmem_ld32(taddr + c * 32, r0);
+            uint4 gw[4];                               // 32 gains (bf16), the same for every row
+            const int nv = p.N - col0 >= 32 ? 8 : (p.N - col0) >> 2;
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              gw[e] = 2 * e < nv ? __ldg(reinterpret_cast<const uint4*>(p.norm_gain + col0) + e) : make_uint4(0, 0, 0, 0);
+            okx = mbar_wait(&xb_bar[xi], (xph >> xi) & 1, abort_flag, p.status);
+            if (!__all_sync(0xffffffffu, okx)) { okx = false; break; }
+            xph ^= 1u << xi;
+            tmem_ld_wait();
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              float4* slot = reinterpret_cast<float4*>(bx + lane * 128 + ((u ^ (lane & 7)) << 4));
+              const float4 y4 = *slot;
+              const float x0 = __uint_as_float(r0[4 * u]) + y4.x, x1 = __uint_as_float(r0[4 * u + 1]) + y4.y;
+              const float x2 = __uint_as_float(r0[4 * u + 2]) + y4.z, x3 = __uint_as_float(r0[4 * u + 3]) + y4.w;
+              if (u < nv) ss += (x0 * x0 + x1 * x1) + (x2 * x2 + x3 * x3);
+              *slot = make_float4(x0, x1, x2, x3);
+              r0[4 * u] = __float_as_uint(x0); r0[4 * u + 1] = __float_as_uint(x1);
+              r0[4 * u + 2] = __float_as_uint(x2); r0[4 * u + 3] = __float_as_uint(x3);
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const uint32_t pk[4] = {gw[e].x, gw[e].y, gw[e].z, gw[e].w};
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                v0[8 * e + 2 * q] = __uint_as_float(r0[8 * e + 2 * q]) * __uint_as_float(pk[q] << 16);
+                v0[8 * e + 2 * q + 1] = __uint_as_float(r0[8 * e + 2 * q + 1]) * __uint_as_float(pk[q] & 0xffff0000u);
+              }
+            }
+            if (h16 && row_ok) note_f16_saturation(v0, p.status);
+            stage_bf16x32(buf_h, lane, (c & 1) * 4, v0, h16);
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&p.tm_out, bx, col0, row_base);
+              if ((c & 1) || c + 1 == n_chunks) tma_store_2d(&p.tm_norm_h, buf_h, n * p.bn + (c >> 1) * 64, row_base);
+              bulk_commit();
+            }
+          }
+          if (!okx) break;
+          finish_row_norm(p, row, row_ok, m * 4 + quarter, n, n_n_tiles, ss, lane);
+          if (lane == 0) bulk_wait_read<0>();         // the staging blocks go back to the alternating use below
+          __syncwarp();
+          epi_sel = 0;
+        } else if (p.norm_gain != nullptr && un.last) {
+          // The same fold in the single-block kernel (reached by a folded step only at sm_budget 1): y is read with
+          // plain loads; the arithmetic, and so every bit of x, h and the sums, is that of the pair form.
+          const float* yrow = p.y_in + size_t(row_ok ? row : 0) * p.N;
+          const bool h16 = p.norm_h_f16 != 0;
+          float ss = 0.f;
+          uint8_t* buf_x = epi_buf;                       // fp32 block of this chunk
+          uint8_t* buf_h = epi_buf + EPI_BUF_BYTES;       // 16-bit block of a pair of chunks
+          for (int c = 0; c < p.bn / 32; ++c) {
+            const int col0 = n * p.bn + c * 32;
+            if (col0 >= p.N) break;
+            tmem_ld32(taddr + c * 32, r0);
+            const int nv = p.N - col0 >= 32 ? 8 : (p.N - col0) >> 2;        // float4s of the chunk inside the row
+            float4 yv[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+              yv[e] = row_ok && e < nv ? __ldcg(reinterpret_cast<const float4*>(yrow + col0) + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+            uint4 gw[4];                                   // 32 gains (bf16), the same for every row
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              gw[e] = 2 * e < nv ? __ldg(reinterpret_cast<const uint4*>(p.norm_gain + col0) + e) : make_uint4(0, 0, 0, 0);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const float x0 = __uint_as_float(r0[4 * e]) + yv[e].x, x1 = __uint_as_float(r0[4 * e + 1]) + yv[e].y;
+              const float x2 = __uint_as_float(r0[4 * e + 2]) + yv[e].z, x3 = __uint_as_float(r0[4 * e + 3]) + yv[e].w;
+              if (e < nv) ss += (x0 * x0 + x1 * x1) + (x2 * x2 + x3 * x3);
+              r0[4 * e] = __float_as_uint(x0); r0[4 * e + 1] = __float_as_uint(x1);
+              r0[4 * e + 2] = __float_as_uint(x2); r0[4 * e + 3] = __float_as_uint(x3);
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const uint32_t pk[4] = {gw[e].x, gw[e].y, gw[e].z, gw[e].w};
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                v0[8 * e + 2 * q] = __uint_as_float(r0[8 * e + 2 * q]) * __uint_as_float(pk[q] << 16);
+                v0[8 * e + 2 * q + 1] = __uint_as_float(r0[8 * e + 2 * q + 1]) * __uint_as_float(pk[q] & 0xffff0000u);
+              }
+            }
+            if (h16 && row_ok) note_f16_saturation(v0, p.status);
+            if (lane == 0) bulk_wait_read<0>();       // both staging blocks have been read by their last stores
+            __syncwarp();
+            stage_f32x32(buf_x, lane, r0);
+            stage_bf16x32(buf_h, lane, (c & 1) * 4, v0, h16);
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&p.tm_out, buf_x, col0, row_base);
+              if ((c & 1) || col0 + 32 >= p.N) tma_store_2d(&p.tm_norm_h, buf_h, n * p.bn + (c >> 1) * 64, row_base);
+              bulk_commit();
+            }
+          }
+          finish_row_norm(p, row, row_ok, m * 4 + quarter, n, n_n_tiles, ss, lane);
+          if (lane == 0) bulk_wait_read<0>();         // the staging blocks go back to the alternating use below
+          __syncwarp();
+          epi_sel = 0;
+        } else
         for (int c = 0; c < p.bn / 32; ++c) {
           const int col0 = n * p.bn + c * 32;
           if (col0 >= p.N) break;
@@ -486,7 +669,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
           tmem_ld_wait();
 #pragma unroll
           for (int e = 0; e < 32; ++e) {
-            const float g = __uint_as_float(r0[e]), u = __uint_as_float(r1[e]);
+            const float g = __uint_as_float(r0[e]) * rs, u = __uint_as_float(r1[e]) * rs;
             v0[e] = __fdividef(g * u, 1.f + __expf(-g));   // silu(g) * u
           }
           if (p.act_f16) note_f16_saturation(v0, p.status);
@@ -523,6 +706,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
             for (int c = 0; c < 4; ++c) {
               tmem_ld32(taddr + half * 128 + c * 32, r0);
               tmem_ld_wait();
+              if (p.in_row_rs) scale32(r0, rs);
               if (bias) add_bias32(r0, bias + vcol + c * 32);
               if (row_ok) {
 #pragma unroll
@@ -542,6 +726,10 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
               tmem_ld32(taddr + half * 128 + lo * 32, r0);
               tmem_ld32(taddr + half * 128 + hi * 32, r1);
               tmem_ld_wait();
+              if (p.in_row_rs) {
+                scale32(r0, rs);
+                scale32(r1, rs);
+              }
               if (bias) {                                        // the bias comes before the rotation
                 add_bias32(r0, bias + vcol + lo * 32);
                 add_bias32(r1, bias + vcol + hi * 32);

@@ -60,6 +60,25 @@ struct GemmParams {
   int* status;               // device status word; with act_f16 the word after it counts saturated act values
   int act_f16;               // GateUp: 1 = write act as fp16, 0 = bf16
   int* smid_log;             // nullable: SM census slots of this launch (see log_smid)
+  // RMSNorm folded into the GEMMs around it: rmsnorm(x) W^T = diag(r) ((x o g) W^T), r = rsqrt(mean(x^2) + eps).
+  //   Resid, producing side (norm_gain non-null): the tile's final segment does not add-reduce its block into the
+  //   output but reads it, adds, writes x back and, from the same registers, emits the next GEMM's A operand
+  //   h = 16-bit(x o g) (not yet normalised) and the sum of x^2 over the tile's columns, one partial per (row, tile
+  //   column), into row_ss[row * ss_stride + tile column]; the warp that delivers a row group's last tile column sums
+  //   the partials in tile-column order and writes r into row_rs[row] (row_group_done: one counter per 32 rows,
+  //   zero at entry and at exit).
+  const __nv_bfloat16* norm_gain;   // [N] gains of the norm that follows, or null
+  CUtensorMap tm_norm_h;     // h [M, N] 16-bit, box 64 x 32, 128-byte swizzle
+  float* row_ss;             // [M][ss_stride]
+  int ss_stride;
+  float* row_rs;             // [M] r of every row, for the consuming GEMM
+  int* row_group_done;       // [ceil(M / 32)]
+  const float* y_in;         // the output as plain memory (the residual stream to read)
+  int norm_h_f16;            // 1 = h in fp16, 0 = bf16
+  //   Qkv / GateUp, consuming side (in_row_rs non-null): every accumulator row is scaled by r of its token before
+  //   bias / RoPE / SiLU.
+  const float* in_row_rs;    // [M]
+  float norm_eps;            // producing side: eps of the norm that follows
 };
 cudaError_t launch_gemm(const GemmParams& p, int sm_budget, cudaStream_t stream);
 cudaError_t gemm_set_attributes();
