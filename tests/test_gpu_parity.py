@@ -552,3 +552,42 @@ def test_a_wait_that_nothing_satisfies_gives_up_with_a_timeout_status():
     torch.cuda.synchronize()
     assert st2.item() == 0
     assert torch.allclose(out, a.float() @ w.float().T, rtol=1e-3, atol=1e-2)
+
+
+# ------------------------------------------------- RMSNorm folded into the GEMMs --
+def test_folded_rmsnorm_step_matches_oracle_and_every_budget(orc):
+    """Two layers whose four projections all run on SM pairs, so that both norms of a layer are folded into the GEMMs
+    around them (the residual GEMM emits the un-normalised 16-bit operand and the row sums of squares, the next GEMM
+    scales its rows): against the oracle on sampled rows, and bit for bit across budgets down to one pair (2) and to
+    the single-block stand-in (1), which must add the same partial sums in the same order."""
+    dims = wl.StageDims(2, 1024, 16, 4, 64, 2048)
+    r = np.random.default_rng(12)
+    batch = wl.BatchSpec([1400, 1100] + [1] * 100, [0, 200] + r.integers(30, 900, size=100).tolist())
+    case = make_case(dims, batch, seed=77, kv_fill=True)
+    rows = np.unique(np.concatenate([np.array([0, 1, 127, 128, 255, 256, 1399, 1400, 2499, 2500, batch.n_tokens - 1]),
+                                     np.linspace(0, batch.n_tokens - 1, 60).astype(np.int64)]))
+    mask = np.zeros(batch.n_tokens, dtype=np.uint8)
+    mask[rows] = 1
+    y_ref = orc.step(case.cfg, case.weights, case.kv_pool.copy(), batch.q_len, batch.ctx_len, case.block_tables, case.x,
+                     last_layer_row_mask=mask)
+    st = make_stage(case)
+    try:
+        outs = {}
+        for budget in (st.sm_count, 37, 2, 1):
+            st.kv_pool.copy_(wl.bits_to_bf16_tensor(case.kv_pool, st.device))
+            outs[budget] = run_step(st, case, budget)
+        y, pool = outs[st.sm_count]
+        err = rel_err(y[rows], y_ref[rows])
+        print(f"folded RMSNorm, 2 layers, {batch.n_tokens} rows: max|err|/RMS on {len(rows)} rows = {err:.2e}")
+        assert err <= TOL
+        for budget, (y_b, pool_b) in outs.items():
+            assert np.array_equal(y_b, y), budget
+            assert np.array_equal(pool_b, pool), budget
+        # the fold leaves one RMSNorm launch per step (the first norm, which has no GEMM in front of it)
+        B.hs_stage_profile_enable(st.handle, True)
+        run_step(st, case, st.sm_count)
+        prof = B.hs_stage_profile_read(st.handle)
+        B.hs_stage_profile_enable(st.handle, False)
+        assert prof["rmsnorm"][1] == 1 and prof["gemm_out"][1] == 2 and prof["gemm_down"][1] == 2
+    finally:
+        st.close()
