@@ -2,6 +2,7 @@
 #include <math.h>
 #include <string.h>
 
+#include <algorithm>
 #include <memory>
 #include <mutex>
 #include <new>
@@ -189,6 +190,10 @@ struct hs_stage {
   CUtensorMap tm_q_attn;                   // Q tiles of the prefill attention (box 64 x tokens per item)
   int32_t* pinned[kRing] = {};
   cudaEvent_t ev[kRing] = {};
+  // The two attention kernels of a layer are independent of each other; with both kinds of work in a step they run
+  // side by side, the decode kernel on a stream of the stage's own, forked from and joined to the caller's stream
+  cudaStream_t aux_stream = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
   bool ev_pending[kRing] = {};
   int ring_pos = 0;
   // optional per-kernel timing
@@ -358,6 +363,13 @@ hs_status_t hs_stage_create(const hs_stage_config_t* cfg, const hs_layer_weights
     return fail("hs_stage_create: fp16 weight copy or tensor-map encoding failed (cuTensorMapEncodeTiled unavailable, or "
                 "a matrix whose row pitch is not a multiple of 16 bytes)");
 
+  if (cudaStreamCreateWithFlags(&s->aux_stream, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&s->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&s->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+    const cudaError_t e = cudaGetLastError();
+    hs_stage_destroy(s.release());
+    return cuda_fail("hs_stage_create: auxiliary stream or event creation", e);
+  }
   for (int i = 0; i < kRing; ++i) {
     if (cudaHostAlloc(reinterpret_cast<void**>(&s->pinned[i]), size_t(s->ml.total) * 4, cudaHostAllocDefault) !=
             cudaSuccess ||
@@ -387,6 +399,9 @@ hs_status_t hs_stage_destroy(hs_stage_t* s) {
       }
       if (s->pinned[i]) cudaFreeHost(s->pinned[i]);
     }
+    if (s->aux_stream) { cudaStreamSynchronize(s->aux_stream); cudaStreamDestroy(s->aux_stream); }
+    if (s->ev_fork) cudaEventDestroy(s->ev_fork);
+    if (s->ev_join) cudaEventDestroy(s->ev_join);
     for (const hs_stage::Timed& t : s->timed) { cudaEventDestroy(t.a); cudaEventDestroy(t.b); }
     for (cudaEvent_t e : s->event_pool) cudaEventDestroy(e);
   }
@@ -535,6 +550,23 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     return HS_ERR_CUDA;
   auto slots = [&](int cls) { return census ? census + cls * kSmidSlots : nullptr; };
 
+  // Split of the SM budget between the two attention kernels when a step has both kinds of work (0 = one after the
+  // other).  The decode kernel is bound by the K / V bytes it streams, the prefill kernel by its key blocks; with the
+  // rates measured on B200 (about 42 GB/s per SM up to 5.5 TB/s; 1.15 us per block of an item; 12 us per launch)
+  //   t_decode(b) = 12 + bytes / min(5.5e6, 42e3 b)    t_prefill(b) = 12 + 1.15 max(longest item, blocks / b)   [us]
+  // and the split is the one with the smallest larger time, taken only if that beats running them in turn by 8 %.
+  // It moves work between SMs, never between results: both kernels give the same bits at any grid size.
+  int decode_sms = 0;
+  if (plan.n_prefill_items > 0 && plan.n_decode_items > 0 && sm_budget >= 16 && !s->profile) {   // (per-kernel timing keeps them apart)
+    auto t_dec = [&](int b) { return 12.0 + double(plan.decode_kv_bytes) / std::min(5.5e6, 42e3 * b); };
+    auto t_pre = [&](int b) { return 12.0 + 1.15 * std::max(double(plan.prefill_longest), double(plan.prefill_blocks) / b); };
+    double best = 0.92 * (t_dec(sm_budget) + t_pre(sm_budget));
+    for (int b = 4; b <= sm_budget - 4; ++b) {
+      const double t = std::max(t_dec(b), t_pre(sm_budget - b));
+      if (t < best) { best = t; decode_sms = b; }
+    }
+  }
+
   for (int l = 0; l < c.n_layers && e == cudaSuccess; ++l) {
     const hs_layer_weights_t& w = s->layers[l];
     const LayerMaps& m = s->maps[l];
@@ -620,10 +652,26 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     a.group_done = meta + s->ml.group_done;
     a.status = status;
     a.smid_log = slots(2);       // prefill in class 2, decode in class 3 (the next slots)
-    if (a.n_prefill_items > 0) { LaunchTimer t(s, 2, stream); where = "prefill attention"; e = launch_attention_prefill(a, sm_budget, stream); }
-    if (e != cudaSuccess) break;
-    if (a.n_decode_items > 0) { LaunchTimer t(s, 3, stream); where = "decode attention"; e = launch_attention_decode(a, sm_budget, stream); }
-    if (e != cudaSuccess) break;
+    if (decode_sms > 0) {
+      // side by side: the decode kernel on the stage's own stream with decode_sms of the budget, the prefill kernel on
+      // the caller's stream with the rest; both are joined before the out-projection
+      AttnParams ad = a;
+      ad.overlap = 0;
+      if (cudaEventRecord(s->ev_fork, stream) != cudaSuccess || cudaStreamWaitEvent(s->aux_stream, s->ev_fork, 0) != cudaSuccess) {
+        e = cudaGetLastError(); where = "attention fork"; break;
+      }
+      { LaunchTimer t(s, 3, s->aux_stream); where = "decode attention"; e = launch_attention_decode(ad, decode_sms, s->aux_stream); }
+      if (e != cudaSuccess) break;
+      if (cudaEventRecord(s->ev_join, s->aux_stream) != cudaSuccess) { e = cudaGetLastError(); where = "attention join"; break; }
+      { LaunchTimer t(s, 2, stream); where = "prefill attention"; e = launch_attention_prefill(a, sm_budget - decode_sms, stream); }
+      if (e != cudaSuccess) break;
+      if (cudaStreamWaitEvent(stream, s->ev_join, 0) != cudaSuccess) { e = cudaGetLastError(); where = "attention join"; break; }
+    } else {
+      if (a.n_prefill_items > 0) { LaunchTimer t(s, 2, stream); where = "prefill attention"; e = launch_attention_prefill(a, sm_budget, stream); }
+      if (e != cudaSuccess) break;
+      if (a.n_decode_items > 0) { LaunchTimer t(s, 3, stream); where = "decode attention"; e = launch_attention_decode(a, sm_budget, stream); }
+      if (e != cudaSuccess) break;
+    }
 
     GemmParams go{};
     go.tm_a = a_rows == 128 ? s->tm_o : s->tm_o_s[a_sel];

@@ -393,6 +393,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
       int s = 0, acc = 0;
       uint32_t ph = 0, acc_ph = 0;
       bool ok = true;
+      const uint64_t a_desc0 = umma_desc_kmajor_sw128(smem_u32(smem));
       while (ok && walk.next(un)) {
         if (!mbar_wait(&tempty[acc], acc_ph ^ 1, abort_flag, p.status)) break;
         tc_fence_after_sync();
@@ -401,18 +402,20 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
         for (int kb = kb_begin; kb < kb_end; ++kb) {
           if (!mbar_wait(&full[s], ph, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after_sync();
-          const uint32_t a_addr = smem_u32(smem + s * STAGE_BYTES);
-          const uint64_t a_desc = umma_desc_kmajor_sw128(a_addr);
-          const uint64_t b_desc = umma_desc_kmajor_sw128(a_addr + b_off);
+          // descriptors of stage s: those of stage 0 plus the stage's offset in the address field (units of 16 bytes;
+          // shared memory is below 256 KB, so nothing carries out of the field): the issuing thread has as little as
+          // possible between two MMAs
+          const uint64_t a_desc = a_desc0 + uint64_t(s * (STAGE_BYTES >> 4));
+          const uint64_t b_desc = a_desc + uint64_t(b_off >> 4);
+          const uint32_t acc0 = kb != kb_begin ? 1u : 0u;
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {  // 16 bf16 = 32 B along K: +2 in the (address / 16) field
-            if (PAIR) umma_bf16_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, ((kb - kb_begin) | k) != 0);
-            else umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, ((kb - kb_begin) | k) != 0);
+            if (PAIR) umma_bf16_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, k != 0 ? 1u : acc0);
+            else umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, k != 0 ? 1u : acc0);
           }
           // frees the stage (in both blocks) once these MMAs have read it
           if (PAIR) {
-            umma_commit_pair(mapa_u32(smem_u32(&empty[s]), 0));
-            umma_commit_pair(mapa_u32(smem_u32(&empty[s]), 1));
+            umma_commit_pair_both(&empty[s]);
           } else {
             umma_commit(&empty[s]);
           }
@@ -420,8 +423,7 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
         }
         if (ok) {
           if (PAIR) {
-            umma_commit_pair(mapa_u32(smem_u32(&tfull[acc]), 0));
-            umma_commit_pair(mapa_u32(smem_u32(&tfull[acc]), 1));
+            umma_commit_pair_both(&tfull[acc]);
           } else {
             umma_commit(&tfull[acc]);
           }

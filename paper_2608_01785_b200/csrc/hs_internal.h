@@ -64,6 +64,10 @@ MetaLayout make_meta_layout(const hs_stage_config_t& c);
 struct StepPlan {
   int n_tokens = 0, n_seqs = 0;
   int n_prefill_items = 0, n_decode_items = 0, n_decode_rows = 0;
+  // work estimates of the two attention kernels (for the split of the SM budget when they run side by side)
+  int64_t prefill_blocks = 0;     // 64-key blocks over all prefill items (an item's two tiles share a block)
+  int prefill_longest = 0;        // blocks of the longest prefill item
+  int64_t decode_kv_bytes = 0;    // K and V bytes the decode items read, one layer
 };
 
 // Validates `b` against `c` and, when `meta` is non-NULL, fills the metadata block (layout `ml`).

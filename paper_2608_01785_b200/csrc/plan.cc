@@ -179,6 +179,7 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
           }
       }
       n_dec_items += c.n_kv_heads * splits;
+      p.decode_kv_bytes += int64_t(keys) * 2 * c.n_kv_heads * c.head_dim * 2;
       ++n_dec_rows;
     } else {
       // a prefill item covers two Q tiles of Mt tokens each (the second one may be short or absent)
@@ -186,6 +187,10 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
         for (int hk = 0; hk < c.n_kv_heads; ++hk) {
           const int nt = std::min(2 * Mt, n - t0);
           pre.push_back(Item{{s, hk, t0, nt}, ctx + t0 + nt});
+          const int keys_item = (c.flags & HS_FLAG_BIDIRECTIONAL) ? ctx + n : ctx + t0 + nt;
+          const int blocks = ceil_div(keys_item, 64);
+          p.prefill_blocks += blocks;
+          p.prefill_longest = std::max(p.prefill_longest, blocks);
         }
     }
     t += n;

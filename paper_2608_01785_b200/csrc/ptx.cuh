@@ -252,6 +252,17 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar_cluster_addr) {
                : "memory");
 }
 
+// The same arrival delivered to the barrier at the same shared-memory offset in both blocks of the pair with one
+// instruction (a commit costs its issuing thread about a hundred cycles; the MMA issuer of a pair signals two
+// blocks after every K block).  `bar` is this block's barrier; mask 3 = both blocks.  This is a signal, not a copy.
+__device__ __forceinline__ void umma_commit_pair_both(uint64_t* bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+          smem_u32(bar)),
+      "h"(static_cast<uint16_t>(3))
+      : "memory");
+}
+
 // ------------------------------------------------------- warp-level MMA ----
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t smem_addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
