@@ -37,7 +37,7 @@ SEED = {"c1_tiny": 0, "c2_shared": 1, "c3_7b": 2, "c4_talker": 3, "c3_decode": 2
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one gate/up GEMM launch per workload, each from one
 # ncu capture of that launch (the config-3 launch was captured on a 2-layer cut of the stage: a layer's launch
 # reads its own weights and the step's activations whatever the depth).  None where no capture exists.
-GATEUP_DRAM_TRAFFIC_BYTES = {"c2_shared": 69989376 + 39707904, "c3_7b": None}
+GATEUP_DRAM_TRAFFIC_BYTES = {"c2_shared": 70058496 + 39722496, "c3_7b": 287605760 + 71187200}
 # Below this length of the timed region a kernel runs at burst clocks and is held against the burst peak; a longer
 # region settles under the power cap and is held against the sustained peak.
 BURST_REGION_MS = 1000.0
@@ -362,7 +362,13 @@ class Measured:
         self.timed_steps(warmup, self.step_fn())
         sampler = ClockSampler(self.dev.index or 0)
         if sample_clocks:
+            # nvidia-smi needs a few hundred milliseconds to deliver its first sample; a short workload keeps
+            # stepping (untimed) until it has, so that the samples are taken under this workload's load
             sampler.start()
+            t_end = time.perf_counter() + 1.5
+            while not sampler.lines and time.perf_counter() < t_end:
+                self.timed_steps(max(warmup, 5), self.step_fn())
+            sampler.lines.clear()
         ms_total = self.timed_steps(steps, self.step_fn())
         clocks = sampler.stop() if sample_clocks else None
         assert self.stage.status() == 0, "device status word is set"
