@@ -208,11 +208,13 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
     }
     first_round = false;
     if (item >= p.n_decode_items || *abort_flag) break;
-    // one 32-byte record: {decode row, kv head, first key, end key} {seq, token row, group's first item, splits}
+    // one 32-byte record: {decode row, kv head, first key, end key} {seq, token row, the group's first partial slot,
+    // splits | index within the group << 16}: the queue hands the items out longest first, the partials of a group
+    // stay in key order
     const int4 it = reinterpret_cast<const int4*>(p.decode_items)[2 * item];
     const int4 dr = reinterpret_cast<const int4*>(p.decode_items)[2 * item + 1];
     const int drow = it.x, hk = it.y, k0 = it.z, k1 = it.w;
-    const int seq = dr.x, tok = dr.y, splits = dr.w;
+    const int seq = dr.x, tok = dr.y, splits = dr.w & 0xffff, part = dr.z + (dr.w >> 16);
     const int n_pages = (k1 - k0 + 15) >> 4;
     const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq + (k0 >> 4);
 
@@ -365,8 +367,8 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
       continue;
     }
     // the item's partial: unnormalised output, running max (log2 domain) and sum, rows = query heads
-    float* po = p.part_o + size_t(item) * 16 * DH;
-    float* pml = p.part_ml + size_t(item) * 16 * 2;
+    float* po = p.part_o + size_t(part) * 16 * DH;
+    float* pml = p.part_ml + size_t(part) * 16 * 2;
 #pragma unroll
     for (int j = 0; j < DH / 8; ++j) {
       const int col = 8 * j + 2 * (lane & 3);

@@ -10,9 +10,10 @@
 namespace hs {
 
 constexpr int kPage = HS_PAGE_SIZE;      // tokens per KV page
-constexpr int kDecodeSplit = 256;        // smallest number of keys per decode split-KV work item (sizes the buffers)
+constexpr int kDecodeSplit = 256;        // run length that sizes the decode item buffers (the planner may pick 128 when the items still fit)
 constexpr int kDecodeWarps = 6;            // warps per block of the decode attention kernel (kernels.h: kDecodeKernelWarps)
 constexpr int kDecodeSplitMax = 512;     // largest number of keys per item the planner may choose
+constexpr int kDecodeTail = 128;         // keys per piece of a sequence's last, incomplete run (the items that end the kernel)
 static_assert(kDecodeSplit % 16 == 0 && kDecodeSplitMax / 16 <= 32, "the decode kernel keeps one page id per lane");
 constexpr int kPrefillRows = 128;        // (token, query head of one KV head) rows per prefill work item
 
@@ -52,7 +53,8 @@ struct MetaLayout {
   int block_tables;                  // [max_seqs * max_pages_per_seq]
   int prefill_items;                 // [max_prefill_items * 4]  {seq, kv_head, first token, tokens (at most two tiles)}
   int decode_items;                  // [max_decode_items * 8]   {decode row, kv_head, first key, end key,
-                                     //                           seq, token row, first item of the group, splits}
+                                     //                           seq, token row, first partial slot of the group,
+                                     //                           splits | index within the group << 16}
   int decode_rows;                   // [max_seqs * 4]           {seq, token row, first item, splits}
   int counters;                      // [n_layers * 2]           work-queue heads, zero at step start
   int group_done;                    // [max_seqs * n_kv_heads]  finished decode splits per group, zero
@@ -74,9 +76,10 @@ struct StepPlan {
 // `page_stamp` is scratch of num_pages entries used to detect a page named by two sequences; `stamp`
 // must be a value not used by an earlier call.  tok_seq (nullable) receives the owning sequence of each
 // token.  Returns HS_OK, HS_ERR_INVALID_ARG or HS_ERR_BAD_BLOCK_TABLE.
-// Keys per decode work item for this batch: 256, 384 or 512, whichever lets the device's warps finish the items in
-// the fewest, shortest rounds.  A function of the batch and of the device's SM count only (never of the budget).
-int pick_decode_split(const hs_stage_config_t& c, const hs_batch_t& b, int sm_count);
+// Keys per decode work item for this batch: 128, 256, 384 or 512, whichever lets the device's warps finish the items
+// in the fewest, shortest rounds (among the sizes whose item count fits max_items).  A function of the batch and of
+// the device's SM count only (never of the budget).
+int pick_decode_split(const hs_stage_config_t& c, const hs_batch_t& b, int sm_count, int max_items);
 hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs_batch_t& b, int sm_count,
                       std::vector<int32_t>& page_stamp, int32_t stamp, int32_t* meta, int32_t* tok_seq,
                       StepPlan* plan);

@@ -156,7 +156,7 @@ extern "C" hs_status_t hs_op_decode_attention_noalloc(const void* q_dev, const v
         int32_t* it = meta + kOffItems + (n_items + hk * splits + j) * 8;
         it[0] = s; it[1] = hk; it[2] = j * kDecodeSplit;
         it[3] = keys < (j + 1) * kDecodeSplit ? keys : (j + 1) * kDecodeSplit;
-        it[4] = s; it[5] = s; it[6] = n_items + hk * splits; it[7] = splits;   // one query row per sequence
+        it[4] = s; it[5] = s; it[6] = n_items + hk * splits; it[7] = splits | (j << 16);   // one query row per sequence
       }
     n_items += n_kv_heads * splits;
   }

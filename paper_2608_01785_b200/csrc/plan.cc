@@ -61,9 +61,10 @@ MetaLayout make_meta_layout(const hs_stage_config_t& c) {
   MetaLayout m{};
   const int G = c.n_q_heads / c.n_kv_heads;
   m.max_prefill_items = c.n_kv_heads * (c.max_tokens / prefill_tokens_per_item(G) + c.max_seqs);
-  // every decode sequence has one ragged split plus one per kDecodeSplit cached keys; cached keys are
-  // bounded by the pool
-  m.max_decode_items = c.n_kv_heads * (c.max_seqs + int((int64_t(c.num_pages) * kPage) / kDecodeSplit) + 1);
+  // a decode sequence of n keys has at most n / kDecodeSplit whole runs and kDecodeSplitMax / kDecodeTail pieces of a
+  // last, incomplete one; cached keys are bounded by the pool
+  m.max_decode_items = c.n_kv_heads * (c.max_seqs * (kDecodeSplitMax / kDecodeTail) +
+                                       int((int64_t(c.num_pages) * kPage) / kDecodeSplit) + 1);
   int off = 0;
   auto take = [&](int n) {
     int o = off;
@@ -86,23 +87,36 @@ MetaLayout make_meta_layout(const hs_stage_config_t& c) {
   return m;
 }
 
-int pick_decode_split(const hs_stage_config_t& c, const hs_batch_t& b, int sm_count) {
-  // Every warp of the decode kernel works through whole items, so the kernel lasts about
-  //   rounds x (pages per item + 8),   rounds = ceil(items / (0.97 x warps of the device)),
-  // in units of the time a warp needs for one page: the items are handed out in rounds (a short last round leaves
-  // most warps idle for a whole item), and an item costs about 8 page times on top of its pages (queue, record,
-  // page ids, first bytes, partial result, its share of the merge).  Measured on B200, 64 sequences of 512..4096
-  // keys, 4 KV heads: 256 keys 72 us, 384 keys 68 us, 512 keys 76 us per launch; 32 sequences: 49 / 39 / 44 us.
-  const int warps = (sm_count > 0 ? sm_count : 148) * kDecodeWarps;
+int decode_items_of(int keys, int split) { return keys / split + ceil_div(keys % split, kDecodeTail); }
+
+int pick_decode_split(const hs_stage_config_t& c, const hs_batch_t& b, int sm_count, int max_items) {
+  // Every warp of the decode kernel works through whole items, longest first.  In units of the time a warp needs for
+  // one page an item costs its pages + 8 (queue, record, page ids, first bytes, partial result, its share of the
+  // merge), the whole runs are handed out in rounds -- a short last round leaves most warps idle for a whole item --
+  // and the pieces of the incomplete runs fill what the last round leaves free, or add rounds of their own:
+  //   cost = rounds x (pages per run + 8) + further rounds of pieces x (pages per piece + 8),
+  //   rounds = ceil(whole runs / (0.97 x warps of the device)).
+  // Measured on B200, 64 sequences of 512..4096 keys, 4 KV heads (model in brackets): 256 keys 72.6 us (72), 384 keys
+  // 67.1 (64), 512 keys 77.8 (80); 16 sequences of 300..800 keys: 128 keys 17 us, 256 keys 21 us.
+  const int64_t W = int64_t((sm_count > 0 ? sm_count : 148) * kDecodeWarps) * 97 / 100;
+  const int piece_cost = kDecodeTail / kPage + 8;
   int best = kDecodeSplit;
   double best_cost = 1e30;
-  for (int split = kDecodeSplit; split <= kDecodeSplitMax; split += 128) {
-    int64_t items = 0;
+  for (int split = kDecodeTail; split <= kDecodeSplitMax; split += 128) {
+    int64_t whole = 0, pieces = 0;
     for (int s = 0; s < b.n_seqs; ++s)
-      if (b.q_len[s] == 1) items += int64_t(c.n_kv_heads) * ceil_div(b.ctx_len[s] + 1, split);
-    if (items == 0) return kDecodeSplit;
-    const double rounds = double((items * 100 + int64_t(warps) * 97 - 1) / (int64_t(warps) * 97));
-    const double cost = rounds * (split / kPage + 8);
+      if (b.q_len[s] == 1) {
+        const int keys = b.ctx_len[s] + 1;
+        whole += int64_t(c.n_kv_heads) * (keys / split);
+        pieces += int64_t(c.n_kv_heads) * ceil_div(keys % split, kDecodeTail);
+      }
+    if (whole + pieces == 0) return kDecodeSplit;
+    if (whole + pieces > max_items) continue;          // (only the smallest size can exceed the buffers)
+    const int run_cost = split / kPage + 8;
+    const int64_t rounds = (whole + W - 1) / W;
+    const int64_t absorbed = (rounds * W - whole) * (run_cost / piece_cost);
+    const int64_t left = pieces > absorbed ? pieces - absorbed : 0;
+    const double cost = double(rounds * run_cost + (left + W - 1) / W * piece_cost);
     if (cost < best_cost - 1e-9) {
       best_cost = cost;
       best = split;
@@ -138,13 +152,15 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
 
   const int G = c.n_q_heads / c.n_kv_heads;
   const int Mt = prefill_tokens_per_item(G);
-  const int split = pick_decode_split(c, b, sm_count);
+  const int split = pick_decode_split(c, b, sm_count, ml.max_decode_items);
   StepPlan p;
   p.n_tokens = b.n_tokens;
   p.n_seqs = b.n_seqs;
 
   struct Item { int32_t v[4]; int32_t cost; };
   std::vector<Item> pre;
+  struct DecItem { int32_t v[8]; int32_t keys; };
+  std::vector<DecItem> dec;
   int n_dec_items = 0, n_dec_rows = 0;
   int t = 0;
   for (int s = 0; s < b.n_seqs; ++s) {
@@ -166,18 +182,23 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
       if (tok_seq) tok_seq[t + j] = s;
     }
     if (n == 1) {
-      // decode: keys 0..ctx split into fixed runs of `split` keys
-      const int keys = ctx + 1, splits = ceil_div(keys, split);
+      // decode: keys 0..ctx cut into whole runs of `split` keys and the rest into pieces of kDecodeTail keys; the items
+      // of a (sequence, KV head) group keep consecutive partial-result slots in key order, whatever the order the
+      // queue hands them out in
+      const int keys = ctx + 1, small = kDecodeTail;
+      const int n_big = keys / split;
+      const int splits = decode_items_of(keys, split);
+      if (splits > 0x7fff) return HS_ERR_INVALID_ARG;      // the item record keeps the index within the group in 15 bits
       if (meta) {
         int32_t* row = meta + ml.decode_rows + n_dec_rows * 4;
         row[0] = s; row[1] = t; row[2] = n_dec_items; row[3] = splits;
-        for (int hk = 0; hk < c.n_kv_heads; ++hk)
-          for (int j = 0; j < splits; ++j) {
-            int32_t* it = meta + ml.decode_items + (n_dec_items + hk * splits + j) * 8;
-            it[0] = n_dec_rows; it[1] = hk; it[2] = j * split; it[3] = std::min(keys, (j + 1) * split);
-            it[4] = s; it[5] = t; it[6] = n_dec_items + hk * splits; it[7] = splits;
-          }
       }
+      for (int hk = 0; hk < c.n_kv_heads; ++hk)
+        for (int j = 0; j < splits; ++j) {
+          const int k0 = j < n_big ? j * split : n_big * split + (j - n_big) * small;
+          const int k1 = j < n_big ? k0 + split : std::min(keys, k0 + small);
+          dec.push_back(DecItem{{n_dec_rows, hk, k0, k1, s, t, n_dec_items + hk * splits, splits | (j << 16)}, k1 - k0});
+        }
       n_dec_items += c.n_kv_heads * splits;
       p.decode_kv_bytes += int64_t(keys) * 2 * c.n_kv_heads * c.head_dim * 2;
       ++n_dec_rows;
@@ -198,7 +219,11 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
   if (int(pre.size()) > ml.max_prefill_items || n_dec_items > ml.max_decode_items) return HS_ERR_INVALID_ARG;
   // longest first, so that the dynamic queue finishes evenly; ties keep batch order
   std::stable_sort(pre.begin(), pre.end(), [](const Item& a, const Item& b2) { return a.cost > b2.cost; });
+  // decode items likewise: the long runs first, the short ones fill the end of the kernel
+  std::stable_sort(dec.begin(), dec.end(), [](const DecItem& a, const DecItem& b2) { return a.keys > b2.keys; });
   if (meta) {
+    for (size_t i = 0; i < dec.size(); ++i)
+      for (int k = 0; k < 8; ++k) meta[ml.decode_items + int(i) * 8 + k] = dec[i].v[k];
     for (size_t i = 0; i < pre.size(); ++i)
       for (int k = 0; k < 4; ++k) meta[ml.prefill_items + int(i) * 4 + k] = pre[i].v[k];
     for (int i = 0; i < c.n_layers * 2; ++i) meta[ml.counters + i] = 0;
