@@ -190,48 +190,73 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
     tma_prefetch_desc(&p.tm_kv);
   }
   __syncthreads();
-  griddep_wait();
-  griddep_launch_dependents();
 
   uint8_t* slots = smem + warp * DC_STAGES * SLOT_BYTES;
   uint64_t* full = full_all + warp * DC_STAGES;
   uint32_t issued = 0, consumed = 0;      // pages this warp has requested / finished, over all its items
+  auto issue = [&](int page, int hk) {      // lane 0: request one page of an item
+    const uint32_t st = issued % DC_STAGES;
+    mbar_expect_tx(&full[st], SLOT_BYTES);
+    load_page<DH>(p, slots + st * SLOT_BYTES, &full[st], 0, page, hk);
+    load_page<DH>(p, slots + st * SLOT_BYTES + G_::PAGE_BYTES, &full[st], 1, page, hk);
+    ++issued;
+  };
 
-  // a warp's first item is its own index in the grid (no round trip to the queue head before the first
-  // page request); the queue hands out the items after those
+  // A warp's first item is its own index in the grid (no round trip to the queue head before the first page request);
+  // the queue hands out the items after those.  The first item's record, its page ids and those of its first pages
+  // that lie wholly inside the cached context are fetched before the wait for the previous kernel: the step's
+  // metadata was copied before any kernel of the step started, and this step writes K / V at positions >= ctx only.
+  int item = blockIdx.x * DC_WARPS + warp;
+  int4 it = make_int4(0, 0, 0, 0), dr = it;
+  int my_page = 0, ahead = 0;             // ahead: pages of the current item already requested
+  if (item < p.n_decode_items) {
+    it = reinterpret_cast<const int4*>(p.decode_items)[2 * item];
+    dr = reinterpret_cast<const int4*>(p.decode_items)[2 * item + 1];
+    const int n_pages = (it.w - it.z + 15) >> 4;
+    my_page = lane < n_pages ? p.block_tables[size_t(dr.x) * p.max_pages_per_seq + (it.z >> 4) + lane] : 0;
+    const int ctx = p.seq_ctx[dr.x];
+#pragma unroll
+    for (int pi = 0; pi < DC_STAGES - 1; ++pi) {
+      const int page = __shfl_sync(0xffffffffu, my_page, pi);
+      const bool stable = pi < n_pages && it.z + (pi + 1) * 16 <= ctx && ahead == pi;
+      if (stable) {
+        if (lane == 0) issue(page, it.y);
+        ++ahead;
+      }
+    }
+  }
+  griddep_wait();
+  griddep_launch_dependents();
+
   bool first_round = true;
   for (;;) {
-    int item = blockIdx.x * DC_WARPS + warp;
     if (!first_round) {
       if (lane == 0) item = int(gridDim.x) * DC_WARPS + atomicAdd(p.counters + 1, 1);
       item = __shfl_sync(0xffffffffu, item, 0);
     }
-    first_round = false;
     if (item >= p.n_decode_items || *abort_flag) break;
     // one 32-byte record: {decode row, kv head, first key, end key} {seq, token row, the group's first partial slot,
     // splits | index within the group << 16}: the queue hands the items out longest first, the partials of a group
     // stay in key order
-    const int4 it = reinterpret_cast<const int4*>(p.decode_items)[2 * item];
-    const int4 dr = reinterpret_cast<const int4*>(p.decode_items)[2 * item + 1];
+    if (!first_round) {
+      it = reinterpret_cast<const int4*>(p.decode_items)[2 * item];
+      dr = reinterpret_cast<const int4*>(p.decode_items)[2 * item + 1];
+      ahead = 0;
+    }
     const int drow = it.x, hk = it.y, k0 = it.z, k1 = it.w;
     const int seq = dr.x, tok = dr.y, splits = dr.w & 0xffff, part = dr.z + (dr.w >> 16);
     const int n_pages = (k1 - k0 + 15) >> 4;
-    const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq + (k0 >> 4);
-
     // the item's page ids, one per lane, fetched with a single load: reading the block table page by page
     // would put one dependent round trip to memory in front of every request
-    const int my_page = lane < n_pages ? table[lane] : 0;      // the planner keeps items within 32 pages
-    auto issue = [&](int page) {            // lane 0: request one page of this item
-      const uint32_t st = issued % DC_STAGES;
-      mbar_expect_tx(&full[st], SLOT_BYTES);
-      load_page<DH>(p, slots + st * SLOT_BYTES, &full[st], 0, page, hk);
-      load_page<DH>(p, slots + st * SLOT_BYTES + G_::PAGE_BYTES, &full[st], 1, page, hk);
-      ++issued;
-    };
+    if (!first_round) {
+      const int32_t* table = p.block_tables + size_t(seq) * p.max_pages_per_seq + (k0 >> 4);
+      my_page = lane < n_pages ? table[lane] : 0;      // the planner keeps items within 32 pages
+    }
+    first_round = false;
 #pragma unroll
     for (int pi = 0; pi < DC_STAGES - 1; ++pi) {
       const int page = __shfl_sync(0xffffffffu, my_page, pi);
-      if (lane == 0 && pi < n_pages) issue(page);
+      if (lane == 0 && pi >= ahead && pi < n_pages) issue(page, hk);
     }
 
     // Q fragments straight from global memory: rows = query heads hk*G .. hk*G + G - 1 of the new token
@@ -255,7 +280,7 @@ __global__ void __launch_bounds__(DC_THREADS, 1) attn_decode_kernel(const __grid
     for (int pi = 0; pi < n_pages; ++pi) {
       // the slot read in the previous iteration is free: keep DC_STAGES - 1 pages in flight
       const int page_ahead = __shfl_sync(0xffffffffu, my_page, (pi + DC_STAGES - 1) & 31);
-      if (lane == 0 && pi + DC_STAGES - 1 < n_pages) issue(page_ahead);
+      if (lane == 0 && pi + DC_STAGES - 1 < n_pages) issue(page_ahead, hk);
       const uint32_t st = consumed % DC_STAGES;
       ok = mbar_wait(&full[st], (consumed / DC_STAGES) & 1, abort_flag, p.status);
       if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }

@@ -345,6 +345,41 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
   if (PAIR) cluster_sync_all();               // the other block's barriers exist before anything targets them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // A small step's A box holds only the rows that exist (32 or 64 instead of 128): the MMA still reads 128
+  // rows starting at the stage's base -- beyond the A box that is the B data of the stage, finite values
+  // that only reach accumulator rows no epilogue stores
+  const bool two_halves = b_two;
+  // One stage's requests of the producer thread: the weight boxes (which also arm the barrier) and the A box.  In a
+  // pair both blocks' bytes are counted on the leader's barrier, which the leader arms for both.
+  auto load_b = [&](int s, int kb, const BSource& b0, const BSource& b1) {
+    uint8_t* st = smem + s * STAGE_BYTES;
+    if (PAIR) {
+      if (rank == 0) mbar_expect_tx(&full[s], 2 * STAGE_BYTES);
+      tma_load_2d_pair(st + b_off, &p.tm_b[b0.map], mapa_u32(smem_u32(&full[s]), 0), kb * BK, b0.row);
+    } else {
+      mbar_expect_tx(&full[s], a_bytes + (two_halves ? 2 * BH_BYTES : BH_BYTES));
+      tma_load_2d(st + b_off, &p.tm_b[b0.map], &full[s], kb * BK, b0.row);
+      if (two_halves) tma_load_2d(st + b_off + BH_BYTES, &p.tm_b[b1.map], &full[s], kb * BK, b1.row);
+    }
+  };
+  auto load_a = [&](int s, int kb, int m, int half) {
+    uint8_t* st = smem + s * STAGE_BYTES;
+    if (PAIR) tma_load_2d_pair(st, &p.tm_a, mapa_u32(smem_u32(&full[s]), 0), kb * BK, (2 * m + int(rank)) * BM);
+    else tma_load_2d(st, &p.tm_a, &full[s], kb * BK, (emulate_pair ? 2 * m + half : m) * BM);
+  };
+  // The weights never change: the producer asks for the weight boxes of its first unit's first stages before the wait
+  // for the previous kernel, and for the A boxes of those stages after it.
+  bool have_unit = false;
+  int b_ahead = 0;
+  if (warp == 0 && lane == 0) {
+    have_unit = walk.next(un);
+    if (have_unit) {
+      const int n = un.tile / n_m_tiles;
+      const BSource b0 = b_source(p, n, PAIR ? int(rank) : 0), b1 = b_source(p, n, 1);
+      b_ahead = un.kb_end - un.kb_begin < STAGES ? un.kb_end - un.kb_begin : STAGES;
+      for (int i = 0; i < b_ahead; ++i) load_b(i, un.kb_begin + i, b0, b1);
+    }
+  }
   griddep_wait();                 // everything above is set-up; the operands belong to the previous kernel until here
   griddep_launch_dependents();
 
@@ -354,32 +389,19 @@ __device__ __forceinline__ void gemm_body(const GemmParams& p) {
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      // A small step's A box holds only the rows that exist (32 or 64 instead of 128): the MMA still reads 128
-      // rows starting at the stage's base -- beyond the A box that is the B data of the stage, finite values
-      // that only reach accumulator rows no epilogue stores
-      const bool two_halves = b_two;
-      while (ok && walk.next(un)) {
+      while (ok && have_unit) {
         const int tile = un.tile;
         const int m = tile % n_m_tiles, n = tile / n_m_tiles;
         const BSource b0 = b_source(p, n, PAIR ? int(rank) : 0), b1 = b_source(p, n, 1);
         const int kb_end = un.kb_end;
         for (int kb = un.kb_begin; kb < kb_end; ++kb) {
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-          uint8_t* st = smem + s * STAGE_BYTES;
-          if (PAIR) {
-            // both blocks' bytes are counted on the leader's barrier, which the leader arms for both
-            const uint32_t bar = mapa_u32(smem_u32(&full[s]), 0);
-            if (rank == 0) mbar_expect_tx(&full[s], 2 * STAGE_BYTES);
-            tma_load_2d_pair(st, &p.tm_a, bar, kb * BK, (2 * m + int(rank)) * BM);
-            tma_load_2d_pair(st + b_off, &p.tm_b[b0.map], bar, kb * BK, b0.row);
-          } else {
-            mbar_expect_tx(&full[s], a_bytes + (two_halves ? 2 * BH_BYTES : BH_BYTES));
-            tma_load_2d(st, &p.tm_a, &full[s], kb * BK, (emulate_pair ? 2 * m + un.half : m) * BM);
-            tma_load_2d(st + b_off, &p.tm_b[b0.map], &full[s], kb * BK, b0.row);
-            if (two_halves) tma_load_2d(st + b_off + BH_BYTES, &p.tm_b[b1.map], &full[s], kb * BK, b1.row);
-          }
+          if (b_ahead > 0) --b_ahead;
+          else load_b(s, kb, b0, b1);
+          load_a(s, kb, m, un.half);
           if (++s == STAGES) { s = 0; ph ^= 1; }
         }
+        have_unit = walk.next(un);
       }
     }
   } else if (warp == 1) {
