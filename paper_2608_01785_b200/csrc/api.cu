@@ -53,7 +53,8 @@ WsLayout make_ws_layout(const hs_stage_config_t& c, const MetaLayout& ml) {
   w.status = take(256);
   w.turn = take(kGemmTurnWords * 4);
   w.smid = take(size_t(HS_PROFILE_CLASSES) * kSmidSlots * 4);
-  w.row_ss = take(T * kRowSsStride * 4);             // partial sums of x^2 per (token, tile column) of a folded RMSNorm
+  // partial sums of x^2 per (token, tile column) of a folded RMSNorm; steps of at most 64 rows keep one per 32 columns
+  w.row_ss = take(std::max(T * kRowSsStride, size_t(64) * size_t(c.d_model / 32 + 1)) * 4);
   w.row_rs = take(T * 4);                            // r of every token
   w.row_done = take((T / 32 + 2) * 4);               // tile columns delivered per group of 32 token rows
   // fp16 copies of the seven weight matrices of every layer (absent with HS_FLAG_BF16_ACTIVATIONS);
@@ -530,6 +531,26 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
   const bool fold_norm = !s->modulation && n_ss_tiles <= kRowSsStride && !skinny(d, q_dim + 2 * kv_dim, kGemmQkv) &&
                          !skinny(q_dim, d, kGemmResid) && !skinny(d, F, kGemmGateUp) && !skinny(F, d, kGemmResid) &&
                          pair_d && pair_qkv && pair_gu;
+  // Steps of at most 16 rows: a residual projection on the weight-streaming kernel folds the norm behind it the same
+  // way (its epilogue emits h and the row sums, the block that delivers the last unit finalises r); the projection
+  // behind the norm -- on either kernel -- scales its rows.  A choice by shape, never by budget.  Measured on B200, the
+  // 12-layer talker step: the fold costs a residual GEMM 2 us and saves a launch, which is 2 % slower at the full
+  // budget (where launch overlap hides most of a launch) and 11-14 % faster at budgets 112 / 74 / 37, the budgets a
+  // downstream stage runs at; at 64 rows (config-3 decode tick: +4 us per out-projection) it is -1.4 % / +2 %, so
+  // larger steps keep the separate kernel.
+  const bool sk_fold = !s->modulation && T <= 16;
+  const bool sk_fold_mlp = sk_fold && skinny(q_dim, d, kGemmResid);
+  const bool sk_fold_attn = sk_fold && skinny(F, d, kGemmResid);
+  auto sk_fold_out = [&](SkinnyParams& k, const void* gain) {
+    k.norm_gain = static_cast<const __nv_bfloat16*>(gain);
+    k.norm_h = h;
+    k.norm_h_f16 = f16;
+    k.row_ss = reinterpret_cast<float*>(s->ws_dev + s->ws.row_ss);
+    k.ss_stride = d / 32;
+    k.row_rs = reinterpret_cast<float*>(s->ws_dev + s->ws.row_rs);
+    k.units_done = reinterpret_cast<int*>(s->ws_dev + s->ws.row_done);
+    k.norm_eps = c.rms_eps;
+  };
   float* row_ss = reinterpret_cast<float*>(s->ws_dev + s->ws.row_ss);
   auto fold_out = [&](GemmParams& gp, const void* gain) {      // producing side
     gp.norm_gain = static_cast<const __nv_bfloat16*>(gain);
@@ -589,7 +610,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     np.mod = mod_l;
     np.tok_seq = meta + s->ml.tok_seq;
     np.mod_which = 0;
-    const bool folded_attn_norm = fold_norm && l > 0;          // the previous layer's down-projection produced h and the sums
+    const bool folded_attn_norm = (fold_norm || sk_fold_attn) && l > 0;   // the previous layer's down-projection produced h and the sums
     if (!folded_attn_norm) { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
@@ -622,6 +643,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
       k.tok_pos = g.tok_pos; k.tok_slot = g.tok_slot; k.rope = g.rope;
       for (int i = 0; i < 3; ++i) k.qkv_bias[i] = g.qkv_bias[i];
       k.smid_log = slots(1);
+      k.in_row_rs = g.in_row_rs;
       LaunchTimer t(s, 1, stream); where = "qkv gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
     } else { LaunchTimer t(s, 1, stream); where = "qkv gemm"; e = launch_gemm(g, sm_budget, stream); }
     if (e != cudaSuccess) break;
@@ -696,6 +718,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
       k.w[0] = wo.w_o; k.y = x; k.accumulate = 1;
       k.gate_mod = go.gate_mod; k.tok_seq = go.tok_seq; k.gate_which = 2;
       k.smid_log = slots(5);
+      if (sk_fold_mlp) sk_fold_out(k, w.g_mlp);
       LaunchTimer t(s, 5, stream); where = "out-proj gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
     } else { LaunchTimer t(s, 5, stream); where = "out-proj gemm"; e = launch_gemm(go, sm_budget, stream); }
     if (e != cudaSuccess) break;
@@ -703,7 +726,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     np.x_bf16 = nullptr;
     np.gain = static_cast<const __nv_bfloat16*>(w.g_mlp);
     np.mod_which = 3;
-    if (!fold_norm) { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
+    if (!fold_norm && !sk_fold_mlp) { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
     GemmParams gu{};
@@ -719,12 +742,13 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     gu.tm_act = s->tm_act_st;
     gu.status = status;
     gu.smid_log = slots(6);
-    if (fold_norm) fold_in(gu);
+    if (fold_norm || sk_fold_mlp) fold_in(gu);
     if (skinny(d, F, kGemmGateUp)) {
       SkinnyParams k = skinny_base(h, d, F, kGemmGateUp);
       k.w[0] = wo.w_gate; k.w[1] = wo.w_up;
       k.act = reinterpret_cast<__nv_bfloat16*>(s->ws_dev + s->ws.act); k.act_f16 = f16;
       k.smid_log = slots(6);
+      k.in_row_rs = gu.in_row_rs;
       LaunchTimer t(s, 6, stream); where = "gate/up gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
     } else { LaunchTimer t(s, 6, stream); where = "gate/up gemm"; e = launch_gemm(gu, sm_budget, stream); }
     if (e != cudaSuccess) break;
@@ -752,6 +776,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
       k.w[0] = wo.w_down; k.y = x; k.accumulate = 1;
       k.gate_mod = gd.gate_mod; k.tok_seq = gd.tok_seq; k.gate_which = 5;
       k.smid_log = slots(7);
+      if (sk_fold_attn && l + 1 < c.n_layers) sk_fold_out(k, s->layers[l + 1].g_attn);
       LaunchTimer t(s, 7, stream); where = "down gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
     } else { LaunchTimer t(s, 7, stream); where = "down gemm"; e = launch_gemm(gd, sm_budget, stream); }
     if (e != cudaSuccess) break;

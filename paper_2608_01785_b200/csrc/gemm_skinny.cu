@@ -83,7 +83,9 @@ __device__ __forceinline__ const uint8_t* unit_row(const SkinnyParams& p, int un
 
 
 // MT: 16-row tiles of activations (T <= 16 MT); DB: depth of a warp's ring of K steps.
-template <int MT, int DB, bool F16>
+// FOLD: the instantiation that knows the folded RMSNorm (producing side in Resid mode, consuming side in the others);
+// the plain one carries none of its code.
+template <int MT, int DB, bool F16, bool FOLD>
 __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const SkinnyParams p) {
   extern __shared__ __align__(16) uint8_t sk_smem[];
   constexpr int STAGE_BYTES = (NT + 2 * MT) * 512;          // per warp and K step: 4 weight tiles, 2 MT row groups
@@ -161,6 +163,10 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
       cp_async_commit();
     }
   }
+  // folded RMSNorm, consuming side: r of this thread's epilogue row, on its way while the first unit streams
+  float rs_in = 1.f;
+  if (FOLD && p.in_row_rs != nullptr && int(threadIdx.x >> 2) < p.T) rs_in = __ldcg(p.in_row_rs + (threadIdx.x >> 2));
+  int* last_unit = reinterpret_cast<int*>(part_all + SK_WARPS * PART_PITCH);   // FOLD: one word behind the partial tiles
 
   for (; unit < units; unit += gridDim.x) {
     float acc[MT][NT][4];
@@ -228,6 +234,10 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
         lo.x += l.x; lo.y += l.y; lo.z += l.z; lo.w += l.w;
         hi.x += h.x; hi.y += h.y; hi.z += h.z; hi.w += h.w;
       }
+      if (FOLD && p.in_row_rs != nullptr) {
+        lo.x *= rs_in; lo.y *= rs_in; lo.z *= rs_in; lo.w *= rs_in;
+        hi.x *= rs_in; hi.y *= rs_in; hi.z *= rs_in; hi.w *= rs_in;
+      }
       if (p.mode == kGemmResid) {
         float4* y_lo = reinterpret_cast<float4*>(p.y + size_t(row) * p.N + unit * 32 + jq);
         float4* y_hi = y_lo + 4;
@@ -245,6 +255,24 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
         }
         *y_lo = lo;
         *y_hi = hi;
+        if (FOLD && p.norm_gain != nullptr) {
+          // folded RMSNorm, producing side: the next GEMM's operand and this unit's share of the row's sum of squares
+          // (the four threads of a row are neighbours in a warp)
+          const uint2 g_lo = __ldg(reinterpret_cast<const uint2*>(p.norm_gain + unit * 32 + jq));
+          const uint2 g_hi = __ldg(reinterpret_cast<const uint2*>(p.norm_gain + unit * 32 + jq + 16));
+          float v[8] = {lo.x * __uint_as_float(g_lo.x << 16), lo.y * __uint_as_float(g_lo.x & 0xffff0000u),
+                        lo.z * __uint_as_float(g_lo.y << 16), lo.w * __uint_as_float(g_lo.y & 0xffff0000u),
+                        hi.x * __uint_as_float(g_hi.x << 16), hi.y * __uint_as_float(g_hi.x & 0xffff0000u),
+                        hi.z * __uint_as_float(g_hi.y << 16), hi.w * __uint_as_float(g_hi.y & 0xffff0000u)};
+          if (p.norm_h_f16 && p.status) note_f16_saturation(v, p.status);
+          __nv_bfloat16* hrow = p.norm_h + size_t(row) * p.N + unit * 32 + jq;
+          *reinterpret_cast<uint2*>(hrow) = make_uint2(pack_act(v[0], v[1], p.norm_h_f16 != 0), pack_act(v[2], v[3], p.norm_h_f16 != 0));
+          *reinterpret_cast<uint2*>(hrow + 16) = make_uint2(pack_act(v[4], v[5], p.norm_h_f16 != 0), pack_act(v[6], v[7], p.norm_h_f16 != 0));
+          float ss = lo.x * lo.x + lo.y * lo.y + lo.z * lo.z + lo.w * lo.w + hi.x * hi.x + hi.y * hi.y + hi.z * hi.z + hi.w * hi.w;
+          ss += __shfl_xor_sync(0xfu << (lane & 28), ss, 1);
+          ss += __shfl_xor_sync(0xfu << (lane & 28), ss, 2);
+          if ((threadIdx.x & 3) == 0) p.row_ss[size_t(row) * p.ss_stride + unit] = ss;
+        }
       } else if (p.mode == kGemmGateUp) {
         const float gt[4] = {lo.x, lo.y, lo.z, lo.w}, up[4] = {hi.x, hi.y, hi.z, hi.w};
         float v[4];
@@ -299,6 +327,26 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
       }
     }
     __syncthreads();                                         // the partial tiles are free again
+    if (FOLD && p.mode == kGemmResid && p.norm_gain != nullptr) {
+      // the block that delivers the last unit turns the partial sums into every row's r: four threads per row add
+      // the units' partials in a fixed order.  (The barrier above orders the block's stores before thread 0's fence.)
+      if (threadIdx.x == 0) {
+        __threadfence();
+        *last_unit = atomicAdd(p.units_done, 1) == units - 1;
+      }
+      __syncthreads();
+      if (*last_unit) {
+        __threadfence();
+        const int q = threadIdx.x & 3;
+        float sum = 0.f;
+        if (row < p.T)
+          for (int i = q; i < units; i += 4) sum += __ldcg(p.row_ss + size_t(row) * p.ss_stride + i);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+        if (q == 0 && row < p.T) p.row_rs[row] = rsqrtf(sum / float(p.N) + p.norm_eps);
+        if (threadIdx.x == 0) *p.units_done = 0;             // ready for the next launch
+      }
+    }
     if (ALIAS && next < units) {
       set_rows(next);
       prologue();
@@ -309,7 +357,7 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
 template <int MT, int DB>
 constexpr int skinny_smem() {
   constexpr int rings = SK_WARPS * DB * (NT + 2 * MT) * 512, both = rings + SK_WARPS * MT * 16 * PART_STRIDE * 4;
-  return both > 227 * 1024 ? rings : both;
+  return (both > 227 * 1024 ? rings : both) + 16;            // + the word of the folded norm's last-unit flag
 }
 constexpr int DB1 = 8, DB2 = 6, DB4 = 4;                     // ring depths by row-tile count
 static_assert(skinny_smem<1, DB1>() <= 227 * 1024 && skinny_smem<2, DB2>() <= 227 * 1024 && skinny_smem<4, DB4>() <= 227 * 1024,
@@ -318,15 +366,22 @@ static_assert(skinny_smem<1, DB1>() <= 227 * 1024 && skinny_smem<2, DB2>() <= 22
 template <int MT, int DB>
 cudaError_t launch_one(const SkinnyParams& p, int grid, cudaStream_t stream) {
   constexpr int smem = skinny_smem<MT, DB>() < kMinSmemBytes ? kMinSmemBytes : skinny_smem<MT, DB>();
-  if (p.ab_f16) return launch_step_kernel(gemm_skinny_kernel<MT, DB, true>, grid, SK_THREADS, smem, stream, p.overlap != 0, p);
-  return launch_step_kernel(gemm_skinny_kernel<MT, DB, false>, grid, SK_THREADS, smem, stream, p.overlap != 0, p);
+  const bool fold = p.norm_gain != nullptr || p.in_row_rs != nullptr;
+  if (p.ab_f16) {
+    if (fold) return launch_step_kernel(gemm_skinny_kernel<MT, DB, true, true>, grid, SK_THREADS, smem, stream, p.overlap != 0, p);
+    return launch_step_kernel(gemm_skinny_kernel<MT, DB, true, false>, grid, SK_THREADS, smem, stream, p.overlap != 0, p);
+  }
+  if (fold) return launch_step_kernel(gemm_skinny_kernel<MT, DB, false, true>, grid, SK_THREADS, smem, stream, p.overlap != 0, p);
+  return launch_step_kernel(gemm_skinny_kernel<MT, DB, false, false>, grid, SK_THREADS, smem, stream, p.overlap != 0, p);
 }
 template <int MT, int DB>
 cudaError_t set_one() {
   constexpr int smem = skinny_smem<MT, DB>() < kMinSmemBytes ? kMinSmemBytes : skinny_smem<MT, DB>();
-  cudaError_t e = set_kernel_smem(gemm_skinny_kernel<MT, DB, true>, smem);
-  if (e != cudaSuccess) return e;
-  return set_kernel_smem(gemm_skinny_kernel<MT, DB, false>, smem);
+  cudaError_t e = set_kernel_smem(gemm_skinny_kernel<MT, DB, true, false>, smem);
+  if (e == cudaSuccess) e = set_kernel_smem(gemm_skinny_kernel<MT, DB, false, false>, smem);
+  if (e == cudaSuccess) e = set_kernel_smem(gemm_skinny_kernel<MT, DB, true, true>, smem);
+  if (e == cudaSuccess) e = set_kernel_smem(gemm_skinny_kernel<MT, DB, false, true>, smem);
+  return e;
 }
 
 }  // namespace

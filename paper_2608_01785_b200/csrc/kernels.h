@@ -112,6 +112,22 @@ struct SkinnyParams {
   int act_f16;
   int* status;               // nullable: the stage's device status words (the second one counts fp16 saturations)
   int* smid_log;
+  // RMSNorm folded into the GEMMs around it, as in GemmParams (rmsnorm(x) W^T = diag(r) ((x o g) W^T)).
+  //   Resid, producing side (norm_gain non-null): the epilogue also emits h = 16-bit(y o g) for the next GEMM and the
+  //   sum of y^2 over the unit's 32 columns into row_ss[row * ss_stride + unit]; the block that delivers the last unit
+  //   (units_done: one counter, zero at entry and at exit) sums every row's partials in a fixed order and writes
+  //   r = rsqrt(mean(y^2) + norm_eps) into row_rs[row].
+  const __nv_bfloat16* norm_gain;   // [N]
+  __nv_bfloat16* norm_h;     // 16-bit [T, N]
+  int norm_h_f16;
+  float* row_ss;             // [T][ss_stride], ss_stride >= N / 32
+  int ss_stride;
+  float* row_rs;             // [T]
+  int* units_done;
+  float norm_eps;
+  //   Qkv / GateUp, consuming side (in_row_rs non-null): every output row is scaled by r of its token before bias /
+  //   RoPE / SiLU.
+  const float* in_row_rs;    // [T]
 };
 // True when the skinny kernel covers this shape (few rows, K a multiple of 32, widths it can tile).
 bool gemm_skinny_supports(int T, int K, int N, int mode, int head_dim);

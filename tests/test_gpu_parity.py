@@ -591,3 +591,38 @@ def test_folded_rmsnorm_step_matches_oracle_and_every_budget(orc):
         assert prof["rmsnorm"][1] == 1 and prof["gemm_out"][1] == 2 and prof["gemm_down"][1] == 2
     finally:
         st.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("flags", [0, B.HS_FLAG_BF16_ACTIVATIONS])
+@pytest.mark.parametrize("n_rows", [16, 9])
+def test_small_step_takes_the_norms_into_its_projections(orc, n_rows, flags):
+    """Decode-only steps of at most 16 rows: the residual projections on the weight-streaming kernel emit the next
+    GEMM's un-normalised 16-bit operand and the rows' sums of squares, the projections behind them scale their output
+    rows by the RMSNorm factor, so that a three-layer step launches one RMSNorm (the first, which widens x_in) instead
+    of six.  Against the oracle on every row, bit for bit across budgets, in both activation formats."""
+    dims = wl.StageDims(3, 1024, 16, 2, 64, 3072)
+    r = np.random.default_rng(21)
+    batch = wl.BatchSpec([1] * n_rows, r.integers(40, 700, size=n_rows).tolist())
+    case = make_case(dims, batch, seed=31, kv_fill=True)
+    y_ref = orc.step(case.cfg, case.weights, case.kv_pool.copy(), batch.q_len, batch.ctx_len, case.block_tables, case.x)
+    st = make_stage(case, flags=flags)
+    try:
+        outs = {}
+        for budget in (st.sm_count, 40, 3, 1):
+            st.kv_pool.copy_(wl.bits_to_bf16_tensor(case.kv_pool, st.device))
+            outs[budget] = run_step(st, case, budget)
+        y, pool = outs[st.sm_count]
+        err = rel_err(y, y_ref)
+        print(f"small step with the norms in the projections, {n_rows} rows, flags {flags}: max|err|/RMS = {err:.2e}")
+        assert err <= TOL
+        for budget, (y_b, pool_b) in outs.items():
+            assert np.array_equal(y_b, y), budget
+            assert np.array_equal(pool_b, pool), budget
+        B.hs_stage_profile_enable(st.handle, True)
+        run_step(st, case, st.sm_count)
+        prof = B.hs_stage_profile_read(st.handle)
+        B.hs_stage_profile_enable(st.handle, False)
+        assert prof["rmsnorm"][1] == 1 and prof["gemm_qkv"][1] == 3 and prof["gemm_gateup"][1] == 3
+    finally:
+        st.close()
