@@ -17,8 +17,13 @@ class Stage:
     weights: per layer, a dict of bf16 CUDA tensors named as in hs_layer_weights_t.
     """
 
+    GUARD_BYTE = 0xA5
+
     def __init__(self, dims, weights: Sequence[Dict[str, torch.Tensor]], num_pages: int, max_tokens: int,
-                 max_seqs: int, max_pages_per_seq: int, max_position: int, device: int = 0, flags: int = 0):
+                 max_seqs: int, max_pages_per_seq: int, max_position: int, device: int = 0, flags: int = 0,
+                 guard_bytes: int = 0):
+        """guard_bytes > 0 (a multiple of 1024) puts that many bytes of a fixed pattern in front of and behind the
+        workspace and the KV pool; guards_intact() tells whether anything wrote there."""
         if not torch.cuda.is_available():
             raise RuntimeError("Stage needs a CUDA device; there is no CPU implementation")
         self.dims = dims
@@ -28,8 +33,18 @@ class Stage:
         if pool_bytes == 0 or ws_bytes == 0:
             raise B.HsError(B.HS_ERR_UNSUPPORTED_SHAPE, "configuration rejected")
         self.weights = [{k: v.to(self.device, torch.bfloat16).contiguous() for k, v in lw.items()} for lw in weights]
-        self.kv_pool = torch.zeros(pool_bytes // 2, dtype=torch.bfloat16, device=self.device)
-        self.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=self.device)
+        assert guard_bytes % 1024 == 0
+        self._guarded = []
+        if guard_bytes:
+            def guarded(n_bytes):
+                raw = torch.full((n_bytes + 2 * guard_bytes,), self.GUARD_BYTE, dtype=torch.uint8, device=self.device)
+                self._guarded.append((raw, guard_bytes))
+                return raw[guard_bytes: guard_bytes + n_bytes]
+            self.kv_pool = guarded(pool_bytes).zero_().view(torch.bfloat16)
+            self.workspace = guarded(ws_bytes)
+        else:
+            self.kv_pool = torch.zeros(pool_bytes // 2, dtype=torch.bfloat16, device=self.device)
+            self.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=self.device)
         ptrs = [{k: v.data_ptr() for k, v in lw.items()} for lw in self.weights]
         self.handle = B.hs_stage_create(self.cfg, ptrs, self.kv_pool.data_ptr(), self.workspace.data_ptr())
         self.sm_count = B.hs_stage_sm_count(self.handle)
@@ -69,6 +84,12 @@ class Stage:
     def saturation_count(self) -> int:
         """fp16 activation values clamped to +-65504 since the stage was created (0 for a well-scaled model)."""
         return B.hs_stage_saturation_count(self.handle)
+
+    def guards_intact(self) -> bool:
+        """True when the guard bytes around the workspace and the KV pool (guard_bytes of the constructor) still hold
+        their pattern."""
+        return all(bool((raw[:g] == self.GUARD_BYTE).all()) and bool((raw[-g:] == self.GUARD_BYTE).all())
+                   for raw, g in self._guarded)
 
     def set_modulation(self, mod) -> None:
         """fp32 device tensor [n_layers, max_seqs, 6, d_model] (or None): per-sequence shift / scale / gate vectors

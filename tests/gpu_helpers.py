@@ -12,13 +12,13 @@ from tests.helpers import Case
 
 
 def make_stage(case: Case, max_tokens: Optional[int] = None, max_position: Optional[int] = None,
-               weights=None, flags: int = 0) -> Stage:
+               weights=None, flags: int = 0, guard_bytes: int = 0) -> Stage:
     """A stage with the case's dims and weights whose pool starts as a copy of the case's pool and whose
     allocator has handed out the case's block tables (the library's allocator must reproduce them)."""
     batch = case.batch
     st = Stage(case.dims, weights if weights is not None else case.weights_t, case.cfg.num_pages,
                max_tokens or batch.n_tokens, batch.n_seqs, case.mpps, max_position or max(batch.total_len()),
-               flags=flags)
+               flags=flags, guard_bytes=guard_bytes)
     st.kv_pool.copy_(wl.bits_to_bf16_tensor(case.kv_pool, st.device))
     tables = [st.kv_alloc(s, t) for s, t in enumerate(batch.total_len())]
     bt = st.block_table_array(tables)

@@ -626,3 +626,54 @@ def test_small_step_takes_the_norms_into_its_projections(orc, n_rows, flags):
         assert prof["rmsnorm"][1] == 1 and prof["gemm_qkv"][1] == 3 and prof["gemm_gateup"][1] == 3
     finally:
         st.close()
+
+
+# ------------------------------------------------ guard bytes around every buffer --
+GUARDED = {
+    # all four projections on SM pairs, both norms folded, stream-K residual GEMMs, both attention kernels side by side
+    "pairs_folded": (wl.StageDims(2, 1024, 16, 4, 64, 2048), [1400, 1100] + [1] * 40, [0, 200] + [57 + 13 * i for i in range(40)]),
+    # single blocks with a K split, ragged row tile
+    "single_blocks": (wl.StageDims(2, 512, 8, 2, 64, 1408), [100, 21, 1], [0, 40, 300]),
+    # weight-streaming kernel with the small-step fold
+    "small_step": (wl.StageDims(2, 1024, 16, 2, 64, 3072), [1] * 11, [33 + 29 * i for i in range(11)]),
+}
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name", sorted(GUARDED))
+def test_a_step_writes_nothing_outside_its_buffers(name):
+    """Guard bytes in front of and behind the workspace, the KV pool, x_in and y_out keep their pattern through steps
+    at several budgets (the step forms differ: SM pairs with folded norms and stream-K, single blocks with a K split,
+    the weight-streaming kernel); y_out is written completely."""
+    dims, q_len, ctx_len = GUARDED[name]
+    batch = wl.BatchSpec(list(q_len), list(ctx_len))
+    case = make_case(dims, batch, seed=5, kv_fill=True)
+    G = 4096
+    st = make_stage(case, guard_bytes=G)
+    try:
+        T, d = batch.n_tokens, dims.d_model
+        x_raw = torch.full((T * d * 2 + 2 * G,), 0xA5, dtype=torch.uint8, device=st.device)
+        y_raw = torch.full((T * d * 4 + 2 * G,), 0xA5, dtype=torch.uint8, device=st.device)
+        x = x_raw[G: G + T * d * 2].view(torch.bfloat16).view(T, d)
+        y = y_raw[G: G + T * d * 4].view(torch.float32).view(T, d)
+        x.copy_(case.x_t.to(st.device))
+        for budget in (st.sm_count, 37, 2, 1):
+            st.kv_pool.copy_(wl.bits_to_bf16_tensor(case.kv_pool, st.device))
+            y.fill_(float("nan"))
+            st.step(st.make_batch(batch.q_len, batch.ctx_len, case.block_tables, x, y), budget)
+            torch.cuda.synchronize()
+            assert st.status() == 0
+            assert st.guards_intact(), (name, budget)
+            for raw in (x_raw, y_raw):
+                assert bool((raw[:G] == 0xA5).all()) and bool((raw[-G:] == 0xA5).all()), (name, budget)
+            assert bool(torch.isfinite(y).all()), (name, budget)
+            assert torch.equal(x, case.x_t.to(st.device)), "x_in is read only"
+        # the step forms the cases are named for were the ones that ran
+        B.hs_stage_profile_enable(st.handle, True)
+        st.step(st.make_batch(batch.q_len, batch.ctx_len, case.block_tables, x, y), st.sm_count)
+        torch.cuda.synchronize()
+        prof = B.hs_stage_profile_read(st.handle)
+        B.hs_stage_profile_enable(st.handle, False)
+        assert prof["rmsnorm"][1] == (4 if name == "single_blocks" else 1)
+    finally:
+        st.close()

@@ -62,6 +62,23 @@ def test_rmsnorm_unit_rms_and_scale_invariance(oracle64):
     assert np.allclose(oracle64.rmsnorm(x1, np.ones(4), 5.0), 2.0 / 3.0, atol=1e-12)
 
 
+def test_rmsnorm_factors_out_of_the_projection_behind_it(oracle64):
+    """rmsnorm(x) W^T = diag(r) ((x o g) W^T) with r = 1 / sqrt(mean(x^2) + eps): the identity behind folding the norm
+    into the GEMMs around it (the 16-bit rounding then falls on x o g instead of on r (x o g))."""
+    r = np.random.default_rng(17)
+    x = r.standard_normal((9, 160)) * np.array([0.01, 0.3, 1, 2, 5, 10, 40, 100, 1000])[:, None]
+    g = 1.0 + 0.3 * r.standard_normal(160)
+    w = r.standard_normal((48, 160)) / math.sqrt(160)
+    eps = float(np.float32(1e-6))                        # the oracle takes eps as a C float
+    rs = 1.0 / np.sqrt((x ** 2).mean(axis=1) + eps)
+    before = oracle64.linear(oracle64.rmsnorm(x, g, eps), w)
+    after = rs[:, None] * oracle64.linear(x * g, w)
+    assert np.allclose(before, after, rtol=1e-12, atol=1e-12)
+    # a mistake in the factor (eps outside the root, the mean over the wrong axis, g left out) does not survive
+    assert not np.allclose(before, (1.0 / (np.sqrt((x ** 2).mean(axis=1)) + eps))[:, None] * oracle64.linear(x * g, w), rtol=1e-9, atol=0)
+    assert not np.allclose(before, rs[:, None] * oracle64.linear(x, w), rtol=1e-3, atol=1e-6)
+
+
 def test_rmsnorm_matches_library(oracle32):
     r = np.random.default_rng(2)
     x = r.standard_normal((7, 96)).astype(np.float32)
