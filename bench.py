@@ -285,6 +285,7 @@ def rooflines(name, dims, batch, prof, steps, ms_step, clocks, budget, sm_count,
     peak_t = (peaks["bf16_burst"] if use_burst else peaks["bf16_sustained"]) * budget / sm_count
     mhz = (clocks or {}).get("sm_mhz")
     out = {}
+    folded = prof["rmsnorm"][1] < prof["gemm_out"][1]      # fewer norm launches than layers: the residual GEMMs carry them
     for cls, flops in gemm_classes(dims, T).items():
         ms, n = prof[cls]
         if not n:
@@ -296,6 +297,10 @@ def rooflines(name, dims, batch, prof, steps, ms_step, clocks, budget, sm_count,
                     "frac_of_sustained_peak": ach / (peaks["bf16_sustained"] * budget / sm_count),
                     "flops_per_launch": flops, "avg_launch_ms": avg_s * 1e3, "launches": n,
                     "ms_x_sm_mhz": avg_s * 1e3 * mhz if mhz else None}
+        if folded and cls in ("gemm_out", "gemm_down"):
+            out[cls]["note"] = ("this launch also does the RMSNorm that follows it (reads the residual stream, adds, writes it "
+                                "back, emits the next GEMM's 16-bit operand and the rows' sums of squares); only the "
+                                "projection's flops are counted")
     _, attn_flops = flops_per_step(dims, batch)
     ms, n = prof["attn_prefill"]
     if n:

@@ -39,7 +39,10 @@ hs_status_t hs_op_gemm_f16(const void *a, const void *w, const float *resid, flo
 /*
  * Diagnosis: device address and size of one of the stage's private intermediates after a step
  * (contents of the LAST layer executed).  name is one of
- *   "h"   [max_tokens, d]      last RMSNorm output            (fp16; bf16 with HS_FLAG_BF16_ACTIVATIONS)
+ *   "h"   [max_tokens, d]      last RMSNorm output            (fp16; bf16 with HS_FLAG_BF16_ACTIVATIONS).  Where
+ *                              the norm is folded into the GEMMs around it (all projections on SM pairs, or a
+ *                              step of at most 16 rows; unconditioned stage) this is 16-bit(x o g), not yet scaled
+ *                              by the row's rsqrt(mean(x^2) + eps): the GEMM behind it applies that factor.
  *   "q"   [max_tokens, Hq*Dh]  queries after RoPE             (bf16)
  *   "o"   [max_tokens, Hq*Dh]  attention output               (fp16; bf16 with the flag)
  *   "act" [max_tokens, F]      silu(gate) * up                (fp16; bf16 with the flag)
@@ -58,8 +61,11 @@ hs_status_t hs_stage_debug_buffer(hs_stage_t *stage, const char *name, void **de
  * events on the step's stream.  hs_stage_profile_read synchronises those events and adds, per
  * kernel class, the elapsed milliseconds to ms[class] and the launch count to launches[class]
  * (host arrays of HS_PROFILE_CLASSES entries, accumulated since the last read), then forgets them.
- * While enabled, the kernels of a step never overlap (the events between them serialise the stream), so the
- * per-class times add up to slightly more than an unprofiled full-budget step takes.
+ * While enabled, the kernels of a step never overlap (the events between them serialise the stream; the prefill
+ * and decode attention kernels of a layer, which otherwise run side by side on two shares of the budget, run one
+ * after the other on the whole budget), so the per-class times add up to more than an unprofiled step takes.
+ * A residual GEMM that folds the RMSNorm behind it is timed with that work (classes 5 and 7); class 0 then counts
+ * the one norm launch a step keeps.
  * Classes: 0 rmsnorm, 1 qkv gemm, 2 prefill attention, 3 decode attention (with the merge of its split
  * partials), 4 unused (always zero; kept so that the class numbers stay what they were),
  * 5 out-proj gemm, 6 gate/up gemm, 7 down gemm.
