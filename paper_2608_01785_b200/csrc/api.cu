@@ -159,6 +159,7 @@ hs_status_t ensure_attributes(int device) {
   if ((e = attention_set_attributes()) != cudaSuccess) return cuda_fail("attention attributes", e);
   if ((e = head_set_attributes()) != cudaSuccess) return cuda_fail("head attributes", e);
   if ((e = gemm_skinny_set_attributes()) != cudaSuccess) return cuda_fail("small-step gemm attributes", e);
+  if ((e = small_step_set_attributes()) != cudaSuccess) return cuda_fail("one-launch small step attributes", e);
   if (device >= 0 && device < 64) g_attrs_set[device] = true;
   return HS_OK;
 }
@@ -465,6 +466,17 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
   if (st != HS_OK) return st;
   s->ring_pos = (slot + 1) % kRing;
 
+  {  // the layers' constants for the one-launch small step travel with the metadata (biases may change between steps)
+    static_assert(sizeof(SmallLayer) == 24 * 4, "MetaLayout::small_layers holds 24 words per layer");
+    SmallLayer* sl = reinterpret_cast<SmallLayer*>(s->pinned[slot] + s->ml.small_layers);
+    for (int l = 0; l < c.n_layers; ++l) {
+      const hs_layer_weights_t& wo = s->operands[l];
+      sl[l] = SmallLayer{wo.w_q, wo.w_k, wo.w_v, wo.w_o, wo.w_gate, wo.w_up, wo.w_down,
+                         static_cast<const __nv_bfloat16*>(s->layers[l].g_attn),
+                         static_cast<const __nv_bfloat16*>(s->layers[l].g_mlp),
+                         {s->qkv_bias[l].b[0], s->qkv_bias[l].b[1], s->qkv_bias[l].b[2]}};
+    }
+  }
   int32_t* meta = reinterpret_cast<int32_t*>(s->ws_dev + s->ws.meta);
   if (cudaMemcpyAsync(meta, s->pinned[slot], size_t(s->ml.total) * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
       cudaEventRecord(s->ev[slot], stream) != cudaSuccess)
@@ -588,6 +600,43 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     }
   }
 
+  auto make_attn = [&](int l) {
+    AttnParams a{};
+    a.tm_kv = s->tm_kv;
+    a.tm_q = s->tm_q_attn;
+    a.prefill_tokens = prefill_tokens_per_item(c.n_q_heads / c.n_kv_heads);
+    a.o_f16 = f16;
+    a.overlap = overlap;
+    a.q = q; a.o = o;
+    a.n_q_heads = c.n_q_heads; a.n_kv_heads = c.n_kv_heads; a.head_dim = Dh;
+    a.num_pages = c.num_pages; a.max_pages_per_seq = c.max_pages_per_seq; a.layer = l;
+    a.seq_tok0 = meta + s->ml.seq_tok0;
+    a.seq_ctx = meta + s->ml.seq_ctx;
+    a.seq_qlen = meta + s->ml.seq_qlen;
+    a.bidirectional = (c.flags & HS_FLAG_BIDIRECTIONAL) ? 1 : 0;
+    a.block_tables = meta + s->ml.block_tables;
+    a.prefill_items = meta + s->ml.prefill_items;
+    a.n_prefill_items = plan.n_prefill_items;
+    a.decode_items = meta + s->ml.decode_items;
+    a.n_decode_items = plan.n_decode_items;
+    a.decode_rows = meta + s->ml.decode_rows;
+    a.n_decode_rows = plan.n_decode_rows;
+    a.part_o = reinterpret_cast<float*>(s->ws_dev + s->ws.part_o);
+    a.part_ml = reinterpret_cast<float*>(s->ws_dev + s->ws.part_ml);
+    a.counters = meta + s->ml.counters + 2 * l;
+    a.group_done = meta + s->ml.group_done;
+    a.status = status;
+    a.smid_log = slots(2);       // prefill in class 2, decode in class 3 (the next slots)
+    return a;
+  };
+  // A decode-only step of at most 16 rows whose projections all run on the weight-streaming kernel with the norms
+  // folded, under a partial budget: after the first norm, ONE cooperative launch does all layers (launch_small_step);
+  // the same device functions on the same units and items, so the same bits as the launches below (which is why this
+  // choice may look at the budget).  At the full budget the separate launches overlap each other's set-up and are the
+  // faster form (talker step 0.40 ms against 0.52); below it they run strictly one after the other (0.58 / 0.60 /
+  // 0.75 ms at 112 / 74 / 37 SMs against 0.52 / 0.54 / 0.69 in one launch).  Not while the per-kernel timers run.
+  const bool one_launch = sk_fold_mlp && sk_fold_attn && skinny(d, q_dim + 2 * kv_dim, kGemmQkv) && skinny(d, F, kGemmGateUp) &&
+                          plan.n_prefill_items == 0 && plan.n_decode_items > 0 && !s->profile && sm_budget < s->sm_count;
   for (int l = 0; l < c.n_layers && e == cudaSuccess; ++l) {
     const hs_layer_weights_t& w = s->layers[l];
     const LayerMaps& m = s->maps[l];
@@ -613,6 +662,29 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     const bool folded_attn_norm = (fold_norm || sk_fold_attn) && l > 0;   // the previous layer's down-projection produced h and the sums
     if (!folded_attn_norm) { LaunchTimer t(s, 0, stream); where = "rmsnorm"; e = launch_rmsnorm(np, sm_budget, stream); }
     if (e != cudaSuccess) break;
+    if (one_launch) {
+      SmallStepParams sp{};
+      sp.attn = make_attn(0);
+      sp.attn.smid_log = nullptr;
+      sp.layers = reinterpret_cast<const SmallLayer*>(meta + s->ml.small_layers);
+      sp.n_layers = c.n_layers; sp.T = T; sp.d = d; sp.F = F; sp.f16 = f16;
+      sp.q_dim = q_dim; sp.kv_dim = kv_dim; sp.head_dim = Dh; sp.n_kv_heads = c.n_kv_heads;
+      sp.x = x; sp.h = h; sp.q = q; sp.o = o;
+      sp.act = reinterpret_cast<__nv_bfloat16*>(s->ws_dev + s->ws.act);
+      sp.kv_pool = s->kv_pool; sp.layer_kv_elems = layer_kv_elems;
+      sp.tok_pos = meta + s->ml.tok_pos; sp.tok_slot = meta + s->ml.tok_slot;
+      sp.rope = reinterpret_cast<const float2*>(s->ws_dev + s->ws.rope);
+      sp.counters = meta + s->ml.counters;
+      sp.row_ss = reinterpret_cast<float*>(s->ws_dev + s->ws.row_ss);
+      sp.row_rs = reinterpret_cast<float*>(s->ws_dev + s->ws.row_rs);
+      sp.units_done = reinterpret_cast<int*>(s->ws_dev + s->ws.row_done);
+      sp.eps = c.rms_eps;
+      sp.grid_bar = meta + s->ml.grid_bar;
+      sp.status = status;
+      sp.smid_log = slots(1);
+      where = "small step"; e = launch_small_step(sp, sm_budget, stream);
+      break;
+    }
 
     GemmParams g{};
     g.tm_a = a_rows == 128 ? s->tm_h : s->tm_h_s[a_sel];
@@ -648,32 +720,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     } else { LaunchTimer t(s, 1, stream); where = "qkv gemm"; e = launch_gemm(g, sm_budget, stream); }
     if (e != cudaSuccess) break;
 
-    AttnParams a{};
-    a.tm_kv = s->tm_kv;
-    a.tm_q = s->tm_q_attn;
-    a.prefill_tokens = prefill_tokens_per_item(c.n_q_heads / c.n_kv_heads);
-    a.o_f16 = f16;
-    a.overlap = overlap;
-    a.q = q; a.o = o;
-    a.n_q_heads = c.n_q_heads; a.n_kv_heads = c.n_kv_heads; a.head_dim = Dh;
-    a.num_pages = c.num_pages; a.max_pages_per_seq = c.max_pages_per_seq; a.layer = l;
-    a.seq_tok0 = meta + s->ml.seq_tok0;
-    a.seq_ctx = meta + s->ml.seq_ctx;
-    a.seq_qlen = meta + s->ml.seq_qlen;
-    a.bidirectional = (c.flags & HS_FLAG_BIDIRECTIONAL) ? 1 : 0;
-    a.block_tables = meta + s->ml.block_tables;
-    a.prefill_items = meta + s->ml.prefill_items;
-    a.n_prefill_items = plan.n_prefill_items;
-    a.decode_items = meta + s->ml.decode_items;
-    a.n_decode_items = plan.n_decode_items;
-    a.decode_rows = meta + s->ml.decode_rows;
-    a.n_decode_rows = plan.n_decode_rows;
-    a.part_o = reinterpret_cast<float*>(s->ws_dev + s->ws.part_o);
-    a.part_ml = reinterpret_cast<float*>(s->ws_dev + s->ws.part_ml);
-    a.counters = meta + s->ml.counters + 2 * l;
-    a.group_done = meta + s->ml.group_done;
-    a.status = status;
-    a.smid_log = slots(2);       // prefill in class 2, decode in class 3 (the next slots)
+    AttnParams a = make_attn(l);
     if (decode_sms > 0) {
       // side by side: the decode kernel on the stage's own stream with decode_sms of the budget, the prefill kernel on
       // the caller's stream with the rest; both are joined before the out-projection

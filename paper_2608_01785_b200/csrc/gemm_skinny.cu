@@ -20,6 +20,9 @@
 // unchanged and every load is a full 16 bytes.
 #include <cuda_fp16.h>
 
+#include <algorithm>
+
+#include "attention_decode.cuh"
 #include "kernels.h"
 #include "ptx.cuh"
 
@@ -85,9 +88,12 @@ __device__ __forceinline__ const uint8_t* unit_row(const SkinnyParams& p, int un
 // MT: 16-row tiles of activations (T <= 16 MT); DB: depth of a warp's ring of K steps.
 // FOLD: the instantiation that knows the folded RMSNorm (producing side in Resid mode, consuming side in the others);
 // the plain one carries none of its code.
-template <int MT, int DB, bool F16, bool FOLD>
-__global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const SkinnyParams p) {
-  extern __shared__ __align__(16) uint8_t sk_smem[];
+// The body is a device function shared by the kernel of its own and by the one-launch small step: the calling
+// thread block (SK_THREADS threads) is number `block` of `n_blocks` working on the launch's units; `wait` is called
+// once by every thread, after the weights of the first steps have been requested, and must return when the
+// activations (the previous kernel's or phase's output) are visible.
+template <int MT, int DB, bool F16, bool FOLD, typename Wait>
+__device__ __forceinline__ void gemm_skinny_body(const SkinnyParams& p, uint8_t* sk_smem, int block, int n_blocks, Wait wait) {
   constexpr int STAGE_BYTES = (NT + 2 * MT) * 512;          // per warp and K step: 4 weight tiles, 2 MT row groups
   constexpr int RING_BYTES = DB * STAGE_BYTES;              // per warp
   constexpr int PART_FLOATS = MT * 16 * PART_STRIDE;        // per warp
@@ -99,7 +105,6 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
   float* part_all = reinterpret_cast<float*>(sk_smem + (ALIAS ? 0 : SK_WARPS * RING_BYTES));
   constexpr int PART_PITCH = ALIAS ? RING_BYTES / 4 : PART_FLOATS;   // floats between two warps' partial tiles
   float* part = part_all + warp * PART_PITCH;
-  log_smid(p.smid_log);
 
   const int units = p.mode == kGemmGateUp ? p.N >> 4 : p.N >> 5;
   // 32-wide K steps, dealt to the warps in turn: warp w takes steps w, w + 8, ...  The eight warps move through
@@ -147,15 +152,22 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
     }
   };
 
-  int unit = blockIdx.x;
+  int unit = block;
   if (unit < units) {                                       // weights never change: fetch them before the wait
     set_rows(unit);
 #pragma unroll
     for (int s = 0; s < DB - 1; ++s)
       if (s < n) issue_b(s, s);
   }
-  griddep_wait();
-  griddep_launch_dependents();
+  // the epilogue row of this thread and what it needs from the step's metadata (written before the step's first kernel)
+  const int e_row = threadIdx.x >> 2, e_jq = (threadIdx.x & 3) * 4;
+  const bool e_ok = e_row < MT * 16 && e_row < p.T;
+  int e_pos = 0, e_slot = 0;
+  if (p.mode == kGemmQkv && e_ok) {
+    e_pos = p.tok_pos[e_row];
+    e_slot = p.tok_slot[e_row];
+  }
+  wait();
   if (unit < units) {
 #pragma unroll
     for (int s = 0; s < DB - 1; ++s) {
@@ -168,7 +180,31 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
   if (FOLD && p.in_row_rs != nullptr && int(threadIdx.x >> 2) < p.T) rs_in = __ldcg(p.in_row_rs + (threadIdx.x >> 2));
   int* last_unit = reinterpret_cast<int*>(part_all + SK_WARPS * PART_PITCH);   // FOLD: one word behind the partial tiles
 
-  for (; unit < units; unit += gridDim.x) {
+  for (; unit < units; unit += n_blocks) {
+    // What the epilogue will read from memory is requested now, so that it has arrived when the K loop ends: the
+    // output block to add to, the gains of a folded norm, the rotation of the row's position.
+    float4 y_pre_lo = make_float4(0.f, 0.f, 0.f, 0.f), y_pre_hi = y_pre_lo, cs0 = y_pre_lo, cs1 = y_pre_lo;
+    uint2 ng_lo = make_uint2(0u, 0u), ng_hi = ng_lo;
+    if (e_ok) {
+      if (p.mode == kGemmResid) {
+        if (p.accumulate) {
+          const float4* y_lo = reinterpret_cast<const float4*>(p.y + size_t(e_row) * p.N + unit * 32 + e_jq);
+          y_pre_lo = __ldcg(y_lo);                           // (through the L2: see the one-launch small step)
+          y_pre_hi = __ldcg(y_lo + 4);
+        }
+        if (FOLD && p.norm_gain != nullptr) {
+          ng_lo = __ldg(reinterpret_cast<const uint2*>(p.norm_gain + unit * 32 + e_jq));
+          ng_hi = __ldg(reinterpret_cast<const uint2*>(p.norm_gain + unit * 32 + e_jq + 16));
+        }
+      } else if (p.mode == kGemmQkv) {
+        const int upr = p.head_dim >> 5, head = unit / upr, sub = unit - head * upr;
+        if (head < p.q_dim / p.head_dim + p.n_kv_heads) {
+          const float4* cs = reinterpret_cast<const float4*>(p.rope + size_t(e_pos) * (p.head_dim >> 1) + sub * 16 + e_jq);
+          cs0 = cs[0];
+          cs1 = cs[1];
+        }
+      }
+    }
     float acc[MT][NT][4];
 #pragma unroll
     for (int i = 0; i < MT; ++i)
@@ -204,7 +240,7 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
     cp_async_wait<0>();
 
     // the next unit's first steps travel while this one is reduced and written (when the rings stay free)
-    const int next = unit + gridDim.x;
+    const int next = unit + n_blocks;
     if (!ALIAS && next < units) {
       set_rows(next);
       prologue();
@@ -249,7 +285,7 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
           hi.x *= g_hi.x; hi.y *= g_hi.y; hi.z *= g_hi.z; hi.w *= g_hi.w;
         }
         if (p.accumulate) {
-          const float4 a = *y_lo, b = *y_hi;
+          const float4 a = y_pre_lo, b = y_pre_hi;
           lo.x += a.x; lo.y += a.y; lo.z += a.z; lo.w += a.w;
           hi.x += b.x; hi.y += b.y; hi.z += b.z; hi.w += b.w;
         }
@@ -258,8 +294,7 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
         if (FOLD && p.norm_gain != nullptr) {
           // folded RMSNorm, producing side: the next GEMM's operand and this unit's share of the row's sum of squares
           // (the four threads of a row are neighbours in a warp)
-          const uint2 g_lo = __ldg(reinterpret_cast<const uint2*>(p.norm_gain + unit * 32 + jq));
-          const uint2 g_hi = __ldg(reinterpret_cast<const uint2*>(p.norm_gain + unit * 32 + jq + 16));
+          const uint2 g_lo = ng_lo, g_hi = ng_hi;
           float v[8] = {lo.x * __uint_as_float(g_lo.x << 16), lo.y * __uint_as_float(g_lo.x & 0xffff0000u),
                         lo.z * __uint_as_float(g_lo.y << 16), lo.w * __uint_as_float(g_lo.y & 0xffff0000u),
                         hi.x * __uint_as_float(g_hi.x << 16), hi.y * __uint_as_float(g_hi.x & 0xffff0000u),
@@ -300,8 +335,7 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
           b[2] += __uint_as_float(wh.y << 16); b[3] += __uint_as_float(wh.y & 0xffff0000u);
         }
         if (head < n_q_heads + p.n_kv_heads) {               // q and k heads are rotated
-          const float4* cs = reinterpret_cast<const float4*>(p.rope + size_t(p.tok_pos[row]) * half + i0);
-          const float4 t0 = cs[0], t1 = cs[1];               // (cos, sin) of pairs i0 .. i0 + 3
+          const float4 t0 = cs0, t1 = cs1;                   // (cos, sin) of pairs i0 .. i0 + 3, requested at the unit's start
           const float c[4] = {t0.x, t0.z, t1.x, t1.z}, sn[4] = {t0.y, t0.w, t1.y, t1.w};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
@@ -318,7 +352,7 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
           dst = p.q_out + size_t(row) * p.q_dim + head * Dh + i0;
         } else {
           const int hk = head - n_q_heads;
-          const int slot = p.tok_slot[row];
+          const int slot = e_slot;
           dst = hk < p.n_kv_heads ? cache_row(p.k_cache, slot, hk, p.n_kv_heads, Dh) + i0
                                   : cache_row(p.v_cache, slot, hk - p.n_kv_heads, p.n_kv_heads, Dh) + i0;
         }
@@ -354,6 +388,16 @@ __global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const Skinny
   }
 }
 
+template <int MT, int DB, bool F16, bool FOLD>
+__global__ void __launch_bounds__(SK_THREADS, 1) gemm_skinny_kernel(const SkinnyParams p) {
+  extern __shared__ __align__(16) uint8_t sk_smem[];
+  log_smid(p.smid_log);
+  gemm_skinny_body<MT, DB, F16, FOLD>(p, sk_smem, int(blockIdx.x), int(gridDim.x), [] {
+    griddep_wait();
+    griddep_launch_dependents();
+  });
+}
+
 template <int MT, int DB>
 constexpr int skinny_smem() {
   constexpr int rings = SK_WARPS * DB * (NT + 2 * MT) * 512, both = rings + SK_WARPS * MT * 16 * PART_STRIDE * 4;
@@ -382,6 +426,142 @@ cudaError_t set_one() {
   if (e == cudaSuccess) e = set_kernel_smem(gemm_skinny_kernel<MT, DB, true, true>, smem);
   if (e == cudaSuccess) e = set_kernel_smem(gemm_skinny_kernel<MT, DB, false, true>, smem);
   return e;
+}
+
+
+// ============================================================ one-launch small step ==
+// Shared memory: the weight-streaming GEMM's rings and partial tiles from offset 0 (the decode attention's page rings
+// use the front of the same area in their phase), the decode attention's mbarriers behind them.
+constexpr int SS_BAR_OFFSET = (skinny_smem<1, DB1>() + 1023) / 1024 * 1024;
+constexpr int SS_SMEM = SS_BAR_OFFSET + 512 + 1024;          // + barriers + room to align the base
+static_assert(SS_SMEM <= 227 * 1024 && SS_SMEM >= kMinSmemBytes, "one block per SM");
+static_assert(DC_WARPS * DC_STAGES * 2 * Geom<128>::PAGE_BYTES <= SS_BAR_OFFSET, "the page rings fit in front of the barriers");
+static_assert(DC_WARPS * 32 <= SK_THREADS, "the decode phase uses the first warps of the block");
+
+// Arrives at the grid barrier and waits until `target` blocks have (bounded: gives up after the wait limit, records
+// HS_ERR_TIMEOUT and returns false in every thread of the block).
+__device__ __forceinline__ bool grid_barrier(int* counter, int target, int* status) {
+  __syncthreads();                      // this block's writes of the phase come before thread 0's fence
+  int failed = 0;
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(counter, 1);
+    const unsigned long long t0 = globaltimer_ns();
+    for (;;) {
+      int seen;
+      asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+      if (seen >= target) break;
+      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        atomicExch(status, kErrTimeout);
+        failed = 1;
+        break;
+      }
+      __nanosleep(32);
+    }
+    __threadfence();
+  }
+  return __syncthreads_or(failed) == 0;
+}
+
+template <int DH, bool F16>
+__global__ void __launch_bounds__(SK_THREADS, 1) small_step_kernel(const __grid_constant__ SmallStepParams p) {
+  extern __shared__ uint8_t ss_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(ss_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* dc_bars = reinterpret_cast<uint64_t*>(smem + SS_BAR_OFFSET);
+  log_smid(p.smid_log);
+  const int block = int(blockIdx.x), grid = int(gridDim.x);
+  const int qkv_n = p.q_dim + 2 * p.kv_dim;
+  const int nb_qkv = min(grid, qkv_n >> 5), nb_attn = min(grid, p.attn.n_decode_items), nb_d = min(grid, p.d >> 5),
+            nb_gu = min(grid, p.F >> 4);
+  int arrived = 0;                      // grid barriers this block has been through
+  bool dead = false;                    // a barrier ran out of time: no further waits, leave after the phase
+  auto barrier = [&] {
+    ++arrived;
+    if (!dead && !grid_barrier(p.grid_bar, arrived * grid, p.status)) dead = true;
+  };
+  auto base = [&](const void* a, int K, int N, int mode) {
+    SkinnyParams k{};
+    k.a = a; k.T = p.T; k.K = K; k.N = N; k.mode = mode;
+    k.ab_f16 = F16 ? 1 : 0;
+    k.status = p.status;
+    return k;
+  };
+  auto fold_out = [&](SkinnyParams& k, const __nv_bfloat16* gain) {
+    k.norm_gain = gain; k.norm_h = p.h; k.norm_h_f16 = F16 ? 1 : 0;
+    k.row_ss = p.row_ss; k.ss_stride = p.d >> 5; k.row_rs = p.row_rs; k.units_done = p.units_done; k.norm_eps = p.eps;
+  };
+  for (int l = 0; l < p.n_layers && !dead; ++l) {
+    const SmallLayer L = p.layers[l];
+    {  // QKV projection + RoPE + cache write (the norm in front of it: the step's first norm kernel, or folded)
+      SkinnyParams k = base(p.h, p.d, qkv_n, kGemmQkv);
+      k.w[0] = L.w_q; k.w[1] = L.w_k; k.w[2] = L.w_v;
+      k.q_dim = p.q_dim; k.kv_dim = p.kv_dim; k.head_dim = p.head_dim; k.n_kv_heads = p.n_kv_heads;
+      k.q_out = p.q;
+      k.k_cache = p.kv_pool + (size_t(l) * 2 + 0) * p.layer_kv_elems;
+      k.v_cache = p.kv_pool + (size_t(l) * 2 + 1) * p.layer_kv_elems;
+      k.tok_pos = p.tok_pos; k.tok_slot = p.tok_slot; k.rope = p.rope;
+      for (int i = 0; i < 3; ++i) k.qkv_bias[i] = L.bias[i];
+      if (l > 0) k.in_row_rs = p.row_rs;
+      auto w = [&] { if (l > 0) barrier(); };
+      if (block < nb_qkv) gemm_skinny_body<1, DB1, F16, true>(k, smem, block, nb_qkv, w);
+      else w();
+    }
+    if (dead) break;
+    {  // decode attention
+      auto w = [&] { barrier(); };
+      if (block < nb_attn) {
+        attn_decode_body<DH>(p.attn, l, p.counters + 2 * l, smem, dc_bars, block, nb_attn, w);
+        if (threadIdx.x == 0)           // the barriers' memory belongs to the next phase's rings no more, but end their life
+          for (int i = 0; i < DC_WARPS * DC_STAGES; ++i) mbar_inval(&dc_bars[i]);
+        __syncthreads();
+      } else {
+        w();
+      }
+    }
+    if (dead) break;
+    {  // out-projection + residual add (+ the MLP norm's operand, sums and r)
+      SkinnyParams k = base(p.o, p.q_dim, p.d, kGemmResid);
+      k.w[0] = L.w_o; k.y = p.x; k.accumulate = 1;
+      fold_out(k, L.g_mlp);
+      auto w = [&] { barrier(); };
+      if (block < nb_d) gemm_skinny_body<1, DB1, F16, true>(k, smem, block, nb_d, w);
+      else w();
+    }
+    if (dead) break;
+    {  // gate / up projection + SwiGLU
+      SkinnyParams k = base(p.h, p.d, p.F, kGemmGateUp);
+      k.w[0] = L.w_gate; k.w[1] = L.w_up;
+      k.act = p.act; k.act_f16 = F16 ? 1 : 0;
+      k.in_row_rs = p.row_rs;
+      auto w = [&] { barrier(); };
+      if (block < nb_gu) gemm_skinny_body<1, DB1, F16, true>(k, smem, block, nb_gu, w);
+      else w();
+    }
+    if (dead) break;
+    {  // down-projection + residual add (+ the next layer's attention norm)
+      SkinnyParams k = base(p.act, p.F, p.d, kGemmResid);
+      k.w[0] = L.w_down; k.y = p.x; k.accumulate = 1;
+      if (l + 1 < p.n_layers) fold_out(k, p.layers[l + 1].g_attn);
+      auto w = [&] { barrier(); };
+      if (block < nb_d) gemm_skinny_body<1, DB1, F16, true>(k, smem, block, nb_d, w);
+      else w();
+    }
+  }
+}
+
+template <int DH, bool F16>
+cudaError_t launch_small_one(const SmallStepParams& p, int grid, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(unsigned(grid), 1, 1);
+  cfg.blockDim = dim3(SK_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = SS_SMEM;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;      // all blocks resident at once: they wait on one another
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, small_step_kernel<DH, F16>, p);
 }
 
 }  // namespace
@@ -430,6 +610,22 @@ cudaError_t gemm_skinny_set_attributes() {
   if (e == cudaSuccess) e = set_one<2, DB2>();
   if (e == cudaSuccess) e = set_one<4, DB4>();
   return e;
+}
+
+cudaError_t small_step_set_attributes() {
+  cudaError_t e = set_kernel_smem(small_step_kernel<64, true>, SS_SMEM);
+  if (e == cudaSuccess) e = set_kernel_smem(small_step_kernel<64, false>, SS_SMEM);
+  if (e == cudaSuccess) e = set_kernel_smem(small_step_kernel<128, true>, SS_SMEM);
+  if (e == cudaSuccess) e = set_kernel_smem(small_step_kernel<128, false>, SS_SMEM);
+  return e;
+}
+
+cudaError_t launch_small_step(const SmallStepParams& p, int sm_budget, cudaStream_t stream) {
+  if (p.T <= 0 || p.T > 16 || p.attn.n_decode_items <= 0) return cudaErrorInvalidValue;
+  const int widest = std::max(std::max((p.q_dim + 2 * p.kv_dim) >> 5, p.attn.n_decode_items), std::max(p.d >> 5, p.F >> 4));
+  const int grid = widest < sm_budget ? widest : sm_budget;
+  if (p.head_dim == 128) return p.f16 ? launch_small_one<128, true>(p, grid, stream) : launch_small_one<128, false>(p, grid, stream);
+  return p.f16 ? launch_small_one<64, true>(p, grid, stream) : launch_small_one<64, false>(p, grid, stream);
 }
 
 cudaError_t launch_gemm_skinny(const SkinnyParams& p, int sm_budget, cudaStream_t stream) {

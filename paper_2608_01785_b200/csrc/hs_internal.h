@@ -58,6 +58,8 @@ struct MetaLayout {
   int decode_rows;                   // [max_seqs * 4]           {seq, token row, first item, splits}
   int counters;                      // [n_layers * 2]           work-queue heads, zero at step start
   int group_done;                    // [max_seqs * n_kv_heads]  finished decode splits per group, zero
+  int grid_bar;                      // [4]                      arrivals at the one-launch small step's grid barriers, zero
+  int small_layers;                  // [n_layers * 24]          SmallLayer records (12 pointers each) of the one-launch small step
   int total;                         // int32 words in the block
   int max_prefill_items, max_decode_items;
 };

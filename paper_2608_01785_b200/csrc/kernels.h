@@ -213,6 +213,36 @@ struct AttnParams {
   int* status;
   int* smid_log;                   // nullable: SM census slots; prefill uses [0, 160), decode [160, 320)
 };
+// ------------------------------------------------- one-launch small step --
+// A whole step of at most 16 decode rows whose four projections run on the weight-streaming kernel, as ONE
+// cooperative launch of at most sm_budget blocks: per layer QKV -> decode attention -> out-projection -> gate/up ->
+// down-projection, the phases separated by bounded grid-wide barriers (a counter in device memory), each phase the
+// same device function with the same unit / item decomposition as the kernel of its own, so that the results are
+// the same bits.  The RMSNorms are folded into the projections (SkinnyParams); the first norm of the step is
+// launched in front of it.
+struct SmallLayer {                // one layer's constants, in device memory (written with the step's metadata)
+  const void* w_q; const void* w_k; const void* w_v; const void* w_o;     // 16-bit operand copies, [out, in]
+  const void* w_gate; const void* w_up; const void* w_down;
+  const __nv_bfloat16* g_attn; const __nv_bfloat16* g_mlp;
+  const __nv_bfloat16* bias[3];    // optional q, k, v biases
+};
+struct SmallStepParams {
+  AttnParams attn;                 // the decode attention's arguments (layer and counters are set per layer)
+  const SmallLayer* layers;
+  int n_layers, T, d, F, f16;
+  int q_dim, kv_dim, head_dim, n_kv_heads;
+  float* x;                        // fp32 residual stream [T, d] (the caller's y_out)
+  __nv_bfloat16* h; __nv_bfloat16* q; __nv_bfloat16* o; __nv_bfloat16* act;
+  __nv_bfloat16* kv_pool; size_t layer_kv_elems;
+  const int32_t* tok_pos; const int32_t* tok_slot; const float2* rope;
+  int* counters;                   // [n_layers * 2] queue heads, zero at entry
+  float* row_ss; float* row_rs; int* units_done; float eps;
+  int* grid_bar;                   // one word, zero at entry: blocks arrived at the grid barriers so far
+  int* status; int* smid_log;
+};
+cudaError_t launch_small_step(const SmallStepParams& p, int sm_budget, cudaStream_t stream);
+cudaError_t small_step_set_attributes();
+
 cudaError_t launch_attention_prefill(const AttnParams& p, int sm_budget, cudaStream_t stream);
 cudaError_t launch_attention_decode(const AttnParams& p, int sm_budget, cudaStream_t stream);
 cudaError_t attention_set_attributes();

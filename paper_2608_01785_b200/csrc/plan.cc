@@ -83,6 +83,8 @@ MetaLayout make_meta_layout(const hs_stage_config_t& c) {
   m.decode_rows = take(c.max_seqs * 4);
   m.counters = take(c.n_layers * 2);
   m.group_done = take(c.max_seqs * c.n_kv_heads);
+  m.grid_bar = take(4);
+  m.small_layers = take(c.n_layers * 24);
   m.total = off;
   return m;
 }
@@ -228,6 +230,7 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
       for (int k = 0; k < 4; ++k) meta[ml.prefill_items + int(i) * 4 + k] = pre[i].v[k];
     for (int i = 0; i < c.n_layers * 2; ++i) meta[ml.counters + i] = 0;
     for (int i = 0; i < c.max_seqs * c.n_kv_heads; ++i) meta[ml.group_done + i] = 0;
+    for (int i = 0; i < 4; ++i) meta[ml.grid_bar + i] = 0;
   }
   p.n_prefill_items = int(pre.size());
   p.n_decode_items = n_dec_items;

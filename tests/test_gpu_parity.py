@@ -619,11 +619,16 @@ def test_small_step_takes_the_norms_into_its_projections(orc, n_rows, flags):
         for budget, (y_b, pool_b) in outs.items():
             assert np.array_equal(y_b, y), budget
             assert np.array_equal(pool_b, pool), budget
+        # the runs above took the one-launch form of the step (after the first norm one cooperative kernel walks all
+        # layers, its phases separated by grid barriers); with the per-kernel timers on, the same step runs as one
+        # launch per kernel: the same bits, one RMSNorm launch
         B.hs_stage_profile_enable(st.handle, True)
-        run_step(st, case, st.sm_count)
+        st.kv_pool.copy_(wl.bits_to_bf16_tensor(case.kv_pool, st.device))
+        y_k, pool_k = run_step(st, case, st.sm_count)
         prof = B.hs_stage_profile_read(st.handle)
         B.hs_stage_profile_enable(st.handle, False)
         assert prof["rmsnorm"][1] == 1 and prof["gemm_qkv"][1] == 3 and prof["gemm_gateup"][1] == 3
+        assert np.array_equal(y_k, y) and np.array_equal(pool_k, pool)
     finally:
         st.close()
 
