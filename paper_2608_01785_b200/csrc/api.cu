@@ -683,7 +683,11 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
       sp.status = status;
       sp.smid_log = slots(1);
       where = "small step"; e = launch_small_step(sp, sm_budget, stream);
-      break;
+      // a device or context that cannot hold the grid resident at once (or knows no cooperative launch) takes the
+      // separate launches below: the same results
+      if (e != cudaErrorCooperativeLaunchTooLarge && e != cudaErrorNotSupported) break;
+      cudaGetLastError();
+      e = cudaSuccess;
     }
 
     GemmParams g{};

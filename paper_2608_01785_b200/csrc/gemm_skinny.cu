@@ -444,8 +444,8 @@ __device__ __forceinline__ bool grid_barrier(int* counter, int target, int* stat
   __syncthreads();                      // this block's writes of the phase come before thread 0's fence
   int failed = 0;
   if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(counter, 1);
+    // release: the block's writes (ordered before this thread by the barrier above) are visible to whoever sees the count
+    asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(counter) : "memory");
     const unsigned long long t0 = globaltimer_ns();
     for (;;) {
       int seen;
@@ -458,9 +458,8 @@ __device__ __forceinline__ bool grid_barrier(int* counter, int target, int* stat
       }
       __nanosleep(32);
     }
-    __threadfence();
   }
-  return __syncthreads_or(failed) == 0;
+  return __syncthreads_or(failed) == 0;   // the acquire above, then this barrier: every thread sees the other blocks' writes
 }
 
 template <int DH, bool F16>
