@@ -553,14 +553,22 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
   const bool sk_fold = !s->modulation && T <= 16;
   const bool sk_fold_mlp = sk_fold && skinny(q_dim, d, kGemmResid);
   const bool sk_fold_attn = sk_fold && skinny(F, d, kGemmResid);
-  auto sk_fold_out = [&](SkinnyParams& k, const void* gain) {
+  // (a weight-streaming GEMM behind the norm adds the rows' partial sums itself; a tiled one reads r, which the
+  // producer's last block then has to finalise)
+  auto sk_fold_out = [&](SkinnyParams& k, const void* gain, bool consumer_is_skinny) {
     k.norm_gain = static_cast<const __nv_bfloat16*>(gain);
     k.norm_h = h;
     k.norm_h_f16 = f16;
     k.row_ss = reinterpret_cast<float*>(s->ws_dev + s->ws.row_ss);
     k.ss_stride = d / 32;
-    k.row_rs = reinterpret_cast<float*>(s->ws_dev + s->ws.row_rs);
-    k.units_done = reinterpret_cast<int*>(s->ws_dev + s->ws.row_done);
+    if (!consumer_is_skinny) {
+      k.row_rs = reinterpret_cast<float*>(s->ws_dev + s->ws.row_rs);
+      k.units_done = reinterpret_cast<int*>(s->ws_dev + s->ws.row_done);
+    }
+    k.norm_eps = c.rms_eps;
+  };
+  auto sk_fold_in = [&](SkinnyParams& k) {
+    k.in_row_ss = reinterpret_cast<const float*>(s->ws_dev + s->ws.row_ss);
     k.norm_eps = c.rms_eps;
   };
   float* row_ss = reinterpret_cast<float*>(s->ws_dev + s->ws.row_ss);
@@ -719,7 +727,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
       k.tok_pos = g.tok_pos; k.tok_slot = g.tok_slot; k.rope = g.rope;
       for (int i = 0; i < 3; ++i) k.qkv_bias[i] = g.qkv_bias[i];
       k.smid_log = slots(1);
-      k.in_row_rs = g.in_row_rs;
+      if (sk_fold_attn && l > 0) sk_fold_in(k);
+      else k.in_row_rs = g.in_row_rs;
       LaunchTimer t(s, 1, stream); where = "qkv gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
     } else { LaunchTimer t(s, 1, stream); where = "qkv gemm"; e = launch_gemm(g, sm_budget, stream); }
     if (e != cudaSuccess) break;
@@ -769,7 +778,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
       k.w[0] = wo.w_o; k.y = x; k.accumulate = 1;
       k.gate_mod = go.gate_mod; k.tok_seq = go.tok_seq; k.gate_which = 2;
       k.smid_log = slots(5);
-      if (sk_fold_mlp) sk_fold_out(k, w.g_mlp);
+      if (sk_fold_mlp) sk_fold_out(k, w.g_mlp, skinny(d, F, kGemmGateUp));
       LaunchTimer t(s, 5, stream); where = "out-proj gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
     } else { LaunchTimer t(s, 5, stream); where = "out-proj gemm"; e = launch_gemm(go, sm_budget, stream); }
     if (e != cudaSuccess) break;
@@ -799,7 +808,8 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
       k.w[0] = wo.w_gate; k.w[1] = wo.w_up;
       k.act = reinterpret_cast<__nv_bfloat16*>(s->ws_dev + s->ws.act); k.act_f16 = f16;
       k.smid_log = slots(6);
-      k.in_row_rs = gu.in_row_rs;
+      if (sk_fold_mlp) sk_fold_in(k);
+      else k.in_row_rs = gu.in_row_rs;
       LaunchTimer t(s, 6, stream); where = "gate/up gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
     } else { LaunchTimer t(s, 6, stream); where = "gate/up gemm"; e = launch_gemm(gu, sm_budget, stream); }
     if (e != cudaSuccess) break;
@@ -827,7 +837,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
       k.w[0] = wo.w_down; k.y = x; k.accumulate = 1;
       k.gate_mod = gd.gate_mod; k.tok_seq = gd.tok_seq; k.gate_which = 5;
       k.smid_log = slots(7);
-      if (sk_fold_attn && l + 1 < c.n_layers) sk_fold_out(k, s->layers[l + 1].g_attn);
+      if (sk_fold_attn && l + 1 < c.n_layers) sk_fold_out(k, s->layers[l + 1].g_attn, skinny(d, q_dim + 2 * kv_dim, kGemmQkv));
       LaunchTimer t(s, 7, stream); where = "down gemm"; e = launch_gemm_skinny(k, sm_budget, stream);
     } else { LaunchTimer t(s, 7, stream); where = "down gemm"; e = launch_gemm(gd, sm_budget, stream); }
     if (e != cudaSuccess) break;

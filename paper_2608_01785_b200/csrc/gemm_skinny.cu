@@ -88,6 +88,19 @@ __device__ __forceinline__ const uint8_t* unit_row(const SkinnyParams& p, int un
 // MT: 16-row tiles of activations (T <= 16 MT); DB: depth of a warp's ring of K steps.
 // FOLD: the instantiation that knows the folded RMSNorm (producing side in Resid mode, consuming side in the others);
 // the plain one carries none of its code.
+// r = rsqrt(mean(x^2) + eps) of row `row` from its n partial sums of squares (one per 32 columns): the four threads
+// of a row (threadIdx & 3) add every fourth partial each and then combine, a fixed order whoever calls.  Called by all
+// threads of a warp.
+__device__ __forceinline__ float row_norm_factor(const float* row_ss, int stride, int n, int row, int T, int width, float eps) {
+  const int q = threadIdx.x & 3;
+  float sum = 0.f;
+  if (row < T)
+    for (int i = q; i < n; i += 4) sum += __ldcg(row_ss + size_t(row) * stride + i);
+  sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+  sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+  return rsqrtf(sum / float(width) + eps);
+}
+
 // The body is a device function shared by the kernel of its own and by the one-launch small step: the calling
 // thread block (SK_THREADS threads) is number `block` of `n_blocks` working on the launch's units; `wait` is called
 // once by every thread, after the weights of the first steps have been requested, and must return when the
@@ -178,6 +191,7 @@ __device__ __forceinline__ void gemm_skinny_body(const SkinnyParams& p, uint8_t*
   // folded RMSNorm, consuming side: r of this thread's epilogue row, on its way while the first unit streams
   float rs_in = 1.f;
   if (FOLD && p.in_row_rs != nullptr && int(threadIdx.x >> 2) < p.T) rs_in = __ldcg(p.in_row_rs + (threadIdx.x >> 2));
+  if (FOLD && p.in_row_ss != nullptr) rs_in = row_norm_factor(p.in_row_ss, p.K >> 5, p.K >> 5, int(threadIdx.x >> 2), p.T, p.K, p.norm_eps);
   int* last_unit = reinterpret_cast<int*>(part_all + SK_WARPS * PART_PITCH);   // FOLD: one word behind the partial tiles
 
   for (; unit < units; unit += n_blocks) {
@@ -270,7 +284,7 @@ __device__ __forceinline__ void gemm_skinny_body(const SkinnyParams& p, uint8_t*
         lo.x += l.x; lo.y += l.y; lo.z += l.z; lo.w += l.w;
         hi.x += h.x; hi.y += h.y; hi.z += h.z; hi.w += h.w;
       }
-      if (FOLD && p.in_row_rs != nullptr) {
+      if (FOLD && (p.in_row_rs != nullptr || p.in_row_ss != nullptr)) {
         lo.x *= rs_in; lo.y *= rs_in; lo.z *= rs_in; lo.w *= rs_in;
         hi.x *= rs_in; hi.y *= rs_in; hi.z *= rs_in; hi.w *= rs_in;
       }
@@ -361,9 +375,9 @@ __device__ __forceinline__ void gemm_skinny_body(const SkinnyParams& p, uint8_t*
       }
     }
     __syncthreads();                                         // the partial tiles are free again
-    if (FOLD && p.mode == kGemmResid && p.norm_gain != nullptr) {
-      // the block that delivers the last unit turns the partial sums into every row's r: four threads per row add
-      // the units' partials in a fixed order.  (The barrier above orders the block's stores before thread 0's fence.)
+    if (FOLD && p.mode == kGemmResid && p.norm_gain != nullptr && p.units_done != nullptr) {
+      // the block that delivers the last unit turns the partial sums into every row's r (for a tiled GEMM behind the
+      // norm).  (The barrier above orders the block's stores before thread 0's fence.)
       if (threadIdx.x == 0) {
         __threadfence();
         *last_unit = atomicAdd(p.units_done, 1) == units - 1;
@@ -371,13 +385,8 @@ __device__ __forceinline__ void gemm_skinny_body(const SkinnyParams& p, uint8_t*
       __syncthreads();
       if (*last_unit) {
         __threadfence();
-        const int q = threadIdx.x & 3;
-        float sum = 0.f;
-        if (row < p.T)
-          for (int i = q; i < units; i += 4) sum += __ldcg(p.row_ss + size_t(row) * p.ss_stride + i);
-        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-        if (q == 0 && row < p.T) p.row_rs[row] = rsqrtf(sum / float(p.N) + p.norm_eps);
+        const float r = row_norm_factor(p.row_ss, p.ss_stride, units, row, p.T, p.N, p.norm_eps);
+        if ((threadIdx.x & 3) == 0 && row < p.T) p.row_rs[row] = r;
         if (threadIdx.x == 0) *p.units_done = 0;             // ready for the next launch
       }
     }
@@ -410,7 +419,7 @@ static_assert(skinny_smem<1, DB1>() <= 227 * 1024 && skinny_smem<2, DB2>() <= 22
 template <int MT, int DB>
 cudaError_t launch_one(const SkinnyParams& p, int grid, cudaStream_t stream) {
   constexpr int smem = skinny_smem<MT, DB>() < kMinSmemBytes ? kMinSmemBytes : skinny_smem<MT, DB>();
-  const bool fold = p.norm_gain != nullptr || p.in_row_rs != nullptr;
+  const bool fold = p.norm_gain != nullptr || p.in_row_rs != nullptr || p.in_row_ss != nullptr;
   if (p.ab_f16) {
     if (fold) return launch_step_kernel(gemm_skinny_kernel<MT, DB, true, true>, grid, SK_THREADS, smem, stream, p.overlap != 0, p);
     return launch_step_kernel(gemm_skinny_kernel<MT, DB, true, false>, grid, SK_THREADS, smem, stream, p.overlap != 0, p);
@@ -487,7 +496,7 @@ __global__ void __launch_bounds__(SK_THREADS, 1) small_step_kernel(const __grid_
   };
   auto fold_out = [&](SkinnyParams& k, const __nv_bfloat16* gain) {
     k.norm_gain = gain; k.norm_h = p.h; k.norm_h_f16 = F16 ? 1 : 0;
-    k.row_ss = p.row_ss; k.ss_stride = p.d >> 5; k.row_rs = p.row_rs; k.units_done = p.units_done; k.norm_eps = p.eps;
+    k.row_ss = p.row_ss; k.ss_stride = p.d >> 5; k.norm_eps = p.eps;     // the consuming GEMM adds the partials itself
   };
   for (int l = 0; l < p.n_layers && !dead; ++l) {
     const SmallLayer L = p.layers[l];
@@ -500,7 +509,7 @@ __global__ void __launch_bounds__(SK_THREADS, 1) small_step_kernel(const __grid_
       k.v_cache = p.kv_pool + (size_t(l) * 2 + 1) * p.layer_kv_elems;
       k.tok_pos = p.tok_pos; k.tok_slot = p.tok_slot; k.rope = p.rope;
       for (int i = 0; i < 3; ++i) k.qkv_bias[i] = L.bias[i];
-      if (l > 0) k.in_row_rs = p.row_rs;
+      if (l > 0) { k.in_row_ss = p.row_ss; k.norm_eps = p.eps; }
       auto w = [&] { if (l > 0) barrier(); };
       if (block < nb_qkv) gemm_skinny_body<1, DB1, F16, true>(k, smem, block, nb_qkv, w);
       else w();
@@ -531,7 +540,7 @@ __global__ void __launch_bounds__(SK_THREADS, 1) small_step_kernel(const __grid_
       SkinnyParams k = base(p.h, p.d, p.F, kGemmGateUp);
       k.w[0] = L.w_gate; k.w[1] = L.w_up;
       k.act = p.act; k.act_f16 = F16 ? 1 : 0;
-      k.in_row_rs = p.row_rs;
+      k.in_row_ss = p.row_ss; k.norm_eps = p.eps;
       auto w = [&] { barrier(); };
       if (block < nb_gu) gemm_skinny_body<1, DB1, F16, true>(k, smem, block, nb_gu, w);
       else w();

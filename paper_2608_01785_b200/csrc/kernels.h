@@ -114,9 +114,10 @@ struct SkinnyParams {
   int* smid_log;
   // RMSNorm folded into the GEMMs around it, as in GemmParams (rmsnorm(x) W^T = diag(r) ((x o g) W^T)).
   //   Resid, producing side (norm_gain non-null): the epilogue also emits h = 16-bit(y o g) for the next GEMM and the
-  //   sum of y^2 over the unit's 32 columns into row_ss[row * ss_stride + unit]; the block that delivers the last unit
-  //   (units_done: one counter, zero at entry and at exit) sums every row's partials in a fixed order and writes
-  //   r = rsqrt(mean(y^2) + norm_eps) into row_rs[row].
+  //   sum of y^2 over the unit's 32 columns into row_ss[row * ss_stride + unit].  When the GEMM behind the norm is the
+  //   tiled kernel (units_done non-null), the block that delivers the last unit (units_done: one counter, zero at entry
+  //   and at exit) sums every row's partials and writes r = rsqrt(mean(y^2) + norm_eps) into row_rs[row]; when it is
+  //   this kernel, that GEMM sums the partials itself (in_row_ss) and the producer's tail stays short.
   const __nv_bfloat16* norm_gain;   // [N]
   __nv_bfloat16* norm_h;     // 16-bit [T, N]
   int norm_h_f16;
@@ -124,10 +125,12 @@ struct SkinnyParams {
   int ss_stride;
   float* row_rs;             // [T]
   int* units_done;
-  float norm_eps;
-  //   Qkv / GateUp, consuming side (in_row_rs non-null): every output row is scaled by r of its token before bias /
-  //   RoPE / SiLU.
+  float norm_eps;            // both sides
+  //   Qkv / GateUp, consuming side: every output row is scaled by r of its token before bias / RoPE / SiLU; r comes
+  //   from in_row_rs[row], or (in_row_ss non-null) from the K / 32 partials in_row_ss[row * (K / 32) + i], which four
+  //   threads per row add in the order the producer's last block would have.
   const float* in_row_rs;    // [T]
+  const float* in_row_ss;    // [T][K / 32]
 };
 // True when the skinny kernel covers this shape (few rows, K a multiple of 32, widths it can tile).
 bool gemm_skinny_supports(int T, int K, int N, int mode, int head_dim);
