@@ -191,7 +191,12 @@ hs_status_t hs_stage_plan(hs_stage_t *stage, const hs_batch_t *batch, int32_t *t
  * the same step rewrites the same slots with the same values.  The caller advances ctx_len itself.
  * With sm_budget < the device's SM count every kernel of the step starts only after the previous one has
  * ended, so that no block of the step ever sits on an SM outside the budget; with sm_budget == SM count
- * (no co-running neighbour) each kernel's set-up overlaps the previous kernel's drain.
+ * (no co-running neighbour) each kernel's set-up overlaps the previous kernel's drain.  A decode-only step of at
+ * most 16 rows under a partial budget runs, after its first RMSNorm, as one cooperative launch of at most sm_budget
+ * blocks whose phases are the same kernels' bodies separated by bounded grid-wide barriers (same results; the
+ * separate launches are used instead where the device refuses a cooperative launch).  With both prefill and decode
+ * work in a step the two attention kernels of a layer run side by side on two shares of the budget, the decode
+ * kernel on a stream of the stage's own that is forked from and joined to cuda_stream by events.
  * Errors (nothing launched): INVALID_ARG, INVALID_BUDGET, BAD_BLOCK_TABLE, NO_DEVICE, CUDA.
  */
 hs_status_t hs_stage_step(hs_stage_t *stage, const hs_batch_t *batch, int32_t sm_budget, void *cuda_stream);
