@@ -684,8 +684,6 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
       sp.rope = reinterpret_cast<const float2*>(s->ws_dev + s->ws.rope);
       sp.counters = meta + s->ml.counters;
       sp.row_ss = reinterpret_cast<float*>(s->ws_dev + s->ws.row_ss);
-      sp.row_rs = reinterpret_cast<float*>(s->ws_dev + s->ws.row_rs);
-      sp.units_done = reinterpret_cast<int*>(s->ws_dev + s->ws.row_done);
       sp.eps = c.rms_eps;
       sp.grid_bar = meta + s->ml.grid_bar;
       sp.status = status;

@@ -203,7 +203,7 @@ struct Unit { int tile, kb_begin, kb_end, seg, last, half; };
 //                     256-row tiles, each unit twice -- once per 128-row half (`half`) -- so that every output
 //                     element still receives the same partial sums in the same order.
 struct UnitWalk {
-  int stream_k, n_tiles, k_blocks, ksplit, kb_per, n_workers, n_slots;
+  int stream_k, n_tiles, k_blocks, ksplit, n_workers, n_slots;
   int halves, n_m_tiles, M;  // halves = 2: a single block standing in for a pair
   int cur;                 // unit (plain) or slot (stream-K) being handed out
   int idx, n_seg, first_tile;
@@ -216,7 +216,6 @@ struct UnitWalk {
     M = p.M;
     n_tiles = n_tiles_; k_blocks = k_blocks_; n_workers = n_workers_;
     ksplit = !pair && p.mode == kGemmResid && p.ksplit > 1 ? p.ksplit : 1;
-    kb_per = (k_blocks + ksplit - 1) / ksplit;
     n_slots = stream_k ? p.stream_k_slots : n_tiles * ksplit;
     cur = worker - n_workers;
     idx = n_seg = 0; first_tile = 0; lo = hi = 0;
@@ -234,8 +233,8 @@ struct UnitWalk {
       if (cur >= n_slots) return false;
       const int ks = cur / n_tiles;
       u.tile = cur - ks * n_tiles;
-      u.kb_begin = ks * kb_per;
-      u.kb_end = min(k_blocks, u.kb_begin + kb_per);
+      u.kb_begin = gemm_split_begin(k_blocks, ksplit, ks);
+      u.kb_end = gemm_split_begin(k_blocks, ksplit, ks + 1);
       u.seg = ks;
       u.last = ks == ksplit - 1;
       return true;
@@ -857,27 +856,25 @@ int gemm_pick_bn(int M, int N, int sm_count) {
 
 int gemm_pick_ksplit(int M, int N, int K, int bn, int sm_count) {
   // Few tiles (small M): split K so that more SMs stream a share of the weights.  The splits of a tile add
-  // their partial sums in split order, one after the other, so every further split shortens the streaming
-  // but lengthens that chain.  Measured on B200 at 64 rows (bn = 128): a block streams a 64-wide K block in
-  // about 0.36 us, a link of the chain costs about 3.5 us.  The split count minimises
-  //   waves * ceil(k_blocks / ks) * 0.36 us + (ks - 1) * 3.5 us        over ks = 1 .. 8
-  // (3584 x 3584 at 64 rows: 2 splits, 23 us instead of 27 with 5; 3584 x 18944: 5 splits).  Depends on the
-  // shape and the device only, never on the SM budget.
+  // their partial sums in split order, one after the other.  Measured on B200 at 64 rows (bn = 128): a block streams
+  // a 64-wide K block in about 0.36 us, a link of the chain costs about 3.5 us -- the time of ten K blocks, which is
+  // how much longer each split is than the one before it (gemm_split_begin), so that only the last link is exposed.
+  // The split count minimises gemm_ksplit_cost_us over ks = 1 .. 8.  Depends on the shape and the device only, never
+  // on the SM budget.
   const int tiles = ((M + BM - 1) / BM) * ((N + bn - 1) / bn);
   const int k_blocks = (K + BK - 1) / BK;
   int best = 1;
   double best_cost = 1e30;
   for (int ks = 1; ks <= 8 && ks <= k_blocks; ++ks) {
-    const int per = (k_blocks + ks - 1) / ks;
+    if (gemm_split_begin(k_blocks, ks, ks - 1) >= k_blocks) continue;      // an empty last split
     const int waves = (tiles * ks + sm_count - 1) / sm_count;
-    const double cost = double(waves) * per * 0.36 + (ks - 1) * 3.5;
+    const double cost = gemm_ksplit_cost_us(k_blocks, ks, waves);
     if (cost < best_cost - 1e-9) {
       best_cost = cost;
       best = ks;
     }
   }
-  const int per = (k_blocks + best - 1) / best;
-  return (k_blocks + per - 1) / per;          // no empty split
+  return best;
 }
 
 int gemm_pick_stream_k(int M, int N, int K, int sm_count) {

@@ -605,7 +605,7 @@ bool gemm_skinny_wins(int T, int K, int N, int mode, int head_dim, int sm_count)
   if (mode == kGemmResid) {
     const int bn = gemm_pick_bn(T, N, sm_count), ks = gemm_pick_ksplit(T, N, K, bn, sm_count);
     const int tiles = (N + bn - 1) / bn, waves = (tiles * ks + sm_count - 1) / sm_count;
-    tiled = double(waves) * ((k_blocks + ks - 1) / ks) * 0.36 + (ks - 1) * 3.5;
+    tiled = gemm_ksplit_cost_us(k_blocks, ks, waves);
   } else {
     const int tiles = (N + 127) / 128, waves = (tiles + sm_count - 1) / sm_count;
     tiled = double(waves) * k_blocks * (mode == kGemmGateUp ? 0.8 : 0.36);

@@ -85,6 +85,27 @@ cudaError_t gemm_set_attributes();
 // Tile width for a Resid-mode GEMM of this shape on a device with sm_count SMs (budget independent).
 int gemm_pick_bn(int M, int N, int sm_count);
 int gemm_pick_ksplit(int M, int N, int K, int bn, int sm_count);
+// Where split i (0 .. ks) of a tile's k_blocks begins.  The splits add their sums one after the other, a link of that
+// chain costing about as long as kSplitSkew K blocks take to stream; so each split is that much longer than the one
+// before it and finishes just when its turn comes, instead of all finishing together and then queueing.  Equal
+// lengths when K is too short for that.  A function of the shape only.
+constexpr int kSplitSkew = 10;
+__host__ __device__ inline int gemm_split_begin(int k_blocks, int ks, int i) {
+  if (i >= ks) return k_blocks;
+  const int tri = kSplitSkew * ks * (ks - 1) / 2;
+  if (ks < 2 || k_blocks < tri + ks * kSplitSkew) {
+    const int per = (k_blocks + ks - 1) / ks;
+    return i * per < k_blocks ? i * per : k_blocks;
+  }
+  return i * ((k_blocks - tri) / ks) + kSplitSkew * i * (i - 1) / 2;
+}
+// Modelled time (us) of a K-split residual GEMM of `waves` rounds on single blocks: the longest split's stream and
+// what of the chain of adds is not hidden behind it.
+inline double gemm_ksplit_cost_us(int k_blocks, int ks, int waves) {
+  const int last = k_blocks - gemm_split_begin(k_blocks, ks, ks - 1);
+  const bool skewed = gemm_split_begin(k_blocks, ks, 1) != (k_blocks + ks - 1) / ks || ks == 1;
+  return double(waves) * last * 0.36 + (ks > 1 ? (skewed ? 3.5 : (ks - 1) * 3.5) : 0.0);
+}
 // Runs for the stream-K form of a Resid-mode GEMM on pairs (one per pair of the device), or 0 when whole tiles
 // already fill their waves well enough (budget independent).
 int gemm_pick_stream_k(int M, int N, int K, int sm_count);
@@ -239,7 +260,7 @@ struct SmallStepParams {
   __nv_bfloat16* kv_pool; size_t layer_kv_elems;
   const int32_t* tok_pos; const int32_t* tok_slot; const float2* rope;
   int* counters;                   // [n_layers * 2] queue heads, zero at entry
-  float* row_ss; float* row_rs; int* units_done; float eps;
+  float* row_ss; float eps;        // partial sums of squares of the folded norms [T][d / 32]; eps of the norms
   int* grid_bar;                   // one word, zero at entry: blocks arrived at the grid barriers so far
   int* status; int* smid_log;
 };
