@@ -11,7 +11,7 @@ namespace hs {
 
 constexpr int kPage = HS_PAGE_SIZE;      // tokens per KV page
 constexpr int kDecodeSplit = 256;        // run length that sizes the decode item buffers (the planner may pick 128 when the items still fit)
-constexpr int kDecodeWarps = 6;            // warps per block of the decode attention kernel (kernels.h: kDecodeKernelWarps)
+constexpr int kDecodeWarps = 8;            // warps per block of the decode attention kernel (kernels.h: kDecodeKernelWarps)
 constexpr int kDecodeSplitMax = 512;     // largest number of keys per item the planner may choose
 constexpr int kDecodeTail = 128;         // keys per piece of a sequence's last, incomplete run (the items that end the kernel)
 static_assert(kDecodeSplit % 16 == 0 && kDecodeSplitMax / 16 <= 32, "the decode kernel keeps one page id per lane");

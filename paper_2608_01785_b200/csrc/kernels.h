@@ -14,7 +14,7 @@ namespace hs {
 constexpr int kMinSmemBytes = 117 * 1024;
 // Warps per block of the decode attention kernel (each works through one item at a time); the planner sizes its
 // work items for sm_count x this many warps.
-constexpr int kDecodeKernelWarps = 6;
+constexpr int kDecodeKernelWarps = 8;
 
 // ------------------------------------------------------------------ GEMM --
 // out = A[M,K] * W^T with W given as up to three row blocks [rows, K] (bf16, K contiguous).  The output
