@@ -106,16 +106,17 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, u
       : "memory");
 }
 
-__device__ __forceinline__ ItemView view_item(const AttnParams& p, int item, int Mt) {
-  const int4 it = reinterpret_cast<const int4*>(p.prefill_items)[item];
+// An item's geometry from its 32-byte record {seq, kv head, first token, tokens} {cached tokens of the sequence, token
+// row of the sequence's first new token, new tokens of the sequence, -}.
+__device__ __forceinline__ ItemView view_item(const AttnParams& p, const int4& it, const int4& sq, int Mt) {
   ItemView v;
   v.seq = it.x; v.hk = it.y; v.tok_begin = it.z; v.n_tok = it.w;
-  v.ctx = p.seq_ctx[v.seq];
-  v.tok0 = p.seq_tok0[v.seq] + v.tok_begin;
+  v.ctx = sq.x;
+  v.tok0 = sq.y + v.tok_begin;
   v.pos0 = v.ctx + v.tok_begin;
   v.n_tok_t[0] = min(v.n_tok, Mt);
   v.n_tok_t[1] = v.n_tok - v.n_tok_t[0];
-  const int all = v.ctx + p.seq_qlen[v.seq];
+  const int all = v.ctx + sq.z;
   v.n_keys = p.bidirectional ? all : v.pos0 + v.n_tok;
   const int keys_a = p.bidirectional ? all : v.pos0 + v.n_tok_t[0];
   v.nblk_t[0] = (keys_a + PF_KEYS - 1) / PF_KEYS;
@@ -189,6 +190,20 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
     // chunk, requested a chunk ahead), so that no round trip to the block table stands in front of a page request.
     const int pi = warp == 8 ? 0 : warp - 10;           // producer index 0..3
     const int kv = pi >> 1, w0 = (pi & 1) * 2;          // K or V; first of its two pages in a block
+    // The lead producer's lane 0 asks the work queue for the next item while it still has a few key blocks of the
+    // current one to request, and for that item's record two blocks later -- so that neither the atomic nor the
+    // record's round trip stands between two items (with items of one key block those two and the sequence's fields,
+    // now part of the record, were most of an item's time).  Asking earlier -- at the item's start -- would hand the
+    // items out before anybody knows which blocks finish early.  A block's first item is its index in the grid.
+    int q_next = int(blockIdx.x);                                   // lane 0 of the lead: the next item's queue index
+    int4 rec_a = make_int4(0, 0, 0, 0), rec_b = rec_a;              // ... and its record
+    auto fetch_record = [&](int idx) {
+      if (idx < p.n_prefill_items) {
+        rec_a = __ldg(reinterpret_cast<const int4*>(p.prefill_items) + 2 * idx);
+        rec_b = __ldg(reinterpret_cast<const int4*>(p.prefill_items) + 2 * idx + 1);
+      }
+    };
+    if (pi == 0 && lane == 0) fetch_record(q_next);
     for (;;) {
       int item = 0;
       bool ok = true;
@@ -196,17 +211,19 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
       if (pi == 0) {
         if (lane == 0) {
           ok = mbar_wait(&bar->ring_empty[rs], rph ^ 1, abort_flag, p.status);
-          if (ok) item = atomicAdd(p.counters, 1);
+          if (ok) {
+            item = q_next;
+            if (item < p.n_prefill_items) v = view_item(p, rec_a, rec_b, Mt);
+            bar->ring_item[rs] = item;
+            bar->ring_view[rs] = v;
+            mbar_arrive(&bar->ring_full[rs]);
+          }
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
-        item = __shfl_sync(0xffffffffu, item, 0);
-        if (item < p.n_prefill_items) v = view_item(p, item, Mt);
-        if (lane == 0) {
-          bar->ring_item[rs] = item;
-          bar->ring_view[rs] = v;
-          mbar_arrive(&bar->ring_full[rs]);
-        }
+        __syncwarp();
+        item = bar->ring_item[rs];
+        v = bar->ring_view[rs];
       } else {
         ok = mbar_wait(&bar->ring_full[rs], rph, abort_flag, p.status);
         if (!__all_sync(0xffffffffu, ok)) break;
@@ -220,22 +237,30 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
       const int32_t* table = p.block_tables + size_t(v.seq) * p.max_pages_per_seq;
       const int n_pages = (v.n_keys + 15) >> 4;
       int pg_next = lane < n_pages ? table[lane] : 0, pg_cur = 0;
-      if (pi == 0 && lane == 0) {
-        // Q tiles: one box of Mt token rows x 64 columns per (tile, head, half)
-        ok = mbar_wait(&bar->q_empty, (n_items_seen & 1) ^ 1, abort_flag, p.status);
+      {
+        // Q tiles: one box of Mt token rows x 64 columns per (tile, head, half) -- up to 32 copies per item, which one
+        // thread would need microseconds to issue.  The four producers take every fourth copy each, one lane per copy.
+        if (lane == 0) ok = mbar_wait(&bar->q_empty, (n_items_seen & 1) ^ 1, abort_flag, p.status);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
         if (ok) {
           const int n_tiles = v.n_tok_t[1] > 0 ? 2 : 1;
-          mbar_expect_tx(&bar->q_full, n_tiles * G * G_::HALVES * Mt * 128);
-          for (int t = 0; t < n_tiles; ++t)
-            for (int g = 0; g < G; ++g)
-              for (int h = 0; h < G_::HALVES; ++h)
-                tma_load_2d(q_smem + t * G_::Q_BYTES + h * 16384 + g * Mt * 128, &p.tm_q, &bar->q_full,
-                            (v.hk * G + g) * DH + h * 64, v.tok0 + t * Mt);
+          const int n_copies = n_tiles * G * G_::HALVES;
+          if (pi == 0 && lane == 0) mbar_expect_tx(&bar->q_full, n_copies * Mt * 128);
+          const int cidx = pi + 4 * lane;                    // copy of this lane: (tile, head, half), half fastest
+          if (cidx < n_copies) {
+            const int h = cidx % G_::HALVES, g = (cidx / G_::HALVES) % G, t = cidx / (G_::HALVES * G);
+            tma_load_2d(q_smem + t * G_::Q_BYTES + h * 16384 + g * Mt * 128, &p.tm_q, &bar->q_full,
+                        (v.hk * G + g) * DH + h * 64, v.tok0 + t * Mt);
+          }
         }
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
       ++n_items_seen;
       for (int kb = 0; kb < v.nblk && ok; ++kb) {
+        if (pi == 0 && lane == 0) {
+          if (kb == max(0, v.nblk - 4)) q_next = int(gridDim.x) + atomicAdd(p.counters, 1);
+          if (kb == v.nblk - 2 && v.nblk > 2) fetch_record(q_next);
+        }
         if ((kb & 7) == 0) {
           pg_cur = pg_next;
           const int idx = (kb + 8) * 4 + lane;
@@ -266,6 +291,7 @@ __global__ void __launch_bounds__(PF_THREADS, 1) attn_prefill_kernel(const __gri
         }
       }
       if (!ok) break;
+      if (pi == 0 && lane == 0 && v.nblk <= 2) fetch_record(q_next);   // (a short item: not before its own requests are out)
       blk_base += v.nblk;
     }
   } else if (warp == 9 || warp == 10) {

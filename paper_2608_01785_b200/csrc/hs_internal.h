@@ -51,7 +51,8 @@ struct MetaLayout {
   int tok_pos, tok_slot, tok_seq;    // [max_tokens]      absolute position / cache slot / sequence index of each new token
   int seq_tok0, seq_ctx, seq_qlen;   // [max_seqs]        first token row, cached tokens, new tokens
   int block_tables;                  // [max_seqs * max_pages_per_seq]
-  int prefill_items;                 // [max_prefill_items * 4]  {seq, kv_head, first token, tokens (at most two tiles)}
+  int prefill_items;                 // [max_prefill_items * 8]  {seq, kv_head, first token, tokens (at most two tiles),
+                                     //                           cached tokens, first token row and new tokens of the sequence, 0}
   int decode_items;                  // [max_decode_items * 8]   {decode row, kv_head, first key, end key,
                                      //                           seq, token row, first partial slot of the group,
                                      //                           splits | index within the group << 16}

@@ -222,7 +222,8 @@ struct AttnParams {
   const int32_t* seq_qlen;   // new tokens per sequence (prefill kernel, bidirectional only)
   int bidirectional;         // prefill kernel: 1 = no causal mask, a row sees every key of its sequence
   const int32_t* block_tables;
-  const int32_t* prefill_items;    // int4 per item
+  const int32_t* prefill_items;    // two int4 per item: {seq, kv head, first token, tokens} {cached tokens, first token
+                                   //                    row and new tokens of the sequence, 0}
   int n_prefill_items;
   const int32_t* decode_items;     // two int4 per item: {decode row, kv head, first key, end key}
                                    //                    {seq, token row, first item of its group, splits}

@@ -78,7 +78,7 @@ MetaLayout make_meta_layout(const hs_stage_config_t& c) {
   m.seq_ctx = take(c.max_seqs);
   m.seq_qlen = take(c.max_seqs);
   m.block_tables = take(c.max_seqs * c.max_pages_per_seq);
-  m.prefill_items = take(m.max_prefill_items * 4);
+  m.prefill_items = take(m.max_prefill_items * 8);
   m.decode_items = take(m.max_decode_items * 8);
   m.decode_rows = take(c.max_seqs * 4);
   m.counters = take(c.n_layers * 2);
@@ -159,7 +159,7 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
   p.n_tokens = b.n_tokens;
   p.n_seqs = b.n_seqs;
 
-  struct Item { int32_t v[4]; int32_t cost; };
+  struct Item { int32_t v[8]; int32_t cost; };
   std::vector<Item> pre;
   struct DecItem { int32_t v[8]; int32_t keys; };
   std::vector<DecItem> dec;
@@ -209,7 +209,7 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
       for (int t0 = 0; t0 < n; t0 += 2 * Mt)
         for (int hk = 0; hk < c.n_kv_heads; ++hk) {
           const int nt = std::min(2 * Mt, n - t0);
-          pre.push_back(Item{{s, hk, t0, nt}, ctx + t0 + nt});
+          pre.push_back(Item{{s, hk, t0, nt, ctx, t, n, 0}, ctx + t0 + nt});
           const int keys_item = (c.flags & HS_FLAG_BIDIRECTIONAL) ? ctx + n : ctx + t0 + nt;
           const int blocks = ceil_div(keys_item, 64);
           p.prefill_blocks += blocks;
@@ -227,7 +227,7 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
     for (size_t i = 0; i < dec.size(); ++i)
       for (int k = 0; k < 8; ++k) meta[ml.decode_items + int(i) * 8 + k] = dec[i].v[k];
     for (size_t i = 0; i < pre.size(); ++i)
-      for (int k = 0; k < 4; ++k) meta[ml.prefill_items + int(i) * 4 + k] = pre[i].v[k];
+      for (int k = 0; k < 8; ++k) meta[ml.prefill_items + int(i) * 8 + k] = pre[i].v[k];
     for (int i = 0; i < c.n_layers * 2; ++i) meta[ml.counters + i] = 0;
     for (int i = 0; i < c.max_seqs * c.n_kv_heads; ++i) meta[ml.group_done + i] = 0;
     for (int i = 0; i < 4; ++i) meta[ml.grid_bar + i] = 0;
