@@ -627,6 +627,7 @@ hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget,
     a.n_prefill_items = plan.n_prefill_items;
     a.decode_items = meta + s->ml.decode_items;
     a.n_decode_items = plan.n_decode_items;
+    a.decode_group = plan.decode_group;
     a.decode_rows = meta + s->ml.decode_rows;
     a.n_decode_rows = plan.n_decode_rows;
     a.part_o = reinterpret_cast<float*>(s->ws_dev + s->ws.part_o);

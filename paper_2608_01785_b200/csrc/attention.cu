@@ -33,7 +33,8 @@ cudaError_t attention_set_attributes() {
 
 cudaError_t launch_attention_decode(const AttnParams& p, int sm_budget, cudaStream_t stream) {
   if (p.n_decode_items <= 0) return cudaSuccess;
-  const int grid = p.n_decode_items < sm_budget ? p.n_decode_items : sm_budget;
+  const int work = p.decode_group ? p.n_decode_items / DC_WARPS : p.n_decode_items;     // groups, or items
+  const int grid = work < sm_budget ? work : sm_budget;
   if (p.head_dim == 128)
     return launch_step_kernel(attn_decode_kernel<128>, grid, DC_THREADS, dc_smem_bytes<128>(), stream, p.overlap != 0, p);
   else

@@ -235,13 +235,22 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams& p, int layer,
   }
   wait();
 
+  // Group mode (p.decode_group, a batch whose items would not fill the device's warps): item 8 g + w is the w-th
+  // eighth of the pages of group g = (sequence, KV head); a block takes whole groups -- g = block, block + n_blocks,
+  // ... -- its eight warps one slice each, and their partial results meet in the block's shared memory instead of in
+  // global memory behind a counter.  Every warp of the block goes through the same barriers whatever happens to it.
+  const bool group_mode = p.decode_group != 0;
   bool first_round = true;
-  for (;;) {
+  for (int round = 0;; ++round) {
     if (!first_round) {
-      if (lane == 0) item = n_blocks * DC_WARPS + atomicAdd(counters + 1, 1);
-      item = __shfl_sync(0xffffffffu, item, 0);
+      if (group_mode) {
+        item = worker ? (block + round * n_blocks) * DC_WARPS + warp : p.n_decode_items;
+      } else {
+        if (lane == 0) item = n_blocks * DC_WARPS + atomicAdd(counters + 1, 1);
+        item = __shfl_sync(0xffffffffu, item, 0);
+      }
     }
-    if (item >= p.n_decode_items || *abort_flag) break;
+    if (item >= p.n_decode_items || (!group_mode && *abort_flag)) break;
     // one 32-byte record: {decode row, kv head, first key, end key} {seq, token row, the group's first partial slot,
     // splits | index within the group << 16}: the queue hands the items out longest first, the partials of a group
     // stay in key order
@@ -366,11 +375,61 @@ __device__ __forceinline__ void attn_decode_body(const AttnParams& p, int layer,
       }
       __syncwarp();                         // every lane is done with this slot before lane 0 refills it
     }
-    if (!ok) break;
+    if (!ok && !group_mode) break;
 
     l_a = quad_sum(l_a);
     l_b = quad_sum(l_b);
     __nv_bfloat16* orow = p.o + size_t(tok) * q_dim + size_t(hk) * G * DH;
+    if (group_mode) {
+      // this slice's partial into the warp's own (now idle) page ring: [16 rows][DH] unnormalised output, then
+      // [16 rows] (max, sum)
+      float* po = reinterpret_cast<float*>(slots);
+      float2* pml = reinterpret_cast<float2*>(slots + 16 * DH * 4);
+#pragma unroll
+      for (int j = 0; j < DH / 8; ++j) {
+        const int col = 8 * j + 2 * (lane & 3);
+        if (ra < G) *reinterpret_cast<float2*>(po + ra * DH + col) = make_float2(o_acc[j][0], o_acc[j][1]);
+        if (rb < G) *reinterpret_cast<float2*>(po + rb * DH + col) = make_float2(o_acc[j][2], o_acc[j][3]);
+      }
+      if ((lane & 3) == 0) {
+        if (ra < G) pml[ra] = make_float2(m_a, l_a);
+        if (rb < G) pml[rb] = make_float2(m_b, l_b);
+      }
+      const bool failed = __syncthreads_or(!ok) != 0;      // the same answer in every warp of the block
+      if (!failed) {
+        // the eight partials are merged in slice order by the whole block: a thread per pair of output columns
+        const bool f16 = p.o_f16 != 0;
+        for (int e = threadIdx.x; e < G * (DH / 2); e += blockDim.x) {
+          const int g = e / (DH / 2), col = 2 * (e - g * (DH / 2));
+          float mm = -INFINITY;
+#pragma unroll
+          for (int w = 0; w < DC_WARPS; ++w)
+            mm = fmaxf(mm, reinterpret_cast<const float2*>(smem + w * DC_STAGES * SLOT_BYTES + 16 * DH * 4)[g].x);
+          float ll = 0.f, o0 = 0.f, o1 = 0.f;
+#pragma unroll
+          for (int w = 0; w < DC_WARPS; ++w) {
+            const uint8_t* base = smem + w * DC_STAGES * SLOT_BYTES;
+            const float2 ml = reinterpret_cast<const float2*>(base + 16 * DH * 4)[g];
+            const float f = exp2f(ml.x - mm);                 // 0 for an empty slice (max = -inf)
+            const float2 v = *reinterpret_cast<const float2*>(reinterpret_cast<const float*>(base) + g * DH + col);
+            ll += f * ml.y;
+            o0 += f * v.x;
+            o1 += f * v.y;
+          }
+          const float inv = 1.f / ll;
+          if (f16) {
+            const float v2[2] = {o0, o1};
+            note_f16_saturation(v2, p.status, inv);
+          }
+          *reinterpret_cast<uint32_t*>(orow + g * DH + col) = pack_act(o0 * inv, o1 * inv, f16);
+        }
+      }
+      // the rings go back to the copy engine: order these generic-proxy accesses before its next writes
+      fence_proxy_async();
+      __syncthreads();
+      if (failed) break;
+      continue;
+    }
     if (splits == 1) {
       // the whole key range was this item: normalise and write the output rows directly
       const float inv_a = 1.f / l_a, inv_b = 1.f / l_b;

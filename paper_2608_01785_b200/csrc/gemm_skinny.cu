@@ -479,7 +479,7 @@ __global__ void __launch_bounds__(SK_THREADS, 1) small_step_kernel(const __grid_
   log_smid(p.smid_log);
   const int block = int(blockIdx.x), grid = int(gridDim.x);
   const int qkv_n = p.q_dim + 2 * p.kv_dim;
-  const int nb_qkv = min(grid, qkv_n >> 5), nb_attn = min(grid, p.attn.n_decode_items), nb_d = min(grid, p.d >> 5),
+  const int nb_qkv = min(grid, qkv_n >> 5), nb_attn = min(grid, p.attn.decode_group ? p.attn.n_decode_items / DC_WARPS : p.attn.n_decode_items), nb_d = min(grid, p.d >> 5),
             nb_gu = min(grid, p.F >> 4);
   int arrived = 0;                      // grid barriers this block has been through
   bool dead = false;                    // a barrier ran out of time: no further waits, leave after the phase
@@ -630,7 +630,8 @@ cudaError_t small_step_set_attributes() {
 
 cudaError_t launch_small_step(const SmallStepParams& p, int sm_budget, cudaStream_t stream) {
   if (p.T <= 0 || p.T > 16 || p.attn.n_decode_items <= 0) return cudaErrorInvalidValue;
-  const int widest = std::max(std::max((p.q_dim + 2 * p.kv_dim) >> 5, p.attn.n_decode_items), std::max(p.d >> 5, p.F >> 4));
+  const int attn_work = p.attn.decode_group ? p.attn.n_decode_items / DC_WARPS : p.attn.n_decode_items;
+  const int widest = std::max(std::max((p.q_dim + 2 * p.kv_dim) >> 5, attn_work), std::max(p.d >> 5, p.F >> 4));
   const int grid = widest < sm_budget ? widest : sm_budget;
   if (p.head_dim == 128) return p.f16 ? launch_small_one<128, true>(p, grid, stream) : launch_small_one<128, false>(p, grid, stream);
   return p.f16 ? launch_small_one<64, true>(p, grid, stream) : launch_small_one<64, false>(p, grid, stream);

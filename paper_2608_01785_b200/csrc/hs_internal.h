@@ -69,6 +69,7 @@ MetaLayout make_meta_layout(const hs_stage_config_t& c);
 struct StepPlan {
   int n_tokens = 0, n_seqs = 0;
   int n_prefill_items = 0, n_decode_items = 0, n_decode_rows = 0;
+  int decode_group = 0;           // 1: decode items are eight page slices per (sequence, KV head), group-major (see plan_step)
   // work estimates of the two attention kernels (for the split of the SM budget when they run side by side)
   int64_t prefill_blocks = 0;     // 64-key blocks over all prefill items (an item's two tiles share a block)
   int prefill_longest = 0;        // blocks of the longest prefill item

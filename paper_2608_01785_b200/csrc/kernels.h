@@ -228,6 +228,8 @@ struct AttnParams {
   const int32_t* decode_items;     // two int4 per item: {decode row, kv head, first key, end key}
                                    //                    {seq, token row, first item of its group, splits}
   int n_decode_items;
+  int decode_group;                // 1: the items are eight page slices per (sequence, KV head) group, group-major; a block
+                                   //    works whole groups and merges their slices in shared memory (small batches)
   const int32_t* decode_rows;      // int4 per decode sequence
   int n_decode_rows;
   float* part_o;                   // [max_decode_items][16][Dh] unnormalised partial outputs

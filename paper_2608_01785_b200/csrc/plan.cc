@@ -63,7 +63,7 @@ MetaLayout make_meta_layout(const hs_stage_config_t& c) {
   m.max_prefill_items = c.n_kv_heads * (c.max_tokens / prefill_tokens_per_item(G) + c.max_seqs);
   // a decode sequence of n keys has at most n / kDecodeSplit whole runs and kDecodeSplitMax / kDecodeTail pieces of a
   // last, incomplete one; cached keys are bounded by the pool
-  m.max_decode_items = c.n_kv_heads * (c.max_seqs * (kDecodeSplitMax / kDecodeTail) +
+  m.max_decode_items = c.n_kv_heads * (c.max_seqs * 2 * (kDecodeSplitMax / kDecodeTail) +
                                        int((int64_t(c.num_pages) * kPage) / kDecodeSplit) + 1);
   int off = 0;
   auto take = [&](int n) {
@@ -155,6 +155,18 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
   const int G = c.n_q_heads / c.n_kv_heads;
   const int Mt = prefill_tokens_per_item(G);
   const int split = pick_decode_split(c, b, sm_count, ml.max_decode_items);
+  // Group mode of the decode attention: when even the smallest run length leaves warps idle (the batch is small) and
+  // every (sequence, KV head) group can have a block of its own, a group's pages are dealt evenly to the eight warps
+  // of one block, whose partial results then meet in shared memory -- no partials in global memory, no counter, no
+  // merging warp.  A function of the batch and the device's SM count, never of the budget.
+  bool group_mode = split == kDecodeTail;
+  {
+    int groups = 0, longest = 0;
+    for (int s = 0; s < b.n_seqs; ++s)
+      if (b.q_len[s] == 1) { groups += c.n_kv_heads; longest = std::max(longest, b.ctx_len[s] + 1); }
+    const int sms = sm_count > 0 ? sm_count : 148;
+    if (groups == 0 || groups > sms || longest > kDecodeWarps * 32 * kPage) group_mode = false;
+  }
   StepPlan p;
   p.n_tokens = b.n_tokens;
   p.n_seqs = b.n_seqs;
@@ -183,7 +195,22 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
       }
       if (tok_seq) tok_seq[t + j] = s;
     }
-    if (n == 1) {
+    if (n == 1 && group_mode) {
+      // decode, group mode: eight slices of the sequence's pages per KV head (the last ones may be empty)
+      const int keys = ctx + 1, pages = ceil_div(keys, kPage), per = ceil_div(pages, kDecodeWarps) * kPage;
+      if (meta) {
+        int32_t* row = meta + ml.decode_rows + n_dec_rows * 4;
+        row[0] = s; row[1] = t; row[2] = n_dec_items; row[3] = kDecodeWarps;
+      }
+      for (int hk = 0; hk < c.n_kv_heads; ++hk)
+        for (int w = 0; w < kDecodeWarps; ++w) {
+          const int k0 = std::min(keys, w * per), k1 = std::min(keys, (w + 1) * per);
+          dec.push_back(DecItem{{n_dec_rows, hk, k0, k1, s, t, 0, 1}, 0});
+        }
+      n_dec_items += c.n_kv_heads * kDecodeWarps;
+      p.decode_kv_bytes += int64_t(keys) * 2 * c.n_kv_heads * c.head_dim * 2;
+      ++n_dec_rows;
+    } else if (n == 1) {
       // decode: keys 0..ctx cut into whole runs of `split` keys and the rest into pieces of kDecodeTail keys; the items
       // of a (sequence, KV head) group keep consecutive partial-result slots in key order, whatever the order the
       // queue hands them out in
@@ -222,7 +249,7 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
   // longest first, so that the dynamic queue finishes evenly; ties keep batch order
   std::stable_sort(pre.begin(), pre.end(), [](const Item& a, const Item& b2) { return a.cost > b2.cost; });
   // decode items likewise: the long runs first, the short ones fill the end of the kernel
-  std::stable_sort(dec.begin(), dec.end(), [](const DecItem& a, const DecItem& b2) { return a.keys > b2.keys; });
+  if (!group_mode) std::stable_sort(dec.begin(), dec.end(), [](const DecItem& a, const DecItem& b2) { return a.keys > b2.keys; });
   if (meta) {
     for (size_t i = 0; i < dec.size(); ++i)
       for (int k = 0; k < 8; ++k) meta[ml.decode_items + int(i) * 8 + k] = dec[i].v[k];
@@ -234,6 +261,7 @@ hs_status_t plan_step(const hs_stage_config_t& c, const MetaLayout& ml, const hs
   }
   p.n_prefill_items = int(pre.size());
   p.n_decode_items = n_dec_items;
+  p.decode_group = group_mode && n_dec_items > 0 ? 1 : 0;
   p.n_decode_rows = n_dec_rows;
   if (plan) *plan = p;
   return HS_OK;

@@ -82,9 +82,11 @@ def test_noalloc_decode_attention_matches_the_stage_path_twice_in_a_row():
             assert B.hs_op_decode_attention_noalloc_status() == B.HS_OK
             got = o_got.float().cpu().numpy()
             assert np.all(np.isfinite(got))
-            # against the existing entry point (the stage sizes its split-KV items by batch, this call uses a
-            # fixed size, so the two may add the same terms in different groupings: tolerance, not bits) ...
-            assert rel_err(got, o_stage) <= TOL
+            # against the existing entry point (the stage sizes its split-KV items by batch -- or deals a group's pages
+            # to the eight warps of one block -- while this call uses a fixed size, so the two add the same terms in
+            # different groupings and round the bf16 output differently by an ulp here and there: tolerance, not
+            # bits; row by row for the reason given below) ...
+            assert max(rel_err(got[s], o_stage[s]) for s in range(n)) <= TOL
             # ... and against the oracle's attention of the same bf16 queries over the same cache
             # (row by row: a sequence of 6 keys has outputs of the size of V itself, one of 1500 keys outputs thirty
             # times smaller, so one RMS over the whole tensor would measure the short rows by the long ones' scale)
