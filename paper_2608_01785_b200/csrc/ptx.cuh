@@ -307,10 +307,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Two fp32 -> packed fp16 (round to nearest even), clamped to the finite fp16 range so that an outlier
 // becomes +-65504 instead of infinity.
 __device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
-  lo = fminf(fmaxf(lo, -65504.f), 65504.f);
-  hi = fminf(fmaxf(hi, -65504.f), 65504.f);
-  __half2 v = __floats2half2_rn(lo, hi);
-  return *reinterpret_cast<uint32_t*>(&v);
+  uint32_t v;     // one instruction: round to nearest even, values beyond the finite range become +-65504
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(v) : "f"(hi), "f"(lo));
+  return v;
 }
 // Packs as fp16 or bf16: the stage's private activations (h, o, act) are fp16 unless it was created with
 // HS_FLAG_BF16_ACTIVATIONS.
