@@ -133,6 +133,32 @@ hs_status_t hs_op_decode_attention_noalloc(const void *q_dev, const void *kv_poo
                                            void *cuda_stream);
 hs_status_t hs_op_decode_attention_noalloc_status(int32_t *status_out);
 
+/*
+ * Host-only diagnosis of the planner: the attention work lists hs_stage_step would build for `batch` (validated as
+ * by hs_stage_plan; works on a stage without a device, which plans for 148 SMs).  The paper has no counterpart: it
+ * leaves the execution of a step to its runtime (Sec. 5).
+ *   decode_items   [decode_cap][8] int32, in the order the kernel's queue hands them out:
+ *                  {decode row, KV head, first key, end key (exclusive), sequence, token row, the group's first
+ *                  partial slot, items of the group | index within the group << 16}; in group mode (*decode_group = 1:
+ *                  a small batch, every (sequence, KV head) group worked by one block) eight page slices per group,
+ *                  group-major, some possibly empty (first key = end key), the last two words unused.
+ *   prefill_items  [prefill_cap][8] int32, longest first: {sequence, KV head, first new token, tokens (at most two Q
+ *                  tiles), cached tokens, token row of the sequence's first new token, new tokens of the sequence, 0}.
+ * Any pointer may be NULL; counts are always written when their pointer is given; at most cap records are copied.
+ * Errors: INVALID_ARG, BAD_BLOCK_TABLE.
+ */
+hs_status_t hs_stage_plan_attention(hs_stage_t *stage, const hs_batch_t *batch, int32_t *decode_items, int32_t decode_cap,
+                                    int32_t *n_decode_items, int32_t *decode_group, int32_t *prefill_items,
+                                    int32_t prefill_cap, int32_t *n_prefill_items);
+
+/*
+ * Host-only: the K block (of 64) at which split i (0 .. ks; i = ks gives k_blocks) of a small step's residual GEMM
+ * begins when its k_blocks are cut into ks splits.  Each split is ten K blocks longer than the one before it (the
+ * splits add their sums one after the other, and a link of that chain takes about as long as ten K blocks take to
+ * stream), or all are equal when K is too short for that.  Returns -1 for ks < 1, k_blocks < 1 or i outside 0 .. ks.
+ */
+int32_t hs_op_gemm_split_begin(int32_t k_blocks, int32_t ks, int32_t i);
+
 #if defined(__GNUC__)
 #pragma GCC visibility pop
 #endif

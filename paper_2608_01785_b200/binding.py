@@ -29,7 +29,7 @@ EXPORTS = ("hs_status_str", "hs_kv_pool_bytes", "hs_workspace_bytes", "hs_stage_
            "hs_spatial_derive_cap", "hs_head_workspace_bytes", "hs_head_create", "hs_head_step", "hs_head_status",
            "hs_head_destroy", "hs_op_embed", "hs_temporal_create", "hs_temporal_step", "hs_temporal_destroy",
            "hs_stage_set_qkv_bias", "hs_stage_set_modulation", "hs_stage_saturation_count", "hs_op_wait_probe",
-           "hs_op_decode_attention_noalloc_status")
+           "hs_op_decode_attention_noalloc_status", "hs_stage_plan_attention", "hs_op_gemm_split_begin")
 PROFILE_CLASSES = ("rmsnorm", "gemm_qkv", "attn_prefill", "attn_decode", "attn_combine", "gemm_out", "gemm_gateup",
                    "gemm_down")
 
@@ -109,6 +109,11 @@ def lib() -> C.CDLL:
         l.hs_kv_free_pages.argtypes = [C.c_void_p]
         l.hs_kv_free_pages.restype = C.c_int32
         l.hs_stage_plan.argtypes = [C.c_void_p, C.POINTER(hs_batch_t), C.c_void_p, C.c_void_p, C.c_void_p]
+        l.hs_stage_plan_attention.argtypes = [C.c_void_p, C.POINTER(hs_batch_t), C.c_void_p, C.c_int32, C.c_void_p,
+                                              C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p]
+        l.hs_stage_plan_attention.restype = C.c_int
+        l.hs_op_gemm_split_begin.argtypes = [C.c_int32, C.c_int32, C.c_int32]
+        l.hs_op_gemm_split_begin.restype = C.c_int32
         l.hs_stage_step.argtypes = [C.c_void_p, C.POINTER(hs_batch_t), C.c_int32, C.c_void_p]
         l.hs_stage_status.argtypes = [C.c_void_p]
         l.hs_stage_sm_count.argtypes = [C.c_void_p]
@@ -236,6 +241,23 @@ def hs_stage_plan(stage: int, batch: Batch):
     if st != HS_OK:
         raise HsError(st, "hs_stage_plan")
     return seq[:n], pos[:n], slot[:n]
+
+
+def hs_stage_plan_attention(stage: int, batch: Batch, cap: int = 1 << 16):
+    """Returns (decode_items [n, 8], decode_group flag, prefill_items [m, 8]) as the planner lists them."""
+    dec = np.zeros((cap, 8), dtype=np.int32)
+    pre = np.zeros((cap, 8), dtype=np.int32)
+    n_dec, grp, n_pre = C.c_int32(0), C.c_int32(0), C.c_int32(0)
+    st = lib().hs_stage_plan_attention(C.c_void_p(stage), C.byref(batch.c), dec.ctypes.data, cap, C.byref(n_dec),
+                                       C.byref(grp), pre.ctypes.data, cap, C.byref(n_pre))
+    if st != HS_OK:
+        raise HsError(st, "hs_stage_plan_attention")
+    assert n_dec.value <= cap and n_pre.value <= cap
+    return dec[: n_dec.value], grp.value, pre[: n_pre.value]
+
+
+def hs_op_gemm_split_begin(k_blocks: int, ks: int, i: int) -> int:
+    return int(lib().hs_op_gemm_split_begin(k_blocks, ks, i))
 
 
 def hs_stage_step(stage: int, batch: Batch, sm_budget: int, cuda_stream: int = 0) -> None:

@@ -444,6 +444,29 @@ hs_status_t hs_stage_plan(hs_stage_t* s, const hs_batch_t* b, int32_t* tok_seq, 
   return HS_OK;
 }
 
+hs_status_t hs_stage_plan_attention(hs_stage_t* s, const hs_batch_t* b, int32_t* decode_items, int32_t decode_cap,
+                                    int32_t* n_decode_items, int32_t* decode_group, int32_t* prefill_items,
+                                    int32_t prefill_cap, int32_t* n_prefill_items) {
+  if (!s || !b || decode_cap < 0 || prefill_cap < 0) return HS_ERR_INVALID_ARG;
+  std::vector<int32_t> meta(s->ml.total);
+  StepPlan plan;
+  const hs_status_t st = plan_step(s->cfg, s->ml, *b, s->sm_count, s->page_stamp, ++s->stamp, meta.data(), nullptr, &plan);
+  if (st != HS_OK) return st;
+  if (n_decode_items) *n_decode_items = plan.n_decode_items;
+  if (decode_group) *decode_group = plan.decode_group;
+  if (n_prefill_items) *n_prefill_items = plan.n_prefill_items;
+  if (decode_items)
+    memcpy(decode_items, meta.data() + s->ml.decode_items, size_t(std::min(decode_cap, plan.n_decode_items)) * 32);
+  if (prefill_items)
+    memcpy(prefill_items, meta.data() + s->ml.prefill_items, size_t(std::min(prefill_cap, plan.n_prefill_items)) * 32);
+  return HS_OK;
+}
+
+int32_t hs_op_gemm_split_begin(int32_t k_blocks, int32_t ks, int32_t i) {
+  if (k_blocks < 1 || ks < 1 || i < 0 || i > ks) return -1;
+  return gemm_split_begin(k_blocks, ks, i);
+}
+
 hs_status_t hs_stage_step(hs_stage_t* s, const hs_batch_t* b, int32_t sm_budget, void* cuda_stream) {
   if (!s || !b) return HS_ERR_INVALID_ARG;
   if (s->cfg.device < 0) return HS_ERR_NO_DEVICE;
